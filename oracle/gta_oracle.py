@@ -1,0 +1,201 @@
+"""ctypes front end of the fp64 CPU oracle (``gta_oracle.c``).
+
+TEST INFRASTRUCTURE ONLY: imported by the tests, by the smoke check and by the
+benchmark's CPU-baseline leg.  It never touches the CUDA library and the CUDA
+library never touches it.
+
+Arrays may be numpy arrays (float32 / float64 / uint16 holding bf16 bit patterns)
+or torch CPU tensors (float32 / float64 / bfloat16); values are handed to the C
+code in their stored form and widened there, exactly, to double.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from dataclasses import dataclass
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "gta_oracle.c")
+_LIB = os.path.join(_HERE, "libgta_oracle.so")
+
+F32, BF16, F64 = 0, 1, 2
+
+
+def build(force: bool = False) -> str:
+    """Compile the C oracle with gcc (OpenMP) next to its source; returns the path."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        tmp = _LIB + f".{os.getpid()}.tmp"
+        subprocess.check_call(
+            ["gcc", "-O2", "-ftree-vectorize", "-fopenmp", "-fPIC", "-shared", "-o", tmp, _SRC, "-lm"]
+        )
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+class _Shape(ctypes.Structure):
+    _fields_ = [
+        ("batch", ctypes.c_int32), ("seq", ctypes.c_int32), ("d_model", ctypes.c_int32),
+        ("n_heads", ctypes.c_int32), ("n_q", ctypes.c_int32), ("n_k", ctypes.c_int32),
+        ("n_c", ctypes.c_int32), ("d_h", ctypes.c_int32), ("d_l", ctypes.c_int32),
+        ("causal", ctypes.c_int32), ("scale", ctypes.c_double),
+    ]
+
+
+@dataclass
+class Shape:
+    """Operator shape in the paper's symbols (Sec. 3.2): B, N, H, n_h, n_q, n_k, n_c, d_h, d_l."""
+    batch: int
+    seq: int
+    d_model: int
+    n_heads: int
+    n_q: int
+    n_k: int
+    n_c: int
+    d_h: int
+    d_l: int
+    causal: int = 1
+    scale: float = 0.0
+
+    def c(self) -> _Shape:
+        return _Shape(self.batch, self.seq, self.d_model, self.n_heads, self.n_q, self.n_k,
+                      self.n_c, self.d_h, self.d_l, self.causal, self.scale)
+
+
+_lib = None
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        L = ctypes.CDLL(build())
+        vp, i32, ip = ctypes.c_void_p, ctypes.c_int32, ctypes.POINTER(ctypes.c_int32)
+        sp = ctypes.POINTER(_Shape)
+        for name in ("gta_oracle_prefill", "gta_oracle_prefill_definition"):
+            f = getattr(L, name)
+            f.argtypes = [sp, i32, vp, vp, vp, vp, vp, vp, vp, i32, vp, i32]
+            f.restype = i32
+        L.gta_oracle_probs.argtypes = [sp, i32, vp, vp, vp]
+        L.gta_oracle_probs.restype = i32
+        L.gta_oracle_decode.argtypes = [sp, i32, vp, vp, vp, vp, i32, vp, vp, vp, vp, i32]
+        L.gta_oracle_decode.restype = i32
+        L.gta_oracle_cache_append.argtypes = [sp, i32, vp, vp, i32, vp, vp, i32, vp, ip]
+        L.gta_oracle_cache_append.restype = i32
+        L.gta_oracle_attention_cost.argtypes = [sp]
+        L.gta_oracle_attention_cost.restype = ctypes.c_double
+        L.gta_oracle_cache_elems.argtypes = [sp]
+        L.gta_oracle_cache_elems.restype = ctypes.c_double
+        L.gta_oracle_num_threads.restype = i32
+        _lib = L
+    return _lib
+
+
+def _as_np(a):
+    """torch CPU tensor or numpy array -> (contiguous numpy array, dtype code)."""
+    if not isinstance(a, np.ndarray):
+        import torch
+        assert a.device.type == "cpu", "the oracle reads host memory only"
+        a = a.contiguous()
+        if a.dtype == torch.bfloat16:
+            a = a.view(torch.int16).numpy().view(np.uint16)
+        else:
+            a = a.numpy()
+    a = np.ascontiguousarray(a)
+    code = {np.dtype(np.float32): F32, np.dtype(np.uint16): BF16, np.dtype(np.float64): F64}[a.dtype]
+    return a, code
+
+
+def _same_dtype(*arrs):
+    conv = [_as_np(a) for a in arrs]
+    codes = {c for _, c in conv}
+    assert len(codes) == 1, "all operator tensors share one storage type"
+    return [a for a, _ in conv], codes.pop()
+
+
+def _ptr(a):
+    return ctypes.c_void_p(a.ctypes.data)
+
+
+def _check(rc, what):
+    if rc != 0:
+        raise RuntimeError(f"{what}: oracle returned {rc} (1 = bad argument, 2 = out of memory)")
+
+
+def num_threads() -> int:
+    return int(lib().gta_oracle_num_threads())
+
+
+def prefill(shape: Shape, q, k, c, x, w_p, w_g, rows=None, n_threads: int = 0, definition=False):
+    """out[B, R, n_h, d_h] (float64).  rows=None -> every position (R = N)."""
+    (q, k, c, x, w_p, w_g), code = _same_dtype(q, k, c, x, w_p, w_g)
+    s = shape
+    assert q.size == s.batch * s.n_q * s.seq * s.d_h and k.size == s.batch * s.n_k * s.seq * s.d_h
+    assert c.size == s.batch * s.n_c * s.seq * s.d_l and x.size == s.batch * s.seq * s.d_model
+    assert w_p.size == s.n_heads * s.d_l * s.d_h and w_g.size == s.d_model * s.n_heads * s.d_h
+    if rows is None:
+        rows_np, n_rows, R = None, 0, s.seq
+    else:
+        rows_np = np.ascontiguousarray(np.asarray(rows, dtype=np.int32))
+        n_rows = R = int(rows_np.size)
+    out = np.zeros((s.batch, R, s.n_heads, s.d_h), dtype=np.float64)
+    fn = lib().gta_oracle_prefill_definition if definition else lib().gta_oracle_prefill
+    cs = s.c()
+    rc = fn(ctypes.byref(cs), code, _ptr(q), _ptr(k), _ptr(c), _ptr(x), _ptr(w_p), _ptr(w_g),
+            _ptr(rows_np) if rows_np is not None else None, n_rows, _ptr(out), n_threads)
+    _check(rc, "prefill")
+    return out
+
+
+def probs(shape: Shape, q, k):
+    """Attention probabilities [B, n_q, N, N] (float64); masked entries are 0."""
+    (q, k), code = _same_dtype(q, k)
+    s = shape
+    out = np.zeros((s.batch, s.n_q, s.seq, s.seq), dtype=np.float64)
+    cs = s.c()
+    _check(lib().gta_oracle_probs(ctypes.byref(cs), code, _ptr(q), _ptr(k), _ptr(out)), "probs")
+    return out
+
+
+def decode(shape: Shape, q, k_cache, c_cache, seq_lens, s_cap: int, x_t, w_p, w_g, n_threads: int = 0):
+    """out[B, n_h, d_h] (float64); seq_lens counts the new token, already appended."""
+    (q, k_cache, c_cache, x_t, w_p, w_g), code = _same_dtype(q, k_cache, c_cache, x_t, w_p, w_g)
+    s = shape
+    assert k_cache.size == s.batch * s.n_k * s_cap * s.d_h
+    assert c_cache.size == s.batch * s.n_c * s_cap * s.d_l
+    lens = np.ascontiguousarray(np.asarray(seq_lens, dtype=np.int32))
+    assert lens.size == s.batch
+    out = np.zeros((s.batch, s.n_heads, s.d_h), dtype=np.float64)
+    cs = s.c()
+    rc = lib().gta_oracle_decode(ctypes.byref(cs), code, _ptr(q), _ptr(k_cache), _ptr(c_cache),
+                                 _ptr(lens), s_cap, _ptr(x_t), _ptr(w_p), _ptr(w_g), _ptr(out),
+                                 n_threads)
+    _check(rc, "decode")
+    return out
+
+
+def cache_append(shape: Shape, k_cache, c_cache, s_cap: int, k_new, c_new, n_new: int, seq_lens):
+    """Byte-exact append.  Returns (k_cache, c_cache, seq_lens, overflowed) as NEW numpy arrays."""
+    (k_cache, c_cache, k_new, c_new), _ = _same_dtype(k_cache, c_cache, k_new, c_new)
+    k_cache, c_cache = k_cache.copy(), c_cache.copy()
+    lens = np.ascontiguousarray(np.asarray(seq_lens, dtype=np.int32)).copy()
+    flag = ctypes.c_int32(0)
+    cs = shape.c()
+    rc = lib().gta_oracle_cache_append(ctypes.byref(cs), k_cache.dtype.itemsize, _ptr(k_cache),
+                                       _ptr(c_cache), s_cap, _ptr(k_new), _ptr(c_new), n_new,
+                                       _ptr(lens), ctypes.byref(flag))
+    _check(rc, "cache_append")
+    return k_cache, c_cache, lens, int(flag.value)
+
+
+def attention_cost(shape: Shape) -> float:
+    """n_q (d_h + d_l) N^2 — Table 3, GTA row, 'Attention' column."""
+    cs = shape.c()
+    return float(lib().gta_oracle_attention_cost(ctypes.byref(cs)))
+
+
+def cache_elems(shape: Shape) -> float:
+    """(n_k d_h + n_c d_l) N — Table 3, GTA row, 'KV Cache per Layer' column."""
+    cs = shape.c()
+    return float(lib().gta_oracle_cache_elems(ctypes.byref(cs)))

@@ -1,0 +1,297 @@
+"""CPU-only pins of the fp64 oracle against what the paper and the mathematics fix.
+
+Every check compares the oracle with something that is not the oracle: a textbook attention
+written here with numpy, an einsum restatement of the definition, closed forms of the softmax,
+invariants (row sums, causality, batch independence, sharing inside a head group) and the
+ratios / cache widths the paper prints.  A dropped term, a wrong head map, a transposed
+operand, a missing sigmoid or an off-by-one in the causal bound fails at least one of them.
+"""
+import numpy as np
+import pytest
+
+from oracle.gta_oracle import Shape
+
+RNG = np.random.default_rng(20250617)
+
+
+def _rand(*shape, scale=1.0):
+    return RNG.standard_normal(shape) * scale
+
+
+def _inputs(s: Shape, n=None):
+    n = s.seq if n is None else n
+    return dict(
+        q=_rand(s.batch, s.n_q, n, s.d_h), k=_rand(s.batch, s.n_k, n, s.d_h),
+        c=_rand(s.batch, s.n_c, n, s.d_l), x=_rand(s.batch, n, s.d_model),
+        w_p=_rand(s.n_heads, s.d_l, s.d_h, scale=s.d_l ** -0.5),
+        w_g=_rand(s.d_model, s.n_heads * s.d_h, scale=s.d_model ** -0.5),
+    )
+
+
+def _softmax_np(s, axis=-1):
+    e = np.exp(s - s.max(axis=axis, keepdims=True))
+    return e / e.sum(axis=axis, keepdims=True)
+
+
+def _einsum_gta(s: Shape, t):
+    """Independent restatement of Sec. 3.2-3.3 with whole-matrix einsums (definition form)."""
+    B, N, nh = s.batch, s.seq, s.n_heads
+    scale = s.scale or s.d_h ** -0.5
+    out = np.zeros((B, N, nh, s.d_h))
+    mask = np.tril(np.ones((N, N), dtype=bool)) if s.causal else np.ones((N, N), dtype=bool)
+    for i in range(nh):
+        g = i * s.n_q // nh
+        kg, cg = g * s.n_k // s.n_q, g * s.n_c // s.n_q
+        S = np.einsum("btd,bjd->btj", t["q"][:, g], t["k"][:, kg]) * scale
+        S = np.where(mask[None], S, -np.inf)
+        P = _softmax_np(S)
+        gate = 1.0 / (1.0 + np.exp(-np.einsum("bth,he->bte", t["x"], t["w_g"][:, i * s.d_h:(i + 1) * s.d_h])))
+        V = np.einsum("bjl,le->bje", t["c"][:, cg], t["w_p"][i])            # C W_P
+        Vt = V[:, None, :, :] * gate[:, :, None, :]                          # V^{(t)}[b,t,j,e]
+        out[:, :, i, :] = np.einsum("btj,btje->bte", P, Vt)
+    return out
+
+
+# ---------------------------------------------------------------- P1: reduction to MHA
+@pytest.mark.parametrize("causal", [1, 0])
+def test_reduces_to_multi_head_attention(oracle, causal):
+    """Group size 1, W_P = slice selector, W_G = 0  =>  0.5 * textbook MHA (sigmoid(0) = 1/2)."""
+    nh, dh, N, B, H = 3, 8, 17, 2, 12
+    s = Shape(B, N, H, nh, nh, nh, 1, dh, nh * dh, causal)
+    t = _inputs(s)
+    t["w_g"][:] = 0.0
+    t["w_p"][:] = 0.0
+    for i in range(nh):
+        t["w_p"][i, i * dh:(i + 1) * dh, :] = np.eye(dh)
+    got = oracle.prefill(s, **t)
+    want = np.zeros_like(got)
+    for b in range(B):
+        for i in range(nh):
+            S = t["q"][b, i] @ t["k"][b, i].T / np.sqrt(dh)
+            if causal:
+                S = np.where(np.tril(np.ones((N, N), dtype=bool)), S, -np.inf)
+            want[b, :, i, :] = _softmax_np(S) @ t["c"][b, 0][:, i * dh:(i + 1) * dh]
+    np.testing.assert_allclose(got, 0.5 * want, rtol=1e-12, atol=1e-14)
+
+
+# ---------------------------------------------------------------- P2: softmax rows
+def test_probability_rows_sum_to_one_and_respect_mask(oracle):
+    s = Shape(2, 19, 8, 4, 2, 1, 1, 8, 16, 1)
+    t = _inputs(s)
+    P = oracle.probs(s, t["q"], t["k"])
+    assert P.shape == (2, 2, 19, 19)
+    np.testing.assert_allclose(P.sum(-1), 1.0, atol=1e-14)
+    assert (P >= 0).all()
+    assert np.all(np.triu(P, k=1) == 0.0)          # nothing above the diagonal
+    assert np.all(np.diagonal(P, axis1=-2, axis2=-1) > 0)  # the diagonal is included
+    # probabilities equal an independent softmax of the scaled scores
+    S = np.einsum("bgtd,bjd->bgtj", t["q"], t["k"][:, 0]) / np.sqrt(8)
+    S = np.where(np.tril(np.ones((19, 19), dtype=bool)), S, -np.inf)
+    np.testing.assert_allclose(P, _softmax_np(S), rtol=1e-12, atol=1e-15)
+
+
+# ---------------------------------------------------------------- P3: causality
+def test_future_tokens_do_not_change_earlier_rows(oracle):
+    s = Shape(1, 24, 16, 4, 2, 2, 1, 8, 16, 1)
+    t = _inputs(s)
+    base = oracle.prefill(s, **t)
+    cut = 13
+    t2 = {k: v.copy() for k, v in t.items()}
+    for name in ("q", "k", "c"):
+        t2[name][:, :, cut:, :] += _rand(*t2[name][:, :, cut:, :].shape)
+    t2["x"][:, cut:, :] += 1.0
+    pert = oracle.prefill(s, **t2)
+    assert np.array_equal(base[:, :cut], pert[:, :cut])        # bit-identical
+    assert not np.allclose(base[:, cut:], pert[:, cut:])
+    # and the non-causal operator does depend on the future
+    s0 = Shape(1, 24, 16, 4, 2, 2, 1, 8, 16, 0)
+    assert not np.allclose(oracle.prefill(s0, **t)[:, :cut], oracle.prefill(s0, **t2)[:, :cut])
+
+
+# ---------------------------------------------------------------- P4: decode == last prefill row
+@pytest.mark.parametrize("n_k,n_c", [(4, 1), (2, 2), (1, 1)])
+def test_decode_equals_last_prefill_row_after_append(oracle, n_k, n_c):
+    B, N, cap = 3, 11, 16
+    s = Shape(B, N, 24, 8, 4, n_k, n_c, 8, 16, 1)
+    t = _inputs(s)
+    full = oracle.prefill(s, **t)
+    # load the first N-1 tokens into empty caches, then append token N-1 as a decode step would
+    k_cache = _rand(B, n_k, cap, s.d_h)   # garbage beyond the live part must not matter
+    c_cache = _rand(B, n_c, cap, s.d_l)
+    lens = np.zeros(B, dtype=np.int32)
+    k_cache, c_cache, lens, ov = oracle.cache_append(
+        s, k_cache, c_cache, cap, t["k"][:, :, :N - 1].copy(), t["c"][:, :, :N - 1].copy(), N - 1, lens)
+    assert ov == 0 and (lens == N - 1).all()
+    k_cache, c_cache, lens, ov = oracle.cache_append(
+        s, k_cache, c_cache, cap, t["k"][:, :, N - 1:].copy(), t["c"][:, :, N - 1:].copy(), 1, lens)
+    assert ov == 0 and (lens == N).all()
+    got = oracle.decode(s, t["q"][:, :, N - 1].copy(), k_cache, c_cache, lens, cap,
+                        t["x"][:, N - 1].copy(), t["w_p"], t["w_g"])
+    np.testing.assert_allclose(got, full[:, N - 1], rtol=1e-12, atol=1e-15)
+
+
+def test_decode_ragged_lengths_and_empty_sequence(oracle):
+    B, cap = 4, 12
+    s = Shape(B, 0, 8, 4, 2, 2, 1, 4, 8, 1)
+    lens = np.array([12, 1, 0, 5], dtype=np.int32)
+    q, xt = _rand(B, 2, 4), _rand(B, 8)
+    kc, cc = _rand(B, 2, cap, 4), _rand(B, 1, cap, 8)
+    w_p, w_g = _rand(4, 8, 4), _rand(8, 16)
+    got = oracle.decode(s, q, kc, cc, lens, cap, xt, w_p, w_g)
+    assert np.all(got[2] == 0.0)
+    # len == 1: attention is the identity on the single cached latent
+    gate = 1 / (1 + np.exp(-(xt[1] @ w_g)))
+    want = np.stack([cc[1, 0, 0] @ w_p[i] for i in range(4)]) * gate.reshape(4, 4)
+    np.testing.assert_allclose(got[1], want, rtol=1e-12)
+    # each sequence equals a one-sequence call (independence from the other lengths)
+    for b in (0, 3):
+        s1 = Shape(1, 0, 8, 4, 2, 2, 1, 4, 8, 1)
+        one = oracle.decode(s1, q[b:b + 1], kc[b:b + 1], cc[b:b + 1], lens[b:b + 1], cap, xt[b:b + 1], w_p, w_g)
+        assert np.array_equal(one[0], got[b])
+
+
+# ---------------------------------------------------------------- P5 / P6: brute force, two forms
+@pytest.mark.parametrize("shape", [
+    Shape(2, 7, 6, 4, 2, 1, 1, 4, 8, 1),      # keys shared by both maps
+    Shape(1, 8, 10, 8, 4, 2, 2, 4, 4, 1),     # two latent groups, d_l == d_h
+    Shape(2, 5, 6, 6, 6, 3, 1, 2, 6, 0),      # non-causal, one head per map
+    Shape(1, 1, 3, 2, 1, 1, 1, 2, 4, 1),      # single token
+    Shape(1, 6, 4, 4, 2, 2, 1, 3, 5, 1, 0.37),  # explicit softmax scale
+])
+def test_matches_einsum_restatement_and_definition_form(oracle, shape):
+    t = _inputs(shape)
+    want = _einsum_gta(shape, t)
+    got = oracle.prefill(shape, **t)
+    got_def = oracle.prefill(shape, **t, definition=True)
+    np.testing.assert_allclose(got, want, rtol=1e-11, atol=1e-14)
+    np.testing.assert_allclose(got_def, want, rtol=1e-11, atol=1e-14)
+    np.testing.assert_allclose(got, got_def, rtol=1e-11, atol=1e-14)     # P6
+    rows = [shape.seq - 1, 0]
+    sub = oracle.prefill(shape, **t, rows=rows)
+    assert np.array_equal(sub, got[:, rows])
+
+
+def test_gate_uses_the_query_token_not_the_key_token(oracle):
+    """Changing x at position j changes row j only (the gate never follows the key index)."""
+    s = Shape(1, 9, 8, 2, 1, 1, 1, 4, 8, 1)
+    t = _inputs(s)
+    base = oracle.prefill(s, **t)
+    t["x"][0, 3] += 2.0
+    pert = oracle.prefill(s, **t)
+    changed = np.any(base != pert, axis=(0, 2, 3))
+    assert changed.tolist() == [j == 3 for j in range(9)]
+
+
+# ---------------------------------------------------------------- P7 / P8: closed forms
+def test_uniform_attention_closed_form(oracle):
+    s = Shape(2, 10, 8, 4, 2, 2, 1, 4, 8, 1)
+    t = _inputs(s)
+    t["q"][:] = 0.0
+    got = oracle.prefill(s, **t)
+    csum = np.cumsum(t["c"][:, 0], axis=1) / np.arange(1, 11)[None, :, None]   # running mean
+    gate = 1 / (1 + np.exp(-(t["x"] @ t["w_g"]))).reshape(2, 10, 4, 4)
+    want = np.einsum("btl,ile->btie", csum, t["w_p"]) * gate
+    np.testing.assert_allclose(got, want, rtol=1e-12, atol=1e-15)
+
+
+def test_one_hot_attention_closed_form(oracle):
+    N, dh = 8, 8
+    s = Shape(1, N, 6, 2, 1, 1, 1, dh, 12, 1)
+    t = _inputs(s)
+    perm = RNG.permutation(N)
+    t["k"][0, 0] = 200.0 * np.eye(dh)[perm]              # key j points along axis perm[j]
+    target = np.array([RNG.integers(0, tt + 1) for tt in range(N)])   # a visible key per row
+    t["q"][0, 0] = np.eye(dh)[perm[target]] * np.sqrt(dh)
+    got = oracle.prefill(s, **t)
+    gate = 1 / (1 + np.exp(-(t["x"][0] @ t["w_g"]))).reshape(N, 2, dh)
+    want = np.einsum("tl,ile->tie", t["c"][0, 0][target], t["w_p"]) * gate
+    np.testing.assert_allclose(got[0], want, rtol=1e-10, atol=1e-12)
+
+
+# ---------------------------------------------------------------- P9: sharing inside a group
+def test_heads_of_one_map_share_probabilities(oracle):
+    s = Shape(1, 12, 8, 4, 2, 2, 1, 4, 8, 1)
+    t = _inputs(s)
+    wg = t["w_g"].reshape(8, 4, 4)
+    t["w_p"][1] = t["w_p"][0]; wg[:, 1] = wg[:, 0]        # heads 0,1: same map (group 0)
+    t["w_p"][2] = t["w_p"][0]; wg[:, 2] = wg[:, 0]        # head 2: other map (group 1)
+    t["w_g"] = wg.reshape(8, 16)
+    out = oracle.prefill(s, **t)
+    assert np.array_equal(out[:, :, 0], out[:, :, 1])
+    assert not np.allclose(out[:, 1:, 0], out[:, 1:, 2])
+    # head -> group map is by contiguous blocks: swapping query groups swaps head blocks
+    t2 = dict(t); t2["q"] = t["q"][:, ::-1].copy(); t2["k"] = t["k"][:, ::-1].copy()
+    out2 = oracle.prefill(s, **t2)
+    assert np.array_equal(out2[:, :, 2], out[:, :, 0])
+
+
+# ---------------------------------------------------------------- P10: printed cost figures
+def test_cost_model_matches_printed_ratios(oracle):
+    """Table 3 closed forms at the 1B hyper-parameters (App. A, model table) give the printed
+    37.5 % attention cost and 30 % cache of GQA-1B; printed cache widths 192 / 320 / 384."""
+    N = 2048
+    gta_1b = Shape(1, N, 1280, 20, 5, 1, 1, 64, 128)
+    gqa_attn = 2 * 20 * 64 * N * N            # 2 n_h d_h N^2
+    gqa_cache = 2 * 5 * 64 * N                # 2 n_k d_h N with 5 KV heads
+    assert oracle.attention_cost(gta_1b) / gqa_attn == pytest.approx(0.375, abs=1e-12)
+    assert oracle.cache_elems(gta_1b) / gqa_cache == pytest.approx(0.30, abs=1e-12)
+    assert oracle.cache_elems(Shape(1, 1, 768, 12, 3, 1, 1, 64, 128)) == 192      # GTA1
+    assert oracle.cache_elems(Shape(1, 1, 1280, 20, 10, 1, 2, 64, 128)) == 320    # GTA4
+    assert oracle.cache_elems(Shape(1, 1, 1280, 10, 5, 1, 1, 128, 256)) == 384    # d_h = 128 ablation
+    assert 192 / 1536 == 0.125 and 320 / 2560 == 0.125 and 192 / 2560 == 0.075    # vs MHA
+
+
+def test_weight_shapes_agree_with_printed_parameter_counts():
+    """The printed parameter totals (in units of 2^20) fix the decoder shapes: W_P is n_h dense
+    d_l x d_h blocks and W_G is H x n_h d_h."""
+    M = 2.0 ** 20
+    layers = 24
+    # GTA1 - GQA at 160M: GQA has K,V = 2*3*64 columns; GTA1 has Q 3*64, K 64, C 128, W_P, W_G
+    H, nh, dh, dl = 768, 12, 64, 128
+    gqa = H * nh * dh + 2 * H * 3 * dh
+    gta1 = H * 3 * dh + H * dh + H * dl + nh * dl * dh + H * nh * dh
+    assert layers * (gta1 - gqa) / M == pytest.approx(160.75 - 158.50, abs=0.006)
+    gta2 = gta1 + H * 3 * dh                                   # six query groups instead of three
+    assert layers * (gta2 - gta1) / M == pytest.approx(164.13 - 160.75, abs=0.006)
+    H, nh = 1280, 20
+    gta3 = H * 5 * dh + H * dh + H * dl + nh * dl * dh + H * nh * dh
+    gta4 = H * 10 * dh + H * dh + H * 2 * dl + nh * dl * dh + H * nh * dh
+    assert layers * (gta4 - gta3) / M == pytest.approx(500.11 - 486.98, abs=0.006)
+
+
+# ---------------------------------------------------------------- P12: independence
+def test_batch_permutation_permutes_outputs(oracle):
+    s = Shape(3, 6, 8, 4, 2, 1, 1, 4, 8, 1)
+    t = _inputs(s)
+    out = oracle.prefill(s, **t)
+    perm = [2, 0, 1]
+    t2 = {k: (v[perm].copy() if k in ("q", "k", "c", "x") else v) for k, v in t.items()}
+    assert np.array_equal(oracle.prefill(s, **t2), out[perm])
+
+
+# ---------------------------------------------------------------- storage types, append
+def test_bf16_and_f32_storage_are_widened_exactly(oracle):
+    import torch
+    s = Shape(1, 9, 8, 4, 2, 2, 1, 4, 8, 1)
+    t = {k: torch.from_numpy(v).to(torch.bfloat16) for k, v in _inputs(s).items()}
+    out_bf = oracle.prefill(s, **t)
+    out_f32 = oracle.prefill(s, **{k: v.float() for k, v in t.items()})
+    out_f64 = oracle.prefill(s, **{k: v.double().numpy() for k, v in t.items()})
+    assert np.array_equal(out_bf, out_f64) and np.array_equal(out_f32, out_f64)
+
+
+def test_cache_append_is_a_byte_copy_with_overflow_skip(oracle):
+    B, cap = 3, 6
+    s = Shape(B, 0, 4, 2, 2, 2, 1, 4, 8, 1)
+    kc = RNG.integers(0, 2 ** 16, (B, 2, cap, 4)).astype(np.uint16)
+    cc = RNG.integers(0, 2 ** 16, (B, 1, cap, 8)).astype(np.uint16)
+    kn = RNG.integers(0, 2 ** 16, (B, 2, 2, 4)).astype(np.uint16)
+    cn = RNG.integers(0, 2 ** 16, (B, 1, 2, 8)).astype(np.uint16)
+    lens = np.array([0, 4, 5], dtype=np.int32)          # the last one would overflow (5 + 2 > 6)
+    k2, c2, l2, ov = oracle.cache_append(s, kc, cc, cap, kn, cn, 2, lens)
+    assert ov == 1 and l2.tolist() == [2, 6, 5]
+    want_k, want_c = kc.copy(), cc.copy()
+    want_k[0, :, 0:2] = kn[0]; want_c[0, :, 0:2] = cn[0]
+    want_k[1, :, 4:6] = kn[1]; want_c[1, :, 4:6] = cn[1]
+    assert np.array_equal(k2, want_k) and np.array_equal(c2, want_c)
+    assert np.array_equal(kc[2], k2[2]) and np.array_equal(cc[2], c2[2])
