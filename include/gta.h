@@ -1,0 +1,177 @@
+/*
+ * gta.h — C ABI of the B200 (sm_100a) GTA attention operator library.
+ *
+ * GTA = Grouped-head latenT Attention.  One attention map is computed per query group
+ * and shared by every head of the group; the probabilities are applied to a compressed
+ * latent value tensor C (d_l wide) instead of per-head values; each head then decodes its
+ * value with its own projection W_P,i and a sigmoid gate computed from the hidden state
+ * of the query token (paper Sec. 3.2 "Input projections and grouping", "Nonlinear value
+ * decoder", and Sec. 3.3 "Efficient attention computation", reformulated equation).
+ *
+ * Symbols (paper Sec. 3.2): B batch, N sequence length, H hidden size (d_model), n_h heads,
+ * n_q / n_k / n_c query / key / latent groups, d_h head dim, d_l latent dim (d_l >= d_h).
+ * Head -> group maps are contiguous blocks:
+ *   q(i) = floor(i * n_q / n_h),  k(i) = floor(q(i) * n_k / n_q),  c(i) = floor(q(i) * n_c / n_q)
+ * which needs n_q | n_h, n_k | n_q and n_c | n_q.
+ *
+ * General rules for every entry point
+ *   - Every tensor pointer is a DEVICE pointer unless it says "host".  The caller owns all
+ *     buffers; the library allocates no device memory and keeps no per-call state.
+ *   - Tensors are dense, row-major, innermost dimension last, base address 16-byte aligned.
+ *   - All work is enqueued on `cuda_stream` (a cudaStream_t cast to void*; NULL = the legacy
+ *     default stream).  No call synchronises the device or the stream.
+ *   - Errors the host can see (null pointer, misalignment, bad divisibility, unsupported
+ *     sizes, workspace too small, not an sm_100 device) are returned as a status code before
+ *     anything is launched.  Conditions only the device can see (a full cache, a bounded wait
+ *     that ran out) are written to `*status_word`, a device int32 the caller zeroes and reads
+ *     after its own synchronisation; kernels only ever raise it (atomic max) and it may be NULL.
+ *   - No entry point aborts, traps or throws.
+ */
+#ifndef GTA_H_
+#define GTA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define GTA_API __attribute__((visibility("default")))
+#else
+#define GTA_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    GTA_OK = 0,
+    GTA_ERR_INVALID_ARG = 1, /* null pointer, misaligned pointer, negative size, bad divisibility */
+    GTA_ERR_UNSUPPORTED = 2, /* shape / dtype / device outside what the kernels cover */
+    GTA_ERR_WORKSPACE = 3,   /* workspace missing or smaller than *_workspace_bytes() */
+    GTA_ERR_CUDA = 4,        /* a CUDA runtime / driver call failed (launch, attribute, tensor map) */
+    GTA_ERR_CACHE_FULL = 5,  /* device-side: an append would exceed S_cap for some sequence */
+    GTA_ERR_TIMEOUT = 6      /* device-side: a bounded wait inside a kernel ran out */
+} gta_status_t;
+
+typedef enum { GTA_F32 = 0, GTA_BF16 = 1 } gta_dtype_t;
+
+typedef struct {
+    int32_t batch;       /* B */
+    int32_t seq;         /* prefill: N (query length = key length).  decode / append: ignored */
+    int32_t d_model;     /* H: row length of x and number of rows of W_G */
+    int32_t n_heads;     /* n_h */
+    int32_t n_q_groups;  /* n_q: number of attention maps; must divide n_h */
+    int32_t n_k_groups;  /* n_k: must divide n_q */
+    int32_t n_c_groups;  /* n_c: must divide n_q */
+    int32_t head_dim;    /* d_h */
+    int32_t latent_dim;  /* d_l */
+    int32_t causal;      /* 1: key j <= query t (diagonal included, App. B.1.1); 0: all keys */
+    int32_t dtype;       /* gta_dtype_t; storage type of EVERY tensor argument */
+    float softmax_scale; /* 0 => 1/sqrt(d_h) (Sec. 3.3) */
+} gta_shape_t;
+
+/*
+ * gta_prefill — causal prefill of the whole operator (Sec. 3.3, reformulated equation, with
+ * the causal sum of App. B.1.1):
+ *   P_g   = Softmax(scale * Q_g K_{k(g)}^T)            one map per query group g
+ *   L_g   = P_g C_{c(g)}                               [N, d_l]
+ *   out_i = (L_{q(i)} W_P,i) (.) Sigmoid(X W_G,i)      per head i; the gate of row t uses x_t
+ * The output projection W_O and RoPE are outside the operator (q, k arrive post-RoPE).
+ *
+ *   q   [B, n_q, N, d_h]      k   [B, n_k, N, d_h]      c  [B, n_c, N, d_l]
+ *   x   [B, N, H]             w_p [n_h, d_l, d_h]       w_g [H, n_h*d_h]
+ *   out [B, N, n_h, d_h]      (written; same dtype as the inputs, round-to-nearest-even)
+ *   workspace: at least gta_prefill_workspace_bytes(shape) bytes, 256-byte aligned; holds
+ *     the normalised latent attention output L between the two kernels; contents undefined
+ *     afterwards.  Calls that share a workspace must be ordered on one stream.
+ * Arithmetic: fp32 accumulation everywhere.  bf16 fast path (tcgen05 tensor cores) when
+ * dtype = bf16, d_h = 128, d_l a multiple of 256, H a multiple of 64; other shapes and fp32
+ * run on the plain-ALU kernels of the same library.  N = 0 or B = 0 is a no-op (GTA_OK).
+ */
+GTA_API size_t gta_prefill_workspace_bytes(const gta_shape_t *shape);
+GTA_API gta_status_t gta_prefill(const gta_shape_t *shape, const void *q, const void *k, const void *c,
+                         const void *x, const void *w_p, const void *w_g, void *out,
+                         void *workspace, size_t workspace_bytes, int32_t *status_word,
+                         void *cuda_stream);
+
+/*
+ * gta_decode — one decode step (App. B.1.3): for every sequence b the new token's queries
+ * attend the seq_lens[b] cached keys / latents (the new token's own entries included, i.e.
+ * gta_cache_append has already run), then the decoder and gate of gta_prefill are applied
+ * with x_t = hidden state of the new token.  Equals row seq_lens[b]-1 of gta_prefill.
+ *
+ *   q        [B, n_q, d_h]                 x_t [B, H]
+ *   k_cache  [B, n_k, S_cap, d_h]          c_cache [B, n_c, S_cap, d_l]
+ *   seq_lens device int32 [B], 0 <= seq_lens[b] <= S_cap (values above S_cap are clamped);
+ *            a sequence with length 0 gets an all-zero output row
+ *   w_p, w_g as in gta_prefill;  out [B, n_h, d_h]
+ *   workspace: at least gta_decode_workspace_bytes(shape, S_cap) bytes, 256-byte aligned
+ *     (split-KV partial results and gate partial sums).
+ * Needs d_h and d_l multiples of 8 (bf16) / 4 (fp32) so that rows are 16-byte vectors,
+ * d_h <= 256, d_l <= 2048.
+ */
+GTA_API size_t gta_decode_workspace_bytes(const gta_shape_t *shape, int32_t S_cap);
+GTA_API gta_status_t gta_decode(const gta_shape_t *shape, const void *q, const void *k_cache,
+                        const void *c_cache, const int32_t *seq_lens, int32_t S_cap,
+                        const void *x_t, const void *w_p, const void *w_g, void *out,
+                        void *workspace, size_t workspace_bytes, int32_t *status_word,
+                        void *cuda_stream);
+
+/*
+ * gta_cache_append — write new keys and latents behind the live part of the caches (the
+ * caches hold K and C of every past token: Sec. 3.3, last paragraph; App. B.1.3).  Pure
+ * byte copy, bit-exact:
+ *   for b with seq_lens[b] + n_new <= S_cap:
+ *     k_cache[b, :, seq_lens[b] + n, :] = k_new[b, :, n, :]   n = 0 .. n_new-1   (c likewise)
+ *     seq_lens[b] += n_new
+ *   a sequence that would overflow is skipped entirely (cache and length unchanged) and
+ *   *status_word is raised to GTA_ERR_CACHE_FULL.
+ *
+ *   k_cache [B, n_k, S_cap, d_h]  c_cache [B, n_c, S_cap, d_l]   (read-modify-write)
+ *   k_new   [B, n_k, n_new, d_h]  c_new   [B, n_c, n_new, d_l]
+ *   seq_lens device int32 [B] in/out.   n_new = 1 per decode step; n_new = N loads a prefill.
+ * Rows must be multiples of 16 bytes (d_h, d_l multiples of 8 for bf16, 4 for fp32).
+ */
+GTA_API gta_status_t gta_cache_append(const gta_shape_t *shape, void *k_cache, void *c_cache,
+                              int32_t S_cap, const void *k_new, const void *c_new,
+                              int32_t n_new, int32_t *seq_lens, int32_t *status_word,
+                              void *cuda_stream);
+
+/*
+ * Profiling aids (no counterpart in the paper): the same calls restricted to a subset of their
+ * kernels, so that each kernel can be timed or captured alone.  `stages` is a bit mask;
+ * gta_prefill_stages: 1 = attention kernel (writes L to the workspace), 2 = decoder + gate
+ * kernel (reads L from the workspace); gta_decode_stages: 1 = gate partial sums, 2 = split-KV
+ * cache kernel, 4 = merge + decoder.  A mask of all stages equals the plain call.  The
+ * workspace must still hold what the skipped stages would have written.
+ */
+GTA_API gta_status_t gta_prefill_stages(const gta_shape_t *shape, const void *q, const void *k,
+                                        const void *c, const void *x, const void *w_p, const void *w_g,
+                                        void *out, void *workspace, size_t workspace_bytes,
+                                        int32_t *status_word, void *cuda_stream, int32_t stages);
+GTA_API gta_status_t gta_decode_stages(const gta_shape_t *shape, const void *q, const void *k_cache,
+                                       const void *c_cache, const int32_t *seq_lens, int32_t S_cap,
+                                       const void *x_t, const void *w_p, const void *w_g, void *out,
+                                       void *workspace, size_t workspace_bytes, int32_t *status_word,
+                                       void *cuda_stream, int32_t stages);
+
+/* Host helpers. */
+GTA_API const char *gta_status_string(gta_status_t status); /* static string, never NULL */
+GTA_API int gta_version(void);                              /* major*10000 + minor*100 + patch */
+
+/*
+ * Which kernel family gta_prefill would use for `shape` on the current device:
+ *   0 = invalid / unsupported, 1 = plain-ALU fp32 kernels, 2 = tcgen05 tensor-core kernels.
+ */
+GTA_API int gta_prefill_path(const gta_shape_t *shape);
+
+/*
+ * Number of kernel launches the last successful call of this thread enqueued (for
+ * benchmark accounting; host-side counter only).
+ */
+GTA_API int gta_last_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GTA_H_ */

@@ -1,0 +1,231 @@
+"""Thin ctypes binding of the C-ABI library (`include/gta.h`): argument marshalling only.
+
+Every step of the operator runs inside the CUDA library; PyTorch is used for device memory,
+streams and host<->device copies.  There is no CPU fallback: if `libgta_b200.so` has not been
+built (``python -m paper_2506_17286_b200.build``) every entry point raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libgta_b200.so")
+
+GTA_OK, GTA_ERR_INVALID_ARG, GTA_ERR_UNSUPPORTED, GTA_ERR_WORKSPACE = 0, 1, 2, 3
+GTA_ERR_CUDA, GTA_ERR_CACHE_FULL, GTA_ERR_TIMEOUT = 4, 5, 6
+GTA_F32, GTA_BF16 = 0, 1
+
+EXPORTS = (
+    "gta_prefill_workspace_bytes", "gta_prefill", "gta_decode_workspace_bytes", "gta_decode",
+    "gta_cache_append", "gta_status_string", "gta_version", "gta_prefill_path", "gta_last_launch_count",
+    "gta_prefill_stages", "gta_decode_stages",
+)
+
+
+class GtaShape(ctypes.Structure):
+    """Mirror of gta_shape_t."""
+    _fields_ = [
+        ("batch", ctypes.c_int32), ("seq", ctypes.c_int32), ("d_model", ctypes.c_int32),
+        ("n_heads", ctypes.c_int32), ("n_q_groups", ctypes.c_int32), ("n_k_groups", ctypes.c_int32),
+        ("n_c_groups", ctypes.c_int32), ("head_dim", ctypes.c_int32), ("latent_dim", ctypes.c_int32),
+        ("causal", ctypes.c_int32), ("dtype", ctypes.c_int32), ("softmax_scale", ctypes.c_float),
+    ]
+
+
+class GtaError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {status_string(status)} (status {status})")
+
+
+_lib = None
+
+
+def lib():
+    """Load the shared library (once).  Raises if it is missing: there is no fallback."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(
+                f"{LIB_PATH} not found: build it with `python -m paper_2506_17286_b200.build` "
+                "(the GTA operator has no CPU or PyTorch fallback)")
+        L = ctypes.CDLL(LIB_PATH)
+        vp, i32, sz = ctypes.c_void_p, ctypes.c_int32, ctypes.c_size_t
+        sp = ctypes.POINTER(GtaShape)
+        L.gta_prefill_workspace_bytes.argtypes = [sp]
+        L.gta_prefill_workspace_bytes.restype = sz
+        L.gta_prefill.argtypes = [sp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp, vp]
+        L.gta_prefill.restype = i32
+        L.gta_prefill_stages.argtypes = [sp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp, vp, i32]
+        L.gta_prefill_stages.restype = i32
+        L.gta_decode_stages.argtypes = [sp, vp, vp, vp, vp, i32, vp, vp, vp, vp, vp, sz, vp, vp, i32]
+        L.gta_decode_stages.restype = i32
+        L.gta_decode_workspace_bytes.argtypes = [sp, i32]
+        L.gta_decode_workspace_bytes.restype = sz
+        L.gta_decode.argtypes = [sp, vp, vp, vp, vp, i32, vp, vp, vp, vp, vp, sz, vp, vp]
+        L.gta_decode.restype = i32
+        L.gta_cache_append.argtypes = [sp, vp, vp, i32, vp, vp, i32, vp, vp, vp]
+        L.gta_cache_append.restype = i32
+        L.gta_status_string.argtypes = [i32]
+        L.gta_status_string.restype = ctypes.c_char_p
+        L.gta_version.restype = i32
+        L.gta_prefill_path.argtypes = [sp]
+        L.gta_prefill_path.restype = i32
+        L.gta_last_launch_count.restype = i32
+        _lib = L
+    return _lib
+
+
+def status_string(status: int) -> str:
+    return lib().gta_status_string(int(status)).decode()
+
+
+def version() -> int:
+    return int(lib().gta_version())
+
+
+def last_launch_count() -> int:
+    return int(lib().gta_last_launch_count())
+
+
+def _dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return GTA_F32
+    if t.dtype == torch.bfloat16:
+        return GTA_BF16
+    raise TypeError(f"unsupported dtype {t.dtype}: the library takes float32 or bfloat16")
+
+
+def _ptr(t):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(stream):
+    s = torch.cuda.current_stream() if stream is None else stream
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+def _check_tensors(*ts):
+    dev, dt = ts[0].device, ts[0].dtype
+    for t in ts:
+        if t.device != dev or t.dtype != dt:
+            raise ValueError("all operator tensors must share one device and one dtype")
+        if not t.is_contiguous():
+            raise ValueError("operator tensors must be contiguous")
+        if t.device.type != "cuda":
+            raise ValueError("operator tensors must live on a CUDA device")
+
+
+def make_shape(*, batch, seq, d_model, n_heads, n_q, n_k, n_c, d_h, d_l, dtype, causal=True,
+               softmax_scale=0.0) -> GtaShape:
+    code = dtype if isinstance(dtype, int) else (GTA_F32 if dtype == torch.float32 else GTA_BF16)
+    return GtaShape(batch, seq, d_model, n_heads, n_q, n_k, n_c, d_h, d_l, int(bool(causal)), code,
+                    float(softmax_scale))
+
+
+def prefill_workspace_bytes(shape: GtaShape) -> int:
+    return int(lib().gta_prefill_workspace_bytes(ctypes.byref(shape)))
+
+
+def decode_workspace_bytes(shape: GtaShape, s_cap: int) -> int:
+    return int(lib().gta_decode_workspace_bytes(ctypes.byref(shape), int(s_cap)))
+
+
+def prefill_path(shape: GtaShape) -> int:
+    return int(lib().gta_prefill_path(ctypes.byref(shape)))
+
+
+def _workspace(nbytes: int, device) -> torch.Tensor:
+    return torch.empty(max(nbytes, 256), dtype=torch.uint8, device=device)
+
+
+def gta_prefill(q, k, c, x, w_p, w_g, *, causal=True, softmax_scale=0.0, out=None, workspace=None,
+                status_word=None, stream=None, stages=3):
+    """out[B, N, n_h, d_h] = GTA prefill.  q [B,n_q,N,d_h], k [B,n_k,N,d_h], c [B,n_c,N,d_l],
+    x [B,N,H], w_p [n_h,d_l,d_h], w_g [H,n_h*d_h]; all on one CUDA device, one dtype."""
+    _check_tensors(q, k, c, x, w_p, w_g)
+    B, n_q, N, d_h = q.shape
+    n_k, n_c, d_l = k.shape[1], c.shape[1], c.shape[3]
+    n_h, H = w_p.shape[0], x.shape[2]
+    if k.shape != (B, n_k, N, d_h) or c.shape != (B, n_c, N, d_l) or x.shape != (B, N, H) \
+            or w_p.shape != (n_h, d_l, d_h) or w_g.shape != (H, n_h * d_h):
+        raise ValueError("inconsistent operator tensor shapes")
+    shape = make_shape(batch=B, seq=N, d_model=H, n_heads=n_h, n_q=n_q, n_k=n_k, n_c=n_c, d_h=d_h, d_l=d_l,
+                       dtype=_dtype_code(q), causal=causal, softmax_scale=softmax_scale)
+    if out is None:
+        out = torch.empty((B, N, n_h, d_h), dtype=q.dtype, device=q.device)
+    need = prefill_workspace_bytes(shape)
+    if workspace is None:
+        workspace = _workspace(need, q.device)
+    args = (ctypes.byref(shape), _ptr(q), _ptr(k), _ptr(c), _ptr(x), _ptr(w_p), _ptr(w_g), _ptr(out),
+            _ptr(workspace), workspace.numel() * workspace.element_size(), _ptr(status_word), _stream(stream))
+    st = lib().gta_prefill(*args) if stages == 3 else lib().gta_prefill_stages(*args, stages)
+    if st != GTA_OK:
+        raise GtaError(st, "gta_prefill")
+    return out
+
+
+def decode_shape(q, k_cache, c_cache, x_t, w_p, causal=True, softmax_scale=0.0) -> GtaShape:
+    B, n_q, d_h = q.shape
+    return make_shape(batch=B, seq=0, d_model=x_t.shape[1], n_heads=w_p.shape[0], n_q=n_q,
+                      n_k=k_cache.shape[1], n_c=c_cache.shape[1], d_h=d_h, d_l=c_cache.shape[3],
+                      dtype=_dtype_code(q), causal=causal, softmax_scale=softmax_scale)
+
+
+def gta_decode(q, k_cache, c_cache, seq_lens, x_t, w_p, w_g, *, softmax_scale=0.0, out=None, workspace=None,
+               status_word=None, stream=None, stages=7):
+    """out[B, n_h, d_h] = one decode step.  q [B,n_q,d_h], k_cache [B,n_k,S_cap,d_h],
+    c_cache [B,n_c,S_cap,d_l], seq_lens int32 [B] (new token included), x_t [B,H]."""
+    _check_tensors(q, k_cache, c_cache, x_t, w_p, w_g)
+    if seq_lens.dtype != torch.int32 or seq_lens.device != q.device or not seq_lens.is_contiguous():
+        raise ValueError("seq_lens must be a contiguous int32 tensor on the operator's device")
+    B, n_q, d_h = q.shape
+    s_cap = k_cache.shape[2]
+    shape = decode_shape(q, k_cache, c_cache, x_t, w_p, softmax_scale=softmax_scale)
+    n_h, d_l, H = shape.n_heads, shape.latent_dim, shape.d_model
+    if k_cache.shape != (B, shape.n_k_groups, s_cap, d_h) or c_cache.shape != (B, shape.n_c_groups, s_cap, d_l) \
+            or x_t.shape != (B, H) or w_p.shape != (n_h, d_l, d_h) or w_g.shape != (H, n_h * d_h) \
+            or seq_lens.shape != (B,):
+        raise ValueError("inconsistent operator tensor shapes")
+    if out is None:
+        out = torch.empty((B, n_h, d_h), dtype=q.dtype, device=q.device)
+    if workspace is None:
+        workspace = _workspace(decode_workspace_bytes(shape, s_cap), q.device)
+    args = (ctypes.byref(shape), _ptr(q), _ptr(k_cache), _ptr(c_cache), _ptr(seq_lens), s_cap, _ptr(x_t),
+            _ptr(w_p), _ptr(w_g), _ptr(out), _ptr(workspace), workspace.numel() * workspace.element_size(),
+            _ptr(status_word), _stream(stream))
+    st = lib().gta_decode(*args) if stages == 7 else lib().gta_decode_stages(*args, stages)
+    if st != GTA_OK:
+        raise GtaError(st, "gta_decode")
+    return out
+
+
+def gta_cache_append(k_cache, c_cache, k_new, c_new, seq_lens, *, status_word=None, stream=None):
+    """In place: rows k_new [B,n_k,n_new,d_h] / c_new [B,n_c,n_new,d_l] go behind seq_lens[b] in the
+    caches and seq_lens advances by n_new.  A full sequence is skipped and raises *status_word."""
+    _check_tensors(k_cache, c_cache, k_new, c_new)
+    if seq_lens.dtype != torch.int32 or seq_lens.device != k_cache.device or not seq_lens.is_contiguous():
+        raise ValueError("seq_lens must be a contiguous int32 tensor on the caches' device")
+    B, n_k, s_cap, d_h = k_cache.shape
+    n_c, d_l = c_cache.shape[1], c_cache.shape[3]
+    n_new = k_new.shape[2]
+    if c_cache.shape != (B, n_c, s_cap, d_l) or k_new.shape != (B, n_k, n_new, d_h) \
+            or c_new.shape != (B, n_c, n_new, d_l) or seq_lens.shape != (B,):
+        raise ValueError("inconsistent cache tensor shapes")
+    n_q = n_k * n_c // _gcd(n_k, n_c)   # any common multiple serves: append ignores the query groups
+    shape = make_shape(batch=B, seq=0, d_model=8, n_heads=n_q, n_q=n_q, n_k=n_k, n_c=n_c, d_h=d_h, d_l=d_l,
+                       dtype=_dtype_code(k_cache))
+    st = lib().gta_cache_append(ctypes.byref(shape), _ptr(k_cache), _ptr(c_cache), s_cap, _ptr(k_new),
+                                _ptr(c_new), n_new, _ptr(seq_lens), _ptr(status_word), _stream(stream))
+    if st != GTA_OK:
+        raise GtaError(st, "gta_cache_append")
+    return seq_lens
+
+
+def _gcd(a, b):
+    while b:
+        a, b = b, a % b
+    return a

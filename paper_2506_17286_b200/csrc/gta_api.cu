@@ -1,0 +1,202 @@
+// C-ABI entry points: argument validation and dispatch to the kernel launchers.
+#include <math.h>
+
+#include "gta_common.cuh"
+#include "gta_sm100.cuh"
+
+namespace {
+
+thread_local int g_last_launches = 0;
+
+bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
+
+// Is the current device a Blackwell data-centre part (compute capability 10.x)?
+gta_status_t check_device() {
+    static thread_local int cached_dev = -1;
+    static thread_local int cached_major = 0;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return GTA_ERR_CUDA;
+    if (dev != cached_dev) {
+        int major = 0;
+        if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess)
+            return GTA_ERR_CUDA;
+        cached_dev = dev;
+        cached_major = major;
+    }
+    return cached_major == 10 ? GTA_OK : GTA_ERR_UNSUPPORTED;
+}
+
+// Shape checks common to all entry points.  `need_seq`: prefill uses shape->seq.
+gta_status_t check_shape(const gta_shape_t* s, bool need_seq, gta::Dims* d) {
+    if (!s) return GTA_ERR_INVALID_ARG;
+    if (s->batch < 0 || (need_seq && s->seq < 0) || s->d_model < 1 || s->n_heads < 1 || s->n_q_groups < 1 ||
+        s->n_k_groups < 1 || s->n_c_groups < 1 || s->head_dim < 1 || s->latent_dim < 1)
+        return GTA_ERR_INVALID_ARG;
+    if (s->n_heads % s->n_q_groups || s->n_q_groups % s->n_k_groups || s->n_q_groups % s->n_c_groups)
+        return GTA_ERR_INVALID_ARG;
+    if (s->dtype != GTA_F32 && s->dtype != GTA_BF16) return GTA_ERR_INVALID_ARG;
+    if (s->causal != 0 && s->causal != 1) return GTA_ERR_INVALID_ARG;
+    if (!(s->softmax_scale >= 0.f) || isinf(s->softmax_scale)) return GTA_ERR_INVALID_ARG;
+    // rows are moved as 16-byte vectors
+    if (s->head_dim % 8 || s->latent_dim % 8 || s->d_model % 8) return GTA_ERR_UNSUPPORTED;
+    if (s->head_dim > 256 || s->batch > 65535 || s->n_q_groups > 65535 || s->n_heads > 65535)
+        return GTA_ERR_UNSUPPORTED;
+    d->B = s->batch; d->N = need_seq ? s->seq : 0; d->H = s->d_model; d->n_h = s->n_heads;
+    d->n_q = s->n_q_groups; d->n_k = s->n_k_groups; d->n_c = s->n_c_groups;
+    d->d_h = s->head_dim; d->d_l = s->latent_dim; d->causal = s->causal;
+    d->scale = s->softmax_scale > 0.f ? s->softmax_scale : 1.0f / sqrtf((float)s->head_dim);
+    return GTA_OK;
+}
+
+size_t elem_size(int dtype) { return dtype == GTA_F32 ? 4 : 2; }
+
+}  // namespace
+
+extern "C" {
+
+const char* gta_status_string(gta_status_t status) {
+    switch (status) {
+        case GTA_OK: return "ok";
+        case GTA_ERR_INVALID_ARG: return "invalid argument";
+        case GTA_ERR_UNSUPPORTED: return "unsupported shape, dtype or device";
+        case GTA_ERR_WORKSPACE: return "workspace missing or too small";
+        case GTA_ERR_CUDA: return "CUDA call failed";
+        case GTA_ERR_CACHE_FULL: return "cache full";
+        case GTA_ERR_TIMEOUT: return "bounded device wait ran out";
+    }
+    return "unknown status";
+}
+
+int gta_version(void) { return 100; }
+
+int gta_last_launch_count(void) { return g_last_launches; }
+
+int gta_prefill_path(const gta_shape_t* shape) {
+    gta::Dims d;
+    if (check_shape(shape, true, &d) != GTA_OK) return 0;
+    if (gta::sm100_prefill_supported(d, shape->dtype)) return 2;
+    if (d.d_l > 1024) return 0;
+    return 1;
+}
+
+size_t gta_prefill_workspace_bytes(const gta_shape_t* shape) {
+    gta::Dims d;
+    if (check_shape(shape, true, &d) != GTA_OK) return 0;
+    // normalised latent attention output L[B, n_q, N, d_l]: fp32 on the plain-ALU path, bf16 on
+    // the tensor-core path; sized for the larger so either path may run.
+    size_t bytes = (size_t)d.B * d.n_q * d.N * d.d_l * sizeof(float);
+    return bytes < 256 ? 256 : ((bytes + 255) & ~(size_t)255);
+}
+
+gta_status_t gta_prefill(const gta_shape_t* shape, const void* q, const void* k, const void* c,
+                         const void* x, const void* w_p, const void* w_g, void* out, void* workspace,
+                         size_t workspace_bytes, int32_t* status_word, void* cuda_stream) {
+    return gta_prefill_stages(shape, q, k, c, x, w_p, w_g, out, workspace, workspace_bytes, status_word,
+                              cuda_stream, 3);
+}
+
+gta_status_t gta_prefill_stages(const gta_shape_t* shape, const void* q, const void* k, const void* c,
+                                const void* x, const void* w_p, const void* w_g, void* out, void* workspace,
+                                size_t workspace_bytes, int32_t* status_word, void* cuda_stream,
+                                int32_t stages) {
+    g_last_launches = 0;
+    if (stages < 1 || stages > 3) return GTA_ERR_INVALID_ARG;
+    gta::Dims d;
+    gta_status_t st = check_shape(shape, true, &d);
+    if (st != GTA_OK) return st;
+    if (!q || !k || !c || !x || !w_p || !w_g || !out) return GTA_ERR_INVALID_ARG;
+    if (!aligned(q, 16) || !aligned(k, 16) || !aligned(c, 16) || !aligned(x, 16) || !aligned(w_p, 16) ||
+        !aligned(w_g, 16) || !aligned(out, 16) || !aligned(status_word, 4))
+        return GTA_ERR_INVALID_ARG;
+    const int path = gta_prefill_path(shape);
+    if (path == 0) return GTA_ERR_UNSUPPORTED;
+    if (d.B == 0 || d.N == 0) return GTA_OK;
+    if (!workspace || !aligned(workspace, 256) || workspace_bytes < gta_prefill_workspace_bytes(shape))
+        return GTA_ERR_WORKSPACE;
+    if ((st = check_device()) != GTA_OK) return st;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    int launches = 0;
+    cudaError_t err;
+    if (path == 2) {
+        st = gta::launch_sm100_prefill(d, q, k, c, x, w_p, w_g, out, workspace, status_word, stream, stages, &launches);
+        if (st != GTA_OK) return st;
+        err = cudaSuccess;
+    } else {
+        err = gta::launch_generic_prefill(d, shape->dtype, q, k, c, x, w_p, w_g, out,
+                                          static_cast<float*>(workspace), stream, stages, &launches);
+    }
+    if (err != cudaSuccess) return GTA_ERR_CUDA;
+    g_last_launches = launches;
+    return GTA_OK;
+}
+
+size_t gta_decode_workspace_bytes(const gta_shape_t* shape, int32_t S_cap) {
+    gta::Dims d;
+    if (check_shape(shape, false, &d) != GTA_OK || S_cap < 0) return 0;
+    return gta::decode_workspace_bytes(d, S_cap);
+}
+
+gta_status_t gta_decode(const gta_shape_t* shape, const void* q, const void* k_cache, const void* c_cache,
+                        const int32_t* seq_lens, int32_t S_cap, const void* x_t, const void* w_p,
+                        const void* w_g, void* out, void* workspace, size_t workspace_bytes,
+                        int32_t* status_word, void* cuda_stream) {
+    return gta_decode_stages(shape, q, k_cache, c_cache, seq_lens, S_cap, x_t, w_p, w_g, out, workspace,
+                             workspace_bytes, status_word, cuda_stream, 7);
+}
+
+gta_status_t gta_decode_stages(const gta_shape_t* shape, const void* q, const void* k_cache,
+                               const void* c_cache, const int32_t* seq_lens, int32_t S_cap, const void* x_t,
+                               const void* w_p, const void* w_g, void* out, void* workspace,
+                               size_t workspace_bytes, int32_t* status_word, void* cuda_stream,
+                               int32_t stages) {
+    g_last_launches = 0;
+    if (stages < 1 || stages > 7) return GTA_ERR_INVALID_ARG;
+    gta::Dims d;
+    gta_status_t st = check_shape(shape, false, &d);
+    if (st != GTA_OK) return st;
+    if (S_cap < 0) return GTA_ERR_INVALID_ARG;
+    if (!q || !seq_lens || !x_t || !w_p || !w_g || !out) return GTA_ERR_INVALID_ARG;
+    if (S_cap > 0 && (!k_cache || !c_cache)) return GTA_ERR_INVALID_ARG;
+    if (!aligned(q, 16) || !aligned(k_cache, 16) || !aligned(c_cache, 16) || !aligned(x_t, 16) ||
+        !aligned(w_p, 16) || !aligned(w_g, 16) || !aligned(out, 16) || !aligned(seq_lens, 4) ||
+        !aligned(status_word, 4))
+        return GTA_ERR_INVALID_ARG;
+    // one latent row is spread over at most 256 threads, 16 bytes each
+    if ((size_t)d.d_l * elem_size(shape->dtype) > 4096) return GTA_ERR_UNSUPPORTED;
+    if (d.B == 0) return GTA_OK;
+    if (!workspace || !aligned(workspace, 256) || workspace_bytes < gta::decode_workspace_bytes(d, S_cap))
+        return GTA_ERR_WORKSPACE;
+    if ((st = check_device()) != GTA_OK) return st;
+    int launches = 0;
+    cudaError_t err = gta::launch_decode(d, shape->dtype, q, k_cache, c_cache, seq_lens, S_cap, x_t, w_p, w_g,
+                                         out, workspace, status_word, static_cast<cudaStream_t>(cuda_stream),
+                                         stages, &launches);
+    if (err != cudaSuccess) return GTA_ERR_CUDA;
+    g_last_launches = launches;
+    return GTA_OK;
+}
+
+gta_status_t gta_cache_append(const gta_shape_t* shape, void* k_cache, void* c_cache, int32_t S_cap,
+                              const void* k_new, const void* c_new, int32_t n_new, int32_t* seq_lens,
+                              int32_t* status_word, void* cuda_stream) {
+    g_last_launches = 0;
+    gta::Dims d;
+    gta_status_t st = check_shape(shape, false, &d);
+    if (st != GTA_OK) return st;
+    if (S_cap < 0 || n_new < 0) return GTA_ERR_INVALID_ARG;
+    if (!k_cache || !c_cache || !k_new || !c_new || !seq_lens) return GTA_ERR_INVALID_ARG;
+    if (!aligned(k_cache, 16) || !aligned(c_cache, 16) || !aligned(k_new, 16) || !aligned(c_new, 16) ||
+        !aligned(seq_lens, 4) || !aligned(status_word, 4))
+        return GTA_ERR_INVALID_ARG;
+    if (d.B == 0 || n_new == 0) return GTA_OK;
+    if ((st = check_device()) != GTA_OK) return st;
+    int launches = 0;
+    cudaError_t err = gta::launch_cache_append(d, (int)elem_size(shape->dtype), k_cache, c_cache, S_cap, k_new,
+                                               c_new, n_new, seq_lens, status_word,
+                                               static_cast<cudaStream_t>(cuda_stream), &launches);
+    if (err != cudaSuccess) return GTA_ERR_CUDA;
+    g_last_launches = launches;
+    return GTA_OK;
+}
+
+}  // extern "C"

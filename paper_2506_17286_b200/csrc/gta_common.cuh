@@ -1,0 +1,61 @@
+// Internal helpers shared by the kernels of the GTA library (not part of the C ABI).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "gta.h"
+
+namespace gta {
+
+// Head -> group maps (contiguous blocks), Sec. 3.2 "Input projections and grouping".
+struct Dims {
+    int B, N, H, n_h, n_q, n_k, n_c, d_h, d_l, causal;
+    float scale;  // softmax scale, already resolved (1/sqrt(d_h) when the caller passed 0)
+    __host__ __device__ int head_to_q(int i) const { return (int)(((long long)i * n_q) / n_h); }
+    __host__ __device__ int q_to_k(int g) const { return (int)(((long long)g * n_k) / n_q); }
+    __host__ __device__ int q_to_c(int g) const { return (int)(((long long)g * n_c) / n_q); }
+};
+
+// Element access that widens the storage type to fp32 / narrows with round-to-nearest-even.
+template <typename T> __device__ __forceinline__ float to_f32(T v);
+template <> __device__ __forceinline__ float to_f32<float>(float v) { return v; }
+template <> __device__ __forceinline__ float to_f32<__nv_bfloat16>(__nv_bfloat16 v) { return __bfloat162float(v); }
+
+template <typename T> __device__ __forceinline__ T from_f32(float v);
+template <> __device__ __forceinline__ float from_f32<float>(float v) { return v; }
+template <> __device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
+
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+    return v;
+}
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+__device__ __forceinline__ void raise_status(int32_t* status_word, int code) {
+    if (status_word) atomicMax(status_word, code);
+}
+
+// Launchers implemented in the .cu files; each returns cudaGetLastError() of its launches and
+// adds the number of launches it made to *launches.
+cudaError_t launch_generic_prefill(const Dims& d, int dtype, const void* q, const void* k, const void* c,
+                                   const void* x, const void* w_p, const void* w_g, void* out,
+                                   float* o_lat_ws, cudaStream_t stream, int stages, int* launches);
+
+cudaError_t launch_decode(const Dims& d, int dtype, const void* q, const void* k_cache, const void* c_cache,
+                          const int32_t* seq_lens, int S_cap, const void* x_t, const void* w_p,
+                          const void* w_g, void* out, void* workspace, int32_t* status_word,
+                          cudaStream_t stream, int stages, int* launches);
+size_t decode_workspace_bytes(const Dims& d, int S_cap);
+
+cudaError_t launch_cache_append(const Dims& d, int elem_size, void* k_cache, void* c_cache, int S_cap,
+                                const void* k_new, const void* c_new, int n_new, int32_t* seq_lens,
+                                int32_t* status_word, cudaStream_t stream, int* launches);
+
+}  // namespace gta

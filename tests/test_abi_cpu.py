@@ -1,0 +1,110 @@
+"""CPU-only checks of the C-ABI library: it loads, exports every declared symbol, and rejects
+bad arguments on the host before anything could be launched (no GPU is touched)."""
+import ctypes
+import os
+import re
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def B():
+    from paper_2506_17286_b200 import build, binding
+    build.build()
+    binding.lib()
+    return binding
+
+
+def _declared_symbols():
+    text = open(os.path.join(ROOT, "include", "gta.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"GTA_API[^;(]*?\b(gta_\w+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported(B):
+    names = _declared_symbols()
+    assert set(names) >= {"gta_prefill", "gta_decode", "gta_cache_append"}
+    L = ctypes.CDLL(B.LIB_PATH)
+    for n in names:
+        assert hasattr(L, n), f"{n} declared in include/gta.h but not exported"
+    assert set(names) == set(B.EXPORTS)
+
+
+def test_version_and_status_strings(B):
+    assert B.version() >= 100
+    seen = {B.status_string(i) for i in range(7)}
+    assert len(seen) == 7 and B.status_string(0) == "ok"
+    assert B.status_string(99) == "unknown status"
+
+
+def _shape(B, **kw):
+    base = dict(batch=2, seq=64, d_model=64, n_heads=4, n_q=2, n_k=2, n_c=1, d_h=32, d_l=64, dtype=B.GTA_BF16)
+    base.update(kw)
+    return B.make_shape(**base)
+
+
+def test_workspace_sizes(B):
+    s = _shape(B)
+    assert B.prefill_workspace_bytes(s) >= 2 * 2 * 64 * 64 * 2
+    assert B.prefill_workspace_bytes(s) % 256 == 0
+    assert B.decode_workspace_bytes(s, 1000) > 0 and B.decode_workspace_bytes(s, 1000) % 256 == 0
+    assert B.decode_workspace_bytes(s, 4000) > B.decode_workspace_bytes(s, 1000)
+    assert B.prefill_workspace_bytes(_shape(B, n_q=3)) == 0       # n_q does not divide n_h
+    assert B.decode_workspace_bytes(s, -1) == 0
+
+
+def test_bad_arguments_are_rejected_on_the_host(B):
+    L = B.lib()
+    good = _shape(B)
+    buf = (ctypes.c_char * 4096)()
+    base = ctypes.addressof(buf)
+    p = ctypes.c_void_p((base + 255) & ~255)          # an aligned (host) address: never dereferenced
+    odd = ctypes.c_void_p(((base + 255) & ~255) + 2)
+    args = [p] * 7
+
+    def prefill(shape, a=args, ws=p, ws_bytes=1 << 40):
+        return L.gta_prefill(ctypes.byref(shape), *a, ws, ws_bytes, None, None)
+
+    assert L.gta_prefill(None, *args, p, 1 << 40, None, None) == B.GTA_ERR_INVALID_ARG
+    assert prefill(good, [None] + args[1:]) == B.GTA_ERR_INVALID_ARG
+    assert prefill(good, [odd] + args[1:]) == B.GTA_ERR_INVALID_ARG
+    assert prefill(_shape(B, n_k=3)) == B.GTA_ERR_INVALID_ARG          # n_k must divide n_q
+    assert prefill(_shape(B, n_c=4)) == B.GTA_ERR_INVALID_ARG          # n_c must divide n_q
+    assert prefill(_shape(B, dtype=7)) == B.GTA_ERR_INVALID_ARG
+    assert prefill(_shape(B, seq=-1)) == B.GTA_ERR_INVALID_ARG
+    assert prefill(_shape(B, softmax_scale=-1.0)) == B.GTA_ERR_INVALID_ARG
+    assert prefill(_shape(B, d_h=20)) == B.GTA_ERR_UNSUPPORTED         # rows must be 16-byte vectors
+    assert prefill(_shape(B, d_h=512, d_l=512)) == B.GTA_ERR_UNSUPPORTED
+    assert prefill(good, ws=None) == B.GTA_ERR_WORKSPACE
+    assert prefill(good, ws_bytes=16) == B.GTA_ERR_WORKSPACE
+    assert prefill(_shape(B, seq=0)) == B.GTA_OK                       # empty problem: no-op
+    assert prefill(_shape(B, batch=0)) == B.GTA_OK
+
+    def decode(shape, s_cap=128, ws=p, ws_bytes=1 << 40, lens=p):
+        return L.gta_decode(ctypes.byref(shape), p, p, p, lens, s_cap, p, p, p, p, ws, ws_bytes, None, None)
+
+    assert decode(good, s_cap=-1) == B.GTA_ERR_INVALID_ARG
+    assert decode(good, lens=None) == B.GTA_ERR_INVALID_ARG
+    assert decode(good, ws_bytes=8) == B.GTA_ERR_WORKSPACE
+    assert decode(_shape(B, d_l=4096)) == B.GTA_ERR_UNSUPPORTED
+    assert decode(_shape(B, batch=0)) == B.GTA_OK
+
+    def append(shape, n_new=1, lens=p):
+        return L.gta_cache_append(ctypes.byref(shape), p, p, 128, p, p, n_new, lens, None, None)
+
+    assert append(good, n_new=-1) == B.GTA_ERR_INVALID_ARG
+    assert append(good, lens=None) == B.GTA_ERR_INVALID_ARG
+    assert append(good, n_new=0) == B.GTA_OK
+
+
+def test_binding_rejects_cpu_tensors_and_missing_library(B, monkeypatch):
+    import torch
+    t = torch.zeros(1, 1, 8, 8)
+    with pytest.raises(ValueError):
+        B.gta_prefill(t, t, t, torch.zeros(1, 8, 8), torch.zeros(1, 8, 8), torch.zeros(8, 8))
+    monkeypatch.setattr(B, "_lib", None)
+    monkeypatch.setattr(B, "LIB_PATH", os.path.join(ROOT, "does_not_exist.so"))
+    with pytest.raises(RuntimeError, match="no CPU or PyTorch fallback"):
+        B.lib()

@@ -1,0 +1,230 @@
+"""GPU parity: the CUDA library (through its C ABI) against the fp64 CPU oracle, element by
+element on identical seeded inputs.  Sizes span several tiles plus ragged tails; the full-size
+workloads are checked on sampled rows / sequences the oracle can compute one by one."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2506_17286_b200 import inputs as I
+from tests.parity_utils import assert_close, cpu, oracle_shape
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def B():
+    if not torch.cuda.is_available():
+        pytest.skip("needs a CUDA device")
+    from paper_2506_17286_b200 import build, binding
+    build.build()
+    binding.lib()
+    return binding
+
+
+def _prefill_case(B, oracle, w, causal=True, rows=None, scale=0.0, project=True):
+    t = I.prefill_inputs(w, device="cuda", project=project)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    out = B.gta_prefill(t["q"], t["k"], t["c"], t["x"], t["w_p"], t["w_g"], causal=causal,
+                        softmax_scale=scale, status_word=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    tc = cpu(t)
+    want = oracle.prefill(oracle_shape(w, causal=int(causal), scale=scale), tc["q"], tc["k"], tc["c"], tc["x"],
+                          tc["w_p"], tc["w_g"], rows=rows)
+    got = out if rows is None else out[:, torch.as_tensor(rows, device=out.device, dtype=torch.long)]
+    return assert_close(got, want, w.torch_dtype(), w.name)
+
+
+# --------------------------------------------------------------------------- prefill
+def test_prefill_config1_tiny_fp32(B, oracle):
+    _prefill_case(B, oracle, I.CONFIGS["c1_tiny_prefill_f32"])
+
+
+SMALL_PREFILL = [
+    # name, dtype, B, N, H, n_h, n_q, n_k, n_c, d_h, d_l
+    ("bf16_tiles_ragged", "bf16", 2, 300, 256, 8, 4, 4, 1, 128, 512),
+    ("bf16_two_slices_long", "bf16", 1, 640, 128, 4, 2, 2, 1, 128, 256),
+    ("bf16_dl1024", "bf16", 1, 257, 192, 4, 2, 2, 1, 128, 1024),
+    ("bf16_shared_keys_two_latents", "bf16", 2, 200, 128, 8, 4, 2, 2, 64, 128),
+    ("bf16_paper_1b_shape", "bf16", 1, 160, 1280, 20, 5, 1, 1, 64, 128),
+    ("f32_general", "f32", 2, 150, 96, 6, 6, 3, 1, 32, 64),
+    ("f32_dh128", "f32", 1, 129, 64, 2, 1, 1, 1, 128, 256),
+]
+
+
+@pytest.mark.parametrize("case", SMALL_PREFILL, ids=[c[0] for c in SMALL_PREFILL])
+def test_prefill_small_shapes(B, oracle, case):
+    name, dt, *dims = case
+    w = I.Workload(name, "prefill", dt, *dims, seed=4242)
+    _prefill_case(B, oracle, w)
+
+
+@pytest.mark.parametrize("N", [1, 2, 127, 128, 129, 255, 256, 384])
+def test_prefill_tile_boundaries_bf16(B, oracle, N):
+    w = I.Workload(f"edge_{N}", "prefill", "bf16", 1, N, 128, 4, 2, 2, 1, 128, 256, seed=77 + N)
+    _prefill_case(B, oracle, w)
+
+
+def test_prefill_non_causal_and_explicit_scale(B, oracle):
+    w = I.Workload("noncausal", "prefill", "bf16", 1, 200, 128, 4, 2, 2, 1, 128, 256, seed=5)
+    _prefill_case(B, oracle, w, causal=False)
+    _prefill_case(B, oracle, w, causal=True, scale=0.05)
+    wf = I.Workload("noncausal_f32", "prefill", "f32", 1, 70, 64, 4, 2, 1, 1, 32, 64, seed=6)
+    _prefill_case(B, oracle, wf, causal=False)
+
+
+def test_prefill_is_deterministic_and_leaves_inputs_untouched(B):
+    w = I.Workload("det", "prefill", "bf16", 2, 300, 256, 8, 4, 4, 1, 128, 512, seed=9)
+    t = I.prefill_inputs(w, device="cuda")
+    before = {k: v.clone() for k, v in t.items()}
+    a = B.gta_prefill(t["q"], t["k"], t["c"], t["x"], t["w_p"], t["w_g"])
+    b = B.gta_prefill(t["q"], t["k"], t["c"], t["x"], t["w_p"], t["w_g"])
+    torch.cuda.synchronize()
+    assert torch.equal(a, b)
+    for k in t:
+        assert torch.equal(t[k], before[k])
+
+
+def _sample_rows(N, n=48, seed=0):
+    rng = np.random.default_rng(seed)
+    fixed = {0, 1, 127, 128, 129, N // 2 - 1, N // 2, N - 129, N - 128, N - 2, N - 1}
+    rows = sorted(r for r in fixed if 0 <= r < N)
+    extra = rng.choice(N, size=max(0, n - len(rows)), replace=False).tolist()
+    return sorted(set(rows) | set(extra))
+
+
+def test_prefill_config2_full_size_sampled_rows(B, oracle):
+    w = I.CONFIGS["c2_prefill_bf16"]
+    _prefill_case(B, oracle, w, rows=_sample_rows(w.seq, 64, seed=2))
+
+
+def test_prefill_config4_full_size_sampled_rows(B, oracle):
+    w = I.CONFIGS["c4_long_prefill_bf16"]
+    _prefill_case(B, oracle, w, rows=_sample_rows(w.seq, 40, seed=4))
+
+
+# --------------------------------------------------------------------------- decode
+def _decode_case(B, oracle, w, seq_lens=None, s_cap=None, sample=None):
+    t = I.decode_inputs(w, device="cuda", s_cap=s_cap, seq_lens=seq_lens)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    out = B.gta_decode(t["q"], t["k_cache"], t["c_cache"], t["seq_lens"], t["x_t"], t["w_p"], t["w_g"],
+                       status_word=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    idx = list(range(w.batch)) if sample is None else sample
+    sel = torch.as_tensor(idx, device="cuda", dtype=torch.long)
+    lens = t["seq_lens"][sel].cpu().numpy()
+    cap = int(lens.max()) if len(idx) else 0
+    ws = I.scaled(w, batch=len(idx))
+    want = oracle.decode(oracle_shape(ws, seq=0), t["q"][sel].cpu(), t["k_cache"][sel][:, :, :cap].contiguous().cpu(),
+                         t["c_cache"][sel][:, :, :cap].contiguous().cpu(), lens, cap, t["x_t"][sel].cpu(),
+                         t["w_p"].cpu(), t["w_g"].cpu())
+    return assert_close(out[sel], want, w.torch_dtype(), w.name)
+
+
+SMALL_DECODE = [
+    # name, dtype, B, H, n_h, n_q, n_k, n_c, d_h, d_l, lens
+    ("bf16_ragged", "bf16", 5, 256, 8, 4, 4, 1, 128, 512, [1, 63, 64, 65, 700]),
+    ("bf16_empty_and_full", "bf16", 4, 128, 4, 2, 2, 1, 128, 256, [0, 512, 1, 300]),
+    ("bf16_shared_keys_two_latents", "bf16", 3, 128, 8, 4, 2, 2, 64, 128, [200, 5, 129]),
+    ("bf16_paper_1b_shape", "bf16", 2, 1280, 20, 5, 1, 1, 64, 128, [333, 1000]),
+    ("bf16_eight_maps", "bf16", 9, 512, 16, 8, 8, 1, 128, 1024, [257, 256, 255, 1, 2, 1000, 64, 128, 511]),
+    ("f32_general", "f32", 3, 96, 6, 6, 3, 1, 32, 64, [100, 7, 260]),
+]
+
+
+@pytest.mark.parametrize("case", SMALL_DECODE, ids=[c[0] for c in SMALL_DECODE])
+def test_decode_small_shapes(B, oracle, case):
+    name, dt, nb, H, n_h, n_q, n_k, n_c, d_h, d_l, lens = case
+    w = I.Workload(name, "decode", dt, nb, 0, H, n_h, n_q, n_k, n_c, d_h, d_l, seed=99)
+    _decode_case(B, oracle, w, seq_lens=lens, s_cap=max(lens) + 13)
+
+
+def test_decode_config3_full_size(B, oracle):
+    _decode_case(B, oracle, I.CONFIGS["c3_decode_bf16"])
+
+
+def test_decode_config5_full_size_sampled_sequences(B, oracle):
+    w = I.CONFIGS["c5_ragged_decode_bf16"]
+    lens = I.decode_seq_lens(w).numpy()
+    order = np.argsort(lens)
+    sample = sorted({int(order[0]), int(order[-1]), int(order[len(order) // 2]), 0, 1, 63, 127, int(order[1])})
+    _decode_case(B, oracle, w, sample=sample)
+
+
+def test_decode_equals_last_prefill_row_on_the_gpu(B):
+    """Append the prefill's keys / latents to empty caches, decode the last token: both library
+    paths must agree within the bf16 tolerance (and with the oracle through the other tests)."""
+    w = I.Workload("p_vs_d", "prefill", "bf16", 3, 333, 256, 8, 4, 4, 1, 128, 512, seed=31)
+    t = I.prefill_inputs(w, device="cuda")
+    full = B.gta_prefill(t["q"], t["k"], t["c"], t["x"], t["w_p"], t["w_g"])
+    cap = 400
+    k_cache = torch.randn(w.batch, w.n_k, cap, w.d_h, device="cuda").to(torch.bfloat16)
+    c_cache = torch.randn(w.batch, w.n_c, cap, w.d_l, device="cuda").to(torch.bfloat16)
+    lens = torch.zeros(w.batch, dtype=torch.int32, device="cuda")
+    B.gta_cache_append(k_cache, c_cache, t["k"][:, :, :-1].contiguous(), t["c"][:, :, :-1].contiguous(), lens)
+    B.gta_cache_append(k_cache, c_cache, t["k"][:, :, -1:].contiguous(), t["c"][:, :, -1:].contiguous(), lens)
+    assert lens.tolist() == [w.seq] * w.batch
+    dec = B.gta_decode(t["q"][:, :, -1].contiguous(), k_cache, c_cache, lens, t["x"][:, -1].contiguous(),
+                       t["w_p"], t["w_g"])
+    torch.cuda.synchronize()
+    assert_close(dec, full[:, -1].double().cpu().numpy(), torch.bfloat16, "decode vs prefill")
+
+
+# --------------------------------------------------------------------------- cache append
+@pytest.mark.parametrize("dt", ["bf16", "f32"])
+@pytest.mark.parametrize("n_new", [1, 3, 700])
+def test_cache_append_is_bit_exact(B, oracle, dt, n_new):
+    tdt = torch.bfloat16 if dt == "bf16" else torch.float32
+    nb, n_k, n_c, d_h, d_l, cap = 6, 4, 2, 64, 128, 1024
+    g = torch.Generator("cpu").manual_seed(123 + n_new)
+    k_cache = torch.randn(nb, n_k, cap, d_h, generator=g).to(tdt)
+    c_cache = torch.randn(nb, n_c, cap, d_l, generator=g).to(tdt)
+    k_new = torch.randn(nb, n_k, n_new, d_h, generator=g).to(tdt)
+    c_new = torch.randn(nb, n_c, n_new, d_l, generator=g).to(tdt)
+    lens = torch.tensor([0, 1, cap - n_new, cap - n_new + 1, cap, 17], dtype=torch.int32)  # two overflow
+    shape = oracle.Shape(nb, 0, 8, 4, 4, n_k, n_c, d_h, d_l)
+    wk, wc, wl, wov = oracle.cache_append(shape, k_cache, c_cache, cap, k_new, c_new, n_new, lens.numpy())
+    assert wov == 1
+
+    dk, dc, dl = k_cache.cuda(), c_cache.cuda(), lens.cuda()
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    B.gta_cache_append(dk, dc, k_new.cuda(), c_new.cuda(), dl, status_word=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == B.GTA_ERR_CACHE_FULL
+    assert dl.cpu().numpy().tolist() == wl.tolist()
+
+    def bits(t):
+        t = t.cpu().contiguous()
+        return t.view(torch.int16).numpy().view(np.uint16) if t.dtype == torch.bfloat16 else t.numpy().view(np.uint32)
+
+    want_k = wk if dt == "bf16" else wk.view(np.uint32)
+    want_c = wc if dt == "bf16" else wc.view(np.uint32)
+    assert np.array_equal(bits(dk), want_k.reshape(bits(dk).shape))
+    assert np.array_equal(bits(dc), want_c.reshape(bits(dc).shape))
+
+
+def test_append_then_decode_sequence_of_steps(B, oracle):
+    """Three decode steps with appends in between track the oracle's cache model exactly."""
+    w = I.Workload("steps", "decode", "bf16", 4, 0, 128, 4, 2, 2, 1, 128, 256, seed=55)
+    lens0 = [10, 64, 0, 127]
+    t = I.decode_inputs(w, device="cuda", s_cap=160, seq_lens=lens0)
+    kc, cc, lens = t["k_cache"].clone(), t["c_cache"].clone(), t["seq_lens"].clone()
+    hk, hc, hl = kc.cpu(), cc.cpu(), lens.cpu().numpy()
+    g = torch.Generator("cpu").manual_seed(8)
+    shape = oracle_shape(w, seq=0)
+    for _ in range(3):
+        k_new = torch.randn(w.batch, w.n_k, 1, w.d_h, generator=g).to(torch.bfloat16)
+        c_new = torch.randn(w.batch, w.n_c, 1, w.d_l, generator=g).to(torch.bfloat16)
+        q = torch.randn(w.batch, w.n_q, w.d_h, generator=g).to(torch.bfloat16)
+        x_t = torch.randn(w.batch, w.d_model, generator=g).to(torch.bfloat16)
+        B.gta_cache_append(kc, cc, k_new.cuda(), c_new.cuda(), lens)
+        out = B.gta_decode(q.cuda(), kc, cc, lens, x_t.cuda(), t["w_p"], t["w_g"])
+        nk, nc, hl, _ = oracle.cache_append(shape, hk, hc, 160, k_new, c_new, 1, hl)
+        hk = torch.from_numpy(nk.view(np.int16)).view(torch.bfloat16).reshape(hk.shape)
+        hc = torch.from_numpy(nc.view(np.int16)).view(torch.bfloat16).reshape(hc.shape)
+        want = oracle.decode(shape, q, hk, hc, hl, 160, x_t, t["w_p"].cpu(), t["w_g"].cpu())
+        torch.cuda.synchronize()
+        assert lens.cpu().numpy().tolist() == hl.tolist()
+        assert torch.equal(kc.cpu(), hk) and torch.equal(cc.cpu(), hc)
+        assert_close(out, want, torch.bfloat16, "step")
