@@ -48,6 +48,9 @@ cudaError_t launch_generic_prefill(const Dims& d, int dtype, const void* q, cons
                                    const void* x, const void* w_p, const void* w_g, void* out,
                                    float* o_lat_ws, cudaStream_t stream, int stages, int* launches);
 
+cudaError_t launch_generic_attention_bf16(const Dims& d, const void* q, const void* k, const void* c,
+                                          void* o_lat_bf16, cudaStream_t stream, int* launches);
+
 cudaError_t launch_decode(const Dims& d, int dtype, const void* q, const void* k_cache, const void* c_cache,
                           const int32_t* seq_lens, int S_cap, const void* x_t, const void* w_p,
                           const void* w_g, void* out, void* workspace, int32_t* status_word,

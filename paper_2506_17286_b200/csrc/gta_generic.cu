@@ -12,10 +12,10 @@ namespace gta {
 constexpr int kAttnWarps = 16;   // query rows per CTA, one warp each
 constexpr int kMaxAccPerLane = 32;  // d_l <= 32 * 32
 
-template <typename T>
+template <typename T, typename TO>
 __global__ void __launch_bounds__(kAttnWarps * 32)
 generic_attention_kernel(Dims d, const T* __restrict__ q, const T* __restrict__ k,
-                         const T* __restrict__ c, float* __restrict__ o_lat) {
+                         const T* __restrict__ c, TO* __restrict__ o_lat) {
     extern __shared__ float q_smem[];  // [kAttnWarps][d_h]
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int t = blockIdx.x * kAttnWarps + warp;
@@ -64,11 +64,11 @@ generic_attention_kernel(Dims d, const T* __restrict__ q, const T* __restrict__ 
         }
     }
     const float inv_l = 1.f / l;
-    float* o_row = o_lat + (((size_t)b * d.n_q + g) * d.N + t) * d.d_l;
+    TO* o_row = o_lat + (((size_t)b * d.n_q + g) * d.N + t) * d.d_l;
 #pragma unroll
     for (int a = 0; a < kMaxAccPerLane; ++a) {
         const int col = lane + 32 * a;
-        if (a < n_acc && col < d.d_l) o_row[col] = acc[a] * inv_l;
+        if (a < n_acc && col < d.d_l) o_row[col] = from_f32<TO>(acc[a] * inv_l);
     }
 }
 
@@ -161,7 +161,7 @@ static cudaError_t launch_typed(const Dims& d, const void* q, const void* k, con
     if (stages & 1) {
         dim3 grid_a((d.N + kAttnWarps - 1) / kAttnWarps, d.n_q, d.B);
         const size_t smem = (size_t)kAttnWarps * d.d_h * sizeof(float);
-        generic_attention_kernel<T><<<grid_a, kAttnWarps * 32, smem, stream>>>(
+        generic_attention_kernel<T, float><<<grid_a, kAttnWarps * 32, smem, stream>>>(
             d, (const T*)q, (const T*)k, (const T*)c, o_lat_ws);
         cudaError_t err = cudaGetLastError();
         if (err != cudaSuccess) return err;
@@ -183,6 +183,18 @@ cudaError_t launch_generic_prefill(const Dims& d, int dtype, const void* q, cons
     if (dtype == GTA_F32)
         return launch_typed<float>(d, q, k, c, x, w_p, w_g, out, o_lat_ws, stream, stages, launches);
     return launch_typed<__nv_bfloat16>(d, q, k, c, x, w_p, w_g, out, o_lat_ws, stream, stages, launches);
+}
+
+// Attention stage only, bf16 storage in and out (L written as bf16): feeds the tensor-core
+// decoder when the tensor-core attention kernel does not cover a shape.
+cudaError_t launch_generic_attention_bf16(const Dims& d, const void* q, const void* k, const void* c,
+                                          void* o_lat_bf16, cudaStream_t stream, int* launches) {
+    dim3 grid_a((d.N + kAttnWarps - 1) / kAttnWarps, d.n_q, d.B);
+    const size_t smem = (size_t)kAttnWarps * d.d_h * sizeof(float);
+    generic_attention_kernel<__nv_bfloat16, __nv_bfloat16><<<grid_a, kAttnWarps * 32, smem, stream>>>(
+        d, (const __nv_bfloat16*)q, (const __nv_bfloat16*)k, (const __nv_bfloat16*)c, (__nv_bfloat16*)o_lat_bf16);
+    *launches += 1;
+    return cudaGetLastError();
 }
 
 }  // namespace gta
