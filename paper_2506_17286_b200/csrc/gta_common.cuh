@@ -57,6 +57,14 @@ cudaError_t launch_decode(const Dims& d, int dtype, const void* q, const void* k
                           cudaStream_t stream, int stages, int* launches);
 size_t decode_workspace_bytes(const Dims& d, int S_cap);
 
+// bf16 bandwidth-oriented decode (persistent streaming kernel + cluster finish kernel).
+bool decode_fast_supported(const Dims& d, int dtype);
+size_t decode_fast_workspace_bytes(const Dims& d);
+cudaError_t launch_decode_fast(const Dims& d, const void* q, const void* k_cache, const void* c_cache,
+                               const int32_t* seq_lens, int S_cap, const void* x_t, const void* w_p,
+                               const void* w_g, void* out, void* workspace, int32_t* status_word,
+                               cudaStream_t stream, int stages, int* launches);
+
 cudaError_t launch_cache_append(const Dims& d, int elem_size, void* k_cache, void* c_cache, int S_cap,
                                 const void* k_new, const void* c_new, int n_new, int32_t* seq_lens,
                                 int32_t* status_word, cudaStream_t stream, int* launches);

@@ -48,7 +48,12 @@ static DecodePlan make_plan(const Dims& d, int S_cap) {
     return p;
 }
 
-size_t decode_workspace_bytes(const Dims& d, int S_cap) { return make_plan(d, S_cap).total; }
+size_t decode_workspace_bytes(const Dims& d, int S_cap) {
+    // sized for whichever kernel family runs (the choice depends on shape and dtype only)
+    const size_t generic = make_plan(d, S_cap).total;
+    const size_t fast = decode_fast_workspace_bytes(d);
+    return generic > fast ? generic : fast;
+}
 
 // ---- 16-byte vector of storage elements, widened to fp32 ----
 template <typename T> struct Vec16;
@@ -392,7 +397,9 @@ cudaError_t launch_decode(const Dims& d, int dtype, const void* q, const void* k
                           const int32_t* seq_lens, int S_cap, const void* x_t, const void* w_p,
                           const void* w_g, void* out, void* workspace, int32_t* status_word,
                           cudaStream_t stream, int stages, int* launches) {
-    (void)status_word;
+    if (decode_fast_supported(d, dtype) && S_cap > 0)
+        return launch_decode_fast(d, q, k_cache, c_cache, seq_lens, S_cap, x_t, w_p, w_g, out, workspace,
+                                  status_word, stream, stages, launches);
     if (dtype == GTA_F32)
         return launch_decode_typed<float>(d, q, k_cache, c_cache, seq_lens, S_cap, x_t, w_p, w_g, out,
                                           workspace, stream, stages, launches);

@@ -24,8 +24,12 @@ def B():
 def _prefill_case(B, oracle, w, causal=True, rows=None, scale=0.0, project=True):
     t = I.prefill_inputs(w, device="cuda", project=project)
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    shape = B.make_shape(batch=w.batch, seq=w.seq, d_model=w.d_model, n_heads=w.n_heads, n_q=w.n_q, n_k=w.n_k,
+                         n_c=w.n_c, d_h=w.d_h, d_l=w.d_l, dtype=w.torch_dtype())
+    # a workspace full of NaN bit patterns: nothing may be read before the library wrote it
+    ws = torch.full((B.prefill_workspace_bytes(shape),), 0xFF, dtype=torch.uint8, device="cuda")
     out = B.gta_prefill(t["q"], t["k"], t["c"], t["x"], t["w_p"], t["w_g"], causal=causal,
-                        softmax_scale=scale, status_word=status)
+                        softmax_scale=scale, status_word=status, workspace=ws)
     torch.cuda.synchronize()
     assert int(status.item()) == 0
     tc = cpu(t)
@@ -107,8 +111,10 @@ def test_prefill_config4_full_size_sampled_rows(B, oracle):
 def _decode_case(B, oracle, w, seq_lens=None, s_cap=None, sample=None):
     t = I.decode_inputs(w, device="cuda", s_cap=s_cap, seq_lens=seq_lens)
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    shape = B.decode_shape(t["q"], t["k_cache"], t["c_cache"], t["x_t"], t["w_p"])
+    ws = torch.full((B.decode_workspace_bytes(shape, t["s_cap"]),), 0xFF, dtype=torch.uint8, device="cuda")
     out = B.gta_decode(t["q"], t["k_cache"], t["c_cache"], t["seq_lens"], t["x_t"], t["w_p"], t["w_g"],
-                       status_word=status)
+                       status_word=status, workspace=ws)
     torch.cuda.synchronize()
     assert int(status.item()) == 0
     idx = list(range(w.batch)) if sample is None else sample
