@@ -133,7 +133,7 @@ gta_status_t gta_prefill_stages(const gta_shape_t* shape, const void* q, const v
 size_t gta_decode_workspace_bytes(const gta_shape_t* shape, int32_t S_cap) {
     gta::Dims d;
     if (check_shape(shape, false, &d) != GTA_OK || S_cap < 0) return 0;
-    return gta::decode_workspace_bytes(d, S_cap);
+    return gta::decode_workspace_bytes(d, shape->dtype, S_cap);
 }
 
 gta_status_t gta_decode(const gta_shape_t* shape, const void* q, const void* k_cache, const void* c_cache,
@@ -164,7 +164,7 @@ gta_status_t gta_decode_stages(const gta_shape_t* shape, const void* q, const vo
     // one latent row is spread over at most 256 threads, 16 bytes each
     if ((size_t)d.d_l * elem_size(shape->dtype) > 4096) return GTA_ERR_UNSUPPORTED;
     if (d.B == 0) return GTA_OK;
-    if (!workspace || !aligned(workspace, 256) || workspace_bytes < gta::decode_workspace_bytes(d, S_cap))
+    if (!workspace || !aligned(workspace, 256) || workspace_bytes < gta::decode_workspace_bytes(d, shape->dtype, S_cap))
         return GTA_ERR_WORKSPACE;
     if ((st = check_device()) != GTA_OK) return st;
     int launches = 0;

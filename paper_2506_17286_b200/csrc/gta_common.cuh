@@ -55,7 +55,7 @@ cudaError_t launch_decode(const Dims& d, int dtype, const void* q, const void* k
                           const int32_t* seq_lens, int S_cap, const void* x_t, const void* w_p,
                           const void* w_g, void* out, void* workspace, int32_t* status_word,
                           cudaStream_t stream, int stages, int* launches);
-size_t decode_workspace_bytes(const Dims& d, int S_cap);
+size_t decode_workspace_bytes(const Dims& d, int dtype, int S_cap);
 
 // bf16 bandwidth-oriented decode (persistent streaming kernel + cluster finish kernel).
 bool decode_fast_supported(const Dims& d, int dtype);

@@ -48,11 +48,10 @@ static DecodePlan make_plan(const Dims& d, int S_cap) {
     return p;
 }
 
-size_t decode_workspace_bytes(const Dims& d, int S_cap) {
-    // sized for whichever kernel family runs (the choice depends on shape and dtype only)
-    const size_t generic = make_plan(d, S_cap).total;
-    const size_t fast = decode_fast_workspace_bytes(d);
-    return generic > fast ? generic : fast;
+size_t decode_workspace_bytes(const Dims& d, int dtype, int S_cap) {
+    // the kernel family is a function of shape and dtype only, so the size is that family's
+    if (decode_fast_supported(d, dtype) && S_cap > 0) return decode_fast_workspace_bytes(d);
+    return make_plan(d, S_cap).total;
 }
 
 // ---- 16-byte vector of storage elements, widened to fp32 ----
