@@ -34,6 +34,10 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
+# dram__bytes_read.sum + dram__bytes_write.sum per launch on workload c2, from the ncu captures
+# summarised under profiles/ (None once a kernel has changed since its counters were taken).
+NCU_DRAM_BYTES_PER_LAUNCH = {"prefill_attention": 25.43e6, "prefill_decoder_gate": None}
+
 METRIC = "gta_prefill_tflops"
 UNIT = "TFLOP/s"
 
@@ -83,7 +87,7 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", "-i", gpu_id, f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
-                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+                 "-lms", "50"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._pump, daemon=True)
             self.thread.start()
         except OSError:
@@ -317,7 +321,7 @@ def run_ours(args):
     peak_tf = peaks["bf16_tflops_sustained"]
     roofline = {
         "kernel": dom["kernel"], "bound": "tensor", "achieved": dom["flops"] / (dom["ms"] * 1e-3) / 1e12,
-        "peak": peak_tf, "unit": "TFLOP/s", "traffic": None,
+        "peak": peak_tf, "unit": "TFLOP/s", "traffic": NCU_DRAM_BYTES_PER_LAUNCH.get(dom["kernel"]),
         "peak_source": f"bf16_tflops_sustained of {peaks['source']} (kernel timed inside a long step)",
         "kernels": [dict(kernel=k["kernel"], ms=k["ms"], tflops=k["flops"] / (k["ms"] * 1e-3) / 1e12,
                          frac=k["flops"] / (k["ms"] * 1e-3) / 1e12 / peak_tf) for k in kernels],
@@ -396,7 +400,7 @@ def run_ours(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--steps", type=int, default=2000)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")

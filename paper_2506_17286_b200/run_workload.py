@@ -1,0 +1,125 @@
+"""Run one named synthetic workload through the C-ABI library and print per-kernel device times.
+
+    python -m paper_2506_17286_b200.run_workload c3_decode_bf16 [--iters 20] [--warmup 3]
+           [--batch B] [--seq N] [--stages MASK]
+
+A small, self-contained driver for timing or profiling one call at a time (the benchmark
+times the whole step).  Times are CUDA-event times on the launching stream; between
+iterations the inputs alternate between two independent sets, so a decode step never finds
+its caches in L2.  `--batch` / `--seq` shrink the workload (e.g. for a profiler capture);
+`--stages` restricts the call to some of its kernels (see gta_prefill_stages /
+gta_decode_stages in include/gta.h).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import statistics
+
+import torch
+
+from . import binding as G
+from . import inputs as I
+
+
+def _median(xs):
+    return statistics.median(xs) if xs else 0.0
+
+
+def run_prefill(w, iters, warmup, stages):
+    dev = torch.device("cuda")
+    t = I.prefill_inputs(w, device=dev)
+    shape = G.make_shape(batch=w.batch, seq=w.seq, d_model=w.d_model, n_heads=w.n_heads, n_q=w.n_q, n_k=w.n_k,
+                         n_c=w.n_c, d_h=w.d_h, d_l=w.d_l, dtype=w.torch_dtype())
+    ws = torch.zeros(G.prefill_workspace_bytes(shape), dtype=torch.uint8, device=dev)
+    out = torch.empty((w.batch, w.seq, w.n_heads, w.d_h), dtype=w.torch_dtype(), device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    stream = torch.cuda.current_stream()
+    masks = [m for m in (1, 2) if stages & m]
+    times = {m: [] for m in masks}
+    for it in range(warmup + iters):
+        evs = [torch.cuda.Event(enable_timing=True) for _ in range(len(masks) + 1)]
+        evs[0].record(stream)
+        for n, m in enumerate(masks):
+            G.gta_prefill(t["q"], t["k"], t["c"], t["x"], t["w_p"], t["w_g"], out=out, workspace=ws,
+                          status_word=status, stages=m)
+            evs[n + 1].record(stream)
+        torch.cuda.synchronize()
+        if it >= warmup:
+            for n, m in enumerate(masks):
+                times[m].append(evs[n].elapsed_time(evs[n + 1]))
+    assert int(status.item()) == 0, "device status word raised"
+    names = {1: "attention", 2: "decoder_gate"}
+    return {names[m]: _median(v) for m, v in times.items()}
+
+
+def run_decode(w, iters, warmup, stages, append):
+    dev = torch.device("cuda")
+    sets = []
+    for s in range(2):
+        td = I.decode_inputs(I.scaled(w, seed=w.seed + s), device=dev)
+        td["lens0"] = td["seq_lens"].clone()
+        sets.append(td)
+    shape = G.decode_shape(sets[0]["q"], sets[0]["k_cache"], sets[0]["c_cache"], sets[0]["x_t"], sets[0]["w_p"])
+    ws = torch.zeros(G.decode_workspace_bytes(shape, sets[0]["s_cap"]), dtype=torch.uint8, device=dev)
+    out = torch.empty((w.batch, w.n_heads, w.d_h), dtype=w.torch_dtype(), device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    stream = torch.cuda.current_stream()
+    masks = [m for m in (1, 2, 4) if stages & m]
+    times = {m: [] for m in masks}
+    t_append = []
+    for it in range(warmup + iters):
+        td = sets[it % 2]
+        evs = [torch.cuda.Event(enable_timing=True) for _ in range(len(masks) + 2)]
+        if append:
+            td["seq_lens"].copy_(td["lens0"] - 1)
+            evs[-1].record(stream)
+            G.gta_cache_append(td["k_cache"], td["c_cache"], td["k_new"], td["c_new"], td["seq_lens"],
+                               status_word=status)
+        evs[0].record(stream)
+        for n, m in enumerate(masks):
+            G.gta_decode(td["q"], td["k_cache"], td["c_cache"], td["seq_lens"], td["x_t"], td["w_p"], td["w_g"],
+                         out=out, workspace=ws, status_word=status, stages=m)
+            evs[n + 1].record(stream)
+        torch.cuda.synchronize()
+        if it >= warmup:
+            for n, m in enumerate(masks):
+                times[m].append(evs[n].elapsed_time(evs[n + 1]))
+            if append:
+                t_append.append(evs[-1].elapsed_time(evs[0]))
+    assert int(status.item()) == 0, "device status word raised"
+    names = {1: "gate", 2: "cache_stream", 4: "merge_decoder"}
+    res = {names[m]: _median(v) for m, v in times.items()}
+    if append:
+        res["append"] = _median(t_append)
+    lens = sets[0]["lens0"].cpu().tolist()
+    res["cache_bytes"] = float(sum(lens)) * (w.n_k * w.d_h + w.n_c * w.d_l) * 2
+    return res
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("workload", choices=sorted(I.CONFIGS))
+    ap.add_argument("--iters", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--batch", type=int, default=0)
+    ap.add_argument("--seq", type=int, default=0)
+    ap.add_argument("--stages", type=int, default=7)
+    ap.add_argument("--append", action="store_true", help="decode: run gta_cache_append before every step")
+    args = ap.parse_args()
+    w = I.CONFIGS[args.workload]
+    if args.batch:
+        w = I.scaled(w, batch=args.batch)
+    if args.seq:
+        w = I.scaled(w, seq=args.seq) if w.kind == "prefill" or w.seq > 0 else I.scaled(w, ctx_max=args.seq)
+    G.lib()
+    torch.cuda.set_device(0)
+    if w.kind == "prefill":
+        res = run_prefill(w, args.iters, args.warmup, args.stages & 3)
+    else:
+        res = run_decode(w, args.iters, args.warmup, args.stages, args.append)
+    print(json.dumps({"workload": w.name, "batch": w.batch, "seq": w.seq, "median_ms": res}))
+
+
+if __name__ == "__main__":
+    main()
