@@ -50,7 +50,8 @@ typedef enum {
     GTA_ERR_WORKSPACE = 3,   /* workspace missing or smaller than *_workspace_bytes() */
     GTA_ERR_CUDA = 4,        /* a CUDA runtime / driver call failed (launch, attribute, tensor map) */
     GTA_ERR_CACHE_FULL = 5,  /* device-side: an append would exceed S_cap for some sequence */
-    GTA_ERR_TIMEOUT = 6      /* device-side: a bounded wait inside a kernel ran out */
+    GTA_ERR_TIMEOUT = 6,     /* device-side: a bounded wait inside a kernel ran out */
+    GTA_ERR_STATIC_SCRATCH = 7 /* gta_decode_static: the problem needs more than GTA_STATIC_SCRATCH_BYTES */
 } gta_status_t;
 
 typedef enum { GTA_F32 = 0, GTA_BF16 = 1 } gta_dtype_t;
@@ -136,6 +137,34 @@ GTA_API gta_status_t gta_cache_append(const gta_shape_t *shape, void *k_cache, v
                               int32_t S_cap, const void *k_new, const void *c_new,
                               int32_t n_new, int32_t *seq_lens, int32_t *status_word,
                               void *cuda_stream);
+
+/*
+ * gta_decode_static — gta_decode without a workspace argument (the paper has no counterpart: this
+ * is a packaging variant of the same decode step, with the same arguments, results and errors).
+ *
+ * It is meant for hosts that cannot allocate device memory at the moment a decode step is due,
+ * for example a serving process whose memory pool took the whole device at start-up, a plug-in
+ * that may not use its host application's allocator, or a loop that cannot afford the device-
+ * wide synchronisation an allocation implies.  The split-KV partial results go to a fixed array
+ * of GTA_STATIC_SCRATCH_BYTES bytes that is part of the library image: every GPU on which the
+ * library is used keeps that much memory until the process exits.  The call itself allocates
+ * and frees nothing, on the host runtime or the device.
+ *
+ *   - A problem whose gta_decode_workspace_bytes() exceeds GTA_STATIC_SCRATCH_BYTES is refused
+ *     with GTA_ERR_STATIC_SCRATCH before anything is launched (for the bf16 kernels the need
+ *     grows with batch * n_q * d_l, not with the context length).
+ *   - The first call on each device looks up the array's device address (once, with that
+ *     device current); make that first call outside any stream capture.
+ *   - All calls on a device share the one array and find in it whatever the previous call left;
+ *     the kernels write every word before they read it, so nothing needs clearing.  Two calls
+ *     that may run on the GPU at the same time (different streams, no ordering) race on it:
+ *     order them, or use gta_decode with separate workspaces.
+ */
+#define GTA_STATIC_SCRATCH_BYTES (16u << 20)
+GTA_API gta_status_t gta_decode_static(const gta_shape_t *shape, const void *q, const void *k_cache,
+                                       const void *c_cache, const int32_t *seq_lens, int32_t S_cap,
+                                       const void *x_t, const void *w_p, const void *w_g, void *out,
+                                       int32_t *status_word, void *cuda_stream);
 
 /*
  * Profiling aids (no counterpart in the paper): the same calls restricted to a subset of their

@@ -15,13 +15,14 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libgta_b200.so")
 
 GTA_OK, GTA_ERR_INVALID_ARG, GTA_ERR_UNSUPPORTED, GTA_ERR_WORKSPACE = 0, 1, 2, 3
-GTA_ERR_CUDA, GTA_ERR_CACHE_FULL, GTA_ERR_TIMEOUT = 4, 5, 6
+GTA_ERR_CUDA, GTA_ERR_CACHE_FULL, GTA_ERR_TIMEOUT, GTA_ERR_STATIC_SCRATCH = 4, 5, 6, 7
+STATIC_SCRATCH_BYTES = 16 << 20
 GTA_F32, GTA_BF16 = 0, 1
 
 EXPORTS = (
     "gta_prefill_workspace_bytes", "gta_prefill", "gta_decode_workspace_bytes", "gta_decode",
     "gta_cache_append", "gta_status_string", "gta_version", "gta_prefill_path", "gta_last_launch_count",
-    "gta_prefill_stages", "gta_decode_stages",
+    "gta_prefill_stages", "gta_decode_stages", "gta_decode_static",
 )
 
 
@@ -67,6 +68,8 @@ def lib():
         L.gta_decode_workspace_bytes.restype = sz
         L.gta_decode.argtypes = [sp, vp, vp, vp, vp, i32, vp, vp, vp, vp, vp, sz, vp, vp]
         L.gta_decode.restype = i32
+        L.gta_decode_static.argtypes = [sp, vp, vp, vp, vp, i32, vp, vp, vp, vp, vp, vp]
+        L.gta_decode_static.restype = i32
         L.gta_cache_append.argtypes = [sp, vp, vp, i32, vp, vp, i32, vp, vp, vp]
         L.gta_cache_append.restype = i32
         L.gta_status_string.argtypes = [i32]
@@ -200,6 +203,34 @@ def gta_decode(q, k_cache, c_cache, seq_lens, x_t, w_p, w_g, *, softmax_scale=0.
     st = lib().gta_decode(*args) if stages == 7 else lib().gta_decode_stages(*args, stages)
     if st != GTA_OK:
         raise GtaError(st, "gta_decode")
+    return out
+
+
+def gta_decode_static(q, k_cache, c_cache, seq_lens, x_t, w_p, w_g, *, softmax_scale=0.0, out=None,
+                      status_word=None, stream=None):
+    """gta_decode for callers that cannot allocate device memory (a pool that owns the whole
+    device, a plug-in barred from the allocator, a loop that cannot take an allocation's device
+    synchronisation): the split-KV scratch is a fixed STATIC_SCRATCH_BYTES array inside the
+    library instead of a workspace tensor.  Pass `out`, and nothing is allocated at all.
+    Raises GtaError(GTA_ERR_STATIC_SCRATCH) when the problem needs more than the array holds.
+    Calls on one device share the array: order them on one stream."""
+    _check_tensors(q, k_cache, c_cache, x_t, w_p, w_g)
+    if seq_lens.dtype != torch.int32 or seq_lens.device != q.device or not seq_lens.is_contiguous():
+        raise ValueError("seq_lens must be a contiguous int32 tensor on the operator's device")
+    B, n_q, d_h = q.shape
+    s_cap = k_cache.shape[2]
+    shape = decode_shape(q, k_cache, c_cache, x_t, w_p, softmax_scale=softmax_scale)
+    n_h, d_l, H = shape.n_heads, shape.latent_dim, shape.d_model
+    if k_cache.shape != (B, shape.n_k_groups, s_cap, d_h) or c_cache.shape != (B, shape.n_c_groups, s_cap, d_l) \
+            or x_t.shape != (B, H) or w_p.shape != (n_h, d_l, d_h) or w_g.shape != (H, n_h * d_h) \
+            or seq_lens.shape != (B,):
+        raise ValueError("inconsistent operator tensor shapes")
+    if out is None:
+        out = torch.empty((B, n_h, d_h), dtype=q.dtype, device=q.device)
+    st = lib().gta_decode_static(ctypes.byref(shape), _ptr(q), _ptr(k_cache), _ptr(c_cache), _ptr(seq_lens), s_cap,
+                                 _ptr(x_t), _ptr(w_p), _ptr(w_g), _ptr(out), _ptr(status_word), _stream(stream))
+    if st != GTA_OK:
+        raise GtaError(st, "gta_decode_static")
     return out
 
 

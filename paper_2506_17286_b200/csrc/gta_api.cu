@@ -63,6 +63,7 @@ const char* gta_status_string(gta_status_t status) {
         case GTA_ERR_CUDA: return "CUDA call failed";
         case GTA_ERR_CACHE_FULL: return "cache full";
         case GTA_ERR_TIMEOUT: return "bounded device wait ran out";
+        case GTA_ERR_STATIC_SCRATCH: return "problem exceeds the built-in scratch array of gta_decode_static";
     }
     return "unknown status";
 }
