@@ -1,23 +1,30 @@
 // Bandwidth-oriented decode for bf16 caches (App. B.1.3), d_h = 128, one latent group.
 //
-//   decode_stream_kernel : persistent, two CTAs per SM.  The live tokens of all sequences are
-//       cut into sub-tiles of TS tokens; CTA c owns the contiguous sub-tile range
-//       [c n / G, (c+1) n / G), so every CTA streams the same number of cache bytes whatever
-//       the length mix.  A producer warp copies each sub-tile (the K rows of every key group and
-//       the latent rows) into a 3-stage shared-memory ring with bulk async copies; 256 consumer
-//       threads compute the scores of all maps, a running softmax (the maximum is only raised
-//       when it grows by more than 2^8) and the latent sums, each latent row being read once and
-//       applied to all maps with packed fp32x2 FMAs.  When the range crosses into the next
-//       sequence, and at its end, the partial (max, sum, latent sum) goes to slot c + b.
-//   decode_finish_kernel : clusters of 8 CTAs per head split the reduction dimensions of the
-//       decoder (d_l) and of the gate (H); every CTA merges the slots of its d_l slice
-//       (log-sum-exp), multiplies by its slices of W_P,i and W_G,i for 32 sequences at a time,
-//       and the cluster adds the eight partial results through distributed shared memory before
-//       the sigmoid gate is applied.
+//   decode_stream_kernel : persistent, one CTA per SM.  The live tokens of all sequences are cut
+//       into sub-tiles of T tokens; CTA c owns the contiguous sub-tile range [c n / G, (c+1) n / G),
+//       so every CTA streams the same number of cache bytes whatever the length mix.  A producer
+//       warp brings each sub-tile (the K rows of every key group and the latent rows) into a
+//       3-stage shared-memory ring with TMA tensor loads (128-byte swizzle, evict-first in L2).
+//       Eight consumer warps compute, per sub-tile, the scores of all maps and the latent sums
+//       with warp-level m16n8k16 MMAs whose M rows are the attention maps (1 .. 8 valid rows of
+//       16): the cache data never passes through the ALUs element by element, which keeps the
+//       kernel on the HBM roofline instead of the issue-slot limit.  Scores go through a small
+//       shared buffer so that every warp can build the probability fragments for its own
+//       d_l / 8 slice of the latent sum; one CTA barrier per sub-tile.  When the range crosses
+//       into the next sequence, and at its end, the partial (max, sum, latent sum) goes to
+//       slot c + b of the workspace.
+//   decode_finish_kernel : clusters of 4 or 8 CTAs per (head, 64-column half) split the reduction
+//       dimensions of the decoder (d_l) and of the gate (H).  Launched with programmatic stream
+//       serialisation: while the stream kernel drains, each CTA requests its weight slice (TMA)
+//       and its hidden-state slice and works out which stream CTAs own which sequence; after the
+//       dependency wait it merges, for 32 sequences at a time, the slots of its d_l slice
+//       (log-sum-exp), multiplies by W_P,i and W_G,i with warp-level MMAs, and the cluster adds the
+//       partial results through distributed shared memory before the sigmoid gate is applied.
 #include <cooperative_groups.h>
 
 #include "gta_common.cuh"
 #include "sm100_ptx.cuh"
+#include "tma_host.cuh"
 
 namespace cg = cooperative_groups;
 
@@ -26,29 +33,31 @@ namespace gta {
 constexpr int kStreamConsumers = 256;
 constexpr int kStreamThreads = kStreamConsumers + 32;
 constexpr int kStreamStages = 3;
-constexpr int kStreamStageBytes = 32768;
+constexpr int kStreamStageBytes = 65536;
 constexpr int kStreamMaxBatch = 512;
-constexpr int kStreamMaxTS = 32;
-constexpr int kFinSplit = 8;
+constexpr int kStreamMaxT = 64;
 constexpr int kFinBlockB = 32;
 constexpr int kFinThreads = 256;
+constexpr int kFinCols = 64;
+constexpr int kFinMaxSlots = 1024;  // >= stream CTAs + batch
 
 struct FastPlan {
-    int TS;        // tokens per sub-tile
+    int T;         // tokens per sub-tile (16, 32 or 64)
     int G;         // stream CTAs
     int slots;     // G + B partial slots
-    size_t off_ml, off_prefix, total;
+    size_t off_ml, total;   // byte offsets in the workspace (part_o at 0)
 };
 
 static size_t align256f(size_t v) { return (v + 255) & ~(size_t)255; }
+static int finish_split(const Dims& d);
 
 bool decode_fast_supported(const Dims& d, int dtype) {
     if (dtype != GTA_BF16 || d.d_h != 128 || d.n_c != 1) return false;
     if (d.d_l != 256 && d.d_l != 512 && d.d_l != 1024) return false;
     if (d.n_q != 1 && d.n_q != 2 && d.n_q != 4 && d.n_q != 8) return false;
-    if (d.B > kStreamMaxBatch || d.H % 64 != 0) return false;
+    if (d.B > kStreamMaxBatch || finish_split(d) == 0) return false;
     const int tok_bytes = (d.n_k * d.d_h + d.d_l) * 2;
-    return tok_bytes * 4 <= kStreamStageBytes;
+    return tok_bytes * 16 <= kStreamStageBytes;
 }
 
 static int sm_count() {
@@ -65,101 +74,79 @@ static int sm_count() {
 static FastPlan make_fast_plan(const Dims& d) {
     FastPlan p;
     const int tok_bytes = (d.n_k * d.d_h + d.d_l) * 2;
-    int ts = 1;
-    while (ts * 2 * tok_bytes <= kStreamStageBytes && ts * 2 <= kStreamMaxTS) ts *= 2;
-    p.TS = ts;
-    p.G = 2 * sm_count();
+    int t = 16;
+    while (t * 2 * tok_bytes <= kStreamStageBytes && t * 2 <= kStreamMaxT) t *= 2;
+    p.T = t;
+    p.G = sm_count() < kFinMaxSlots - kStreamMaxBatch ? sm_count() : kFinMaxSlots - kStreamMaxBatch;
     p.slots = p.G + d.B;
     const size_t part_o = (size_t)p.slots * d.n_q * d.d_l * sizeof(float);
     const size_t part_ml = (size_t)p.slots * d.n_q * 2 * sizeof(float);
     p.off_ml = align256f(part_o);
-    p.off_prefix = p.off_ml + align256f(part_ml);
-    p.total = p.off_prefix + align256f((size_t)(d.B + 1) * sizeof(int32_t));
+    p.total = p.off_ml + align256f(part_ml);
     return p;
 }
 
 size_t decode_fast_workspace_bytes(const Dims& d) { return make_fast_plan(d).total; }
 
 // ---------------------------------------------------------------------------------------------
-// Bulk async copy global -> shared, completion counted on `bar`; the cache bytes are read once, so
-// they are marked evict-first in L2 (the weights of the finish kernel stay resident).
-__device__ __forceinline__ uint64_t l2_evict_first_policy() {
-    uint64_t pol;
-    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
-    return pol;
-}
-__device__ __forceinline__ void bulk_copy_g2s(void* dst, const void* src, uint32_t bytes, uint64_t* bar,
-                                              uint64_t policy) {
-    asm volatile(
-        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
-        ::"r"(ptx::smem_addr(dst)), "l"(reinterpret_cast<uint64_t>(src)), "r"(bytes), "r"(ptx::smem_addr(bar)),
-          "l"(policy)
-        : "memory");
-}
 __device__ __forceinline__ void consumer_sync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
 
-__device__ __forceinline__ uint64_t pack2(float lo, float hi) {
-    return (uint64_t)__float_as_uint(lo) | ((uint64_t)__float_as_uint(hi) << 32);
-}
-__device__ __forceinline__ void ffma2(uint64_t& acc, uint64_t a, uint64_t b) {
-    asm("fma.rn.f32x2 %0, %1, %2, %0;" : "+l"(acc) : "l"(a), "l"(b));
-}
-__device__ __forceinline__ uint64_t fmul2(uint64_t a, uint64_t b) {
-    uint64_t r;
-    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
-    return r;
-}
 __device__ __forceinline__ float ex2f(float x) {
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&v);
+}
 __device__ __forceinline__ int clamp_len(int len, int S_cap) { return len < 0 ? 0 : (len > S_cap ? S_cap : len); }
 
-// Which stream CTA owns sub-tile `st` when n sub-tiles are dealt to G CTAs in contiguous ranges
-// [c n / G, (c + 1) n / G).
-__device__ __forceinline__ int owner_of(long long st, long long n, int G) {
-    int c = (int)((st * G) / n);
-    while (c + 1 < G && ((long long)(c + 1) * n) / G <= st) ++c;
-    while (c > 0 && ((long long)c * n) / G > st) --c;
-    return c;
-}
-
-// With fewer sub-tiles than CTAs some CTAs own nothing and never write their slot.
-__device__ __forceinline__ bool owns_any(int c, long long n, int G) {
-    return ((long long)c * n) / G < ((long long)(c + 1) * n) / G;
-}
-
-template <int NQ>
-__global__ void __launch_bounds__(kStreamThreads, 2)
-decode_stream_kernel(Dims d, int TS, int S_cap, const __nv_bfloat16* __restrict__ q,
-                     const __nv_bfloat16* __restrict__ k_cache, const __nv_bfloat16* __restrict__ c_cache,
-                     const int32_t* __restrict__ seq_lens, float* __restrict__ part_o, float* __restrict__ part_ml,
-                     int32_t* __restrict__ prefix_g, int32_t* status_word) {
-    extern __shared__ __align__(128) uint8_t smem[];
-    uint8_t* ring = smem;                                                    // 3 x 32 KB
-    float* q_s = reinterpret_cast<float*>(smem + kStreamStages * kStreamStageBytes);   // [NQ][128]
-    float2* p2_s = reinterpret_cast<float2*>(q_s + NQ * 128);                // [2][TS][NQ] pairs (p, p)
-    float* a_s = reinterpret_cast<float*>(p2_s + 2 * kStreamMaxTS * NQ);     // [2][NQ] rescale factors
-    float* red = a_s + 2 * NQ;                                               // [R][d_l / 2]; scan scratch at start
-    int32_t* prefix = reinterpret_cast<int32_t*>(red + 1024);                // [B + 1]
-    int32_t* scan_tmp = reinterpret_cast<int32_t*>(red);                     // [kStreamThreads] (start-up only)
-    uint64_t* full_bar = reinterpret_cast<uint64_t*>(prefix + kStreamMaxBatch + 2);
-    full_bar = reinterpret_cast<uint64_t*>((reinterpret_cast<uintptr_t>(full_bar) + 7) & ~(uintptr_t)7);
+// Shared-memory layout of one ring stage (all tiles are [T rows][64 bf16] = T x 128 bytes with
+// the 128-byte TMA swizzle: the 16-byte chunk c of row r sits at chunk c ^ (r & 7)):
+//   K tiles : key group kg, half h (columns 64 h .. 64 h + 63)  at (2 kg + h) T 128
+//   C tiles : latent columns 64 j .. 64 j + 63                   at c_off + j T 128
+template <int NT>   // NT = d_l / 64 = MMA n-tiles (8 latent columns each) per consumer warp
+__global__ void __launch_bounds__(kStreamThreads, 1)
+decode_stream_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_c, Dims d,
+                     int T, int S_cap, const __nv_bfloat16* __restrict__ q, const int32_t* __restrict__ seq_lens,
+                     float* __restrict__ part_o, float* __restrict__ part_ml, int32_t* status_word) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    uint8_t* ring = smem;                                                              // 3 x 64 KB
+    float* s_buf = reinterpret_cast<float*>(smem + kStreamStages * kStreamStageBytes);   // [2][n_q][T]
+    int32_t* prefix = reinterpret_cast<int32_t*>(s_buf + 2 * 8 * kStreamMaxT);           // [B + 1]
+    int32_t* scan_tmp = prefix + kStreamMaxBatch + 2;                                    // [kStreamThreads]
+    uint64_t* full_bar = reinterpret_cast<uint64_t*>(scan_tmp + kStreamThreads);
     uint64_t* empty_bar = full_bar + kStreamStages;
     volatile int* abort_flag = reinterpret_cast<volatile int*>(empty_bar + kStreamStages);
     volatile int* drain_flag = abort_flag + 1;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int G = gridDim.x, cta = blockIdx.x;
+    const int NQ = d.n_q;
+    // the finish kernel may be scheduled as soon as SMs free up: it prefetches its weights and
+    // then waits for this whole grid before it touches the partial results
+    ptx::grid_launch_dependents();
+    if (tid == kStreamConsumers) {   // the descriptors are on their way while the prefix sum runs
+        ptx::prefetch_tensormap(&tm_k);
+        ptx::prefetch_tensormap(&tm_c);
+    }
 
-    // ---- exclusive prefix sum of the sub-tile counts: prefix[b] = sum_{b' < b} ceil(len / TS)
+    // ---- exclusive prefix sum of the sub-tile counts: prefix[b] = sum_{b' < b} ceil(len / T)
+    //      (thread t owns sequences [t per, (t + 1) per); warp scan, then a scan of the warp totals)
     {
         const int per = (d.B + kStreamThreads - 1) / kStreamThreads;
         const int lo = min(tid * per, d.B), hi = min(lo + per, d.B);
         int sum = 0;
-        for (int b = lo; b < hi; ++b) sum += (clamp_len(seq_lens[b], S_cap) + TS - 1) / TS;
-        scan_tmp[tid] = sum;
+        for (int b = lo; b < hi; ++b) sum += (clamp_len(seq_lens[b], S_cap) + T - 1) / T;
+        int incl = sum;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int v = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += v;
+        }
+        if (lane == 31) scan_tmp[warp] = incl;
         if (tid == 0) {
             for (int s = 0; s < kStreamStages; ++s) { ptx::mbar_init(&full_bar[s], 1); ptx::mbar_init(&empty_bar[s], 8); }
             *abort_flag = 0;
@@ -167,23 +154,20 @@ decode_stream_kernel(Dims d, int TS, int S_cap, const __nv_bfloat16* __restrict_
             ptx::fence_mbar_init();
         }
         __syncthreads();
-        int base = 0;
-        for (int t = 0; t < tid; ++t) base += scan_tmp[t];
+        int base = incl - sum;
+        for (int w = 0; w < warp; ++w) base += scan_tmp[w];
         for (int b = lo; b < hi; ++b) {
             prefix[b] = base;
-            base += (clamp_len(seq_lens[b], S_cap) + TS - 1) / TS;
+            base += (clamp_len(seq_lens[b], S_cap) + T - 1) / T;
         }
-        if (hi == d.B && lo < d.B) prefix[d.B] = base;
-        if (d.B == 0 && tid == 0) prefix[0] = 0;
+        if (tid == kStreamThreads - 1) prefix[d.B] = base;
         __syncthreads();
-        if (cta == 0)
-            for (int b = tid; b <= d.B; b += kStreamThreads) prefix_g[b] = prefix[b];
     }
     const long long n_st = prefix[d.B];
     const long long st_begin = ((long long)cta * n_st) / G, st_end = ((long long)(cta + 1) * n_st) / G;
-    if (st_begin >= st_end) return;      // uniform: nothing armed, nothing allocated
+    if (st_begin >= st_end) return;      // uniform: nothing armed
     int b0;
-    {   // largest b with prefix[b] <= st_begin and a non-empty sequence
+    {   // largest b with prefix[b] <= st_begin: a non-empty sequence, since st_begin < n_st
         int lo = 0, hi = d.B - 1;
         while (lo < hi) {
             const int mid = (lo + hi + 1) >> 1;
@@ -191,34 +175,43 @@ decode_stream_kernel(Dims d, int TS, int S_cap, const __nv_bfloat16* __restrict_
         }
         b0 = lo;
     }
-    const int tok_bytes_k = d.n_k * 256;
-    const int row_bytes_c = d.d_l * 2;
-    const uint32_t c_off = (uint32_t)d.n_k * TS * 256;   // latent rows start here inside a stage
+    const uint32_t tile_bytes = (uint32_t)T * 128;
+    const uint32_t c_off = (uint32_t)d.n_k * 2 * tile_bytes;
+    const uint32_t stage_tx = c_off + (uint32_t)NT * tile_bytes;
 
     if (warp == kStreamConsumers / 32) {
         // ------------------------------------------------------------------ producer
-        if (lane == 0) {
-            const uint64_t policy = l2_evict_first_policy();
+        // Lane 0 waits for the stage and arms its barrier; then every lane issues one of the (up
+        // to 32) tensor loads of the sub-tile, so that issuing them does not pace the stream.
+        {
+            const uint64_t policy = ptx::l2_evict_first_policy();
+            const int n_k_ops = 2 * d.n_k;
             int b = b0;
             long long k = st_begin - prefix[b0];
             int it = 0;
+            bool ok = true;
             for (long long st = st_begin; st < st_end; ++st, ++it, ++k) {
                 while (k >= prefix[b + 1] - prefix[b]) { ++b; k = 0; }
                 const int s = it % kStreamStages;
                 const uint32_t ph = (it / kStreamStages) & 1;
-                if (!ptx::mbar_wait(&empty_bar[s], ph ^ 1, abort_flag)) break;
-                const int len = clamp_len(seq_lens[b], S_cap);
-                const int tok0 = (int)k * TS;
-                const int n_valid = min(TS, len - tok0);
+                if (lane == 0) {
+                    ok = ptx::mbar_wait(&empty_bar[s], ph ^ 1, abort_flag);
+                    if (ok) ptx::mbar_arrive_expect_tx(&full_bar[s], stage_tx);
+                }
+                ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
+                if (!ok) break;
+                const int tok0 = (int)k * T;
                 uint8_t* stage = ring + s * kStreamStageBytes;
-                ptx::mbar_arrive_expect_tx(&full_bar[s], (uint32_t)n_valid * (tok_bytes_k + row_bytes_c));
-                for (int kg = 0; kg < d.n_k; ++kg)
-                    bulk_copy_g2s(stage + kg * TS * 256,
-                                  k_cache + (((size_t)b * d.n_k + kg) * S_cap + tok0) * 128, n_valid * 256, &full_bar[s], policy);
-                bulk_copy_g2s(stage + c_off, c_cache + ((size_t)b * S_cap + tok0) * d.d_l, n_valid * row_bytes_c,
-                              &full_bar[s], policy);
+                for (int op = lane; op < n_k_ops + NT; op += 32) {
+                    if (op < n_k_ops)
+                        ptx::tma_load_3d_hint(stage + op * tile_bytes, &tm_k, &full_bar[s], (op & 1) * 64, tok0,
+                                              b * d.n_k + (op >> 1), policy);
+                    else
+                        ptx::tma_load_3d_hint(stage + c_off + (op - n_k_ops) * tile_bytes, &tm_c, &full_bar[s],
+                                              (op - n_k_ops) * 64, tok0, b, policy);
+                }
             }
-            if (*abort_flag) {
+            if (lane == 0 && *abort_flag) {
                 for (int back = 1; back <= kStreamStages && it - back >= 0; ++back) {
                     const int iq = it - back;
                     ptx::mbar_wait(&full_bar[iq % kStreamStages], (iq / kStreamStages) & 1, drain_flag);
@@ -227,58 +220,45 @@ decode_stream_kernel(Dims d, int TS, int S_cap, const __nv_bfloat16* __restrict_
         }
     } else {
         // ------------------------------------------------------------------ consumers
-        const int tpr = d.d_l / 8;                 // threads per latent row (32, 64 or 128)
-        const int R = kStreamConsumers / tpr;      // latent rows in flight
-        const int r = tid / tpr, v = tid % tpr;
-        const int qpk = NQ / d.n_k;
-        const int n_it = (TS + 7) / 8;             // score iterations: 8 key rows per warp and iteration
+        const int quad = lane >> 2, sub = lane & 3;       // MMA fragment coordinates
+        const int mat = lane >> 3, mrow = lane & 7;       // ldmatrix: which 8x8 matrix, which row of it
+        const int qpk = NQ / d.n_k;                       // maps per key group
+        const int kg_w = warp % d.n_k;                    // this warp scores key group kg_w (n_k divides 8)
+        const int KT = T >> 4;                            // 16-token MMA k-steps per sub-tile
+        const int n_units = (T >> 3) * d.n_k;             // (8-token n-tile, key group) scoring units
         const float c_scale = d.scale * 1.4426950408889634f;
-        const int quad = lane >> 2, ql = lane & 3;
-        float m_run = -INFINITY, l_run = 0.f;      // softmax state of map `warp` (warps < NQ)
-        uint64_t acc[NQ][4];
+        const uint32_t ring_addr = ptx::smem_addr(ring);
+        const bool map_lane = quad < NQ;                  // this lane carries softmax state of map `quad`
+        float m_run = -INFINITY, l_run = 0.f;
+        float acc[NT][4];
 #pragma unroll
-        for (int g = 0; g < NQ; ++g)
-#pragma unroll
-            for (int e = 0; e < 4; ++e) acc[g][e] = 0ull;
+        for (int n = 0; n < NT; ++n) acc[n][0] = acc[n][1] = acc[n][2] = acc[n][3] = 0.f;
+        uint32_t qa[8][2];                                // A fragments of Q for key group kg_w
 
         auto load_q = [&](int b) {
-            for (int e = tid; e < NQ * 128; e += kStreamConsumers)
-                q_s[e] = __bfloat162float(q[(size_t)b * NQ * 128 + e]);
-            m_run = -INFINITY;
-            l_run = 0.f;
-            consumer_sync();
+            const uint32_t* qrow =
+                reinterpret_cast<const uint32_t*>(q + ((size_t)b * NQ + kg_w * qpk + (quad < qpk ? quad : 0)) * 128);
+#pragma unroll
+            for (int ks = 0; ks < 8; ++ks) {
+                qa[ks][0] = quad < qpk ? __ldg(qrow + 8 * ks + sub) : 0u;
+                qa[ks][1] = quad < qpk ? __ldg(qrow + 8 * ks + 4 + sub) : 0u;
+            }
         };
         auto flush = [&](int b) {
             const int slot = cta + b;
-            const int half_cols = d.d_l / 2;
+            if (map_lane) {
+                float* o = part_o + ((size_t)slot * NQ + quad) * d.d_l + warp * (NT * 8) + 2 * sub;
 #pragma unroll
-            for (int g = 0; g < NQ; ++g) {
-                for (int h = 0; h < 2; ++h) {
-                    consumer_sync();
-                    if ((v * 8) / half_cols == h) {
-                        float* dst = red + r * half_cols + (v * 8 - h * half_cols);
-#pragma unroll
-                        for (int e = 0; e < 4; ++e) {
-                            dst[2 * e] = __uint_as_float((uint32_t)acc[g][e]);
-                            dst[2 * e + 1] = __uint_as_float((uint32_t)(acc[g][e] >> 32));
-                        }
-                    }
-                    consumer_sync();
-                    float* out_row = part_o + ((size_t)slot * NQ + g) * d.d_l + h * half_cols;
-                    for (int col = tid; col < half_cols; col += kStreamConsumers) {
-                        float s = 0.f;
-                        for (int rr = 0; rr < R; ++rr) s += red[rr * half_cols + col];
-                        out_row[col] = s;
-                    }
+                for (int n = 0; n < NT; ++n) *reinterpret_cast<float2*>(o + 8 * n) = make_float2(acc[n][0], acc[n][1]);
+                if (warp == 0 && sub == 0) {
+                    part_ml[((size_t)slot * NQ + quad) * 2] = m_run;
+                    part_ml[((size_t)slot * NQ + quad) * 2 + 1] = l_run;
                 }
+            }
 #pragma unroll
-                for (int e = 0; e < 4; ++e) acc[g][e] = 0ull;
-            }
-            if (warp < NQ && lane == 0) {
-                part_ml[((size_t)slot * NQ + warp) * 2] = m_run;
-                part_ml[((size_t)slot * NQ + warp) * 2 + 1] = l_run;
-            }
-            consumer_sync();
+            for (int n = 0; n < NT; ++n) acc[n][0] = acc[n][1] = acc[n][2] = acc[n][3] = 0.f;
+            m_run = -INFINITY;
+            l_run = 0.f;
         };
 
         int b = b0;
@@ -298,95 +278,103 @@ decode_stream_kernel(Dims d, int TS, int S_cap, const __nv_bfloat16* __restrict_
             ok = __all_sync(0xffffffffu, ptx::mbar_wait(&full_bar[s], ph, abort_flag));
             if (!ok) break;
             const int len = clamp_len(seq_lens[b], S_cap);
-            const int n_valid = min(TS, len - (int)k * TS);
-            const uint8_t* stage = ring + s * kStreamStageBytes;
-            float2* p2 = p2_s + (it & 1) * kStreamMaxTS * NQ;     // [TS][NQ] pairs (p, p)
-            float* alpha_s = a_s + (it & 1) * NQ;
+            const int n_valid = min(T, len - (int)k * T);
+            const uint32_t stage = ring_addr + s * kStreamStageBytes;
+            float* sb = s_buf + (it & 1) * (NQ * T);
 
-            // ---- scores + running softmax of map `warp`: a quad of lanes per key row
-            if (warp < NQ) {
-                const int g = warp, kg = g / qpk;
-                const float* qv = q_s + g * 128;
-                float sc[4];
-                float m_loc = -INFINITY;
+            // ---- scores of the maps of key group kg_w, 8 tokens per unit: S = Q K^T
+            for (int u = warp; u < n_units; u += 8) {
+                const int nt = u / d.n_k;
+                const int token = nt * 8 + mrow;
+                const uint32_t krow = stage + (uint32_t)(2 * kg_w) * tile_bytes + token * 128;
+                float sc[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-                for (int i8 = 0; i8 < 4; ++i8) {
-                    sc[i8] = -INFINITY;
-                    if (i8 < n_it) {
-                        const int tok = i8 * 8 + quad;
-                        const uint8_t* row = stage + (size_t)(kg * TS + min(tok, TS - 1)) * 256;
-                        float dot = 0.f;
-#pragma unroll
-                        for (int u = 0; u < 4; ++u) {
-                            const int vec = ql + 4 * u;
-                            const uint4 kv = *reinterpret_cast<const uint4*>(row + vec * 16);
-                            const float4 qa = *reinterpret_cast<const float4*>(qv + vec * 8);
-                            const float4 qb = *reinterpret_cast<const float4*>(qv + vec * 8 + 4);
-                            dot = fmaf(qa.x, __uint_as_float(kv.x << 16), dot);
-                            dot = fmaf(qa.y, __uint_as_float(kv.x & 0xffff0000u), dot);
-                            dot = fmaf(qa.z, __uint_as_float(kv.y << 16), dot);
-                            dot = fmaf(qa.w, __uint_as_float(kv.y & 0xffff0000u), dot);
-                            dot = fmaf(qb.x, __uint_as_float(kv.z << 16), dot);
-                            dot = fmaf(qb.y, __uint_as_float(kv.z & 0xffff0000u), dot);
-                            dot = fmaf(qb.z, __uint_as_float(kv.w << 16), dot);
-                            dot = fmaf(qb.w, __uint_as_float(kv.w & 0xffff0000u), dot);
-                        }
-                        dot += __shfl_xor_sync(0xffffffffu, dot, 1);
-                        dot += __shfl_xor_sync(0xffffffffu, dot, 2);
-                        if (tok < n_valid) sc[i8] = dot * c_scale;
-                        m_loc = fmaxf(m_loc, sc[i8]);
-                    }
+                for (int kp = 0; kp < 4; ++kp) {
+                    const int chunk = 4 * kp + mat;     // 16-byte chunk of the 256-byte K row
+                    uint32_t k0, k1, k2, k3;
+                    ptx::ldsm_x4(krow + (chunk >> 3) * tile_bytes + (((chunk & 7) ^ (token & 7)) << 4), k0, k1, k2, k3);
+                    ptx::mma_bf16_16816(sc, qa[2 * kp][0], 0u, qa[2 * kp][1], 0u, k0, k1);
+                    ptx::mma_bf16_16816(sc, qa[2 * kp + 1][0], 0u, qa[2 * kp + 1][1], 0u, k2, k3);
                 }
-                m_loc = fmaxf(m_loc, __shfl_xor_sync(0xffffffffu, m_loc, 4));
-                m_loc = fmaxf(m_loc, __shfl_xor_sync(0xffffffffu, m_loc, 8));
-                m_loc = fmaxf(m_loc, __shfl_xor_sync(0xffffffffu, m_loc, 16));
-                float alpha = 1.f;
-                if (m_loc > m_run + 8.f) { alpha = ex2f(m_run - m_loc); m_run = m_loc; }
-                float sum = 0.f;
-#pragma unroll
-                for (int i8 = 0; i8 < 4; ++i8) {
-                    if (i8 < n_it) {
-                        const int tok = i8 * 8 + quad;
-                        const float p = ex2f(sc[i8] - m_run);
-                        sum += p;
-                        if (ql == 0 && tok < TS) p2[tok * NQ + g] = make_float2(p, p);
-                    }
+                if (quad < qpk) {
+                    const int t0 = nt * 8 + 2 * sub;
+                    float2 v;
+                    v.x = t0 < n_valid ? sc[0] * c_scale : -INFINITY;
+                    v.y = t0 + 1 < n_valid ? sc[1] * c_scale : -INFINITY;
+                    *reinterpret_cast<float2*>(sb + (kg_w * qpk + quad) * T + t0) = v;
                 }
-                sum += __shfl_xor_sync(0xffffffffu, sum, 4);
-                sum += __shfl_xor_sync(0xffffffffu, sum, 8);
-                sum += __shfl_xor_sync(0xffffffffu, sum, 16);
-                l_run = l_run * alpha + sum;     // every lane of a quad holds the same p: sum counts each token once
-                if (lane == 0) alpha_s[g] = alpha;
+            }
+            // ---- rows past the live length hold whatever the cache holds there: their
+            //      probabilities are zero, so the latent rows are cleared (0 x garbage could be NaN)
+            if (n_valid < T) {
+                const int vec_per_row = NT * 8;          // 16-byte vectors per latent row
+                const int n_vec = (T - n_valid) * vec_per_row;
+                for (int idx = tid; idx < n_vec; idx += kStreamConsumers) {
+                    const int row = n_valid + idx / vec_per_row, v = idx % vec_per_row;
+                    uint8_t* p = ring + s * kStreamStageBytes + c_off + (v >> 3) * tile_bytes + row * 128 + (v & 7) * 16;
+                    *reinterpret_cast<uint4*>(p) = make_uint4(0u, 0u, 0u, 0u);
+                }
+                ptx::fence_proxy_async_smem();   // the next TMA write of this stage follows generic writes
             }
             consumer_sync();
-            // ---- latent sums: each row read once, applied to all maps
+
+            // ---- softmax state of map `quad` (every warp keeps its own copy) and the probability
+            //      fragments: lane (quad, sub) holds tokens 16 kt + 2 sub + {0, 1, 8, 9}
+            uint32_t pa[4][2];
+            float alpha = 1.f;
             {
-                bool rescale = false;
+                float sv[4][4];
+                float m_t = -INFINITY;
 #pragma unroll
-                for (int g = 0; g < NQ; ++g) rescale |= (alpha_s[g] != 1.f);
-                if (rescale) {
-#pragma unroll
-                    for (int g = 0; g < NQ; ++g) {
-                        const uint64_t a2 = pack2(alpha_s[g], alpha_s[g]);
-#pragma unroll
-                        for (int e = 0; e < 4; ++e) acc[g][e] = fmul2(acc[g][e], a2);
+                for (int kt = 0; kt < 4; ++kt) {
+                    if (kt < KT && map_lane) {
+                        const float2 x = *reinterpret_cast<const float2*>(sb + quad * T + 16 * kt + 2 * sub);
+                        const float2 y = *reinterpret_cast<const float2*>(sb + quad * T + 16 * kt + 8 + 2 * sub);
+                        sv[kt][0] = x.x; sv[kt][1] = x.y; sv[kt][2] = y.x; sv[kt][3] = y.y;
+                    } else {
+                        sv[kt][0] = sv[kt][1] = sv[kt][2] = sv[kt][3] = -INFINITY;
                     }
+                    m_t = fmaxf(fmaxf(m_t, fmaxf(sv[kt][0], sv[kt][1])), fmaxf(sv[kt][2], sv[kt][3]));
                 }
-                const uint8_t* c_rows = stage + c_off + v * 16;
-#pragma unroll 2
-                for (int j = r; j < n_valid; j += R) {
-                    const uint4 cv = *reinterpret_cast<const uint4*>(c_rows + (size_t)j * row_bytes_c);
-                    const uint32_t w[4] = {cv.x, cv.y, cv.z, cv.w};
-                    uint64_t c2[4];
+                m_t = fmaxf(m_t, __shfl_xor_sync(0xffffffffu, m_t, 1));
+                m_t = fmaxf(m_t, __shfl_xor_sync(0xffffffffu, m_t, 2));
+                const float m_new = fmaxf(m_run, m_t);     // finite on map lanes: token 0 of a tile is live
+                const float m_sub = map_lane ? m_new : 0.f;
+                alpha = map_lane ? ex2f(m_run - m_new) : 1.f;
+                float sum = 0.f;
 #pragma unroll
-                    for (int e = 0; e < 4; ++e)
-                        c2[e] = (uint64_t)(w[e] << 16) | ((uint64_t)(w[e] & 0xffff0000u) << 32);
-                    const uint64_t* pj = reinterpret_cast<const uint64_t*>(p2 + j * NQ);
+                for (int kt = 0; kt < 4; ++kt) {
+                    const float p0 = ex2f(sv[kt][0] - m_sub), p1 = ex2f(sv[kt][1] - m_sub);
+                    const float p2 = ex2f(sv[kt][2] - m_sub), p3 = ex2f(sv[kt][3] - m_sub);
+                    sum += (p0 + p1) + (p2 + p3);
+                    pa[kt][0] = pack_bf16(p0, p1);
+                    pa[kt][1] = pack_bf16(p2, p3);
+                }
+                sum += __shfl_xor_sync(0xffffffffu, sum, 1);
+                sum += __shfl_xor_sync(0xffffffffu, sum, 2);
+                l_run = l_run * alpha + sum;
+                m_run = m_new;
+            }
 #pragma unroll
-                    for (int g = 0; g < NQ; ++g) {
-                        const uint64_t pp = pj[g];
+            for (int n = 0; n < NT; ++n) { acc[n][0] *= alpha; acc[n][1] *= alpha; }
+
+            // ---- latent sums of this warp's d_l / 8 columns, all maps at once: O += P C
+            {
+                const uint32_t cbase = stage + c_off;
 #pragma unroll
-                        for (int e = 0; e < 4; ++e) ffma2(acc[g][e], pp, c2[e]);
+                for (int kt = 0; kt < 4; ++kt) {
+                    if (kt < KT) {
+                        const int token = 16 * kt + (mat & 1) * 8 + mrow;
+                        const uint32_t crow = cbase + token * 128;
+#pragma unroll
+                        for (int np = 0; np < NT / 2; ++np) {
+                            const int chunk = warp * NT + 2 * np + (mat >> 1);   // 16-byte chunk of the latent row
+                            uint32_t c0, c1, c2, c3;
+                            ptx::ldsm_x4_trans(crow + (chunk >> 3) * tile_bytes + (((chunk & 7) ^ (token & 7)) << 4),
+                                               c0, c1, c2, c3);
+                            ptx::mma_bf16_16816(acc[2 * np], pa[kt][0], 0u, pa[kt][1], 0u, c0, c1);
+                            ptx::mma_bf16_16816(acc[2 * np + 1], pa[kt][0], 0u, pa[kt][1], 0u, c2, c3);
+                        }
                     }
                 }
             }
@@ -400,152 +388,345 @@ decode_stream_kernel(Dims d, int TS, int S_cap, const __nv_bfloat16* __restrict_
 }
 
 // ---------------------------------------------------------------------------------------------
-// Dynamic shared memory (floats): o_s [d_l/8][32] | x_s [H/8][32] | part_s [2][32][128] |
-//                                  mrg [32][4] (max, 1/sum, first slot, last slot)
-__global__ void __cluster_dims__(kFinSplit, 1, 1) __launch_bounds__(kFinThreads)
-decode_finish_cluster_kernel(Dims d, int G, int TS, int S_cap, const int32_t* __restrict__ seq_lens,
-                             const int32_t* __restrict__ prefix_g, const float* __restrict__ part_o,
-                             const float* __restrict__ part_ml, const __nv_bfloat16* __restrict__ x_t,
-                             const __nv_bfloat16* __restrict__ w_p, const __nv_bfloat16* __restrict__ w_g,
-                             __nv_bfloat16* __restrict__ out) {
+// One CTA = one head, 64 of its 128 output columns, 1 / S of the reduction dimensions (S = cluster
+// size, 4 or 8).  Dynamic shared memory:
+//   w_s [(d_l + H) / S rows][64 bf16] (swizzled weight slice: W_P rows first) |
+//   a_s [32][KA + 8 bf16] (merged latent slice, then hidden-state slice, per sequence) |
+//   part_s [2][32][64] fp32 (partial decoder / gate sums) | ml_s, w_all [slots] | prefix_s, rng_s [B] |
+//   bound_s [G + 1] | scan scratch | barrier
+struct FinSmem {
+    uint32_t a_off, part_off, ml_off, w_all_off, prefix_off, rng_off, bound_off, scan_off, bar_off, total;
+};
+__host__ __device__ inline FinSmem fin_smem_layout(int KA) {
+    FinSmem L;
+    L.a_off = (uint32_t)KA * 128u;
+    L.part_off = L.a_off + (uint32_t)kFinBlockB * (KA + 8) * 2;
+    L.ml_off = L.part_off + 2u * kFinBlockB * kFinCols * 4;
+    L.w_all_off = L.ml_off + kFinMaxSlots * 8;
+    L.prefix_off = L.w_all_off + kFinMaxSlots * 4;
+    L.rng_off = L.prefix_off + (kStreamMaxBatch + 2) * 4;
+    L.bound_off = L.rng_off + 2 * kStreamMaxBatch * 4;
+    L.scan_off = L.bound_off + (kFinMaxSlots - kStreamMaxBatch + 2) * 4;
+    L.bar_off = L.scan_off + 8 * 4;
+    L.total = L.bar_off + 16 + 1024;   // + slack to align the base to 1024 bytes
+    return L;
+}
+
+__device__ __forceinline__ void cp_async_16(void* dst, const void* src) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(ptx::smem_addr(dst)), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
+
+// Merge of the split-KV partial latent sums of one block of 32 sequences into a_s (bf16).  A
+// thread owns one 4-column chunk of its CTA's d_l slice for SQ sequences (SQ x dls / 4 = 256
+// threads x ... : dls = 64, 128, 256 -> SQ = 2, 4, 8).  Loads go out in rounds of up to kFinRound
+// slots per sequence, all of a round in flight at once.
+struct FinMergeArgs {
+    const float* part_o; const float* w_all;
+    const int32_t* rng_s;    // [B][2] first / last stream CTA that owns sub-tiles of the sequence
+    __nv_bfloat16* a_s;
+    int n_q, d_l, g, col_base, dls, a_stride, b0, nb, tid;
+};
+constexpr int kFinMaxSQ = 8;
+struct FinMergeRegs { float4 v[32]; };
+
+template <int SQ>
+__device__ __forceinline__ void fin_merge_load(const FinMergeArgs& a, FinMergeRegs& r, int j0) {
+    constexpr int kRound = 32 / SQ;              // slots per sequence and round
+    const int tps = a.dls / 4;                   // threads per sequence
+    const int chunk = a.tid % tps, bgrp = a.tid / tps, nbg = kFinThreads / tps;
+#pragma unroll
+    for (int sq = 0; sq < SQ; ++sq) {
+        const int bb = bgrp + sq * nbg, b = a.b0 + bb;
+        const int c_lo = bb < a.nb ? a.rng_s[2 * b] : 0, c_hi = bb < a.nb ? a.rng_s[2 * b + 1] : -1;
+#pragma unroll
+        for (int j = 0; j < kRound; ++j) {
+            const int c = c_lo + j0 + j;
+            float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (c <= c_hi)
+                v = *reinterpret_cast<const float4*>(a.part_o + ((size_t)(c + b) * a.n_q + a.g) * a.d_l + a.col_base + 4 * chunk);
+            r.v[sq * kRound + j] = v;
+        }
+    }
+}
+
+template <int SQ>
+__device__ __forceinline__ void fin_merge_finish(const FinMergeArgs& a, FinMergeRegs& r) {
+    constexpr int kRound = 32 / SQ;
+    const int tps = a.dls / 4;
+    const int chunk = a.tid % tps, bgrp = a.tid / tps, nbg = kFinThreads / tps;
+    float4 sum[SQ];
+#pragma unroll
+    for (int sq = 0; sq < SQ; ++sq) sum[sq] = make_float4(0.f, 0.f, 0.f, 0.f);
+    int n_max = 0;
+#pragma unroll
+    for (int sq = 0; sq < SQ; ++sq) {
+        const int bb = bgrp + sq * nbg, b = a.b0 + bb;
+        if (bb < a.nb) n_max = max(n_max, a.rng_s[2 * b + 1] - a.rng_s[2 * b] + 1);
+    }
+    for (int j0 = 0;; j0 += kRound) {
+#pragma unroll
+        for (int sq = 0; sq < SQ; ++sq) {
+            const int bb = bgrp + sq * nbg, b = a.b0 + bb;
+            const int c_lo = bb < a.nb ? a.rng_s[2 * b] : 0, c_hi = bb < a.nb ? a.rng_s[2 * b + 1] : -1;
+#pragma unroll
+            for (int j = 0; j < kRound; ++j) {
+                const int c = c_lo + j0 + j;
+                if (c <= c_hi) {
+                    const float w = a.w_all[c + b];   // 0 for a CTA that owns nothing: its slot holds stale bits
+                    if (w != 0.f) {
+                        const float4 v = r.v[sq * kRound + j];
+                        sum[sq].x = fmaf(v.x, w, sum[sq].x); sum[sq].y = fmaf(v.y, w, sum[sq].y);
+                        sum[sq].z = fmaf(v.z, w, sum[sq].z); sum[sq].w = fmaf(v.w, w, sum[sq].w);
+                    }
+                }
+            }
+        }
+        if (j0 + kRound >= n_max) break;
+        fin_merge_load<SQ>(a, r, j0 + kRound);   // sequences that span more CTAs than one round covers
+    }
+#pragma unroll
+    for (int sq = 0; sq < SQ; ++sq) {
+        const int bb = bgrp + sq * nbg;
+        uint2 packed;
+        packed.x = pack_bf16(sum[sq].x, sum[sq].y);
+        packed.y = pack_bf16(sum[sq].z, sum[sq].w);
+        *reinterpret_cast<uint2*>(a.a_s + bb * a.a_stride + 4 * chunk) = packed;
+    }
+}
+
+__global__ void __launch_bounds__(kFinThreads)
+decode_finish_kernel(const __grid_constant__ CUtensorMap tm_wp, const __grid_constant__ CUtensorMap tm_wg, Dims d,
+                     int G, int T, int S_cap, const int32_t* __restrict__ seq_lens,
+                     const float* __restrict__ part_o, const float* __restrict__ part_ml,
+                     const __nv_bfloat16* __restrict__ x_t, __nv_bfloat16* __restrict__ out, int32_t* status_word) {
     cg::cluster_group cluster = cg::this_cluster();
-    extern __shared__ __align__(16) float fsm[];
-    const int dl8 = d.d_l / kFinSplit, h8 = d.H / kFinSplit;
-    float* o_s = fsm;
-    float* x_s = o_s + dl8 * kFinBlockB;
-    float* part_s = x_s + h8 * kFinBlockB;
-    float* mrg = part_s + 2 * kFinBlockB * 128;
-    const int split = blockIdx.x;            // = rank inside the cluster
-    const int i = blockIdx.y;                // head
+    const int S = (int)cluster.num_blocks();     // = gridDim.x
+    extern __shared__ uint8_t fin_raw[];
+    uint8_t* fsm = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(fin_raw) + 1023) & ~(uintptr_t)1023);
+    const int dls = d.d_l / S, hs = d.H / S;     // this CTA's slice of the latent and of the hidden dimension
+    const int KA = dls + hs, a_stride = KA + 8;  // bf16 elements per a_s row (row = 16-byte multiple)
+    const FinSmem L = fin_smem_layout(KA);
+    uint8_t* w_s = fsm;
+    __nv_bfloat16* a_s = reinterpret_cast<__nv_bfloat16*>(fsm + L.a_off);
+    float* part_s = reinterpret_cast<float*>(fsm + L.part_off);
+    float2* ml_s = reinterpret_cast<float2*>(fsm + L.ml_off);             // (max, sum) of map g per slot
+    float* w_all = reinterpret_cast<float*>(fsm + L.w_all_off);           // merge weight per slot
+    int32_t* prefix_s = reinterpret_cast<int32_t*>(fsm + L.prefix_off);   // [B + 1]
+    int32_t* rng_s = reinterpret_cast<int32_t*>(fsm + L.rng_off);         // [B][2] first / last owning CTA
+    int32_t* bound_s = reinterpret_cast<int32_t*>(fsm + L.bound_off);     // [G + 1] first sub-tile of CTA c
+    int32_t* scan_s = reinterpret_cast<int32_t*>(fsm + L.scan_off);
+    uint64_t* w_bar = reinterpret_cast<uint64_t*>(fsm + L.bar_off);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(w_bar + 1);
+
+    const int split = blockIdx.x;                // = rank inside the cluster
+    const int i = blockIdx.y >> 1;               // head
+    const int col0 = (blockIdx.y & 1) * kFinCols;   // first of this CTA's output columns inside the head
     const int g = d.head_to_q(i);
-    const int tid = threadIdx.x;
-    const long long n_st = prefix_g[d.B];
-    const int n_cols = d.n_h * 128;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int quad = lane >> 2, sub = lane & 3, mat = lane >> 3, mrow = lane & 7;
+
+    // ---- weight slice: independent of the stream kernel's results, so it is requested first
+    if (tid == 0) {
+        ptx::mbar_init(w_bar, 1);
+        *abort_flag = 0;
+        ptx::fence_mbar_init();
+        ptx::mbar_arrive_expect_tx(w_bar, (uint32_t)KA * 128);
+        ptx::tma_load_3d(w_s, &tm_wp, w_bar, col0, split * dls, i);
+        for (int r0 = 0; r0 < hs; r0 += 256)
+            ptx::tma_load_2d(w_s + (size_t)(dls + r0) * 128, &tm_wg, w_bar, i * 128 + col0, split * hs + r0);
+    }
+    // ---- also independent of it: the hidden-state slice of a block of sequences (asynchronous copies)
+    auto load_x = [&](int b0, int nb) {
+        const int xv = hs / 8;                      // 16-byte vectors per sequence
+        for (int idx = tid; idx < kFinBlockB * xv; idx += kFinThreads) {
+            const int xb = idx / xv, v = idx % xv;
+            __nv_bfloat16* dst = a_s + xb * a_stride + dls + v * 8;
+            if (xb < nb) cp_async_16(dst, x_t + (size_t)(b0 + xb) * d.H + split * hs + v * 8);
+            else *reinterpret_cast<uint4*>(dst) = make_uint4(0u, 0u, 0u, 0u);
+        }
+    };
+    load_x(0, min(kFinBlockB, d.B));
+    // ---- and which stream CTAs own sub-tiles of which sequence.  Same
+    //      arithmetic as in the stream kernel: prefix sums of ceil(len / T), ranges c n / G.  This
+    //      runs while the stream kernel drains (the launch is programmatically serialised).
+    {
+        const int per = (d.B + kFinThreads - 1) / kFinThreads;
+        const int lo = min(tid * per, d.B), hi = min(lo + per, d.B);
+        int sum = 0;
+        for (int b = lo; b < hi; ++b) sum += (clamp_len(seq_lens[b], S_cap) + T - 1) / T;
+        int incl = sum;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int v = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += v;
+        }
+        if (lane == 31) scan_s[warp] = incl;
+        __syncthreads();
+        int base = incl - sum;
+        for (int w = 0; w < warp; ++w) base += scan_s[w];
+        for (int b = lo; b < hi; ++b) {
+            prefix_s[b] = base;
+            base += (clamp_len(seq_lens[b], S_cap) + T - 1) / T;
+        }
+        if (tid == kFinThreads - 1) prefix_s[d.B] = base;
+        __syncthreads();
+        const long long n_st = prefix_s[d.B];
+        for (int c = tid; c <= G; c += kFinThreads) bound_s[c] = (int32_t)(((long long)c * n_st) / G);
+        // the owner of sub-tile st is the largest c with floor(c n / G) <= st = floor(((st + 1) G - 1) / n)
+        for (int b = tid; b < d.B; b += kFinThreads) {
+            const long long s_lo = prefix_s[b], s_hi = prefix_s[b + 1];
+            int c_lo = 0, c_hi = -1;
+            if (s_hi > s_lo) {
+                c_lo = (int)(((s_lo + 1) * G - 1) / n_st);
+                c_hi = (int)((s_hi * G - 1) / n_st);
+            }
+            rng_s[2 * b] = c_lo;
+            rng_s[2 * b + 1] = c_hi;
+        }
+    }
+    __syncthreads();
+    ptx::grid_dependency_wait();   // everything below reads what the stream kernel wrote
+    const uint32_t w_addr = ptx::smem_addr(w_s), a_addr = ptx::smem_addr(a_s);
+
+    // ---- for this head's map, the (max, sum) pair of every slot (slots nobody wrote hold stale
+    //      bits that are never used)
+    const int n_slots = G + d.B;
+    for (int j = tid; j < n_slots; j += kFinThreads)
+        ml_s[j] = *reinterpret_cast<const float2*>(part_ml + ((size_t)j * d.n_q + g) * 2);
 
     for (int b0 = 0; b0 < d.B; b0 += kFinBlockB) {
         const int nb = min(kFinBlockB, d.B - b0);
-        // ---- per sequence: slot range, merged maximum and 1 / merged sum
-        if (tid < kFinBlockB) {
-            float M = -INFINITY, inv_l = 0.f;
-            int c_lo = 0, c_hi = -1;
-            if (tid < nb) {
-                const int b = b0 + tid;
-                const long long s_lo = prefix_g[b], s_hi = prefix_g[b + 1];
-                if (s_hi > s_lo) {
-                    c_lo = owner_of(s_lo, n_st, G);
-                    c_hi = owner_of(s_hi - 1, n_st, G);
-                    for (int c = c_lo; c <= c_hi; ++c)
-                        if (owns_any(c, n_st, G)) M = fmaxf(M, part_ml[((size_t)(c + b) * d.n_q + g) * 2]);
-                    float l = 0.f;
-                    for (int c = c_lo; c <= c_hi; ++c) {
-                        if (!owns_any(c, n_st, G)) continue;
-                        const float* ml = part_ml + ((size_t)(c + b) * d.n_q + g) * 2;
-                        l = fmaf(ml[1], ex2f(ml[0] - M), l);
+        if (b0 > 0) load_x(b0, nb);   // (block 0: already requested before the dependency wait)
+        // ---- merged latent slice (bf16): a thread owns one 4-column chunk of SQ sequences.  The
+        //      first round of partial-result loads is issued before the merge weights exist (block 0
+        //      computes them meanwhile), so their latency overlaps that work.
+        const FinMergeArgs ma = {part_o, w_all, rng_s, a_s, d.n_q, d.d_l, g, split * dls, dls, a_stride, b0, nb, tid};
+        FinMergeRegs mr;
+        if (dls == 64) fin_merge_load<2>(ma, mr, 0);
+        else if (dls == 128) fin_merge_load<4>(ma, mr, 0);
+        else fin_merge_load<8>(ma, mr, 0);
+        if (b0 == 0) {
+            __syncthreads();   // the (max, sum) pairs are in shared memory
+            // per sequence (eight lanes each): the normalised merge weight of each of its slots c + b:
+            //      w = 2^(m_slot - M) / sum_slots l_slot 2^(m_slot - M)
+            for (int b8 = 0; b8 < d.B; b8 += kFinThreads / 8) {
+                const int b = b8 + (tid >> 3), l8 = tid & 7;
+                const bool live = b < d.B;
+                const int c_lo = live ? rng_s[2 * b] : 0, c_hi = live ? rng_s[2 * b + 1] : -1;
+                float M = -INFINITY, l = 0.f;
+                for (int c = c_lo + l8; c <= c_hi; c += 8)
+                    if (bound_s[c] < bound_s[c + 1]) M = fmaxf(M, ml_s[c + b].x);
+                M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, 1));
+                M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, 2));
+                M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, 4));
+                for (int c = c_lo + l8; c <= c_hi; c += 8) {
+                    float w = 0.f;
+                    if (bound_s[c] < bound_s[c + 1]) {   // a CTA with an empty range wrote nothing
+                        w = ex2f(ml_s[c + b].x - M);
+                        l = fmaf(ml_s[c + b].y, w, l);
                     }
-                    inv_l = 1.f / l;
+                    w_all[c + b] = w;
                 }
-            }
-            mrg[tid * 4] = M; mrg[tid * 4 + 1] = inv_l;
-            mrg[tid * 4 + 2] = __int_as_float(c_lo); mrg[tid * 4 + 3] = __int_as_float(c_hi);
-        }
-        __syncthreads();
-        // ---- merged latent slice o_s[l][bb] and hidden-state slice x_s[h][bb]
-        {
-            const int bb = tid >> 3, l8 = tid & 7;
-            const float M = mrg[bb * 4], inv_l = mrg[bb * 4 + 1];
-            const int c_lo = __float_as_int(mrg[bb * 4 + 2]), c_hi = __float_as_int(mrg[bb * 4 + 3]);
-            const int b = b0 + bb;
-            for (int l0 = 0; l0 < dl8; l0 += 8 * 4) {
-                float sum[4] = {0.f, 0.f, 0.f, 0.f};
-                for (int c = c_lo; c <= c_hi; ++c) {
-                    if (!owns_any(c, n_st, G)) continue;
-                    const size_t pi = (size_t)(c + b) * d.n_q + g;
-                    const float w = ex2f(part_ml[pi * 2] - M);
-                    const float* po = part_o + pi * d.d_l + split * dl8 + l0 + l8;
-#pragma unroll
-                    for (int u = 0; u < 4; ++u) sum[u] = fmaf(po[u * 8], w, sum[u]);
-                }
-#pragma unroll
-                for (int u = 0; u < 4; ++u) o_s[(l0 + l8 + u * 8) * kFinBlockB + bb] = sum[u] * inv_l;
-            }
-            for (int h = l8; h < h8; h += 8)
-                x_s[h * kFinBlockB + bb] = bb < nb ? __bfloat162float(x_t[(size_t)b * d.H + split * h8 + h]) : 0.f;
-        }
-        __syncthreads();
-        // ---- partial decoder and gate sums: one output column per thread, two K halves
-        {
-            const int e = tid & 127, kh = tid >> 7;
-            float acc_y[kFinBlockB], acc_z[kFinBlockB];
-#pragma unroll
-            for (int bb = 0; bb < kFinBlockB; ++bb) { acc_y[bb] = 0.f; acc_z[bb] = 0.f; }
-            {
-                const int l_lo = kh * (dl8 / 2), l_hi = l_lo + dl8 / 2;
-                const __nv_bfloat16* wp = w_p + ((size_t)i * d.d_l + split * dl8) * 128 + e;
-#pragma unroll 4
-                for (int l = l_lo; l < l_hi; ++l) {
-                    const float w = __bfloat162float(wp[(size_t)l * 128]);
-                    const float4* ov = reinterpret_cast<const float4*>(o_s + l * kFinBlockB);
-#pragma unroll
-                    for (int b4 = 0; b4 < kFinBlockB / 4; ++b4) {
-                        const float4 o4 = ov[b4];
-                        acc_y[4 * b4] = fmaf(o4.x, w, acc_y[4 * b4]);
-                        acc_y[4 * b4 + 1] = fmaf(o4.y, w, acc_y[4 * b4 + 1]);
-                        acc_y[4 * b4 + 2] = fmaf(o4.z, w, acc_y[4 * b4 + 2]);
-                        acc_y[4 * b4 + 3] = fmaf(o4.w, w, acc_y[4 * b4 + 3]);
-                    }
-                }
-            }
-            {
-                const int h_lo = kh * (h8 / 2), h_hi = (kh == 0) ? h8 / 2 : h8;
-                const __nv_bfloat16* wg = w_g + (size_t)(split * h8) * n_cols + i * 128 + e;
-#pragma unroll 4
-                for (int h = h_lo; h < h_hi; ++h) {
-                    const float w = __bfloat162float(wg[(size_t)h * n_cols]);
-                    const float4* xv = reinterpret_cast<const float4*>(x_s + h * kFinBlockB);
-#pragma unroll
-                    for (int b4 = 0; b4 < kFinBlockB / 4; ++b4) {
-                        const float4 x4 = xv[b4];
-                        acc_z[4 * b4] = fmaf(x4.x, w, acc_z[4 * b4]);
-                        acc_z[4 * b4 + 1] = fmaf(x4.y, w, acc_z[4 * b4 + 1]);
-                        acc_z[4 * b4 + 2] = fmaf(x4.z, w, acc_z[4 * b4 + 2]);
-                        acc_z[4 * b4 + 3] = fmaf(x4.w, w, acc_z[4 * b4 + 3]);
-                    }
-                }
-            }
-            if (kh == 1) {
-#pragma unroll
-                for (int bb = 0; bb < kFinBlockB; ++bb) {
-                    part_s[bb * 128 + e] = acc_y[bb];
-                    part_s[(kFinBlockB + bb) * 128 + e] = acc_z[bb];
-                }
+                l += __shfl_xor_sync(0xffffffffu, l, 1);
+                l += __shfl_xor_sync(0xffffffffu, l, 2);
+                l += __shfl_xor_sync(0xffffffffu, l, 4);
+                const float inv_l = 1.f / l;
+                for (int c = c_lo + l8; c <= c_hi; c += 8) w_all[c + b] *= inv_l;
             }
             __syncthreads();
-            if (kh == 0) {
+        }
+        if (dls == 64) fin_merge_finish<2>(ma, mr);
+        else if (dls == 128) fin_merge_finish<4>(ma, mr);
+        else fin_merge_finish<8>(ma, mr);
+        cp_async_wait_all();
+        __syncthreads();
+        if (b0 == 0) ptx::mbar_wait(w_bar, 0, abort_flag);   // on give-up the results are wrong and the status word says so
+        // ---- partial sums: warp w owns output columns 8 w .. 8 w + 7; rows = the 32 sequences
+        {
+            // four accumulator sets per m-tile, used round-robin over the k-steps: the dependent
+            // chain of MMAs is a quarter as long (the loop is latency-bound, not throughput-bound)
+            float acc[2][4][4] = {};     // [y / z][set][fragment], m-tile 0
+            float bcc[2][4][4] = {};     // same, m-tile 1
+            const int a_row = (mat & 1) * 8 + mrow, a_col = (mat >> 1) * 8;
+            const int n_ks = KA / 16, ks_y = dls / 16;
+            for (int ks0 = 0; ks0 < n_ks; ks0 += 4) {
 #pragma unroll
-                for (int bb = 0; bb < kFinBlockB; ++bb) {
-                    part_s[bb * 128 + e] += acc_y[bb];
-                    part_s[(kFinBlockB + bb) * 128 + e] += acc_z[bb];
+                for (int u = 0; u < 4; ++u) {
+                    const int ks = ks0 + u;
+                    if (ks >= n_ks) break;
+                    const int yz = ks < ks_y ? 0 : 1;
+                    const int krow = 16 * ks + (lane & 15);
+                    uint32_t w0, w1;
+                    ptx::ldsm_x2_trans(w_addr + krow * 128 + ((warp ^ (krow & 7)) << 4), w0, w1);
+                    uint32_t a0, a1, a2, a3;
+                    ptx::ldsm_x4(a_addr + (uint32_t)(a_row * a_stride + 16 * ks + a_col) * 2, a0, a1, a2, a3);
+                    uint32_t e0, e1, e2, e3;
+                    ptx::ldsm_x4(a_addr + (uint32_t)((16 + a_row) * a_stride + 16 * ks + a_col) * 2, e0, e1, e2, e3);
+                    if (yz == 0) {
+                        ptx::mma_bf16_16816(acc[0][u], a0, a1, a2, a3, w0, w1);
+                        ptx::mma_bf16_16816(bcc[0][u], e0, e1, e2, e3, w0, w1);
+                    } else {
+                        ptx::mma_bf16_16816(acc[1][u], a0, a1, a2, a3, w0, w1);
+                        ptx::mma_bf16_16816(bcc[1][u], e0, e1, e2, e3, w0, w1);
+                    }
                 }
+            }
+            float acc_y[2][4], acc_z[2][4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                acc_y[0][e] = (acc[0][0][e] + acc[0][1][e]) + (acc[0][2][e] + acc[0][3][e]);
+                acc_y[1][e] = (bcc[0][0][e] + bcc[0][1][e]) + (bcc[0][2][e] + bcc[0][3][e]);
+                acc_z[0][e] = (acc[1][0][e] + acc[1][1][e]) + (acc[1][2][e] + acc[1][3][e]);
+                acc_z[1][e] = (bcc[1][0][e] + bcc[1][1][e]) + (bcc[1][2][e] + bcc[1][3][e]);
+            }
+#pragma unroll
+            for (int mt = 0; mt < 2; ++mt) {
+                float* py = part_s + (mt * 16 + quad) * kFinCols + warp * 8 + 2 * sub;
+                float* pz = py + kFinBlockB * kFinCols;
+                *reinterpret_cast<float2*>(py) = make_float2(acc_y[mt][0], acc_y[mt][1]);
+                *reinterpret_cast<float2*>(py + 8 * kFinCols) = make_float2(acc_y[mt][2], acc_y[mt][3]);
+                *reinterpret_cast<float2*>(pz) = make_float2(acc_z[mt][0], acc_z[mt][1]);
+                *reinterpret_cast<float2*>(pz + 8 * kFinCols) = make_float2(acc_z[mt][2], acc_z[mt][3]);
             }
         }
         cluster.sync();
-        // ---- cluster reduction: rank r finishes sequences [4 r, 4 r + 4) of this block
-        for (int idx = tid; idx < (kFinBlockB / kFinSplit) * 128; idx += kFinThreads) {
-            const int bb = split * (kFinBlockB / kFinSplit) + idx / 128, e = idx % 128;
-            float y = 0.f, z = 0.f;
+        // ---- cluster reduction: rank r finishes sequences [r 32 / S, (r + 1) 32 / S) of this block
+        const int rows_per_rank = kFinBlockB / S;
+        for (int idx = tid; idx < rows_per_rank * kFinCols; idx += kFinThreads) {
+            const int bb = split * rows_per_rank + idx / kFinCols, e = idx % kFinCols;
+            float yv[8], zv[8];
 #pragma unroll
-            for (int rk = 0; rk < kFinSplit; ++rk) {
-                const float* remote = cluster.map_shared_rank(part_s, rk);
-                y += remote[bb * 128 + e];
-                z += remote[(kFinBlockB + bb) * 128 + e];
+            for (int rk = 0; rk < 8; ++rk) {      // all remote loads in flight together
+                yv[rk] = zv[rk] = 0.f;
+                if (rk < S) {
+                    const float* remote = cluster.map_shared_rank(part_s, rk);
+                    yv[rk] = remote[bb * kFinCols + e];
+                    zv[rk] = remote[(kFinBlockB + bb) * kFinCols + e];
+                }
             }
+            const float y = ((yv[0] + yv[1]) + (yv[2] + yv[3])) + ((yv[4] + yv[5]) + (yv[6] + yv[7]));
+            const float z = ((zv[0] + zv[1]) + (zv[2] + zv[3])) + ((zv[4] + zv[5]) + (zv[6] + zv[7]));
             if (bb < nb) {
                 const float gate = __fdividef(1.f, 1.f + __expf(-z));
-                out[((size_t)(b0 + bb) * d.n_h + i) * 128 + e] = __float2bfloat16_rn(y * gate);
+                out[((size_t)(b0 + bb) * d.n_h + i) * 128 + col0 + e] = __float2bfloat16_rn(y * gate);
             }
         }
         cluster.sync();   // the partial sums may be overwritten (next block) or the CTA may exit
     }
+    if (tid == 0 && *abort_flag) raise_status(status_word, GTA_ERR_TIMEOUT);
+}
+
+// Cluster size (= split of the reduction dimensions) of the finish kernel: 4 when the larger
+// weight slice still fits in shared memory (fewer CTAs per cluster pack onto the GPCs in one wave),
+// else 8; 0 if neither split gives whole MMA steps and whole TMA boxes.
+static int finish_split(const Dims& d) {
+    for (int S = 4; S <= 8; S *= 2) {
+        const int hs = d.H / S, dls = d.d_l / S;
+        if (d.H % (16 * S) != 0 || (hs > 256 && hs % 256 != 0) || dls > 256) continue;
+        if (fin_smem_layout(dls + hs).total <= 200u * 1024u) return S;
+    }
+    return 0;
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -556,42 +737,70 @@ cudaError_t launch_decode_fast(const Dims& d, const void* q, const void* k_cache
     const FastPlan p = make_fast_plan(d);
     float* part_o = reinterpret_cast<float*>(workspace);
     float* part_ml = reinterpret_cast<float*>(static_cast<char*>(workspace) + p.off_ml);
-    int32_t* prefix_g = reinterpret_cast<int32_t*>(static_cast<char*>(workspace) + p.off_prefix);
     cudaError_t err;
     if (stages & 2) {
-        const size_t smem = (size_t)kStreamStages * kStreamStageBytes +
-                            (size_t)(d.n_q * 128 + 4 * kStreamMaxTS * d.n_q + 2 * d.n_q + 1024) * sizeof(float) +
-                            (size_t)(kStreamMaxBatch + 2) * sizeof(int32_t) + 8 +
-                            2 * kStreamStages * sizeof(uint64_t) + 16;
-#define GTA_LAUNCH_STREAM(NQ)                                                                              \
+        CUtensorMap tm_k, tm_c;
+        const uint32_t box[3] = {64, (uint32_t)p.T, 1};
+        const uint64_t dk[3] = {128, (uint64_t)S_cap, (uint64_t)d.B * d.n_k};
+        const uint64_t dc[3] = {(uint64_t)d.d_l, (uint64_t)S_cap, (uint64_t)d.B};
+        if (!make_bf16_map(&tm_k, k_cache, 3, dk, box) || !make_bf16_map(&tm_c, c_cache, 3, dc, box))
+            return cudaErrorInvalidValue;
+        const size_t smem = (size_t)kStreamStages * kStreamStageBytes + 2 * 8 * kStreamMaxT * sizeof(float) +
+                            (size_t)(kStreamMaxBatch + 2 + kStreamThreads) * sizeof(int32_t) +
+                            2 * kStreamStages * sizeof(uint64_t) + 16 + 1024;
+#define GTA_LAUNCH_STREAM(NT)                                                                              \
         do {                                                                                               \
-            auto kern = decode_stream_kernel<NQ>;                                                          \
+            auto kern = decode_stream_kernel<NT>;                                                          \
             err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);      \
             if (err != cudaSuccess) return err;                                                            \
-            kern<<<p.G, kStreamThreads, smem, stream>>>(d, p.TS, S_cap, (const __nv_bfloat16*)q,           \
-                                                        (const __nv_bfloat16*)k_cache,                     \
-                                                        (const __nv_bfloat16*)c_cache, seq_lens, part_o,   \
-                                                        part_ml, prefix_g, status_word);                   \
+            kern<<<p.G, kStreamThreads, smem, stream>>>(tm_k, tm_c, d, p.T, S_cap, (const __nv_bfloat16*)q, \
+                                                        seq_lens, part_o, part_ml, status_word);           \
         } while (0)
-        switch (d.n_q) {
-            case 1: GTA_LAUNCH_STREAM(1); break;
-            case 2: GTA_LAUNCH_STREAM(2); break;
-            case 4: GTA_LAUNCH_STREAM(4); break;
-            default: GTA_LAUNCH_STREAM(8); break;
+        switch (d.d_l) {
+            case 256: GTA_LAUNCH_STREAM(4); break;
+            case 512: GTA_LAUNCH_STREAM(8); break;
+            default: GTA_LAUNCH_STREAM(16); break;
         }
 #undef GTA_LAUNCH_STREAM
         if ((err = cudaGetLastError()) != cudaSuccess) return err;
         *launches += 1;
     }
     if (stages & 4) {
-        const size_t smem = ((size_t)(d.d_l / kFinSplit + d.H / kFinSplit) * kFinBlockB + 2 * kFinBlockB * 128 +
-                             kFinBlockB * 4) * sizeof(float);
-        err = cudaFuncSetAttribute(decode_finish_cluster_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        const int S = finish_split(d);
+        const int dls = d.d_l / S, hs = d.H / S, KA = dls + hs;
+        CUtensorMap tm_wp, tm_wg;
+        {
+            const uint64_t dims[3] = {128, (uint64_t)d.d_l, (uint64_t)d.n_h};
+            const uint32_t box[3] = {64, (uint32_t)dls, 1};
+            if (!make_bf16_map(&tm_wp, w_p, 3, dims, box)) return cudaErrorInvalidValue;
+        }
+        {
+            const uint64_t dims[2] = {(uint64_t)d.n_h * 128, (uint64_t)d.H};
+            const uint32_t box[2] = {64, (uint32_t)(hs < 256 ? hs : 256)};
+            if (!make_bf16_map(&tm_wg, w_g, 2, dims, box)) return cudaErrorInvalidValue;
+        }
+        const size_t smem = fin_smem_layout(KA).total;
+        err = cudaFuncSetAttribute(decode_finish_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (err != cudaSuccess) return err;
-        dim3 grid(kFinSplit, d.n_h);
-        decode_finish_cluster_kernel<<<grid, kFinThreads, smem, stream>>>(
-            d, p.G, p.TS, S_cap, seq_lens, prefix_g, part_o, part_ml, (const __nv_bfloat16*)x_t,
-            (const __nv_bfloat16*)w_p, (const __nv_bfloat16*)w_g, (__nv_bfloat16*)out);
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(S, d.n_h * 2);
+        cfg.blockDim = dim3(kFinThreads);
+        cfg.dynamicSmemBytes = smem;
+        cfg.stream = stream;
+        cudaLaunchAttribute attr[2];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = S;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        // the kernel may be scheduled while the stream kernel drains; it waits for it on the device
+        attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[1].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 2;
+        err = cudaLaunchKernelEx(&cfg, decode_finish_kernel, tm_wp, tm_wg, d, p.G, p.T, S_cap, seq_lens,
+                                 (const float*)part_o, (const float*)part_ml, (const __nv_bfloat16*)x_t,
+                                 (__nv_bfloat16*)out, status_word);
+        if (err != cudaSuccess) return err;
         if ((err = cudaGetLastError()) != cudaSuccess) return err;
         *launches += 1;
     }

@@ -10,48 +10,9 @@
 #include <cuda.h>
 
 #include "sm100_ptx.cuh"
+#include "tma_host.cuh"
 
 namespace gta {
-
-// --------------------------------------------------------------------------- host: tensor maps
-namespace {
-
-using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_fn() {
-    static EncodeTiledFn fn = [] {
-        void* p = nullptr;
-        cudaDriverEntryPointQueryResult q;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
-            q != cudaDriverEntryPointSuccess)
-            p = nullptr;
-        return reinterpret_cast<EncodeTiledFn>(p);
-    }();
-    return fn;
-}
-
-// bf16 tensor, `rank` dims (innermost first), 128-byte swizzle, zero fill outside the tensor.
-bool make_map(CUtensorMap* m, const void* base, int rank, const uint64_t* dims, const uint32_t* box) {
-    EncodeTiledFn fn = encode_fn();
-    if (!fn) return false;
-    cuuint64_t gdim[5], gstride[5];
-    cuuint32_t bx[5], estr[5];
-    uint64_t stride = 2;
-    for (int i = 0; i < rank; ++i) {
-        gdim[i] = dims[i];
-        bx[i] = box[i];
-        estr[i] = 1;
-        stride *= dims[i];
-        if (i < rank - 1) gstride[i] = stride;   // byte stride of dimension i+1
-    }
-    return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void*>(base), gdim, gstride, bx, estr,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
-}  // namespace
 
 // --------------------------------------------------------------------------- decoder + gate kernel
 constexpr int kDecStages = 4;
@@ -492,7 +453,7 @@ gta_status_t launch_sm100_prefill(const Dims& d, const void* q, const void* k, c
         const uint64_t dq[3] = {(uint64_t)d.d_h, (uint64_t)d.N, (uint64_t)d.B * d.n_q};
         const uint64_t dk[3] = {(uint64_t)d.d_h, (uint64_t)d.N, (uint64_t)d.B * d.n_k};
         const uint64_t dc[3] = {(uint64_t)d.d_l, (uint64_t)d.N, (uint64_t)d.B * d.n_c};
-        if (!make_map(&tm_q, q, 3, dq, box) || !make_map(&tm_k, k, 3, dk, box) || !make_map(&tm_c, c, 3, dc, box))
+        if (!make_bf16_map(&tm_q, q, 3, dq, box) || !make_bf16_map(&tm_k, k, 3, dk, box) || !make_bf16_map(&tm_c, c, 3, dc, box))
             return GTA_ERR_CUDA;
         if (cudaFuncSetAttribute(sm100_attention_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  (int)kAttnSmemTotal) != cudaSuccess)
@@ -512,22 +473,22 @@ gta_status_t launch_sm100_prefill(const Dims& d, const void* q, const void* k, c
         {
             const uint64_t dims[3] = {(uint64_t)d.d_l, (uint64_t)d.N, (uint64_t)d.B * d.n_q};
             const uint32_t box[3] = {kBlockK, kTileM, 1};
-            if (!make_map(&tm_l, workspace, 3, dims, box)) return GTA_ERR_CUDA;
+            if (!make_bf16_map(&tm_l, workspace, 3, dims, box)) return GTA_ERR_CUDA;
         }
         {
             const uint64_t dims[3] = {(uint64_t)d.H, (uint64_t)d.N, (uint64_t)d.B};
             const uint32_t box[3] = {kBlockK, kTileM, 1};
-            if (!make_map(&tm_x, x, 3, dims, box)) return GTA_ERR_CUDA;
+            if (!make_bf16_map(&tm_x, x, 3, dims, box)) return GTA_ERR_CUDA;
         }
         {
             const uint64_t dims[3] = {(uint64_t)d.d_h, (uint64_t)d.d_l, (uint64_t)d.n_h};
             const uint32_t box[3] = {64, kBlockK, 1};
-            if (!make_map(&tm_wp, w_p, 3, dims, box)) return GTA_ERR_CUDA;
+            if (!make_bf16_map(&tm_wp, w_p, 3, dims, box)) return GTA_ERR_CUDA;
         }
         {
             const uint64_t dims[2] = {(uint64_t)d.n_h * d.d_h, (uint64_t)d.H};
             const uint32_t box[2] = {64, kBlockK};
-            if (!make_map(&tm_wg, w_g, 2, dims, box)) return GTA_ERR_CUDA;
+            if (!make_bf16_map(&tm_wg, w_g, 2, dims, box)) return GTA_ERR_CUDA;
         }
         gta_status_t st = pair ? launch_decoder<256>(d, tm_l, tm_x, tm_wp, tm_wg, out, status_word, stream)
                                : launch_decoder<128>(d, tm_l, tm_x, tm_wp, tm_wg, out, status_word, stream);
