@@ -13,4 +13,8 @@ gta_status_t launch_sm100_prefill(const Dims& d, const void* q, const void* k, c
                                   const void* w_p, const void* w_g, void* out, void* workspace,
                                   int32_t* status_word, cudaStream_t stream, int stages, int* launches);
 
+// Decoder + gate kernel alone: out = (L W_P) (.) sigmoid(X W_G) with L[B, n_q, N, d_l] in bf16.
+gta_status_t launch_sm100_decoder(const Dims& d, const void* l_bf16, const void* x, const void* w_p, const void* w_g,
+                                  void* out, int32_t* status_word, cudaStream_t stream);
+
 }  // namespace gta

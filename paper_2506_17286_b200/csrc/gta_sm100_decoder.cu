@@ -1,0 +1,321 @@
+// tcgen05 / TMA decoder + gate kernel of the bf16 prefill path (d_h = 128):
+//     out_i = (L_{q(i)} W_P,i) (.) sigmoid(X W_G,i)          (Sec. 3.3, reformulated equation)
+//
+// Persistent: one CTA per SM walks a static list of work items.  An item is a tile of 128 token
+// rows x two heads of one attention map (256 output columns); what does not divide evenly over the
+// CTAs is cut into single-head items (128 columns) so that the last wave is short.  Roles:
+//   warp 0      TMA producer: 4-stage ring of {A tile 128 x 64, B tile 64 x NT}, gate operands
+//               (X, W_G) first, then decoder operands (L, W_P); it runs ahead into the next item.
+//   warp 1      tcgen05.mma issuer: acc_G (K = H) then acc_P (K = d_l), side by side in TMEM.
+//   warps 2-9   epilogue, two warps per TMEM lane quarter (one per head): as soon as acc_G is
+//               complete they turn it into sigmoid gates held in registers (packed bf16) and hand
+//               the columns back, so the MUFU work hides under the acc_P MMAs; when acc_P is
+//               complete they multiply, round and store, while the next item's gate MMAs run.
+#include "gta_sm100.cuh"
+
+#include <cuda.h>
+
+#include "sm100_ptx.cuh"
+#include "tma_host.cuh"
+
+namespace gta {
+
+namespace {
+
+constexpr int kDecStages = 4;
+constexpr int kDecThreads = 320;
+constexpr int kTileM = 128;        // token rows per item
+constexpr int kBlockK = 64;        // K elements per pipeline stage (one 128-byte swizzle row)
+constexpr uint32_t kATileBytes = kTileM * kBlockK * 2;   // 16 KB
+constexpr uint32_t kBGroupBytes = kBlockK * 64 * 2;      // 64 K-rows x 64 columns = 8 KB
+constexpr uint32_t kStageBytes = kATileBytes + 4 * kBGroupBytes;   // 48 KB
+constexpr uint32_t kBarOffset = kDecStages * kStageBytes;
+constexpr uint32_t kDecSmemTotal = kBarOffset + 256 + 1024;        // barriers + alignment slack
+
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&v);
+}
+// sigmoid(z) = 1/2 + 1/2 tanh(z / 2): one MUFU operation
+__device__ __forceinline__ float sigmoid_tanh(float z) {
+    float t;
+    asm("tanh.approx.f32 %0, %1;" : "=f"(t) : "f"(0.5f * z));
+    return fmaf(0.5f, t, 0.5f);
+}
+
+// Static schedule.  U units (128 rows x head pair, or x single head when a map has an odd number
+// of heads) over G CTAs: every CTA takes q = U / G whole units; the r = U mod G left over are cut
+// in two single-head halves when that makes the tail shorter (2 r <= G), else handed out whole.
+struct Schedule {
+    int n_hp;       // units per row tile (head pairs, or heads)
+    int pair;       // 1: a unit is two heads
+    int RT;         // row tiles per sequence
+    int q, r, split_tail;
+};
+
+struct Item {
+    int b, t0, i0, nt;   // batch entry, first token row, first head, columns (128 or 256)
+};
+
+__device__ __forceinline__ int items_of_cta(const Schedule& s, int cta, int G) {
+    if (s.split_tail) return s.q + ((cta < 2 * s.r) ? 1 : 0);
+    return s.q + ((cta < s.r) ? 1 : 0);
+}
+
+__device__ __forceinline__ Item item_of(const Schedule& s, int cta, int G, int n) {
+    int u, half = -1;
+    if (n < s.q) u = cta * s.q + n;
+    else if (s.split_tail) { u = G * s.q + (cta >> 1); half = cta & 1; }
+    else u = G * s.q + cta;
+    Item it;
+    const int hp = u % s.n_hp;
+    const int rt = (u / s.n_hp) % s.RT;
+    it.b = u / (s.n_hp * s.RT);
+    it.t0 = rt * kTileM;
+    if (s.pair) {
+        it.i0 = 2 * hp + (half < 0 ? 0 : half);
+        it.nt = half < 0 ? 256 : 128;
+    } else {
+        it.i0 = hp;
+        it.nt = 128;
+    }
+    return it;
+}
+
+__global__ void __launch_bounds__(kDecThreads, 1)
+sm100_decoder_kernel(const __grid_constant__ CUtensorMap tm_l, const __grid_constant__ CUtensorMap tm_x,
+                     const __grid_constant__ CUtensorMap tm_wp, const __grid_constant__ CUtensorMap tm_wg,
+                     Dims d, Schedule sch, __nv_bfloat16* __restrict__ out, int32_t* status_word) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + kBarOffset);
+    uint64_t* empty_bar = full_bar + kDecStages;
+    uint64_t* accg_full = empty_bar + kDecStages;
+    uint64_t* accg_free = accg_full + 1;
+    uint64_t* accp_full = accg_free + 1;
+    uint64_t* accp_free = accp_full + 1;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(accp_free + 1);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+    volatile int* drain_flag = abort_flag + 1;   // never raised: lets the drain wait run to its limit
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int G = gridDim.x, cta = blockIdx.x;
+    const int n_items = items_of_cta(sch, cta, G);
+    const int ks_g = d.H / kBlockK, ks_p = d.d_l / kBlockK, ks_total = ks_g + ks_p;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kDecStages; ++s) { ptx::mbar_init(&full_bar[s], 1); ptx::mbar_init(&empty_bar[s], 1); }
+        ptx::mbar_init(accg_full, 1);
+        ptx::mbar_init(accg_free, 8);
+        ptx::mbar_init(accp_full, 1);
+        ptx::mbar_init(accp_free, 8);
+        *abort_flag = 0;
+        *drain_flag = 0;
+        ptx::fence_mbar_init();
+    }
+    if (warp == 1) ptx::tmem_alloc(tmem_slot, 512);
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    ptx::tc_fence_after_sync();
+    const uint32_t tmem_base = *tmem_slot;
+    const uint32_t tmem_p = tmem_base, tmem_g = tmem_base + 256;
+
+    if (warp == 0) {
+        if (ptx::elect_one()) {
+            ptx::prefetch_tensormap(&tm_l); ptx::prefetch_tensormap(&tm_x);
+            ptx::prefetch_tensormap(&tm_wp); ptx::prefetch_tensormap(&tm_wg);
+            int it = 0;            // ring iteration, runs on across items
+            bool ok = true;
+            for (int n = 0; n < n_items && ok; ++n) {
+                const Item w = item_of(sch, cta, G, n);
+                const int g = d.head_to_q(w.i0);
+                const int n_grp = w.nt / 64;
+                const uint32_t tx = kATileBytes + (uint32_t)n_grp * kBGroupBytes;
+                for (int ks = 0; ks < ks_total; ++ks, ++it) {
+                    const int s = it % kDecStages;
+                    const uint32_t ph = (it / kDecStages) & 1;
+                    ok = ptx::mbar_wait(&empty_bar[s], ph ^ 1, abort_flag);
+                    if (!ok) break;
+                    uint8_t* a_s = smem + s * kStageBytes;
+                    uint8_t* b_s = a_s + kATileBytes;
+                    ptx::mbar_arrive_expect_tx(&full_bar[s], tx);
+                    if (ks < ks_g) {
+                        ptx::tma_load_3d(a_s, &tm_x, &full_bar[s], ks * kBlockK, w.t0, w.b);
+                        for (int grp = 0; grp < n_grp; ++grp)
+                            ptx::tma_load_2d(b_s + grp * kBGroupBytes, &tm_wg, &full_bar[s], w.i0 * 128 + grp * 64,
+                                             ks * kBlockK);
+                    } else {
+                        const int kk = ks - ks_g;
+                        ptx::tma_load_3d(a_s, &tm_l, &full_bar[s], kk * kBlockK, w.t0, w.b * d.n_q + g);
+                        for (int grp = 0; grp < n_grp; ++grp)
+                            ptx::tma_load_3d(b_s + grp * kBGroupBytes, &tm_wp, &full_bar[s], (grp & 1) * 64,
+                                             kk * kBlockK, w.i0 + (grp >> 1));
+                    }
+                }
+            }
+            if (*abort_flag) {   // drain: every armed stage either lands or the wait gives up
+                for (int back = 1; back <= kDecStages && it - back >= 0; ++back) {
+                    const int kq = it - back;
+                    ptx::mbar_wait(&full_bar[kq % kDecStages], (kq / kDecStages) & 1, drain_flag);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        if (ptx::elect_one()) {
+            int it = 0;
+            bool ok = true;
+            for (int n = 0; n < n_items && ok; ++n) {
+                const Item w = item_of(sch, cta, G, n);
+                const uint32_t idesc = ptx::make_idesc_bf16(kTileM, w.nt, 0, 1);   // A K-major, B MN-major
+                for (int ks = 0; ks < ks_total; ++ks, ++it) {
+                    // the accumulator about to be overwritten must have been read by the epilogue
+                    if (ks == 0) ok = ptx::mbar_wait(accg_free, (n & 1) ^ 1, abort_flag);
+                    else if (ks == ks_g) ok = ptx::mbar_wait(accp_free, (n & 1) ^ 1, abort_flag);
+                    if (!ok) break;
+                    const int s = it % kDecStages;
+                    const uint32_t ph = (it / kDecStages) & 1;
+                    ok = ptx::mbar_wait(&full_bar[s], ph, abort_flag);
+                    if (!ok) break;
+                    ptx::tc_fence_after_sync();
+                    const uint32_t a_addr = ptx::smem_addr(smem + s * kStageBytes);
+                    const uint32_t b_addr = a_addr + kATileBytes;
+                    const uint32_t d_tmem = ks < ks_g ? tmem_g : tmem_p;
+                    const bool first = (ks == 0) || (ks == ks_g);
+#pragma unroll
+                    for (int k4 = 0; k4 < kBlockK / 16; ++k4) {
+                        const uint64_t a_desc = ptx::make_smem_desc(a_addr + k4 * 32, 16, 1024);
+                        const uint64_t b_desc = ptx::make_smem_desc(b_addr + k4 * 16 * 128, 64 * 128, 1024);
+                        ptx::mma_ss(d_tmem, a_desc, b_desc, idesc, (first && k4 == 0) ? 0u : 1u);
+                    }
+                    ptx::tc_commit(&empty_bar[s]);
+                    if (ks == ks_g - 1) ptx::tc_commit(accg_full);
+                    if (ks == ks_total - 1) ptx::tc_commit(accp_full);
+                }
+            }
+        }
+    } else {
+        // epilogue: warp w may touch TMEM lanes [32 (w % 4), 32 (w % 4) + 32); the two warps of a
+        // quarter take one half of the item's columns each (= one head of a pair)
+        const int quarter = warp & 3;
+        const int half = (warp - 2) >> 2;
+        const int row = quarter * 32 + lane;
+        const uint32_t lane_base = ((uint32_t)(quarter * 32) << 16);
+        bool ok = true;
+        for (int n = 0; n < n_items && ok; ++n) {
+            const Item w = item_of(sch, cta, G, n);
+            const int cols = w.nt / 2;               // this warp's columns: 128 or 64
+            const int c0 = half * cols;
+            const int t = w.t0 + row;
+            uint32_t gate[64];                       // sigmoid gates, packed bf16 pairs
+            ok = __all_sync(0xffffffffu, ptx::mbar_wait(accg_full, n & 1, abort_flag));
+            if (!ok) break;
+            ptx::tc_fence_after_sync();
+#pragma unroll
+            for (int ch = 0; ch < 4; ++ch) {
+                if (ch * 32 < cols) {
+                    uint32_t z[32];
+                    ptx::tmem_ld32(tmem_g + lane_base + c0 + ch * 32, z);
+                    ptx::tmem_wait_ld();
+#pragma unroll
+                    for (int e = 0; e < 16; ++e)
+                        gate[ch * 16 + e] = pack_bf16x2(sigmoid_tanh(__uint_as_float(z[2 * e])),
+                                                        sigmoid_tanh(__uint_as_float(z[2 * e + 1])));
+                }
+            }
+            ptx::tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(accg_free);
+
+            ok = __all_sync(0xffffffffu, ptx::mbar_wait(accp_full, n & 1, abort_flag));
+            if (!ok) break;
+            ptx::tc_fence_after_sync();
+            // columns [c0, c0 + cols) of the item = head i0 + (c0 / 128), columns (c0 % 128) ..
+            __nv_bfloat16* o_row = out + (((size_t)w.b * d.N + (t < d.N ? t : 0)) * d.n_h + w.i0) * 128 + c0;
+#pragma unroll
+            for (int ch = 0; ch < 4; ++ch) {
+                if (ch * 32 < cols) {
+                    uint32_t p[32];
+                    ptx::tmem_ld32(tmem_p + lane_base + c0 + ch * 32, p);
+                    ptx::tmem_wait_ld();
+                    uint32_t packed[16];
+#pragma unroll
+                    for (int e = 0; e < 16; ++e) {
+                        const uint32_t gg = gate[ch * 16 + e];
+                        const float g0 = __uint_as_float(gg << 16), g1 = __uint_as_float(gg & 0xffff0000u);
+                        packed[e] = pack_bf16x2(__uint_as_float(p[2 * e]) * g0, __uint_as_float(p[2 * e + 1]) * g1);
+                    }
+                    if (t < d.N) {
+                        uint4* dst = reinterpret_cast<uint4*>(o_row + ch * 32);
+#pragma unroll
+                        for (int v = 0; v < 4; ++v)
+                            dst[v] = make_uint4(packed[4 * v], packed[4 * v + 1], packed[4 * v + 2], packed[4 * v + 3]);
+                    }
+                }
+            }
+            ptx::tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(accp_free);
+        }
+    }
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 1) ptx::tmem_dealloc(tmem_base, 512);
+    if (threadIdx.x == 0 && *abort_flag) raise_status(status_word, GTA_ERR_TIMEOUT);
+}
+
+int sm_count() {
+    static int n = [] {
+        int dev = 0, v = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v <= 0)
+            v = 148;
+        return v;
+    }();
+    return n;
+}
+
+}  // namespace
+
+gta_status_t launch_sm100_decoder(const Dims& d, const void* l_bf16, const void* x, const void* w_p, const void* w_g,
+                                  void* out, int32_t* status_word, cudaStream_t stream) {
+    CUtensorMap tm_l, tm_x, tm_wp, tm_wg;
+    {
+        const uint64_t dims[3] = {(uint64_t)d.d_l, (uint64_t)d.N, (uint64_t)d.B * d.n_q};
+        const uint32_t box[3] = {kBlockK, kTileM, 1};
+        if (!make_bf16_map(&tm_l, l_bf16, 3, dims, box)) return GTA_ERR_CUDA;
+    }
+    {
+        const uint64_t dims[3] = {(uint64_t)d.H, (uint64_t)d.N, (uint64_t)d.B};
+        const uint32_t box[3] = {kBlockK, kTileM, 1};
+        if (!make_bf16_map(&tm_x, x, 3, dims, box)) return GTA_ERR_CUDA;
+    }
+    {
+        const uint64_t dims[3] = {(uint64_t)d.d_h, (uint64_t)d.d_l, (uint64_t)d.n_h};
+        const uint32_t box[3] = {64, kBlockK, 1};
+        if (!make_bf16_map(&tm_wp, w_p, 3, dims, box)) return GTA_ERR_CUDA;
+    }
+    {
+        const uint64_t dims[2] = {(uint64_t)d.n_h * d.d_h, (uint64_t)d.H};
+        const uint32_t box[2] = {64, kBlockK};
+        if (!make_bf16_map(&tm_wg, w_g, 2, dims, box)) return GTA_ERR_CUDA;
+    }
+    Schedule s;
+    s.pair = (d.n_h / d.n_q) % 2 == 0 ? 1 : 0;
+    s.n_hp = s.pair ? d.n_h / 2 : d.n_h;
+    s.RT = (d.N + kTileM - 1) / kTileM;
+    const long long U = (long long)d.B * s.RT * s.n_hp;
+    if (U > 0x3fffffffLL) return GTA_ERR_UNSUPPORTED;
+    const int sms = sm_count();
+    const int G = U < sms ? (int)U : sms;
+    s.q = (int)(U / G);
+    s.r = (int)(U % G);
+    s.split_tail = (s.pair && 2 * s.r <= G) ? 1 : 0;
+    if (cudaFuncSetAttribute(sm100_decoder_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)kDecSmemTotal) != cudaSuccess)
+        return GTA_ERR_CUDA;
+    sm100_decoder_kernel<<<G, kDecThreads, kDecSmemTotal, stream>>>(tm_l, tm_x, tm_wp, tm_wg, d, s,
+                                                                    (__nv_bfloat16*)out, status_word);
+    return cudaGetLastError() == cudaSuccess ? GTA_OK : GTA_ERR_CUDA;
+}
+
+}  // namespace gta
