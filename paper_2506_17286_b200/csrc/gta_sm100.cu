@@ -18,16 +18,21 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
 }
 
 // --------------------------------------------------------------------------- attention kernel
-// One CTA = one 128-row query tile of one attention map x one 256-column slice of the latent
+// A work item = one 128-row query tile of one attention map x one 256-column slice of the latent
 // (the 128 x d_l fp32 output does not fit the 512 TMEM columns next to the score tiles, so d_l is
-// cut in slices of 256 and each slice CTA recomputes the scores).  Per 128-key tile j:
+// cut in slices of 256 and each slice item recomputes the scores).  Persistent: one CTA per SM
+// walks a static list of items, heaviest (latest) query tiles first, dealt to the CTAs in snake
+// order so that every CTA gets about the same number of key tiles.  Per 128-key tile j:
 //   S_j = Q K_j^T            tcgen05.mma, smem x smem -> TMEM (two S buffers, ping-pong)
-//   P_j = exp2(S_j c - m)    128 softmax threads, one row each; P_j (bf16) overwrites S_j in TMEM
+//   P_j = exp2(S_j c - m)    256 softmax threads, two per row (64 keys each, row maximum exchanged
+//                            through shared memory); P_j (bf16) overwrites S_j in TMEM
 //   O  += P_j C_j            tcgen05.mma, TMEM x smem (C is the MN-major B operand) -> TMEM
 // The running maximum is only raised when it grows by more than 2^8 (the accumulators stay in
 // range and O needs rescaling on few tiles); O is divided by the row sum at the end and written
-// as bf16 to L[B, n_q, N, d_l].
-constexpr int kAttnThreads = 192;
+// as bf16 to L[B, n_q, N, d_l].  The K / C ring and the score pipeline run on across items: the
+// next item's Q is requested as soon as the last QK^T of the current item has been issued, and
+// its first score tile is computed while the current item's output is being stored.
+constexpr int kAttnThreads = 320;
 constexpr int kKeyTile = 128;
 constexpr int kSlice = 256;
 constexpr uint32_t kQBytes = 128 * 128 * 2;            // 32 KB
@@ -35,13 +40,38 @@ constexpr uint32_t kKStageBytes = kKeyTile * 128 * 2;  // 32 KB
 constexpr uint32_t kCStageBytes = kKeyTile * kSlice * 2;  // 64 KB
 constexpr uint32_t kAttnKOff = kQBytes;
 constexpr uint32_t kAttnCOff = kAttnKOff + 2 * kKStageBytes;
-constexpr uint32_t kAttnBarOff = kAttnCOff + 2 * kCStageBytes;
-constexpr uint32_t kAttnSmemTotal = kAttnBarOff + 256 + 1024;
+constexpr uint32_t kAttnXchgOff = kAttnCOff + 2 * kCStageBytes;          // float [2][4][2][32]
+constexpr uint32_t kAttnBarOff = kAttnXchgOff + 2 * 4 * 2 * 32 * 4;
+constexpr uint32_t kAttnAlignSlack = 768;   // the 227 KB limit leaves no more; checked in the kernel
+constexpr uint32_t kAttnSmemTotal = kAttnBarOff + 256 + kAttnAlignSlack;
+static_assert(kAttnSmemTotal <= 232448, "attention kernel shared memory exceeds the per-CTA limit");
 
 __device__ __forceinline__ float fast_exp2(float x) {
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
+}
+__device__ __forceinline__ void pair_sync(int quarter) {   // the two softmax warps of a TMEM lane quarter
+    asm volatile("bar.sync %0, 64;" ::"r"(quarter + 1) : "memory");
+}
+
+struct AttnItem {
+    int b, g, slice, qi, n_tiles;
+};
+
+// Item `n` of CTA `cta`: position p in the list sorted by descending query tile, rounds dealt
+// alternately left-to-right and right-to-left.  Returns false past the end of the list.
+__device__ __forceinline__ bool attn_item(const Dims& d, int n_qt, int n_slices, long long total, int G, int cta,
+                                          int n, AttnItem* it) {
+    const long long p = (long long)n * G + ((n & 1) ? (G - 1 - cta) : cta);
+    if (p >= total) return false;
+    long long r = p;
+    it->slice = (int)(r % n_slices); r /= n_slices;
+    it->g = (int)(r % d.n_q); r /= d.n_q;
+    it->b = (int)(r % d.B); r /= d.B;
+    it->qi = n_qt - 1 - (int)r;
+    it->n_tiles = d.causal ? it->qi + 1 : n_qt;
+    return true;
 }
 
 __global__ void __launch_bounds__(kAttnThreads, 1)
@@ -50,40 +80,42 @@ sm100_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                        int32_t* status_word) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    float* xchg = reinterpret_cast<float*>(smem + kAttnXchgOff);
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kAttnBarOff);
     uint64_t* q_full = bars;            // 1
-    uint64_t* k_full = bars + 1;        // 2
-    uint64_t* k_empty = bars + 3;       // 2
-    uint64_t* c_full = bars + 5;        // 2
-    uint64_t* c_empty = bars + 7;       // 2
-    uint64_t* s_full = bars + 9;        // 2
-    uint64_t* p_full = bars + 11;       // 2
-    uint64_t* o_done = bars + 13;       // 1
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 14);
+    uint64_t* q_empty = bars + 1;       // 1
+    uint64_t* k_full = bars + 2;        // 2
+    uint64_t* k_empty = bars + 4;       // 2
+    uint64_t* c_full = bars + 6;        // 2
+    uint64_t* c_empty = bars + 8;       // 2
+    uint64_t* s_full = bars + 10;       // 2
+    uint64_t* p_full = bars + 12;       // 2
+    uint64_t* o_done = bars + 14;       // 1
+    uint64_t* o_free = bars + 15;       // 1
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 16);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
     volatile int* drain_flag = abort_flag + 1;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    // heaviest (latest) query tiles first
+    const int G = gridDim.x, cta = blockIdx.x;
+    if ((uint32_t)(smem - smem_raw) > kAttnAlignSlack) {   // uniform; cannot happen with a 256-byte aligned window
+        if (threadIdx.x == 0) raise_status(status_word, GTA_ERR_CUDA);
+        return;
+    }
     const int n_slices = d.d_l / kSlice;
     const int n_qt = (d.N + 127) / 128;
-    int bid = blockIdx.x;
-    const int slice = bid % n_slices; bid /= n_slices;
-    const int g = bid % d.n_q; bid /= d.n_q;
-    const int b = bid % d.B; bid /= d.B;
-    const int qi = n_qt - 1 - bid;
-    const int q0 = qi * 128;
-    const int kg = d.q_to_k(g), cg = d.q_to_c(g);
-    const int n_tiles = d.causal ? qi + 1 : n_qt;
+    const long long total = (long long)n_qt * n_slices * d.n_q * d.B;
 
     if (threadIdx.x == 0) {
         ptx::mbar_init(q_full, 1);
+        ptx::mbar_init(q_empty, 1);
         for (int s = 0; s < 2; ++s) {
             ptx::mbar_init(&k_full[s], 1); ptx::mbar_init(&k_empty[s], 1);
             ptx::mbar_init(&c_full[s], 1); ptx::mbar_init(&c_empty[s], 1);
-            ptx::mbar_init(&s_full[s], 1); ptx::mbar_init(&p_full[s], 128);
+            ptx::mbar_init(&s_full[s], 1); ptx::mbar_init(&p_full[s], 256);
         }
         ptx::mbar_init(o_done, 1);
+        ptx::mbar_init(o_free, 256);
         *abort_flag = 0;
         *drain_flag = 0;
         ptx::fence_mbar_init();
@@ -98,33 +130,41 @@ sm100_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     if (warp == 0) {
         if (ptx::elect_one()) {
             ptx::prefetch_tensormap(&tm_q); ptx::prefetch_tensormap(&tm_k); ptx::prefetch_tensormap(&tm_c);
-            ptx::mbar_arrive_expect_tx(q_full, kQBytes);
-            ptx::tma_load_3d(smem, &tm_q, q_full, 0, q0, b * d.n_q + g);
-            ptx::tma_load_3d(smem + 16384, &tm_q, q_full, 64, q0, b * d.n_q + g);
-            int j = 0;
+            int tj = 0;                 // key tiles issued so far (ring position), across items
             bool ok = true;
-            for (; j < n_tiles && ok; ++j) {
-                const int s = j & 1;
-                const uint32_t ph = (j >> 1) & 1;
-                ok = ptx::mbar_wait(&k_empty[s], ph ^ 1, abort_flag);
+            bool q_armed = false;
+            AttnItem w;
+            for (int n = 0; ok && attn_item(d, n_qt, n_slices, total, G, cta, n, &w); ++n) {
+                const int kg = d.q_to_k(w.g), cg = d.q_to_c(w.g);
+                ok = ptx::mbar_wait(q_empty, (n & 1) ^ 1, abort_flag);
                 if (!ok) break;
-                uint8_t* k_s = smem + kAttnKOff + s * kKStageBytes;
-                ptx::mbar_arrive_expect_tx(&k_full[s], kKStageBytes);
-                ptx::tma_load_3d(k_s, &tm_k, &k_full[s], 0, j * kKeyTile, b * d.n_k + kg);
-                ptx::tma_load_3d(k_s + 16384, &tm_k, &k_full[s], 64, j * kKeyTile, b * d.n_k + kg);
-                ok = ptx::mbar_wait(&c_empty[s], ph ^ 1, abort_flag);
-                if (!ok) { ++j; break; }
-                uint8_t* c_s = smem + kAttnCOff + s * kCStageBytes;
-                ptx::mbar_arrive_expect_tx(&c_full[s], kCStageBytes);
+                ptx::mbar_arrive_expect_tx(q_full, kQBytes);
+                ptx::tma_load_3d(smem, &tm_q, q_full, 0, w.qi * 128, w.b * d.n_q + w.g);
+                ptx::tma_load_3d(smem + 16384, &tm_q, q_full, 64, w.qi * 128, w.b * d.n_q + w.g);
+                q_armed = true;
+                for (int j = 0; j < w.n_tiles; ++j, ++tj) {
+                    const int s = tj & 1;
+                    const uint32_t ph = (tj >> 1) & 1;
+                    ok = ptx::mbar_wait(&k_empty[s], ph ^ 1, abort_flag);
+                    if (!ok) break;
+                    uint8_t* k_s = smem + kAttnKOff + s * kKStageBytes;
+                    ptx::mbar_arrive_expect_tx(&k_full[s], kKStageBytes);
+                    ptx::tma_load_3d(k_s, &tm_k, &k_full[s], 0, j * kKeyTile, w.b * d.n_k + kg);
+                    ptx::tma_load_3d(k_s + 16384, &tm_k, &k_full[s], 64, j * kKeyTile, w.b * d.n_k + kg);
+                    ok = ptx::mbar_wait(&c_empty[s], ph ^ 1, abort_flag);
+                    if (!ok) { ++tj; break; }
+                    uint8_t* c_s = smem + kAttnCOff + s * kCStageBytes;
+                    ptx::mbar_arrive_expect_tx(&c_full[s], kCStageBytes);
 #pragma unroll
-                for (int grp = 0; grp < kSlice / 64; ++grp)
-                    ptx::tma_load_3d(c_s + grp * 16384, &tm_c, &c_full[s], slice * kSlice + grp * 64, j * kKeyTile,
-                                     b * d.n_c + cg);
+                    for (int grp = 0; grp < kSlice / 64; ++grp)
+                        ptx::tma_load_3d(c_s + grp * 16384, &tm_c, &c_full[s], w.slice * kSlice + grp * 64,
+                                         j * kKeyTile, w.b * d.n_c + cg);
+                }
             }
             if (*abort_flag) {   // drain what was armed (bounded), so no copy lands after exit
-                ptx::mbar_wait(q_full, 0, drain_flag);
-                for (int back = 1; back <= 2 && j - back >= 0; ++back) {
-                    const int jq = j - back;
+                if (q_armed) ptx::mbar_wait(q_full, 0, drain_flag), ptx::mbar_wait(q_full, 1, drain_flag);
+                for (int back = 1; back <= 2 && tj - back >= 0; ++back) {
+                    const int jq = tj - back;
                     ptx::mbar_wait(&k_full[jq & 1], (jq >> 1) & 1, drain_flag);
                     ptx::mbar_wait(&c_full[jq & 1], (jq >> 1) & 1, drain_flag);
                 }
@@ -135,141 +175,173 @@ sm100_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
             constexpr uint32_t idesc_qk = ptx::make_idesc_bf16(128, kKeyTile, 0, 0);   // both K-major
             constexpr uint32_t idesc_pv = ptx::make_idesc_bf16(128, kSlice, 0, 1);     // B = C, MN-major
             const uint32_t q_addr = ptx::smem_addr(smem);
-            auto issue_qk = [&](int j) {
-                const uint32_t k_addr = ptx::smem_addr(smem + kAttnKOff + (j & 1) * kKStageBytes);
-                const uint32_t s_tmem = tmem_base + (j & 1) * 128;
+            bool ok = true;
+            // S = Q K^T of ring tile tj; `first` / `last`: first / last key tile of its item n
+            auto issue_qk = [&](int tj, int n, bool first, bool last) {
+                if (first) ok = ptx::mbar_wait(q_full, n & 1, abort_flag);
+                if (ok) ok = ptx::mbar_wait(&k_full[tj & 1], (tj >> 1) & 1, abort_flag);
+                if (!ok) return;
+                ptx::tc_fence_after_sync();
+                const uint32_t k_addr = ptx::smem_addr(smem + kAttnKOff + (tj & 1) * kKStageBytes);
+                const uint32_t s_tmem = tmem_base + (tj & 1) * 128;
 #pragma unroll
                 for (int k8 = 0; k8 < 8; ++k8) {
                     const uint32_t off = (k8 >> 2) * 16384 + (k8 & 3) * 32;
                     ptx::mma_ss(s_tmem, ptx::make_smem_desc(q_addr + off, 16, 1024),
                                 ptx::make_smem_desc(k_addr + off, 16, 1024), idesc_qk, k8 ? 1u : 0u);
                 }
-                ptx::tc_commit(&s_full[j & 1]);
-                ptx::tc_commit(&k_empty[j & 1]);
+                ptx::tc_commit(&s_full[tj & 1]);
+                ptx::tc_commit(&k_empty[tj & 1]);
+                if (last) ptx::tc_commit(q_empty);
             };
-            bool ok = ptx::mbar_wait(q_full, 0, abort_flag) && ptx::mbar_wait(&k_full[0], 0, abort_flag);
-            if (ok) {
-                ptx::tc_fence_after_sync();
-                issue_qk(0);
-            }
-            for (int j = 0; j < n_tiles && ok; ++j) {
-                if (j + 1 < n_tiles) {
-                    ok = ptx::mbar_wait(&k_full[(j + 1) & 1], ((j + 1) >> 1) & 1, abort_flag);
+            int tj = 0;
+            AttnItem w, nxt;
+            bool have = attn_item(d, n_qt, n_slices, total, G, cta, 0, &w);
+            if (have) issue_qk(0, 0, true, w.n_tiles == 1);
+            for (int n = 0; have && ok; ++n) {
+                const bool have_next = attn_item(d, n_qt, n_slices, total, G, cta, n + 1, &nxt);
+                for (int j = 0; j < w.n_tiles && ok; ++j, ++tj) {
+                    // look ahead: the next score tile, of this item or of the next one
+                    if (j + 1 < w.n_tiles) issue_qk(tj + 1, n, false, j + 2 == w.n_tiles);
+                    else if (have_next) issue_qk(tj + 1, n + 1, true, nxt.n_tiles == 1);
+                    if (!ok) break;
+                    ok = ptx::mbar_wait(&p_full[tj & 1], (tj >> 1) & 1, abort_flag) &&
+                         ptx::mbar_wait(&c_full[tj & 1], (tj >> 1) & 1, abort_flag);
+                    if (ok && j == 0 && n > 0) ok = ptx::mbar_wait(o_free, (n - 1) & 1, abort_flag);
                     if (!ok) break;
                     ptx::tc_fence_after_sync();
-                    issue_qk(j + 1);
-                }
-                ok = ptx::mbar_wait(&p_full[j & 1], (j >> 1) & 1, abort_flag) &&
-                     ptx::mbar_wait(&c_full[j & 1], (j >> 1) & 1, abort_flag);
-                if (!ok) break;
-                ptx::tc_fence_after_sync();
-                const uint32_t c_addr = ptx::smem_addr(smem + kAttnCOff + (j & 1) * kCStageBytes);
-                const uint32_t p_tmem = tmem_base + (j & 1) * 128;
+                    const uint32_t c_addr = ptx::smem_addr(smem + kAttnCOff + (tj & 1) * kCStageBytes);
+                    const uint32_t p_tmem = tmem_base + (tj & 1) * 128;
 #pragma unroll
-                for (int k8 = 0; k8 < 8; ++k8)
-                    ptx::mma_ts(tmem_o, p_tmem + k8 * 8, ptx::make_smem_desc(c_addr + k8 * 2048, 16384, 1024),
-                                idesc_pv, (j > 0 || k8 > 0) ? 1u : 0u);
-                ptx::tc_commit(o_done);
-                ptx::tc_commit(&c_empty[j & 1]);
+                    for (int k8 = 0; k8 < 8; ++k8)
+                        ptx::mma_ts(tmem_o, p_tmem + k8 * 8, ptx::make_smem_desc(c_addr + k8 * 2048, 16384, 1024),
+                                    idesc_pv, (j > 0 || k8 > 0) ? 1u : 0u);
+                    ptx::tc_commit(o_done);
+                    ptx::tc_commit(&c_empty[tj & 1]);
+                }
+                w = nxt;
+                have = have_next;
             }
         }
     } else {
         const int quarter = warp & 3;
+        const int half = (warp - 2) >> 2;            // which 64 keys of a tile / which 128 output columns
         const int row = quarter * 32 + lane;
-        const int t = q0 + row;
         const uint32_t lane_base = ((uint32_t)(quarter * 32) << 16);
         const float c_scale = d.scale * 1.4426950408889634f;
-        float m = -INFINITY, l = 0.f;
         bool ok = true;
-        for (int j = 0; j < n_tiles && ok; ++j) {
-            ok = __all_sync(0xffffffffu, ptx::mbar_wait(&s_full[j & 1], (j >> 1) & 1, abort_flag));
-            if (!ok) break;   // warp-uniform: the TMEM instructions below are warp-collective
-            ptx::tc_fence_after_sync();
-            const uint32_t s_tmem = tmem_base + lane_base + (j & 1) * 128;
-            float sv[128];
-#pragma unroll
-            for (int ch = 0; ch < 4; ++ch) {
-                uint32_t r[32];
-                ptx::tmem_ld32(s_tmem + ch * 32, r);
-                ptx::tmem_wait_ld();
-#pragma unroll
-                for (int e = 0; e < 32; ++e) sv[ch * 32 + e] = __uint_as_float(r[e]) * c_scale;
-            }
-            // mask: keys past the sequence end, and (causal) keys after the query, on boundary tiles
-            const int key0 = j * kKeyTile;
-            const int last_key = d.causal ? min(t, d.N - 1) : d.N - 1;
-            if (key0 + kKeyTile - 1 > last_key) {
-#pragma unroll
-                for (int e = 0; e < 128; ++e)
-                    if (key0 + e > last_key) sv[e] = -INFINITY;
-            }
-            float m_tile = sv[0];
-#pragma unroll
-            for (int e = 1; e < 128; ++e) m_tile = fmaxf(m_tile, sv[e]);
-            float alpha = 1.f;
-            bool raise = m_tile > m + 8.f;     // also true on the first tile (m = -inf)
-            if (raise) {
-                alpha = fast_exp2(m - m_tile);
-                m = m_tile;
-            }
-            const float neg_m = (m == -INFINITY) ? 0.f : -m;   // a fully masked row keeps p = 0
-            float sum = 0.f;
-            uint32_t packed[64];
-#pragma unroll
-            for (int e = 0; e < 64; ++e) {
-                const float p0 = fast_exp2(sv[2 * e] + neg_m);
-                const float p1 = fast_exp2(sv[2 * e + 1] + neg_m);
-                sum += p0 + p1;
-                packed[e] = pack_bf16x2(p0, p1);
-            }
-            l = l * alpha + sum;
-            // P_j (bf16 pairs) over the first 64 columns of S_j
-            {
-                uint32_t (*pk)[32] = reinterpret_cast<uint32_t (*)[32]>(packed);
-                ptx::tmem_st32(s_tmem, pk[0]);
-                ptx::tmem_st32(s_tmem + 32, pk[1]);
-            }
-            if (j > 0 && __any_sync(0xffffffffu, raise)) {
-                ok = __all_sync(0xffffffffu, ptx::mbar_wait(o_done, (j - 1) & 1, abort_flag));
-                if (!ok) break;
+        int tj = 0;
+        AttnItem w;
+        for (int n = 0; ok && attn_item(d, n_qt, n_slices, total, G, cta, n, &w); ++n) {
+            const int t = w.qi * 128 + row;
+            float m = -INFINITY, l = 0.f;            // m in scaled (log2) units; l = this thread's share of the row sum
+            for (int j = 0; j < w.n_tiles && ok; ++j, ++tj) {
+                ok = __all_sync(0xffffffffu, ptx::mbar_wait(&s_full[tj & 1], (tj >> 1) & 1, abort_flag));
+                if (!ok) break;   // warp-uniform: the TMEM instructions below are warp-collective
                 ptx::tc_fence_after_sync();
-#pragma unroll 1
-                for (int ch = 0; ch < kSlice / 32; ++ch) {
-                    uint32_t r[32];
-                    ptx::tmem_ld32(tmem_o + lane_base + ch * 32, r);
+                const uint32_t s_tmem = tmem_base + lane_base + (tj & 1) * 128;
+                float sv[64];
+                {
+                    uint32_t r0[32], r1[32];
+                    ptx::tmem_ld32(s_tmem + half * 64, r0);
+                    ptx::tmem_ld32(s_tmem + half * 64 + 32, r1);
                     ptx::tmem_wait_ld();
 #pragma unroll
-                    for (int e = 0; e < 32; ++e) r[e] = __float_as_uint(__uint_as_float(r[e]) * alpha);
-                    ptx::tmem_st32(tmem_o + lane_base + ch * 32, r);
+                    for (int e = 0; e < 32; ++e) { sv[e] = __uint_as_float(r0[e]); sv[32 + e] = __uint_as_float(r1[e]); }
                 }
-            }
-            ptx::tmem_wait_st();
-            ptx::tc_fence_before_sync();
-            ptx::mbar_arrive(&p_full[j & 1]);
-        }
-        if (ok) ok = __all_sync(0xffffffffu, ptx::mbar_wait(o_done, (n_tiles - 1) & 1, abort_flag));
-        if (ok) {
-            ptx::tc_fence_after_sync();
-            const float inv_l = 1.f / l;
-            __nv_bfloat16* o_row = o_lat + (((size_t)b * d.n_q + g) * d.N + (t < d.N ? t : 0)) * d.d_l + slice * kSlice;
+                // mask: keys past the sequence end, and (causal) keys after the query, on boundary tiles
+                const int key0 = j * kKeyTile + half * 64;
+                const int last_key = d.causal ? min(t, d.N - 1) : d.N - 1;
+                if (key0 + 63 > last_key) {
+#pragma unroll
+                    for (int e = 0; e < 64; ++e)
+                        if (key0 + e > last_key) sv[e] = -INFINITY;
+                }
+                float mx[4] = {sv[0], sv[1], sv[2], sv[3]};
+#pragma unroll
+                for (int e = 4; e < 64; e += 4) {
+                    mx[0] = fmaxf(mx[0], sv[e]); mx[1] = fmaxf(mx[1], sv[e + 1]);
+                    mx[2] = fmaxf(mx[2], sv[e + 2]); mx[3] = fmaxf(mx[3], sv[e + 3]);
+                }
+                const float m_half = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * c_scale;   // c_scale > 0
+                float* xs = xchg + (tj & 1) * 256 + quarter * 64;
+                xs[half * 32 + lane] = m_half;
+                pair_sync(quarter);
+                const float m_tile = fmaxf(m_half, xs[(half ^ 1) * 32 + lane]);
+                float alpha = 1.f;
+                const bool raise = m_tile > m + 8.f;     // also true on the first tile (m = -inf); same in both halves
+                if (raise) {
+                    alpha = fast_exp2(m - m_tile);
+                    m = m_tile;
+                }
+                const float neg_m = (m == -INFINITY) ? 0.f : -m;   // a fully masked row keeps p = 0
+                float sum[4] = {0.f, 0.f, 0.f, 0.f};
+                uint32_t packed[32];
+#pragma unroll
+                for (int e = 0; e < 32; ++e) {
+                    const float p0 = fast_exp2(fmaf(sv[2 * e], c_scale, neg_m));
+                    const float p1 = fast_exp2(fmaf(sv[2 * e + 1], c_scale, neg_m));
+                    sum[e & 3] += p0 + p1;
+                    packed[e] = pack_bf16x2(p0, p1);
+                }
+                l = l * alpha + ((sum[0] + sum[1]) + (sum[2] + sum[3]));
+                // P_j (bf16 pairs): this thread's 64 keys = packed columns [32 half, 32 half + 32) of S_j
+                ptx::tmem_st32(s_tmem + half * 32, packed);
+                if (j > 0) {
+                    // Every completion of o_done is waited for, in order, whether or not O has to be
+                    // rescaled: a parity wait is only meaningful one phase at a time, and the
+                    // epilogue's wait below must not find the barrier two phases behind.
+                    ok = __all_sync(0xffffffffu, ptx::mbar_wait(o_done, (tj - 1) & 1, abort_flag));
+                    if (!ok) break;
+                    if (__any_sync(0xffffffffu, raise)) {
+                        ptx::tc_fence_after_sync();
 #pragma unroll 1
-            for (int ch = 0; ch < kSlice / 32; ++ch) {
+                        for (int ch = 0; ch < 4; ++ch) {     // this thread's 128 of the 256 output columns
+                            uint32_t r[32];
+                            ptx::tmem_ld32(tmem_o + lane_base + half * 128 + ch * 32, r);
+                            ptx::tmem_wait_ld();
+#pragma unroll
+                            for (int e = 0; e < 32; ++e) r[e] = __float_as_uint(__uint_as_float(r[e]) * alpha);
+                            ptx::tmem_st32(tmem_o + lane_base + half * 128 + ch * 32, r);
+                        }
+                    }
+                }
+                ptx::tmem_wait_st();
+                ptx::tc_fence_before_sync();
+                ptx::mbar_arrive(&p_full[tj & 1]);
+            }
+            if (!ok) break;
+            // ---- item epilogue: whole row sum, normalise, store this thread's 128 columns
+            float* xs = xchg + (tj & 1) * 256 + quarter * 64;   // tj already points past the item: next parity
+            xs[half * 32 + lane] = l;
+            pair_sync(quarter);
+            const float inv_l = 1.f / (l + xs[(half ^ 1) * 32 + lane]);
+            ok = __all_sync(0xffffffffu, ptx::mbar_wait(o_done, (tj - 1) & 1, abort_flag));
+            if (!ok) break;
+            ptx::tc_fence_after_sync();
+            __nv_bfloat16* o_row = o_lat + (((size_t)w.b * d.n_q + w.g) * d.N + (t < d.N ? t : 0)) * d.d_l +
+                                   w.slice * kSlice + half * 128;
+#pragma unroll 1
+            for (int ch = 0; ch < 4; ++ch) {
                 uint32_t r[32];
-                ptx::tmem_ld32(tmem_o + lane_base + ch * 32, r);
+                ptx::tmem_ld32(tmem_o + lane_base + half * 128 + ch * 32, r);
                 ptx::tmem_wait_ld();
                 if (t < d.N) {
                     uint4* dst = reinterpret_cast<uint4*>(o_row + ch * 32);
 #pragma unroll
                     for (int v = 0; v < 4; ++v) {
-                        uint32_t w[4];
+                        uint32_t ww[4];
 #pragma unroll
                         for (int e = 0; e < 4; ++e)
-                            w[e] = pack_bf16x2(__uint_as_float(r[8 * v + 2 * e]) * inv_l,
-                                               __uint_as_float(r[8 * v + 2 * e + 1]) * inv_l);
-                        dst[v] = make_uint4(w[0], w[1], w[2], w[3]);
+                            ww[e] = pack_bf16x2(__uint_as_float(r[8 * v + 2 * e]) * inv_l,
+                                                __uint_as_float(r[8 * v + 2 * e + 1]) * inv_l);
+                        dst[v] = make_uint4(ww[0], ww[1], ww[2], ww[3]);
                     }
                 }
             }
+            ptx::tc_fence_before_sync();
+            ptx::mbar_arrive(o_free);
+            pair_sync(quarter);   // the exchange slot may be rewritten by the next tile of the same parity
         }
     }
     ptx::tc_fence_before_sync();
@@ -298,9 +370,14 @@ gta_status_t launch_sm100_prefill(const Dims& d, const void* q, const void* k, c
                                  (int)kAttnSmemTotal) != cudaSuccess)
             return GTA_ERR_CUDA;
         const int n_qt = (d.N + 127) / 128;
-        const long long n_cta = (long long)n_qt * (d.d_l / kSlice) * d.n_q * d.B;
-        if (n_cta > 0x7fffffffLL) return GTA_ERR_UNSUPPORTED;
-        sm100_attention_kernel<<<(unsigned)n_cta, kAttnThreads, kAttnSmemTotal, stream>>>(
+        const long long n_items = (long long)n_qt * (d.d_l / kSlice) * d.n_q * d.B;
+        if (n_items > 0x3fffffffLL) return GTA_ERR_UNSUPPORTED;
+        int dev = 0, sms = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
+            return GTA_ERR_CUDA;
+        const unsigned n_cta = (unsigned)(n_items < sms ? n_items : sms);
+        sm100_attention_kernel<<<n_cta, kAttnThreads, kAttnSmemTotal, stream>>>(
             tm_q, tm_k, tm_c, d, (__nv_bfloat16*)workspace, status_word);
         if (cudaGetLastError() != cudaSuccess) return GTA_ERR_CUDA;
         *launches += 1;
