@@ -1,12 +1,17 @@
 // tcgen05 / TMA decoder + gate kernel of the bf16 prefill path (d_h = 128):
 //     out_i = (L_{q(i)} W_P,i) (.) sigmoid(X W_G,i)          (Sec. 3.3, reformulated equation)
 //
-// Persistent: one CTA per SM walks a static list of work items.  An item is a tile of 128 token
-// rows x two heads of one attention map (256 output columns); what does not divide evenly over the
-// CTAs is cut into single-head items (128 columns) so that the last wave is short.  Roles:
-//   warp 0      TMA producer: 4-stage ring of {A tile 128 x 64, B tile 64 x NT}, gate operands
-//               (X, W_G) first, then decoder operands (L, W_P); it runs ahead into the next item.
-//   warp 1      tcgen05.mma issuer: acc_G (K = H) then acc_P (K = d_l), side by side in TMEM.
+// Persistent CTA pairs (clusters of 2, tcgen05 cta_group::2): a pair walks a static list of work
+// items.  An item is a tile of 256 token rows x two heads of one attention map (256 output
+// columns): each CTA of the pair owns 128 of the rows and stages its own A rows plus HALF of the
+// item's weight columns, so a weight tile crosses L2 -> shared memory once per 256 rows.  What
+// does not divide evenly over the pairs is cut into single-head items (128 columns) so that the
+// last wave is short.  Roles in each CTA:
+//   warp 0      TMA producer: 6-stage ring of {A tile 128 x 64, B tile 64 x NT/2}, gate operands
+//               (X, W_G) first, then decoder operands (L, W_P); byte counts of both CTAs go to the
+//               leader's barrier; it runs ahead into the next item.
+//   warp 1      (leader CTA only) tcgen05.mma issuer, M = 256: acc_G (K = H) then acc_P (K = d_l),
+//               side by side in each CTA's TMEM; completions are multicast to both CTAs' barriers.
 //   warps 2-9   epilogue, two warps per TMEM lane quarter (one per head): as soon as acc_G is
 //               complete they turn it into sigmoid gates held in registers (packed bf16) and hand
 //               the columns back, so the MUFU work hides under the acc_P MMAs; when acc_P is
@@ -22,13 +27,13 @@ namespace gta {
 
 namespace {
 
-constexpr int kDecStages = 4;
+constexpr int kDecStages = 6;
 constexpr int kDecThreads = 320;
-constexpr int kTileM = 128;        // token rows per item
+constexpr int kTileM = 128;        // token rows per CTA and item
 constexpr int kBlockK = 64;        // K elements per pipeline stage (one 128-byte swizzle row)
 constexpr uint32_t kATileBytes = kTileM * kBlockK * 2;   // 16 KB
 constexpr uint32_t kBGroupBytes = kBlockK * 64 * 2;      // 64 K-rows x 64 columns = 8 KB
-constexpr uint32_t kStageBytes = kATileBytes + 4 * kBGroupBytes;   // 48 KB
+constexpr uint32_t kStageBytes = kATileBytes + 2 * kBGroupBytes;   // 32 KB per CTA
 constexpr uint32_t kBarOffset = kDecStages * kStageBytes;
 constexpr uint32_t kDecSmemTotal = kBarOffset + 256 + 1024;        // barriers + alignment slack
 
@@ -43,35 +48,35 @@ __device__ __forceinline__ float sigmoid_tanh(float z) {
     return fmaf(0.5f, t, 0.5f);
 }
 
-// Static schedule.  U units (128 rows x head pair, or x single head when a map has an odd number
-// of heads) over G CTAs: every CTA takes q = U / G whole units; the r = U mod G left over are cut
-// in two single-head halves when that makes the tail shorter (2 r <= G), else handed out whole.
+// Static schedule.  U units (256 rows x head pair, or x single head when a map has an odd number
+// of heads) over G CTA pairs: every pair takes q = U / G whole units; the r = U mod G left over are
+// cut in two single-head halves when that makes the tail shorter (2 r <= G), else handed out whole.
 struct Schedule {
     int n_hp;       // units per row tile (head pairs, or heads)
     int pair;       // 1: a unit is two heads
-    int RT;         // row tiles per sequence
+    int RT;         // 256-row tiles per sequence
     int q, r, split_tail;
 };
 
 struct Item {
-    int b, t0, i0, nt;   // batch entry, first token row, first head, columns (128 or 256)
+    int b, t0, i0, nt;   // batch entry, first token row (of the pair), first head, columns (128 or 256)
 };
 
-__device__ __forceinline__ int items_of_cta(const Schedule& s, int cta, int G) {
-    if (s.split_tail) return s.q + ((cta < 2 * s.r) ? 1 : 0);
-    return s.q + ((cta < s.r) ? 1 : 0);
+__device__ __forceinline__ int items_of_pair(const Schedule& s, int pr) {
+    if (s.split_tail) return s.q + ((pr < 2 * s.r) ? 1 : 0);
+    return s.q + ((pr < s.r) ? 1 : 0);
 }
 
-__device__ __forceinline__ Item item_of(const Schedule& s, int cta, int G, int n) {
+__device__ __forceinline__ Item item_of(const Schedule& s, int pr, int G, int n) {
     int u, half = -1;
-    if (n < s.q) u = cta * s.q + n;
-    else if (s.split_tail) { u = G * s.q + (cta >> 1); half = cta & 1; }
-    else u = G * s.q + cta;
+    if (n < s.q) u = pr * s.q + n;
+    else if (s.split_tail) { u = G * s.q + (pr >> 1); half = pr & 1; }
+    else u = G * s.q + pr;
     Item it;
     const int hp = u % s.n_hp;
     const int rt = (u / s.n_hp) % s.RT;
     it.b = u / (s.n_hp * s.RT);
-    it.t0 = rt * kTileM;
+    it.t0 = rt * 2 * kTileM;
     if (s.pair) {
         it.i0 = 2 * hp + (half < 0 ? 0 : half);
         it.nt = half < 0 ? 256 : 128;
@@ -88,34 +93,37 @@ sm100_decoder_kernel(const __grid_constant__ CUtensorMap tm_l, const __grid_cons
                      Dims d, Schedule sch, __nv_bfloat16* __restrict__ out, int32_t* status_word) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-    uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + kBarOffset);
-    uint64_t* empty_bar = full_bar + kDecStages;
-    uint64_t* accg_full = empty_bar + kDecStages;
-    uint64_t* accg_free = accg_full + 1;
-    uint64_t* accp_full = accg_free + 1;
-    uint64_t* accp_free = accp_full + 1;
+    uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + kBarOffset);   // used in the leader CTA
+    uint64_t* empty_bar = full_bar + kDecStages;                             // both CTAs
+    uint64_t* accg_full = empty_bar + kDecStages;                            // both CTAs
+    uint64_t* accp_full = accg_full + 1;                                     // both CTAs
+    uint64_t* accg_free = accp_full + 1;                                     // leader CTA: 16 warps arrive
+    uint64_t* accp_free = accg_free + 1;                                     // leader CTA
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(accp_free + 1);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
     volatile int* drain_flag = abort_flag + 1;   // never raised: lets the drain wait run to its limit
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int G = gridDim.x, cta = blockIdx.x;
-    const int n_items = items_of_cta(sch, cta, G);
+    const uint32_t rank = ptx::cluster_ctarank();          // 0 = leader
+    const int G = gridDim.x >> 1, pr = blockIdx.x >> 1;    // CTA pairs, this pair
+    const int n_items = items_of_pair(sch, pr);
     const int ks_g = d.H / kBlockK, ks_p = d.d_l / kBlockK, ks_total = ks_g + ks_p;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < kDecStages; ++s) { ptx::mbar_init(&full_bar[s], 1); ptx::mbar_init(&empty_bar[s], 1); }
+        for (int s = 0; s < kDecStages; ++s) { ptx::mbar_init(&full_bar[s], 2); ptx::mbar_init(&empty_bar[s], 1); }
         ptx::mbar_init(accg_full, 1);
-        ptx::mbar_init(accg_free, 8);
         ptx::mbar_init(accp_full, 1);
-        ptx::mbar_init(accp_free, 8);
+        ptx::mbar_init(accg_free, 16);
+        ptx::mbar_init(accp_free, 16);
         *abort_flag = 0;
         *drain_flag = 0;
         ptx::fence_mbar_init();
     }
-    if (warp == 1) ptx::tmem_alloc(tmem_slot, 512);
+    if (warp == 1) ptx::tmem_alloc_pair(tmem_slot, 512);
     ptx::tc_fence_before_sync();
     __syncthreads();
+    ptx::cluster_arrive();     // the peer's barriers exist before anything is signalled to them
+    ptx::cluster_wait();
     ptx::tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
     const uint32_t tmem_p = tmem_base, tmem_g = tmem_base + 256;
@@ -127,9 +135,12 @@ sm100_decoder_kernel(const __grid_constant__ CUtensorMap tm_l, const __grid_cons
             int it = 0;            // ring iteration, runs on across items
             bool ok = true;
             for (int n = 0; n < n_items && ok; ++n) {
-                const Item w = item_of(sch, cta, G, n);
+                const Item w = item_of(sch, pr, G, n);
+                const int t0 = w.t0 + (int)rank * kTileM;          // this CTA's rows
+                const int n_grp = w.nt / 128;                      // 64-column groups of this CTA's weight half
+                const int col0 = (int)rank * (w.nt / 2);           // first of this CTA's columns inside the item
+                const int head = w.i0 + col0 / 128, hcol = col0 % 128;
                 const int g = d.head_to_q(w.i0);
-                const int n_grp = w.nt / 64;
                 const uint32_t tx = kATileBytes + (uint32_t)n_grp * kBGroupBytes;
                 for (int ks = 0; ks < ks_total; ++ks, ++it) {
                     const int s = it % kDecStages;
@@ -138,22 +149,23 @@ sm100_decoder_kernel(const __grid_constant__ CUtensorMap tm_l, const __grid_cons
                     if (!ok) break;
                     uint8_t* a_s = smem + s * kStageBytes;
                     uint8_t* b_s = a_s + kATileBytes;
-                    ptx::mbar_arrive_expect_tx(&full_bar[s], tx);
+                    const uint32_t bar = ptx::map_to_cta(ptx::smem_addr(&full_bar[s]), 0);   // the leader's
+                    ptx::mbar_arrive_expect_tx_cluster(bar, tx);
                     if (ks < ks_g) {
-                        ptx::tma_load_3d(a_s, &tm_x, &full_bar[s], ks * kBlockK, w.t0, w.b);
+                        ptx::tma_load_3d_pair(a_s, &tm_x, bar, ks * kBlockK, t0, w.b);
                         for (int grp = 0; grp < n_grp; ++grp)
-                            ptx::tma_load_2d(b_s + grp * kBGroupBytes, &tm_wg, &full_bar[s], w.i0 * 128 + grp * 64,
-                                             ks * kBlockK);
+                            ptx::tma_load_2d_pair(b_s + grp * kBGroupBytes, &tm_wg, bar, head * 128 + hcol + grp * 64,
+                                                  ks * kBlockK);
                     } else {
                         const int kk = ks - ks_g;
-                        ptx::tma_load_3d(a_s, &tm_l, &full_bar[s], kk * kBlockK, w.t0, w.b * d.n_q + g);
+                        ptx::tma_load_3d_pair(a_s, &tm_l, bar, kk * kBlockK, t0, w.b * d.n_q + g);
                         for (int grp = 0; grp < n_grp; ++grp)
-                            ptx::tma_load_3d(b_s + grp * kBGroupBytes, &tm_wp, &full_bar[s], (grp & 1) * 64,
-                                             kk * kBlockK, w.i0 + (grp >> 1));
+                            ptx::tma_load_3d_pair(b_s + grp * kBGroupBytes, &tm_wp, bar, hcol + grp * 64, kk * kBlockK,
+                                                  head);
                     }
                 }
             }
-            if (*abort_flag) {   // drain: every armed stage either lands or the wait gives up
+            if (*abort_flag && rank == 0) {   // drain: every armed stage either lands or the wait gives up
                 for (int back = 1; back <= kDecStages && it - back >= 0; ++back) {
                     const int kq = it - back;
                     ptx::mbar_wait(&full_bar[kq % kDecStages], (kq / kDecStages) & 1, drain_flag);
@@ -161,14 +173,14 @@ sm100_decoder_kernel(const __grid_constant__ CUtensorMap tm_l, const __grid_cons
             }
         }
     } else if (warp == 1) {
-        if (ptx::elect_one()) {
+        if (rank == 0 && ptx::elect_one()) {
             int it = 0;
             bool ok = true;
             for (int n = 0; n < n_items && ok; ++n) {
-                const Item w = item_of(sch, cta, G, n);
-                const uint32_t idesc = ptx::make_idesc_bf16(kTileM, w.nt, 0, 1);   // A K-major, B MN-major
+                const Item w = item_of(sch, pr, G, n);
+                const uint32_t idesc = ptx::make_idesc_bf16(2 * kTileM, w.nt, 0, 1);   // A K-major, B MN-major
                 for (int ks = 0; ks < ks_total; ++ks, ++it) {
-                    // the accumulator about to be overwritten must have been read by the epilogue
+                    // the accumulator about to be overwritten must have been read by both epilogues
                     if (ks == 0) ok = ptx::mbar_wait(accg_free, (n & 1) ^ 1, abort_flag);
                     else if (ks == ks_g) ok = ptx::mbar_wait(accp_free, (n & 1) ^ 1, abort_flag);
                     if (!ok) break;
@@ -185,11 +197,11 @@ sm100_decoder_kernel(const __grid_constant__ CUtensorMap tm_l, const __grid_cons
                     for (int k4 = 0; k4 < kBlockK / 16; ++k4) {
                         const uint64_t a_desc = ptx::make_smem_desc(a_addr + k4 * 32, 16, 1024);
                         const uint64_t b_desc = ptx::make_smem_desc(b_addr + k4 * 16 * 128, 64 * 128, 1024);
-                        ptx::mma_ss(d_tmem, a_desc, b_desc, idesc, (first && k4 == 0) ? 0u : 1u);
+                        ptx::mma_ss_pair(d_tmem, a_desc, b_desc, idesc, (first && k4 == 0) ? 0u : 1u);
                     }
-                    ptx::tc_commit(&empty_bar[s]);
-                    if (ks == ks_g - 1) ptx::tc_commit(accg_full);
-                    if (ks == ks_total - 1) ptx::tc_commit(accp_full);
+                    ptx::tc_commit_pair(&empty_bar[s], 3);
+                    if (ks == ks_g - 1) ptx::tc_commit_pair(accg_full, 3);
+                    if (ks == ks_total - 1) ptx::tc_commit_pair(accp_full, 3);
                 }
             }
         }
@@ -200,12 +212,14 @@ sm100_decoder_kernel(const __grid_constant__ CUtensorMap tm_l, const __grid_cons
         const int half = (warp - 2) >> 2;
         const int row = quarter * 32 + lane;
         const uint32_t lane_base = ((uint32_t)(quarter * 32) << 16);
+        const uint32_t accg_free_leader = ptx::map_to_cta(ptx::smem_addr(accg_free), 0);
+        const uint32_t accp_free_leader = ptx::map_to_cta(ptx::smem_addr(accp_free), 0);
         bool ok = true;
         for (int n = 0; n < n_items && ok; ++n) {
-            const Item w = item_of(sch, cta, G, n);
+            const Item w = item_of(sch, pr, G, n);
             const int cols = w.nt / 2;               // this warp's columns: 128 or 64
             const int c0 = half * cols;
-            const int t = w.t0 + row;
+            const int t = w.t0 + (int)rank * kTileM + row;
             uint32_t gate[64];                       // sigmoid gates, packed bf16 pairs
             ok = __all_sync(0xffffffffu, ptx::mbar_wait(accg_full, n & 1, abort_flag));
             if (!ok) break;
@@ -224,7 +238,7 @@ sm100_decoder_kernel(const __grid_constant__ CUtensorMap tm_l, const __grid_cons
             }
             ptx::tc_fence_before_sync();
             __syncwarp();
-            if (lane == 0) ptx::mbar_arrive(accg_free);
+            if (lane == 0) ptx::mbar_arrive_cluster(accg_free_leader);
 
             ok = __all_sync(0xffffffffu, ptx::mbar_wait(accp_full, n & 1, abort_flag));
             if (!ok) break;
@@ -254,12 +268,14 @@ sm100_decoder_kernel(const __grid_constant__ CUtensorMap tm_l, const __grid_cons
             }
             ptx::tc_fence_before_sync();
             __syncwarp();
-            if (lane == 0) ptx::mbar_arrive(accp_free);
+            if (lane == 0) ptx::mbar_arrive_cluster(accp_free_leader);
         }
     }
     ptx::tc_fence_before_sync();
     __syncthreads();
-    if (warp == 1) ptx::tmem_dealloc(tmem_base, 512);
+    ptx::cluster_arrive();     // neither CTA leaves (or frees TMEM) while the other may still signal it
+    ptx::cluster_wait();
+    if (warp == 1) ptx::tmem_dealloc_pair(tmem_base, 512);
     if (threadIdx.x == 0 && *abort_flag) raise_status(status_word, GTA_ERR_TIMEOUT);
 }
 
@@ -302,19 +318,44 @@ gta_status_t launch_sm100_decoder(const Dims& d, const void* l_bf16, const void*
     Schedule s;
     s.pair = (d.n_h / d.n_q) % 2 == 0 ? 1 : 0;
     s.n_hp = s.pair ? d.n_h / 2 : d.n_h;
-    s.RT = (d.N + kTileM - 1) / kTileM;
+    s.RT = (d.N + 2 * kTileM - 1) / (2 * kTileM);
     const long long U = (long long)d.B * s.RT * s.n_hp;
     if (U > 0x3fffffffLL) return GTA_ERR_UNSUPPORTED;
-    const int sms = sm_count();
-    const int G = U < sms ? (int)U : sms;
-    s.q = (int)(U / G);
-    s.r = (int)(U % G);
-    s.split_tail = (s.pair && 2 * s.r <= G) ? 1 : 0;
     if (cudaFuncSetAttribute(sm100_decoder_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)kDecSmemTotal) != cudaSuccess)
         return GTA_ERR_CUDA;
-    sm100_decoder_kernel<<<G, kDecThreads, kDecSmemTotal, stream>>>(tm_l, tm_x, tm_wp, tm_wg, d, s,
-                                                                    (__nv_bfloat16*)out, status_word);
+    cudaLaunchConfig_t cfg = {};
+    cfg.blockDim = dim3(kDecThreads);
+    cfg.dynamicSmemBytes = kDecSmemTotal;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    // A persistent grid must be resident at once: as many pairs as the device can hold (not every
+    // pair of SMs can host a cluster), asked once per device.
+    static thread_local int cached_dev = -1, cached_pairs = 0;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return GTA_ERR_CUDA;
+    if (dev != cached_dev) {
+        cfg.gridDim = dim3(2 * (sm_count() / 2));
+        int n = 0;
+        if (cudaOccupancyMaxActiveClusters(&n, sm100_decoder_kernel, &cfg) != cudaSuccess || n < 1) return GTA_ERR_CUDA;
+        cached_dev = dev;
+        cached_pairs = n;
+    }
+    const int pairs = cached_pairs;
+    const int G = U < pairs ? (int)U : pairs;
+    s.q = (int)(U / G);
+    s.r = (int)(U % G);
+    s.split_tail = (s.pair && 2 * s.r <= G) ? 1 : 0;
+    cfg.gridDim = dim3(2 * G);
+    if (cudaLaunchKernelEx(&cfg, sm100_decoder_kernel, tm_l, tm_x, tm_wp, tm_wg, d, s, (__nv_bfloat16*)out,
+                           status_word) != cudaSuccess)
+        return GTA_ERR_CUDA;
     return cudaGetLastError() == cudaSuccess ? GTA_OK : GTA_ERR_CUDA;
 }
 
