@@ -18,29 +18,32 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
 }
 
 // --------------------------------------------------------------------------- attention kernel
-// A work item = one 128-row query tile of one attention map x one 256-column slice of the latent
-// (the 128 x d_l fp32 output does not fit the 512 TMEM columns next to the score tiles, so d_l is
-// cut in slices of 256 and each slice item recomputes the scores).  Persistent: one CTA per SM
-// walks a static list of items, heaviest (latest) query tiles first, dealt to the CTAs in snake
-// order so that every CTA gets about the same number of key tiles.  Per 128-key tile j:
-//   S_j = Q K_j^T            tcgen05.mma, smem x smem -> TMEM (two S buffers, ping-pong)
-//   P_j = exp2(S_j c - m)    256 softmax threads, two per row (64 keys each, row maximum exchanged
-//                            through shared memory); P_j (bf16) overwrites S_j in TMEM
-//   O  += P_j C_j            tcgen05.mma, TMEM x smem (C is the MN-major B operand) -> TMEM
+// A work item = two adjacent 128-row query tiles of one attention map x one 256-column slice of
+// the latent, run by a CTA pair (cluster of 2, tcgen05 cta_group::2): each CTA owns one query tile
+// (its own S / P / O in its own TMEM) and stages HALF of every key tile (64 of the 128 keys for
+// S = Q K^T, 128 of the 256 latent columns for O += P C), so K and C cross L2 -> shared memory once
+// per 256 query rows and the ring is four key tiles deep.  (The 128 x d_l fp32 output does not fit
+// the 512 TMEM columns next to the score tiles, so d_l is cut in slices of 256 and each slice item
+// recomputes the scores.)  Persistent: a pair walks a static list of items, heaviest (latest)
+// query tiles first, dealt to the pairs in snake order.  Per 128-key tile j:
+//   S_j = Q K_j^T            tcgen05.mma M = 256, smem x smem -> TMEM (two S buffers, ping-pong)
+//   P_j = exp2(S_j c - m)    256 softmax threads per CTA, two per row (64 keys each, row maximum
+//                            exchanged through shared memory); P_j (bf16) overwrites S_j in TMEM
+//   O  += P_j C_j            tcgen05.mma M = 256, TMEM x smem (C is the MN-major B operand) -> TMEM
 // The running maximum is only raised when it grows by more than 2^8 (the accumulators stay in
 // range and O needs rescaling on few tiles); O is divided by the row sum at the end and written
-// as bf16 to L[B, n_q, N, d_l].  The K / C ring and the score pipeline run on across items: the
-// next item's Q is requested as soon as the last QK^T of the current item has been issued, and
-// its first score tile is computed while the current item's output is being stored.
+// as bf16 to L[B, n_q, N, d_l].  The ring and the score pipeline run on across items.  The lower
+// query tile of a pair sees one fully masked key tile per item (its probabilities are zero).
 constexpr int kAttnThreads = 320;
+constexpr int kAttnStages = 4;
 constexpr int kKeyTile = 128;
 constexpr int kSlice = 256;
-constexpr uint32_t kQBytes = 128 * 128 * 2;            // 32 KB
-constexpr uint32_t kKStageBytes = kKeyTile * 128 * 2;  // 32 KB
-constexpr uint32_t kCStageBytes = kKeyTile * kSlice * 2;  // 64 KB
-constexpr uint32_t kAttnKOff = kQBytes;
-constexpr uint32_t kAttnCOff = kAttnKOff + 2 * kKStageBytes;
-constexpr uint32_t kAttnXchgOff = kAttnCOff + 2 * kCStageBytes;          // float [2][4][2][32]
+constexpr uint32_t kQBytes = 128 * 128 * 2;                 // 32 KB: this CTA's query tile
+constexpr uint32_t kKHalfBytes = (kKeyTile / 2) * 128 * 2;  // 16 KB: this CTA's 64 keys
+constexpr uint32_t kCHalfBytes = kKeyTile * (kSlice / 2) * 2;   // 32 KB: this CTA's 128 latent columns
+constexpr uint32_t kAttnStageBytes = kKHalfBytes + kCHalfBytes;   // 48 KB
+constexpr uint32_t kAttnRingOff = kQBytes;
+constexpr uint32_t kAttnXchgOff = kAttnRingOff + kAttnStages * kAttnStageBytes;   // float [2][4][2][32]
 constexpr uint32_t kAttnBarOff = kAttnXchgOff + 2 * 4 * 2 * 32 * 4;
 constexpr uint32_t kAttnAlignSlack = 768;   // the 227 KB limit leaves no more; checked in the kernel
 constexpr uint32_t kAttnSmemTotal = kAttnBarOff + 256 + kAttnAlignSlack;
@@ -51,26 +54,39 @@ __device__ __forceinline__ float fast_exp2(float x) {
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
+// 2^x on the FMA pipe (x <= ~8; anything below -126 gives ~1e-38): round to the nearest integer with
+// the 1.5 * 2^23 trick, cubic for the fraction in [-1/2, 1/2] (relative error < 8e-5, well inside the
+// bf16 rounding of P), exponent patched in with integer arithmetic.  Used for one element in four so
+// that the MUFU unit, which paces the exponential phase, carries three quarters of them.
+__device__ __forceinline__ float poly_exp2(float x) {
+    x = fmaxf(x, -126.f);
+    const float t = x + 12582912.f;
+    const float f = x - (t - 12582912.f);
+    float p = fmaf(f, 0.05517165f, 0.24261113f);
+    p = fmaf(f, p, 0.69326097f);
+    p = fmaf(f, p, 0.99992806f);
+    return __int_as_float(__float_as_int(p) + (__float_as_int(t) << 23));
+}
 __device__ __forceinline__ void pair_sync(int quarter) {   // the two softmax warps of a TMEM lane quarter
     asm volatile("bar.sync %0, 64;" ::"r"(quarter + 1) : "memory");
 }
 
 struct AttnItem {
-    int b, g, slice, qi, n_tiles;
+    int b, g, slice, qp, n_tiles;   // qp: pair of query tiles (2 qp, 2 qp + 1)
 };
 
-// Item `n` of CTA `cta`: position p in the list sorted by descending query tile, rounds dealt
+// Item `n` of CTA pair `pr`: position p in the list sorted by descending query tile, rounds dealt
 // alternately left-to-right and right-to-left.  Returns false past the end of the list.
-__device__ __forceinline__ bool attn_item(const Dims& d, int n_qt, int n_slices, long long total, int G, int cta,
-                                          int n, AttnItem* it) {
-    const long long p = (long long)n * G + ((n & 1) ? (G - 1 - cta) : cta);
+__device__ __forceinline__ bool attn_item(const Dims& d, int n_qt, int n_qp, int n_slices, long long total, int G,
+                                          int pr, int n, AttnItem* it) {
+    const long long p = (long long)n * G + ((n & 1) ? (G - 1 - pr) : pr);
     if (p >= total) return false;
     long long r = p;
     it->slice = (int)(r % n_slices); r /= n_slices;
     it->g = (int)(r % d.n_q); r /= d.n_q;
     it->b = (int)(r % d.B); r /= d.B;
-    it->qi = n_qt - 1 - (int)r;
-    it->n_tiles = d.causal ? it->qi + 1 : n_qt;
+    it->qp = n_qp - 1 - (int)r;
+    it->n_tiles = d.causal ? min(2 * it->qp + 2, n_qt) : n_qt;
     return true;
 }
 
@@ -82,47 +98,43 @@ sm100_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     float* xchg = reinterpret_cast<float*>(smem + kAttnXchgOff);
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kAttnBarOff);
-    uint64_t* q_full = bars;            // 1
-    uint64_t* q_empty = bars + 1;       // 1
-    uint64_t* k_full = bars + 2;        // 2
-    uint64_t* k_empty = bars + 4;       // 2
-    uint64_t* c_full = bars + 6;        // 2
-    uint64_t* c_empty = bars + 8;       // 2
-    uint64_t* s_full = bars + 10;       // 2
-    uint64_t* p_full = bars + 12;       // 2
-    uint64_t* o_done = bars + 14;       // 1
-    uint64_t* o_free = bars + 15;       // 1
+    uint64_t* q_full = bars;            // leader CTA; both producers arrive
+    uint64_t* q_empty = bars + 1;       // both CTAs (multicast commit)
+    uint64_t* full = bars + 2;          // [4] leader CTA; both producers arrive
+    uint64_t* empty = bars + 6;         // [4] both CTAs (multicast commit)
+    uint64_t* s_full = bars + 10;       // [2] both CTAs (multicast commit)
+    uint64_t* p_full = bars + 12;       // [2] leader CTA; 16 softmax warps arrive
+    uint64_t* o_done = bars + 14;       // both CTAs (multicast commit)
+    uint64_t* o_free = bars + 15;       // leader CTA; 16 softmax warps arrive
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 16);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
     volatile int* drain_flag = abort_flag + 1;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int G = gridDim.x, cta = blockIdx.x;
-    if ((uint32_t)(smem - smem_raw) > kAttnAlignSlack) {   // uniform; cannot happen with a 256-byte aligned window
-        if (threadIdx.x == 0) raise_status(status_word, GTA_ERR_CUDA);
-        return;
-    }
+    const uint32_t rank = ptx::cluster_ctarank();          // 0 = leader
+    const int G = gridDim.x >> 1, pr = blockIdx.x >> 1;    // CTA pairs, this pair
+    const bool bad_align = (uint32_t)(smem - smem_raw) > kAttnAlignSlack;   // cannot happen with a 256-byte aligned window
     const int n_slices = d.d_l / kSlice;
-    const int n_qt = (d.N + 127) / 128;
-    const long long total = (long long)n_qt * n_slices * d.n_q * d.B;
+    const int n_qt = (d.N + 127) / 128, n_qp = (n_qt + 1) / 2;
+    const long long total = bad_align ? 0 : (long long)n_qp * n_slices * d.n_q * d.B;
 
     if (threadIdx.x == 0) {
-        ptx::mbar_init(q_full, 1);
+        ptx::mbar_init(q_full, 2);
         ptx::mbar_init(q_empty, 1);
-        for (int s = 0; s < 2; ++s) {
-            ptx::mbar_init(&k_full[s], 1); ptx::mbar_init(&k_empty[s], 1);
-            ptx::mbar_init(&c_full[s], 1); ptx::mbar_init(&c_empty[s], 1);
-            ptx::mbar_init(&s_full[s], 1); ptx::mbar_init(&p_full[s], 256);
-        }
+        for (int s = 0; s < kAttnStages; ++s) { ptx::mbar_init(&full[s], 2); ptx::mbar_init(&empty[s], 1); }
+        for (int s = 0; s < 2; ++s) { ptx::mbar_init(&s_full[s], 1); ptx::mbar_init(&p_full[s], 16); }
         ptx::mbar_init(o_done, 1);
-        ptx::mbar_init(o_free, 256);
+        ptx::mbar_init(o_free, 16);
         *abort_flag = 0;
         *drain_flag = 0;
         ptx::fence_mbar_init();
+        if (bad_align) raise_status(status_word, GTA_ERR_CUDA);
     }
-    if (warp == 1) ptx::tmem_alloc(tmem_slot, 512);
+    if (warp == 1) ptx::tmem_alloc_pair(tmem_slot, 512);
     ptx::tc_fence_before_sync();
     __syncthreads();
+    ptx::cluster_arrive();     // the peer's barriers exist before anything is signalled to them
+    ptx::cluster_wait();
     ptx::tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
     const uint32_t tmem_o = tmem_base + 256;
@@ -130,94 +142,93 @@ sm100_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     if (warp == 0) {
         if (ptx::elect_one()) {
             ptx::prefetch_tensormap(&tm_q); ptx::prefetch_tensormap(&tm_k); ptx::prefetch_tensormap(&tm_c);
+            const uint32_t q_full_leader = ptx::map_to_cta(ptx::smem_addr(q_full), 0);
             int tj = 0;                 // key tiles issued so far (ring position), across items
             bool ok = true;
-            bool q_armed = false;
             AttnItem w;
-            for (int n = 0; ok && attn_item(d, n_qt, n_slices, total, G, cta, n, &w); ++n) {
+            for (int n = 0; ok && attn_item(d, n_qt, n_qp, n_slices, total, G, pr, n, &w); ++n) {
                 const int kg = d.q_to_k(w.g), cg = d.q_to_c(w.g);
+                const int q0 = (2 * w.qp + (int)rank) * 128;       // this CTA's query rows
                 ok = ptx::mbar_wait(q_empty, (n & 1) ^ 1, abort_flag);
                 if (!ok) break;
-                ptx::mbar_arrive_expect_tx(q_full, kQBytes);
-                ptx::tma_load_3d(smem, &tm_q, q_full, 0, w.qi * 128, w.b * d.n_q + w.g);
-                ptx::tma_load_3d(smem + 16384, &tm_q, q_full, 64, w.qi * 128, w.b * d.n_q + w.g);
-                q_armed = true;
+                ptx::mbar_arrive_expect_tx_cluster(q_full_leader, kQBytes);
+                ptx::tma_load_3d_pair(smem, &tm_q, q_full_leader, 0, q0, w.b * d.n_q + w.g);
+                ptx::tma_load_3d_pair(smem + 16384, &tm_q, q_full_leader, 64, q0, w.b * d.n_q + w.g);
                 for (int j = 0; j < w.n_tiles; ++j, ++tj) {
-                    const int s = tj & 1;
-                    const uint32_t ph = (tj >> 1) & 1;
-                    ok = ptx::mbar_wait(&k_empty[s], ph ^ 1, abort_flag);
+                    const int s = tj % kAttnStages;
+                    const uint32_t ph = (tj / kAttnStages) & 1;
+                    ok = ptx::mbar_wait(&empty[s], ph ^ 1, abort_flag);
                     if (!ok) break;
-                    uint8_t* k_s = smem + kAttnKOff + s * kKStageBytes;
-                    ptx::mbar_arrive_expect_tx(&k_full[s], kKStageBytes);
-                    ptx::tma_load_3d(k_s, &tm_k, &k_full[s], 0, j * kKeyTile, w.b * d.n_k + kg);
-                    ptx::tma_load_3d(k_s + 16384, &tm_k, &k_full[s], 64, j * kKeyTile, w.b * d.n_k + kg);
-                    ok = ptx::mbar_wait(&c_empty[s], ph ^ 1, abort_flag);
-                    if (!ok) { ++tj; break; }
-                    uint8_t* c_s = smem + kAttnCOff + s * kCStageBytes;
-                    ptx::mbar_arrive_expect_tx(&c_full[s], kCStageBytes);
-#pragma unroll
-                    for (int grp = 0; grp < kSlice / 64; ++grp)
-                        ptx::tma_load_3d(c_s + grp * 16384, &tm_c, &c_full[s], w.slice * kSlice + grp * 64,
-                                         j * kKeyTile, w.b * d.n_c + cg);
+                    uint8_t* k_s = smem + kAttnRingOff + s * kAttnStageBytes;
+                    uint8_t* c_s = k_s + kKHalfBytes;
+                    const uint32_t bar = ptx::map_to_cta(ptx::smem_addr(&full[s]), 0);
+                    ptx::mbar_arrive_expect_tx_cluster(bar, kAttnStageBytes);
+                    const int key0 = j * kKeyTile + (int)rank * 64;         // this CTA's 64 keys of the tile
+                    ptx::tma_load_3d_pair(k_s, &tm_k, bar, 0, key0, w.b * d.n_k + kg);
+                    ptx::tma_load_3d_pair(k_s + 8192, &tm_k, bar, 64, key0, w.b * d.n_k + kg);
+                    const int col0 = w.slice * kSlice + (int)rank * 128;     // this CTA's 128 latent columns
+                    ptx::tma_load_3d_pair(c_s, &tm_c, bar, col0, j * kKeyTile, w.b * d.n_c + cg);
+                    ptx::tma_load_3d_pair(c_s + 16384, &tm_c, bar, col0 + 64, j * kKeyTile, w.b * d.n_c + cg);
                 }
             }
-            if (*abort_flag) {   // drain what was armed (bounded), so no copy lands after exit
-                if (q_armed) ptx::mbar_wait(q_full, 0, drain_flag), ptx::mbar_wait(q_full, 1, drain_flag);
-                for (int back = 1; back <= 2 && tj - back >= 0; ++back) {
+            if (*abort_flag && rank == 0) {   // drain what was armed (bounded), so no copy lands after exit
+                ptx::mbar_wait(q_full, 0, drain_flag);
+                ptx::mbar_wait(q_full, 1, drain_flag);
+                for (int back = 1; back <= kAttnStages && tj - back >= 0; ++back) {
                     const int jq = tj - back;
-                    ptx::mbar_wait(&k_full[jq & 1], (jq >> 1) & 1, drain_flag);
-                    ptx::mbar_wait(&c_full[jq & 1], (jq >> 1) & 1, drain_flag);
+                    ptx::mbar_wait(&full[jq % kAttnStages], (jq / kAttnStages) & 1, drain_flag);
                 }
             }
         }
     } else if (warp == 1) {
-        if (ptx::elect_one()) {
-            constexpr uint32_t idesc_qk = ptx::make_idesc_bf16(128, kKeyTile, 0, 0);   // both K-major
-            constexpr uint32_t idesc_pv = ptx::make_idesc_bf16(128, kSlice, 0, 1);     // B = C, MN-major
+        if (rank == 0 && ptx::elect_one()) {
+            constexpr uint32_t idesc_qk = ptx::make_idesc_bf16(256, kKeyTile, 0, 0);   // both K-major
+            constexpr uint32_t idesc_pv = ptx::make_idesc_bf16(256, kSlice, 0, 1);     // B = C, MN-major
             const uint32_t q_addr = ptx::smem_addr(smem);
             bool ok = true;
             // S = Q K^T of ring tile tj; `first` / `last`: first / last key tile of its item n
             auto issue_qk = [&](int tj, int n, bool first, bool last) {
                 if (first) ok = ptx::mbar_wait(q_full, n & 1, abort_flag);
-                if (ok) ok = ptx::mbar_wait(&k_full[tj & 1], (tj >> 1) & 1, abort_flag);
+                if (ok) ok = ptx::mbar_wait(&full[tj % kAttnStages], (tj / kAttnStages) & 1, abort_flag);
                 if (!ok) return;
                 ptx::tc_fence_after_sync();
-                const uint32_t k_addr = ptx::smem_addr(smem + kAttnKOff + (tj & 1) * kKStageBytes);
+                const uint32_t k_addr = ptx::smem_addr(smem + kAttnRingOff + (tj % kAttnStages) * kAttnStageBytes);
                 const uint32_t s_tmem = tmem_base + (tj & 1) * 128;
 #pragma unroll
-                for (int k8 = 0; k8 < 8; ++k8) {
-                    const uint32_t off = (k8 >> 2) * 16384 + (k8 & 3) * 32;
-                    ptx::mma_ss(s_tmem, ptx::make_smem_desc(q_addr + off, 16, 1024),
-                                ptx::make_smem_desc(k_addr + off, 16, 1024), idesc_qk, k8 ? 1u : 0u);
-                }
-                ptx::tc_commit(&s_full[tj & 1]);
-                ptx::tc_commit(&k_empty[tj & 1]);
-                if (last) ptx::tc_commit(q_empty);
+                for (int k8 = 0; k8 < 8; ++k8)
+                    ptx::mma_ss_pair(s_tmem, ptx::make_smem_desc(q_addr + (k8 >> 2) * 16384 + (k8 & 3) * 32, 16, 1024),
+                                     ptx::make_smem_desc(k_addr + (k8 >> 2) * 8192 + (k8 & 3) * 32, 16, 1024), idesc_qk,
+                                     k8 ? 1u : 0u);
+                ptx::tc_commit_pair(&s_full[tj & 1], 3);
+                if (last) ptx::tc_commit_pair(q_empty, 3);
             };
             int tj = 0;
             AttnItem w, nxt;
-            bool have = attn_item(d, n_qt, n_slices, total, G, cta, 0, &w);
+            bool have = attn_item(d, n_qt, n_qp, n_slices, total, G, pr, 0, &w);
             if (have) issue_qk(0, 0, true, w.n_tiles == 1);
             for (int n = 0; have && ok; ++n) {
-                const bool have_next = attn_item(d, n_qt, n_slices, total, G, cta, n + 1, &nxt);
+                const bool have_next = attn_item(d, n_qt, n_qp, n_slices, total, G, pr, n + 1, &nxt);
                 for (int j = 0; j < w.n_tiles && ok; ++j, ++tj) {
-                    // look ahead: the next score tile, of this item or of the next one
+                    // look ahead: the item's next score tile goes to the tensor pipe before this
+                    // tile's P C, so the softmax warps never wait for scores
                     if (j + 1 < w.n_tiles) issue_qk(tj + 1, n, false, j + 2 == w.n_tiles);
-                    else if (have_next) issue_qk(tj + 1, n + 1, true, nxt.n_tiles == 1);
                     if (!ok) break;
-                    ok = ptx::mbar_wait(&p_full[tj & 1], (tj >> 1) & 1, abort_flag) &&
-                         ptx::mbar_wait(&c_full[tj & 1], (tj >> 1) & 1, abort_flag);
+                    ok = ptx::mbar_wait(&p_full[tj & 1], (tj >> 1) & 1, abort_flag);
                     if (ok && j == 0 && n > 0) ok = ptx::mbar_wait(o_free, (n - 1) & 1, abort_flag);
                     if (!ok) break;
                     ptx::tc_fence_after_sync();
-                    const uint32_t c_addr = ptx::smem_addr(smem + kAttnCOff + (tj & 1) * kCStageBytes);
+                    const uint32_t c_addr =
+                        ptx::smem_addr(smem + kAttnRingOff + (tj % kAttnStages) * kAttnStageBytes + kKHalfBytes);
                     const uint32_t p_tmem = tmem_base + (tj & 1) * 128;
 #pragma unroll
                     for (int k8 = 0; k8 < 8; ++k8)
-                        ptx::mma_ts(tmem_o, p_tmem + k8 * 8, ptx::make_smem_desc(c_addr + k8 * 2048, 16384, 1024),
-                                    idesc_pv, (j > 0 || k8 > 0) ? 1u : 0u);
-                    ptx::tc_commit(o_done);
-                    ptx::tc_commit(&c_empty[tj & 1]);
+                        ptx::mma_ts_pair(tmem_o, p_tmem + k8 * 8, ptx::make_smem_desc(c_addr + k8 * 2048, 16384, 1024),
+                                         idesc_pv, (j > 0 || k8 > 0) ? 1u : 0u);
+                    ptx::tc_commit_pair(o_done, 3);
+                    ptx::tc_commit_pair(&empty[tj % kAttnStages], 3);
+                    // ... but the NEXT item's first score tile has to wait for that item's Q, which can
+                    // only be requested once this item's last Q K^T is done: it goes after the last P C
+                    if (j + 1 == w.n_tiles && have_next) issue_qk(tj + 1, n + 1, true, nxt.n_tiles == 1);
                 }
                 w = nxt;
                 have = have_next;
@@ -229,11 +240,14 @@ sm100_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         const int row = quarter * 32 + lane;
         const uint32_t lane_base = ((uint32_t)(quarter * 32) << 16);
         const float c_scale = d.scale * 1.4426950408889634f;
+        const uint32_t p_full_leader[2] = {ptx::map_to_cta(ptx::smem_addr(&p_full[0]), 0),
+                                           ptx::map_to_cta(ptx::smem_addr(&p_full[1]), 0)};
+        const uint32_t o_free_leader = ptx::map_to_cta(ptx::smem_addr(o_free), 0);
         bool ok = true;
         int tj = 0;
         AttnItem w;
-        for (int n = 0; ok && attn_item(d, n_qt, n_slices, total, G, cta, n, &w); ++n) {
-            const int t = w.qi * 128 + row;
+        for (int n = 0; ok && attn_item(d, n_qt, n_qp, n_slices, total, G, pr, n, &w); ++n) {
+            const int t = (2 * w.qp + (int)rank) * 128 + row;
             float m = -INFINITY, l = 0.f;            // m in scaled (log2) units; l = this thread's share of the row sum
             for (int j = 0; j < w.n_tiles && ok; ++j, ++tj) {
                 ok = __all_sync(0xffffffffu, ptx::mbar_wait(&s_full[tj & 1], (tj >> 1) & 1, abort_flag));
@@ -269,7 +283,7 @@ sm100_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                 pair_sync(quarter);
                 const float m_tile = fmaxf(m_half, xs[(half ^ 1) * 32 + lane]);
                 float alpha = 1.f;
-                const bool raise = m_tile > m + 8.f;     // also true on the first tile (m = -inf); same in both halves
+                const bool raise = m_tile > m + 8.f;     // also true on the first live tile (m = -inf); same in both halves
                 if (raise) {
                     alpha = fast_exp2(m - m_tile);
                     m = m_tile;
@@ -279,8 +293,9 @@ sm100_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                 uint32_t packed[32];
 #pragma unroll
                 for (int e = 0; e < 32; ++e) {
-                    const float p0 = fast_exp2(fmaf(sv[2 * e], c_scale, neg_m));
-                    const float p1 = fast_exp2(fmaf(sv[2 * e + 1], c_scale, neg_m));
+                    const float x0 = fmaf(sv[2 * e], c_scale, neg_m), x1 = fmaf(sv[2 * e + 1], c_scale, neg_m);
+                    const float p0 = fast_exp2(x0);
+                    const float p1 = (e & 1) ? poly_exp2(x1) : fast_exp2(x1);
                     sum[e & 3] += p0 + p1;
                     packed[e] = pack_bf16x2(p0, p1);
                 }
@@ -308,7 +323,8 @@ sm100_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                 }
                 ptx::tmem_wait_st();
                 ptx::tc_fence_before_sync();
-                ptx::mbar_arrive(&p_full[tj & 1]);
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive_cluster(p_full_leader[tj & 1]);
             }
             if (!ok) break;
             // ---- item epilogue: whole row sum, normalise, store this thread's 128 columns
@@ -327,26 +343,28 @@ sm100_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                 ptx::tmem_ld32(tmem_o + lane_base + half * 128 + ch * 32, r);
                 ptx::tmem_wait_ld();
                 if (t < d.N) {
-                    uint4* dst = reinterpret_cast<uint4*>(o_row + ch * 32);
 #pragma unroll
-                    for (int v = 0; v < 4; ++v) {
-                        uint32_t ww[4];
+                    for (int v = 0; v < 2; ++v) {      // 2 x 32 bytes: whole sectors, half as many stores
+                        uint32_t ww[8];
 #pragma unroll
-                        for (int e = 0; e < 4; ++e)
-                            ww[e] = pack_bf16x2(__uint_as_float(r[8 * v + 2 * e]) * inv_l,
-                                                __uint_as_float(r[8 * v + 2 * e + 1]) * inv_l);
-                        dst[v] = make_uint4(ww[0], ww[1], ww[2], ww[3]);
+                        for (int e = 0; e < 8; ++e)
+                            ww[e] = pack_bf16x2(__uint_as_float(r[16 * v + 2 * e]) * inv_l,
+                                                __uint_as_float(r[16 * v + 2 * e + 1]) * inv_l);
+                        ptx::st_global_256(o_row + ch * 32 + v * 16, ww);
                     }
                 }
             }
             ptx::tc_fence_before_sync();
-            ptx::mbar_arrive(o_free);
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive_cluster(o_free_leader);
             pair_sync(quarter);   // the exchange slot may be rewritten by the next tile of the same parity
         }
     }
     ptx::tc_fence_before_sync();
     __syncthreads();
-    if (warp == 1) ptx::tmem_dealloc(tmem_base, 512);
+    ptx::cluster_arrive();     // neither CTA leaves (or frees TMEM) while the other may still signal it
+    ptx::cluster_wait();
+    if (warp == 1) ptx::tmem_dealloc_pair(tmem_base, 512);
     if (threadIdx.x == 0 && *abort_flag) raise_status(status_word, GTA_ERR_TIMEOUT);
 }
 
@@ -360,25 +378,49 @@ gta_status_t launch_sm100_prefill(const Dims& d, const void* q, const void* k, c
                                   int32_t* status_word, cudaStream_t stream, int stages, int* launches) {
     if (stages & 1) {
         CUtensorMap tm_q, tm_k, tm_c;
-        const uint32_t box[3] = {64, 128, 1};
+        const uint32_t box[3] = {64, 128, 1}, box_k[3] = {64, 64, 1};
         const uint64_t dq[3] = {(uint64_t)d.d_h, (uint64_t)d.N, (uint64_t)d.B * d.n_q};
         const uint64_t dk[3] = {(uint64_t)d.d_h, (uint64_t)d.N, (uint64_t)d.B * d.n_k};
         const uint64_t dc[3] = {(uint64_t)d.d_l, (uint64_t)d.N, (uint64_t)d.B * d.n_c};
-        if (!make_bf16_map(&tm_q, q, 3, dq, box) || !make_bf16_map(&tm_k, k, 3, dk, box) || !make_bf16_map(&tm_c, c, 3, dc, box))
+        if (!make_bf16_map(&tm_q, q, 3, dq, box) || !make_bf16_map(&tm_k, k, 3, dk, box_k) ||
+            !make_bf16_map(&tm_c, c, 3, dc, box))
             return GTA_ERR_CUDA;
         if (cudaFuncSetAttribute(sm100_attention_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  (int)kAttnSmemTotal) != cudaSuccess)
             return GTA_ERR_CUDA;
-        const int n_qt = (d.N + 127) / 128;
-        const long long n_items = (long long)n_qt * (d.d_l / kSlice) * d.n_q * d.B;
+        const int n_qt = (d.N + 127) / 128, n_qp = (n_qt + 1) / 2;
+        const long long n_items = (long long)n_qp * (d.d_l / kSlice) * d.n_q * d.B;
         if (n_items > 0x3fffffffLL) return GTA_ERR_UNSUPPORTED;
+        cudaLaunchConfig_t cfg = {};
+        cfg.blockDim = dim3(kAttnThreads);
+        cfg.dynamicSmemBytes = kAttnSmemTotal;
+        cfg.stream = stream;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = 2;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        // a persistent grid must be resident at once: as many CTA pairs as the device can hold
+        static thread_local int cached_dev = -1, cached_pairs = 0;
         int dev = 0, sms = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess ||
-            cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
+        if (cudaGetDevice(&dev) != cudaSuccess) return GTA_ERR_CUDA;
+        if (dev != cached_dev) {
+            if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 2)
+                return GTA_ERR_CUDA;
+            cfg.gridDim = dim3(2 * (sms / 2));
+            int n = 0;
+            if (cudaOccupancyMaxActiveClusters(&n, sm100_attention_kernel, &cfg) != cudaSuccess || n < 1)
+                return GTA_ERR_CUDA;
+            cached_dev = dev;
+            cached_pairs = n;
+        }
+        const int pairs = (int)(n_items < cached_pairs ? n_items : cached_pairs);
+        cfg.gridDim = dim3(2 * pairs);
+        if (cudaLaunchKernelEx(&cfg, sm100_attention_kernel, tm_q, tm_k, tm_c, d, (__nv_bfloat16*)workspace,
+                               status_word) != cudaSuccess)
             return GTA_ERR_CUDA;
-        const unsigned n_cta = (unsigned)(n_items < sms ? n_items : sms);
-        sm100_attention_kernel<<<n_cta, kAttnThreads, kAttnSmemTotal, stream>>>(
-            tm_q, tm_k, tm_c, d, (__nv_bfloat16*)workspace, status_word);
         if (cudaGetLastError() != cudaSuccess) return GTA_ERR_CUDA;
         *launches += 1;
     }

@@ -259,10 +259,12 @@ sm100_decoder_kernel(const __grid_constant__ CUtensorMap tm_l, const __grid_cons
                         packed[e] = pack_bf16x2(__uint_as_float(p[2 * e]) * g0, __uint_as_float(p[2 * e + 1]) * g1);
                     }
                     if (t < d.N) {
-                        uint4* dst = reinterpret_cast<uint4*>(o_row + ch * 32);
 #pragma unroll
-                        for (int v = 0; v < 4; ++v)
-                            dst[v] = make_uint4(packed[4 * v], packed[4 * v + 1], packed[4 * v + 2], packed[4 * v + 3]);
+                        for (int v = 0; v < 2; ++v) {      // 2 x 32 bytes: whole sectors, half as many stores
+                            const uint32_t ww[8] = {packed[8 * v], packed[8 * v + 1], packed[8 * v + 2], packed[8 * v + 3],
+                                                    packed[8 * v + 4], packed[8 * v + 5], packed[8 * v + 6], packed[8 * v + 7]};
+                            ptx::st_global_256(o_row + ch * 32 + v * 16, ww);
+                        }
                     }
                 }
             }
