@@ -133,6 +133,11 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
         ptx::prefetch_tensormap(&tm_c);
     }
 
+    // This kernel is itself launched with programmatic stream serialisation: it may have been
+    // scheduled while the kernel before it in the stream (a cache append, the previous decode
+    // step) was still draining, and must not read that kernel's results (lengths, caches) earlier.
+    ptx::grid_dependency_wait();
+
     // ---- exclusive prefix sum of the sub-tile counts: prefix[b] = sum_{b' < b} ceil(len / T)
     //      (thread t owns sequences [t per, (t + 1) per); warp scan, then a scan of the warp totals)
     {
@@ -753,8 +758,19 @@ cudaError_t launch_decode_fast(const Dims& d, const void* q, const void* k_cache
             auto kern = decode_stream_kernel<NT>;                                                          \
             err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);      \
             if (err != cudaSuccess) return err;                                                            \
-            kern<<<p.G, kStreamThreads, smem, stream>>>(tm_k, tm_c, d, p.T, S_cap, (const __nv_bfloat16*)q, \
-                                                        seq_lens, part_o, part_ml, status_word);           \
+            cudaLaunchConfig_t cfg = {};                                                                   \
+            cfg.gridDim = dim3(p.G);                                                                       \
+            cfg.blockDim = dim3(kStreamThreads);                                                           \
+            cfg.dynamicSmemBytes = smem;                                                                   \
+            cfg.stream = stream;                                                                           \
+            cudaLaunchAttribute attr[1];                                                                   \
+            attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;                               \
+            attr[0].val.programmaticStreamSerializationAllowed = 1;                                        \
+            cfg.attrs = attr;                                                                              \
+            cfg.numAttrs = 1;                                                                              \
+            err = cudaLaunchKernelEx(&cfg, kern, tm_k, tm_c, d, p.T, S_cap, (const __nv_bfloat16*)q,       \
+                                     seq_lens, part_o, part_ml, status_word);                              \
+            if (err != cudaSuccess) return err;                                                            \
         } while (0)
         switch (d.d_l) {
             case 256: GTA_LAUNCH_STREAM(4); break;
