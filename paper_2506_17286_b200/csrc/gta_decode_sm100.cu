@@ -13,7 +13,9 @@
 //       d_l / 8 slice of the latent sum; one CTA barrier per sub-tile.  When the range crosses
 //       into the next sequence, and at its end, the partial (max, sum, latent sum) goes to
 //       slot c + b of the workspace.
-//   decode_finish_kernel : clusters of 4 or 8 CTAs per (head, 64-column half) split the reduction
+//   decode_merge_kernel (batches of more than 16): log-sum-exp merge of the slots into L (bf16);
+//       the tcgen05 decoder + gate kernel of the prefill path then runs with the batch as its token axis.
+//   decode_finish_kernel (small batches): clusters of 4 or 8 CTAs per (head, 64-column half) split the reduction
 //       dimensions of the decoder (d_l) and of the gate (H).  Launched with programmatic stream
 //       serialisation: while the stream kernel drains, each CTA requests its weight slice (TMA)
 //       and its hidden-state slice and works out which stream CTAs own which sequence; after the
@@ -23,6 +25,7 @@
 #include <cooperative_groups.h>
 
 #include "gta_common.cuh"
+#include "gta_sm100.cuh"
 #include "sm100_ptx.cuh"
 #include "tma_host.cuh"
 
@@ -45,8 +48,10 @@ struct FastPlan {
     int T;         // tokens per sub-tile (16, 32 or 64)
     int G;         // stream CTAs
     int slots;     // G + B partial slots
-    size_t off_ml, total;   // byte offsets in the workspace (part_o at 0)
+    size_t off_ml, off_rng, off_bound, off_l, total;   // byte offsets in the workspace (part_o at 0)
 };
+constexpr int kFinMaxBatchClusters = 16;   // larger batches finish through the merge kernel + the tcgen05 decoder kernel
+                                           // (measured: faster from 32 sequences on; the weights then feed 128-row MMAs)
 
 static size_t align256f(size_t v) { return (v + 255) & ~(size_t)255; }
 static int finish_split(const Dims& d);
@@ -82,7 +87,10 @@ static FastPlan make_fast_plan(const Dims& d) {
     const size_t part_o = (size_t)p.slots * d.n_q * d.d_l * sizeof(float);
     const size_t part_ml = (size_t)p.slots * d.n_q * 2 * sizeof(float);
     p.off_ml = align256f(part_o);
-    p.total = p.off_ml + align256f(part_ml);
+    p.off_rng = p.off_ml + align256f(part_ml);
+    p.off_bound = p.off_rng + align256f((size_t)d.B * 2 * sizeof(int32_t));
+    p.off_l = p.off_bound + align256f((size_t)(p.G + 1) * sizeof(int32_t));
+    p.total = p.off_l + align256f((size_t)d.n_q * d.B * d.d_l * sizeof(__nv_bfloat16));
     return p;
 }
 
@@ -110,7 +118,8 @@ template <int NT>   // NT = d_l / 64 = MMA n-tiles (8 latent columns each) per c
 __global__ void __launch_bounds__(kStreamThreads, 1)
 decode_stream_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_c, Dims d,
                      int T, int S_cap, const __nv_bfloat16* __restrict__ q, const int32_t* __restrict__ seq_lens,
-                     float* __restrict__ part_o, float* __restrict__ part_ml, int32_t* status_word) {
+                     float* __restrict__ part_o, float* __restrict__ part_ml, int32_t* __restrict__ rng_g,
+                     int32_t* __restrict__ bound_g, int32_t* status_word) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     uint8_t* ring = smem;                                                              // 3 x 64 KB
@@ -170,6 +179,25 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
     }
     const long long n_st = prefix[d.B];
     const long long st_begin = ((long long)cta * n_st) / G, st_end = ((long long)(cta + 1) * n_st) / G;
+    // ---- tables for the merge kernel (large batches): bound_g[c] = first sub-tile of CTA c, and for
+    //      sequence b the CTAs c_lo .. c_hi that own its sub-tiles (CTA c answers for b = c, c + G, ...).
+    //      The owner of sub-tile st is the largest c with floor(c n / G) <= st = floor(((st + 1) G - 1) / n).
+    if (rng_g != nullptr) {
+        if (tid == 0) {
+            bound_g[cta] = (int32_t)st_begin;
+            if (cta == 0) bound_g[G] = (int32_t)n_st;
+        }
+        for (int b = cta + tid * G; b < d.B; b += G * kStreamThreads) {
+            const long long s_lo = prefix[b], s_hi = prefix[b + 1];
+            int c_lo = 0, c_hi = -1;
+            if (s_hi > s_lo) {
+                c_lo = (int)(((s_lo + 1) * G - 1) / n_st);
+                c_hi = (int)((s_hi * G - 1) / n_st);
+            }
+            rng_g[2 * b] = c_lo;
+            rng_g[2 * b + 1] = c_hi;
+        }
+    }
     if (st_begin >= st_end) return;      // uniform: nothing armed
     int b0;
     {   // largest b with prefix[b] <= st_begin: a non-empty sequence, since st_begin < n_st
@@ -735,6 +763,44 @@ static int finish_split(const Dims& d) {
 }
 
 // ---------------------------------------------------------------------------------------------
+// Large batches: log-sum-exp merge of the split-KV slots of one (attention map, sequence) pair per
+// CTA into the normalised latent L[n_q][B][d_l] (bf16), which the tcgen05 decoder + gate kernel of
+// the prefill path then consumes with the batch in the role of the token axis.
+__global__ void __launch_bounds__(256)
+decode_merge_kernel(Dims d, int G, const int32_t* __restrict__ rng_g, const int32_t* __restrict__ bound_g,
+                    const float* __restrict__ part_o, const float* __restrict__ part_ml,
+                    __nv_bfloat16* __restrict__ l_out) {
+    ptx::grid_launch_dependents();
+    ptx::grid_dependency_wait();
+    const int g = blockIdx.x, b = blockIdx.y;
+    const int c_lo = rng_g[2 * b], c_hi = rng_g[2 * b + 1];
+    float M = -INFINITY, l = 0.f;
+    for (int c = c_lo; c <= c_hi; ++c)
+        if (bound_g[c] < bound_g[c + 1]) M = fmaxf(M, part_ml[((size_t)(c + b) * d.n_q + g) * 2]);
+    for (int c = c_lo; c <= c_hi; ++c)
+        if (bound_g[c] < bound_g[c + 1]) {   // a CTA with an empty range wrote nothing
+            const float* ml = part_ml + ((size_t)(c + b) * d.n_q + g) * 2;
+            l = fmaf(ml[1], ex2f(ml[0] - M), l);
+        }
+    const float inv_l = c_hi >= c_lo ? 1.f / l : 0.f;
+    for (int col = threadIdx.x * 4; col < d.d_l; col += 256 * 4) {
+        float4 sum = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int c = c_lo; c <= c_hi; ++c) {
+            if (!(bound_g[c] < bound_g[c + 1])) continue;
+            const size_t pi = (size_t)(c + b) * d.n_q + g;
+            const float w = ex2f(part_ml[pi * 2] - M) * inv_l;
+            const float4 v = *reinterpret_cast<const float4*>(part_o + pi * d.d_l + col);
+            sum.x = fmaf(v.x, w, sum.x); sum.y = fmaf(v.y, w, sum.y);
+            sum.z = fmaf(v.z, w, sum.z); sum.w = fmaf(v.w, w, sum.w);
+        }
+        uint2 packed;
+        packed.x = pack_bf16(sum.x, sum.y);
+        packed.y = pack_bf16(sum.z, sum.w);
+        *reinterpret_cast<uint2*>(l_out + ((size_t)g * d.B + b) * d.d_l + col) = packed;
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
 cudaError_t launch_decode_fast(const Dims& d, const void* q, const void* k_cache, const void* c_cache,
                                const int32_t* seq_lens, int S_cap, const void* x_t, const void* w_p,
                                const void* w_g, void* out, void* workspace, int32_t* status_word,
@@ -742,6 +808,10 @@ cudaError_t launch_decode_fast(const Dims& d, const void* q, const void* k_cache
     const FastPlan p = make_fast_plan(d);
     float* part_o = reinterpret_cast<float*>(workspace);
     float* part_ml = reinterpret_cast<float*>(static_cast<char*>(workspace) + p.off_ml);
+    int32_t* rng_g = reinterpret_cast<int32_t*>(static_cast<char*>(workspace) + p.off_rng);
+    int32_t* bound_g = reinterpret_cast<int32_t*>(static_cast<char*>(workspace) + p.off_bound);
+    __nv_bfloat16* l_g = reinterpret_cast<__nv_bfloat16*>(static_cast<char*>(workspace) + p.off_l);
+    const bool big_batch = d.B > kFinMaxBatchClusters;
     cudaError_t err;
     if (stages & 2) {
         CUtensorMap tm_k, tm_c;
@@ -769,7 +839,8 @@ cudaError_t launch_decode_fast(const Dims& d, const void* q, const void* k_cache
             cfg.attrs = attr;                                                                              \
             cfg.numAttrs = 1;                                                                              \
             err = cudaLaunchKernelEx(&cfg, kern, tm_k, tm_c, d, p.T, S_cap, (const __nv_bfloat16*)q,       \
-                                     seq_lens, part_o, part_ml, status_word);                              \
+                                     seq_lens, part_o, part_ml, big_batch ? rng_g : (int32_t*)nullptr,     \
+                                     bound_g, status_word);                                                \
             if (err != cudaSuccess) return err;                                                            \
         } while (0)
         switch (d.d_l) {
@@ -781,7 +852,26 @@ cudaError_t launch_decode_fast(const Dims& d, const void* q, const void* k_cache
         if ((err = cudaGetLastError()) != cudaSuccess) return err;
         *launches += 1;
     }
-    if (stages & 4) {
+    if ((stages & 4) && big_batch) {
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(d.n_q, d.B);
+        cfg.blockDim = dim3(256);
+        cfg.stream = stream;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        err = cudaLaunchKernelEx(&cfg, decode_merge_kernel, d, p.G, (const int32_t*)rng_g, (const int32_t*)bound_g,
+                                 (const float*)part_o, (const float*)part_ml, l_g);
+        if (err != cudaSuccess) return err;
+        // the batch takes the role of the token axis: L [n_q][B][d_l], x_t [B][H], out [B][n_h][d_h]
+        Dims dd = d;
+        dd.B = 1;
+        dd.N = d.B;
+        if (launch_sm100_decoder(dd, l_g, x_t, w_p, w_g, out, status_word, stream) != GTA_OK) return cudaErrorUnknown;
+        *launches += 2;
+    } else if (stages & 4) {
         const int S = finish_split(d);
         const int dls = d.d_l / S, hs = d.H / S, KA = dls + hs;
         CUtensorMap tm_wp, tm_wg;

@@ -113,6 +113,9 @@ sm100_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = ptx::cluster_ctarank();          // 0 = leader
     const int G = gridDim.x >> 1, pr = blockIdx.x >> 1;    // CTA pairs, this pair
+    // the decoder + gate kernel may be scheduled as SMs free up: its gate phase does not need L, and
+    // it waits for this whole grid before it reads L
+    ptx::grid_launch_dependents();
     const bool bad_align = (uint32_t)(smem - smem_raw) > kAttnAlignSlack;   // cannot happen with a 256-byte aligned window
     const int n_slices = d.d_l / kSlice;
     const int n_qt = (d.N + 127) / 128, n_qp = (n_qt + 1) / 2;

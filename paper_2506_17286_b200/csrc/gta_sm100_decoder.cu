@@ -134,6 +134,7 @@ sm100_decoder_kernel(const __grid_constant__ CUtensorMap tm_l, const __grid_cons
             ptx::prefetch_tensormap(&tm_wp); ptx::prefetch_tensormap(&tm_wg);
             int it = 0;            // ring iteration, runs on across items
             bool ok = true;
+            bool l_ready = false;
             for (int n = 0; n < n_items && ok; ++n) {
                 const Item w = item_of(sch, pr, G, n);
                 const int t0 = w.t0 + (int)rank * kTileM;          // this CTA's rows
@@ -158,6 +159,10 @@ sm100_decoder_kernel(const __grid_constant__ CUtensorMap tm_l, const __grid_cons
                                                   ks * kBlockK);
                     } else {
                         const int kk = ks - ks_g;
+                        // L comes from the kernel before this one in the stream; this kernel is
+                        // launched with programmatic serialisation, so the gate phase above (X, W_G
+                        // only) may already have run while that kernel was draining
+                        if (!l_ready) { ptx::grid_dependency_wait(); l_ready = true; }
                         ptx::tma_load_3d_pair(a_s, &tm_l, bar, kk * kBlockK, t0, w.b * d.n_q + g);
                         for (int grp = 0; grp < n_grp; ++grp)
                             ptx::tma_load_3d_pair(b_s + grp * kBGroupBytes, &tm_wp, bar, hcol + grp * 64, kk * kBlockK,
@@ -321,7 +326,7 @@ gta_status_t launch_sm100_decoder(const Dims& d, const void* l_bf16, const void*
     s.pair = (d.n_h / d.n_q) % 2 == 0 ? 1 : 0;
     s.n_hp = s.pair ? d.n_h / 2 : d.n_h;
     s.RT = (d.N + 2 * kTileM - 1) / (2 * kTileM);
-    const long long U = (long long)d.B * s.RT * s.n_hp;
+    long long U = (long long)d.B * s.RT * s.n_hp;
     if (U > 0x3fffffffLL) return GTA_ERR_UNSUPPORTED;
     if (cudaFuncSetAttribute(sm100_decoder_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)kDecSmemTotal) != cudaSuccess)
@@ -330,13 +335,15 @@ gta_status_t launch_sm100_decoder(const Dims& d, const void* l_bf16, const void*
     cfg.blockDim = dim3(kDecThreads);
     cfg.dynamicSmemBytes = kDecSmemTotal;
     cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = 2;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = 1;   // the occupancy query below takes the cluster attribute only
     // A persistent grid must be resident at once: as many pairs as the device can hold (not every
     // pair of SMs can host a cluster), asked once per device.
     static thread_local int cached_dev = -1, cached_pairs = 0;
@@ -350,11 +357,17 @@ gta_status_t launch_sm100_decoder(const Dims& d, const void* l_bf16, const void*
         cached_pairs = n;
     }
     const int pairs = cached_pairs;
+    if (s.pair && 2 * U <= pairs) {   // few units (e.g. a decode batch): single heads keep twice as many SMs busy
+        s.pair = 0;
+        s.n_hp = d.n_h;
+        U *= 2;
+    }
     const int G = U < pairs ? (int)U : pairs;
     s.q = (int)(U / G);
     s.r = (int)(U % G);
     s.split_tail = (s.pair && 2 * s.r <= G) ? 1 : 0;
     cfg.gridDim = dim3(2 * G);
+    cfg.numAttrs = 2;
     if (cudaLaunchKernelEx(&cfg, sm100_decoder_kernel, tm_l, tm_x, tm_wp, tm_wg, d, s, (__nv_bfloat16*)out,
                            status_word) != cudaSuccess)
         return GTA_ERR_CUDA;

@@ -157,6 +157,9 @@ SMALL_DECODE = [
     ("bf16_paper_1b_shape", "bf16", 2, 1280, 20, 5, 1, 1, 64, 128, [333, 1000]),
     ("bf16_eight_maps", "bf16", 9, 512, 16, 8, 8, 1, 128, 1024, [257, 256, 255, 1, 2, 1000, 64, 128, 511]),
     ("f32_general", "f32", 3, 96, 6, 6, 3, 1, 32, 64, [100, 7, 260]),
+    # more than 32 sequences: the finish goes through the merge kernel + the tensor-core decoder kernel
+    ("bf16_batch_40", "bf16", 40, 256, 8, 4, 4, 1, 128, 512, [1 + (37 * i) % 300 for i in range(40)]),
+    ("bf16_batch_33_odd_heads", "bf16", 33, 128, 3, 1, 1, 1, 128, 256, [0 if i == 5 else 1 + (91 * i) % 500 for i in range(33)]),
 ]
 
 
