@@ -27,14 +27,14 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
 // recomputes the scores.)  Persistent: a pair walks a static list of items, heaviest (latest)
 // query tiles first, dealt to the pairs in snake order.  Per 128-key tile j:
 //   S_j = Q K_j^T            tcgen05.mma M = 256, smem x smem -> TMEM (two S buffers, ping-pong)
-//   P_j = exp2(S_j c - m)    256 softmax threads per CTA, two per row (64 keys each, row maximum
+//   P_j = exp2(S_j c - m)    512 softmax threads per CTA, four per row (32 keys each, row maximum
 //                            exchanged through shared memory); P_j (bf16) overwrites S_j in TMEM
 //   O  += P_j C_j            tcgen05.mma M = 256, TMEM x smem (C is the MN-major B operand) -> TMEM
 // The running maximum is only raised when it grows by more than 2^8 (the accumulators stay in
 // range and O needs rescaling on few tiles); O is divided by the row sum at the end and written
 // as bf16 to L[B, n_q, N, d_l].  The ring and the score pipeline run on across items.  The lower
 // query tile of a pair sees one fully masked key tile per item (its probabilities are zero).
-constexpr int kAttnThreads = 320;
+constexpr int kAttnThreads = 64 + 512;   // TMA warp, MMA warp, 16 softmax warps
 constexpr int kAttnStages = 4;
 constexpr int kKeyTile = 128;
 constexpr int kSlice = 256;
@@ -43,7 +43,7 @@ constexpr uint32_t kKHalfBytes = (kKeyTile / 2) * 128 * 2;  // 16 KB: this CTA's
 constexpr uint32_t kCHalfBytes = kKeyTile * (kSlice / 2) * 2;   // 32 KB: this CTA's 128 latent columns
 constexpr uint32_t kAttnStageBytes = kKHalfBytes + kCHalfBytes;   // 48 KB
 constexpr uint32_t kAttnRingOff = kQBytes;
-constexpr uint32_t kAttnXchgOff = kAttnRingOff + kAttnStages * kAttnStageBytes;   // float [2][4][2][32]
+constexpr uint32_t kAttnXchgOff = kAttnRingOff + kAttnStages * kAttnStageBytes;   // 2 KB, per lane quarter: bf16 [2][4][32] or float [4][32]
 constexpr uint32_t kAttnBarOff = kAttnXchgOff + 2 * 4 * 2 * 32 * 4;
 constexpr uint32_t kAttnAlignSlack = 768;   // the 227 KB limit leaves no more; checked in the kernel
 constexpr uint32_t kAttnSmemTotal = kAttnBarOff + 256 + kAttnAlignSlack;
@@ -54,23 +54,31 @@ __device__ __forceinline__ float fast_exp2(float x) {
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
-// 2^x on the FMA pipe (x <= ~8; anything below -126 gives ~1e-38): round to the nearest integer with
-// the 1.5 * 2^23 trick, cubic for the fraction in [-1/2, 1/2] (relative error < 8e-5, well inside the
-// bf16 rounding of P), exponent patched in with integer arithmetic.  Used for one element in four so
-// that the MUFU unit, which paces the exponential phase, carries three quarters of them.
-__device__ __forceinline__ float poly_exp2(float x) {
-    x = fmaxf(x, -126.f);
-    const float t = x + 12582912.f;
-    const float f = x - (t - 12582912.f);
-    float p = fmaf(f, 0.05517165f, 0.24261113f);
-    p = fmaf(f, p, 0.69326097f);
-    p = fmaf(f, p, 0.99992806f);
-    return __int_as_float(__float_as_int(p) + (__float_as_int(t) << 23));
+// 2^x for a pair of values on the FMA pipe (x <= ~8; anything below -126 gives ~1e-38): round to the
+// nearest integer with the 1.5 * 2^23 trick, cubic for the fraction in [-1/2, 1/2] (relative error
+// < 8e-5, well inside the bf16 rounding of P), exponent patched in with integer arithmetic.  Used for
+// some of the pairs so that the MUFU unit, which paces the exponential phase, carries fewer of them.
+__device__ __forceinline__ void poly_exp2_pair(uint64_t x2, float& p0, float& p1) {
+    float x0, x1;
+    ptx::f32x2_split(x2, x0, x1);
+    x2 = ptx::f32x2(fmaxf(x0, -126.f), fmaxf(x1, -126.f));
+    const uint64_t t2 = ptx::add2(x2, ptx::f32x2(12582912.f, 12582912.f));
+    const uint64_t u2 = ptx::add2(t2, ptx::f32x2(-12582912.f, -12582912.f));
+    const uint64_t f2 = ptx::fma2(u2, ptx::f32x2(-1.f, -1.f), x2);
+    uint64_t q2 = ptx::fma2(f2, ptx::f32x2(0.05517165f, 0.05517165f), ptx::f32x2(0.24261113f, 0.24261113f));
+    q2 = ptx::fma2(f2, q2, ptx::f32x2(0.69326097f, 0.69326097f));
+    q2 = ptx::fma2(f2, q2, ptx::f32x2(0.99992806f, 0.99992806f));
+    float q0, q1, t0, t1;
+    ptx::f32x2_split(q2, q0, q1);
+    ptx::f32x2_split(t2, t0, t1);
+    p0 = __int_as_float(__float_as_int(q0) + (__float_as_int(t0) << 23));
+    p1 = __int_as_float(__float_as_int(q1) + (__float_as_int(t1) << 23));
 }
-__device__ __forceinline__ void pair_sync(int quarter) {   // the two softmax warps of a TMEM lane quarter
-    asm volatile("bar.sync %0, 64;" ::"r"(quarter + 1) : "memory");
+// which of every eight pairs of exponentials run on the FMA pipe instead of the MUFU unit
+__device__ constexpr bool kPolyPair[8] = {false, false, true, false, false, true, false, true};
+__device__ __forceinline__ void quarter_sync(int quarter) {   // the four softmax warps of a TMEM lane quarter
+    asm volatile("bar.sync %0, 128;" ::"r"(quarter + 1) : "memory");
 }
-
 struct AttnItem {
     int b, g, slice, qp, n_tiles;   // qp: pair of query tiles (2 qp, 2 qp + 1)
 };
@@ -103,9 +111,9 @@ sm100_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     uint64_t* full = bars + 2;          // [4] leader CTA; both producers arrive
     uint64_t* empty = bars + 6;         // [4] both CTAs (multicast commit)
     uint64_t* s_full = bars + 10;       // [2] both CTAs (multicast commit)
-    uint64_t* p_full = bars + 12;       // [2] leader CTA; 16 softmax warps arrive
+    uint64_t* p_full = bars + 12;       // [2] leader CTA; 32 softmax warps arrive
     uint64_t* o_done = bars + 14;       // both CTAs (multicast commit)
-    uint64_t* o_free = bars + 15;       // leader CTA; 16 softmax warps arrive
+    uint64_t* o_free = bars + 15;       // leader CTA; 32 softmax warps arrive
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 16);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
     volatile int* drain_flag = abort_flag + 1;
@@ -125,9 +133,9 @@ sm100_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         ptx::mbar_init(q_full, 2);
         ptx::mbar_init(q_empty, 1);
         for (int s = 0; s < kAttnStages; ++s) { ptx::mbar_init(&full[s], 2); ptx::mbar_init(&empty[s], 1); }
-        for (int s = 0; s < 2; ++s) { ptx::mbar_init(&s_full[s], 1); ptx::mbar_init(&p_full[s], 16); }
+        for (int s = 0; s < 2; ++s) { ptx::mbar_init(&s_full[s], 1); ptx::mbar_init(&p_full[s], 32); }
         ptx::mbar_init(o_done, 1);
-        ptx::mbar_init(o_free, 16);
+        ptx::mbar_init(o_free, 32);
         *abort_flag = 0;
         *drain_flag = 0;
         ptx::fence_mbar_init();
@@ -238,14 +246,19 @@ sm100_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
             }
         }
     } else {
+        // 16 softmax warps: four per TMEM lane quarter (warp % 4), each thread 32 of the 128 keys of its
+        // row and 64 of the 256 output columns.  Four warps per scheduler hide the latencies of the
+        // TMEM loads, the exchange and the exponentials behind one another.
         const int quarter = warp & 3;
-        const int half = (warp - 2) >> 2;            // which 64 keys of a tile / which 128 output columns
+        const int part = (warp - 2) >> 2;            // which 32 keys of a tile / which 64 output columns
         const int row = quarter * 32 + lane;
         const uint32_t lane_base = ((uint32_t)(quarter * 32) << 16);
         const float c_scale = d.scale * 1.4426950408889634f;
         const uint32_t p_full_leader[2] = {ptx::map_to_cta(ptx::smem_addr(&p_full[0]), 0),
                                            ptx::map_to_cta(ptx::smem_addr(&p_full[1]), 0)};
         const uint32_t o_free_leader = ptx::map_to_cta(ptx::smem_addr(o_free), 0);
+        __nv_bfloat16* xm = reinterpret_cast<__nv_bfloat16*>(xchg);   // [4 quarters][2][4][32] partial row maxima
+        float* xl = xchg + quarter * 128;                             // [4][32] partial row sums (item end)
         bool ok = true;
         int tj = 0;
         AttnItem w;
@@ -257,54 +270,65 @@ sm100_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                 if (!ok) break;   // warp-uniform: the TMEM instructions below are warp-collective
                 ptx::tc_fence_after_sync();
                 const uint32_t s_tmem = tmem_base + lane_base + (tj & 1) * 128;
-                float sv[64];
+                float sv[32];
                 {
-                    uint32_t r0[32], r1[32];
-                    ptx::tmem_ld32(s_tmem + half * 64, r0);
-                    ptx::tmem_ld32(s_tmem + half * 64 + 32, r1);
+                    uint32_t r0[32];
+                    ptx::tmem_ld32(s_tmem + part * 32, r0);
                     ptx::tmem_wait_ld();
 #pragma unroll
-                    for (int e = 0; e < 32; ++e) { sv[e] = __uint_as_float(r0[e]); sv[32 + e] = __uint_as_float(r1[e]); }
+                    for (int e = 0; e < 32; ++e) sv[e] = __uint_as_float(r0[e]);
                 }
                 // mask: keys past the sequence end, and (causal) keys after the query, on boundary tiles
-                const int key0 = j * kKeyTile + half * 64;
+                const int key0 = j * kKeyTile + part * 32;
                 const int last_key = d.causal ? min(t, d.N - 1) : d.N - 1;
-                if (key0 + 63 > last_key) {
+                if (key0 + 31 > last_key) {
 #pragma unroll
-                    for (int e = 0; e < 64; ++e)
+                    for (int e = 0; e < 32; ++e)
                         if (key0 + e > last_key) sv[e] = -INFINITY;
                 }
-                float mx[4] = {sv[0], sv[1], sv[2], sv[3]};
+                float mx[2] = {ptx::max3(sv[0], sv[1], sv[2]), ptx::max3(sv[3], sv[4], sv[5])};
 #pragma unroll
-                for (int e = 4; e < 64; e += 4) {
-                    mx[0] = fmaxf(mx[0], sv[e]); mx[1] = fmaxf(mx[1], sv[e + 1]);
-                    mx[2] = fmaxf(mx[2], sv[e + 2]); mx[3] = fmaxf(mx[3], sv[e + 3]);
+                for (int e = 6; e < 30; e += 4) {
+                    mx[0] = ptx::max3(mx[0], sv[e], sv[e + 1]);
+                    mx[1] = ptx::max3(mx[1], sv[e + 2], sv[e + 3]);
                 }
-                const float m_half = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * c_scale;   // c_scale > 0
-                float* xs = xchg + (tj & 1) * 256 + quarter * 64;
-                xs[half * 32 + lane] = m_half;
-                pair_sync(quarter);
-                const float m_tile = fmaxf(m_half, xs[(half ^ 1) * 32 + lane]);
+                const float m_part = ptx::max3(mx[0], mx[1], fmaxf(sv[30], sv[31])) * c_scale;   // c_scale > 0
+                __nv_bfloat16* xs = xm + (quarter * 2 + (tj & 1)) * 128;   // 512 bytes per quarter, shared with xl
+                xs[part * 32 + lane] = __float2bfloat16_ru(m_part);
+                quarter_sync(quarter);
+                const float m_tile = fmaxf(fmaxf(__bfloat162float(xs[lane]), __bfloat162float(xs[32 + lane])),
+                                           fmaxf(__bfloat162float(xs[64 + lane]), __bfloat162float(xs[96 + lane])));
                 float alpha = 1.f;
-                const bool raise = m_tile > m + 8.f;     // also true on the first live tile (m = -inf); same in both halves
+                const bool raise = m_tile > m + 8.f;     // also true on the first live tile (m = -inf); same in all four threads
                 if (raise) {
                     alpha = fast_exp2(m - m_tile);
                     m = m_tile;
                 }
                 const float neg_m = (m == -INFINITY) ? 0.f : -m;   // a fully masked row keeps p = 0
-                float sum[4] = {0.f, 0.f, 0.f, 0.f};
-                uint32_t packed[32];
+                const uint64_t cs2 = ptx::f32x2(c_scale, c_scale), nm2 = ptx::f32x2(neg_m, neg_m);
+                uint64_t sum2[2] = {0ull, 0ull};         // two-wide fp32 arithmetic: half the issue slots
+                uint32_t packed[16];
 #pragma unroll
-                for (int e = 0; e < 32; ++e) {
-                    const float x0 = fmaf(sv[2 * e], c_scale, neg_m), x1 = fmaf(sv[2 * e + 1], c_scale, neg_m);
-                    const float p0 = fast_exp2(x0);
-                    const float p1 = (e & 1) ? poly_exp2(x1) : fast_exp2(x1);
-                    sum[e & 3] += p0 + p1;
+                for (int e = 0; e < 16; ++e) {
+                    const uint64_t x2 = ptx::fma2(ptx::f32x2(sv[2 * e], sv[2 * e + 1]), cs2, nm2);
+                    float p0, p1;
+                    if (kPolyPair[e & 7]) {
+                        poly_exp2_pair(x2, p0, p1);
+                    } else {
+                        float x0, x1;
+                        ptx::f32x2_split(x2, x0, x1);
+                        p0 = fast_exp2(x0);
+                        p1 = fast_exp2(x1);
+                    }
+                    sum2[e & 1] = ptx::add2(sum2[e & 1], ptx::f32x2(p0, p1));
                     packed[e] = pack_bf16x2(p0, p1);
                 }
-                l = l * alpha + ((sum[0] + sum[1]) + (sum[2] + sum[3]));
-                // P_j (bf16 pairs): this thread's 64 keys = packed columns [32 half, 32 half + 32) of S_j
-                ptx::tmem_st32(s_tmem + half * 32, packed);
+                float s0, s1;
+                ptx::f32x2_split(ptx::add2(sum2[0], sum2[1]), s0, s1);
+                l = l * alpha + (s0 + s1);
+                // P_j (bf16 pairs): this thread's 32 keys = packed columns [16 part, 16 part + 16) of S_j
+                // (columns that other threads of the row read as scores: they did so before the exchange)
+                ptx::tmem_st16(s_tmem + part * 16, packed);
                 if (j > 0) {
                     // Every completion of o_done is waited for, in order, whether or not O has to be
                     // rescaled: a parity wait is only meaningful one phase at a time, and the
@@ -314,13 +338,19 @@ sm100_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                     if (__any_sync(0xffffffffu, raise)) {
                         ptx::tc_fence_after_sync();
 #pragma unroll 1
-                        for (int ch = 0; ch < 4; ++ch) {     // this thread's 128 of the 256 output columns
+                        for (int ch = 0; ch < 2; ++ch) {     // this thread's 64 of the 256 output columns
                             uint32_t r[32];
-                            ptx::tmem_ld32(tmem_o + lane_base + half * 128 + ch * 32, r);
+                            ptx::tmem_ld32(tmem_o + lane_base + part * 64 + ch * 32, r);
                             ptx::tmem_wait_ld();
+                            const uint64_t a2 = ptx::f32x2(alpha, alpha);
 #pragma unroll
-                            for (int e = 0; e < 32; ++e) r[e] = __float_as_uint(__uint_as_float(r[e]) * alpha);
-                            ptx::tmem_st32(tmem_o + lane_base + half * 128 + ch * 32, r);
+                            for (int e = 0; e < 32; e += 2) {
+                                float v0, v1;
+                                ptx::f32x2_split(ptx::mul2(ptx::f32x2(__uint_as_float(r[e]), __uint_as_float(r[e + 1])), a2), v0, v1);
+                                r[e] = __float_as_uint(v0);
+                                r[e + 1] = __float_as_uint(v1);
+                            }
+                            ptx::tmem_st32(tmem_o + lane_base + part * 64 + ch * 32, r);
                         }
                     }
                 }
@@ -330,20 +360,20 @@ sm100_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                 if (lane == 0) ptx::mbar_arrive_cluster(p_full_leader[tj & 1]);
             }
             if (!ok) break;
-            // ---- item epilogue: whole row sum, normalise, store this thread's 128 columns
-            float* xs = xchg + (tj & 1) * 256 + quarter * 64;   // tj already points past the item: next parity
-            xs[half * 32 + lane] = l;
-            pair_sync(quarter);
-            const float inv_l = 1.f / (l + xs[(half ^ 1) * 32 + lane]);
+            // ---- item epilogue: whole row sum, normalise, store this thread's 64 columns
+            quarter_sync(quarter);                   // everybody has read the last tile's partial maxima
+            xl[part * 32 + lane] = l;
+            quarter_sync(quarter);
+            const float inv_l = 1.f / ((xl[lane] + xl[32 + lane]) + (xl[64 + lane] + xl[96 + lane]));
             ok = __all_sync(0xffffffffu, ptx::mbar_wait(o_done, (tj - 1) & 1, abort_flag));
             if (!ok) break;
             ptx::tc_fence_after_sync();
             __nv_bfloat16* o_row = o_lat + (((size_t)w.b * d.n_q + w.g) * d.N + (t < d.N ? t : 0)) * d.d_l +
-                                   w.slice * kSlice + half * 128;
+                                   w.slice * kSlice + part * 64;
 #pragma unroll 1
-            for (int ch = 0; ch < 4; ++ch) {
+            for (int ch = 0; ch < 2; ++ch) {
                 uint32_t r[32];
-                ptx::tmem_ld32(tmem_o + lane_base + half * 128 + ch * 32, r);
+                ptx::tmem_ld32(tmem_o + lane_base + part * 64 + ch * 32, r);
                 ptx::tmem_wait_ld();
                 if (t < d.N) {
 #pragma unroll
@@ -360,7 +390,7 @@ sm100_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
             ptx::tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive_cluster(o_free_leader);
-            pair_sync(quarter);   // the exchange slot may be rewritten by the next tile of the same parity
+            quarter_sync(quarter);   // the exchange area is rewritten by the next item's first tile
         }
     }
     ptx::tc_fence_before_sync();
