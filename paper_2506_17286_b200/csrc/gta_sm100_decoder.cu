@@ -16,6 +16,12 @@
 //               complete they turn it into sigmoid gates held in registers (packed bf16) and hand
 //               the columns back, so the MUFU work hides under the acc_P MMAs; when acc_P is
 //               complete they multiply, round and store, while the next item's gate MMAs run.
+//
+// When all token rows fit one 128-row tile (a decode batch, a very short prompt) the second CTA of a
+// pair would hold no rows at all, and a head per pair leaves most SMs idle while each pair spends
+// its time on MMAs over padding.  That case runs the same kernel without pairs (template parameter
+// kPair = false: plain clusters of one, cta_group::1, M = 128) on items of HALF a head (64
+// columns), twice as many CTAs each with half the MMA time.
 #include "gta_sm100.cuh"
 
 #include <cuda.h>
@@ -35,7 +41,15 @@ constexpr uint32_t kATileBytes = kTileM * kBlockK * 2;   // 16 KB
 constexpr uint32_t kBGroupBytes = kBlockK * 64 * 2;      // 64 K-rows x 64 columns = 8 KB
 constexpr uint32_t kStageBytes = kATileBytes + 2 * kBGroupBytes;   // 32 KB per CTA
 constexpr uint32_t kBarOffset = kDecStages * kStageBytes;
-constexpr uint32_t kDecSmemTotal = kBarOffset + 256 + 1024;        // barriers + alignment slack
+constexpr uint32_t kBarBytes = 512;
+constexpr uint32_t kDecSmemTotal = kBarOffset + kBarBytes + 1024;  // barriers + alignment slack
+// Without CTA pairs (one row tile): the A tile holds only the rows that exist, rounded up to the
+// 8-row swizzle atom, which leaves room for a much deeper ring -- with one item per CTA and few
+// CTAs, the bytes in flight per SM are what paces the kernel.  The MMA still reads 128 rows: the
+// rows past the tile are whatever follows in shared memory (other tiles), and only feed
+// accumulator rows that are never stored.
+constexpr int kMaxStages = 16;
+constexpr uint32_t kSoloRingBytes = 200 * 1024;
 
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
@@ -52,14 +66,16 @@ __device__ __forceinline__ float sigmoid_tanh(float z) {
 // of heads) over G CTA pairs: every pair takes q = U / G whole units; the r = U mod G left over are
 // cut in two single-head halves when that makes the tail shorter (2 r <= G), else handed out whole.
 struct Schedule {
-    int n_hp;       // units per row tile (head pairs, or heads)
+    int n_hp;       // units per row tile (head pairs, heads, or (without CTA pairs) half heads)
     int pair;       // 1: a unit is two heads
     int RT;         // 256-row tiles per sequence
     int q, r, split_tail;
+    int n_stages;        // ring depth
+    uint32_t a_bytes;    // bytes of an A tile in the ring
 };
 
 struct Item {
-    int b, t0, i0, nt;   // batch entry, first token row (of the pair), first head, columns (128 or 256)
+    int b, t0, i0, hc, nt;   // batch entry, first token row, first head, first column inside it, columns
 };
 
 __device__ __forceinline__ int items_of_pair(const Schedule& s, int pr) {
@@ -67,6 +83,7 @@ __device__ __forceinline__ int items_of_pair(const Schedule& s, int pr) {
     return s.q + ((pr < s.r) ? 1 : 0);
 }
 
+template <bool kPair>
 __device__ __forceinline__ Item item_of(const Schedule& s, int pr, int G, int n) {
     int u, half = -1;
     if (n < s.q) u = pr * s.q + n;
@@ -76,6 +93,14 @@ __device__ __forceinline__ Item item_of(const Schedule& s, int pr, int G, int n)
     const int hp = u % s.n_hp;
     const int rt = (u / s.n_hp) % s.RT;
     it.b = u / (s.n_hp * s.RT);
+    it.hc = 0;
+    if (!kPair) {            // half a head on one CTA
+        it.t0 = rt * kTileM;
+        it.i0 = hp >> 1;
+        it.hc = (hp & 1) * 64;
+        it.nt = 64;
+        return it;
+    }
     it.t0 = rt * 2 * kTileM;
     if (s.pair) {
         it.i0 = 2 * hp + (half < 0 ? 0 : half);
@@ -87,15 +112,23 @@ __device__ __forceinline__ Item item_of(const Schedule& s, int pr, int G, int n)
     return it;
 }
 
+template <bool kPair>
 __global__ void __launch_bounds__(kDecThreads, 1)
 sm100_decoder_kernel(const __grid_constant__ CUtensorMap tm_l, const __grid_constant__ CUtensorMap tm_x,
                      const __grid_constant__ CUtensorMap tm_wp, const __grid_constant__ CUtensorMap tm_wg,
                      Dims d, Schedule sch, __nv_bfloat16* __restrict__ out, int32_t* status_word) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-    uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + kBarOffset);   // used in the leader CTA
-    uint64_t* empty_bar = full_bar + kDecStages;                             // both CTAs
-    uint64_t* accg_full = empty_bar + kDecStages;                            // both CTAs
+    // ring: pairs keep {A, B} of a stage side by side; without pairs all A tiles come first, then all B tiles
+    const int n_stages = kPair ? kDecStages : sch.n_stages;
+    const uint32_t a_stride = kPair ? kStageBytes : sch.a_bytes;
+    const uint32_t b_base = kPair ? kATileBytes : (uint32_t)n_stages * sch.a_bytes;
+    const uint32_t b_stride = kPair ? kStageBytes : kBGroupBytes;
+    const uint32_t a_tile_bytes = kPair ? kATileBytes : sch.a_bytes;
+    const uint32_t bar_off = kPair ? kBarOffset : (uint32_t)n_stages * (sch.a_bytes + kBGroupBytes);
+    uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + bar_off);       // used in the leader CTA
+    uint64_t* empty_bar = full_bar + kMaxStages;                             // both CTAs
+    uint64_t* accg_full = empty_bar + kMaxStages;                            // both CTAs
     uint64_t* accp_full = accg_full + 1;                                     // both CTAs
     uint64_t* accg_free = accp_full + 1;                                     // leader CTA: 16 warps arrive
     uint64_t* accp_free = accg_free + 1;                                     // leader CTA
@@ -104,26 +137,32 @@ sm100_decoder_kernel(const __grid_constant__ CUtensorMap tm_l, const __grid_cons
     volatile int* drain_flag = abort_flag + 1;   // never raised: lets the drain wait run to its limit
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const uint32_t rank = ptx::cluster_ctarank();          // 0 = leader
-    const int G = gridDim.x >> 1, pr = blockIdx.x >> 1;    // CTA pairs, this pair
+    const uint32_t rank = kPair ? ptx::cluster_ctarank() : 0u;          // 0 = leader
+    const int G = kPair ? gridDim.x >> 1 : gridDim.x;                   // CTA pairs (or CTAs)
+    const int pr = kPair ? blockIdx.x >> 1 : blockIdx.x;                // this pair
     const int n_items = items_of_pair(sch, pr);
     const int ks_g = d.H / kBlockK, ks_p = d.d_l / kBlockK, ks_total = ks_g + ks_p;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < kDecStages; ++s) { ptx::mbar_init(&full_bar[s], 2); ptx::mbar_init(&empty_bar[s], 1); }
+        for (int s = 0; s < n_stages; ++s) { ptx::mbar_init(&full_bar[s], kPair ? 2 : 1); ptx::mbar_init(&empty_bar[s], 1); }
         ptx::mbar_init(accg_full, 1);
         ptx::mbar_init(accp_full, 1);
-        ptx::mbar_init(accg_free, 16);
-        ptx::mbar_init(accp_free, 16);
+        ptx::mbar_init(accg_free, kPair ? 16 : 8);
+        ptx::mbar_init(accp_free, kPair ? 16 : 8);
         *abort_flag = 0;
         *drain_flag = 0;
         ptx::fence_mbar_init();
     }
-    if (warp == 1) ptx::tmem_alloc_pair(tmem_slot, 512);
+    if (warp == 1) {
+        if (kPair) ptx::tmem_alloc_pair(tmem_slot, 512);
+        else ptx::tmem_alloc(tmem_slot, 512);
+    }
     ptx::tc_fence_before_sync();
     __syncthreads();
-    ptx::cluster_arrive();     // the peer's barriers exist before anything is signalled to them
-    ptx::cluster_wait();
+    if (kPair) {
+        ptx::cluster_arrive();     // the peer's barriers exist before anything is signalled to them
+        ptx::cluster_wait();
+    }
     ptx::tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
     const uint32_t tmem_p = tmem_base, tmem_g = tmem_base + 256;
@@ -133,23 +172,41 @@ sm100_decoder_kernel(const __grid_constant__ CUtensorMap tm_l, const __grid_cons
             ptx::prefetch_tensormap(&tm_l); ptx::prefetch_tensormap(&tm_x);
             ptx::prefetch_tensormap(&tm_wp); ptx::prefetch_tensormap(&tm_wg);
             int it = 0;            // ring iteration, runs on across items
+            int s = 0;             // its stage and phase, kept as counters (no division in the loop)
+            uint32_t ph = 0;
             bool ok = true;
             bool l_ready = false;
             for (int n = 0; n < n_items && ok; ++n) {
-                const Item w = item_of(sch, pr, G, n);
+                const Item w = item_of<kPair>(sch, pr, G, n);
                 const int t0 = w.t0 + (int)rank * kTileM;          // this CTA's rows
-                const int n_grp = w.nt / 128;                      // 64-column groups of this CTA's weight half
+                const int n_grp = kPair ? w.nt / 128 : w.nt / 64;  // 64-column groups this CTA stages
                 const int col0 = (int)rank * (w.nt / 2);           // first of this CTA's columns inside the item
-                const int head = w.i0 + col0 / 128, hcol = col0 % 128;
+                const int head = w.i0 + col0 / 128, hcol = w.hc + col0 % 128;
                 const int g = d.head_to_q(w.i0);
-                const uint32_t tx = kATileBytes + (uint32_t)n_grp * kBGroupBytes;
-                for (int ks = 0; ks < ks_total; ++ks, ++it) {
-                    const int s = it % kDecStages;
-                    const uint32_t ph = (it / kDecStages) & 1;
+                const uint32_t tx = a_tile_bytes + (uint32_t)n_grp * kBGroupBytes;
+                for (int ks = 0; ks < ks_total; ++ks, ++it, s = (s + 1 == n_stages) ? 0 : s + 1, ph ^= (s == 0)) {
                     ok = ptx::mbar_wait(&empty_bar[s], ph ^ 1, abort_flag);
                     if (!ok) break;
-                    uint8_t* a_s = smem + s * kStageBytes;
-                    uint8_t* b_s = a_s + kATileBytes;
+                    uint8_t* a_s = smem + s * a_stride;
+                    uint8_t* b_s = smem + b_base + s * b_stride;
+                    if (!kPair) {
+                        uint64_t* bar = &full_bar[s];
+                        ptx::mbar_arrive_expect_tx(bar, tx);
+                        if (ks < ks_g) {
+                            ptx::tma_load_3d(a_s, &tm_x, bar, ks * kBlockK, t0, w.b);
+                            for (int grp = 0; grp < n_grp; ++grp)
+                                ptx::tma_load_2d(b_s + grp * kBGroupBytes, &tm_wg, bar, head * 128 + hcol + grp * 64,
+                                                 ks * kBlockK);
+                        } else {
+                            const int kk = ks - ks_g;
+                            if (!l_ready) { ptx::grid_dependency_wait(); l_ready = true; }
+                            ptx::tma_load_3d(a_s, &tm_l, bar, kk * kBlockK, t0, w.b * d.n_q + g);
+                            for (int grp = 0; grp < n_grp; ++grp)
+                                ptx::tma_load_3d(b_s + grp * kBGroupBytes, &tm_wp, bar, hcol + grp * 64, kk * kBlockK,
+                                                 head);
+                        }
+                        continue;
+                    }
                     const uint32_t bar = ptx::map_to_cta(ptx::smem_addr(&full_bar[s]), 0);   // the leader's
                     ptx::mbar_arrive_expect_tx_cluster(bar, tx);
                     if (ks < ks_g) {
@@ -171,42 +228,48 @@ sm100_decoder_kernel(const __grid_constant__ CUtensorMap tm_l, const __grid_cons
                 }
             }
             if (*abort_flag && rank == 0) {   // drain: every armed stage either lands or the wait gives up
-                for (int back = 1; back <= kDecStages && it - back >= 0; ++back) {
+                for (int back = 1; back <= n_stages && it - back >= 0; ++back) {
                     const int kq = it - back;
-                    ptx::mbar_wait(&full_bar[kq % kDecStages], (kq / kDecStages) & 1, drain_flag);
+                    ptx::mbar_wait(&full_bar[kq % n_stages], (kq / n_stages) & 1, drain_flag);
                 }
             }
         }
     } else if (warp == 1) {
         if (rank == 0 && ptx::elect_one()) {
-            int it = 0;
+            int it = 0, s = 0;
+            uint32_t ph = 0;
             bool ok = true;
             for (int n = 0; n < n_items && ok; ++n) {
-                const Item w = item_of(sch, pr, G, n);
-                const uint32_t idesc = ptx::make_idesc_bf16(2 * kTileM, w.nt, 0, 1);   // A K-major, B MN-major
-                for (int ks = 0; ks < ks_total; ++ks, ++it) {
+                const Item w = item_of<kPair>(sch, pr, G, n);
+                const uint32_t idesc = ptx::make_idesc_bf16(kPair ? 2 * kTileM : kTileM, w.nt, 0, 1);   // A K-major, B MN-major
+                for (int ks = 0; ks < ks_total; ++ks, ++it, s = (s + 1 == n_stages) ? 0 : s + 1, ph ^= (s == 0)) {
                     // the accumulator about to be overwritten must have been read by both epilogues
                     if (ks == 0) ok = ptx::mbar_wait(accg_free, (n & 1) ^ 1, abort_flag);
                     else if (ks == ks_g) ok = ptx::mbar_wait(accp_free, (n & 1) ^ 1, abort_flag);
                     if (!ok) break;
-                    const int s = it % kDecStages;
-                    const uint32_t ph = (it / kDecStages) & 1;
                     ok = ptx::mbar_wait(&full_bar[s], ph, abort_flag);
                     if (!ok) break;
                     ptx::tc_fence_after_sync();
-                    const uint32_t a_addr = ptx::smem_addr(smem + s * kStageBytes);
-                    const uint32_t b_addr = a_addr + kATileBytes;
+                    const uint32_t a_addr = ptx::smem_addr(smem + s * a_stride);
+                    const uint32_t b_addr = ptx::smem_addr(smem + b_base + s * b_stride);
                     const uint32_t d_tmem = ks < ks_g ? tmem_g : tmem_p;
                     const bool first = (ks == 0) || (ks == ks_g);
 #pragma unroll
                     for (int k4 = 0; k4 < kBlockK / 16; ++k4) {
                         const uint64_t a_desc = ptx::make_smem_desc(a_addr + k4 * 32, 16, 1024);
                         const uint64_t b_desc = ptx::make_smem_desc(b_addr + k4 * 16 * 128, 64 * 128, 1024);
-                        ptx::mma_ss_pair(d_tmem, a_desc, b_desc, idesc, (first && k4 == 0) ? 0u : 1u);
+                        if (kPair) ptx::mma_ss_pair(d_tmem, a_desc, b_desc, idesc, (first && k4 == 0) ? 0u : 1u);
+                        else ptx::mma_ss(d_tmem, a_desc, b_desc, idesc, (first && k4 == 0) ? 0u : 1u);
                     }
-                    ptx::tc_commit_pair(&empty_bar[s], 3);
-                    if (ks == ks_g - 1) ptx::tc_commit_pair(accg_full, 3);
-                    if (ks == ks_total - 1) ptx::tc_commit_pair(accp_full, 3);
+                    if (kPair) {
+                        ptx::tc_commit_pair(&empty_bar[s], 3);
+                        if (ks == ks_g - 1) ptx::tc_commit_pair(accg_full, 3);
+                        if (ks == ks_total - 1) ptx::tc_commit_pair(accp_full, 3);
+                    } else {
+                        ptx::tc_commit(&empty_bar[s]);
+                        if (ks == ks_g - 1) ptx::tc_commit(accg_full);
+                        if (ks == ks_total - 1) ptx::tc_commit(accp_full);
+                    }
                 }
             }
         }
@@ -221,8 +284,8 @@ sm100_decoder_kernel(const __grid_constant__ CUtensorMap tm_l, const __grid_cons
         const uint32_t accp_free_leader = ptx::map_to_cta(ptx::smem_addr(accp_free), 0);
         bool ok = true;
         for (int n = 0; n < n_items && ok; ++n) {
-            const Item w = item_of(sch, pr, G, n);
-            const int cols = w.nt / 2;               // this warp's columns: 128 or 64
+            const Item w = item_of<kPair>(sch, pr, G, n);
+            const int cols = w.nt / 2;               // this warp's columns: 128, 64 or 32
             const int c0 = half * cols;
             const int t = w.t0 + (int)rank * kTileM + row;
             uint32_t gate[64];                       // sigmoid gates, packed bf16 pairs
@@ -243,13 +306,16 @@ sm100_decoder_kernel(const __grid_constant__ CUtensorMap tm_l, const __grid_cons
             }
             ptx::tc_fence_before_sync();
             __syncwarp();
-            if (lane == 0) ptx::mbar_arrive_cluster(accg_free_leader);
+            if (lane == 0) {
+                if (kPair) ptx::mbar_arrive_cluster(accg_free_leader);
+                else ptx::mbar_arrive(accg_free);
+            }
 
             ok = __all_sync(0xffffffffu, ptx::mbar_wait(accp_full, n & 1, abort_flag));
             if (!ok) break;
             ptx::tc_fence_after_sync();
             // columns [c0, c0 + cols) of the item = head i0 + (c0 / 128), columns (c0 % 128) ..
-            __nv_bfloat16* o_row = out + (((size_t)w.b * d.N + (t < d.N ? t : 0)) * d.n_h + w.i0) * 128 + c0;
+            __nv_bfloat16* o_row = out + (((size_t)w.b * d.N + (t < d.N ? t : 0)) * d.n_h + w.i0) * 128 + w.hc + c0;
 #pragma unroll
             for (int ch = 0; ch < 4; ++ch) {
                 if (ch * 32 < cols) {
@@ -275,14 +341,22 @@ sm100_decoder_kernel(const __grid_constant__ CUtensorMap tm_l, const __grid_cons
             }
             ptx::tc_fence_before_sync();
             __syncwarp();
-            if (lane == 0) ptx::mbar_arrive_cluster(accp_free_leader);
+            if (lane == 0) {
+                if (kPair) ptx::mbar_arrive_cluster(accp_free_leader);
+                else ptx::mbar_arrive(accp_free);
+            }
         }
     }
     ptx::tc_fence_before_sync();
     __syncthreads();
-    ptx::cluster_arrive();     // neither CTA leaves (or frees TMEM) while the other may still signal it
-    ptx::cluster_wait();
-    if (warp == 1) ptx::tmem_dealloc_pair(tmem_base, 512);
+    if (kPair) {
+        ptx::cluster_arrive();     // neither CTA leaves (or frees TMEM) while the other may still signal it
+        ptx::cluster_wait();
+    }
+    if (warp == 1) {
+        if (kPair) ptx::tmem_dealloc_pair(tmem_base, 512);
+        else ptx::tmem_dealloc(tmem_base, 512);
+    }
     if (threadIdx.x == 0 && *abort_flag) raise_status(status_word, GTA_ERR_TIMEOUT);
 }
 
@@ -302,14 +376,16 @@ int sm_count() {
 gta_status_t launch_sm100_decoder(const Dims& d, const void* l_bf16, const void* x, const void* w_p, const void* w_g,
                                   void* out, int32_t* status_word, cudaStream_t stream) {
     CUtensorMap tm_l, tm_x, tm_wp, tm_wg;
+    const bool solo = d.N <= kTileM;                                    // one row tile: no CTA pairs
+    const uint32_t a_rows = solo ? (uint32_t)((d.N + 7) & ~7) : kTileM; // rows of an A tile
     {
         const uint64_t dims[3] = {(uint64_t)d.d_l, (uint64_t)d.N, (uint64_t)d.B * d.n_q};
-        const uint32_t box[3] = {kBlockK, kTileM, 1};
+        const uint32_t box[3] = {kBlockK, a_rows, 1};
         if (!make_bf16_map(&tm_l, l_bf16, 3, dims, box)) return GTA_ERR_CUDA;
     }
     {
         const uint64_t dims[3] = {(uint64_t)d.H, (uint64_t)d.N, (uint64_t)d.B};
-        const uint32_t box[3] = {kBlockK, kTileM, 1};
+        const uint32_t box[3] = {kBlockK, a_rows, 1};
         if (!make_bf16_map(&tm_x, x, 3, dims, box)) return GTA_ERR_CUDA;
     }
     {
@@ -322,20 +398,54 @@ gta_status_t launch_sm100_decoder(const Dims& d, const void* l_bf16, const void*
         const uint32_t box[2] = {64, kBlockK};
         if (!make_bf16_map(&tm_wg, w_g, 2, dims, box)) return GTA_ERR_CUDA;
     }
-    Schedule s;
-    s.pair = (d.n_h / d.n_q) % 2 == 0 ? 1 : 0;
-    s.n_hp = s.pair ? d.n_h / 2 : d.n_h;
-    s.RT = (d.N + 2 * kTileM - 1) / (2 * kTileM);
-    long long U = (long long)d.B * s.RT * s.n_hp;
-    if (U > 0x3fffffffLL) return GTA_ERR_UNSUPPORTED;
-    if (cudaFuncSetAttribute(sm100_decoder_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             (int)kDecSmemTotal) != cudaSuccess)
-        return GTA_ERR_CUDA;
     cudaLaunchConfig_t cfg = {};
     cfg.blockDim = dim3(kDecThreads);
     cfg.dynamicSmemBytes = kDecSmemTotal;
     cfg.stream = stream;
     cudaLaunchAttribute attr[2];
+    if (solo) {
+        // half-head items over as many SMs as there are items
+        Schedule s;
+        s.a_bytes = a_rows * kBlockK * 2;
+        s.n_stages = (int)(kSoloRingBytes / (s.a_bytes + kBGroupBytes));
+        if (s.n_stages > kMaxStages) s.n_stages = kMaxStages;
+        // the MMA reads 16 KB from every A tile: the B tiles behind the last one must cover that
+        if ((uint32_t)s.n_stages * kBGroupBytes < kATileBytes) return GTA_ERR_UNSUPPORTED;
+        const uint32_t smem_bytes = (uint32_t)s.n_stages * (s.a_bytes + kBGroupBytes) + kBarBytes + 1024;
+        cfg.dynamicSmemBytes = smem_bytes;
+        s.pair = 0;
+        s.n_hp = 2 * d.n_h;
+        s.RT = 1;
+        const long long U = (long long)d.B * s.n_hp;
+        if (U > 0x3fffffffLL) return GTA_ERR_UNSUPPORTED;
+        if (cudaFuncSetAttribute(sm100_decoder_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)smem_bytes) != cudaSuccess)
+            return GTA_ERR_CUDA;
+        const int G = U < sm_count() ? (int)U : sm_count();
+        s.q = (int)(U / G);
+        s.r = (int)(U % G);
+        s.split_tail = 0;
+        cfg.gridDim = dim3(G);
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        if (cudaLaunchKernelEx(&cfg, sm100_decoder_kernel<false>, tm_l, tm_x, tm_wp, tm_wg, d, s, (__nv_bfloat16*)out,
+                               status_word) != cudaSuccess)
+            return GTA_ERR_CUDA;
+        return cudaGetLastError() == cudaSuccess ? GTA_OK : GTA_ERR_CUDA;
+    }
+    Schedule s;
+    s.n_stages = kDecStages;
+    s.a_bytes = kATileBytes;
+    s.pair = (d.n_h / d.n_q) % 2 == 0 ? 1 : 0;
+    s.n_hp = s.pair ? d.n_h / 2 : d.n_h;
+    s.RT = (d.N + 2 * kTileM - 1) / (2 * kTileM);
+    long long U = (long long)d.B * s.RT * s.n_hp;
+    if (U > 0x3fffffffLL) return GTA_ERR_UNSUPPORTED;
+    if (cudaFuncSetAttribute(sm100_decoder_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)kDecSmemTotal) != cudaSuccess)
+        return GTA_ERR_CUDA;
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = 2;
     attr[0].val.clusterDim.y = 1;
@@ -352,7 +462,7 @@ gta_status_t launch_sm100_decoder(const Dims& d, const void* l_bf16, const void*
     if (dev != cached_dev) {
         cfg.gridDim = dim3(2 * (sm_count() / 2));
         int n = 0;
-        if (cudaOccupancyMaxActiveClusters(&n, sm100_decoder_kernel, &cfg) != cudaSuccess || n < 1) return GTA_ERR_CUDA;
+        if (cudaOccupancyMaxActiveClusters(&n, sm100_decoder_kernel<true>, &cfg) != cudaSuccess || n < 1) return GTA_ERR_CUDA;
         cached_dev = dev;
         cached_pairs = n;
     }
@@ -368,7 +478,7 @@ gta_status_t launch_sm100_decoder(const Dims& d, const void* l_bf16, const void*
     s.split_tail = (s.pair && 2 * s.r <= G) ? 1 : 0;
     cfg.gridDim = dim3(2 * G);
     cfg.numAttrs = 2;
-    if (cudaLaunchKernelEx(&cfg, sm100_decoder_kernel, tm_l, tm_x, tm_wp, tm_wg, d, s, (__nv_bfloat16*)out,
+    if (cudaLaunchKernelEx(&cfg, sm100_decoder_kernel<true>, tm_l, tm_x, tm_wp, tm_wg, d, s, (__nv_bfloat16*)out,
                            status_word) != cudaSuccess)
         return GTA_ERR_CUDA;
     return cudaGetLastError() == cudaSuccess ? GTA_OK : GTA_ERR_CUDA;
