@@ -48,7 +48,7 @@ struct FastPlan {
     int T;         // tokens per sub-tile (16, 32 or 64)
     int G;         // stream CTAs
     int slots;     // G + B partial slots
-    size_t off_ml, off_rng, off_bound, off_l, total;   // byte offsets in the workspace (part_o at 0)
+    size_t off_ml, off_l, total;   // byte offsets in the workspace (part_o at 0)
 };
 constexpr int kFinMaxBatchClusters = 16;   // larger batches finish through the merge kernel + the tcgen05 decoder kernel
                                            // (measured: faster from 32 sequences on; the weights then feed 128-row MMAs)
@@ -87,9 +87,7 @@ static FastPlan make_fast_plan(const Dims& d) {
     const size_t part_o = (size_t)p.slots * d.n_q * d.d_l * sizeof(float);
     const size_t part_ml = (size_t)p.slots * d.n_q * 2 * sizeof(float);
     p.off_ml = align256f(part_o);
-    p.off_rng = p.off_ml + align256f(part_ml);
-    p.off_bound = p.off_rng + align256f((size_t)d.B * 2 * sizeof(int32_t));
-    p.off_l = p.off_bound + align256f((size_t)(p.G + 1) * sizeof(int32_t));
+    p.off_l = p.off_ml + align256f(part_ml);
     p.total = p.off_l + align256f((size_t)d.n_q * d.B * d.d_l * sizeof(__nv_bfloat16));
     return p;
 }
@@ -118,8 +116,7 @@ template <int NT>   // NT = d_l / 64 = MMA n-tiles (8 latent columns each) per c
 __global__ void __launch_bounds__(kStreamThreads, 1)
 decode_stream_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_c, Dims d,
                      int T, int S_cap, const __nv_bfloat16* __restrict__ q, const int32_t* __restrict__ seq_lens,
-                     float* __restrict__ part_o, float* __restrict__ part_ml, int32_t* __restrict__ rng_g,
-                     int32_t* __restrict__ bound_g, int32_t* status_word) {
+                     float* __restrict__ part_o, float* __restrict__ part_ml, int32_t* status_word) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     uint8_t* ring = smem;                                                              // 3 x 64 KB
@@ -179,25 +176,6 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
     }
     const long long n_st = prefix[d.B];
     const long long st_begin = ((long long)cta * n_st) / G, st_end = ((long long)(cta + 1) * n_st) / G;
-    // ---- tables for the merge kernel (large batches): bound_g[c] = first sub-tile of CTA c, and for
-    //      sequence b the CTAs c_lo .. c_hi that own its sub-tiles (CTA c answers for b = c, c + G, ...).
-    //      The owner of sub-tile st is the largest c with floor(c n / G) <= st = floor(((st + 1) G - 1) / n).
-    if (rng_g != nullptr) {
-        if (tid == 0) {
-            bound_g[cta] = (int32_t)st_begin;
-            if (cta == 0) bound_g[G] = (int32_t)n_st;
-        }
-        for (int b = cta + tid * G; b < d.B; b += G * kStreamThreads) {
-            const long long s_lo = prefix[b], s_hi = prefix[b + 1];
-            int c_lo = 0, c_hi = -1;
-            if (s_hi > s_lo) {
-                c_lo = (int)(((s_lo + 1) * G - 1) / n_st);
-                c_hi = (int)((s_hi * G - 1) / n_st);
-            }
-            rng_g[2 * b] = c_lo;
-            rng_g[2 * b + 1] = c_hi;
-        }
-    }
     if (st_begin >= st_end) return;      // uniform: nothing armed
     int b0;
     {   // largest b with prefix[b] <= st_begin: a non-empty sequence, since st_begin < n_st
@@ -766,38 +744,88 @@ static int finish_split(const Dims& d) {
 // Large batches: log-sum-exp merge of the split-KV slots of one (attention map, sequence) pair per
 // CTA into the normalised latent L[n_q][B][d_l] (bf16), which the tcgen05 decoder + gate kernel of
 // the prefill path then consumes with the batch in the role of the token axis.
+// Launched with programmatic stream serialisation: while the stream kernel still runs, the CTA
+// works out from the sequence lengths (inputs, not results of that kernel) which stream CTAs own
+// sub-tiles of its sequence -- the same arithmetic as in the stream kernel: prefix sums of
+// ceil(len / T), ranges c n / G -- so that after the dependency wait a single round of loads
+// (every slot's (max, sum) pair and its partial sums together) is all that is left.
 __global__ void __launch_bounds__(256)
-decode_merge_kernel(Dims d, int G, const int32_t* __restrict__ rng_g, const int32_t* __restrict__ bound_g,
+decode_merge_kernel(Dims d, int G, int T, int S_cap, const int32_t* __restrict__ seq_lens,
                     const float* __restrict__ part_o, const float* __restrict__ part_ml,
                     __nv_bfloat16* __restrict__ l_out) {
+    __shared__ long long red_s[2][8];
+    __shared__ int live_s[kFinMaxSlots];        // slot j of the range holds something
     ptx::grid_launch_dependents();
-    ptx::grid_dependency_wait();
-    const int g = blockIdx.x, b = blockIdx.y;
-    const int c_lo = rng_g[2 * b], c_hi = rng_g[2 * b + 1];
-    float M = -INFINITY, l = 0.f;
-    for (int c = c_lo; c <= c_hi; ++c)
-        if (bound_g[c] < bound_g[c + 1]) M = fmaxf(M, part_ml[((size_t)(c + b) * d.n_q + g) * 2]);
-    for (int c = c_lo; c <= c_hi; ++c)
-        if (bound_g[c] < bound_g[c + 1]) {   // a CTA with an empty range wrote nothing
-            const float* ml = part_ml + ((size_t)(c + b) * d.n_q + g) * 2;
-            l = fmaf(ml[1], ex2f(ml[0] - M), l);
-        }
-    const float inv_l = c_hi >= c_lo ? 1.f / l : 0.f;
-    for (int col = threadIdx.x * 4; col < d.d_l; col += 256 * 4) {
-        float4 sum = make_float4(0.f, 0.f, 0.f, 0.f);
-        for (int c = c_lo; c <= c_hi; ++c) {
-            if (!(bound_g[c] < bound_g[c + 1])) continue;
-            const size_t pi = (size_t)(c + b) * d.n_q + g;
-            const float w = ex2f(part_ml[pi * 2] - M) * inv_l;
-            const float4 v = *reinterpret_cast<const float4*>(part_o + pi * d.d_l + col);
-            sum.x = fmaf(v.x, w, sum.x); sum.y = fmaf(v.y, w, sum.y);
-            sum.z = fmaf(v.z, w, sum.z); sum.w = fmaf(v.w, w, sum.w);
-        }
-        uint2 packed;
-        packed.x = pack_bf16(sum.x, sum.y);
-        packed.y = pack_bf16(sum.z, sum.w);
-        *reinterpret_cast<uint2*>(l_out + ((size_t)g * d.B + b) * d.d_l + col) = packed;
+    const int g = blockIdx.x, b = blockIdx.y, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    long long before = 0, total = 0;            // sub-tiles of the sequences before b, of all sequences
+    for (int i = tid; i < d.B; i += 256) {
+        const int n = (clamp_len(seq_lens[i], S_cap) + T - 1) / T;
+        total += n;
+        if (i < b) before += n;
     }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        before += __shfl_xor_sync(0xffffffffu, before, o);
+        total += __shfl_xor_sync(0xffffffffu, total, o);
+    }
+    if (lane == 0) { red_s[0][warp] = before; red_s[1][warp] = total; }
+    __syncthreads();
+    long long s_lo = 0, n_st = 0;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) { s_lo += red_s[0][w]; n_st += red_s[1][w]; }
+    const long long s_hi = s_lo + (clamp_len(seq_lens[b], S_cap) + T - 1) / T;
+    // the owner of sub-tile st is the largest c with floor(c n / G) <= st = floor(((st + 1) G - 1) / n)
+    int c_lo = 0, c_hi = -1;
+    if (s_hi > s_lo) {
+        c_lo = (int)(((s_lo + 1) * G - 1) / n_st);
+        c_hi = (int)((s_hi * G - 1) / n_st);
+    }
+    for (int j = tid; c_lo + j <= c_hi; j += 256) {   // a CTA with an empty range wrote nothing
+        const int c = c_lo + j;
+        live_s[j] = ((long long)c * n_st) / G < ((long long)(c + 1) * n_st) / G;
+    }
+    __syncthreads();
+    ptx::grid_dependency_wait();
+
+    const int col = tid * 4;
+    if (col >= d.d_l) return;
+    float M = -INFINITY, l = 0.f;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int c0 = c_lo; c0 <= c_hi; c0 += 8) {       // eight slots per round of loads
+        float2 ml[8];
+        float4 v[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const int c = c0 + j;
+            ml[j] = make_float2(-INFINITY, 0.f);
+            v[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (c <= c_hi && live_s[c - c_lo]) {
+                const size_t pi = (size_t)(c + b) * d.n_q + g;
+                ml[j] = *reinterpret_cast<const float2*>(part_ml + pi * 2);
+                v[j] = *reinterpret_cast<const float4*>(part_o + pi * d.d_l + col);
+            }
+        }
+        float Mn = M;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) Mn = fmaxf(Mn, ml[j].x);
+        if (Mn == -INFINITY) continue;               // nothing live so far
+        const float scale = ex2f(M - Mn);            // 0 on the first live round (M = -inf)
+        l *= scale;
+        acc.x *= scale; acc.y *= scale; acc.z *= scale; acc.w *= scale;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const float w = ex2f(ml[j].x - Mn);      // 0 for a slot that is not there
+            l = fmaf(ml[j].y, w, l);
+            acc.x = fmaf(v[j].x, w, acc.x); acc.y = fmaf(v[j].y, w, acc.y);
+            acc.z = fmaf(v[j].z, w, acc.z); acc.w = fmaf(v[j].w, w, acc.w);
+        }
+        M = Mn;
+    }
+    const float inv_l = l > 0.f ? 1.f / l : 0.f;     // an empty sequence gives zeros
+    uint2 packed;
+    packed.x = pack_bf16(acc.x * inv_l, acc.y * inv_l);
+    packed.y = pack_bf16(acc.z * inv_l, acc.w * inv_l);
+    *reinterpret_cast<uint2*>(l_out + ((size_t)g * d.B + b) * d.d_l + col) = packed;
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -808,8 +836,6 @@ cudaError_t launch_decode_fast(const Dims& d, const void* q, const void* k_cache
     const FastPlan p = make_fast_plan(d);
     float* part_o = reinterpret_cast<float*>(workspace);
     float* part_ml = reinterpret_cast<float*>(static_cast<char*>(workspace) + p.off_ml);
-    int32_t* rng_g = reinterpret_cast<int32_t*>(static_cast<char*>(workspace) + p.off_rng);
-    int32_t* bound_g = reinterpret_cast<int32_t*>(static_cast<char*>(workspace) + p.off_bound);
     __nv_bfloat16* l_g = reinterpret_cast<__nv_bfloat16*>(static_cast<char*>(workspace) + p.off_l);
     const bool big_batch = d.B > kFinMaxBatchClusters;
     cudaError_t err;
@@ -839,8 +865,7 @@ cudaError_t launch_decode_fast(const Dims& d, const void* q, const void* k_cache
             cfg.attrs = attr;                                                                              \
             cfg.numAttrs = 1;                                                                              \
             err = cudaLaunchKernelEx(&cfg, kern, tm_k, tm_c, d, p.T, S_cap, (const __nv_bfloat16*)q,       \
-                                     seq_lens, part_o, part_ml, big_batch ? rng_g : (int32_t*)nullptr,     \
-                                     bound_g, status_word);                                                \
+                                     seq_lens, part_o, part_ml, status_word);                              \
             if (err != cudaSuccess) return err;                                                            \
         } while (0)
         switch (d.d_l) {
@@ -862,8 +887,8 @@ cudaError_t launch_decode_fast(const Dims& d, const void* q, const void* k_cache
         attr[0].val.programmaticStreamSerializationAllowed = 1;
         cfg.attrs = attr;
         cfg.numAttrs = 1;
-        err = cudaLaunchKernelEx(&cfg, decode_merge_kernel, d, p.G, (const int32_t*)rng_g, (const int32_t*)bound_g,
-                                 (const float*)part_o, (const float*)part_ml, l_g);
+        err = cudaLaunchKernelEx(&cfg, decode_merge_kernel, d, p.G, p.T, S_cap, seq_lens, (const float*)part_o,
+                                 (const float*)part_ml, l_g);
         if (err != cudaSuccess) return err;
         // the batch takes the role of the token axis: L [n_q][B][d_l], x_t [B][H], out [B][n_h][d_h]
         Dims dd = d;
