@@ -131,9 +131,6 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int G = gridDim.x, cta = blockIdx.x;
     const int NQ = d.n_q;
-    // the finish kernel may be scheduled as soon as SMs free up: it prefetches its weights and
-    // then waits for this whole grid before it touches the partial results
-    ptx::grid_launch_dependents();
     if (tid == kStreamConsumers) {   // the descriptors are on their way while the prefix sum runs
         ptx::prefetch_tensormap(&tm_k);
         ptx::prefetch_tensormap(&tm_c);
@@ -143,6 +140,10 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
     // scheduled while the kernel before it in the stream (a cache append, the previous decode
     // step) was still draining, and must not read that kernel's results (lengths, caches) earlier.
     ptx::grid_dependency_wait();
+    // Only now may the kernels after this one be scheduled: they read inputs (sequence lengths,
+    // hidden states, weights) before their own dependency wait, which orders them against this
+    // kernel alone -- whatever ran before this kernel is complete and visible from here on.
+    ptx::grid_launch_dependents();
 
     // ---- exclusive prefix sum of the sub-tile counts: prefix[b] = sum_{b' < b} ceil(len / T)
     //      (thread t owns sequences [t per, (t + 1) per); warp scan, then a scan of the warp totals)

@@ -22,7 +22,7 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
 // the latent, run by a CTA pair (cluster of 2, tcgen05 cta_group::2): each CTA owns one query tile
 // (its own S / P / O in its own TMEM) and stages HALF of every key tile (64 of the 128 keys for
 // S = Q K^T, 128 of the 256 latent columns for O += P C), so K and C cross L2 -> shared memory once
-// per 256 query rows and the ring is four key tiles deep.  (The 128 x d_l fp32 output does not fit
+// per 256 query rows and the ring is three key tiles deep.  (The 128 x d_l fp32 output does not fit
 // the 512 TMEM columns next to the score tiles, so d_l is cut in slices of 256 and each slice item
 // recomputes the scores.)  Persistent: a pair walks a static list of items, heaviest (latest)
 // query tiles first, dealt to the pairs in snake order.  Per 128-key tile j:
@@ -31,11 +31,12 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
 //                            exchanged through shared memory); P_j (bf16) overwrites S_j in TMEM
 //   O  += P_j C_j            tcgen05.mma M = 256, TMEM x smem (C is the MN-major B operand) -> TMEM
 // The running maximum is only raised when it grows by more than 2^8 (the accumulators stay in
-// range and O needs rescaling on few tiles); O is divided by the row sum at the end and written
-// as bf16 to L[B, n_q, N, d_l].  The ring and the score pipeline run on across items.  The lower
+// range and O needs rescaling on few tiles); O is divided by the row sum at the end, staged in
+// shared memory as bf16 and written to L[B, n_q, N, d_l] with TMA tensor stores (whole 128-byte
+// lines, clipped at the sequence end, off the load/store units).  The ring and the score pipeline run on across items.  The lower
 // query tile of a pair sees one fully masked key tile per item (its probabilities are zero).
 constexpr int kAttnThreads = 64 + 512;   // TMA warp, MMA warp, 16 softmax warps
-constexpr int kAttnStages = 4;
+constexpr int kAttnStages = 3;
 constexpr int kKeyTile = 128;
 constexpr int kSlice = 256;
 constexpr uint32_t kQBytes = 128 * 128 * 2;                 // 32 KB: this CTA's query tile
@@ -43,9 +44,11 @@ constexpr uint32_t kKHalfBytes = (kKeyTile / 2) * 128 * 2;  // 16 KB: this CTA's
 constexpr uint32_t kCHalfBytes = kKeyTile * (kSlice / 2) * 2;   // 32 KB: this CTA's 128 latent columns
 constexpr uint32_t kAttnStageBytes = kKHalfBytes + kCHalfBytes;   // 48 KB
 constexpr uint32_t kAttnRingOff = kQBytes;
-constexpr uint32_t kAttnXchgOff = kAttnRingOff + kAttnStages * kAttnStageBytes;   // 2 KB, per lane quarter: bf16 [2][4][32] or float [4][32]
+constexpr uint32_t kAttnOutOff = kAttnRingOff + kAttnStages * kAttnStageBytes;   // 32 KB: two 128 x 64 output boxes
+constexpr uint32_t kAttnOutBoxBytes = 128 * 64 * 2;
+constexpr uint32_t kAttnXchgOff = kAttnOutOff + 2 * kAttnOutBoxBytes;   // 2 KB, per lane quarter: bf16 [2][4][32] or float [4][32]
 constexpr uint32_t kAttnBarOff = kAttnXchgOff + 2 * 4 * 2 * 32 * 4;
-constexpr uint32_t kAttnAlignSlack = 768;   // the 227 KB limit leaves no more; checked in the kernel
+constexpr uint32_t kAttnAlignSlack = 1024;  // checked in the kernel
 constexpr uint32_t kAttnSmemTotal = kAttnBarOff + 256 + kAttnAlignSlack;
 static_assert(kAttnSmemTotal <= 232448, "attention kernel shared memory exceeds the per-CTA limit");
 
@@ -76,6 +79,9 @@ __device__ __forceinline__ void poly_exp2_pair(uint64_t x2, float& p0, float& p1
 }
 // which of every eight pairs of exponentials run on the FMA pipe instead of the MUFU unit
 __device__ constexpr bool kPolyPair[8] = {false, false, true, false, false, true, false, true};
+__device__ __forceinline__ void softmax_sync() {   // all 16 softmax warps
+    asm volatile("bar.sync 5, 512;" ::: "memory");
+}
 __device__ __forceinline__ void quarter_sync(int quarter) {   // the four softmax warps of a TMEM lane quarter
     asm volatile("bar.sync %0, 128;" ::"r"(quarter + 1) : "memory");
 }
@@ -100,7 +106,7 @@ __device__ __forceinline__ bool attn_item(const Dims& d, int n_qt, int n_qp, int
 
 __global__ void __launch_bounds__(kAttnThreads, 1)
 sm100_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
-                       const __grid_constant__ CUtensorMap tm_c, Dims d, __nv_bfloat16* __restrict__ o_lat,
+                       const __grid_constant__ CUtensorMap tm_c, const __grid_constant__ CUtensorMap tm_o, Dims d,
                        int32_t* status_word) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -121,9 +127,6 @@ sm100_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = ptx::cluster_ctarank();          // 0 = leader
     const int G = gridDim.x >> 1, pr = blockIdx.x >> 1;    // CTA pairs, this pair
-    // the decoder + gate kernel may be scheduled as SMs free up: its gate phase does not need L, and
-    // it waits for this whole grid before it reads L
-    ptx::grid_launch_dependents();
     const bool bad_align = (uint32_t)(smem - smem_raw) > kAttnAlignSlack;   // cannot happen with a 256-byte aligned window
     const int n_slices = d.d_l / kSlice;
     const int n_qt = (d.N + 127) / 128, n_qp = (n_qt + 1) / 2;
@@ -139,7 +142,6 @@ sm100_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         *abort_flag = 0;
         *drain_flag = 0;
         ptx::fence_mbar_init();
-        if (bad_align) raise_status(status_word, GTA_ERR_CUDA);
     }
     if (warp == 1) ptx::tmem_alloc_pair(tmem_slot, 512);
     ptx::tc_fence_before_sync();
@@ -147,6 +149,13 @@ sm100_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     ptx::cluster_arrive();     // the peer's barriers exist before anything is signalled to them
     ptx::cluster_wait();
     ptx::tc_fence_after_sync();
+    // The kernel is launched with programmatic stream serialisation: everything above may have run
+    // while the kernel before it in the stream was draining; nothing of global memory is touched
+    // before this wait.  Only then may the decoder + gate kernel be scheduled (as SMs free up): its
+    // gate phase reads X and W_G before its own wait, which orders it against this kernel alone.
+    ptx::grid_dependency_wait();
+    ptx::grid_launch_dependents();
+    if (threadIdx.x == 0 && bad_align) raise_status(status_word, GTA_ERR_CUDA);
     const uint32_t tmem_base = *tmem_slot;
     const uint32_t tmem_o = tmem_base + 256;
 
@@ -259,15 +268,18 @@ sm100_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         const uint32_t o_free_leader = ptx::map_to_cta(ptx::smem_addr(o_free), 0);
         __nv_bfloat16* xm = reinterpret_cast<__nv_bfloat16*>(xchg);   // [4 quarters][2][4][32] partial row maxima
         float* xl = xchg + quarter * 128;                             // [4][32] partial row sums (item end)
+        const bool store_issuer = warp == 2 && lane == 0;
+        // A wait that gives up raises the CTA's abort flag, after which every wait returns at once:
+        // these warps then run their loops to the end all the same (on meaningless data), so that
+        // the named barriers below are always reached by all of their threads.
         bool ok = true;
         int tj = 0;
         AttnItem w;
-        for (int n = 0; ok && attn_item(d, n_qt, n_qp, n_slices, total, G, pr, n, &w); ++n) {
+        for (int n = 0; attn_item(d, n_qt, n_qp, n_slices, total, G, pr, n, &w); ++n) {
             const int t = (2 * w.qp + (int)rank) * 128 + row;
             float m = -INFINITY, l = 0.f;            // m in scaled (log2) units; l = this thread's share of the row sum
-            for (int j = 0; j < w.n_tiles && ok; ++j, ++tj) {
+            for (int j = 0; j < w.n_tiles; ++j, ++tj) {
                 ok = __all_sync(0xffffffffu, ptx::mbar_wait(&s_full[tj & 1], (tj >> 1) & 1, abort_flag));
-                if (!ok) break;   // warp-uniform: the TMEM instructions below are warp-collective
                 ptx::tc_fence_after_sync();
                 const uint32_t s_tmem = tmem_base + lane_base + (tj & 1) * 128;
                 float sv[32];
@@ -334,7 +346,6 @@ sm100_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                     // rescaled: a parity wait is only meaningful one phase at a time, and the
                     // epilogue's wait below must not find the barrier two phases behind.
                     ok = __all_sync(0xffffffffu, ptx::mbar_wait(o_done, (tj - 1) & 1, abort_flag));
-                    if (!ok) break;
                     if (__any_sync(0xffffffffu, raise)) {
                         ptx::tc_fence_after_sync();
 #pragma unroll 1
@@ -359,39 +370,52 @@ sm100_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                 __syncwarp();
                 if (lane == 0) ptx::mbar_arrive_cluster(p_full_leader[tj & 1]);
             }
-            if (!ok) break;
             // ---- item epilogue: whole row sum, normalise, store this thread's 64 columns
             quarter_sync(quarter);                   // everybody has read the last tile's partial maxima
             xl[part * 32 + lane] = l;
             quarter_sync(quarter);
             const float inv_l = 1.f / ((xl[lane] + xl[32 + lane]) + (xl[64 + lane] + xl[96 + lane]));
             ok = __all_sync(0xffffffffu, ptx::mbar_wait(o_done, (tj - 1) & 1, abort_flag));
-            if (!ok) break;
             ptx::tc_fence_after_sync();
-            __nv_bfloat16* o_row = o_lat + (((size_t)w.b * d.n_q + w.g) * d.N + (t < d.N ? t : 0)) * d.d_l +
-                                   w.slice * kSlice + part * 64;
+            // Two passes of 128 columns: thread (row, part) takes columns 32 part .. 32 part + 31 of
+            // the pass, rounds them to bf16 into the staging boxes (box = 64 columns x 128 rows,
+            // 128-byte swizzle: 16-byte chunk c of row r sits at chunk c ^ (r & 7)), and one thread
+            // stores the two boxes with TMA.
+            const int q0 = (2 * w.qp + (int)rank) * 128;
+            uint8_t* box_row = smem + kAttnOutOff + (part >> 1) * kAttnOutBoxBytes + row * 128;
 #pragma unroll 1
-            for (int ch = 0; ch < 2; ++ch) {
+            for (int pass = 0; pass < 2; ++pass) {
                 uint32_t r[32];
-                ptx::tmem_ld32(tmem_o + lane_base + part * 64 + ch * 32, r);
+                ptx::tmem_ld32(tmem_o + lane_base + pass * 128 + part * 32, r);
                 ptx::tmem_wait_ld();
-                if (t < d.N) {
+                if (pass == 1) {      // O has been read completely: the next item's sums may start
+                    ptx::tc_fence_before_sync();
+                    __syncwarp();
+                    if (lane == 0) ptx::mbar_arrive_cluster(o_free_leader);
+                }
+                uint32_t pk[16];
 #pragma unroll
-                    for (int v = 0; v < 2; ++v) {      // 2 x 32 bytes: whole sectors, half as many stores
-                        uint32_t ww[8];
+                for (int e = 0; e < 16; ++e)
+                    pk[e] = pack_bf16x2(__uint_as_float(r[2 * e]) * inv_l, __uint_as_float(r[2 * e + 1]) * inv_l);
+                if (store_issuer) ptx::bulk_wait_group_read_all();   // the stores before have read the boxes
+                softmax_sync();
 #pragma unroll
-                        for (int e = 0; e < 8; ++e)
-                            ww[e] = pack_bf16x2(__uint_as_float(r[16 * v + 2 * e]) * inv_l,
-                                                __uint_as_float(r[16 * v + 2 * e + 1]) * inv_l);
-                        ptx::st_global_256(o_row + ch * 32 + v * 16, ww);
-                    }
+                for (int c = 0; c < 4; ++c) {
+                    const int chunk = ((part & 1) * 4 + c) ^ (row & 7);
+                    *reinterpret_cast<uint4*>(box_row + chunk * 16) =
+                        make_uint4(pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
+                }
+                ptx::fence_proxy_async_smem();
+                softmax_sync();
+                if (store_issuer && q0 < d.N) {
+                    for (int bx = 0; bx < 2; ++bx)
+                        ptx::tma_store_3d(&tm_o, smem + kAttnOutOff + bx * kAttnOutBoxBytes,
+                                          w.slice * kSlice + pass * 128 + bx * 64, q0, w.b * d.n_q + w.g);
+                    ptx::bulk_commit_group();
                 }
             }
-            ptx::tc_fence_before_sync();
-            __syncwarp();
-            if (lane == 0) ptx::mbar_arrive_cluster(o_free_leader);
-            quarter_sync(quarter);   // the exchange area is rewritten by the next item's first tile
         }
+        if (store_issuer) ptx::bulk_wait_group_read_all();   // shared memory stays valid until the stores have read it
     }
     ptx::tc_fence_before_sync();
     __syncthreads();
@@ -410,7 +434,7 @@ gta_status_t launch_sm100_prefill(const Dims& d, const void* q, const void* k, c
                                   const void* w_p, const void* w_g, void* out, void* workspace,
                                   int32_t* status_word, cudaStream_t stream, int stages, int* launches) {
     if (stages & 1) {
-        CUtensorMap tm_q, tm_k, tm_c;
+        CUtensorMap tm_q, tm_k, tm_c, tm_o;
         const uint32_t box[3] = {64, 128, 1}, box_k[3] = {64, 64, 1};
         const uint64_t dq[3] = {(uint64_t)d.d_h, (uint64_t)d.N, (uint64_t)d.B * d.n_q};
         const uint64_t dk[3] = {(uint64_t)d.d_h, (uint64_t)d.N, (uint64_t)d.B * d.n_k};
@@ -418,6 +442,11 @@ gta_status_t launch_sm100_prefill(const Dims& d, const void* q, const void* k, c
         if (!make_bf16_map(&tm_q, q, 3, dq, box) || !make_bf16_map(&tm_k, k, 3, dk, box_k) ||
             !make_bf16_map(&tm_c, c, 3, dc, box))
             return GTA_ERR_CUDA;
+        {   // L [B n_q][N][d_l], stored in boxes of 128 rows x 64 columns
+            const uint64_t dl[3] = {(uint64_t)d.d_l, (uint64_t)d.N, (uint64_t)d.B * d.n_q};
+            const uint32_t box_o[3] = {64, 128, 1};
+            if (!make_bf16_map(&tm_o, workspace, 3, dl, box_o)) return GTA_ERR_CUDA;
+        }
         if (cudaFuncSetAttribute(sm100_attention_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  (int)kAttnSmemTotal) != cudaSuccess)
             return GTA_ERR_CUDA;
@@ -428,13 +457,15 @@ gta_status_t launch_sm100_prefill(const Dims& d, const void* q, const void* k, c
         cfg.blockDim = dim3(kAttnThreads);
         cfg.dynamicSmemBytes = kAttnSmemTotal;
         cfg.stream = stream;
-        cudaLaunchAttribute attr[1];
+        cudaLaunchAttribute attr[2];
         attr[0].id = cudaLaunchAttributeClusterDimension;
         attr[0].val.clusterDim.x = 2;
         attr[0].val.clusterDim.y = 1;
         attr[0].val.clusterDim.z = 1;
+        attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[1].val.programmaticStreamSerializationAllowed = 1;
         cfg.attrs = attr;
-        cfg.numAttrs = 1;
+        cfg.numAttrs = 1;   // the occupancy query below takes the cluster attribute only
         // a persistent grid must be resident at once: as many CTA pairs as the device can hold
         static thread_local int cached_dev = -1, cached_pairs = 0;
         int dev = 0, sms = 0;
@@ -451,7 +482,8 @@ gta_status_t launch_sm100_prefill(const Dims& d, const void* q, const void* k, c
         }
         const int pairs = (int)(n_items < cached_pairs ? n_items : cached_pairs);
         cfg.gridDim = dim3(2 * pairs);
-        if (cudaLaunchKernelEx(&cfg, sm100_attention_kernel, tm_q, tm_k, tm_c, d, (__nv_bfloat16*)workspace,
+        cfg.numAttrs = 2;
+        if (cudaLaunchKernelEx(&cfg, sm100_attention_kernel, tm_q, tm_k, tm_c, tm_o, d,
                                status_word) != cudaSuccess)
             return GTA_ERR_CUDA;
         if (cudaGetLastError() != cudaSuccess) return GTA_ERR_CUDA;
