@@ -53,6 +53,9 @@ SMALL_PREFILL = [
     ("bf16_paper_1b_shape", "bf16", 1, 160, 1280, 20, 5, 1, 1, 64, 128),
     ("f32_general", "f32", 2, 150, 96, 6, 6, 3, 1, 32, 64),
     ("f32_dh128", "f32", 1, 129, 64, 2, 1, 1, 1, 128, 256),
+    # all rows in one 128-row tile: the decoder + gate kernel runs without CTA pairs on half-head items
+    ("bf16_short_batch3_odd_heads", "bf16", 3, 100, 192, 6, 2, 2, 1, 128, 256),
+    ("bf16_short_one_token", "bf16", 5, 1, 128, 4, 4, 4, 1, 128, 512),
 ]
 
 
@@ -157,7 +160,11 @@ SMALL_DECODE = [
     ("bf16_paper_1b_shape", "bf16", 2, 1280, 20, 5, 1, 1, 64, 128, [333, 1000]),
     ("bf16_eight_maps", "bf16", 9, 512, 16, 8, 8, 1, 128, 1024, [257, 256, 255, 1, 2, 1000, 64, 128, 511]),
     ("f32_general", "f32", 3, 96, 6, 6, 3, 1, 32, 64, [100, 7, 260]),
-    # more than 32 sequences: the finish goes through the merge kernel + the tensor-core decoder kernel
+    # more than 16 sequences: the finish goes through the merge kernel + the tensor-core decoder kernel
+    # (without CTA pairs up to 128 sequences, with them above)
+    ("bf16_batch_17", "bf16", 17, 192, 4, 2, 2, 1, 128, 256, [1 + (53 * i) % 400 for i in range(17)]),
+    ("bf16_batch_128", "bf16", 128, 128, 4, 4, 4, 1, 128, 256, [(29 * i) % 150 for i in range(128)]),
+    ("bf16_batch_200", "bf16", 200, 128, 4, 2, 2, 1, 128, 512, [1 + (31 * i) % 90 for i in range(200)]),
     ("bf16_batch_40", "bf16", 40, 256, 8, 4, 4, 1, 128, 512, [1 + (37 * i) % 300 for i in range(40)]),
     ("bf16_batch_33_odd_heads", "bf16", 33, 128, 3, 1, 1, 1, 128, 256, [0 if i == 5 else 1 + (91 * i) % 500 for i in range(33)]),
 ]
