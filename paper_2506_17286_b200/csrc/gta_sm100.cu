@@ -93,12 +93,14 @@ struct AttnItem {
 // alternately left-to-right and right-to-left.  Returns false past the end of the list.
 __device__ __forceinline__ bool attn_item(const Dims& d, int n_qt, int n_qp, int n_slices, long long total, int G,
                                           int pr, int n, AttnItem* it) {
-    const long long p = (long long)n * G + ((n & 1) ? (G - 1 - pr) : pr);
-    if (p >= total) return false;
-    long long r = p;
-    it->slice = (int)(r % n_slices); r /= n_slices;
-    it->g = (int)(r % d.n_q); r /= d.n_q;
-    it->b = (int)(r % d.B); r /= d.B;
+    // the host refuses more than 2^30 items, so 32-bit arithmetic is enough (64-bit divisions are
+    // slow enough to show at every item boundary)
+    const long long p64 = (long long)n * G + ((n & 1) ? (G - 1 - pr) : pr);
+    if (p64 >= total) return false;
+    unsigned r = (unsigned)p64;
+    it->slice = (int)(r % (unsigned)n_slices); r /= (unsigned)n_slices;
+    it->g = (int)(r % (unsigned)d.n_q); r /= (unsigned)d.n_q;
+    it->b = (int)(r % (unsigned)d.B); r /= (unsigned)d.B;
     it->qp = n_qp - 1 - (int)r;
     it->n_tiles = d.causal ? min(2 * it->qp + 2, n_qt) : n_qt;
     return true;
