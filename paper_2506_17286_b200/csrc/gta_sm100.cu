@@ -31,11 +31,13 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
 //                            exchanged through shared memory); P_j (bf16) overwrites S_j in TMEM
 //   O  += P_j C_j            tcgen05.mma M = 256, TMEM x smem (C is the MN-major B operand) -> TMEM
 // The running maximum is only raised when it grows by more than 2^8 (the accumulators stay in
-// range and O needs rescaling on few tiles); O is divided by the row sum at the end, staged in
-// shared memory as bf16 and written to L[B, n_q, N, d_l] with TMA tensor stores (whole 128-byte
-// lines, clipped at the sequence end, off the load/store units).  The ring and the score pipeline run on across items.  The lower
+// range and O needs rescaling on few tiles).  At the end of an item the softmax threads only hand
+// their row sums over: four epilogue warps (one per TMEM lane quarter) divide O by the row sum,
+// stage it in shared memory as bf16 and write it to L[B, n_q, N, d_l] with TMA tensor stores
+// (whole 128-byte lines, clipped at the sequence end), while the softmax threads are already on
+// the first score tile of the next item.  The ring and the score pipeline run on across items.  The lower
 // query tile of a pair sees one fully masked key tile per item (its probabilities are zero).
-constexpr int kAttnThreads = 64 + 512;   // TMA warp, MMA warp, 16 softmax warps
+constexpr int kAttnThreads = 64 + 512 + 128;   // TMA warp, MMA warp, 16 softmax warps, 4 epilogue warps
 constexpr int kAttnStages = 3;
 constexpr int kKeyTile = 128;
 constexpr int kSlice = 256;
@@ -47,7 +49,8 @@ constexpr uint32_t kAttnRingOff = kQBytes;
 constexpr uint32_t kAttnOutOff = kAttnRingOff + kAttnStages * kAttnStageBytes;   // 32 KB: two 128 x 64 output boxes
 constexpr uint32_t kAttnOutBoxBytes = 128 * 64 * 2;
 constexpr uint32_t kAttnXchgOff = kAttnOutOff + 2 * kAttnOutBoxBytes;   // 2 KB, per lane quarter: bf16 [2][4][32] or float [4][32]
-constexpr uint32_t kAttnBarOff = kAttnXchgOff + 2 * 4 * 2 * 32 * 4;
+constexpr uint32_t kAttnSumOff = kAttnXchgOff + 2 * 4 * 2 * 32 * 4;      // 4 KB: float [2 items][4 quarters][4 parts][32] row sums
+constexpr uint32_t kAttnBarOff = kAttnSumOff + 2 * 4 * 4 * 32 * 4;
 constexpr uint32_t kAttnAlignSlack = 1024;  // checked in the kernel
 constexpr uint32_t kAttnSmemTotal = kAttnBarOff + 256 + kAttnAlignSlack;
 static_assert(kAttnSmemTotal <= 232448, "attention kernel shared memory exceeds the per-CTA limit");
@@ -79,8 +82,8 @@ __device__ __forceinline__ void poly_exp2_pair(uint64_t x2, float& p0, float& p1
 }
 // which of every eight pairs of exponentials run on the FMA pipe instead of the MUFU unit
 __device__ constexpr bool kPolyPair[8] = {false, false, true, false, false, true, false, true};
-__device__ __forceinline__ void softmax_sync() {   // all 16 softmax warps
-    asm volatile("bar.sync 5, 512;" ::: "memory");
+__device__ __forceinline__ void epilogue_sync() {   // the four epilogue warps
+    asm volatile("bar.sync 5, 128;" ::: "memory");
 }
 __device__ __forceinline__ void quarter_sync(int quarter) {   // the four softmax warps of a TMEM lane quarter
     asm volatile("bar.sync %0, 128;" ::"r"(quarter + 1) : "memory");
@@ -121,8 +124,10 @@ sm100_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     uint64_t* s_full = bars + 10;       // [2] both CTAs (multicast commit)
     uint64_t* p_full = bars + 12;       // [2] leader CTA; 32 softmax warps arrive
     uint64_t* o_done = bars + 14;       // both CTAs (multicast commit)
-    uint64_t* o_free = bars + 15;       // leader CTA; 32 softmax warps arrive
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 16);
+    uint64_t* o_free = bars + 15;       // leader CTA; 8 epilogue warps arrive
+    uint64_t* epi_ready = bars + 16;    // this CTA; its 16 softmax warps arrive (row sums of an item are in place)
+    uint64_t* o_item = bars + 17;       // both CTAs (multicast commit): the last sum of an item is complete
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 18);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
     volatile int* drain_flag = abort_flag + 1;
 
@@ -140,7 +145,9 @@ sm100_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         for (int s = 0; s < kAttnStages; ++s) { ptx::mbar_init(&full[s], 2); ptx::mbar_init(&empty[s], 1); }
         for (int s = 0; s < 2; ++s) { ptx::mbar_init(&s_full[s], 1); ptx::mbar_init(&p_full[s], 32); }
         ptx::mbar_init(o_done, 1);
-        ptx::mbar_init(o_free, 32);
+        ptx::mbar_init(o_free, 8);
+        ptx::mbar_init(epi_ready, 16);
+        ptx::mbar_init(o_item, 1);
         *abort_flag = 0;
         *drain_flag = 0;
         ptx::fence_mbar_init();
@@ -247,6 +254,7 @@ sm100_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                         ptx::mma_ts_pair(tmem_o, p_tmem + k8 * 8, ptx::make_smem_desc(c_addr + k8 * 2048, 16384, 1024),
                                          idesc_pv, (j > 0 || k8 > 0) ? 1u : 0u);
                     ptx::tc_commit_pair(o_done, 3);
+                    if (j + 1 == w.n_tiles) ptx::tc_commit_pair(o_item, 3);   // for the epilogue warps
                     ptx::tc_commit_pair(&empty[tj % kAttnStages], 3);
                     // ... but the NEXT item's first score tile has to wait for that item's Q, which can
                     // only be requested once this item's last Q K^T is done: it goes after the last P C
@@ -256,7 +264,7 @@ sm100_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                 have = have_next;
             }
         }
-    } else {
+    } else if (warp < 18) {
         // 16 softmax warps: four per TMEM lane quarter (warp % 4), each thread 32 of the 128 keys of its
         // row and 64 of the 256 output columns.  Four warps per scheduler hide the latencies of the
         // TMEM loads, the exchange and the exponentials behind one another.
@@ -267,10 +275,8 @@ sm100_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         const float c_scale = d.scale * 1.4426950408889634f;
         const uint32_t p_full_leader[2] = {ptx::map_to_cta(ptx::smem_addr(&p_full[0]), 0),
                                            ptx::map_to_cta(ptx::smem_addr(&p_full[1]), 0)};
-        const uint32_t o_free_leader = ptx::map_to_cta(ptx::smem_addr(o_free), 0);
         __nv_bfloat16* xm = reinterpret_cast<__nv_bfloat16*>(xchg);   // [4 quarters][2][4][32] partial row maxima
-        float* xl = xchg + quarter * 128;                             // [4][32] partial row sums (item end)
-        const bool store_issuer = warp == 2 && lane == 0;
+        float* xsum = reinterpret_cast<float*>(smem + kAttnSumOff);
         // A wait that gives up raises the CTA's abort flag, after which every wait returns at once:
         // these warps then run their loops to the end all the same (on meaningless data), so that
         // the named barriers below are always reached by all of their threads.
@@ -343,12 +349,12 @@ sm100_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                 // P_j (bf16 pairs): this thread's 32 keys = packed columns [16 part, 16 part + 16) of S_j
                 // (columns that other threads of the row read as scores: they did so before the exchange)
                 ptx::tmem_st16(s_tmem + part * 16, packed);
-                if (j > 0) {
+                if (tj > 0) {
                     // Every completion of o_done is waited for, in order, whether or not O has to be
-                    // rescaled: a parity wait is only meaningful one phase at a time, and the
-                    // epilogue's wait below must not find the barrier two phases behind.
+                    // rescaled (on the first tile of an item it never is): a parity wait is only
+                    // meaningful one phase at a time.
                     ok = __all_sync(0xffffffffu, ptx::mbar_wait(o_done, (tj - 1) & 1, abort_flag));
-                    if (__any_sync(0xffffffffu, raise)) {
+                    if (j > 0 && __any_sync(0xffffffffu, raise)) {
                         ptx::tc_fence_after_sync();
 #pragma unroll 1
                         for (int ch = 0; ch < 2; ++ch) {     // this thread's 64 of the 256 output columns
@@ -372,43 +378,61 @@ sm100_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                 __syncwarp();
                 if (lane == 0) ptx::mbar_arrive_cluster(p_full_leader[tj & 1]);
             }
-            // ---- item epilogue: whole row sum, normalise, store this thread's 64 columns
-            quarter_sync(quarter);                   // everybody has read the last tile's partial maxima
-            xl[part * 32 + lane] = l;
-            quarter_sync(quarter);
-            const float inv_l = 1.f / ((xl[lane] + xl[32 + lane]) + (xl[64 + lane] + xl[96 + lane]));
-            ok = __all_sync(0xffffffffu, ptx::mbar_wait(o_done, (tj - 1) & 1, abort_flag));
+            // ---- end of the item: the row sums go to the epilogue warps (double-buffered by item:
+            //      the epilogue of item n reads them before it hands O back, which the sums of
+            //      item n + 1 wait for, long before item n + 2 ends)
+            xsum[(((n & 1) * 4 + quarter) * 4 + part) * 32 + lane] = l;
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(epi_ready);
+        }
+    } else {
+        // 4 epilogue warps, one per TMEM lane quarter, a row per thread.  After the last sum of an item
+        // (o_item: one completion per item, and the next cannot come before this item's O has been
+        // handed back) they divide O by the row sum, round to bf16 into the staging boxes (box = 64 columns x
+        // 128 rows, 128-byte swizzle: 16-byte chunk c of row r sits at chunk c ^ (r & 7)) and store
+        // them with TMA: two passes of 128 columns.  O is handed back as soon as it has been read.
+        const int quarter = warp & 3;
+        const int row = quarter * 32 + lane;
+        const uint32_t lane_base = ((uint32_t)(quarter * 32) << 16);
+        const uint32_t o_free_leader = ptx::map_to_cta(ptx::smem_addr(o_free), 0);
+        const float* xsum = reinterpret_cast<const float*>(smem + kAttnSumOff);
+        const bool store_issuer = warp == 18 && lane == 0;
+        bool ok = true;      // as for the softmax warps: on a wait that gave up the loops run to their end
+        AttnItem w;
+        for (int n = 0; attn_item(d, n_qt, n_qp, n_slices, total, G, pr, n, &w); ++n) {
+            ok = __all_sync(0xffffffffu, ptx::mbar_wait_backoff(o_item, n & 1, abort_flag, 100));
+            ok = __all_sync(0xffffffffu, ptx::mbar_wait(epi_ready, n & 1, abort_flag));
             ptx::tc_fence_after_sync();
-            // Two passes of 128 columns: thread (row, part) takes columns 32 part .. 32 part + 31 of
-            // the pass, rounds them to bf16 into the staging boxes (box = 64 columns x 128 rows,
-            // 128-byte swizzle: 16-byte chunk c of row r sits at chunk c ^ (r & 7)), and one thread
-            // stores the two boxes with TMA.
+            const float* xs = xsum + ((n & 1) * 4 + quarter) * 128;
+            const float inv_l = 1.f / ((xs[lane] + xs[32 + lane]) + (xs[64 + lane] + xs[96 + lane]));
             const int q0 = (2 * w.qp + (int)rank) * 128;
-            uint8_t* box_row = smem + kAttnOutOff + (part >> 1) * kAttnOutBoxBytes + row * 128;
 #pragma unroll 1
             for (int pass = 0; pass < 2; ++pass) {
-                uint32_t r[32];
-                ptx::tmem_ld32(tmem_o + lane_base + pass * 128 + part * 32, r);
-                ptx::tmem_wait_ld();
+                if (store_issuer) ptx::bulk_wait_group_read_all();   // the stores before have read the boxes
+                epilogue_sync();
+#pragma unroll 1
+                for (int ch = 0; ch < 4; ++ch) {     // 32 columns at a time: box ch / 2, chunks 4 (ch % 2) ..
+                    uint32_t r[32];
+                    ptx::tmem_ld32(tmem_o + lane_base + pass * 128 + ch * 32, r);
+                    ptx::tmem_wait_ld();
+                    uint8_t* box_row = smem + kAttnOutOff + (ch >> 1) * kAttnOutBoxBytes + row * 128;
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        const int chunk = ((ch & 1) * 4 + c) ^ (row & 7);
+                        *reinterpret_cast<uint4*>(box_row + chunk * 16) = make_uint4(
+                            pack_bf16x2(__uint_as_float(r[8 * c]) * inv_l, __uint_as_float(r[8 * c + 1]) * inv_l),
+                            pack_bf16x2(__uint_as_float(r[8 * c + 2]) * inv_l, __uint_as_float(r[8 * c + 3]) * inv_l),
+                            pack_bf16x2(__uint_as_float(r[8 * c + 4]) * inv_l, __uint_as_float(r[8 * c + 5]) * inv_l),
+                            pack_bf16x2(__uint_as_float(r[8 * c + 6]) * inv_l, __uint_as_float(r[8 * c + 7]) * inv_l));
+                    }
+                }
                 if (pass == 1) {      // O has been read completely: the next item's sums may start
                     ptx::tc_fence_before_sync();
                     __syncwarp();
                     if (lane == 0) ptx::mbar_arrive_cluster(o_free_leader);
                 }
-                uint32_t pk[16];
-#pragma unroll
-                for (int e = 0; e < 16; ++e)
-                    pk[e] = pack_bf16x2(__uint_as_float(r[2 * e]) * inv_l, __uint_as_float(r[2 * e + 1]) * inv_l);
-                if (store_issuer) ptx::bulk_wait_group_read_all();   // the stores before have read the boxes
-                softmax_sync();
-#pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    const int chunk = ((part & 1) * 4 + c) ^ (row & 7);
-                    *reinterpret_cast<uint4*>(box_row + chunk * 16) =
-                        make_uint4(pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
-                }
                 ptx::fence_proxy_async_smem();
-                softmax_sync();
+                epilogue_sync();
                 if (store_issuer && q0 < d.N) {
                     for (int bx = 0; bx < 2; ++bx)
                         ptx::tma_store_3d(&tm_o, smem + kAttnOutOff + bx * kAttnOutBoxBytes,
