@@ -46,7 +46,10 @@ constexpr uint32_t kKHalfBytes = (kKeyTile / 2) * 128 * 2;  // 16 KB: this CTA's
 constexpr uint32_t kCHalfBytes = kKeyTile * (kSlice / 2) * 2;   // 32 KB: this CTA's 128 latent columns
 constexpr uint32_t kAttnStageBytes = kKHalfBytes + kCHalfBytes;   // 48 KB
 constexpr uint32_t kAttnRingOff = kQBytes;
-constexpr uint32_t kAttnOutOff = kAttnRingOff + kAttnStages * kAttnStageBytes;   // 32 KB: two 128 x 64 output boxes
+// Two 32 KB buffers alternate between two roles: buffer n & 1 holds the query tile of item n, then
+// (once the item's last Q K^T is done) the two 128 x 64 output boxes of its epilogue, then the query
+// tile of item n + 2.  So the next item's Q is loaded long before the current item ends.
+constexpr uint32_t kAttnOutOff = kAttnRingOff + kAttnStages * kAttnStageBytes;   // the second buffer (the first is at 0)
 constexpr uint32_t kAttnOutBoxBytes = 128 * 64 * 2;
 constexpr uint32_t kAttnXchgOff = kAttnOutOff + 2 * kAttnOutBoxBytes;   // 2 KB, per lane quarter: bf16 [2][4][32] or float [4][32]
 constexpr uint32_t kAttnSumOff = kAttnXchgOff + 2 * 4 * 2 * 32 * 4;      // 4 KB: float [2 items][4 quarters][4 parts][32] row sums
@@ -118,7 +121,7 @@ sm100_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     float* xchg = reinterpret_cast<float*>(smem + kAttnXchgOff);
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kAttnBarOff);
     uint64_t* q_full = bars;            // leader CTA; both producers arrive
-    uint64_t* q_empty = bars + 1;       // both CTAs (multicast commit)
+    uint64_t* stage_free = bars + 1;    // this CTA; its epilogue's stores have read the buffer (one thread arrives)
     uint64_t* full = bars + 2;          // [4] leader CTA; both producers arrive
     uint64_t* empty = bars + 6;         // [4] both CTAs (multicast commit)
     uint64_t* s_full = bars + 10;       // [2] both CTAs (multicast commit)
@@ -141,7 +144,7 @@ sm100_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
 
     if (threadIdx.x == 0) {
         ptx::mbar_init(q_full, 2);
-        ptx::mbar_init(q_empty, 1);
+        ptx::mbar_init(stage_free, 1);
         for (int s = 0; s < kAttnStages; ++s) { ptx::mbar_init(&full[s], 2); ptx::mbar_init(&empty[s], 1); }
         for (int s = 0; s < 2; ++s) { ptx::mbar_init(&s_full[s], 1); ptx::mbar_init(&p_full[s], 32); }
         ptx::mbar_init(o_done, 1);
@@ -178,11 +181,14 @@ sm100_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
             for (int n = 0; ok && attn_item(d, n_qt, n_qp, n_slices, total, G, pr, n, &w); ++n) {
                 const int kg = d.q_to_k(w.g), cg = d.q_to_c(w.g);
                 const int q0 = (2 * w.qp + (int)rank) * 128;       // this CTA's query rows
-                ok = ptx::mbar_wait(q_empty, (n & 1) ^ 1, abort_flag);
+                // buffer n & 1 is free once the epilogue of item n - 2 has stored out of it (which
+                // also means every Q K^T of that item is done); every completion is waited for, in order
+                if (n >= 2) ok = ptx::mbar_wait(stage_free, n & 1, abort_flag);
                 if (!ok) break;
+                uint8_t* q_s = smem + ((n & 1) ? kAttnOutOff : 0u);
                 ptx::mbar_arrive_expect_tx_cluster(q_full_leader, kQBytes);
-                ptx::tma_load_3d_pair(smem, &tm_q, q_full_leader, 0, q0, w.b * d.n_q + w.g);
-                ptx::tma_load_3d_pair(smem + 16384, &tm_q, q_full_leader, 64, q0, w.b * d.n_q + w.g);
+                ptx::tma_load_3d_pair(q_s, &tm_q, q_full_leader, 0, q0, w.b * d.n_q + w.g);
+                ptx::tma_load_3d_pair(q_s + 16384, &tm_q, q_full_leader, 64, q0, w.b * d.n_q + w.g);
                 for (int j = 0; j < w.n_tiles; ++j, ++tj) {
                     const int s = tj % kAttnStages;
                     const uint32_t ph = (tj / kAttnStages) & 1;
@@ -213,14 +219,14 @@ sm100_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         if (rank == 0 && ptx::elect_one()) {
             constexpr uint32_t idesc_qk = ptx::make_idesc_bf16(256, kKeyTile, 0, 0);   // both K-major
             constexpr uint32_t idesc_pv = ptx::make_idesc_bf16(256, kSlice, 0, 1);     // B = C, MN-major
-            const uint32_t q_addr = ptx::smem_addr(smem);
             bool ok = true;
-            // S = Q K^T of ring tile tj; `first` / `last`: first / last key tile of its item n
-            auto issue_qk = [&](int tj, int n, bool first, bool last) {
+            // S = Q K^T of ring tile tj; `first`: first key tile of its item n
+            auto issue_qk = [&](int tj, int n, bool first) {
                 if (first) ok = ptx::mbar_wait(q_full, n & 1, abort_flag);
                 if (ok) ok = ptx::mbar_wait(&full[tj % kAttnStages], (tj / kAttnStages) & 1, abort_flag);
                 if (!ok) return;
                 ptx::tc_fence_after_sync();
+                const uint32_t q_addr = ptx::smem_addr(smem + ((n & 1) ? kAttnOutOff : 0u));
                 const uint32_t k_addr = ptx::smem_addr(smem + kAttnRingOff + (tj % kAttnStages) * kAttnStageBytes);
                 const uint32_t s_tmem = tmem_base + (tj & 1) * 128;
 #pragma unroll
@@ -229,18 +235,25 @@ sm100_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                                      ptx::make_smem_desc(k_addr + (k8 >> 2) * 8192 + (k8 & 3) * 32, 16, 1024), idesc_qk,
                                      k8 ? 1u : 0u);
                 ptx::tc_commit_pair(&s_full[tj & 1], 3);
-                if (last) ptx::tc_commit_pair(q_empty, 3);
             };
             int tj = 0;
             AttnItem w, nxt;
             bool have = attn_item(d, n_qt, n_qp, n_slices, total, G, pr, 0, &w);
-            if (have) issue_qk(0, 0, true, w.n_tiles == 1);
+            if (have) issue_qk(0, 0, true);
             for (int n = 0; have && ok; ++n) {
                 const bool have_next = attn_item(d, n_qt, n_qp, n_slices, total, G, pr, n + 1, &nxt);
                 for (int j = 0; j < w.n_tiles && ok; ++j, ++tj) {
-                    // look ahead: the item's next score tile goes to the tensor pipe before this
-                    // tile's P C, so the softmax warps never wait for scores
-                    if (j + 1 < w.n_tiles) issue_qk(tj + 1, n, false, j + 2 == w.n_tiles);
+                    // look ahead: the next score tile goes to the tensor pipe before this tile's P C, so
+                    // the softmax warps never wait for scores.  Across items too, when the next
+                    // item's Q has landed (it normally has: it is loaded into the other buffer well
+                    // before this item ends); otherwise after this item's last P C, below.
+                    bool next_item_early = false;
+                    if (j + 1 < w.n_tiles) {
+                        issue_qk(tj + 1, n, false);
+                    } else if (have_next && ptx::mbar_test_wait(q_full, (n + 1) & 1)) {
+                        issue_qk(tj + 1, n + 1, true);
+                        next_item_early = true;
+                    }
                     if (!ok) break;
                     ok = ptx::mbar_wait(&p_full[tj & 1], (tj >> 1) & 1, abort_flag);
                     if (ok && j == 0 && n > 0) ok = ptx::mbar_wait(o_free, (n - 1) & 1, abort_flag);
@@ -256,9 +269,8 @@ sm100_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                     ptx::tc_commit_pair(o_done, 3);
                     if (j + 1 == w.n_tiles) ptx::tc_commit_pair(o_item, 3);   // for the epilogue warps
                     ptx::tc_commit_pair(&empty[tj % kAttnStages], 3);
-                    // ... but the NEXT item's first score tile has to wait for that item's Q, which can
-                    // only be requested once this item's last Q K^T is done: it goes after the last P C
-                    if (j + 1 == w.n_tiles && have_next) issue_qk(tj + 1, n + 1, true, nxt.n_tiles == 1);
+                    if (j + 1 == w.n_tiles && have_next && !next_item_early)
+                        issue_qk(tj + 1, n + 1, true);
                 }
                 w = nxt;
                 have = have_next;
@@ -406,42 +418,58 @@ sm100_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
             const float* xs = xsum + ((n & 1) * 4 + quarter) * 128;
             const float inv_l = 1.f / ((xs[lane] + xs[32 + lane]) + (xs[64 + lane] + xs[96 + lane]));
             const int q0 = (2 * w.qp + (int)rank) * 128;
+            const uint64_t inv2 = ptx::f32x2(inv_l, inv_l);
+            uint8_t* stage = smem + ((n & 1) ? kAttnOutOff : 0u);    // the buffer that held this item's Q
+            // Four passes of 64 columns = one box each, the two halves of the buffer used alternately:
+            // a pass only waits for the store of the pass before last.  O is handed back as soon as
+            // its last columns are in registers.
 #pragma unroll 1
-            for (int pass = 0; pass < 2; ++pass) {
-                if (store_issuer) ptx::bulk_wait_group_read_all();   // the stores before have read the boxes
-                epilogue_sync();
+            for (int pass = 0; pass < 4; ++pass) {
+                uint8_t* box_row = stage + (pass & 1) * kAttnOutBoxBytes + row * 128;
+                if (pass >= 2) {
+                    if (store_issuer) ptx::bulk_wait_group_read_but_one();
+                    epilogue_sync();
+                }
 #pragma unroll 1
-                for (int ch = 0; ch < 4; ++ch) {     // 32 columns at a time: box ch / 2, chunks 4 (ch % 2) ..
+                for (int ch = 0; ch < 2; ++ch) {     // 32 columns at a time: 16-byte chunks 4 ch .. 4 ch + 3 of the row
                     uint32_t r[32];
-                    ptx::tmem_ld32(tmem_o + lane_base + pass * 128 + ch * 32, r);
+                    ptx::tmem_ld32(tmem_o + lane_base + pass * 64 + ch * 32, r);
                     ptx::tmem_wait_ld();
-                    uint8_t* box_row = smem + kAttnOutOff + (ch >> 1) * kAttnOutBoxBytes + row * 128;
+                    if (pass == 3 && ch == 1) {      // O has been read completely: the next item's sums may start
+                        ptx::tc_fence_before_sync();
+                        __syncwarp();
+                        if (lane == 0) ptx::mbar_arrive_cluster(o_free_leader);
+                    }
+                    // two-wide multiplies: these warps share their schedulers with the softmax warps,
+                    // and every issue slot they need delays handing O back
+                    uint32_t pk[16];
+#pragma unroll
+                    for (int e = 0; e < 16; ++e) {
+                        float v0, v1;
+                        ptx::f32x2_split(ptx::mul2(ptx::f32x2(__uint_as_float(r[2 * e]), __uint_as_float(r[2 * e + 1])), inv2), v0, v1);
+                        pk[e] = pack_bf16x2(v0, v1);
+                    }
 #pragma unroll
                     for (int c = 0; c < 4; ++c) {
-                        const int chunk = ((ch & 1) * 4 + c) ^ (row & 7);
-                        *reinterpret_cast<uint4*>(box_row + chunk * 16) = make_uint4(
-                            pack_bf16x2(__uint_as_float(r[8 * c]) * inv_l, __uint_as_float(r[8 * c + 1]) * inv_l),
-                            pack_bf16x2(__uint_as_float(r[8 * c + 2]) * inv_l, __uint_as_float(r[8 * c + 3]) * inv_l),
-                            pack_bf16x2(__uint_as_float(r[8 * c + 4]) * inv_l, __uint_as_float(r[8 * c + 5]) * inv_l),
-                            pack_bf16x2(__uint_as_float(r[8 * c + 6]) * inv_l, __uint_as_float(r[8 * c + 7]) * inv_l));
+                        const int chunk = (ch * 4 + c) ^ (row & 7);
+                        *reinterpret_cast<uint4*>(box_row + chunk * 16) =
+                            make_uint4(pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
                     }
-                }
-                if (pass == 1) {      // O has been read completely: the next item's sums may start
-                    ptx::tc_fence_before_sync();
-                    __syncwarp();
-                    if (lane == 0) ptx::mbar_arrive_cluster(o_free_leader);
                 }
                 ptx::fence_proxy_async_smem();
                 epilogue_sync();
                 if (store_issuer && q0 < d.N) {
-                    for (int bx = 0; bx < 2; ++bx)
-                        ptx::tma_store_3d(&tm_o, smem + kAttnOutOff + bx * kAttnOutBoxBytes,
-                                          w.slice * kSlice + pass * 128 + bx * 64, q0, w.b * d.n_q + w.g);
+                    ptx::tma_store_3d(&tm_o, stage + (pass & 1) * kAttnOutBoxBytes, w.slice * kSlice + pass * 64, q0,
+                                      w.b * d.n_q + w.g);
                     ptx::bulk_commit_group();
                 }
             }
+            // the buffer may take the query tile of item n + 2 once the stores have read it
+            if (store_issuer) {
+                ptx::bulk_wait_group_read_all();
+                ptx::mbar_arrive(stage_free);
+            }
         }
-        if (store_issuer) ptx::bulk_wait_group_read_all();   // shared memory stays valid until the stores have read it
     }
     ptx::tc_fence_before_sync();
     __syncthreads();
