@@ -187,6 +187,24 @@ def run_reference(args):
     return 0
 
 
+# ----------------------------------------------------------------------------- ranks
+def max_over_ranks(value, dist=None, device="cpu"):
+    """The largest of `value` over all ranks of the default process group (every rank gets it); the
+    value itself without a process group.  Times of a multi-GPU run are reduced with this."""
+    if dist is None:
+        return float(value)
+    import torch
+    t = torch.tensor([float(value)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_rate(work_per_rank, world, ms):
+    """Aggregate rate of `world` independent replicas that each did `work_per_rank` in `ms`
+    milliseconds (the maximum over ranks): replicas only, no collective on the path."""
+    return world * work_per_rank / (ms * 1e-3)
+
+
 # ----------------------------------------------------------------------------- our arm
 def run_ours(args):
     import torch
@@ -352,22 +370,18 @@ def run_ours(args):
     t_decode_leg = sum(e[2].elapsed_time(e[4]) for e in ev) / K
     t_decode = sum(e[3].elapsed_time(e[4]) for e in ev) / K
 
-    def max_over_ranks(v):
-        if dist is None:
-            return v
-        t = torch.tensor([v], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+    def max_over_ranks_(v):
+        return max_over_ranks(v, dist, dev)
 
-    total_ms = max_over_ranks(total_ms)
-    t_attn, t_dec_k, t_prefill = max_over_ranks(t_attn), max_over_ranks(t_dec_k), max_over_ranks(t_prefill)
-    t_decode, t_decode_leg = max_over_ranks(t_decode), max_over_ranks(t_decode_leg)
-    t_decode_b2b = max_over_ranks(t_decode_b2b)
-    t_decode_call = max_over_ranks(t_decode_call)
+    total_ms = max_over_ranks_(total_ms)
+    t_attn, t_dec_k, t_prefill = max_over_ranks_(t_attn), max_over_ranks_(t_dec_k), max_over_ranks_(t_prefill)
+    t_decode, t_decode_leg = max_over_ranks_(t_decode), max_over_ranks_(t_decode_leg)
+    t_decode_b2b = max_over_ranks_(t_decode_b2b)
+    t_decode_call = max_over_ranks_(t_decode_call)
 
     fl = prefill_flops(wp)
     by = decode_bytes(wd, [wd.seq] * wd.batch)
-    value = world * fl["total"] / (t_prefill * 1e-3) / 1e12
+    value = whole_job_rate(fl["total"], world, t_prefill) / 1e12
     path = G.prefill_path(shape_p)
 
     # ---- roofline of the dominant prefill kernel, and of the decode call
@@ -461,7 +475,7 @@ def run_ours(args):
         e2e_serial_step()
     b.record(stream)
     barrier()
-    e2e_serial_ms = max_over_ranks(a.elapsed_time(b) / e2e_steps)
+    e2e_serial_ms = max_over_ranks_(a.elapsed_time(b) / e2e_steps)
     e2e_run(4)
     barrier()
     a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -469,7 +483,7 @@ def run_ours(args):
     e2e_run(e2e_steps)
     b.record(stream)
     barrier()
-    e2e_ms = max_over_ranks(a.elapsed_time(b) / e2e_steps)
+    e2e_ms = max_over_ranks_(a.elapsed_time(b) / e2e_steps)
     assert int(status.item()) == 0, "device status word raised during the benchmark"
     e2e = {"value": world * fl["total"] / (e2e_ms * 1e-3) / 1e12, "unit": UNIT, "h2d_bytes_per_step": h2d,
            "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms, "steps": e2e_steps,
