@@ -1,4 +1,4 @@
-// tcgen05 / TMA decoder + gate kernel of the bf16 prefill path (d_h = 128):
+// tcgen05 / TMA decoder + gate kernel of the bf16 prefill path (d_h = 64 or 128):
 //     out_i = (L_{q(i)} W_P,i) (.) sigmoid(X W_G,i)          (Sec. 3.3, reformulated equation)
 //
 // Persistent CTA pairs (clusters of 2, tcgen05 cta_group::2): a pair walks a static list of work
@@ -62,12 +62,14 @@ __device__ __forceinline__ float sigmoid_tanh(float z) {
     return fmaf(0.5f, t, 0.5f);
 }
 
-// Static schedule.  U units (256 rows x head pair, or x single head when a map has an odd number
-// of heads) over G CTA pairs: every pair takes q = U / G whole units; the r = U mod G left over are
-// cut in two single-head halves when that makes the tail shorter (2 r <= G), else handed out whole.
+// Static schedule.  The output columns of a token (n_h d_h of them, head after head) are cut in
+// blocks of 256 -- or 128 where the heads of an attention map do not fill a multiple of 256 -- that
+// never straddle two maps.  U units (256 rows x column block) over G CTA pairs: every pair takes
+// q = U / G whole units; the r = U mod G left over are cut in two halves (128 columns) when that
+// makes the tail shorter (2 r <= G), else handed out whole.
 struct Schedule {
-    int n_hp;       // units per row tile (head pairs, heads, or (without CTA pairs) half heads)
-    int pair;       // 1: a unit is two heads
+    int n_hp;       // column blocks per row tile
+    int pair;       // 1: a block is 256 columns (else 128; 64 without CTA pairs)
     int RT;         // 256-row tiles per sequence
     int q, r, split_tail;
     int n_stages;        // ring depth
@@ -75,7 +77,7 @@ struct Schedule {
 };
 
 struct Item {
-    int b, t0, i0, hc, nt;   // batch entry, first token row, first head, first column inside it, columns
+    int b, t0, f0, nt;   // batch entry, first token row, first output column (of n_h d_h), columns
 };
 
 __device__ __forceinline__ int items_of_pair(const Schedule& s, int pr) {
@@ -93,20 +95,18 @@ __device__ __forceinline__ Item item_of(const Schedule& s, int pr, int G, int n)
     const int hp = u % s.n_hp;
     const int rt = (u / s.n_hp) % s.RT;
     it.b = u / (s.n_hp * s.RT);
-    it.hc = 0;
-    if (!kPair) {            // half a head on one CTA
+    if (!kPair) {            // 64 columns on one CTA
         it.t0 = rt * kTileM;
-        it.i0 = hp >> 1;
-        it.hc = (hp & 1) * 64;
+        it.f0 = hp * 64;
         it.nt = 64;
         return it;
     }
     it.t0 = rt * 2 * kTileM;
     if (s.pair) {
-        it.i0 = 2 * hp + (half < 0 ? 0 : half);
+        it.f0 = 256 * hp + (half < 0 ? 0 : 128 * half);
         it.nt = half < 0 ? 256 : 128;
     } else {
-        it.i0 = hp;
+        it.f0 = 128 * hp;
         it.nt = 128;
     }
     return it;
@@ -181,8 +181,11 @@ sm100_decoder_kernel(const __grid_constant__ CUtensorMap tm_l, const __grid_cons
                 const int t0 = w.t0 + (int)rank * kTileM;          // this CTA's rows
                 const int n_grp = kPair ? w.nt / 128 : w.nt / 64;  // 64-column groups this CTA stages
                 const int col0 = (int)rank * (w.nt / 2);           // first of this CTA's columns inside the item
-                const int head = w.i0 + col0 / 128, hcol = w.hc + col0 % 128;
-                const int g = d.head_to_q(w.i0);
+                const int fc = w.f0 + col0;                         // this CTA's first output column
+                const int g = d.head_to_q(w.f0 / d.d_h);           // a block never straddles two maps
+                // head and column inside it of the (up to two) 64-column groups this CTA stages
+                const int wp_head[2] = {fc / d.d_h, (fc + 64) / d.d_h};
+                const int wp_col[2] = {fc % d.d_h, (fc + 64) % d.d_h};
                 const uint32_t tx = a_tile_bytes + (uint32_t)n_grp * kBGroupBytes;
                 for (int ks = 0; ks < ks_total; ++ks, ++it, s = (s + 1 == n_stages) ? 0 : s + 1, ph ^= (s == 0)) {
                     ok = ptx::mbar_wait(&empty_bar[s], ph ^ 1, abort_flag);
@@ -195,15 +198,14 @@ sm100_decoder_kernel(const __grid_constant__ CUtensorMap tm_l, const __grid_cons
                         if (ks < ks_g) {
                             ptx::tma_load_3d(a_s, &tm_x, bar, ks * kBlockK, t0, w.b);
                             for (int grp = 0; grp < n_grp; ++grp)
-                                ptx::tma_load_2d(b_s + grp * kBGroupBytes, &tm_wg, bar, head * 128 + hcol + grp * 64,
-                                                 ks * kBlockK);
+                                ptx::tma_load_2d(b_s + grp * kBGroupBytes, &tm_wg, bar, fc + grp * 64, ks * kBlockK);
                         } else {
                             const int kk = ks - ks_g;
                             if (!l_ready) { ptx::grid_dependency_wait(); l_ready = true; }
                             ptx::tma_load_3d(a_s, &tm_l, bar, kk * kBlockK, t0, w.b * d.n_q + g);
                             for (int grp = 0; grp < n_grp; ++grp)
-                                ptx::tma_load_3d(b_s + grp * kBGroupBytes, &tm_wp, bar, hcol + grp * 64, kk * kBlockK,
-                                                 head);
+                                ptx::tma_load_3d(b_s + grp * kBGroupBytes, &tm_wp, bar, wp_col[grp], kk * kBlockK,
+                                                 wp_head[grp]);
                         }
                         continue;
                     }
@@ -212,8 +214,7 @@ sm100_decoder_kernel(const __grid_constant__ CUtensorMap tm_l, const __grid_cons
                     if (ks < ks_g) {
                         ptx::tma_load_3d_pair(a_s, &tm_x, bar, ks * kBlockK, t0, w.b);
                         for (int grp = 0; grp < n_grp; ++grp)
-                            ptx::tma_load_2d_pair(b_s + grp * kBGroupBytes, &tm_wg, bar, head * 128 + hcol + grp * 64,
-                                                  ks * kBlockK);
+                            ptx::tma_load_2d_pair(b_s + grp * kBGroupBytes, &tm_wg, bar, fc + grp * 64, ks * kBlockK);
                     } else {
                         const int kk = ks - ks_g;
                         // L comes from the kernel before this one in the stream; this kernel is
@@ -222,8 +223,8 @@ sm100_decoder_kernel(const __grid_constant__ CUtensorMap tm_l, const __grid_cons
                         if (!l_ready) { ptx::grid_dependency_wait(); l_ready = true; }
                         ptx::tma_load_3d_pair(a_s, &tm_l, bar, kk * kBlockK, t0, w.b * d.n_q + g);
                         for (int grp = 0; grp < n_grp; ++grp)
-                            ptx::tma_load_3d_pair(b_s + grp * kBGroupBytes, &tm_wp, bar, hcol + grp * 64, kk * kBlockK,
-                                                  head);
+                            ptx::tma_load_3d_pair(b_s + grp * kBGroupBytes, &tm_wp, bar, wp_col[grp], kk * kBlockK,
+                                                  wp_head[grp]);
                     }
                 }
             }
@@ -314,8 +315,8 @@ sm100_decoder_kernel(const __grid_constant__ CUtensorMap tm_l, const __grid_cons
             ok = __all_sync(0xffffffffu, ptx::mbar_wait(accp_full, n & 1, abort_flag));
             if (!ok) break;
             ptx::tc_fence_after_sync();
-            // columns [c0, c0 + cols) of the item = head i0 + (c0 / 128), columns (c0 % 128) ..
-            __nv_bfloat16* o_row = out + (((size_t)w.b * d.N + (t < d.N ? t : 0)) * d.n_h + w.i0) * 128 + w.hc + c0;
+            // columns [c0, c0 + cols) of the item = output columns f0 + c0 .. of the token (head after head)
+            __nv_bfloat16* o_row = out + ((size_t)w.b * d.N + (t < d.N ? t : 0)) * ((size_t)d.n_h * d.d_h) + w.f0 + c0;
 #pragma unroll
             for (int ch = 0; ch < 4; ++ch) {
                 if (ch * 32 < cols) {
@@ -414,7 +415,7 @@ gta_status_t launch_sm100_decoder(const Dims& d, const void* l_bf16, const void*
         const uint32_t smem_bytes = (uint32_t)s.n_stages * (s.a_bytes + kBGroupBytes) + kBarBytes + 1024;
         cfg.dynamicSmemBytes = smem_bytes;
         s.pair = 0;
-        s.n_hp = 2 * d.n_h;
+        s.n_hp = d.n_h * d.d_h / 64;
         s.RT = 1;
         const long long U = (long long)d.B * s.n_hp;
         if (U > 0x3fffffffLL) return GTA_ERR_UNSUPPORTED;
@@ -438,8 +439,10 @@ gta_status_t launch_sm100_decoder(const Dims& d, const void* l_bf16, const void*
     Schedule s;
     s.n_stages = kDecStages;
     s.a_bytes = kATileBytes;
-    s.pair = (d.n_h / d.n_q) % 2 == 0 ? 1 : 0;
-    s.n_hp = s.pair ? d.n_h / 2 : d.n_h;
+    const int map_cols = (d.n_h / d.n_q) * d.d_h;      // output columns of one attention map
+    if (map_cols % 128 != 0) return GTA_ERR_UNSUPPORTED;
+    s.pair = map_cols % 256 == 0 ? 1 : 0;
+    s.n_hp = d.n_h * d.d_h / (s.pair ? 256 : 128);
     s.RT = (d.N + 2 * kTileM - 1) / (2 * kTileM);
     long long U = (long long)d.B * s.RT * s.n_hp;
     if (U > 0x3fffffffLL) return GTA_ERR_UNSUPPORTED;
@@ -467,9 +470,9 @@ gta_status_t launch_sm100_decoder(const Dims& d, const void* l_bf16, const void*
         cached_pairs = n;
     }
     const int pairs = cached_pairs;
-    if (s.pair && 2 * U <= pairs) {   // few units (e.g. a decode batch): single heads keep twice as many SMs busy
+    if (s.pair && 2 * U <= pairs) {   // few units: 128-column blocks keep twice as many SMs busy
         s.pair = 0;
-        s.n_hp = d.n_h;
+        s.n_hp *= 2;
         U *= 2;
     }
     const int G = U < pairs ? (int)U : pairs;
