@@ -40,7 +40,7 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
 constexpr int kAttnThreads = 64 + 512 + 128;   // TMA warp, MMA warp, 16 softmax warps, 4 epilogue warps
 constexpr int kAttnStages = 3;
 constexpr int kKeyTile = 128;
-constexpr int kSlice = 256;
+constexpr int kSlice = 256;      // widest latent slice of an item (template parameter SLICE: 256 or 128)
 constexpr uint32_t kQBytes = 128 * 128 * 2;                 // 32 KB: this CTA's query tile
 constexpr uint32_t kKHalfBytes = (kKeyTile / 2) * 128 * 2;  // 16 KB: this CTA's 64 keys
 constexpr uint32_t kCHalfBytes = kKeyTile * (kSlice / 2) * 2;   // 32 KB: this CTA's 128 latent columns
@@ -112,6 +112,9 @@ __device__ __forceinline__ bool attn_item(const Dims& d, int n_qt, int n_qp, int
     return true;
 }
 
+// DH: head dimension of Q and K (64 or 128); SLICE: latent columns per item (128 or 256).  The
+// shared-memory layout is the one of the largest case; the smaller ones use the front of each area.
+template <int DH, int SLICE>
 __global__ void __launch_bounds__(kAttnThreads, 1)
 sm100_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                        const __grid_constant__ CUtensorMap tm_c, const __grid_constant__ CUtensorMap tm_o, Dims d,
@@ -138,7 +141,10 @@ sm100_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     const uint32_t rank = ptx::cluster_ctarank();          // 0 = leader
     const int G = gridDim.x >> 1, pr = blockIdx.x >> 1;    // CTA pairs, this pair
     const bool bad_align = (uint32_t)(smem - smem_raw) > kAttnAlignSlack;   // cannot happen with a 256-byte aligned window
-    const int n_slices = d.d_l / kSlice;
+    constexpr uint32_t kQLoadBytes = 128 * DH * 2;                 // this CTA's query tile
+    constexpr uint32_t kKLoadBytes = (kKeyTile / 2) * DH * 2;      // this CTA's 64 keys
+    constexpr uint32_t kCLoadBytes = kKeyTile * (SLICE / 2) * 2;   // this CTA's SLICE / 2 latent columns
+    const int n_slices = d.d_l / SLICE;
     const int n_qt = (d.N + 127) / 128, n_qp = (n_qt + 1) / 2;
     const long long total = bad_align ? 0 : (long long)n_qp * n_slices * d.n_q * d.B;
 
@@ -186,9 +192,9 @@ sm100_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                 if (n >= 2) ok = ptx::mbar_wait(stage_free, n & 1, abort_flag);
                 if (!ok) break;
                 uint8_t* q_s = smem + ((n & 1) ? kAttnOutOff : 0u);
-                ptx::mbar_arrive_expect_tx_cluster(q_full_leader, kQBytes);
+                ptx::mbar_arrive_expect_tx_cluster(q_full_leader, kQLoadBytes);
                 ptx::tma_load_3d_pair(q_s, &tm_q, q_full_leader, 0, q0, w.b * d.n_q + w.g);
-                ptx::tma_load_3d_pair(q_s + 16384, &tm_q, q_full_leader, 64, q0, w.b * d.n_q + w.g);
+                if (DH == 128) ptx::tma_load_3d_pair(q_s + 16384, &tm_q, q_full_leader, 64, q0, w.b * d.n_q + w.g);
                 for (int j = 0; j < w.n_tiles; ++j, ++tj) {
                     const int s = tj % kAttnStages;
                     const uint32_t ph = (tj / kAttnStages) & 1;
@@ -197,13 +203,14 @@ sm100_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                     uint8_t* k_s = smem + kAttnRingOff + s * kAttnStageBytes;
                     uint8_t* c_s = k_s + kKHalfBytes;
                     const uint32_t bar = ptx::map_to_cta(ptx::smem_addr(&full[s]), 0);
-                    ptx::mbar_arrive_expect_tx_cluster(bar, kAttnStageBytes);
+                    ptx::mbar_arrive_expect_tx_cluster(bar, kKLoadBytes + kCLoadBytes);
                     const int key0 = j * kKeyTile + (int)rank * 64;         // this CTA's 64 keys of the tile
                     ptx::tma_load_3d_pair(k_s, &tm_k, bar, 0, key0, w.b * d.n_k + kg);
-                    ptx::tma_load_3d_pair(k_s + 8192, &tm_k, bar, 64, key0, w.b * d.n_k + kg);
-                    const int col0 = w.slice * kSlice + (int)rank * 128;     // this CTA's 128 latent columns
+                    if (DH == 128) ptx::tma_load_3d_pair(k_s + 8192, &tm_k, bar, 64, key0, w.b * d.n_k + kg);
+                    const int col0 = w.slice * SLICE + (int)rank * (SLICE / 2);     // this CTA's latent columns
                     ptx::tma_load_3d_pair(c_s, &tm_c, bar, col0, j * kKeyTile, w.b * d.n_c + cg);
-                    ptx::tma_load_3d_pair(c_s + 16384, &tm_c, bar, col0 + 64, j * kKeyTile, w.b * d.n_c + cg);
+                    if (SLICE == 256)
+                        ptx::tma_load_3d_pair(c_s + 16384, &tm_c, bar, col0 + 64, j * kKeyTile, w.b * d.n_c + cg);
                 }
             }
             if (*abort_flag && rank == 0) {   // drain what was armed (bounded), so no copy lands after exit
@@ -218,7 +225,7 @@ sm100_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     } else if (warp == 1) {
         if (rank == 0 && ptx::elect_one()) {
             constexpr uint32_t idesc_qk = ptx::make_idesc_bf16(256, kKeyTile, 0, 0);   // both K-major
-            constexpr uint32_t idesc_pv = ptx::make_idesc_bf16(256, kSlice, 0, 1);     // B = C, MN-major
+            constexpr uint32_t idesc_pv = ptx::make_idesc_bf16(256, SLICE, 0, 1);      // B = C, MN-major
             bool ok = true;
             // S = Q K^T of ring tile tj; `first`: first key tile of its item n
             auto issue_qk = [&](int tj, int n, bool first) {
@@ -230,7 +237,7 @@ sm100_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                 const uint32_t k_addr = ptx::smem_addr(smem + kAttnRingOff + (tj % kAttnStages) * kAttnStageBytes);
                 const uint32_t s_tmem = tmem_base + (tj & 1) * 128;
 #pragma unroll
-                for (int k8 = 0; k8 < 8; ++k8)
+                for (int k8 = 0; k8 < DH / 16; ++k8)
                     ptx::mma_ss_pair(s_tmem, ptx::make_smem_desc(q_addr + (k8 >> 2) * 16384 + (k8 & 3) * 32, 16, 1024),
                                      ptx::make_smem_desc(k_addr + (k8 >> 2) * 8192 + (k8 & 3) * 32, 16, 1024), idesc_qk,
                                      k8 ? 1u : 0u);
@@ -369,9 +376,9 @@ sm100_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                     if (j > 0 && __any_sync(0xffffffffu, raise)) {
                         ptx::tc_fence_after_sync();
 #pragma unroll 1
-                        for (int ch = 0; ch < 2; ++ch) {     // this thread's 64 of the 256 output columns
+                        for (int ch = 0; ch < SLICE / 128; ++ch) {     // this thread's quarter of the output columns
                             uint32_t r[32];
-                            ptx::tmem_ld32(tmem_o + lane_base + part * 64 + ch * 32, r);
+                            ptx::tmem_ld32(tmem_o + lane_base + part * (SLICE / 4) + ch * 32, r);
                             ptx::tmem_wait_ld();
                             const uint64_t a2 = ptx::f32x2(alpha, alpha);
 #pragma unroll
@@ -381,7 +388,7 @@ sm100_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                                 r[e] = __float_as_uint(v0);
                                 r[e + 1] = __float_as_uint(v1);
                             }
-                            ptx::tmem_st32(tmem_o + lane_base + part * 64 + ch * 32, r);
+                            ptx::tmem_st32(tmem_o + lane_base + part * (SLICE / 4) + ch * 32, r);
                         }
                     }
                 }
@@ -424,7 +431,7 @@ sm100_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
             // a pass only waits for the store of the pass before last.  O is handed back as soon as
             // its last columns are in registers.
 #pragma unroll 1
-            for (int pass = 0; pass < 4; ++pass) {
+            for (int pass = 0; pass < SLICE / 64; ++pass) {
                 uint8_t* box_row = stage + (pass & 1) * kAttnOutBoxBytes + row * 128;
                 if (pass >= 2) {
                     if (store_issuer) ptx::bulk_wait_group_read_but_one();
@@ -435,7 +442,7 @@ sm100_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                     uint32_t r[32];
                     ptx::tmem_ld32(tmem_o + lane_base + pass * 64 + ch * 32, r);
                     ptx::tmem_wait_ld();
-                    if (pass == 3 && ch == 1) {      // O has been read completely: the next item's sums may start
+                    if (pass == SLICE / 64 - 1 && ch == 1) {      // O has been read completely: the next item's sums may start
                         ptx::tc_fence_before_sync();
                         __syncwarp();
                         if (lane == 0) ptx::mbar_arrive_cluster(o_free_leader);
@@ -459,7 +466,7 @@ sm100_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                 ptx::fence_proxy_async_smem();
                 epilogue_sync();
                 if (store_issuer && q0 < d.N) {
-                    ptx::tma_store_3d(&tm_o, stage + (pass & 1) * kAttnOutBoxBytes, w.slice * kSlice + pass * 64, q0,
+                    ptx::tma_store_3d(&tm_o, stage + (pass & 1) * kAttnOutBoxBytes, w.slice * SLICE + pass * 64, q0,
                                       w.b * d.n_q + w.g);
                     ptx::bulk_commit_group();
                 }
@@ -481,7 +488,54 @@ sm100_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
 
 // --------------------------------------------------------------------------- host side
 bool sm100_prefill_supported(const Dims& d, int dtype) {
-    return dtype == GTA_BF16 && d.d_h == 128 && d.d_l % 256 == 0 && d.d_l <= 1024 && d.H % 64 == 0 && d.N >= 1;
+    // the decoder + gate kernel cuts the output columns in blocks of at least 128 inside one attention map
+    const bool blocks_ok = d.n_q > 0 && ((d.n_h / d.n_q) * d.d_h) % 128 == 0;
+    return dtype == GTA_BF16 && (d.d_h == 128 || d.d_h == 64) && d.d_l % 128 == 0 && d.d_l <= 1024 &&
+           d.H % 64 == 0 && d.N >= 1 && blocks_ok;
+}
+
+// One instantiation of the attention kernel: its occupancy (asked once per device) and its launch.
+template <int DH, int SLICE>
+static gta_status_t launch_attention(const Dims& d, const CUtensorMap& tm_q, const CUtensorMap& tm_k,
+                                     const CUtensorMap& tm_c, const CUtensorMap& tm_o, int32_t* status_word,
+                                     cudaStream_t stream) {
+    auto kern = sm100_attention_kernel<DH, SLICE>;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAttnSmemTotal) != cudaSuccess)
+        return GTA_ERR_CUDA;
+    const int n_qt = (d.N + 127) / 128, n_qp = (n_qt + 1) / 2;
+    const long long n_items = (long long)n_qp * (d.d_l / SLICE) * d.n_q * d.B;
+    if (n_items > 0x3fffffffLL) return GTA_ERR_UNSUPPORTED;
+    cudaLaunchConfig_t cfg = {};
+    cfg.blockDim = dim3(kAttnThreads);
+    cfg.dynamicSmemBytes = kAttnSmemTotal;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;   // the occupancy query below takes the cluster attribute only
+    // a persistent grid must be resident at once: as many CTA pairs as the device can hold
+    static thread_local int cached_dev = -1, cached_pairs = 0;
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return GTA_ERR_CUDA;
+    if (dev != cached_dev) {
+        if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 2)
+            return GTA_ERR_CUDA;
+        cfg.gridDim = dim3(2 * (sms / 2));
+        int n = 0;
+        if (cudaOccupancyMaxActiveClusters(&n, kern, &cfg) != cudaSuccess || n < 1) return GTA_ERR_CUDA;
+        cached_dev = dev;
+        cached_pairs = n;
+    }
+    const int pairs = (int)(n_items < cached_pairs ? n_items : cached_pairs);
+    cfg.gridDim = dim3(2 * pairs);
+    cfg.numAttrs = 2;
+    if (cudaLaunchKernelEx(&cfg, kern, tm_q, tm_k, tm_c, tm_o, d, status_word) != cudaSuccess) return GTA_ERR_CUDA;
+    return cudaGetLastError() == cudaSuccess ? GTA_OK : GTA_ERR_CUDA;
 }
 
 gta_status_t launch_sm100_prefill(const Dims& d, const void* q, const void* k, const void* c, const void* x,
@@ -501,45 +555,14 @@ gta_status_t launch_sm100_prefill(const Dims& d, const void* q, const void* k, c
             const uint32_t box_o[3] = {64, 128, 1};
             if (!make_bf16_map(&tm_o, workspace, 3, dl, box_o)) return GTA_ERR_CUDA;
         }
-        if (cudaFuncSetAttribute(sm100_attention_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 (int)kAttnSmemTotal) != cudaSuccess)
-            return GTA_ERR_CUDA;
-        const int n_qt = (d.N + 127) / 128, n_qp = (n_qt + 1) / 2;
-        const long long n_items = (long long)n_qp * (d.d_l / kSlice) * d.n_q * d.B;
-        if (n_items > 0x3fffffffLL) return GTA_ERR_UNSUPPORTED;
-        cudaLaunchConfig_t cfg = {};
-        cfg.blockDim = dim3(kAttnThreads);
-        cfg.dynamicSmemBytes = kAttnSmemTotal;
-        cfg.stream = stream;
-        cudaLaunchAttribute attr[2];
-        attr[0].id = cudaLaunchAttributeClusterDimension;
-        attr[0].val.clusterDim.x = 2;
-        attr[0].val.clusterDim.y = 1;
-        attr[0].val.clusterDim.z = 1;
-        attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-        attr[1].val.programmaticStreamSerializationAllowed = 1;
-        cfg.attrs = attr;
-        cfg.numAttrs = 1;   // the occupancy query below takes the cluster attribute only
-        // a persistent grid must be resident at once: as many CTA pairs as the device can hold
-        static thread_local int cached_dev = -1, cached_pairs = 0;
-        int dev = 0, sms = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess) return GTA_ERR_CUDA;
-        if (dev != cached_dev) {
-            if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 2)
-                return GTA_ERR_CUDA;
-            cfg.gridDim = dim3(2 * (sms / 2));
-            int n = 0;
-            if (cudaOccupancyMaxActiveClusters(&n, sm100_attention_kernel, &cfg) != cudaSuccess || n < 1)
-                return GTA_ERR_CUDA;
-            cached_dev = dev;
-            cached_pairs = n;
-        }
-        const int pairs = (int)(n_items < cached_pairs ? n_items : cached_pairs);
-        cfg.gridDim = dim3(2 * pairs);
-        cfg.numAttrs = 2;
-        if (cudaLaunchKernelEx(&cfg, sm100_attention_kernel, tm_q, tm_k, tm_c, tm_o, d,
-                               status_word) != cudaSuccess)
-            return GTA_ERR_CUDA;
+        gta_status_t st;
+        if (d.d_h == 128)
+            st = d.d_l % 256 == 0 ? launch_attention<128, 256>(d, tm_q, tm_k, tm_c, tm_o, status_word, stream)
+                                  : launch_attention<128, 128>(d, tm_q, tm_k, tm_c, tm_o, status_word, stream);
+        else
+            st = d.d_l % 256 == 0 ? launch_attention<64, 256>(d, tm_q, tm_k, tm_c, tm_o, status_word, stream)
+                                  : launch_attention<64, 128>(d, tm_q, tm_k, tm_c, tm_o, status_word, stream);
+        if (st != GTA_OK) return st;
         if (cudaGetLastError() != cudaSuccess) return GTA_ERR_CUDA;
         *launches += 1;
     }

@@ -56,6 +56,10 @@ SMALL_PREFILL = [
     # all rows in one 128-row tile: the decoder + gate kernel runs without CTA pairs on half-head items
     ("bf16_short_batch3_odd_heads", "bf16", 3, 100, 192, 6, 2, 2, 1, 128, 256),
     ("bf16_short_one_token", "bf16", 5, 1, 128, 4, 4, 4, 1, 128, 512),
+    # head dimension 64 and 128-column latent slices on the tensor-core path
+    ("bf16_dh64_dl256_long", "bf16", 2, 700, 192, 8, 2, 1, 1, 64, 256),
+    ("bf16_dh128_dl128", "bf16", 1, 400, 128, 4, 2, 2, 1, 128, 128),
+    ("bf16_dh64_dl384_two_latents", "bf16", 1, 300, 128, 4, 2, 2, 2, 64, 384),
 ]
 
 
