@@ -86,8 +86,10 @@ typedef struct {
  *     the normalised latent attention output L between the two kernels; contents undefined
  *     afterwards.  Calls that share a workspace must be ordered on one stream.
  * Arithmetic: fp32 accumulation everywhere.  bf16 fast path (tcgen05 tensor cores) when
- * dtype = bf16, d_h = 128, d_l a multiple of 256, H a multiple of 64; other shapes and fp32
- * run on the plain-ALU kernels of the same library.  N = 0 or B = 0 is a no-op (GTA_OK).
+ * dtype = bf16, d_h = 64 or 128, d_l a multiple of 128 (at most 1024), H a multiple of 64 and
+ * the heads of one attention map fill a multiple of 128 output columns ((n_h / n_q) d_h);
+ * other shapes and fp32 run on the plain-ALU kernels of the same library (gta_prefill_path
+ * tells which).  N = 0 or B = 0 is a no-op (GTA_OK).
  */
 GTA_API size_t gta_prefill_workspace_bytes(const gta_shape_t *shape);
 GTA_API gta_status_t gta_prefill(const gta_shape_t *shape, const void *q, const void *k, const void *c,

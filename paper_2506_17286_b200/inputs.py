@@ -48,6 +48,9 @@ CONFIGS = {
     "c4_long_prefill_bf16": Workload("c4_long_prefill_bf16", "prefill", "bf16", 1, 16384, 4096, 32, 8, 8, 1, 128, 1024, seed=1004),
     "c5_ragged_decode_bf16": Workload("c5_ragged_decode_bf16", "decode", "bf16", 128, 0, 4096, 32, 8, 8, 1, 128, 1024,
                                       ctx_min=1024, ctx_max=32768, seed=1005),
+    # beyond the five: the layer shape of the paper's 1B model (20 heads in 5 maps sharing one key
+    # group and one latent group, d_h = 64, d_l = 128, H = 1280; cache 192 elements per token)
+    "x1_gta1b_prefill_bf16": Workload("x1_gta1b_prefill_bf16", "prefill", "bf16", 8, 2048, 1280, 20, 5, 1, 1, 64, 128, seed=1011),
 }
 
 

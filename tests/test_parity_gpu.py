@@ -135,6 +135,13 @@ def test_prefill_config4_full_size_sampled_rows(B, oracle):
     _prefill_case(B, oracle, w, rows=_sample_rows(w.seq, 40, seed=4))
 
 
+def test_prefill_paper_1b_layer_shape_full_size_sampled_rows(B, oracle):
+    # 20 heads in 5 maps over one key group and one latent group, d_h = 64, d_l = 128: the tensor-core
+    # path with 64-wide heads, 128-column slices and several items per CTA pair
+    w = I.CONFIGS["x1_gta1b_prefill_bf16"]
+    _prefill_case(B, oracle, w, rows=_sample_rows(w.seq, 48, seed=11))
+
+
 # --------------------------------------------------------------------------- decode
 def _decode_case(B, oracle, w, seq_lens=None, s_cap=None, sample=None):
     t = I.decode_inputs(w, device="cuda", s_cap=s_cap, seq_lens=seq_lens)
