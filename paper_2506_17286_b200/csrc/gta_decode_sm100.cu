@@ -57,10 +57,16 @@ static size_t align256f(size_t v) { return (v + 255) & ~(size_t)255; }
 static int finish_split(const Dims& d);
 
 bool decode_fast_supported(const Dims& d, int dtype) {
-    if (dtype != GTA_BF16 || d.d_h != 128 || d.n_c != 1) return false;
-    if (d.d_l != 256 && d.d_l != 512 && d.d_l != 1024) return false;
-    if (d.n_q != 1 && d.n_q != 2 && d.n_q != 4 && d.n_q != 8) return false;
-    if (d.B > kStreamMaxBatch || finish_split(d) == 0) return false;
+    if (dtype != GTA_BF16 || (d.d_h != 128 && d.d_h != 64) || d.n_c != 1) return false;
+    if (d.d_l != 128 && d.d_l != 256 && d.d_l != 512 && d.d_l != 1024) return false;
+    if (d.n_q < 1 || d.n_q > 8) return false;                    // the maps are the rows of the warp-level MMAs
+    if (d.n_k != 1 && d.n_k != 2 && d.n_k != 4 && d.n_k != 8) return false;   // key groups are dealt to the 8 warps
+    if (d.H % 64 != 0 || d.B > kStreamMaxBatch) return false;
+    // the finish: clusters (small batches; written for d_h = 128, power-of-two map counts, d_l >= 256), else the
+    // merge kernel + the tcgen05 decoder kernel, which cuts the output columns in blocks inside one attention map
+    const bool clusters = d.B <= kFinMaxBatchClusters && d.d_h == 128 && d.d_l >= 256 && (d.n_q & (d.n_q - 1)) == 0;
+    if (clusters && finish_split(d) == 0) return false;
+    if (!clusters && ((d.n_h / d.n_q) * d.d_h) % (d.B > 128 ? 128 : 64) != 0) return false;
     const int tok_bytes = (d.n_k * d.d_h + d.d_l) * 2;
     return tok_bytes * 16 <= kStreamStageBytes;
 }
@@ -110,9 +116,11 @@ __device__ __forceinline__ int clamp_len(int len, int S_cap) { return len < 0 ? 
 
 // Shared-memory layout of one ring stage (all tiles are [T rows][64 bf16] = T x 128 bytes with
 // the 128-byte TMA swizzle: the 16-byte chunk c of row r sits at chunk c ^ (r & 7)):
-//   K tiles : key group kg, half h (columns 64 h .. 64 h + 63)  at (2 kg + h) T 128
+//   K tiles : key group kg, half h (columns 64 h .. 64 h + 63)  at (KH kg + h) T 128
 //   C tiles : latent columns 64 j .. 64 j + 63                   at c_off + j T 128
-template <int NT>   // NT = d_l / 64 = MMA n-tiles (8 latent columns each) per consumer warp
+// NT = d_l / 64 = MMA n-tiles (8 latent columns each) per consumer warp; KH = d_h / 64 = 64-column
+// tiles per key row
+template <int NT, int KH>
 __global__ void __launch_bounds__(kStreamThreads, 1)
 decode_stream_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_c, Dims d,
                      int T, int S_cap, const __nv_bfloat16* __restrict__ q, const int32_t* __restrict__ seq_lens,
@@ -188,7 +196,7 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
         b0 = lo;
     }
     const uint32_t tile_bytes = (uint32_t)T * 128;
-    const uint32_t c_off = (uint32_t)d.n_k * 2 * tile_bytes;
+    const uint32_t c_off = (uint32_t)d.n_k * KH * tile_bytes;
     const uint32_t stage_tx = c_off + (uint32_t)NT * tile_bytes;
 
     if (warp == kStreamConsumers / 32) {
@@ -197,7 +205,7 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
         // to 32) tensor loads of the sub-tile, so that issuing them does not pace the stream.
         {
             const uint64_t policy = ptx::l2_evict_first_policy();
-            const int n_k_ops = 2 * d.n_k;
+            const int n_k_ops = KH * d.n_k;
             int b = b0;
             long long k = st_begin - prefix[b0];
             int it = 0;
@@ -216,8 +224,8 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
                 uint8_t* stage = ring + s * kStreamStageBytes;
                 for (int op = lane; op < n_k_ops + NT; op += 32) {
                     if (op < n_k_ops)
-                        ptx::tma_load_3d_hint(stage + op * tile_bytes, &tm_k, &full_bar[s], (op & 1) * 64, tok0,
-                                              b * d.n_k + (op >> 1), policy);
+                        ptx::tma_load_3d_hint(stage + op * tile_bytes, &tm_k, &full_bar[s], (op % KH) * 64, tok0,
+                                              b * d.n_k + op / KH, policy);
                     else
                         ptx::tma_load_3d_hint(stage + c_off + (op - n_k_ops) * tile_bytes, &tm_c, &full_bar[s],
                                               (op - n_k_ops) * 64, tok0, b, policy);
@@ -245,13 +253,13 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
         float acc[NT][4];
 #pragma unroll
         for (int n = 0; n < NT; ++n) acc[n][0] = acc[n][1] = acc[n][2] = acc[n][3] = 0.f;
-        uint32_t qa[8][2];                                // A fragments of Q for key group kg_w
+        uint32_t qa[4 * KH][2];                           // A fragments of Q for key group kg_w
 
         auto load_q = [&](int b) {
             const uint32_t* qrow =
-                reinterpret_cast<const uint32_t*>(q + ((size_t)b * NQ + kg_w * qpk + (quad < qpk ? quad : 0)) * 128);
+                reinterpret_cast<const uint32_t*>(q + ((size_t)b * NQ + kg_w * qpk + (quad < qpk ? quad : 0)) * (64 * KH));
 #pragma unroll
-            for (int ks = 0; ks < 8; ++ks) {
+            for (int ks = 0; ks < 4 * KH; ++ks) {
                 qa[ks][0] = quad < qpk ? __ldg(qrow + 8 * ks + sub) : 0u;
                 qa[ks][1] = quad < qpk ? __ldg(qrow + 8 * ks + 4 + sub) : 0u;
             }
@@ -298,11 +306,11 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
             for (int u = warp; u < n_units; u += 8) {
                 const int nt = u / d.n_k;
                 const int token = nt * 8 + mrow;
-                const uint32_t krow = stage + (uint32_t)(2 * kg_w) * tile_bytes + token * 128;
+                const uint32_t krow = stage + (uint32_t)(KH * kg_w) * tile_bytes + token * 128;
                 float sc[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-                for (int kp = 0; kp < 4; ++kp) {
-                    const int chunk = 4 * kp + mat;     // 16-byte chunk of the 256-byte K row
+                for (int kp = 0; kp < 2 * KH; ++kp) {
+                    const int chunk = 4 * kp + mat;     // 16-byte chunk of the K row (128 KH bytes)
                     uint32_t k0, k1, k2, k3;
                     ptx::ldsm_x4(krow + (chunk >> 3) * tile_bytes + (((chunk & 7) ^ (token & 7)) << 4), k0, k1, k2, k3);
                     ptx::mma_bf16_16816(sc, qa[2 * kp][0], 0u, qa[2 * kp][1], 0u, k0, k1);
@@ -838,21 +846,21 @@ cudaError_t launch_decode_fast(const Dims& d, const void* q, const void* k_cache
     float* part_o = reinterpret_cast<float*>(workspace);
     float* part_ml = reinterpret_cast<float*>(static_cast<char*>(workspace) + p.off_ml);
     __nv_bfloat16* l_g = reinterpret_cast<__nv_bfloat16*>(static_cast<char*>(workspace) + p.off_l);
-    const bool big_batch = d.B > kFinMaxBatchClusters;
+    const bool big_batch = !(d.B <= kFinMaxBatchClusters && d.d_h == 128 && d.d_l >= 256 && (d.n_q & (d.n_q - 1)) == 0);
     cudaError_t err;
     if (stages & 2) {
         CUtensorMap tm_k, tm_c;
         const uint32_t box[3] = {64, (uint32_t)p.T, 1};
-        const uint64_t dk[3] = {128, (uint64_t)S_cap, (uint64_t)d.B * d.n_k};
+        const uint64_t dk[3] = {(uint64_t)d.d_h, (uint64_t)S_cap, (uint64_t)d.B * d.n_k};
         const uint64_t dc[3] = {(uint64_t)d.d_l, (uint64_t)S_cap, (uint64_t)d.B};
         if (!make_bf16_map(&tm_k, k_cache, 3, dk, box) || !make_bf16_map(&tm_c, c_cache, 3, dc, box))
             return cudaErrorInvalidValue;
         const size_t smem = (size_t)kStreamStages * kStreamStageBytes + 2 * 8 * kStreamMaxT * sizeof(float) +
                             (size_t)(kStreamMaxBatch + 2 + kStreamThreads) * sizeof(int32_t) +
                             2 * kStreamStages * sizeof(uint64_t) + 16 + 1024;
-#define GTA_LAUNCH_STREAM(NT)                                                                              \
+#define GTA_LAUNCH_STREAM_(NT, KH)                                                                         \
         do {                                                                                               \
-            auto kern = decode_stream_kernel<NT>;                                                          \
+            auto kern = decode_stream_kernel<NT, KH>;                                                      \
             err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);      \
             if (err != cudaSuccess) return err;                                                            \
             cudaLaunchConfig_t cfg = {};                                                                   \
@@ -869,12 +877,19 @@ cudaError_t launch_decode_fast(const Dims& d, const void* q, const void* k_cache
                                      seq_lens, part_o, part_ml, status_word);                              \
             if (err != cudaSuccess) return err;                                                            \
         } while (0)
+#define GTA_LAUNCH_STREAM(NT)                                                                              \
+        do {                                                                                               \
+            if (d.d_h == 128) GTA_LAUNCH_STREAM_(NT, 2);                                                   \
+            else GTA_LAUNCH_STREAM_(NT, 1);                                                                \
+        } while (0)
         switch (d.d_l) {
+            case 128: GTA_LAUNCH_STREAM(2); break;
             case 256: GTA_LAUNCH_STREAM(4); break;
             case 512: GTA_LAUNCH_STREAM(8); break;
             default: GTA_LAUNCH_STREAM(16); break;
         }
 #undef GTA_LAUNCH_STREAM
+#undef GTA_LAUNCH_STREAM_
         if ((err = cudaGetLastError()) != cudaSuccess) return err;
         *launches += 1;
     }

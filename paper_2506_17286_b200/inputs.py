@@ -51,6 +51,7 @@ CONFIGS = {
     # beyond the five: the layer shape of the paper's 1B model (20 heads in 5 maps sharing one key
     # group and one latent group, d_h = 64, d_l = 128, H = 1280; cache 192 elements per token)
     "x1_gta1b_prefill_bf16": Workload("x1_gta1b_prefill_bf16", "prefill", "bf16", 8, 2048, 1280, 20, 5, 1, 1, 64, 128, seed=1011),
+    "x2_gta1b_decode_bf16": Workload("x2_gta1b_decode_bf16", "decode", "bf16", 128, 8192, 1280, 20, 5, 1, 1, 64, 128, seed=1012),
 }
 
 

@@ -177,6 +177,11 @@ SMALL_DECODE = [
     ("bf16_batch_128", "bf16", 128, 128, 4, 4, 4, 1, 128, 256, [(29 * i) % 150 for i in range(128)]),
     ("bf16_batch_200", "bf16", 200, 128, 4, 2, 2, 1, 128, 512, [1 + (31 * i) % 90 for i in range(200)]),
     ("bf16_batch_40", "bf16", 40, 256, 8, 4, 4, 1, 128, 512, [1 + (37 * i) % 300 for i in range(40)]),
+    # head dimension 64, latent width 128, map counts that are no power of two, shared keys: the stream kernel's
+    # other instantiations, finished by the merge kernel + the decoder kernel whatever the batch
+    ("bf16_dh64_three_maps_batch_40", "bf16", 40, 192, 6, 3, 1, 1, 64, 128, [1 + (41 * i) % 700 for i in range(40)]),
+    ("bf16_dh64_dl512_small_batch", "bf16", 3, 128, 8, 4, 2, 1, 64, 512, [70, 1, 513]),
+    ("bf16_dh128_five_maps", "bf16", 7, 256, 10, 5, 1, 1, 128, 256, [300, 0, 64, 65, 1000, 17, 2]),
     ("bf16_batch_33_odd_heads", "bf16", 33, 128, 3, 1, 1, 1, 128, 256, [0 if i == 5 else 1 + (91 * i) % 500 for i in range(33)]),
 ]
 
