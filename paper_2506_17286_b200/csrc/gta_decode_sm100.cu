@@ -38,7 +38,7 @@ constexpr int kStreamThreads = kStreamConsumers + 32;
 constexpr int kStreamStages = 3;
 constexpr int kStreamStageBytes = 65536;
 constexpr int kStreamMaxBatch = 512;
-constexpr int kStreamMaxT = 64;
+constexpr int kStreamMaxT = 128;     // tokens per sub-tile: at most 64, or 128 for the narrowest caches (d_l = 128)
 constexpr int kFinBlockB = 32;
 constexpr int kFinThreads = 256;
 constexpr int kFinCols = 64;
@@ -86,7 +86,8 @@ static FastPlan make_fast_plan(const Dims& d) {
     FastPlan p;
     const int tok_bytes = (d.n_k * d.d_h + d.d_l) * 2;
     int t = 16;
-    while (t * 2 * tok_bytes <= kStreamStageBytes && t * 2 <= kStreamMaxT) t *= 2;
+    const int t_max = d.d_l == 128 ? 128 : 64;       // matches the KTM of the stream kernel's instantiation
+    while (t * 2 * tok_bytes <= kStreamStageBytes && t * 2 <= t_max) t *= 2;
     p.T = t;
     p.G = sm_count() < kFinMaxSlots - kStreamMaxBatch ? sm_count() : kFinMaxSlots - kStreamMaxBatch;
     p.slots = p.G + d.B;
@@ -119,8 +120,9 @@ __device__ __forceinline__ int clamp_len(int len, int S_cap) { return len < 0 ? 
 //   K tiles : key group kg, half h (columns 64 h .. 64 h + 63)  at (KH kg + h) T 128
 //   C tiles : latent columns 64 j .. 64 j + 63                   at c_off + j T 128
 // NT = d_l / 64 = MMA n-tiles (8 latent columns each) per consumer warp; KH = d_h / 64 = 64-column
-// tiles per key row
-template <int NT, int KH>
+// tiles per key row; KTM = most 16-token MMA k-steps per sub-tile (sub-tiles of up to 16 KTM tokens:
+// the narrower a cached token, the more tokens a sub-tile needs to be worth its fixed cost)
+template <int NT, int KH, int KTM>
 __global__ void __launch_bounds__(kStreamThreads, 1)
 decode_stream_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_c, Dims d,
                      int T, int S_cap, const __nv_bfloat16* __restrict__ q, const int32_t* __restrict__ seq_lens,
@@ -340,13 +342,13 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
 
             // ---- softmax state of map `quad` (every warp keeps its own copy) and the probability
             //      fragments: lane (quad, sub) holds tokens 16 kt + 2 sub + {0, 1, 8, 9}
-            uint32_t pa[4][2];
+            uint32_t pa[KTM][2];
             float alpha = 1.f;
             {
-                float sv[4][4];
+                float sv[KTM][4];
                 float m_t = -INFINITY;
 #pragma unroll
-                for (int kt = 0; kt < 4; ++kt) {
+                for (int kt = 0; kt < KTM; ++kt) {
                     if (kt < KT && map_lane) {
                         const float2 x = *reinterpret_cast<const float2*>(sb + quad * T + 16 * kt + 2 * sub);
                         const float2 y = *reinterpret_cast<const float2*>(sb + quad * T + 16 * kt + 8 + 2 * sub);
@@ -363,7 +365,7 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
                 alpha = map_lane ? ex2f(m_run - m_new) : 1.f;
                 float sum = 0.f;
 #pragma unroll
-                for (int kt = 0; kt < 4; ++kt) {
+                for (int kt = 0; kt < KTM; ++kt) {
                     const float p0 = ex2f(sv[kt][0] - m_sub), p1 = ex2f(sv[kt][1] - m_sub);
                     const float p2 = ex2f(sv[kt][2] - m_sub), p3 = ex2f(sv[kt][3] - m_sub);
                     sum += (p0 + p1) + (p2 + p3);
@@ -382,7 +384,7 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
             {
                 const uint32_t cbase = stage + c_off;
 #pragma unroll
-                for (int kt = 0; kt < 4; ++kt) {
+                for (int kt = 0; kt < KTM; ++kt) {
                     if (kt < KT) {
                         const int token = 16 * kt + (mat & 1) * 8 + mrow;
                         const uint32_t crow = cbase + token * 128;
@@ -860,7 +862,7 @@ cudaError_t launch_decode_fast(const Dims& d, const void* q, const void* k_cache
                             2 * kStreamStages * sizeof(uint64_t) + 16 + 1024;
 #define GTA_LAUNCH_STREAM_(NT, KH)                                                                         \
         do {                                                                                               \
-            auto kern = decode_stream_kernel<NT, KH>;                                                      \
+            auto kern = decode_stream_kernel<NT, KH, (NT == 2 ? 8 : 4)>;                                   \
             err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);      \
             if (err != cudaSuccess) return err;                                                            \
             cudaLaunchConfig_t cfg = {};                                                                   \
