@@ -98,6 +98,23 @@ GTA_API gta_status_t gta_prefill(const gta_shape_t *shape, const void *q, const 
                          void *cuda_stream);
 
 /*
+ * gta_prefill_chunk — gta_prefill for a chunk of queries against longer keys and latents that
+ * already sit in a cache: the N = shape->seq query tokens are the LAST N of kv_len attended
+ * positions, so with causal = 1 query t attends keys 0 .. t + kv_len - N (the causal sum of
+ * App. B.1.1 over the whole sequence, restricted to the chunk's rows); row t of the result
+ * equals row kv_len - N + t of gta_prefill over all kv_len tokens.
+ *
+ *   q   [B, n_q, N, d_h]          x   [B, N, H]        out [B, N, n_h, d_h]
+ *   k   [B, n_k, kv_cap, d_h]     c   [B, n_c, kv_cap, d_l]    rows 0 .. kv_len-1 are read
+ *   N <= kv_len <= kv_cap (else GTA_ERR_INVALID_ARG); kv_len = kv_cap = N is gta_prefill.
+ * Workspace, weights, arithmetic, paths and errors as for gta_prefill.
+ */
+GTA_API gta_status_t gta_prefill_chunk(const gta_shape_t *shape, int32_t kv_len, int32_t kv_cap,
+                                       const void *q, const void *k, const void *c, const void *x,
+                                       const void *w_p, const void *w_g, void *out, void *workspace,
+                                       size_t workspace_bytes, int32_t *status_word, void *cuda_stream);
+
+/*
  * gta_decode — one decode step (App. B.1.3): for every sequence b the new token's queries
  * attend the seq_lens[b] cached keys / latents (the new token's own entries included, i.e.
  * gta_cache_append has already run), then the decoder and gate of gta_prefill are applied

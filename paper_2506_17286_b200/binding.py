@@ -22,7 +22,7 @@ GTA_F32, GTA_BF16 = 0, 1
 EXPORTS = (
     "gta_prefill_workspace_bytes", "gta_prefill", "gta_decode_workspace_bytes", "gta_decode",
     "gta_cache_append", "gta_status_string", "gta_version", "gta_prefill_path", "gta_last_launch_count",
-    "gta_prefill_stages", "gta_decode_stages", "gta_decode_static",
+    "gta_prefill_stages", "gta_decode_stages", "gta_decode_static", "gta_prefill_chunk",
 )
 
 
@@ -62,6 +62,8 @@ def lib():
         L.gta_prefill.restype = i32
         L.gta_prefill_stages.argtypes = [sp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp, vp, i32]
         L.gta_prefill_stages.restype = i32
+        L.gta_prefill_chunk.argtypes = [sp, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp, vp]
+        L.gta_prefill_chunk.restype = i32
         L.gta_decode_stages.argtypes = [sp, vp, vp, vp, vp, i32, vp, vp, vp, vp, vp, sz, vp, vp, i32]
         L.gta_decode_stages.restype = i32
         L.gta_decode_workspace_bytes.argtypes = [sp, i32]
@@ -168,6 +170,32 @@ def gta_prefill(q, k, c, x, w_p, w_g, *, causal=True, softmax_scale=0.0, out=Non
     st = lib().gta_prefill(*args) if stages == 3 else lib().gta_prefill_stages(*args, stages)
     if st != GTA_OK:
         raise GtaError(st, "gta_prefill")
+    return out
+
+
+def gta_prefill_chunk(q, k, c, x, w_p, w_g, kv_len, *, causal=True, softmax_scale=0.0, out=None, workspace=None,
+                      status_word=None, stream=None):
+    """gta_prefill for the last N of kv_len positions.  q [B,n_q,N,d_h], x [B,N,H]; k [B,n_k,kv_cap,d_h],
+    c [B,n_c,kv_cap,d_l] of which rows 0 .. kv_len-1 are attended."""
+    _check_tensors(q, k, c, x, w_p, w_g)
+    B, n_q, N, d_h = q.shape
+    n_k, kv_cap, n_c, d_l = k.shape[1], k.shape[2], c.shape[1], c.shape[3]
+    n_h, H = w_p.shape[0], x.shape[2]
+    if k.shape != (B, n_k, kv_cap, d_h) or c.shape != (B, n_c, kv_cap, d_l) or x.shape != (B, N, H) \
+            or w_p.shape != (n_h, d_l, d_h) or w_g.shape != (H, n_h * d_h):
+        raise ValueError("inconsistent operator tensor shapes")
+    shape = make_shape(batch=B, seq=N, d_model=H, n_heads=n_h, n_q=n_q, n_k=n_k, n_c=n_c, d_h=d_h, d_l=d_l,
+                       dtype=_dtype_code(q), causal=causal, softmax_scale=softmax_scale)
+    if out is None:
+        out = torch.empty((B, N, n_h, d_h), dtype=q.dtype, device=q.device)
+    need = prefill_workspace_bytes(shape)
+    if workspace is None:
+        workspace = _workspace(need, q.device)
+    st = lib().gta_prefill_chunk(ctypes.byref(shape), int(kv_len), int(kv_cap), _ptr(q), _ptr(k), _ptr(c), _ptr(x),
+                                 _ptr(w_p), _ptr(w_g), _ptr(out), _ptr(workspace),
+                                 workspace.numel() * workspace.element_size(), _ptr(status_word), _stream(stream))
+    if st != GTA_OK:
+        raise GtaError(st, "gta_prefill_chunk")
     return out
 
 

@@ -45,12 +45,19 @@ gta_status_t check_shape(const gta_shape_t* s, bool need_seq, gta::Dims* d) {
     d->n_q = s->n_q_groups; d->n_k = s->n_k_groups; d->n_c = s->n_c_groups;
     d->d_h = s->head_dim; d->d_l = s->latent_dim; d->causal = s->causal;
     d->scale = s->softmax_scale > 0.f ? s->softmax_scale : 1.0f / sqrtf((float)s->head_dim);
+    d->Nk = d->N;
+    d->S = d->N;
     return GTA_OK;
 }
 
 size_t elem_size(int dtype) { return dtype == GTA_F32 ? 4 : 2; }
 
 }  // namespace
+
+static gta_status_t prefill_impl(const gta_shape_t* shape, int32_t kv_len, int32_t kv_cap, const void* q,
+                                 const void* k, const void* c, const void* x, const void* w_p, const void* w_g,
+                                 void* out, void* workspace, size_t workspace_bytes, int32_t* status_word,
+                                 void* cuda_stream, int32_t stages);
 
 extern "C" {
 
@@ -100,11 +107,34 @@ gta_status_t gta_prefill_stages(const gta_shape_t* shape, const void* q, const v
                                 const void* x, const void* w_p, const void* w_g, void* out, void* workspace,
                                 size_t workspace_bytes, int32_t* status_word, void* cuda_stream,
                                 int32_t stages) {
+    if (!shape) return GTA_ERR_INVALID_ARG;
+    return prefill_impl(shape, shape->seq, shape->seq, q, k, c, x, w_p, w_g, out, workspace, workspace_bytes,
+                        status_word, cuda_stream, stages);
+}
+
+gta_status_t gta_prefill_chunk(const gta_shape_t* shape, int32_t kv_len, int32_t kv_cap, const void* q,
+                               const void* k, const void* c, const void* x, const void* w_p, const void* w_g,
+                               void* out, void* workspace, size_t workspace_bytes, int32_t* status_word,
+                               void* cuda_stream) {
+    if (!shape) return GTA_ERR_INVALID_ARG;
+    if (kv_len < shape->seq || kv_cap < kv_len) return GTA_ERR_INVALID_ARG;
+    return prefill_impl(shape, kv_len, kv_cap, q, k, c, x, w_p, w_g, out, workspace, workspace_bytes, status_word,
+                        cuda_stream, 3);
+}
+
+}  // extern "C"
+
+static gta_status_t prefill_impl(const gta_shape_t* shape, int32_t kv_len, int32_t kv_cap, const void* q,
+                                 const void* k, const void* c, const void* x, const void* w_p, const void* w_g,
+                                 void* out, void* workspace, size_t workspace_bytes, int32_t* status_word,
+                                 void* cuda_stream, int32_t stages) {
     g_last_launches = 0;
     if (stages < 1 || stages > 3) return GTA_ERR_INVALID_ARG;
     gta::Dims d;
     gta_status_t st = check_shape(shape, true, &d);
     if (st != GTA_OK) return st;
+    d.Nk = kv_len;
+    d.S = kv_cap;
     if (!q || !k || !c || !x || !w_p || !w_g || !out) return GTA_ERR_INVALID_ARG;
     if (!aligned(q, 16) || !aligned(k, 16) || !aligned(c, 16) || !aligned(x, 16) || !aligned(w_p, 16) ||
         !aligned(w_g, 16) || !aligned(out, 16) || !aligned(status_word, 4))
@@ -130,6 +160,8 @@ gta_status_t gta_prefill_stages(const gta_shape_t* shape, const void* q, const v
     g_last_launches = launches;
     return GTA_OK;
 }
+
+extern "C" {
 
 size_t gta_decode_workspace_bytes(const gta_shape_t* shape, int32_t S_cap) {
     gta::Dims d;

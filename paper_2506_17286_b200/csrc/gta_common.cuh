@@ -13,6 +13,10 @@ namespace gta {
 struct Dims {
     int B, N, H, n_h, n_q, n_k, n_c, d_h, d_l, causal;
     float scale;  // softmax scale, already resolved (1/sqrt(d_h) when the caller passed 0)
+    // Prefill of a chunk against longer K / C (a cache): the N queries are the LAST N of Nk attended
+    // positions (query t sees keys 0 .. t + Nk - N), and K / C rows are S apart per group.  A plain
+    // prefill has Nk = S = N.
+    int Nk, S;
     __host__ __device__ int head_to_q(int i) const { return (int)(((long long)i * n_q) / n_h); }
     __host__ __device__ int q_to_k(int g) const { return (int)(((long long)g * n_k) / n_q); }
     __host__ __device__ int q_to_c(int g) const { return (int)(((long long)g * n_c) / n_q); }

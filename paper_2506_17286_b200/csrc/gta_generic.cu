@@ -23,13 +23,13 @@ generic_attention_kernel(Dims d, const T* __restrict__ q, const T* __restrict__ 
     if (t >= d.N) return;  // no block-wide barrier below
     const int kg = d.q_to_k(g), cg = d.q_to_c(g);
     const T* q_row = q + (((size_t)b * d.n_q + g) * d.N + t) * d.d_h;
-    const T* k_base = k + ((size_t)b * d.n_k + kg) * (size_t)d.N * d.d_h;
-    const T* c_base = c + ((size_t)b * d.n_c + cg) * (size_t)d.N * d.d_l;
+    const T* k_base = k + ((size_t)b * d.n_k + kg) * (size_t)d.S * d.d_h;
+    const T* c_base = c + ((size_t)b * d.n_c + cg) * (size_t)d.S * d.d_l;
     float* qs = q_smem + warp * d.d_h;
     for (int e = lane; e < d.d_h; e += 32) qs[e] = to_f32(q_row[e]);
     __syncwarp();
 
-    const int n_keys = d.causal ? t + 1 : d.N;
+    const int n_keys = d.causal ? t + 1 + (d.Nk - d.N) : d.Nk;
     const int n_acc = (d.d_l + 31) / 32;
     float acc[kMaxAccPerLane];
 #pragma unroll

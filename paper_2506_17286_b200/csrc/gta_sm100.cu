@@ -97,7 +97,7 @@ struct AttnItem {
 
 // Item `n` of CTA pair `pr`: position p in the list sorted by descending query tile, rounds dealt
 // alternately left-to-right and right-to-left.  Returns false past the end of the list.
-__device__ __forceinline__ bool attn_item(const Dims& d, int n_qt, int n_qp, int n_slices, long long total, int G,
+__device__ __forceinline__ bool attn_item(const Dims& d, int n_kt, int n_qp, int n_slices, long long total, int G,
                                           int pr, int n, AttnItem* it) {
     // the host refuses more than 2^30 items, so 32-bit arithmetic is enough (64-bit divisions are
     // slow enough to show at every item boundary)
@@ -108,7 +108,8 @@ __device__ __forceinline__ bool attn_item(const Dims& d, int n_qt, int n_qp, int
     it->g = (int)(r % (unsigned)d.n_q); r /= (unsigned)d.n_q;
     it->b = (int)(r % (unsigned)d.B); r /= (unsigned)d.B;
     it->qp = n_qp - 1 - (int)r;
-    it->n_tiles = d.causal ? min(2 * it->qp + 2, n_qt) : n_qt;
+    // key tiles the pair's 256 query rows see: up to their last row's key (2 qp + 2) 128 - 1 + Nk - N
+    it->n_tiles = d.causal ? min((((2 * it->qp + 2) * 128 - 1 + d.Nk - d.N) >> 7) + 1, n_kt) : n_kt;
     return true;
 }
 
@@ -146,6 +147,7 @@ sm100_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     constexpr uint32_t kCLoadBytes = kKeyTile * (SLICE / 2) * 2;   // this CTA's SLICE / 2 latent columns
     const int n_slices = d.d_l / SLICE;
     const int n_qt = (d.N + 127) / 128, n_qp = (n_qt + 1) / 2;
+    const int n_kt = (d.Nk + 127) / 128;          // key tiles
     const long long total = bad_align ? 0 : (long long)n_qp * n_slices * d.n_q * d.B;
 
     if (threadIdx.x == 0) {
@@ -184,7 +186,7 @@ sm100_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
             int tj = 0;                 // key tiles issued so far (ring position), across items
             bool ok = true;
             AttnItem w;
-            for (int n = 0; ok && attn_item(d, n_qt, n_qp, n_slices, total, G, pr, n, &w); ++n) {
+            for (int n = 0; ok && attn_item(d, n_kt, n_qp, n_slices, total, G, pr, n, &w); ++n) {
                 const int kg = d.q_to_k(w.g), cg = d.q_to_c(w.g);
                 const int q0 = (2 * w.qp + (int)rank) * 128;       // this CTA's query rows
                 // buffer n & 1 is free once the epilogue of item n - 2 has stored out of it (which
@@ -245,10 +247,10 @@ sm100_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
             };
             int tj = 0;
             AttnItem w, nxt;
-            bool have = attn_item(d, n_qt, n_qp, n_slices, total, G, pr, 0, &w);
+            bool have = attn_item(d, n_kt, n_qp, n_slices, total, G, pr, 0, &w);
             if (have) issue_qk(0, 0, true);
             for (int n = 0; have && ok; ++n) {
-                const bool have_next = attn_item(d, n_qt, n_qp, n_slices, total, G, pr, n + 1, &nxt);
+                const bool have_next = attn_item(d, n_kt, n_qp, n_slices, total, G, pr, n + 1, &nxt);
                 for (int j = 0; j < w.n_tiles && ok; ++j, ++tj) {
                     // look ahead: the next score tile goes to the tensor pipe before this tile's P C, so
                     // the softmax warps never wait for scores.  Across items too, when the next
@@ -302,7 +304,7 @@ sm100_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         bool ok = true;
         int tj = 0;
         AttnItem w;
-        for (int n = 0; attn_item(d, n_qt, n_qp, n_slices, total, G, pr, n, &w); ++n) {
+        for (int n = 0; attn_item(d, n_kt, n_qp, n_slices, total, G, pr, n, &w); ++n) {
             const int t = (2 * w.qp + (int)rank) * 128 + row;
             float m = -INFINITY, l = 0.f;            // m in scaled (log2) units; l = this thread's share of the row sum
             for (int j = 0; j < w.n_tiles; ++j, ++tj) {
@@ -319,7 +321,7 @@ sm100_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                 }
                 // mask: keys past the sequence end, and (causal) keys after the query, on boundary tiles
                 const int key0 = j * kKeyTile + part * 32;
-                const int last_key = d.causal ? min(t, d.N - 1) : d.N - 1;
+                const int last_key = d.causal ? min(t + d.Nk - d.N, d.Nk - 1) : d.Nk - 1;
                 if (key0 + 31 > last_key) {
 #pragma unroll
                     for (int e = 0; e < 32; ++e)
@@ -418,7 +420,7 @@ sm100_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         const bool store_issuer = warp == 18 && lane == 0;
         bool ok = true;      // as for the softmax warps: on a wait that gave up the loops run to their end
         AttnItem w;
-        for (int n = 0; attn_item(d, n_qt, n_qp, n_slices, total, G, pr, n, &w); ++n) {
+        for (int n = 0; attn_item(d, n_kt, n_qp, n_slices, total, G, pr, n, &w); ++n) {
             ok = __all_sync(0xffffffffu, ptx::mbar_wait_backoff(o_item, n & 1, abort_flag, 100));
             ok = __all_sync(0xffffffffu, ptx::mbar_wait(epi_ready, n & 1, abort_flag));
             ptx::tc_fence_after_sync();
@@ -545,8 +547,8 @@ gta_status_t launch_sm100_prefill(const Dims& d, const void* q, const void* k, c
         CUtensorMap tm_q, tm_k, tm_c, tm_o;
         const uint32_t box[3] = {64, 128, 1}, box_k[3] = {64, 64, 1};
         const uint64_t dq[3] = {(uint64_t)d.d_h, (uint64_t)d.N, (uint64_t)d.B * d.n_q};
-        const uint64_t dk[3] = {(uint64_t)d.d_h, (uint64_t)d.N, (uint64_t)d.B * d.n_k};
-        const uint64_t dc[3] = {(uint64_t)d.d_l, (uint64_t)d.N, (uint64_t)d.B * d.n_c};
+        const uint64_t dk[3] = {(uint64_t)d.d_h, (uint64_t)d.S, (uint64_t)d.B * d.n_k};
+        const uint64_t dc[3] = {(uint64_t)d.d_l, (uint64_t)d.S, (uint64_t)d.B * d.n_c};
         if (!make_bf16_map(&tm_q, q, 3, dq, box) || !make_bf16_map(&tm_k, k, 3, dk, box_k) ||
             !make_bf16_map(&tm_c, c, 3, dc, box))
             return GTA_ERR_CUDA;

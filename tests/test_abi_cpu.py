@@ -82,6 +82,15 @@ def test_bad_arguments_are_rejected_on_the_host(B):
     assert prefill(_shape(B, seq=0)) == B.GTA_OK                       # empty problem: no-op
     assert prefill(_shape(B, batch=0)) == B.GTA_OK
 
+    def chunk(shape, kv_len, kv_cap):
+        return L.gta_prefill_chunk(ctypes.byref(shape), kv_len, kv_cap, *args, p, 1 << 40, None, None)
+
+    n = good.seq
+    assert chunk(good, n - 1, n) == B.GTA_ERR_INVALID_ARG              # fewer keys than queries
+    assert chunk(good, n + 8, n + 4) == B.GTA_ERR_INVALID_ARG          # more keys than the buffers hold
+    assert L.gta_prefill_chunk(None, 8, 8, *args, p, 1 << 40, None, None) == B.GTA_ERR_INVALID_ARG
+    assert chunk(_shape(B, seq=0), 16, 16) == B.GTA_OK                 # no queries: no-op
+
     def decode(shape, s_cap=128, ws=p, ws_bytes=1 << 40, lens=p):
         return L.gta_decode(ctypes.byref(shape), p, p, p, lens, s_cap, p, p, p, p, ws, ws_bytes, None, None)
 

@@ -142,6 +142,44 @@ def test_prefill_paper_1b_layer_shape_full_size_sampled_rows(B, oracle):
     _prefill_case(B, oracle, w, rows=_sample_rows(w.seq, 48, seed=11))
 
 
+# --------------------------------------------------------------------------- chunked prefill
+CHUNKS = [
+    # name, dtype, B, kv_len, N (queries = the last N positions), kv_cap, H, n_h, n_q, n_k, n_c, d_h, d_l, causal
+    ("bf16_chunk_mid", "bf16", 2, 700, 300, 768, 256, 8, 4, 4, 1, 128, 512, True),
+    ("bf16_chunk_one_query", "bf16", 3, 513, 1, 513, 128, 4, 2, 2, 1, 128, 256, True),
+    ("bf16_chunk_whole", "bf16", 1, 260, 260, 300, 128, 4, 2, 2, 1, 128, 256, True),
+    ("bf16_chunk_dh64", "bf16", 2, 1000, 129, 1024, 192, 8, 2, 1, 1, 64, 128, True),
+    ("bf16_chunk_non_causal", "bf16", 1, 400, 100, 400, 128, 4, 2, 2, 1, 128, 256, False),
+    ("bf16_chunk_plain_alu_shape", "bf16", 2, 300, 77, 320, 128, 6, 6, 3, 1, 32, 64, True),
+    ("f32_chunk", "f32", 1, 200, 50, 256, 96, 6, 6, 3, 1, 32, 64, True),
+]
+
+
+@pytest.mark.parametrize("case", CHUNKS, ids=[c[0] for c in CHUNKS])
+def test_prefill_chunk_against_a_longer_cache(B, oracle, case):
+    """The chunk's rows must equal the same rows of a prefill over all kv_len tokens (oracle); the
+    cache rows past kv_len hold finite garbage that must not be read into the result."""
+    name, dt, nb, kv_len, N, kv_cap, H, n_h, n_q, n_k, n_c, d_h, d_l, causal = case
+    w = I.Workload(name, "prefill", dt, nb, kv_len, H, n_h, n_q, n_k, n_c, d_h, d_l, seed=321)
+    t = I.prefill_inputs(w, device="cuda")
+    first = kv_len - N
+    gen = torch.Generator(device="cuda").manual_seed(5)
+    k = torch.randn((nb, n_k, kv_cap, d_h), generator=gen, device="cuda").to(w.torch_dtype())
+    c = torch.randn((nb, n_c, kv_cap, d_l), generator=gen, device="cuda").to(w.torch_dtype())
+    k[:, :, :kv_len] = t["k"]
+    c[:, :, :kv_len] = t["c"]
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    out = B.gta_prefill_chunk(t["q"][:, :, first:].contiguous(), k, c, t["x"][:, first:].contiguous(), t["w_p"],
+                              t["w_g"], kv_len, causal=causal, status_word=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    tc = cpu(t)
+    rows = list(range(first, kv_len))
+    want = oracle.prefill(oracle_shape(w, causal=int(causal)), tc["q"], tc["k"], tc["c"], tc["x"], tc["w_p"], tc["w_g"],
+                          rows=rows)
+    assert_close(out, want, w.torch_dtype(), name)
+
+
 # --------------------------------------------------------------------------- decode
 def _decode_case(B, oracle, w, seq_lens=None, s_cap=None, sample=None):
     t = I.decode_inputs(w, device="cuda", s_cap=s_cap, seq_lens=seq_lens)
