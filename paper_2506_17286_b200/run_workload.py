@@ -26,6 +26,40 @@ def _median(xs):
     return statistics.median(xs) if xs else 0.0
 
 
+def run_prefill_chunk(w, iters, warmup, kv_len):
+    """The last w.seq positions of a kv_len-token context as one chunk (gta_prefill_chunk)."""
+    dev = torch.device("cuda")
+    t = I.prefill_inputs(w, device=dev)
+    gen = torch.Generator(device=dev).manual_seed(w.seed)
+    k = torch.randn((w.batch, w.n_k, kv_len, w.d_h), generator=gen, device=dev).to(w.torch_dtype())
+    c = torch.randn((w.batch, w.n_c, kv_len, w.d_l), generator=gen, device=dev).to(w.torch_dtype())
+    shape = G.make_shape(batch=w.batch, seq=w.seq, d_model=w.d_model, n_heads=w.n_heads, n_q=w.n_q, n_k=w.n_k,
+                         n_c=w.n_c, d_h=w.d_h, d_l=w.d_l, dtype=w.torch_dtype())
+    ws = torch.zeros(G.prefill_workspace_bytes(shape), dtype=torch.uint8, device=dev)
+    out = torch.empty((w.batch, w.seq, w.n_heads, w.d_h), dtype=w.torch_dtype(), device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    stream = torch.cuda.current_stream()
+
+    def step():
+        G.gta_prefill_chunk(t["q"], k, c, t["x"], t["w_p"], t["w_g"], kv_len, out=out, workspace=ws,
+                            status_word=status)
+
+    for _ in range(warmup):
+        step()
+    torch.cuda.synchronize()
+    times = []
+    for rep in range(3):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(iters):
+            step()
+        e1.record(stream)
+        torch.cuda.synchronize()
+        times.append(e0.elapsed_time(e1) / iters)
+    assert int(status.item()) == 0, "device status word raised"
+    return {"whole_call": _median(times), "kv_len": kv_len}
+
+
 def run_prefill(w, iters, warmup, stages):
     dev = torch.device("cuda")
     t = I.prefill_inputs(w, device=dev)
@@ -128,6 +162,8 @@ def main():
     ap.add_argument("--seq", type=int, default=0)
     ap.add_argument("--stages", type=int, default=7)
     ap.add_argument("--append", action="store_true", help="decode: run gta_cache_append before every step")
+    ap.add_argument("--kv-len", type=int, default=0,
+                    help="prefill: treat the workload's tokens as the last chunk of a context of this length")
     args = ap.parse_args()
     w = I.CONFIGS[args.workload]
     if args.batch:
@@ -136,7 +172,9 @@ def main():
         w = I.scaled(w, seq=args.seq) if w.kind == "prefill" or w.seq > 0 else I.scaled(w, ctx_max=args.seq)
     G.lib()
     torch.cuda.set_device(0)
-    if w.kind == "prefill":
+    if w.kind == "prefill" and args.kv_len > w.seq:
+        res = run_prefill_chunk(w, args.iters, args.warmup, args.kv_len)
+    elif w.kind == "prefill":
         res = run_prefill(w, args.iters, args.warmup, args.stages & 3)
     else:
         res = run_decode(w, args.iters, args.warmup, args.stages, args.append)
