@@ -129,7 +129,7 @@ GTA_API gta_status_t gta_prefill_chunk(const gta_shape_t *shape, int32_t kv_len,
  *     (split-KV partial results and gate partial sums).
  * Needs d_h and d_l multiples of 8 (bf16) / 4 (fp32) so that rows are 16-byte vectors,
  * d_h <= 256, d_l <= 2048.  bf16 fast path (TMA-streamed caches, tensor-core decoder) when
- * d_h = 64 or 128, d_l = 128, 256, 512 or 1024, n_q <= 8, n_k = 1, 2, 4 or 8, n_c = 1, H a
+ * d_h = 64 or 128, d_l = 128, 256, 512 or 1024, n_q <= 8, n_k = 1, 2, 4 or 8, H a
  * multiple of 64, B <= 512 and the heads of one attention map fill a multiple of 64 output
  * columns (128 for B > 128); everything else runs on the plain-ALU kernels.
  */

@@ -57,17 +57,18 @@ static size_t align256f(size_t v) { return (v + 255) & ~(size_t)255; }
 static int finish_split(const Dims& d);
 
 bool decode_fast_supported(const Dims& d, int dtype) {
-    if (dtype != GTA_BF16 || (d.d_h != 128 && d.d_h != 64) || d.n_c != 1) return false;
+    if (dtype != GTA_BF16 || (d.d_h != 128 && d.d_h != 64)) return false;
     if (d.d_l != 128 && d.d_l != 256 && d.d_l != 512 && d.d_l != 1024) return false;
     if (d.n_q < 1 || d.n_q > 8) return false;                    // the maps are the rows of the warp-level MMAs
     if (d.n_k != 1 && d.n_k != 2 && d.n_k != 4 && d.n_k != 8) return false;   // key groups are dealt to the 8 warps
     if (d.H % 64 != 0 || d.B > kStreamMaxBatch) return false;
     // the finish: clusters (small batches; written for d_h = 128, power-of-two map counts, d_l >= 256), else the
     // merge kernel + the tcgen05 decoder kernel, which cuts the output columns in blocks inside one attention map
-    const bool clusters = d.B <= kFinMaxBatchClusters && d.d_h == 128 && d.d_l >= 256 && (d.n_q & (d.n_q - 1)) == 0;
+    const bool clusters = d.B <= kFinMaxBatchClusters && d.d_h == 128 && d.d_l >= 256 && (d.n_q & (d.n_q - 1)) == 0 &&
+                          d.n_c == 1;
     if (clusters && finish_split(d) == 0) return false;
     if (!clusters && ((d.n_h / d.n_q) * d.d_h) % (d.B > 128 ? 128 : 64) != 0) return false;
-    const int tok_bytes = (d.n_k * d.d_h + d.d_l) * 2;
+    const int tok_bytes = (d.n_k * d.d_h + d.n_c * d.d_l) * 2;
     return tok_bytes * 16 <= kStreamStageBytes;
 }
 
@@ -84,7 +85,7 @@ static int sm_count() {
 
 static FastPlan make_fast_plan(const Dims& d) {
     FastPlan p;
-    const int tok_bytes = (d.n_k * d.d_h + d.d_l) * 2;
+    const int tok_bytes = (d.n_k * d.d_h + d.n_c * d.d_l) * 2;
     int t = 16;
     const int t_max = d.d_l == 128 ? 128 : 64;       // matches the KTM of the stream kernel's instantiation
     while (t * 2 * tok_bytes <= kStreamStageBytes && t * 2 <= t_max) t *= 2;
@@ -118,11 +119,12 @@ __device__ __forceinline__ int clamp_len(int len, int S_cap) { return len < 0 ? 
 // Shared-memory layout of one ring stage (all tiles are [T rows][64 bf16] = T x 128 bytes with
 // the 128-byte TMA swizzle: the 16-byte chunk c of row r sits at chunk c ^ (r & 7)):
 //   K tiles : key group kg, half h (columns 64 h .. 64 h + 63)  at (KH kg + h) T 128
-//   C tiles : latent columns 64 j .. 64 j + 63                   at c_off + j T 128
+//   C tiles : latent group cg, columns 64 j .. 64 j + 63         at c_off + (NT cg + j) T 128
 // NT = d_l / 64 = MMA n-tiles (8 latent columns each) per consumer warp; KH = d_h / 64 = 64-column
 // tiles per key row; KTM = most 16-token MMA k-steps per sub-tile (sub-tiles of up to 16 KTM tokens:
 // the narrower a cached token, the more tokens a sub-tile needs to be worth its fixed cost)
-template <int NT, int KH, int KTM>
+// ONE_C: a single latent group (the latent-sum loop then has no group pass and no masking)
+template <int NT, int KH, int KTM, bool ONE_C>
 __global__ void __launch_bounds__(kStreamThreads, 1)
 decode_stream_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_c, Dims d,
                      int T, int S_cap, const __nv_bfloat16* __restrict__ q, const int32_t* __restrict__ seq_lens,
@@ -199,7 +201,8 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
     }
     const uint32_t tile_bytes = (uint32_t)T * 128;
     const uint32_t c_off = (uint32_t)d.n_k * KH * tile_bytes;
-    const uint32_t stage_tx = c_off + (uint32_t)NT * tile_bytes;
+    const int n_c_tiles = ONE_C ? NT : d.n_c * NT;
+    const uint32_t stage_tx = c_off + (uint32_t)n_c_tiles * tile_bytes;
 
     if (warp == kStreamConsumers / 32) {
         // ------------------------------------------------------------------ producer
@@ -224,13 +227,13 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
                 if (!ok) break;
                 const int tok0 = (int)k * T;
                 uint8_t* stage = ring + s * kStreamStageBytes;
-                for (int op = lane; op < n_k_ops + NT; op += 32) {
+                for (int op = lane; op < n_k_ops + n_c_tiles; op += 32) {
                     if (op < n_k_ops)
                         ptx::tma_load_3d_hint(stage + op * tile_bytes, &tm_k, &full_bar[s], (op % KH) * 64, tok0,
                                               b * d.n_k + op / KH, policy);
                     else
                         ptx::tma_load_3d_hint(stage + c_off + (op - n_k_ops) * tile_bytes, &tm_c, &full_bar[s],
-                                              (op - n_k_ops) * 64, tok0, b, policy);
+                                              ((op - n_k_ops) % NT) * 64, tok0, b * d.n_c + (op - n_k_ops) / NT, policy);
                 }
             }
             if (lane == 0 && *abort_flag) {
@@ -329,10 +332,10 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
             // ---- rows past the live length hold whatever the cache holds there: their
             //      probabilities are zero, so the latent rows are cleared (0 x garbage could be NaN)
             if (n_valid < T) {
-                const int vec_per_row = NT * 8;          // 16-byte vectors per latent row
+                const int vec_per_row = n_c_tiles * 8;   // 16-byte vectors per token over all latent groups
                 const int n_vec = (T - n_valid) * vec_per_row;
                 for (int idx = tid; idx < n_vec; idx += kStreamConsumers) {
-                    const int row = n_valid + idx / vec_per_row, v = idx % vec_per_row;
+                    const int row = n_valid + idx / vec_per_row, v = idx % vec_per_row;   // v >> 3 = tile (group, 64 columns)
                     uint8_t* p = ring + s * kStreamStageBytes + c_off + (v >> 3) * tile_bytes + row * 128 + (v & 7) * 16;
                     *reinterpret_cast<uint4*>(p) = make_uint4(0u, 0u, 0u, 0u);
                 }
@@ -380,12 +383,17 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
 #pragma unroll
             for (int n = 0; n < NT; ++n) { acc[n][0] *= alpha; acc[n][1] *= alpha; }
 
-            // ---- latent sums of this warp's d_l / 8 columns, all maps at once: O += P C
-            {
-                const uint32_t cbase = stage + c_off;
+            // ---- latent sums of this warp's d_l / 8 columns, all maps at once: O += P C.  With several
+            //      latent groups, one pass per group with the probabilities of the other groups' maps
+            //      zeroed (a lane's fragment registers belong to its own map's row).
+            const int n_c_loop = ONE_C ? 1 : d.n_c;
+            for (int cg = 0; cg < n_c_loop; ++cg) {
+                const uint32_t cbase = stage + c_off + (uint32_t)(cg * NT) * tile_bytes;
+                const bool mine = ONE_C || d.q_to_c(quad < NQ ? quad : 0) == cg;
 #pragma unroll
                 for (int kt = 0; kt < KTM; ++kt) {
                     if (kt < KT) {
+                        const uint32_t a0 = mine ? pa[kt][0] : 0u, a2 = mine ? pa[kt][1] : 0u;
                         const int token = 16 * kt + (mat & 1) * 8 + mrow;
                         const uint32_t crow = cbase + token * 128;
 #pragma unroll
@@ -394,8 +402,8 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
                             uint32_t c0, c1, c2, c3;
                             ptx::ldsm_x4_trans(crow + (chunk >> 3) * tile_bytes + (((chunk & 7) ^ (token & 7)) << 4),
                                                c0, c1, c2, c3);
-                            ptx::mma_bf16_16816(acc[2 * np], pa[kt][0], 0u, pa[kt][1], 0u, c0, c1);
-                            ptx::mma_bf16_16816(acc[2 * np + 1], pa[kt][0], 0u, pa[kt][1], 0u, c2, c3);
+                            ptx::mma_bf16_16816(acc[2 * np], a0, 0u, a2, 0u, c0, c1);
+                            ptx::mma_bf16_16816(acc[2 * np + 1], a0, 0u, a2, 0u, c2, c3);
                         }
                     }
                 }
@@ -848,21 +856,22 @@ cudaError_t launch_decode_fast(const Dims& d, const void* q, const void* k_cache
     float* part_o = reinterpret_cast<float*>(workspace);
     float* part_ml = reinterpret_cast<float*>(static_cast<char*>(workspace) + p.off_ml);
     __nv_bfloat16* l_g = reinterpret_cast<__nv_bfloat16*>(static_cast<char*>(workspace) + p.off_l);
-    const bool big_batch = !(d.B <= kFinMaxBatchClusters && d.d_h == 128 && d.d_l >= 256 && (d.n_q & (d.n_q - 1)) == 0);
+    const bool big_batch = !(d.B <= kFinMaxBatchClusters && d.d_h == 128 && d.d_l >= 256 &&
+                             (d.n_q & (d.n_q - 1)) == 0 && d.n_c == 1);
     cudaError_t err;
     if (stages & 2) {
         CUtensorMap tm_k, tm_c;
         const uint32_t box[3] = {64, (uint32_t)p.T, 1};
         const uint64_t dk[3] = {(uint64_t)d.d_h, (uint64_t)S_cap, (uint64_t)d.B * d.n_k};
-        const uint64_t dc[3] = {(uint64_t)d.d_l, (uint64_t)S_cap, (uint64_t)d.B};
+        const uint64_t dc[3] = {(uint64_t)d.d_l, (uint64_t)S_cap, (uint64_t)d.B * d.n_c};
         if (!make_bf16_map(&tm_k, k_cache, 3, dk, box) || !make_bf16_map(&tm_c, c_cache, 3, dc, box))
             return cudaErrorInvalidValue;
         const size_t smem = (size_t)kStreamStages * kStreamStageBytes + 2 * 8 * kStreamMaxT * sizeof(float) +
                             (size_t)(kStreamMaxBatch + 2 + kStreamThreads) * sizeof(int32_t) +
                             2 * kStreamStages * sizeof(uint64_t) + 16 + 1024;
-#define GTA_LAUNCH_STREAM_(NT, KH)                                                                         \
+#define GTA_LAUNCH_STREAM_(NT, KH, ONE)                                                                    \
         do {                                                                                               \
-            auto kern = decode_stream_kernel<NT, KH, (NT == 2 ? 8 : 4)>;                                   \
+            auto kern = decode_stream_kernel<NT, KH, (NT == 2 ? 8 : 4), ONE>;                              \
             err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);      \
             if (err != cudaSuccess) return err;                                                            \
             cudaLaunchConfig_t cfg = {};                                                                   \
@@ -881,8 +890,10 @@ cudaError_t launch_decode_fast(const Dims& d, const void* q, const void* k_cache
         } while (0)
 #define GTA_LAUNCH_STREAM(NT)                                                                              \
         do {                                                                                               \
-            if (d.d_h == 128) GTA_LAUNCH_STREAM_(NT, 2);                                                   \
-            else GTA_LAUNCH_STREAM_(NT, 1);                                                                \
+            if (d.d_h == 128 && d.n_c == 1) GTA_LAUNCH_STREAM_(NT, 2, true);                               \
+            else if (d.d_h == 128) GTA_LAUNCH_STREAM_(NT, 2, false);                                       \
+            else if (d.n_c == 1) GTA_LAUNCH_STREAM_(NT, 1, true);                                          \
+            else GTA_LAUNCH_STREAM_(NT, 1, false);                                                         \
         } while (0)
         switch (d.d_l) {
             case 128: GTA_LAUNCH_STREAM(2); break;

@@ -220,6 +220,8 @@ SMALL_DECODE = [
     ("bf16_dh64_three_maps_batch_40", "bf16", 40, 192, 6, 3, 1, 1, 64, 128, [1 + (41 * i) % 700 for i in range(40)]),
     ("bf16_dh64_dl512_small_batch", "bf16", 3, 128, 8, 4, 2, 1, 64, 512, [70, 1, 513]),
     ("bf16_dh128_five_maps", "bf16", 7, 256, 10, 5, 1, 1, 128, 256, [300, 0, 64, 65, 1000, 17, 2]),
+    ("bf16_two_latents_batch_20", "bf16", 20, 256, 8, 4, 4, 2, 128, 256, [1 + (67 * i) % 500 for i in range(20)]),
+    ("bf16_four_latents_dl128", "bf16", 5, 128, 8, 8, 2, 4, 64, 128, [129, 1, 64, 400, 33]),
     ("bf16_batch_33_odd_heads", "bf16", 33, 128, 3, 1, 1, 1, 128, 256, [0 if i == 5 else 1 + (91 * i) % 500 for i in range(33)]),
 ]
 
