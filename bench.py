@@ -235,11 +235,15 @@ def run_ours(args):
     out_p = torch.empty((wp.batch, wp.seq, wp.n_heads, wp.d_h), dtype=torch.bfloat16, device=dev)
     status = torch.zeros(1, dtype=torch.int32, device=dev)
     # ---- decode leg buffers: two cache sets, read alternately
+    LENS_POOL = max(64, (max(args.steps, 20) + 1) // 2 + 8)   # length vectors per set: one per step of the longest loop
     sets = []
     for s in range(2):
         td = I.decode_inputs(I.scaled(wd, seed=wd.seed + s), device=dev, s_cap=wd.seq + 64)
         td["seq_lens"] -= 1            # the step's append brings the length back to wd.seq
         td["lens0"] = td["seq_lens"].clone()
+        # One length vector per step, all set to wd.seq - 1 before a loop starts: the append of a step
+        # advances its own vector, so no rewind copy sits between the steps of a timed region.
+        td["pool"] = td["lens0"].unsqueeze(0).repeat(LENS_POOL, 1).contiguous()
         sets.append(td)
     shape_d = G.decode_shape(sets[0]["q"], sets[0]["k_cache"], sets[0]["c_cache"], sets[0]["x_t"], sets[0]["w_p"])
     ws_d = torch.empty(G.decode_workspace_bytes(shape_d, wd.seq + 64), dtype=torch.uint8, device=dev)
@@ -262,15 +266,18 @@ def run_ours(args):
                       status_word=status, stages=2)
         launches["n"] += G.last_launch_count()
 
+    def reset_lens():
+        for td in sets:
+            td["pool"].copy_(td["lens0"].unsqueeze(0).expand(LENS_POOL, -1))
+
     def decode_leg(i, evs=None):
         td = sets[i % 2]
-        td["seq_lens"].copy_(td["lens0"])                 # 128-byte device copy: rewind the lengths
-        G.gta_cache_append(td["k_cache"], td["c_cache"], td["k_new"], td["c_new"], td["seq_lens"],
-                           status_word=status)
+        lens = td["pool"][(i // 2) % LENS_POOL]            # this step's own length vector (wd.seq - 1)
+        G.gta_cache_append(td["k_cache"], td["c_cache"], td["k_new"], td["c_new"], lens, status_word=status)
         launches["n"] += G.last_launch_count()
         if evs is not None:
             evs[0].record(stream)
-        G.gta_decode(td["q"], td["k_cache"], td["c_cache"], td["seq_lens"], td["x_t"], td["w_p"], td["w_g"],
+        G.gta_decode(td["q"], td["k_cache"], td["c_cache"], lens, td["x_t"], td["w_p"], td["w_g"],
                      out=out_d, workspace=ws_d, status_word=status)
         launches["n"] += G.last_launch_count()
 
@@ -294,6 +301,7 @@ def run_ours(args):
     time.sleep(0.8)                       # let nvidia-smi deliver its first samples
     for i in range(3):                    # keep the GPU warm after the sleep (untimed)
         prefill_leg(); decode_leg(i)
+    reset_lens()
     launches["n"] = 0
     barrier()
     t_wall0 = time.time()
@@ -319,6 +327,7 @@ def run_ours(args):
     evk = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(K_k)]
     for i in range(3):
         prefill_leg(evk[0][1]); decode_leg(i)
+    reset_lens()
     barrier()
     for i in range(K_k):
         evk[i][0].record(stream)
@@ -333,6 +342,7 @@ def run_ours(args):
     K_d = max(K, 20)
     for i in range(3):
         decode_leg(i)
+    reset_lens()
     barrier()
     d0, d1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     d0.record(stream)
@@ -342,7 +352,7 @@ def run_ours(args):
     barrier()
     t_decode_b2b = d0.elapsed_time(d1) / K_d
     assert int(status.item()) == 0, "device status word raised during the benchmark"
-    # ---- the gta_decode call alone, back to back (no append, no length rewind; same alternation)
+    # ---- the gta_decode call alone, back to back (no append; same alternation)
     for td in sets:
         td["seq_lens"].copy_(td["lens0"] + 1)
 
@@ -414,8 +424,8 @@ def run_ours(args):
                              "bytes = live cache + weights + vectors",
                      "with_append": {"achieved": by["total"] / (t_decode_b2b * 1e-3) / 1e9,
                                      "frac": by["total"] / (t_decode_b2b * 1e-3) / 1e9 / peaks["hbm_gbs"],
-                                     "note": "loop of length rewind copy (benchmark's own, 128 bytes) + "
-                                             "gta_cache_append + gta_decode"}},
+                                     "note": "loop of gta_cache_append + gta_decode (each step on its own "
+                                             "length vector, prepared before the loop)"}},
     }
     decode["roofline"]["frac"] = decode["roofline"]["achieved"] / decode["roofline"]["peak"]
 
