@@ -1,6 +1,7 @@
 // Cache append: bit-exact 16-byte copies of the new key / latent rows behind the live part of
 // each sequence's caches, then the length update (Sec. 3.3 last paragraph; App. B.1.3).
 #include "gta_common.cuh"
+#include "sm100_ptx.cuh"
 
 namespace gta {
 
@@ -40,6 +41,11 @@ __device__ __forceinline__ void append_copy(const AppendArgs& a, int b, int len,
 // One CTA per sequence: copy, then advance the length (few new rows, e.g. one decode step).
 __global__ void __launch_bounds__(kAppendThreads)
 append_small_kernel(AppendArgs a, int32_t* __restrict__ seq_lens, int32_t* status_word) {
+    // Launched with programmatic stream serialisation (the launch latency of a decode step's first
+    // kernel hides behind the step before): nothing is read or written before the kernel ahead in
+    // the stream is complete, and only then may the kernel behind this one be scheduled.
+    ptx::grid_dependency_wait();
+    ptx::grid_launch_dependents();
     const int b = blockIdx.x;
     const int len = seq_lens[b];
     __syncthreads();   // every thread has read the old length before thread 0 rewrites it
@@ -80,7 +86,17 @@ cudaError_t launch_cache_append(const Dims& d, int elem_size, void* k_cache, voi
     a.c_row_vecs = d.d_l * elem_size / 16;
     const long long vecs_per_seq = (long long)n_new * ((long long)d.n_k * a.k_row_vecs + (long long)d.n_c * a.c_row_vecs);
     if (vecs_per_seq <= 8 * kAppendThreads) {
-        append_small_kernel<<<d.B, kAppendThreads, 0, stream>>>(a, seq_lens, status_word);
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(d.B);
+        cfg.blockDim = dim3(kAppendThreads);
+        cfg.stream = stream;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        cudaError_t e = cudaLaunchKernelEx(&cfg, append_small_kernel, a, seq_lens, status_word);
+        if (e != cudaSuccess) return e;
         *launches += 1;
         return cudaGetLastError();
     }
