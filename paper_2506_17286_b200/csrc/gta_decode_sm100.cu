@@ -1,4 +1,4 @@
-// Bandwidth-oriented decode for bf16 caches (App. B.1.3), d_h = 128, one latent group.
+// Bandwidth-oriented decode for bf16 caches (App. B.1.3): d_h = 64 or 128, up to 8 attention maps.
 //
 //   decode_stream_kernel : persistent, one CTA per SM.  The live tokens of all sequences are cut
 //       into sub-tiles of T tokens; CTA c owns the contiguous sub-tile range [c n / G, (c+1) n / G),
@@ -13,23 +13,13 @@
 //       d_l / 8 slice of the latent sum; one CTA barrier per sub-tile.  When the range crosses
 //       into the next sequence, and at its end, the partial (max, sum, latent sum) goes to
 //       slot c + b of the workspace.
-//   decode_merge_kernel (batches of more than 16): log-sum-exp merge of the slots into L (bf16);
-//       the tcgen05 decoder + gate kernel of the prefill path then runs with the batch as its token axis.
-//   decode_finish_kernel (small batches): clusters of 4 or 8 CTAs per (head, 64-column half) split the reduction
-//       dimensions of the decoder (d_l) and of the gate (H).  Launched with programmatic stream
-//       serialisation: while the stream kernel drains, each CTA requests its weight slice (TMA)
-//       and its hidden-state slice and works out which stream CTAs own which sequence; after the
-//       dependency wait it merges, for 32 sequences at a time, the slots of its d_l slice
-//       (log-sum-exp), multiplies by W_P,i and W_G,i with warp-level MMAs, and the cluster adds the
-//       partial results through distributed shared memory before the sigmoid gate is applied.
-#include <cooperative_groups.h>
-
+//   decode_merge_kernel : log-sum-exp merge of the slots into the normalised latent L (bf16); the
+//       tcgen05 decoder + gate kernel of the prefill path then runs with the batch as its token
+//       axis.  Both are launched with programmatic stream serialisation behind the stream kernel.
 #include "gta_common.cuh"
 #include "gta_sm100.cuh"
 #include "sm100_ptx.cuh"
 #include "tma_host.cuh"
-
-namespace cg = cooperative_groups;
 
 namespace gta {
 
@@ -39,9 +29,6 @@ constexpr int kStreamStages = 3;
 constexpr int kStreamStageBytes = 65536;
 constexpr int kStreamMaxBatch = 512;
 constexpr int kStreamMaxT = 128;     // tokens per sub-tile: at most 64, or 128 for the narrowest caches (d_l = 128)
-constexpr int kFinBlockB = 32;
-constexpr int kFinThreads = 256;
-constexpr int kFinCols = 64;
 constexpr int kFinMaxSlots = 1024;  // >= stream CTAs + batch
 
 struct FastPlan {
@@ -50,11 +37,8 @@ struct FastPlan {
     int slots;     // G + B partial slots
     size_t off_ml, off_l, total;   // byte offsets in the workspace (part_o at 0)
 };
-constexpr int kFinMaxBatchClusters = 16;   // larger batches finish through the merge kernel + the tcgen05 decoder kernel
-                                           // (measured: faster from 32 sequences on; the weights then feed 128-row MMAs)
 
 static size_t align256f(size_t v) { return (v + 255) & ~(size_t)255; }
-static int finish_split(const Dims& d);
 
 bool decode_fast_supported(const Dims& d, int dtype) {
     if (dtype != GTA_BF16 || (d.d_h != 128 && d.d_h != 64)) return false;
@@ -62,12 +46,8 @@ bool decode_fast_supported(const Dims& d, int dtype) {
     if (d.n_q < 1 || d.n_q > 8) return false;                    // the maps are the rows of the warp-level MMAs
     if (d.n_k != 1 && d.n_k != 2 && d.n_k != 4 && d.n_k != 8) return false;   // key groups are dealt to the 8 warps
     if (d.H % 64 != 0 || d.B > kStreamMaxBatch) return false;
-    // the finish: clusters (small batches; written for d_h = 128, power-of-two map counts, d_l >= 256), else the
-    // merge kernel + the tcgen05 decoder kernel, which cuts the output columns in blocks inside one attention map
-    const bool clusters = d.B <= kFinMaxBatchClusters && d.d_h == 128 && d.d_l >= 256 && (d.n_q & (d.n_q - 1)) == 0 &&
-                          d.n_c == 1;
-    if (clusters && finish_split(d) == 0) return false;
-    if (!clusters && ((d.n_h / d.n_q) * d.d_h) % (d.B > 128 ? 128 : 64) != 0) return false;
+    // the finish (merge kernel + tcgen05 decoder kernel) cuts the output columns in blocks inside one attention map
+    if (((d.n_h / d.n_q) * d.d_h) % (d.B > 128 ? 128 : 64) != 0) return false;
     const int tok_bytes = (d.n_k * d.d_h + d.n_c * d.d_l) * 2;
     return tok_bytes * 16 <= kStreamStageBytes;
 }
@@ -418,349 +398,7 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
 }
 
 // ---------------------------------------------------------------------------------------------
-// One CTA = one head, 64 of its 128 output columns, 1 / S of the reduction dimensions (S = cluster
-// size, 4 or 8).  Dynamic shared memory:
-//   w_s [(d_l + H) / S rows][64 bf16] (swizzled weight slice: W_P rows first) |
-//   a_s [32][KA + 8 bf16] (merged latent slice, then hidden-state slice, per sequence) |
-//   part_s [2][32][64] fp32 (partial decoder / gate sums) | ml_s, w_all [slots] | prefix_s, rng_s [B] |
-//   bound_s [G + 1] | scan scratch | barrier
-struct FinSmem {
-    uint32_t a_off, part_off, ml_off, w_all_off, prefix_off, rng_off, bound_off, scan_off, bar_off, total;
-};
-__host__ __device__ inline FinSmem fin_smem_layout(int KA) {
-    FinSmem L;
-    L.a_off = (uint32_t)KA * 128u;
-    L.part_off = L.a_off + (uint32_t)kFinBlockB * (KA + 8) * 2;
-    L.ml_off = L.part_off + 2u * kFinBlockB * kFinCols * 4;
-    L.w_all_off = L.ml_off + kFinMaxSlots * 8;
-    L.prefix_off = L.w_all_off + kFinMaxSlots * 4;
-    L.rng_off = L.prefix_off + (kStreamMaxBatch + 2) * 4;
-    L.bound_off = L.rng_off + 2 * kStreamMaxBatch * 4;
-    L.scan_off = L.bound_off + (kFinMaxSlots - kStreamMaxBatch + 2) * 4;
-    L.bar_off = L.scan_off + 8 * 4;
-    L.total = L.bar_off + 16 + 1024;   // + slack to align the base to 1024 bytes
-    return L;
-}
-
-__device__ __forceinline__ void cp_async_16(void* dst, const void* src) {
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(ptx::smem_addr(dst)), "l"(src) : "memory");
-}
-__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
-
-// Merge of the split-KV partial latent sums of one block of 32 sequences into a_s (bf16).  A
-// thread owns one 4-column chunk of its CTA's d_l slice for SQ sequences (SQ x dls / 4 = 256
-// threads x ... : dls = 64, 128, 256 -> SQ = 2, 4, 8).  Loads go out in rounds of up to kFinRound
-// slots per sequence, all of a round in flight at once.
-struct FinMergeArgs {
-    const float* part_o; const float* w_all;
-    const int32_t* rng_s;    // [B][2] first / last stream CTA that owns sub-tiles of the sequence
-    __nv_bfloat16* a_s;
-    int n_q, d_l, g, col_base, dls, a_stride, b0, nb, tid;
-};
-constexpr int kFinMaxSQ = 8;
-struct FinMergeRegs { float4 v[32]; };
-
-template <int SQ>
-__device__ __forceinline__ void fin_merge_load(const FinMergeArgs& a, FinMergeRegs& r, int j0) {
-    constexpr int kRound = 32 / SQ;              // slots per sequence and round
-    const int tps = a.dls / 4;                   // threads per sequence
-    const int chunk = a.tid % tps, bgrp = a.tid / tps, nbg = kFinThreads / tps;
-#pragma unroll
-    for (int sq = 0; sq < SQ; ++sq) {
-        const int bb = bgrp + sq * nbg, b = a.b0 + bb;
-        const int c_lo = bb < a.nb ? a.rng_s[2 * b] : 0, c_hi = bb < a.nb ? a.rng_s[2 * b + 1] : -1;
-#pragma unroll
-        for (int j = 0; j < kRound; ++j) {
-            const int c = c_lo + j0 + j;
-            float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (c <= c_hi)
-                v = *reinterpret_cast<const float4*>(a.part_o + ((size_t)(c + b) * a.n_q + a.g) * a.d_l + a.col_base + 4 * chunk);
-            r.v[sq * kRound + j] = v;
-        }
-    }
-}
-
-template <int SQ>
-__device__ __forceinline__ void fin_merge_finish(const FinMergeArgs& a, FinMergeRegs& r) {
-    constexpr int kRound = 32 / SQ;
-    const int tps = a.dls / 4;
-    const int chunk = a.tid % tps, bgrp = a.tid / tps, nbg = kFinThreads / tps;
-    float4 sum[SQ];
-#pragma unroll
-    for (int sq = 0; sq < SQ; ++sq) sum[sq] = make_float4(0.f, 0.f, 0.f, 0.f);
-    int n_max = 0;
-#pragma unroll
-    for (int sq = 0; sq < SQ; ++sq) {
-        const int bb = bgrp + sq * nbg, b = a.b0 + bb;
-        if (bb < a.nb) n_max = max(n_max, a.rng_s[2 * b + 1] - a.rng_s[2 * b] + 1);
-    }
-    for (int j0 = 0;; j0 += kRound) {
-#pragma unroll
-        for (int sq = 0; sq < SQ; ++sq) {
-            const int bb = bgrp + sq * nbg, b = a.b0 + bb;
-            const int c_lo = bb < a.nb ? a.rng_s[2 * b] : 0, c_hi = bb < a.nb ? a.rng_s[2 * b + 1] : -1;
-#pragma unroll
-            for (int j = 0; j < kRound; ++j) {
-                const int c = c_lo + j0 + j;
-                if (c <= c_hi) {
-                    const float w = a.w_all[c + b];   // 0 for a CTA that owns nothing: its slot holds stale bits
-                    if (w != 0.f) {
-                        const float4 v = r.v[sq * kRound + j];
-                        sum[sq].x = fmaf(v.x, w, sum[sq].x); sum[sq].y = fmaf(v.y, w, sum[sq].y);
-                        sum[sq].z = fmaf(v.z, w, sum[sq].z); sum[sq].w = fmaf(v.w, w, sum[sq].w);
-                    }
-                }
-            }
-        }
-        if (j0 + kRound >= n_max) break;
-        fin_merge_load<SQ>(a, r, j0 + kRound);   // sequences that span more CTAs than one round covers
-    }
-#pragma unroll
-    for (int sq = 0; sq < SQ; ++sq) {
-        const int bb = bgrp + sq * nbg;
-        uint2 packed;
-        packed.x = pack_bf16(sum[sq].x, sum[sq].y);
-        packed.y = pack_bf16(sum[sq].z, sum[sq].w);
-        *reinterpret_cast<uint2*>(a.a_s + bb * a.a_stride + 4 * chunk) = packed;
-    }
-}
-
-__global__ void __launch_bounds__(kFinThreads)
-decode_finish_kernel(const __grid_constant__ CUtensorMap tm_wp, const __grid_constant__ CUtensorMap tm_wg, Dims d,
-                     int G, int T, int S_cap, const int32_t* __restrict__ seq_lens,
-                     const float* __restrict__ part_o, const float* __restrict__ part_ml,
-                     const __nv_bfloat16* __restrict__ x_t, __nv_bfloat16* __restrict__ out, int32_t* status_word) {
-    cg::cluster_group cluster = cg::this_cluster();
-    const int S = (int)cluster.num_blocks();     // = gridDim.x
-    extern __shared__ uint8_t fin_raw[];
-    uint8_t* fsm = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(fin_raw) + 1023) & ~(uintptr_t)1023);
-    const int dls = d.d_l / S, hs = d.H / S;     // this CTA's slice of the latent and of the hidden dimension
-    const int KA = dls + hs, a_stride = KA + 8;  // bf16 elements per a_s row (row = 16-byte multiple)
-    const FinSmem L = fin_smem_layout(KA);
-    uint8_t* w_s = fsm;
-    __nv_bfloat16* a_s = reinterpret_cast<__nv_bfloat16*>(fsm + L.a_off);
-    float* part_s = reinterpret_cast<float*>(fsm + L.part_off);
-    float2* ml_s = reinterpret_cast<float2*>(fsm + L.ml_off);             // (max, sum) of map g per slot
-    float* w_all = reinterpret_cast<float*>(fsm + L.w_all_off);           // merge weight per slot
-    int32_t* prefix_s = reinterpret_cast<int32_t*>(fsm + L.prefix_off);   // [B + 1]
-    int32_t* rng_s = reinterpret_cast<int32_t*>(fsm + L.rng_off);         // [B][2] first / last owning CTA
-    int32_t* bound_s = reinterpret_cast<int32_t*>(fsm + L.bound_off);     // [G + 1] first sub-tile of CTA c
-    int32_t* scan_s = reinterpret_cast<int32_t*>(fsm + L.scan_off);
-    uint64_t* w_bar = reinterpret_cast<uint64_t*>(fsm + L.bar_off);
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(w_bar + 1);
-
-    const int split = blockIdx.x;                // = rank inside the cluster
-    const int i = blockIdx.y >> 1;               // head
-    const int col0 = (blockIdx.y & 1) * kFinCols;   // first of this CTA's output columns inside the head
-    const int g = d.head_to_q(i);
-    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int quad = lane >> 2, sub = lane & 3, mat = lane >> 3, mrow = lane & 7;
-
-    // ---- weight slice: independent of the stream kernel's results, so it is requested first
-    if (tid == 0) {
-        ptx::mbar_init(w_bar, 1);
-        *abort_flag = 0;
-        ptx::fence_mbar_init();
-        ptx::mbar_arrive_expect_tx(w_bar, (uint32_t)KA * 128);
-        ptx::tma_load_3d(w_s, &tm_wp, w_bar, col0, split * dls, i);
-        for (int r0 = 0; r0 < hs; r0 += 256)
-            ptx::tma_load_2d(w_s + (size_t)(dls + r0) * 128, &tm_wg, w_bar, i * 128 + col0, split * hs + r0);
-    }
-    // ---- also independent of it: the hidden-state slice of a block of sequences (asynchronous copies)
-    auto load_x = [&](int b0, int nb) {
-        const int xv = hs / 8;                      // 16-byte vectors per sequence
-        for (int idx = tid; idx < kFinBlockB * xv; idx += kFinThreads) {
-            const int xb = idx / xv, v = idx % xv;
-            __nv_bfloat16* dst = a_s + xb * a_stride + dls + v * 8;
-            if (xb < nb) cp_async_16(dst, x_t + (size_t)(b0 + xb) * d.H + split * hs + v * 8);
-            else *reinterpret_cast<uint4*>(dst) = make_uint4(0u, 0u, 0u, 0u);
-        }
-    };
-    load_x(0, min(kFinBlockB, d.B));
-    // ---- and which stream CTAs own sub-tiles of which sequence.  Same
-    //      arithmetic as in the stream kernel: prefix sums of ceil(len / T), ranges c n / G.  This
-    //      runs while the stream kernel drains (the launch is programmatically serialised).
-    {
-        const int per = (d.B + kFinThreads - 1) / kFinThreads;
-        const int lo = min(tid * per, d.B), hi = min(lo + per, d.B);
-        int sum = 0;
-        for (int b = lo; b < hi; ++b) sum += (clamp_len(seq_lens[b], S_cap) + T - 1) / T;
-        int incl = sum;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const int v = __shfl_up_sync(0xffffffffu, incl, o);
-            if (lane >= o) incl += v;
-        }
-        if (lane == 31) scan_s[warp] = incl;
-        __syncthreads();
-        int base = incl - sum;
-        for (int w = 0; w < warp; ++w) base += scan_s[w];
-        for (int b = lo; b < hi; ++b) {
-            prefix_s[b] = base;
-            base += (clamp_len(seq_lens[b], S_cap) + T - 1) / T;
-        }
-        if (tid == kFinThreads - 1) prefix_s[d.B] = base;
-        __syncthreads();
-        const long long n_st = prefix_s[d.B];
-        for (int c = tid; c <= G; c += kFinThreads) bound_s[c] = (int32_t)(((long long)c * n_st) / G);
-        // the owner of sub-tile st is the largest c with floor(c n / G) <= st = floor(((st + 1) G - 1) / n)
-        for (int b = tid; b < d.B; b += kFinThreads) {
-            const long long s_lo = prefix_s[b], s_hi = prefix_s[b + 1];
-            int c_lo = 0, c_hi = -1;
-            if (s_hi > s_lo) {
-                c_lo = (int)(((s_lo + 1) * G - 1) / n_st);
-                c_hi = (int)((s_hi * G - 1) / n_st);
-            }
-            rng_s[2 * b] = c_lo;
-            rng_s[2 * b + 1] = c_hi;
-        }
-    }
-    __syncthreads();
-    ptx::grid_dependency_wait();   // everything below reads what the stream kernel wrote
-    const uint32_t w_addr = ptx::smem_addr(w_s), a_addr = ptx::smem_addr(a_s);
-
-    // ---- for this head's map, the (max, sum) pair of every slot (slots nobody wrote hold stale
-    //      bits that are never used)
-    const int n_slots = G + d.B;
-    for (int j = tid; j < n_slots; j += kFinThreads)
-        ml_s[j] = *reinterpret_cast<const float2*>(part_ml + ((size_t)j * d.n_q + g) * 2);
-
-    for (int b0 = 0; b0 < d.B; b0 += kFinBlockB) {
-        const int nb = min(kFinBlockB, d.B - b0);
-        if (b0 > 0) load_x(b0, nb);   // (block 0: already requested before the dependency wait)
-        // ---- merged latent slice (bf16): a thread owns one 4-column chunk of SQ sequences.  The
-        //      first round of partial-result loads is issued before the merge weights exist (block 0
-        //      computes them meanwhile), so their latency overlaps that work.
-        const FinMergeArgs ma = {part_o, w_all, rng_s, a_s, d.n_q, d.d_l, g, split * dls, dls, a_stride, b0, nb, tid};
-        FinMergeRegs mr;
-        if (dls == 64) fin_merge_load<2>(ma, mr, 0);
-        else if (dls == 128) fin_merge_load<4>(ma, mr, 0);
-        else fin_merge_load<8>(ma, mr, 0);
-        if (b0 == 0) {
-            __syncthreads();   // the (max, sum) pairs are in shared memory
-            // per sequence (eight lanes each): the normalised merge weight of each of its slots c + b:
-            //      w = 2^(m_slot - M) / sum_slots l_slot 2^(m_slot - M)
-            for (int b8 = 0; b8 < d.B; b8 += kFinThreads / 8) {
-                const int b = b8 + (tid >> 3), l8 = tid & 7;
-                const bool live = b < d.B;
-                const int c_lo = live ? rng_s[2 * b] : 0, c_hi = live ? rng_s[2 * b + 1] : -1;
-                float M = -INFINITY, l = 0.f;
-                for (int c = c_lo + l8; c <= c_hi; c += 8)
-                    if (bound_s[c] < bound_s[c + 1]) M = fmaxf(M, ml_s[c + b].x);
-                M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, 1));
-                M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, 2));
-                M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, 4));
-                for (int c = c_lo + l8; c <= c_hi; c += 8) {
-                    float w = 0.f;
-                    if (bound_s[c] < bound_s[c + 1]) {   // a CTA with an empty range wrote nothing
-                        w = ex2f(ml_s[c + b].x - M);
-                        l = fmaf(ml_s[c + b].y, w, l);
-                    }
-                    w_all[c + b] = w;
-                }
-                l += __shfl_xor_sync(0xffffffffu, l, 1);
-                l += __shfl_xor_sync(0xffffffffu, l, 2);
-                l += __shfl_xor_sync(0xffffffffu, l, 4);
-                const float inv_l = 1.f / l;
-                for (int c = c_lo + l8; c <= c_hi; c += 8) w_all[c + b] *= inv_l;
-            }
-            __syncthreads();
-        }
-        if (dls == 64) fin_merge_finish<2>(ma, mr);
-        else if (dls == 128) fin_merge_finish<4>(ma, mr);
-        else fin_merge_finish<8>(ma, mr);
-        cp_async_wait_all();
-        __syncthreads();
-        if (b0 == 0) ptx::mbar_wait(w_bar, 0, abort_flag);   // on give-up the results are wrong and the status word says so
-        // ---- partial sums: warp w owns output columns 8 w .. 8 w + 7; rows = the 32 sequences
-        {
-            // four accumulator sets per m-tile, used round-robin over the k-steps: the dependent
-            // chain of MMAs is a quarter as long (the loop is latency-bound, not throughput-bound)
-            float acc[2][4][4] = {};     // [y / z][set][fragment], m-tile 0
-            float bcc[2][4][4] = {};     // same, m-tile 1
-            const int a_row = (mat & 1) * 8 + mrow, a_col = (mat >> 1) * 8;
-            const int n_ks = KA / 16, ks_y = dls / 16;
-            for (int ks0 = 0; ks0 < n_ks; ks0 += 4) {
-#pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    const int ks = ks0 + u;
-                    if (ks >= n_ks) break;
-                    const int yz = ks < ks_y ? 0 : 1;
-                    const int krow = 16 * ks + (lane & 15);
-                    uint32_t w0, w1;
-                    ptx::ldsm_x2_trans(w_addr + krow * 128 + ((warp ^ (krow & 7)) << 4), w0, w1);
-                    uint32_t a0, a1, a2, a3;
-                    ptx::ldsm_x4(a_addr + (uint32_t)(a_row * a_stride + 16 * ks + a_col) * 2, a0, a1, a2, a3);
-                    uint32_t e0, e1, e2, e3;
-                    ptx::ldsm_x4(a_addr + (uint32_t)((16 + a_row) * a_stride + 16 * ks + a_col) * 2, e0, e1, e2, e3);
-                    if (yz == 0) {
-                        ptx::mma_bf16_16816(acc[0][u], a0, a1, a2, a3, w0, w1);
-                        ptx::mma_bf16_16816(bcc[0][u], e0, e1, e2, e3, w0, w1);
-                    } else {
-                        ptx::mma_bf16_16816(acc[1][u], a0, a1, a2, a3, w0, w1);
-                        ptx::mma_bf16_16816(bcc[1][u], e0, e1, e2, e3, w0, w1);
-                    }
-                }
-            }
-            float acc_y[2][4], acc_z[2][4];
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                acc_y[0][e] = (acc[0][0][e] + acc[0][1][e]) + (acc[0][2][e] + acc[0][3][e]);
-                acc_y[1][e] = (bcc[0][0][e] + bcc[0][1][e]) + (bcc[0][2][e] + bcc[0][3][e]);
-                acc_z[0][e] = (acc[1][0][e] + acc[1][1][e]) + (acc[1][2][e] + acc[1][3][e]);
-                acc_z[1][e] = (bcc[1][0][e] + bcc[1][1][e]) + (bcc[1][2][e] + bcc[1][3][e]);
-            }
-#pragma unroll
-            for (int mt = 0; mt < 2; ++mt) {
-                float* py = part_s + (mt * 16 + quad) * kFinCols + warp * 8 + 2 * sub;
-                float* pz = py + kFinBlockB * kFinCols;
-                *reinterpret_cast<float2*>(py) = make_float2(acc_y[mt][0], acc_y[mt][1]);
-                *reinterpret_cast<float2*>(py + 8 * kFinCols) = make_float2(acc_y[mt][2], acc_y[mt][3]);
-                *reinterpret_cast<float2*>(pz) = make_float2(acc_z[mt][0], acc_z[mt][1]);
-                *reinterpret_cast<float2*>(pz + 8 * kFinCols) = make_float2(acc_z[mt][2], acc_z[mt][3]);
-            }
-        }
-        cluster.sync();
-        // ---- cluster reduction: rank r finishes sequences [r 32 / S, (r + 1) 32 / S) of this block
-        const int rows_per_rank = kFinBlockB / S;
-        for (int idx = tid; idx < rows_per_rank * kFinCols; idx += kFinThreads) {
-            const int bb = split * rows_per_rank + idx / kFinCols, e = idx % kFinCols;
-            float yv[8], zv[8];
-#pragma unroll
-            for (int rk = 0; rk < 8; ++rk) {      // all remote loads in flight together
-                yv[rk] = zv[rk] = 0.f;
-                if (rk < S) {
-                    const float* remote = cluster.map_shared_rank(part_s, rk);
-                    yv[rk] = remote[bb * kFinCols + e];
-                    zv[rk] = remote[(kFinBlockB + bb) * kFinCols + e];
-                }
-            }
-            const float y = ((yv[0] + yv[1]) + (yv[2] + yv[3])) + ((yv[4] + yv[5]) + (yv[6] + yv[7]));
-            const float z = ((zv[0] + zv[1]) + (zv[2] + zv[3])) + ((zv[4] + zv[5]) + (zv[6] + zv[7]));
-            if (bb < nb) {
-                const float gate = __fdividef(1.f, 1.f + __expf(-z));
-                out[((size_t)(b0 + bb) * d.n_h + i) * 128 + col0 + e] = __float2bfloat16_rn(y * gate);
-            }
-        }
-        cluster.sync();   // the partial sums may be overwritten (next block) or the CTA may exit
-    }
-    if (tid == 0 && *abort_flag) raise_status(status_word, GTA_ERR_TIMEOUT);
-}
-
-// Cluster size (= split of the reduction dimensions) of the finish kernel: 4 when the larger
-// weight slice still fits in shared memory (fewer CTAs per cluster pack onto the GPCs in one wave),
-// else 8; 0 if neither split gives whole MMA steps and whole TMA boxes.
-static int finish_split(const Dims& d) {
-    for (int S = 4; S <= 8; S *= 2) {
-        const int hs = d.H / S, dls = d.d_l / S;
-        if (d.H % (16 * S) != 0 || (hs > 256 && hs % 256 != 0) || dls > 256) continue;
-        if (fin_smem_layout(dls + hs).total <= 200u * 1024u) return S;
-    }
-    return 0;
-}
-
-// ---------------------------------------------------------------------------------------------
-// Large batches: log-sum-exp merge of the split-KV slots of one (attention map, sequence) pair per
+// Log-sum-exp merge of the split-KV slots of one (attention map, sequence) pair per
 // CTA into the normalised latent L[n_q][B][d_l] (bf16), which the tcgen05 decoder + gate kernel of
 // the prefill path then consumes with the batch in the role of the token axis.
 // Launched with programmatic stream serialisation: while the stream kernel still runs, the CTA
@@ -856,8 +494,6 @@ cudaError_t launch_decode_fast(const Dims& d, const void* q, const void* k_cache
     float* part_o = reinterpret_cast<float*>(workspace);
     float* part_ml = reinterpret_cast<float*>(static_cast<char*>(workspace) + p.off_ml);
     __nv_bfloat16* l_g = reinterpret_cast<__nv_bfloat16*>(static_cast<char*>(workspace) + p.off_l);
-    const bool big_batch = !(d.B <= kFinMaxBatchClusters && d.d_h == 128 && d.d_l >= 256 &&
-                             (d.n_q & (d.n_q - 1)) == 0 && d.n_c == 1);
     cudaError_t err;
     if (stages & 2) {
         CUtensorMap tm_k, tm_c;
@@ -906,7 +542,7 @@ cudaError_t launch_decode_fast(const Dims& d, const void* q, const void* k_cache
         if ((err = cudaGetLastError()) != cudaSuccess) return err;
         *launches += 1;
     }
-    if ((stages & 4) && big_batch) {
+    if (stages & 4) {
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3(d.n_q, d.B);
         cfg.blockDim = dim3(256);
@@ -925,44 +561,6 @@ cudaError_t launch_decode_fast(const Dims& d, const void* q, const void* k_cache
         dd.N = d.B;
         if (launch_sm100_decoder(dd, l_g, x_t, w_p, w_g, out, status_word, stream) != GTA_OK) return cudaErrorUnknown;
         *launches += 2;
-    } else if (stages & 4) {
-        const int S = finish_split(d);
-        const int dls = d.d_l / S, hs = d.H / S, KA = dls + hs;
-        CUtensorMap tm_wp, tm_wg;
-        {
-            const uint64_t dims[3] = {128, (uint64_t)d.d_l, (uint64_t)d.n_h};
-            const uint32_t box[3] = {64, (uint32_t)dls, 1};
-            if (!make_bf16_map(&tm_wp, w_p, 3, dims, box)) return cudaErrorInvalidValue;
-        }
-        {
-            const uint64_t dims[2] = {(uint64_t)d.n_h * 128, (uint64_t)d.H};
-            const uint32_t box[2] = {64, (uint32_t)(hs < 256 ? hs : 256)};
-            if (!make_bf16_map(&tm_wg, w_g, 2, dims, box)) return cudaErrorInvalidValue;
-        }
-        const size_t smem = fin_smem_layout(KA).total;
-        err = cudaFuncSetAttribute(decode_finish_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (err != cudaSuccess) return err;
-        cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3(S, d.n_h * 2);
-        cfg.blockDim = dim3(kFinThreads);
-        cfg.dynamicSmemBytes = smem;
-        cfg.stream = stream;
-        cudaLaunchAttribute attr[2];
-        attr[0].id = cudaLaunchAttributeClusterDimension;
-        attr[0].val.clusterDim.x = S;
-        attr[0].val.clusterDim.y = 1;
-        attr[0].val.clusterDim.z = 1;
-        // the kernel may be scheduled while the stream kernel drains; it waits for it on the device
-        attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-        attr[1].val.programmaticStreamSerializationAllowed = 1;
-        cfg.attrs = attr;
-        cfg.numAttrs = 2;
-        err = cudaLaunchKernelEx(&cfg, decode_finish_kernel, tm_wp, tm_wg, d, p.G, p.T, S_cap, seq_lens,
-                                 (const float*)part_o, (const float*)part_ml, (const __nv_bfloat16*)x_t,
-                                 (__nv_bfloat16*)out, status_word);
-        if (err != cudaSuccess) return err;
-        if ((err = cudaGetLastError()) != cudaSuccess) return err;
-        *launches += 1;
     }
     return cudaSuccess;
 }

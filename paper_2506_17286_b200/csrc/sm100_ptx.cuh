@@ -1,6 +1,7 @@
 // Inline-PTX wrappers for the sm_100a features the tensor-core kernels use: mbarriers, TMA
 // tensor loads, tensor memory (TMEM) management, tcgen05.mma / ld / st, and the shared-memory
-// and instruction descriptors of tcgen05.mma.  No cluster multicast is used anywhere.
+// and instruction descriptors of tcgen05.mma.  No TMA load uses cluster multicast (only tcgen05.commit
+// signals the barriers of both CTAs of a pair).
 #pragma once
 
 #include <cuda.h>
