@@ -28,13 +28,14 @@ constexpr int kStreamThreads = kStreamConsumers + 32;
 constexpr int kStreamStages = 3;
 constexpr int kStreamStageBytes = 65536;
 constexpr int kStreamMaxBatch = 512;
-constexpr int kStreamMaxT = 128;     // tokens per sub-tile: at most 64, or 128 for the narrowest caches (d_l = 128)
+constexpr int kStreamMaxT = 64;      // tokens per sub-tile
 constexpr int kFinMaxSlots = 1024;  // >= stream CTAs + batch
 
 struct FastPlan {
     int T;         // tokens per sub-tile (16, 32 or 64)
     int G;         // stream CTAs
     int slots;     // G + B partial slots
+    int occ;       // stream CTAs per SM (1, or 2 for narrow caches)
     size_t off_ml, off_l, total;   // byte offsets in the workspace (part_o at 0)
 };
 
@@ -67,10 +68,14 @@ static FastPlan make_fast_plan(const Dims& d) {
     FastPlan p;
     const int tok_bytes = (d.n_k * d.d_h + d.n_c * d.d_l) * 2;
     int t = 16;
-    const int t_max = d.d_l == 128 ? 128 : 64;       // matches the KTM of the stream kernel's instantiation
-    while (t * 2 * tok_bytes <= kStreamStageBytes && t * 2 <= t_max) t *= 2;
+    // Narrow caches (a 64-token sub-tile within 32 KB): two CTAs per SM with half-size ring stages.  The
+    // work per byte is the same, but a sub-tile is small against its fixed latency chain (barrier,
+    // score -> softmax -> latent sum), which two independent CTAs on an SM hide behind one another.
+    p.occ = (d.d_l == 128 && kStreamMaxT * tok_bytes <= kStreamStageBytes / 2) ? 2 : 1;
+    while (t * 2 * tok_bytes <= kStreamStageBytes / p.occ && t * 2 <= kStreamMaxT) t *= 2;
     p.T = t;
-    p.G = sm_count() < kFinMaxSlots - kStreamMaxBatch ? sm_count() : kFinMaxSlots - kStreamMaxBatch;
+    const int ctas = p.occ * sm_count();
+    p.G = ctas < kFinMaxSlots - kStreamMaxBatch ? ctas : kFinMaxSlots - kStreamMaxBatch;
     p.slots = p.G + d.B;
     const size_t part_o = (size_t)p.slots * d.n_q * d.d_l * sizeof(float);
     const size_t part_ml = (size_t)p.slots * d.n_q * 2 * sizeof(float);
@@ -101,18 +106,19 @@ __device__ __forceinline__ int clamp_len(int len, int S_cap) { return len < 0 ? 
 //   K tiles : key group kg, half h (columns 64 h .. 64 h + 63)  at (KH kg + h) T 128
 //   C tiles : latent group cg, columns 64 j .. 64 j + 63         at c_off + (NT cg + j) T 128
 // NT = d_l / 64 = MMA n-tiles (8 latent columns each) per consumer warp; KH = d_h / 64 = 64-column
-// tiles per key row; KTM = most 16-token MMA k-steps per sub-tile (sub-tiles of up to 16 KTM tokens:
-// the narrower a cached token, the more tokens a sub-tile needs to be worth its fixed cost)
-// ONE_C: a single latent group (the latent-sum loop then has no group pass and no masking)
-template <int NT, int KH, int KTM, bool ONE_C>
-__global__ void __launch_bounds__(kStreamThreads, 1)
+// tiles per key row; ONE_C: a single latent group (the latent-sum loop then has no group pass and no
+// masking); OCC: CTAs per SM (ring stages of 64 KB / OCC)
+template <int NT, int KH, bool ONE_C, int OCC>
+__global__ void __launch_bounds__(kStreamThreads, OCC)
 decode_stream_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_c, Dims d,
                      int T, int S_cap, const __nv_bfloat16* __restrict__ q, const int32_t* __restrict__ seq_lens,
                      float* __restrict__ part_o, float* __restrict__ part_ml, int32_t* status_word) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     uint8_t* ring = smem;                                                              // 3 x 64 KB
-    float* s_buf = reinterpret_cast<float*>(smem + kStreamStages * kStreamStageBytes);   // [2][n_q][T]
+    constexpr int KTM = kStreamMaxT / 16;                     // most 16-token MMA k-steps per sub-tile
+    constexpr int kStageBytes = kStreamStageBytes / OCC;
+    float* s_buf = reinterpret_cast<float*>(smem + kStreamStages * kStageBytes);   // [2][n_q][T]
     int32_t* prefix = reinterpret_cast<int32_t*>(s_buf + 2 * 8 * kStreamMaxT);           // [B + 1]
     int32_t* scan_tmp = prefix + kStreamMaxBatch + 2;                                    // [kStreamThreads]
     uint64_t* full_bar = reinterpret_cast<uint64_t*>(scan_tmp + kStreamThreads);
@@ -206,7 +212,7 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
                 ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
                 if (!ok) break;
                 const int tok0 = (int)k * T;
-                uint8_t* stage = ring + s * kStreamStageBytes;
+                uint8_t* stage = ring + s * kStageBytes;
                 for (int op = lane; op < n_k_ops + n_c_tiles; op += 32) {
                     if (op < n_k_ops)
                         ptx::tma_load_3d_hint(stage + op * tile_bytes, &tm_k, &full_bar[s], (op % KH) * 64, tok0,
@@ -284,7 +290,7 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
             if (!ok) break;
             const int len = clamp_len(seq_lens[b], S_cap);
             const int n_valid = min(T, len - (int)k * T);
-            const uint32_t stage = ring_addr + s * kStreamStageBytes;
+            const uint32_t stage = ring_addr + s * kStageBytes;
             float* sb = s_buf + (it & 1) * (NQ * T);
 
             // ---- scores of the maps of key group kg_w, 8 tokens per unit: S = Q K^T
@@ -316,7 +322,7 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
                 const int n_vec = (T - n_valid) * vec_per_row;
                 for (int idx = tid; idx < n_vec; idx += kStreamConsumers) {
                     const int row = n_valid + idx / vec_per_row, v = idx % vec_per_row;   // v >> 3 = tile (group, 64 columns)
-                    uint8_t* p = ring + s * kStreamStageBytes + c_off + (v >> 3) * tile_bytes + row * 128 + (v & 7) * 16;
+                    uint8_t* p = ring + s * kStageBytes + c_off + (v >> 3) * tile_bytes + row * 128 + (v & 7) * 16;
                     *reinterpret_cast<uint4*>(p) = make_uint4(0u, 0u, 0u, 0u);
                 }
                 ptx::fence_proxy_async_smem();   // the next TMA write of this stage follows generic writes
@@ -502,12 +508,12 @@ cudaError_t launch_decode_fast(const Dims& d, const void* q, const void* k_cache
         const uint64_t dc[3] = {(uint64_t)d.d_l, (uint64_t)S_cap, (uint64_t)d.B * d.n_c};
         if (!make_bf16_map(&tm_k, k_cache, 3, dk, box) || !make_bf16_map(&tm_c, c_cache, 3, dc, box))
             return cudaErrorInvalidValue;
-        const size_t smem = (size_t)kStreamStages * kStreamStageBytes + 2 * 8 * kStreamMaxT * sizeof(float) +
+        const size_t smem = (size_t)kStreamStages * (kStreamStageBytes / p.occ) + 2 * 8 * kStreamMaxT * sizeof(float) +
                             (size_t)(kStreamMaxBatch + 2 + kStreamThreads) * sizeof(int32_t) +
                             2 * kStreamStages * sizeof(uint64_t) + 16 + 1024;
-#define GTA_LAUNCH_STREAM_(NT, KH, ONE)                                                                    \
+#define GTA_LAUNCH_STREAM_(NT, KH, ONE, OCC)                                                               \
         do {                                                                                               \
-            auto kern = decode_stream_kernel<NT, KH, (NT == 2 ? 8 : 4), ONE>;                              \
+            auto kern = decode_stream_kernel<NT, KH, ONE, OCC>;                                            \
             err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);      \
             if (err != cudaSuccess) return err;                                                            \
             cudaLaunchConfig_t cfg = {};                                                                   \
@@ -526,18 +532,29 @@ cudaError_t launch_decode_fast(const Dims& d, const void* q, const void* k_cache
         } while (0)
 #define GTA_LAUNCH_STREAM(NT)                                                                              \
         do {                                                                                               \
-            if (d.d_h == 128 && d.n_c == 1) GTA_LAUNCH_STREAM_(NT, 2, true);                               \
-            else if (d.d_h == 128) GTA_LAUNCH_STREAM_(NT, 2, false);                                       \
-            else if (d.n_c == 1) GTA_LAUNCH_STREAM_(NT, 1, true);                                          \
-            else GTA_LAUNCH_STREAM_(NT, 1, false);                                                         \
+            if (d.d_h == 128 && d.n_c == 1) GTA_LAUNCH_STREAM_(NT, 2, true, 1);                            \
+            else if (d.d_h == 128) GTA_LAUNCH_STREAM_(NT, 2, false, 1);                                    \
+            else if (d.n_c == 1) GTA_LAUNCH_STREAM_(NT, 1, true, 1);                                       \
+            else GTA_LAUNCH_STREAM_(NT, 1, false, 1);                                                      \
+        } while (0)
+#define GTA_LAUNCH_STREAM_NARROW()   /* d_l = 128, two CTAs per SM */                                      \
+        do {                                                                                               \
+            if (d.d_h == 128 && d.n_c == 1) GTA_LAUNCH_STREAM_(2, 2, true, 2);                             \
+            else if (d.d_h == 128) GTA_LAUNCH_STREAM_(2, 2, false, 2);                                     \
+            else if (d.n_c == 1) GTA_LAUNCH_STREAM_(2, 1, true, 2);                                        \
+            else GTA_LAUNCH_STREAM_(2, 1, false, 2);                                                       \
         } while (0)
         switch (d.d_l) {
-            case 128: GTA_LAUNCH_STREAM(2); break;
+            case 128:
+                if (p.occ == 2) GTA_LAUNCH_STREAM_NARROW();
+                else GTA_LAUNCH_STREAM(2);
+                break;
             case 256: GTA_LAUNCH_STREAM(4); break;
             case 512: GTA_LAUNCH_STREAM(8); break;
             default: GTA_LAUNCH_STREAM(16); break;
         }
 #undef GTA_LAUNCH_STREAM
+#undef GTA_LAUNCH_STREAM_NARROW
 #undef GTA_LAUNCH_STREAM_
         if ((err = cudaGetLastError()) != cudaSuccess) return err;
         *launches += 1;
