@@ -51,7 +51,8 @@ typedef enum {
     GTA_ERR_CUDA = 4,        /* a CUDA runtime / driver call failed (launch, attribute, tensor map) */
     GTA_ERR_CACHE_FULL = 5,  /* device-side: an append would exceed S_cap for some sequence */
     GTA_ERR_TIMEOUT = 6,     /* device-side: a bounded wait inside a kernel ran out */
-    GTA_ERR_STATIC_SCRATCH = 7 /* gta_decode_static: the problem needs more than GTA_STATIC_SCRATCH_BYTES */
+    GTA_ERR_STATIC_SCRATCH = 7, /* gta_decode_static: the problem needs more than GTA_STATIC_SCRATCH_BYTES */
+    GTA_ERR_BAD_PAGE = 8     /* device-side: a block-table entry in use lies outside [0, n_pages) */
 } gta_status_t;
 
 typedef enum { GTA_F32 = 0, GTA_BF16 = 1 } gta_dtype_t;
@@ -159,6 +160,45 @@ GTA_API gta_status_t gta_cache_append(const gta_shape_t *shape, void *k_cache, v
                               int32_t S_cap, const void *k_new, const void *c_new,
                               int32_t n_new, int32_t *seq_lens, int32_t *status_word,
                               void *cuda_stream);
+
+/*
+ * gta_decode_paged / gta_cache_append_paged — gta_decode and gta_cache_append over a paged cache
+ * (the paper keeps K and C of every past token, Sec. 3.3 last paragraph and App. B.1.3, and says
+ * nothing on where the rows live: the operation is the same, only the addressing differs).
+ * The rows of all sequences sit in two pools of fixed-size pages,
+ *
+ *   k_pool [n_pages, n_k, page_size, d_h]      c_pool [n_pages, n_c, page_size, d_l]
+ *   block_table device int32 [B, max_pages]
+ *
+ * and cached token t of sequence b is row t % page_size of page block_table[b, t / page_size]
+ * (the same page number in both pools).  The capacity of a sequence is page_size * max_pages
+ * tokens, which takes the place of S_cap everywhere (length clamp, GTA_ERR_CACHE_FULL).  Only the
+ * entries that cover live tokens (for the append: live and new tokens) are read; the others may
+ * hold anything.  An entry in use outside [0, n_pages) raises *status_word to GTA_ERR_BAD_PAGE;
+ * no memory outside the pools is touched, the affected sequences' results (or appended rows) are
+ * unspecified.  The caller owns the block table and the assignment of pages; two sequences must
+ * not append to the same page.
+ *
+ * Host-side errors: GTA_ERR_INVALID_ARG for a null or misaligned block table or a non-positive
+ * page_size, n_pages or max_pages (or page_size * max_pages above INT32_MAX); otherwise as
+ * gta_decode / gta_cache_append.  workspace: gta_decode_paged_workspace_bytes(shape, page_size,
+ * max_pages).  The bf16 fast path of gta_decode applies when, in addition to its shape rules,
+ * page_size is a multiple of 64; other page sizes run on the plain-ALU kernels.
+ */
+GTA_API size_t gta_decode_paged_workspace_bytes(const gta_shape_t *shape, int32_t page_size,
+                                                int32_t max_pages);
+GTA_API gta_status_t gta_decode_paged(const gta_shape_t *shape, const void *q, const void *k_pool,
+                                      const void *c_pool, const int32_t *block_table,
+                                      int32_t page_size, int32_t n_pages, int32_t max_pages,
+                                      const int32_t *seq_lens, const void *x_t, const void *w_p,
+                                      const void *w_g, void *out, void *workspace,
+                                      size_t workspace_bytes, int32_t *status_word,
+                                      void *cuda_stream);
+GTA_API gta_status_t gta_cache_append_paged(const gta_shape_t *shape, void *k_pool, void *c_pool,
+                                            const int32_t *block_table, int32_t page_size,
+                                            int32_t n_pages, int32_t max_pages, const void *k_new,
+                                            const void *c_new, int32_t n_new, int32_t *seq_lens,
+                                            int32_t *status_word, void *cuda_stream);
 
 /*
  * gta_decode_static — gta_decode without a workspace argument (the paper has no counterpart: this

@@ -189,6 +189,59 @@ def cache_append(shape: Shape, k_cache, c_cache, s_cap: int, k_new, c_new, n_new
     return k_cache, c_cache, lens, int(flag.value)
 
 
+def paged_view(pool, block_table, page_size: int):
+    """The contiguous cache [B, groups, max_pages * page_size, width] that a paged pool
+    [n_pages, groups, page_size, width] and a block table [B, max_pages] describe: cached token t
+    of sequence b is row t % page_size of page block_table[b, t // page_size] (the caches hold K
+    and C of every past token, Sec. 3.3 last paragraph; paging changes where a row lives, not what
+    it holds).  Rows under a negative entry stay zero.  Written token by token on purpose."""
+    pool, _ = _as_np(pool)
+    table = np.asarray(block_table, dtype=np.int64)
+    n_seq, max_pages = table.shape
+    groups, width = pool.shape[1], pool.shape[3]
+    assert pool.shape[2] == page_size
+    view = np.zeros((n_seq, groups, max_pages * page_size, width), dtype=pool.dtype)
+    for b in range(n_seq):
+        for t in range(max_pages * page_size):
+            page = table[b, t // page_size]
+            if page >= 0:
+                view[b, :, t, :] = pool[page, :, t % page_size, :]
+    return view
+
+
+def decode_paged(shape: Shape, q, k_pool, c_pool, block_table, page_size: int, seq_lens, x_t, w_p, w_g,
+                 n_threads: int = 0):
+    """decode() over a paged cache: the pools are read through paged_view, nothing else changes."""
+    k_cache = paged_view(k_pool, block_table, page_size)
+    c_cache = paged_view(c_pool, block_table, page_size)
+    q, _ = _as_np(q); x_t, _ = _as_np(x_t); w_p, _ = _as_np(w_p); w_g, _ = _as_np(w_g)
+    return decode(shape, q, k_cache, c_cache, seq_lens, k_cache.shape[2], x_t, w_p, w_g, n_threads)
+
+
+def cache_append_paged(k_pool, c_pool, block_table, page_size: int, k_new, c_new, seq_lens):
+    """Byte-exact append into a paged cache: new row n of sequence b becomes cached token
+    seq_lens[b] + n, i.e. row (seq_lens[b] + n) % page_size of the page the block table names for
+    it; a sequence whose new rows would pass max_pages * page_size is skipped whole.  Returns
+    (k_pool, c_pool, seq_lens, overflowed) as NEW numpy arrays."""
+    (k_pool, c_pool, k_new, c_new), _ = _same_dtype(k_pool, c_pool, k_new, c_new)
+    k_pool, c_pool = k_pool.copy(), c_pool.copy()
+    table = np.asarray(block_table, dtype=np.int64)
+    lens = np.asarray(seq_lens, dtype=np.int32).copy()
+    n_new = k_new.shape[2]
+    overflowed = 0
+    for b in range(table.shape[0]):
+        if lens[b] < 0 or lens[b] + n_new > table.shape[1] * page_size:
+            overflowed = 1
+            continue
+        for n in range(n_new):
+            t = int(lens[b]) + n
+            page = table[b, t // page_size]
+            k_pool[page, :, t % page_size, :] = k_new[b, :, n, :]
+            c_pool[page, :, t % page_size, :] = c_new[b, :, n, :]
+        lens[b] += n_new
+    return k_pool, c_pool, lens, overflowed
+
+
 def attention_cost(shape: Shape) -> float:
     """n_q (d_h + d_l) N^2 — Table 3, GTA row, 'Attention' column."""
     cs = shape.c()

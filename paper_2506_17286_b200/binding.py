@@ -16,6 +16,7 @@ LIB_PATH = os.path.join(_HERE, "libgta_b200.so")
 
 GTA_OK, GTA_ERR_INVALID_ARG, GTA_ERR_UNSUPPORTED, GTA_ERR_WORKSPACE = 0, 1, 2, 3
 GTA_ERR_CUDA, GTA_ERR_CACHE_FULL, GTA_ERR_TIMEOUT, GTA_ERR_STATIC_SCRATCH = 4, 5, 6, 7
+GTA_ERR_BAD_PAGE = 8
 STATIC_SCRATCH_BYTES = 16 << 20
 GTA_F32, GTA_BF16 = 0, 1
 
@@ -23,6 +24,7 @@ EXPORTS = (
     "gta_prefill_workspace_bytes", "gta_prefill", "gta_decode_workspace_bytes", "gta_decode",
     "gta_cache_append", "gta_status_string", "gta_version", "gta_prefill_path", "gta_last_launch_count",
     "gta_prefill_stages", "gta_decode_stages", "gta_decode_static", "gta_prefill_chunk",
+    "gta_decode_paged_workspace_bytes", "gta_decode_paged", "gta_cache_append_paged",
 )
 
 
@@ -74,6 +76,12 @@ def lib():
         L.gta_decode_static.restype = i32
         L.gta_cache_append.argtypes = [sp, vp, vp, i32, vp, vp, i32, vp, vp, vp]
         L.gta_cache_append.restype = i32
+        L.gta_decode_paged_workspace_bytes.argtypes = [sp, i32, i32]
+        L.gta_decode_paged_workspace_bytes.restype = sz
+        L.gta_decode_paged.argtypes = [sp, vp, vp, vp, vp, i32, i32, i32, vp, vp, vp, vp, vp, vp, sz, vp, vp]
+        L.gta_decode_paged.restype = i32
+        L.gta_cache_append_paged.argtypes = [sp, vp, vp, vp, i32, i32, i32, vp, vp, i32, vp, vp, vp]
+        L.gta_cache_append_paged.restype = i32
         L.gta_status_string.argtypes = [i32]
         L.gta_status_string.restype = ctypes.c_char_p
         L.gta_version.restype = i32
@@ -281,6 +289,69 @@ def gta_cache_append(k_cache, c_cache, k_new, c_new, seq_lens, *, status_word=No
                                 _ptr(c_new), n_new, _ptr(seq_lens), _ptr(status_word), _stream(stream))
     if st != GTA_OK:
         raise GtaError(st, "gta_cache_append")
+    return seq_lens
+
+
+def _check_paged(k_pool, c_pool, block_table, seq_lens):
+    if block_table.dtype != torch.int32 or block_table.device != k_pool.device or not block_table.is_contiguous() \
+            or block_table.dim() != 2:
+        raise ValueError("block_table must be a contiguous int32 [B, max_pages] tensor on the pools' device")
+    if seq_lens.dtype != torch.int32 or seq_lens.device != k_pool.device or not seq_lens.is_contiguous():
+        raise ValueError("seq_lens must be a contiguous int32 tensor on the pools' device")
+    n_pages, n_k, page_size, d_h = k_pool.shape
+    n_c, d_l = c_pool.shape[1], c_pool.shape[3]
+    if c_pool.shape != (n_pages, n_c, page_size, d_l) or seq_lens.shape != (block_table.shape[0],):
+        raise ValueError("inconsistent pool tensor shapes")
+    return n_pages, page_size, block_table.shape[1]
+
+
+def decode_paged_workspace_bytes(shape: GtaShape, page_size: int, max_pages: int) -> int:
+    return int(lib().gta_decode_paged_workspace_bytes(ctypes.byref(shape), int(page_size), int(max_pages)))
+
+
+def gta_decode_paged(q, k_pool, c_pool, block_table, seq_lens, x_t, w_p, w_g, *, softmax_scale=0.0, out=None,
+                     workspace=None, status_word=None, stream=None):
+    """gta_decode over a paged cache.  k_pool [n_pages,n_k,page_size,d_h], c_pool [n_pages,n_c,page_size,d_l],
+    block_table int32 [B,max_pages]: token t of sequence b is row t % page_size of page block_table[b, t // page_size]."""
+    _check_tensors(q, k_pool, c_pool, x_t, w_p, w_g)
+    n_pages, page_size, max_pages = _check_paged(k_pool, c_pool, block_table, seq_lens)
+    B, n_q, d_h = q.shape
+    shape = decode_shape(q, k_pool, c_pool, x_t, w_p, softmax_scale=softmax_scale)
+    n_h, d_l, H = shape.n_heads, shape.latent_dim, shape.d_model
+    if k_pool.shape[3] != d_h or x_t.shape != (B, H) or w_p.shape != (n_h, d_l, d_h) \
+            or w_g.shape != (H, n_h * d_h) or block_table.shape[0] != B:
+        raise ValueError("inconsistent operator tensor shapes")
+    if out is None:
+        out = torch.empty((B, n_h, d_h), dtype=q.dtype, device=q.device)
+    if workspace is None:
+        workspace = _workspace(decode_paged_workspace_bytes(shape, page_size, max_pages), q.device)
+    st = lib().gta_decode_paged(ctypes.byref(shape), _ptr(q), _ptr(k_pool), _ptr(c_pool), _ptr(block_table),
+                                page_size, n_pages, max_pages, _ptr(seq_lens), _ptr(x_t), _ptr(w_p), _ptr(w_g),
+                                _ptr(out), _ptr(workspace), workspace.numel() * workspace.element_size(),
+                                _ptr(status_word), _stream(stream))
+    if st != GTA_OK:
+        raise GtaError(st, "gta_decode_paged")
+    return out
+
+
+def gta_cache_append_paged(k_pool, c_pool, block_table, k_new, c_new, seq_lens, *, status_word=None, stream=None):
+    """gta_cache_append over a paged cache: the new rows go to the pages the block table names for positions
+    seq_lens[b] .. seq_lens[b] + n_new - 1, and seq_lens advances by n_new."""
+    _check_tensors(k_pool, c_pool, k_new, c_new)
+    n_pages, page_size, max_pages = _check_paged(k_pool, c_pool, block_table, seq_lens)
+    B = block_table.shape[0]
+    n_k, d_h, n_c, d_l = k_pool.shape[1], k_pool.shape[3], c_pool.shape[1], c_pool.shape[3]
+    n_new = k_new.shape[2]
+    if k_new.shape != (B, n_k, n_new, d_h) or c_new.shape != (B, n_c, n_new, d_l):
+        raise ValueError("inconsistent cache tensor shapes")
+    n_q = n_k * n_c // _gcd(n_k, n_c)
+    shape = make_shape(batch=B, seq=0, d_model=8, n_heads=n_q, n_q=n_q, n_k=n_k, n_c=n_c, d_h=d_h, d_l=d_l,
+                       dtype=_dtype_code(k_pool))
+    st = lib().gta_cache_append_paged(ctypes.byref(shape), _ptr(k_pool), _ptr(c_pool), _ptr(block_table), page_size,
+                                      n_pages, max_pages, _ptr(k_new), _ptr(c_new), n_new, _ptr(seq_lens),
+                                      _ptr(status_word), _stream(stream))
+    if st != GTA_OK:
+        raise GtaError(st, "gta_cache_append_paged")
     return seq_lens
 
 

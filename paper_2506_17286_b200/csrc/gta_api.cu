@@ -58,6 +58,13 @@ static gta_status_t prefill_impl(const gta_shape_t* shape, int32_t kv_len, int32
                                  const void* k, const void* c, const void* x, const void* w_p, const void* w_g,
                                  void* out, void* workspace, size_t workspace_bytes, int32_t* status_word,
                                  void* cuda_stream, int32_t stages);
+static gta_status_t decode_impl(const gta_shape_t* shape, const void* q, const void* k_cache, const void* c_cache,
+                                const int32_t* seq_lens, int32_t S_cap, const void* x_t, const void* w_p,
+                                const void* w_g, void* out, void* workspace, size_t workspace_bytes,
+                                int32_t* status_word, void* cuda_stream, int32_t stages, const gta::PageMap& pm);
+static gta_status_t append_impl(const gta_shape_t* shape, void* k_cache, void* c_cache, int32_t S_cap,
+                                const void* k_new, const void* c_new, int32_t n_new, int32_t* seq_lens,
+                                int32_t* status_word, void* cuda_stream, const gta::PageMap& pm);
 
 extern "C" {
 
@@ -71,6 +78,7 @@ const char* gta_status_string(gta_status_t status) {
         case GTA_ERR_CACHE_FULL: return "cache full";
         case GTA_ERR_TIMEOUT: return "bounded device wait ran out";
         case GTA_ERR_STATIC_SCRATCH: return "problem exceeds the built-in scratch array of gta_decode_static";
+        case GTA_ERR_BAD_PAGE: return "block-table entry outside the page pool";
     }
     return "unknown status";
 }
@@ -182,6 +190,61 @@ gta_status_t gta_decode_stages(const gta_shape_t* shape, const void* q, const vo
                                const void* w_p, const void* w_g, void* out, void* workspace,
                                size_t workspace_bytes, int32_t* status_word, void* cuda_stream,
                                int32_t stages) {
+    return decode_impl(shape, q, k_cache, c_cache, seq_lens, S_cap, x_t, w_p, w_g, out, workspace, workspace_bytes,
+                       status_word, cuda_stream, stages, gta::PageMap());
+}
+
+// A block table is usable when it is there, 4-byte aligned, and the pool geometry is positive.
+static bool page_args_ok(const int32_t* block_table, int32_t page_size, int32_t n_pages, int32_t max_pages) {
+    return block_table && aligned(block_table, 4) && page_size > 0 && n_pages > 0 && max_pages > 0 &&
+           (long long)page_size * max_pages <= INT32_MAX;
+}
+
+size_t gta_decode_paged_workspace_bytes(const gta_shape_t* shape, int32_t page_size, int32_t max_pages) {
+    gta::Dims d;
+    if (check_shape(shape, false, &d) != GTA_OK || page_size <= 0 || max_pages <= 0 ||
+        (long long)page_size * max_pages > INT32_MAX)
+        return 0;
+    return gta::decode_workspace_bytes(d, shape->dtype, page_size * max_pages, page_size);
+}
+
+gta_status_t gta_decode_paged(const gta_shape_t* shape, const void* q, const void* k_pool, const void* c_pool,
+                              const int32_t* block_table, int32_t page_size, int32_t n_pages, int32_t max_pages,
+                              const int32_t* seq_lens, const void* x_t, const void* w_p, const void* w_g,
+                              void* out, void* workspace, size_t workspace_bytes, int32_t* status_word,
+                              void* cuda_stream) {
+    g_last_launches = 0;
+    if (!page_args_ok(block_table, page_size, n_pages, max_pages)) return GTA_ERR_INVALID_ARG;
+    gta::PageMap pm;
+    pm.table = block_table;
+    pm.page_size = page_size;
+    pm.max_pages = max_pages;
+    pm.n_pages = n_pages;
+    return decode_impl(shape, q, k_pool, c_pool, seq_lens, page_size * max_pages, x_t, w_p, w_g, out, workspace,
+                       workspace_bytes, status_word, cuda_stream, 7, pm);
+}
+
+gta_status_t gta_cache_append_paged(const gta_shape_t* shape, void* k_pool, void* c_pool,
+                                    const int32_t* block_table, int32_t page_size, int32_t n_pages,
+                                    int32_t max_pages, const void* k_new, const void* c_new, int32_t n_new,
+                                    int32_t* seq_lens, int32_t* status_word, void* cuda_stream) {
+    g_last_launches = 0;
+    if (!page_args_ok(block_table, page_size, n_pages, max_pages)) return GTA_ERR_INVALID_ARG;
+    gta::PageMap pm;
+    pm.table = block_table;
+    pm.page_size = page_size;
+    pm.max_pages = max_pages;
+    pm.n_pages = n_pages;
+    return append_impl(shape, k_pool, c_pool, page_size * max_pages, k_new, c_new, n_new, seq_lens, status_word,
+                       cuda_stream, pm);
+}
+
+}  // extern "C"
+
+static gta_status_t decode_impl(const gta_shape_t* shape, const void* q, const void* k_cache, const void* c_cache,
+                                const int32_t* seq_lens, int32_t S_cap, const void* x_t, const void* w_p,
+                                const void* w_g, void* out, void* workspace, size_t workspace_bytes,
+                                int32_t* status_word, void* cuda_stream, int32_t stages, const gta::PageMap& pm) {
     g_last_launches = 0;
     if (stages < 1 || stages > 7) return GTA_ERR_INVALID_ARG;
     gta::Dims d;
@@ -197,21 +260,29 @@ gta_status_t gta_decode_stages(const gta_shape_t* shape, const void* q, const vo
     // one latent row is spread over at most 256 threads, 16 bytes each
     if ((size_t)d.d_l * elem_size(shape->dtype) > 4096) return GTA_ERR_UNSUPPORTED;
     if (d.B == 0) return GTA_OK;
-    if (!workspace || !aligned(workspace, 256) || workspace_bytes < gta::decode_workspace_bytes(d, shape->dtype, S_cap))
+    if (!workspace || !aligned(workspace, 256) ||
+        workspace_bytes < gta::decode_workspace_bytes(d, shape->dtype, S_cap, pm.table ? pm.page_size : 0))
         return GTA_ERR_WORKSPACE;
     if ((st = check_device()) != GTA_OK) return st;
     int launches = 0;
     cudaError_t err = gta::launch_decode(d, shape->dtype, q, k_cache, c_cache, seq_lens, S_cap, x_t, w_p, w_g,
                                          out, workspace, status_word, static_cast<cudaStream_t>(cuda_stream),
-                                         stages, &launches);
+                                         stages, &launches, pm);
     if (err != cudaSuccess) return GTA_ERR_CUDA;
     g_last_launches = launches;
     return GTA_OK;
 }
 
-gta_status_t gta_cache_append(const gta_shape_t* shape, void* k_cache, void* c_cache, int32_t S_cap,
-                              const void* k_new, const void* c_new, int32_t n_new, int32_t* seq_lens,
-                              int32_t* status_word, void* cuda_stream) {
+extern "C" gta_status_t gta_cache_append(const gta_shape_t* shape, void* k_cache, void* c_cache, int32_t S_cap,
+                                         const void* k_new, const void* c_new, int32_t n_new, int32_t* seq_lens,
+                                         int32_t* status_word, void* cuda_stream) {
+    return append_impl(shape, k_cache, c_cache, S_cap, k_new, c_new, n_new, seq_lens, status_word, cuda_stream,
+                       gta::PageMap());
+}
+
+static gta_status_t append_impl(const gta_shape_t* shape, void* k_cache, void* c_cache, int32_t S_cap,
+                                const void* k_new, const void* c_new, int32_t n_new, int32_t* seq_lens,
+                                int32_t* status_word, void* cuda_stream, const gta::PageMap& pm) {
     g_last_launches = 0;
     gta::Dims d;
     gta_status_t st = check_shape(shape, false, &d);
@@ -226,10 +297,8 @@ gta_status_t gta_cache_append(const gta_shape_t* shape, void* k_cache, void* c_c
     int launches = 0;
     cudaError_t err = gta::launch_cache_append(d, (int)elem_size(shape->dtype), k_cache, c_cache, S_cap, k_new,
                                                c_new, n_new, seq_lens, status_word,
-                                               static_cast<cudaStream_t>(cuda_stream), &launches);
+                                               static_cast<cudaStream_t>(cuda_stream), &launches, pm);
     if (err != cudaSuccess) return GTA_ERR_CUDA;
     g_last_launches = launches;
     return GTA_OK;
 }
-
-}  // extern "C"

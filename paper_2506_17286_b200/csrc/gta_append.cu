@@ -12,6 +12,8 @@ struct AppendArgs {
     const uint4* k_new; const uint4* c_new;
     int B, n_k, n_c, S_cap, n_new;
     int k_row_vecs, c_row_vecs;   // 16-byte vectors per row
+    PageMap pm;                   // table == nullptr: contiguous caches
+    int32_t* status_word;
 };
 
 // Copies slice `part` of `n_parts` of sequence b's new rows.  Does not touch seq_lens.
@@ -25,15 +27,19 @@ __device__ __forceinline__ void append_copy(const AppendArgs& a, int b, int len,
             const int v = (int)(idx % a.k_row_vecs);
             const long long row = idx / a.k_row_vecs;          // g * n_new + n
             const int n = (int)(row % a.n_new), g = (int)(row / a.n_new);
-            a.k_cache[(((size_t)b * a.n_k + g) * a.S_cap + len + n) * a.k_row_vecs + v] =
-                a.k_new[(((size_t)b * a.n_k + g) * a.n_new + n) * a.k_row_vecs + v];
+            const long long dst = cache_row(a.pm, b, a.n_k, g, a.S_cap, len + n, a.status_word);
+            if (dst >= 0)
+                a.k_cache[(size_t)dst * a.k_row_vecs + v] =
+                    a.k_new[(((size_t)b * a.n_k + g) * a.n_new + n) * a.k_row_vecs + v];
         } else {
             const long long cidx = idx - k_vecs;
             const int v = (int)(cidx % a.c_row_vecs);
             const long long row = cidx / a.c_row_vecs;
             const int n = (int)(row % a.n_new), g = (int)(row / a.n_new);
-            a.c_cache[(((size_t)b * a.n_c + g) * a.S_cap + len + n) * a.c_row_vecs + v] =
-                a.c_new[(((size_t)b * a.n_c + g) * a.n_new + n) * a.c_row_vecs + v];
+            const long long dst = cache_row(a.pm, b, a.n_c, g, a.S_cap, len + n, a.status_word);
+            if (dst >= 0)
+                a.c_cache[(size_t)dst * a.c_row_vecs + v] =
+                    a.c_new[(((size_t)b * a.n_c + g) * a.n_new + n) * a.c_row_vecs + v];
         }
     }
 }
@@ -77,8 +83,10 @@ __global__ void append_advance_kernel(int B, int S_cap, int n_new, int32_t* __re
 
 cudaError_t launch_cache_append(const Dims& d, int elem_size, void* k_cache, void* c_cache, int S_cap,
                                 const void* k_new, const void* c_new, int n_new, int32_t* seq_lens,
-                                int32_t* status_word, cudaStream_t stream, int* launches) {
+                                int32_t* status_word, cudaStream_t stream, int* launches, const PageMap& pm) {
     AppendArgs a;
+    a.pm = pm;
+    a.status_word = status_word;
     a.k_cache = (uint4*)k_cache; a.c_cache = (uint4*)c_cache;
     a.k_new = (const uint4*)k_new; a.c_new = (const uint4*)c_new;
     a.B = d.B; a.n_k = d.n_k; a.n_c = d.n_c; a.S_cap = S_cap; a.n_new = n_new;

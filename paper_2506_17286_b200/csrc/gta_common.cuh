@@ -46,6 +46,35 @@ __device__ __forceinline__ void raise_status(int32_t* status_word, int code) {
     if (status_word) atomicMax(status_word, code);
 }
 
+// Where the cached rows of a sequence live (decode and append).  table == nullptr: caches
+// [B][groups][S_cap][width], the rows of one (sequence, group) contiguous.  Otherwise a paged pool
+// [n_pages][groups][page_size][width]: token t of sequence b is row t % page_size of page
+// table[b * max_pages + t / page_size], and S_cap = max_pages * page_size.
+struct PageMap {
+    const int32_t* table = nullptr;
+    int page_size = 0, max_pages = 0, n_pages = 0;
+};
+
+// Page that holds token t of sequence b; an entry outside the pool raises GTA_ERR_BAD_PAGE and
+// yields -1 (the caller skips the access).
+__device__ __forceinline__ int page_of(const PageMap& pm, int b, int t, int32_t* status_word) {
+    const int page = pm.table[(size_t)b * pm.max_pages + t / pm.page_size];
+    if (page < 0 || page >= pm.n_pages) {
+        raise_status(status_word, GTA_ERR_BAD_PAGE);
+        return -1;
+    }
+    return page;
+}
+
+// Row index (in rows of the cache tensor) of token t of group g of sequence b, or -1 (bad page).
+__device__ __forceinline__ long long cache_row(const PageMap& pm, int b, int groups, int g, int S_cap, int t,
+                                               int32_t* status_word) {
+    if (pm.table == nullptr) return ((long long)b * groups + g) * S_cap + t;
+    const int page = page_of(pm, b, t, status_word);
+    if (page < 0) return -1;
+    return ((long long)page * groups + g) * pm.page_size + t % pm.page_size;
+}
+
 // Launchers implemented in the .cu files; each returns cudaGetLastError() of its launches and
 // adds the number of launches it made to *launches.
 cudaError_t launch_generic_prefill(const Dims& d, int dtype, const void* q, const void* k, const void* c,
@@ -58,19 +87,20 @@ cudaError_t launch_generic_attention_bf16(const Dims& d, const void* q, const vo
 cudaError_t launch_decode(const Dims& d, int dtype, const void* q, const void* k_cache, const void* c_cache,
                           const int32_t* seq_lens, int S_cap, const void* x_t, const void* w_p,
                           const void* w_g, void* out, void* workspace, int32_t* status_word,
-                          cudaStream_t stream, int stages, int* launches);
-size_t decode_workspace_bytes(const Dims& d, int dtype, int S_cap);
+                          cudaStream_t stream, int stages, int* launches, const PageMap& pm = PageMap());
+size_t decode_workspace_bytes(const Dims& d, int dtype, int S_cap, int page_size = 0);
 
 // bf16 bandwidth-oriented decode (persistent streaming kernel + cluster finish kernel).
-bool decode_fast_supported(const Dims& d, int dtype);
+bool decode_fast_supported(const Dims& d, int dtype, int page_size = 0);
 size_t decode_fast_workspace_bytes(const Dims& d);
 cudaError_t launch_decode_fast(const Dims& d, const void* q, const void* k_cache, const void* c_cache,
                                const int32_t* seq_lens, int S_cap, const void* x_t, const void* w_p,
                                const void* w_g, void* out, void* workspace, int32_t* status_word,
-                               cudaStream_t stream, int stages, int* launches);
+                               cudaStream_t stream, int stages, int* launches, const PageMap& pm = PageMap());
 
 cudaError_t launch_cache_append(const Dims& d, int elem_size, void* k_cache, void* c_cache, int S_cap,
                                 const void* k_new, const void* c_new, int n_new, int32_t* seq_lens,
-                                int32_t* status_word, cudaStream_t stream, int* launches);
+                                int32_t* status_word, cudaStream_t stream, int* launches,
+                                const PageMap& pm = PageMap());
 
 }  // namespace gta

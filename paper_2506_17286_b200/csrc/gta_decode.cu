@@ -48,9 +48,9 @@ static DecodePlan make_plan(const Dims& d, int S_cap) {
     return p;
 }
 
-size_t decode_workspace_bytes(const Dims& d, int dtype, int S_cap) {
-    // the kernel family is a function of shape and dtype only, so the size is that family's
-    if (decode_fast_supported(d, dtype) && S_cap > 0) return decode_fast_workspace_bytes(d);
+size_t decode_workspace_bytes(const Dims& d, int dtype, int S_cap, int page_size) {
+    // the kernel family is a function of shape, dtype and page size only, so the size is that family's
+    if (decode_fast_supported(d, dtype, page_size) && S_cap > 0) return decode_fast_workspace_bytes(d);
     return make_plan(d, S_cap).total;
 }
 
@@ -87,7 +87,7 @@ __global__ void __launch_bounds__(kDecodeThreads)
 decode_partial_kernel(Dims d, int chunk, int n_chunks, int S_cap, const T* __restrict__ q,
                       const T* __restrict__ k_cache, const T* __restrict__ c_cache,
                       const int32_t* __restrict__ seq_lens, float* __restrict__ part_o,
-                      float* __restrict__ part_ml) {
+                      float* __restrict__ part_ml, PageMap pm, int32_t* status_word) {
     constexpr int VEC = Vec16<T>::N;
     const int b = blockIdx.y, ck = blockIdx.x;
     int len = seq_lens[b];
@@ -120,7 +120,9 @@ decode_partial_kernel(Dims d, int chunk, int n_chunks, int S_cap, const T* __res
             const int kg = it / n_row_iters;
             const int j = (it % n_row_iters) * rows_per_warp + sub;
             const bool live = j < n_tok;
-            const T* k_row = k_cache + (((size_t)b * d.n_k + kg) * S_cap + j_begin + (live ? j : 0)) * d.d_h;
+            // (a block-table entry outside the pool raises the status word; row 0 of the pool stands in)
+            const long long k_idx = cache_row(pm, b, d.n_k, kg, S_cap, j_begin + (live ? j : 0), status_word);
+            const T* k_row = k_cache + (size_t)(k_idx < 0 ? 0 : k_idx) * d.d_h;
             for (int gi = 0; gi < q_per_k; ++gi) {
                 const int g = kg * q_per_k + gi;
                 float dot = 0.f;
@@ -167,7 +169,10 @@ decode_partial_kernel(Dims d, int chunk, int n_chunks, int S_cap, const T* __res
     const int r = tid / tpr, v = tid % tpr;
     const int maps_per_c = d.n_q / d.n_c;
     for (int cg = 0; cg < d.n_c; ++cg) {
-        const T* c_base = c_cache + (((size_t)b * d.n_c + cg) * S_cap + j_begin) * d.d_l + v * VEC;
+        auto c_row = [&](int j) -> const T* {   // latent row of token j_begin + j, this thread's vector
+            const long long idx = cache_row(pm, b, d.n_c, cg, S_cap, j_begin + j, status_word);
+            return c_cache + (size_t)(idx < 0 ? 0 : idx) * d.d_l + v * VEC;
+        };
         for (int g0 = cg * maps_per_c; g0 < (cg + 1) * maps_per_c; g0 += NGB) {
             float acc[NGB][VEC];
 #pragma unroll
@@ -179,7 +184,7 @@ decode_partial_kernel(Dims d, int chunk, int n_chunks, int S_cap, const T* __res
                 for (; j + 3 * R < n_tok; j += 4 * R) {   // four independent 16-byte loads in flight
                     float cv[4][VEC];
 #pragma unroll
-                    for (int u = 0; u < 4; ++u) Vec16<T>::load(c_base + (size_t)(j + u * R) * d.d_l, cv[u]);
+                    for (int u = 0; u < 4; ++u) Vec16<T>::load(c_row(j + u * R), cv[u]);
 #pragma unroll
                     for (int u = 0; u < 4; ++u) {
                         const float* pj = p_s + (j + u * R) * d.n_q + g0;
@@ -193,7 +198,7 @@ decode_partial_kernel(Dims d, int chunk, int n_chunks, int S_cap, const T* __res
                 }
                 for (; j < n_tok; j += R) {
                     float cv[VEC];
-                    Vec16<T>::load(c_base + (size_t)j * d.d_l, cv);
+                    Vec16<T>::load(c_row(j), cv);
                     const float* pj = p_s + j * d.n_q + g0;
 #pragma unroll
                     for (int gi = 0; gi < NGB; ++gi) {
@@ -335,8 +340,8 @@ decode_finish_kernel(Dims d, int chunk, int n_chunks, int S_cap, int gate_splits
 template <typename T>
 static cudaError_t launch_decode_typed(const Dims& d, const void* q, const void* k_cache, const void* c_cache,
                                        const int32_t* seq_lens, int S_cap, const void* x_t, const void* w_p,
-                                       const void* w_g, void* out, void* workspace, cudaStream_t stream,
-                                       int stages, int* launches) {
+                                       const void* w_g, void* out, void* workspace, int32_t* status_word,
+                                       cudaStream_t stream, int stages, int* launches, const PageMap& pm) {
     constexpr int VEC = Vec16<T>::N;
     const DecodePlan p = make_plan(d, S_cap);
     float* part_o = reinterpret_cast<float*>(workspace);
@@ -365,7 +370,7 @@ static cudaError_t launch_decode_typed(const Dims& d, const void* q, const void*
             }                                                                                          \
             kern<<<grid, kDecodeThreads, smem, stream>>>(d, p.chunk, p.n_chunks, S_cap, (const T*)q,   \
                                                          (const T*)k_cache, (const T*)c_cache, seq_lens, \
-                                                         part_o, part_ml);                             \
+                                                         part_o, part_ml, pm, status_word);            \
         } while (0)
         if (maps_per_c % 8 == 0) GTA_LAUNCH_PARTIAL(8);
         else if (maps_per_c % 4 == 0) GTA_LAUNCH_PARTIAL(4);
@@ -395,15 +400,15 @@ static cudaError_t launch_decode_typed(const Dims& d, const void* q, const void*
 cudaError_t launch_decode(const Dims& d, int dtype, const void* q, const void* k_cache, const void* c_cache,
                           const int32_t* seq_lens, int S_cap, const void* x_t, const void* w_p,
                           const void* w_g, void* out, void* workspace, int32_t* status_word,
-                          cudaStream_t stream, int stages, int* launches) {
-    if (decode_fast_supported(d, dtype) && S_cap > 0)
+                          cudaStream_t stream, int stages, int* launches, const PageMap& pm) {
+    if (decode_fast_supported(d, dtype, pm.table ? pm.page_size : 0) && S_cap > 0)
         return launch_decode_fast(d, q, k_cache, c_cache, seq_lens, S_cap, x_t, w_p, w_g, out, workspace,
-                                  status_word, stream, stages, launches);
+                                  status_word, stream, stages, launches, pm);
     if (dtype == GTA_F32)
         return launch_decode_typed<float>(d, q, k_cache, c_cache, seq_lens, S_cap, x_t, w_p, w_g, out,
-                                          workspace, stream, stages, launches);
+                                          workspace, status_word, stream, stages, launches, pm);
     return launch_decode_typed<__nv_bfloat16>(d, q, k_cache, c_cache, seq_lens, S_cap, x_t, w_p, w_g, out,
-                                              workspace, stream, stages, launches);
+                                              workspace, status_word, stream, stages, launches, pm);
 }
 
 }  // namespace gta

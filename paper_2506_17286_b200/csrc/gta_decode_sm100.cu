@@ -41,8 +41,9 @@ struct FastPlan {
 
 static size_t align256f(size_t v) { return (v + 255) & ~(size_t)255; }
 
-bool decode_fast_supported(const Dims& d, int dtype) {
+bool decode_fast_supported(const Dims& d, int dtype, int page_size) {
     if (dtype != GTA_BF16 || (d.d_h != 128 && d.d_h != 64)) return false;
+    if (page_size % kStreamMaxT != 0) return false;              // a sub-tile never straddles two pages
     if (d.d_l != 128 && d.d_l != 256 && d.d_l != 512 && d.d_l != 1024) return false;
     if (d.n_q < 1 || d.n_q > 8) return false;                    // the maps are the rows of the warp-level MMAs
     if (d.n_k != 1 && d.n_k != 2 && d.n_k != 4 && d.n_k != 8) return false;   // key groups are dealt to the 8 warps
@@ -112,7 +113,7 @@ template <int NT, int KH, bool ONE_C, int OCC>
 __global__ void __launch_bounds__(kStreamThreads, OCC)
 decode_stream_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_c, Dims d,
                      int T, int S_cap, const __nv_bfloat16* __restrict__ q, const int32_t* __restrict__ seq_lens,
-                     float* __restrict__ part_o, float* __restrict__ part_ml, int32_t* status_word) {
+                     float* __restrict__ part_o, float* __restrict__ part_ml, int32_t* status_word, PageMap pm) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     uint8_t* ring = smem;                                                              // 3 x 64 KB
@@ -205,21 +206,30 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
                 while (k >= prefix[b + 1] - prefix[b]) { ++b; k = 0; }
                 const int s = it % kStreamStages;
                 const uint32_t ph = (it / kStreamStages) & 1;
+                // Contiguous caches: rows tok0 .. of plane b groups + g.  Paged pool: the sub-tile lies inside
+                // one page (T divides the page size), at rows tok0 % page_size .. of plane page groups + g; the
+                // block-table entry is fetched before the wait for the stage.  An entry outside the pool raises
+                // the status word, and the load (of page 0 then) still completes the stage.
+                int tok0 = (int)k * T, plane = b;
+                if (pm.table != nullptr) {
+                    const int page = page_of(pm, b, tok0, lane == 0 ? status_word : nullptr);
+                    plane = page < 0 ? 0 : page;
+                    tok0 %= pm.page_size;
+                }
                 if (lane == 0) {
                     ok = ptx::mbar_wait(&empty_bar[s], ph ^ 1, abort_flag);
                     if (ok) ptx::mbar_arrive_expect_tx(&full_bar[s], stage_tx);
                 }
                 ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
                 if (!ok) break;
-                const int tok0 = (int)k * T;
                 uint8_t* stage = ring + s * kStageBytes;
                 for (int op = lane; op < n_k_ops + n_c_tiles; op += 32) {
                     if (op < n_k_ops)
                         ptx::tma_load_3d_hint(stage + op * tile_bytes, &tm_k, &full_bar[s], (op % KH) * 64, tok0,
-                                              b * d.n_k + op / KH, policy);
+                                              plane * d.n_k + op / KH, policy);
                     else
                         ptx::tma_load_3d_hint(stage + c_off + (op - n_k_ops) * tile_bytes, &tm_c, &full_bar[s],
-                                              ((op - n_k_ops) % NT) * 64, tok0, b * d.n_c + (op - n_k_ops) / NT, policy);
+                                              ((op - n_k_ops) % NT) * 64, tok0, plane * d.n_c + (op - n_k_ops) / NT, policy);
                 }
             }
             if (lane == 0 && *abort_flag) {
@@ -495,7 +505,7 @@ decode_merge_kernel(Dims d, int G, int T, int S_cap, const int32_t* __restrict__
 cudaError_t launch_decode_fast(const Dims& d, const void* q, const void* k_cache, const void* c_cache,
                                const int32_t* seq_lens, int S_cap, const void* x_t, const void* w_p,
                                const void* w_g, void* out, void* workspace, int32_t* status_word,
-                               cudaStream_t stream, int stages, int* launches) {
+                               cudaStream_t stream, int stages, int* launches, const PageMap& pm) {
     const FastPlan p = make_fast_plan(d);
     float* part_o = reinterpret_cast<float*>(workspace);
     float* part_ml = reinterpret_cast<float*>(static_cast<char*>(workspace) + p.off_ml);
@@ -504,8 +514,11 @@ cudaError_t launch_decode_fast(const Dims& d, const void* q, const void* k_cache
     if (stages & 2) {
         CUtensorMap tm_k, tm_c;
         const uint32_t box[3] = {64, (uint32_t)p.T, 1};
-        const uint64_t dk[3] = {(uint64_t)d.d_h, (uint64_t)S_cap, (uint64_t)d.B * d.n_k};
-        const uint64_t dc[3] = {(uint64_t)d.d_l, (uint64_t)S_cap, (uint64_t)d.B * d.n_c};
+        // planes of rows: one per (sequence, group), S_cap rows each -- or one per (page, group), page_size rows
+        const uint64_t rows = pm.table ? (uint64_t)pm.page_size : (uint64_t)S_cap;
+        const uint64_t outer = pm.table ? (uint64_t)pm.n_pages : (uint64_t)d.B;
+        const uint64_t dk[3] = {(uint64_t)d.d_h, rows, outer * d.n_k};
+        const uint64_t dc[3] = {(uint64_t)d.d_l, rows, outer * d.n_c};
         if (!make_bf16_map(&tm_k, k_cache, 3, dk, box) || !make_bf16_map(&tm_c, c_cache, 3, dc, box))
             return cudaErrorInvalidValue;
         const size_t smem = (size_t)kStreamStages * (kStreamStageBytes / p.occ) + 2 * 8 * kStreamMaxT * sizeof(float) +
@@ -527,7 +540,7 @@ cudaError_t launch_decode_fast(const Dims& d, const void* q, const void* k_cache
             cfg.attrs = attr;                                                                              \
             cfg.numAttrs = 1;                                                                              \
             err = cudaLaunchKernelEx(&cfg, kern, tm_k, tm_c, d, p.T, S_cap, (const __nv_bfloat16*)q,       \
-                                     seq_lens, part_o, part_ml, status_word);                              \
+                                     seq_lens, part_o, part_ml, status_word, pm);                          \
             if (err != cudaSuccess) return err;                                                            \
         } while (0)
 #define GTA_LAUNCH_STREAM(NT)                                                                              \

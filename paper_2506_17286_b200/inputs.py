@@ -132,3 +132,35 @@ def decode_inputs(w: Workload, device="cpu", s_cap: int | None = None, seq_lens=
     out = {name: t.to(dev).to(dt).contiguous() for name, t in small.items()}
     out.update(k_cache=k_cache, c_cache=c_cache, seq_lens=lens.to(dev), s_cap=s_cap)
     return out
+
+
+def paginate(t: dict, page_size: int, seed: int = 0, spare_pages: int = 3) -> dict:
+    """The decode inputs `t` (from decode_inputs) with the caches laid out as a paged pool.
+
+    Adds k_pool [n_pages, n_k, page_size, d_h], c_pool [n_pages, n_c, page_size, d_l],
+    block_table int32 [B, max_pages] and page_size; max_pages = ceil(s_cap / page_size), and token
+    t of sequence b sits in row t % page_size of page block_table[b, t // page_size].  The pages of
+    all sequences are dealt out by a seeded random permutation of the pool (`spare_pages` pages stay
+    unassigned); rows no sequence maps to hold N(0,1) values.  Pure data movement.
+    """
+    k_cache, c_cache = t["k_cache"], t["c_cache"]
+    B, n_k, s_cap, d_h = k_cache.shape
+    n_c, d_l = c_cache.shape[1], c_cache.shape[3]
+    dev, dt = k_cache.device, k_cache.dtype
+    max_pages = max(1, -(-s_cap // page_size))
+    n_pages = B * max_pages + spare_pages
+    gen = torch.Generator("cpu").manual_seed(seed + 4242)
+    table = torch.randperm(n_pages, generator=gen)[: B * max_pages].reshape(B, max_pages).to(torch.int32)
+    dgen = torch.Generator(dev).manual_seed(seed + 4243)
+    k_pool = torch.randn((n_pages, n_k, page_size, d_h), generator=dgen, dtype=torch.float32, device=dev).to(dt)
+    c_pool = torch.randn((n_pages, n_c, page_size, d_l), generator=dgen, dtype=torch.float32, device=dev).to(dt)
+    idx = table.to(dev).long()
+    for b in range(B):
+        for j in range(max_pages):
+            lo, hi = j * page_size, min((j + 1) * page_size, s_cap)
+            k_pool[idx[b, j], :, : hi - lo] = k_cache[b, :, lo:hi]
+            c_pool[idx[b, j], :, : hi - lo] = c_cache[b, :, lo:hi]
+    out = dict(t)
+    out.update(k_pool=k_pool, c_pool=c_pool, block_table=table.to(dev).contiguous(), page_size=page_size,
+               max_pages=max_pages, n_pages=n_pages)
+    return out

@@ -1,7 +1,7 @@
 """Run one named synthetic workload through the C-ABI library and print per-kernel device times.
 
     python -m paper_2506_17286_b200.run_workload c3_decode_bf16 [--iters 20] [--warmup 3]
-           [--batch B] [--seq N] [--stages MASK]
+           [--batch B] [--seq N] [--stages MASK] [--append] [--page-size P] [--kv-len L]
 
 A small, self-contained driver for timing or profiling one call at a time (the benchmark
 times the whole step).  Times are CUDA-event times on the launching stream; between
@@ -96,6 +96,50 @@ def run_prefill(w, iters, warmup, stages):
     return {names[m]: _median(v) for m, v in times.items()}
 
 
+def run_decode_paged(w, iters, warmup, append, page_size):
+    """The decode workload with its caches in a paged pool (gta_decode_paged, whole call only)."""
+    dev = torch.device("cuda")
+    sets = []
+    for s in range(2):
+        td = I.paginate(I.decode_inputs(I.scaled(w, seed=w.seed + s), device=dev), page_size, seed=w.seed + s)
+        del td["k_cache"], td["c_cache"]
+        td["lens0"] = td["seq_lens"].clone()
+        sets.append(td)
+    td = sets[0]
+    shape = G.decode_shape(td["q"], td["k_pool"], td["c_pool"], td["x_t"], td["w_p"])
+    ws = torch.zeros(G.decode_paged_workspace_bytes(shape, page_size, td["max_pages"]), dtype=torch.uint8, device=dev)
+    out = torch.empty((w.batch, w.n_heads, w.d_h), dtype=w.torch_dtype(), device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    stream = torch.cuda.current_stream()
+
+    def step(it):
+        td = sets[it % 2]
+        if append:
+            td["seq_lens"].copy_(td["lens0"] - 1)
+            G.gta_cache_append_paged(td["k_pool"], td["c_pool"], td["block_table"], td["k_new"], td["c_new"],
+                                     td["seq_lens"], status_word=status)
+        G.gta_decode_paged(td["q"], td["k_pool"], td["c_pool"], td["block_table"], td["seq_lens"], td["x_t"],
+                           td["w_p"], td["w_g"], out=out, workspace=ws, status_word=status)
+
+    for it in range(warmup):
+        step(it)
+    torch.cuda.synchronize()
+    times = []
+    for rep in range(3):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for it in range(iters):
+            step(it)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        times.append(e0.elapsed_time(e1) / iters)
+    assert int(status.item()) == 0, "device status word raised"
+    lens = sets[0]["lens0"].cpu().tolist()
+    return {"whole_call": _median(times), "append_included": bool(append), "page_size": page_size,
+            "launches": G.last_launch_count(),
+            "cache_bytes": float(sum(lens)) * (w.n_k * w.d_h + w.n_c * w.d_l) * 2}
+
+
 def run_decode(w, iters, warmup, stages, append):
     dev = torch.device("cuda")
     sets = []
@@ -164,6 +208,8 @@ def main():
     ap.add_argument("--append", action="store_true", help="decode: run gta_cache_append before every step")
     ap.add_argument("--kv-len", type=int, default=0,
                     help="prefill: treat the workload's tokens as the last chunk of a context of this length")
+    ap.add_argument("--page-size", type=int, default=0,
+                    help="decode: keep the caches in a paged pool with pages of this many tokens")
     args = ap.parse_args()
     w = I.CONFIGS[args.workload]
     if args.batch:
@@ -176,6 +222,8 @@ def main():
         res = run_prefill_chunk(w, args.iters, args.warmup, args.kv_len)
     elif w.kind == "prefill":
         res = run_prefill(w, args.iters, args.warmup, args.stages & 3)
+    elif args.page_size > 0:
+        res = run_decode_paged(w, args.iters, args.warmup, args.append, args.page_size)
     else:
         res = run_decode(w, args.iters, args.warmup, args.stages, args.append)
     print(json.dumps({"workload": w.name, "batch": w.batch, "seq": w.seq, "median_ms": res}))

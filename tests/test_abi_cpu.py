@@ -34,8 +34,8 @@ def test_every_declared_symbol_is_exported(B):
 
 def test_version_and_status_strings(B):
     assert B.version() >= 100
-    seen = {B.status_string(i) for i in range(7)}
-    assert len(seen) == 7 and B.status_string(0) == "ok"
+    seen = {B.status_string(i) for i in range(9)}
+    assert len(seen) == 9 and B.status_string(0) == "ok"
     assert B.status_string(99) == "unknown status"
 
 
@@ -106,6 +106,29 @@ def test_bad_arguments_are_rejected_on_the_host(B):
     assert append(good, n_new=-1) == B.GTA_ERR_INVALID_ARG
     assert append(good, lens=None) == B.GTA_ERR_INVALID_ARG
     assert append(good, n_new=0) == B.GTA_OK
+
+    def decode_paged(shape, table=p, page_size=64, n_pages=10, max_pages=4, ws_bytes=1 << 40):
+        return L.gta_decode_paged(ctypes.byref(shape), p, p, p, table, page_size, n_pages, max_pages, p, p, p, p, p,
+                                  p, ws_bytes, None, None)
+
+    assert decode_paged(good, table=None) == B.GTA_ERR_INVALID_ARG
+    assert decode_paged(good, table=odd) == B.GTA_ERR_INVALID_ARG
+    assert decode_paged(good, page_size=0) == B.GTA_ERR_INVALID_ARG
+    assert decode_paged(good, n_pages=0) == B.GTA_ERR_INVALID_ARG
+    assert decode_paged(good, max_pages=-3) == B.GTA_ERR_INVALID_ARG
+    assert decode_paged(good, page_size=1 << 20, max_pages=1 << 12) == B.GTA_ERR_INVALID_ARG   # capacity over int32
+    assert decode_paged(good, ws_bytes=8) == B.GTA_ERR_WORKSPACE
+    assert decode_paged(_shape(B, batch=0)) == B.GTA_OK
+    assert B.decode_paged_workspace_bytes(good, 64, 4) == B.decode_workspace_bytes(good, 256)
+    assert B.decode_paged_workspace_bytes(good, 0, 4) == 0
+
+    def append_paged(shape, table=p, page_size=64, n_new=1):
+        return L.gta_cache_append_paged(ctypes.byref(shape), p, p, table, page_size, 10, 4, p, p, n_new, p, None, None)
+
+    assert append_paged(good, table=None) == B.GTA_ERR_INVALID_ARG
+    assert append_paged(good, page_size=-1) == B.GTA_ERR_INVALID_ARG
+    assert append_paged(good, n_new=-1) == B.GTA_ERR_INVALID_ARG
+    assert append_paged(good, n_new=0) == B.GTA_OK
 
 
 def test_binding_rejects_cpu_tensors_and_missing_library(B, monkeypatch):

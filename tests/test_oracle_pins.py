@@ -295,3 +295,61 @@ def test_cache_append_is_a_byte_copy_with_overflow_skip(oracle):
     want_k[1, :, 4:6] = kn[1]; want_c[1, :, 4:6] = cn[1]
     assert np.array_equal(k2, want_k) and np.array_equal(c2, want_c)
     assert np.array_equal(kc[2], k2[2]) and np.array_equal(cc[2], c2[2])
+
+
+# --------------------------------------------------------------------------- paged cache
+def _paged_problem(page_size, lens, seed=5):
+    """A decode problem over contiguous caches plus the same caches scattered into a shuffled pool."""
+    rng = np.random.default_rng(seed)
+    B = len(lens)
+    s = Shape(B, 0, 12, 4, 4, 2, 1, 8, 16, 1)
+    max_pages = -(-max(max(lens), 1) // page_size) + 1
+    cap = max_pages * page_size
+    kc = rng.standard_normal((B, s.n_k, cap, s.d_h)); cc = rng.standard_normal((B, s.n_c, cap, s.d_l))
+    n_pages = B * max_pages + 2
+    table = rng.permutation(n_pages)[: B * max_pages].reshape(B, max_pages)
+    kp = rng.standard_normal((n_pages, s.n_k, page_size, s.d_h)); cp = rng.standard_normal((n_pages, s.n_c, page_size, s.d_l))
+    # scatter by slices (the oracle's view goes token by token: two different index computations)
+    for b in range(B):
+        for j in range(max_pages):
+            kp[table[b, j]] = kc[b, :, j * page_size:(j + 1) * page_size]
+            cp[table[b, j]] = cc[b, :, j * page_size:(j + 1) * page_size]
+    rest = dict(q=rng.standard_normal((B, s.n_q, s.d_h)), x_t=rng.standard_normal((B, s.d_model)),
+                w_p=rng.standard_normal((s.n_heads, s.d_l, s.d_h)) * 0.25,
+                w_g=rng.standard_normal((s.d_model, s.n_heads * s.d_h)) * 0.3)
+    return s, kc, cc, kp, cp, table, cap, rest
+
+
+@pytest.mark.parametrize("page_size", [1, 4, 7])
+def test_paged_decode_does_not_depend_on_where_the_pages_lie(oracle, page_size):
+    lens = [0, 1, page_size, page_size + 1, 3 * page_size - 1, 19]
+    s, kc, cc, kp, cp, table, cap, r = _paged_problem(page_size, lens)
+    assert np.array_equal(oracle.paged_view(kp, table, page_size), kc)
+    assert np.array_equal(oracle.paged_view(cp, table, page_size), cc)
+    want = oracle.decode(s, r["q"], kc, cc, lens, cap, r["x_t"], r["w_p"], r["w_g"])
+    got = oracle.decode_paged(s, r["q"], kp, cp, table, page_size, lens, r["x_t"], r["w_p"], r["w_g"])
+    assert np.array_equal(got, want)
+    # pages no live token maps to may be unassigned
+    holes = table.copy()
+    for b, n in enumerate(lens):
+        holes[b, -(-n // page_size):] = -1
+    got = oracle.decode_paged(s, r["q"], kp, cp, holes, page_size, lens, r["x_t"], r["w_p"], r["w_g"])
+    assert np.array_equal(got, want)
+
+
+@pytest.mark.parametrize("n_new", [1, 5])
+def test_paged_append_equals_contiguous_append_seen_through_the_block_table(oracle, n_new):
+    page_size, lens = 4, [0, 3, 4, 10, 17]
+    s, kc, cc, kp, cp, table, cap, _ = _paged_problem(page_size, lens, seed=9)
+    lens = np.array(lens, dtype=np.int32)
+    lens[-1] = cap - n_new + 1                       # the last sequence would overflow
+    rng = np.random.default_rng(3)
+    kn = rng.standard_normal((len(lens), s.n_k, n_new, s.d_h)); cn = rng.standard_normal((len(lens), s.n_c, n_new, s.d_l))
+    wk, wc, wl, wov = oracle.cache_append(s, kc, cc, cap, kn, cn, n_new, lens)
+    gk, gc, gl, gov = oracle.cache_append_paged(kp, cp, table, page_size, kn, cn, lens)
+    assert gov == wov == 1 and gl.tolist() == wl.tolist()
+    assert np.array_equal(oracle.paged_view(gk, table, page_size), wk)
+    assert np.array_equal(oracle.paged_view(gc, table, page_size), wc)
+    # pages outside the block table are untouched
+    unused = sorted(set(range(kp.shape[0])) - set(table.ravel().tolist()))
+    assert np.array_equal(gk[unused], kp[unused]) and np.array_equal(gc[unused], cp[unused])

@@ -321,3 +321,157 @@ def test_append_then_decode_sequence_of_steps(B, oracle):
         assert lens.cpu().numpy().tolist() == hl.tolist()
         assert torch.equal(kc.cpu(), hk) and torch.equal(cc.cpu(), hc)
         assert_close(out, want, torch.bfloat16, "step")
+
+
+# --------------------------------------------------------------------------- paged cache
+def _paged_decode_case(B, oracle, w, page_size, seq_lens=None, s_cap=None, sample=None, holes=True):
+    """gta_decode_paged against the oracle reading the same pools through the same block table."""
+    t = I.paginate(I.decode_inputs(w, device="cuda", s_cap=s_cap, seq_lens=seq_lens), page_size, seed=w.seed)
+    table = t["block_table"].clone()
+    if holes:   # entries no live token maps to are never read: poison them
+        lens_h = t["seq_lens"].cpu().tolist()
+        for b, n in enumerate(lens_h):
+            table[b, -(-n // page_size):] = -7
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    shape = B.decode_shape(t["q"], t["k_pool"], t["c_pool"], t["x_t"], t["w_p"])
+    ws = torch.full((B.decode_paged_workspace_bytes(shape, page_size, t["max_pages"]),), 0xFF, dtype=torch.uint8,
+                    device="cuda")
+    out = B.gta_decode_paged(t["q"], t["k_pool"], t["c_pool"], table, t["seq_lens"], t["x_t"], t["w_p"], t["w_g"],
+                             status_word=status, workspace=ws)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    idx = list(range(w.batch)) if sample is None else sample
+    sel = torch.as_tensor(idx, device="cuda", dtype=torch.long)
+    lens = t["seq_lens"][sel].cpu().numpy()
+    # the oracle sees the pages of the sampled sequences only, renumbered (its view walks every entry)
+    n_used = max(1, -(-int(lens.max()) // page_size)) if len(idx) else 1
+    sub = t["block_table"][sel][:, :n_used].cpu().numpy()
+    pages, inverse = np.unique(sub, return_inverse=True)
+    pp = torch.as_tensor(pages, device="cuda", dtype=torch.long)
+    want = oracle.decode_paged(oracle_shape(I.scaled(w, batch=len(idx)), seq=0), t["q"][sel].cpu(),
+                               t["k_pool"][pp].cpu(), t["c_pool"][pp].cpu(), inverse.reshape(sub.shape), page_size,
+                               lens, t["x_t"][sel].cpu(), t["w_p"].cpu(), t["w_g"].cpu())
+    return assert_close(out[sel], want, w.torch_dtype(), w.name)
+
+
+PAGED_DECODE = [
+    # name, dtype, B, H, n_h, n_q, n_k, n_c, d_h, d_l, page_size, lens
+    ("bf16_pages_of_64", "bf16", 6, 256, 8, 4, 4, 1, 128, 512, 64, [1, 63, 64, 65, 700, 0]),
+    ("bf16_pages_of_128_batch_40", "bf16", 40, 256, 8, 4, 4, 1, 128, 512, 128, [1 + (37 * i) % 600 for i in range(40)]),
+    ("bf16_pages_of_256_paper_1b_shape", "bf16", 3, 1280, 20, 5, 1, 1, 64, 128, 256, [333, 1000, 256]),
+    ("bf16_pages_of_64_two_latents", "bf16", 5, 256, 8, 4, 4, 2, 128, 256, 64, [129, 1, 64, 400, 33]),
+    # page sizes the streaming kernel does not take (no multiple of 64), and fp32: the plain-ALU kernels
+    ("bf16_pages_of_16", "bf16", 4, 128, 4, 2, 2, 1, 128, 256, 16, [0, 512, 1, 300]),
+    ("bf16_pages_of_48", "bf16", 3, 128, 8, 4, 2, 2, 64, 128, 48, [200, 5, 129]),
+    ("f32_pages_of_5", "f32", 3, 96, 6, 6, 3, 1, 32, 64, 5, [100, 7, 260]),
+]
+
+
+@pytest.mark.parametrize("case", PAGED_DECODE, ids=[c[0] for c in PAGED_DECODE])
+def test_decode_paged_small_shapes(B, oracle, case):
+    name, dt, nb, H, n_h, n_q, n_k, n_c, d_h, d_l, page_size, lens = case
+    w = I.Workload(name, "decode", dt, nb, 0, H, n_h, n_q, n_k, n_c, d_h, d_l, seed=77)
+    _paged_decode_case(B, oracle, w, page_size, seq_lens=lens, s_cap=max(lens) + 13)
+
+
+def test_decode_paged_config3_full_size_sampled_sequences(B, oracle):
+    w = I.CONFIGS["c3_decode_bf16"]
+    _paged_decode_case(B, oracle, w, 64, sample=[0, w.batch // 2, w.batch - 1])
+
+
+def test_decode_paged_is_bitwise_the_contiguous_decode_on_the_streaming_path(B):
+    """Same kernels, same order of operations: only the tile addresses differ."""
+    w = I.Workload("paged_vs_flat", "decode", "bf16", 9, 0, 256, 8, 4, 4, 1, 128, 512, seed=3)
+    lens = [257, 256, 255, 1, 2, 1000, 64, 128, 511]
+    t = I.paginate(I.decode_inputs(w, device="cuda", s_cap=1024, seq_lens=lens), 128, seed=1)
+    flat = B.gta_decode(t["q"], t["k_cache"], t["c_cache"], t["seq_lens"], t["x_t"], t["w_p"], t["w_g"])
+    paged = B.gta_decode_paged(t["q"], t["k_pool"], t["c_pool"], t["block_table"], t["seq_lens"], t["x_t"],
+                               t["w_p"], t["w_g"])
+    torch.cuda.synchronize()
+    assert torch.equal(flat, paged)
+
+
+@pytest.mark.parametrize("dt", ["bf16", "f32"])
+@pytest.mark.parametrize("n_new", [1, 3, 200])
+def test_cache_append_paged_is_bit_exact(B, oracle, dt, n_new):
+    tdt = torch.bfloat16 if dt == "bf16" else torch.float32
+    nb, n_k, n_c, d_h, d_l, page_size, max_pages = 6, 4, 2, 64, 128, 64, 5
+    cap = page_size * max_pages
+    g = torch.Generator("cpu").manual_seed(321 + n_new)
+    n_pages = nb * max_pages + 4
+    k_pool = torch.randn(n_pages, n_k, page_size, d_h, generator=g).to(tdt)
+    c_pool = torch.randn(n_pages, n_c, page_size, d_l, generator=g).to(tdt)
+    k_new = torch.randn(nb, n_k, n_new, d_h, generator=g).to(tdt)
+    c_new = torch.randn(nb, n_c, n_new, d_l, generator=g).to(tdt)
+    table = torch.randperm(n_pages, generator=g)[: nb * max_pages].reshape(nb, max_pages).to(torch.int32)
+    # page boundaries inside the new rows, a full sequence and one that would overflow
+    lens = torch.tensor([0, page_size - 1, cap - n_new, cap - n_new + 1, cap, 2 * page_size - 2], dtype=torch.int32)
+    wk, wc, wl, wov = oracle.cache_append_paged(k_pool, c_pool, table.numpy(), page_size, k_new, c_new, lens.numpy())
+    assert wov == 1
+
+    dk, dc, dl = k_pool.cuda(), c_pool.cuda(), lens.cuda()
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    B.gta_cache_append_paged(dk, dc, table.cuda(), k_new.cuda(), c_new.cuda(), dl, status_word=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == B.GTA_ERR_CACHE_FULL
+    assert dl.cpu().numpy().tolist() == wl.tolist()
+
+    def bits(t):
+        t = t.cpu().contiguous()
+        return t.view(torch.int16).numpy().view(np.uint16) if t.dtype == torch.bfloat16 else t.numpy().view(np.uint32)
+
+    want_k = wk if dt == "bf16" else wk.view(np.uint32)
+    want_c = wc if dt == "bf16" else wc.view(np.uint32)
+    assert np.array_equal(bits(dk), want_k.reshape(bits(dk).shape))
+    assert np.array_equal(bits(dc), want_c.reshape(bits(dc).shape))
+
+
+def test_paged_append_then_decode_sequence_of_steps(B, oracle):
+    """Decode steps over a paged cache, each after an append that may open a new page."""
+    w = I.Workload("paged_steps", "decode", "bf16", 4, 0, 128, 4, 2, 2, 1, 128, 256, seed=56)
+    page_size = 64
+    t = I.paginate(I.decode_inputs(w, device="cuda", s_cap=192, seq_lens=[10, 63, 0, 127]), page_size, seed=2)
+    kp, cp, lens, table = t["k_pool"].clone(), t["c_pool"].clone(), t["seq_lens"].clone(), t["block_table"]
+    hk, hc, hl, ht = kp.cpu(), cp.cpu(), lens.cpu().numpy(), table.cpu().numpy()
+    g = torch.Generator("cpu").manual_seed(9)
+    shape = oracle_shape(w, seq=0)
+    for _ in range(3):
+        k_new = torch.randn(w.batch, w.n_k, 1, w.d_h, generator=g).to(torch.bfloat16)
+        c_new = torch.randn(w.batch, w.n_c, 1, w.d_l, generator=g).to(torch.bfloat16)
+        q = torch.randn(w.batch, w.n_q, w.d_h, generator=g).to(torch.bfloat16)
+        x_t = torch.randn(w.batch, w.d_model, generator=g).to(torch.bfloat16)
+        B.gta_cache_append_paged(kp, cp, table, k_new.cuda(), c_new.cuda(), lens)
+        out = B.gta_decode_paged(q.cuda(), kp, cp, table, lens, x_t.cuda(), t["w_p"], t["w_g"])
+        nk, nc, hl, _ = oracle.cache_append_paged(hk, hc, ht, page_size, k_new, c_new, hl)
+        hk = torch.from_numpy(nk.view(np.int16)).view(torch.bfloat16).reshape(hk.shape)
+        hc = torch.from_numpy(nc.view(np.int16)).view(torch.bfloat16).reshape(hc.shape)
+        want = oracle.decode_paged(shape, q, hk, hc, ht, page_size, hl, x_t, t["w_p"].cpu(), t["w_g"].cpu())
+        torch.cuda.synchronize()
+        assert lens.cpu().numpy().tolist() == hl.tolist()
+        assert torch.equal(kp.cpu(), hk) and torch.equal(cp.cpu(), hc)
+        assert_close(out, want, torch.bfloat16, "paged step")
+
+
+@pytest.mark.parametrize("page_size", [64, 16])
+def test_block_table_entry_outside_the_pool_raises_the_status_word(B, page_size):
+    """Both kernel families check the entries they use: the call completes, touches nothing outside the
+    pools and reports GTA_ERR_BAD_PAGE."""
+    w = I.Workload("bad_page", "decode", "bf16", 3, 0, 128, 4, 2, 2, 1, 128, 256, seed=4)
+    t = I.paginate(I.decode_inputs(w, device="cuda", s_cap=256, seq_lens=[100, 200, 30]), page_size, seed=3)
+    table = t["block_table"].clone()
+    table[1, 1] = t["n_pages"] + 5
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    out = B.gta_decode_paged(t["q"], t["k_pool"], t["c_pool"], table, t["seq_lens"], t["x_t"], t["w_p"], t["w_g"],
+                             status_word=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == B.GTA_ERR_BAD_PAGE
+    assert torch.isfinite(out.float()).all()
+    # the append refuses the row as well: sequence 1's next token falls into the bad page when it starts there
+    lens = torch.tensor([100, page_size, 30], dtype=torch.int32, device="cuda")
+    status.zero_()
+    before_k, before_c = t["k_pool"].clone(), t["c_pool"].clone()
+    B.gta_cache_append_paged(t["k_pool"], t["c_pool"], table, t["k_new"], t["c_new"], lens, status_word=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == B.GTA_ERR_BAD_PAGE
+    changed = (t["k_pool"] != before_k).flatten(1).any(1).sum().item()
+    assert changed == 2   # the two good sequences wrote one row each, each in a page of its own
