@@ -372,6 +372,29 @@ def run_ours(args):
     barrier()
     t_decode_call = d2.elapsed_time(d3) / K_d
     assert int(status.item()) == 0, "device status word raised during the benchmark"
+    # ---- the same call over a paged cache (pages of 64 tokens dealt out at random), back to back
+    page_size = 64
+    psets = [I.paginate(td, page_size, seed=wd.seed + i) for i, td in enumerate(sets)]
+    ws_pg = torch.zeros(G.decode_paged_workspace_bytes(shape_d, page_size, psets[0]["max_pages"]), dtype=torch.uint8,
+                        device=dev)
+
+    def decode_paged_call(i):
+        td = psets[i % 2]
+        G.gta_decode_paged(td["q"], td["k_pool"], td["c_pool"], td["block_table"], td["seq_lens"], td["x_t"],
+                           td["w_p"], td["w_g"], out=out_d, workspace=ws_pg, status_word=status)
+
+    for i in range(3):
+        decode_paged_call(i)
+    barrier()
+    d4, d5 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    d4.record(stream)
+    for i in range(K_d):
+        decode_paged_call(i)
+    d5.record(stream)
+    barrier()
+    t_decode_paged = d4.elapsed_time(d5) / K_d
+    assert int(status.item()) == 0, "device status word raised during the benchmark"
+    del psets, ws_pg
 
     total_ms = e_start.elapsed_time(e_end)
     t_attn = sum(e[0].elapsed_time(e[1]) for e in evk) / K_k
@@ -388,6 +411,7 @@ def run_ours(args):
     t_decode, t_decode_leg = max_over_ranks_(t_decode), max_over_ranks_(t_decode_leg)
     t_decode_b2b = max_over_ranks_(t_decode_b2b)
     t_decode_call = max_over_ranks_(t_decode_call)
+    t_decode_paged = max_over_ranks_(t_decode_paged)
 
     fl = prefill_flops(wp)
     by = decode_bytes(wd, [wd.seq] * wd.batch)
@@ -428,6 +452,11 @@ def run_ours(args):
                                              "length vector, prepared before the loop)"}},
     }
     decode["roofline"]["frac"] = decode["roofline"]["achieved"] / decode["roofline"]["peak"]
+    decode["paged"] = {"page_size": page_size, "ms_decode_call": t_decode_paged,
+                       "achieved": by["total"] / (t_decode_paged * 1e-3) / 1e9,
+                       "frac": by["total"] / (t_decode_paged * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                       "note": "gta_decode_paged back to back on the same caches scattered over a pool of 64-token "
+                               "pages in random order"}
 
     # ---- end to end: pinned host buffers -> device -> gta_prefill -> pinned host buffer, every step.
     #      Copies and compute run on three streams with double-buffered device inputs and outputs, so
