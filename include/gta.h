@@ -201,6 +201,38 @@ GTA_API gta_status_t gta_cache_append_paged(const gta_shape_t *shape, void *k_po
                                             int32_t *status_word, void *cuda_stream);
 
 /*
+ * gta_layer_prefill — the whole attention layer of App. B.1.1 for a chunk of N tokens per sequence
+ * that starts at position pos0 (pos0 = 0: a prompt):
+ *
+ *   [q | k | c]_t = x_t W_qkc                 one matrix, columns = the n_q query groups (d_h each), then
+ *                                             the n_k key groups (d_h each), then the n_c latent groups (d_l each)
+ *   q, k <- RoPE(q, k; position pos0 + t)     per d_h-vector, pairs of neighbouring elements (2i, 2i+1)
+ *                                             rotated by (pos0 + t) rope_base^(-2i/d_h)  (RoFormer, which the
+ *                                             paper cites; the paper does not fix the pairing or the base)
+ *   k_cache[b, :, pos0 + t, :] = k_t,  c_cache[b, :, pos0 + t, :] = c_t       (the prefill's bulk append)
+ *   o_t = gta_prefill_chunk of the chunk's queries over cache rows 0 .. pos0 + N - 1, gated by x_t
+ *   u_t = [o_{t,1}; ...; o_{t,n_h}] W_o
+ *
+ *   x [B, N, H]   w_qkc [H, (n_q + n_k) d_h + n_c d_l]   w_p, w_g as in gta_prefill   w_o [n_h d_h, H]
+ *   k_cache [B, n_k, S_cap, d_h]   c_cache [B, n_c, S_cap, d_l]   (rows pos0 .. pos0 + N - 1 are written,
+ *   rows below pos0 are read, rows above are left alone; no length vector is read or written)
+ *   u [B, N, H]   workspace: gta_layer_prefill_workspace_bytes(shape), 256-byte aligned (q, the gated
+ *   heads and the operator's own workspace).
+ * q, k, c and the gated heads are rounded to the storage type where they are stored (the caches and
+ * the workspace), as every tensor of the operator is.
+ * bf16 only, on the tensor-core kernels: H a multiple of 128, d_h = 64 or 128, d_l a multiple of 64,
+ * (n_q + n_k) d_h + n_c d_l a multiple of 128; otherwise GTA_ERR_UNSUPPORTED.  GTA_ERR_INVALID_ARG
+ * also for pos0 < 0, pos0 + N > S_cap, rope_base <= 1 or a non-causal shape.
+ */
+GTA_API size_t gta_layer_prefill_workspace_bytes(const gta_shape_t *shape);
+GTA_API gta_status_t gta_layer_prefill(const gta_shape_t *shape, int32_t pos0, int32_t S_cap,
+                                       float rope_base, const void *x, const void *w_qkc,
+                                       const void *w_p, const void *w_g, const void *w_o,
+                                       void *k_cache, void *c_cache, void *u, void *workspace,
+                                       size_t workspace_bytes, int32_t *status_word,
+                                       void *cuda_stream);
+
+/*
  * gta_decode_static — gta_decode without a workspace argument (the paper has no counterpart: this
  * is a packaging variant of the same decode step, with the same arguments, results and errors).
  *

@@ -242,6 +242,76 @@ def cache_append_paged(k_pool, c_pool, block_table, page_size: int, k_new, c_new
     return k_pool, c_pool, lens, overflowed
 
 
+def _to_f64(a):
+    """Operator tensor in any accepted storage form -> float64 numpy array (exact widening)."""
+    a, code = _as_np(a)
+    if code == BF16:
+        return (a.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+    return a.astype(np.float64)
+
+
+def round_to_storage(a, storage: int):
+    """float64 array rounded to the storage type (round to nearest even), returned as float64: what a
+    tensor holds after it has been written to a bf16 / fp32 buffer."""
+    a = np.asarray(a, dtype=np.float64)
+    if storage == F64:
+        return a.copy()
+    f = a.astype(np.float32)
+    if storage == F32:
+        return f.astype(np.float64)
+    bits = f.view(np.uint32).astype(np.uint64)
+    bits = ((bits + 0x7FFF + ((bits >> 16) & 1)) >> 16) << 16
+    return bits.astype(np.uint32).view(np.float32).astype(np.float64)
+
+
+def rope(v, positions, base: float = 10000.0):
+    """Rotary position embedding of RoFormer (the RoPE the layer definition of App. B.1.1 applies to
+    q and k): in a vector of even width d, elements (2i, 2i+1) form a pair that is rotated by the
+    angle  position * base^(-2i/d).  v [..., N, d] float64, positions [N]."""
+    v = np.asarray(v, dtype=np.float64)
+    d = v.shape[-1]
+    assert d % 2 == 0 and v.shape[-2] == len(positions)
+    out = np.empty_like(v)
+    for i in range(d // 2):
+        theta = base ** (-2.0 * i / d)
+        ang = np.asarray(positions, dtype=np.float64) * theta
+        x0, x1 = v[..., 2 * i], v[..., 2 * i + 1]
+        out[..., 2 * i] = x0 * np.cos(ang) - x1 * np.sin(ang)
+        out[..., 2 * i + 1] = x0 * np.sin(ang) + x1 * np.cos(ang)
+    return out
+
+
+def layer_prefill(shape: Shape, x, w_qkc, w_p, w_g, w_o, rope_base: float = 10000.0, storage: int = BF16,
+                  n_threads: int = 0):
+    """The attention layer of App. B.1.1 over a prompt (positions 0 .. N-1):
+        q_t, k_t = RoPE(x_t W_Q), RoPE(x_t W_K);  c_t = x_t W_C        (W_qkc = [W_Q | W_K | W_C], groups
+                                                                         side by side, d_h / d_h / d_l wide)
+        o_t = the operator (prefill) on q, k, c, gated by x_t;          u_t = [o_t,1; ...; o_t,n_h] W_O
+    Tensors that the layer stores between its steps (q, the K and C caches, the gated heads) are rounded
+    to `storage` there; everything else is float64.  Returns dict(u, q, k, c, o) as float64 arrays:
+    u [B, N, H], q [B, n_q, N, d_h], k [B, n_k, N, d_h], c [B, n_c, N, d_l], o [B, N, n_h, d_h]."""
+    s = shape
+    x64, w_qkc, w_o = _to_f64(x), _to_f64(w_qkc), _to_f64(w_o)
+    B, N = s.batch, s.seq
+    Dq, Dk, Dc = s.n_q * s.d_h, s.n_k * s.d_h, s.n_c * s.d_l
+    assert x64.shape == (B, N, s.d_model) and w_qkc.shape == (s.d_model, Dq + Dk + Dc)
+    assert w_o.shape == (s.n_heads * s.d_h, s.d_model)
+    y = x64 @ w_qkc
+    pos = np.arange(N)
+
+    def grouped(cols, groups, width):
+        return cols.reshape(B, N, groups, width).transpose(0, 2, 1, 3)
+
+    q = round_to_storage(rope(grouped(y[..., :Dq], s.n_q, s.d_h), pos, rope_base), storage)
+    k = round_to_storage(rope(grouped(y[..., Dq:Dq + Dk], s.n_k, s.d_h), pos, rope_base), storage)
+    c = round_to_storage(grouped(y[..., Dq + Dk:], s.n_c, s.d_l), storage)
+    o = prefill(s, np.ascontiguousarray(q), np.ascontiguousarray(k), np.ascontiguousarray(c), x64,
+                _to_f64(w_p), _to_f64(w_g), n_threads=n_threads)
+    o = round_to_storage(o, storage)
+    u = o.reshape(B, N, s.n_heads * s.d_h) @ w_o
+    return dict(u=u, q=q, k=k, c=c, o=o)
+
+
 def attention_cost(shape: Shape) -> float:
     """n_q (d_h + d_l) N^2 — Table 3, GTA row, 'Attention' column."""
     cs = shape.c()

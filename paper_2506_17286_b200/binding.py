@@ -25,6 +25,7 @@ EXPORTS = (
     "gta_cache_append", "gta_status_string", "gta_version", "gta_prefill_path", "gta_last_launch_count",
     "gta_prefill_stages", "gta_decode_stages", "gta_decode_static", "gta_prefill_chunk",
     "gta_decode_paged_workspace_bytes", "gta_decode_paged", "gta_cache_append_paged",
+    "gta_layer_prefill_workspace_bytes", "gta_layer_prefill",
 )
 
 
@@ -82,6 +83,10 @@ def lib():
         L.gta_decode_paged.restype = i32
         L.gta_cache_append_paged.argtypes = [sp, vp, vp, vp, i32, i32, i32, vp, vp, i32, vp, vp, vp]
         L.gta_cache_append_paged.restype = i32
+        L.gta_layer_prefill_workspace_bytes.argtypes = [sp]
+        L.gta_layer_prefill_workspace_bytes.restype = sz
+        L.gta_layer_prefill.argtypes = [sp, i32, i32, ctypes.c_float, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp, vp]
+        L.gta_layer_prefill.restype = i32
         L.gta_status_string.argtypes = [i32]
         L.gta_status_string.restype = ctypes.c_char_p
         L.gta_version.restype = i32
@@ -204,6 +209,38 @@ def gta_prefill_chunk(q, k, c, x, w_p, w_g, kv_len, *, causal=True, softmax_scal
                                  workspace.numel() * workspace.element_size(), _ptr(status_word), _stream(stream))
     if st != GTA_OK:
         raise GtaError(st, "gta_prefill_chunk")
+    return out
+
+
+def layer_prefill_workspace_bytes(shape: GtaShape) -> int:
+    return int(lib().gta_layer_prefill_workspace_bytes(ctypes.byref(shape)))
+
+
+def gta_layer_prefill(x, w_qkc, w_p, w_g, w_o, k_cache, c_cache, *, pos0=0, rope_base=10000.0, n_q, softmax_scale=0.0,
+                      out=None, workspace=None, status_word=None, stream=None):
+    """u[B, N, H] = the whole attention layer for a chunk that starts at position pos0: projections + RoPE, keys
+    and latents written to rows pos0 .. pos0+N-1 of the caches, the operator, the output projection.
+    x [B,N,H], w_qkc [H,(n_q+n_k)d_h+n_c d_l], w_o [n_h d_h,H], k_cache [B,n_k,S_cap,d_h], c_cache [B,n_c,S_cap,d_l]."""
+    _check_tensors(x, w_qkc, w_p, w_g, w_o, k_cache, c_cache)
+    B, N, H = x.shape
+    n_h, d_l, d_h = w_p.shape
+    n_k, s_cap, n_c = k_cache.shape[1], k_cache.shape[2], c_cache.shape[1]
+    if k_cache.shape != (B, n_k, s_cap, d_h) or c_cache.shape != (B, n_c, s_cap, d_l) \
+            or w_qkc.shape != (H, (n_q + n_k) * d_h + n_c * d_l) or w_g.shape != (H, n_h * d_h) \
+            or w_o.shape != (n_h * d_h, H):
+        raise ValueError("inconsistent layer tensor shapes")
+    shape = make_shape(batch=B, seq=N, d_model=H, n_heads=n_h, n_q=n_q, n_k=n_k, n_c=n_c, d_h=d_h, d_l=d_l,
+                       dtype=_dtype_code(x), causal=True, softmax_scale=softmax_scale)
+    if out is None:
+        out = torch.empty((B, N, H), dtype=x.dtype, device=x.device)
+    if workspace is None:
+        workspace = _workspace(layer_prefill_workspace_bytes(shape), x.device)
+    st = lib().gta_layer_prefill(ctypes.byref(shape), int(pos0), int(s_cap), float(rope_base), _ptr(x), _ptr(w_qkc),
+                                 _ptr(w_p), _ptr(w_g), _ptr(w_o), _ptr(k_cache), _ptr(c_cache), _ptr(out),
+                                 _ptr(workspace), workspace.numel() * workspace.element_size(), _ptr(status_word),
+                                 _stream(stream))
+    if st != GTA_OK:
+        raise GtaError(st, "gta_layer_prefill")
     return out
 
 

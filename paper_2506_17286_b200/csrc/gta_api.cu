@@ -241,6 +241,58 @@ gta_status_t gta_cache_append_paged(const gta_shape_t* shape, void* k_pool, void
 
 }  // extern "C"
 
+// ---- whole attention layer (App. B.1.1): projections + RoPE + cache write, operator, output projection
+static size_t align256(size_t v) { return (v + 255) & ~(size_t)255; }
+
+extern "C" size_t gta_layer_prefill_workspace_bytes(const gta_shape_t* shape) {
+    gta::Dims d;
+    if (check_shape(shape, true, &d) != GTA_OK) return 0;
+    const size_t es = elem_size(shape->dtype);
+    const size_t q_bytes = align256((size_t)d.B * d.n_q * d.N * d.d_h * es);
+    const size_t o_bytes = align256((size_t)d.B * d.N * d.n_h * d.d_h * es);
+    return q_bytes + o_bytes + gta_prefill_workspace_bytes(shape);
+}
+
+extern "C" gta_status_t gta_layer_prefill(const gta_shape_t* shape, int32_t pos0, int32_t S_cap, float rope_base,
+                                          const void* x, const void* w_qkc, const void* w_p, const void* w_g,
+                                          const void* w_o, void* k_cache, void* c_cache, void* u, void* workspace,
+                                          size_t workspace_bytes, int32_t* status_word, void* cuda_stream) {
+    g_last_launches = 0;
+    gta::Dims d;
+    gta_status_t st = check_shape(shape, true, &d);
+    if (st != GTA_OK) return st;
+    if (pos0 < 0 || S_cap < 0 || (long long)pos0 + d.N > S_cap || !(rope_base > 1.0f)) return GTA_ERR_INVALID_ARG;
+    if (!d.causal) return GTA_ERR_INVALID_ARG;      // a chunk written behind a cache is causal by construction
+    if (!x || !w_qkc || !w_p || !w_g || !w_o || !k_cache || !c_cache || !u) return GTA_ERR_INVALID_ARG;
+    if (!aligned(x, 16) || !aligned(w_qkc, 16) || !aligned(w_p, 16) || !aligned(w_g, 16) || !aligned(w_o, 16) ||
+        !aligned(k_cache, 16) || !aligned(c_cache, 16) || !aligned(u, 16) || !aligned(status_word, 4))
+        return GTA_ERR_INVALID_ARG;
+    if (!gta::sm100_linear_supported(d, shape->dtype) || gta_prefill_path(shape) == 0) return GTA_ERR_UNSUPPORTED;
+    if (d.B == 0 || d.N == 0) return GTA_OK;
+    if (!workspace || !aligned(workspace, 256) || workspace_bytes < gta_layer_prefill_workspace_bytes(shape))
+        return GTA_ERR_WORKSPACE;
+    if ((st = check_device()) != GTA_OK) return st;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const size_t es = elem_size(shape->dtype);
+    char* ws = static_cast<char*>(workspace);
+    void* q_ws = ws;
+    void* o_ws = ws + align256((size_t)d.B * d.n_q * d.N * d.d_h * es);
+    char* op_ws = static_cast<char*>(o_ws) + align256((size_t)d.B * d.N * d.n_h * d.d_h * es);
+    const size_t op_ws_bytes = workspace_bytes - (size_t)(op_ws - ws);
+    st = gta::launch_sm100_project(d, pos0, S_cap, (double)rope_base, x, w_qkc, q_ws, k_cache, c_cache, status_word,
+                                   stream);
+    if (st != GTA_OK) return st;
+    // the chunk's queries against everything the caches now hold for these sequences
+    st = prefill_impl(shape, pos0 + d.N, S_cap, q_ws, k_cache, c_cache, x, w_p, w_g, o_ws, op_ws, op_ws_bytes,
+                      status_word, cuda_stream, 3);
+    if (st != GTA_OK) return st;
+    const int op_launches = g_last_launches;
+    st = gta::launch_sm100_matmul((long long)d.B * d.N, d.n_h * d.d_h, d.H, o_ws, w_o, u, status_word, stream);
+    if (st != GTA_OK) return st;
+    g_last_launches = op_launches + 2;
+    return GTA_OK;
+}
+
 static gta_status_t decode_impl(const gta_shape_t* shape, const void* q, const void* k_cache, const void* c_cache,
                                 const int32_t* seq_lens, int32_t S_cap, const void* x_t, const void* w_p,
                                 const void* w_g, void* out, void* workspace, size_t workspace_bytes,

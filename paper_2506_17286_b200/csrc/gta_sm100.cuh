@@ -17,4 +17,18 @@ gta_status_t launch_sm100_prefill(const Dims& d, const void* q, const void* k, c
 gta_status_t launch_sm100_decoder(const Dims& d, const void* l_bf16, const void* x, const void* w_p, const void* w_g,
                                   void* out, int32_t* status_word, cudaStream_t stream);
 
+// Linear maps of the attention layer around the operator (App. B.1.1), bf16 with fp32 accumulation.
+// True when the tcgen05 kernel covers the layer's projections for this shape.
+bool sm100_linear_supported(const Dims& d, int dtype);
+
+// [Q | K | C] = X W_qkc for the B x N tokens of a chunk that starts at position pos0: RoPE on q and k,
+// q to q_out [B, n_q, N, d_h], k and c to rows pos0 + t of the caches [B, groups, S_cap, width].
+gta_status_t launch_sm100_project(const Dims& d, int pos0, int S_cap, double rope_base, const void* x,
+                                  const void* w_qkc, void* q_out, void* k_cache, void* c_cache,
+                                  int32_t* status_word, cudaStream_t stream);
+
+// C[M, n_cols] = A[M, K] W[K, n_cols], row-major.
+gta_status_t launch_sm100_matmul(long long M, int K, int n_cols, const void* a, const void* w, void* c_out,
+                                 int32_t* status_word, cudaStream_t stream);
+
 }  // namespace gta

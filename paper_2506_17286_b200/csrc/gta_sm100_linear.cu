@@ -1,0 +1,356 @@
+// tcgen05 / TMA linear maps of the attention layer around the operator (App. B.1.1):
+//
+//   input projections   [Q | K | C] = H_in [W_Q | W_K | W_C],  q and k then pass through RoPE and every
+//                       column block goes straight to where the operator reads it: q to [B, n_q, N, d_h],
+//                       k and c to rows pos0 + t of the caches (the prefill's bulk append);
+//   output projection   u_t = W_O [o_{t,1} (.) g_{t,1}; ...]  (the operator's output times W_O).
+//
+// One kernel, C[M, n_cols] = A[M, K] W[K, n_cols] in bf16 with fp32 accumulation, two epilogues.
+// Persistent CTA pairs (clusters of 2, tcgen05 cta_group::2, M = 256): a pair walks the (row tile,
+// column block) units pr, pr + G, ...; a column block is 256 columns (128 at the ragged end).  Each
+// CTA owns 128 of the unit's rows and stages its own A rows plus half of the unit's weight columns.
+//   warp 0      TMA producer, 6-stage ring of {A tile 128 x 64, W tile 64 x block / 2}
+//   warp 1      (leader CTA) MMA issuer; two accumulators of 256 TMEM columns alternate between
+//               units, so the epilogue of unit n overlaps the MMAs of unit n + 1
+//   warps 2-9   epilogue: TMEM -> registers -> (RoPE) -> bf16 -> global, one token row per thread
+//
+// RoPE (RoFormer, which the paper cites): the pairs are neighbouring elements (2 i, 2 i + 1) of a
+// d_h-vector, rotated by the angle pos theta_i with theta_i = base^(-2 i / d_h).  The angle is formed
+// and reduced to [-pi, pi] in double precision (theta_i comes from the host as doubles), so that
+// long contexts do not lose the phase; sine and cosine are then single precision.
+#include "gta_sm100.cuh"
+
+#include <cuda.h>
+#include <math.h>
+
+#include "sm100_ptx.cuh"
+#include "tma_host.cuh"
+
+namespace gta {
+
+namespace {
+
+constexpr int kLinStages = 6;
+constexpr int kLinThreads = 320;
+constexpr int kTileM = 128;        // rows per CTA and unit
+constexpr int kBlockK = 64;        // K elements per pipeline stage (one 128-byte swizzle row)
+constexpr uint32_t kATileBytes = kTileM * kBlockK * 2;   // 16 KB
+constexpr uint32_t kBGroupBytes = kBlockK * 64 * 2;      // 64 K-rows x 64 columns = 8 KB
+constexpr uint32_t kStageBytes = kATileBytes + 2 * kBGroupBytes;   // 32 KB per CTA
+constexpr uint32_t kBarOffset = kLinStages * kStageBytes;
+constexpr uint32_t kLinSmemTotal = kBarOffset + 512 + 1024;        // barriers + alignment slack
+constexpr int kMaxRopePairs = 64;  // d_h <= 128
+
+struct LinArgs {
+    int M, K, n_cols;        // C[M, n_cols] = A[M, K] W[K, n_cols]
+    int n_cb;                // column blocks (256 wide, the last one possibly 128)
+    int n_units;             // row tiles (256 rows) x column blocks
+    // plain epilogue
+    __nv_bfloat16* c_out;    // [M, n_cols]
+    // projection epilogue: row = b N + t
+    Dims d;
+    int pos0, S_cap;         // position of token 0 of the chunk; rows per cache plane
+    __nv_bfloat16* q_out;    // [B, n_q, N, d_h]
+    __nv_bfloat16* k_cache;  // [B, n_k, S_cap, d_h]
+    __nv_bfloat16* c_cache;  // [B, n_c, S_cap, d_l]
+    double theta[kMaxRopePairs];
+};
+
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&v);
+}
+
+// kProject: the epilogue of the input projections (RoPE + scatter); otherwise a plain row-major store
+template <bool kProject>
+__global__ void __launch_bounds__(kLinThreads, 1)
+sm100_linear_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_w,
+                    const __grid_constant__ LinArgs a, int32_t* status_word) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + kBarOffset);    // used in the leader CTA
+    uint64_t* empty_bar = full_bar + kLinStages;                             // both CTAs
+    uint64_t* acc_full = empty_bar + kLinStages;                             // [2] both CTAs
+    uint64_t* acc_free = acc_full + 2;                                       // [2] leader CTA: 16 warps arrive
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_free + 2);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+    volatile int* drain_flag = abort_flag + 1;   // never raised: lets the drain wait run to its limit
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = ptx::cluster_ctarank();                       // 0 = leader
+    const int G = gridDim.x >> 1, pr = blockIdx.x >> 1;
+    const int n_items = pr < a.n_units ? (a.n_units - pr + G - 1) / G : 0;
+    const int ks_total = a.K / kBlockK;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kLinStages; ++s) { ptx::mbar_init(&full_bar[s], 2); ptx::mbar_init(&empty_bar[s], 1); }
+        for (int j = 0; j < 2; ++j) { ptx::mbar_init(&acc_full[j], 1); ptx::mbar_init(&acc_free[j], 16); }
+        *abort_flag = 0;
+        *drain_flag = 0;
+        ptx::fence_mbar_init();
+    }
+    if (warp == 1) ptx::tmem_alloc_pair(tmem_slot, 512);
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    ptx::cluster_arrive();     // the peer's barriers exist before anything is signalled to them
+    ptx::cluster_wait();
+    ptx::tc_fence_after_sync();
+    const uint32_t tmem_base = *tmem_slot;
+
+    // unit n of this pair: column block cb (consecutive pairs share a row tile), first row, first column, width
+    auto unit = [&](int n, int& row0, int& f0, int& nt) {
+        const int u = pr + n * G;
+        const int cb = u % a.n_cb;
+        row0 = (u / a.n_cb) * 2 * kTileM;
+        f0 = cb * 256;
+        nt = a.n_cols - f0 < 256 ? a.n_cols - f0 : 256;
+    };
+
+    if (warp == 0) {
+        if (ptx::elect_one()) {
+            ptx::prefetch_tensormap(&tm_a);
+            ptx::prefetch_tensormap(&tm_w);
+            // A may be the result of the kernel before this one in the stream
+            ptx::grid_dependency_wait();
+            int it = 0, s = 0;
+            uint32_t ph = 0;
+            bool ok = true;
+            for (int n = 0; n < n_items && ok; ++n) {
+                int row0, f0, nt;
+                unit(n, row0, f0, nt);
+                const int r0 = row0 + (int)rank * kTileM;          // this CTA's rows
+                const int n_grp = nt / 128;                         // 64-column groups this CTA stages
+                const int fc = f0 + (int)rank * (nt / 2);           // this CTA's first weight column
+                const uint32_t tx = kATileBytes + (uint32_t)n_grp * kBGroupBytes;
+                const uint32_t bar_base = ptx::map_to_cta(ptx::smem_addr(&full_bar[0]), 0);   // the leader's
+                for (int ks = 0; ks < ks_total; ++ks, ++it, s = (s + 1 == kLinStages) ? 0 : s + 1, ph ^= (s == 0)) {
+                    ok = ptx::mbar_wait(&empty_bar[s], ph ^ 1, abort_flag);
+                    if (!ok) break;
+                    uint8_t* a_s = smem + s * kStageBytes;
+                    uint8_t* b_s = a_s + kATileBytes;
+                    const uint32_t bar = bar_base + (uint32_t)s * 8;
+                    ptx::mbar_arrive_expect_tx_cluster(bar, tx);
+                    ptx::tma_load_2d_pair(a_s, &tm_a, bar, ks * kBlockK, r0);
+                    for (int grp = 0; grp < n_grp; ++grp)
+                        ptx::tma_load_2d_pair(b_s + grp * kBGroupBytes, &tm_w, bar, fc + grp * 64, ks * kBlockK);
+                }
+            }
+            if (*abort_flag && rank == 0) {   // drain: every armed stage either lands or the wait gives up
+                for (int back = 1; back <= kLinStages && it - back >= 0; ++back) {
+                    const int kq = it - back;
+                    ptx::mbar_wait(&full_bar[kq % kLinStages], (kq / kLinStages) & 1, drain_flag);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        if (rank == 0 && ptx::elect_one()) {
+            int it = 0, s = 0;
+            uint32_t ph = 0;
+            bool ok = true;
+            for (int n = 0; n < n_items && ok; ++n) {
+                int row0, f0, nt;
+                unit(n, row0, f0, nt);
+                const uint32_t idesc = ptx::make_idesc_bf16(2 * kTileM, nt, 0, 1);   // A K-major, W MN-major
+                const uint32_t d_tmem = tmem_base + (uint32_t)(n & 1) * 256;
+                // the accumulator about to be overwritten (unit n - 2) must have been read by both epilogues
+                ok = ptx::mbar_wait(&acc_free[n & 1], ((n >> 1) & 1) ^ 1, abort_flag);
+                for (int ks = 0; ks < ks_total && ok; ++ks, ++it, s = (s + 1 == kLinStages) ? 0 : s + 1, ph ^= (s == 0)) {
+                    ok = ptx::mbar_wait(&full_bar[s], ph, abort_flag);
+                    if (!ok) break;
+                    ptx::tc_fence_after_sync();
+                    const uint32_t a_addr = ptx::smem_addr(smem + s * kStageBytes);
+                    const uint32_t b_addr = a_addr + kATileBytes;
+#pragma unroll
+                    for (int k4 = 0; k4 < kBlockK / 16; ++k4) {
+                        const uint64_t a_desc = ptx::make_smem_desc(a_addr + k4 * 32, 16, 1024);
+                        const uint64_t b_desc = ptx::make_smem_desc(b_addr + k4 * 16 * 128, 64 * 128, 1024);
+                        ptx::mma_ss_pair(d_tmem, a_desc, b_desc, idesc, (ks == 0 && k4 == 0) ? 0u : 1u);
+                    }
+                    ptx::tc_commit_pair(&empty_bar[s], 3);
+                    if (ks == ks_total - 1) ptx::tc_commit_pair(&acc_full[n & 1], 3);
+                }
+            }
+        }
+    } else {
+        // epilogue: warp w may touch TMEM lanes [32 (w % 4), 32 (w % 4) + 32); the two warps of a
+        // quarter take one half of the unit's columns each
+        const int quarter = warp & 3;
+        const int half = (warp - 2) >> 2;
+        const int row_in_tile = quarter * 32 + lane;
+        const uint32_t lane_base = ((uint32_t)(quarter * 32) << 16);
+        const uint32_t acc_free_leader[2] = {ptx::map_to_cta(ptx::smem_addr(&acc_free[0]), 0),
+                                             ptx::map_to_cta(ptx::smem_addr(&acc_free[1]), 0)};
+        const int Dq = a.d.n_q * a.d.d_h, Dk = a.d.n_k * a.d.d_h;
+        bool ok = true;
+        for (int n = 0; n < n_items && ok; ++n) {
+            int row0, f0, nt;
+            unit(n, row0, f0, nt);
+            const int cols = nt / 2;                 // this warp's columns: 128 or 64
+            const int c0 = half * cols;
+            const int row = row0 + (int)rank * kTileM + row_in_tile;
+            const bool live = row < a.M;
+            const int b = kProject ? (live ? row / a.d.N : 0) : 0;
+            const int t = kProject ? (live ? row - b * a.d.N : 0) : 0;
+            const uint32_t acc = tmem_base + (uint32_t)(n & 1) * 256 + lane_base + c0;
+            ok = __all_sync(0xffffffffu, ptx::mbar_wait(&acc_full[n & 1], (n >> 1) & 1, abort_flag));
+            if (!ok) break;
+            ptx::tc_fence_after_sync();
+#pragma unroll
+            for (int ch = 0; ch < 4; ++ch) {
+                if (ch * 32 < cols) {
+                    uint32_t v[32];
+                    ptx::tmem_ld32(acc + ch * 32, v);
+                    ptx::tmem_wait_ld();
+                    const int col = f0 + c0 + ch * 32;     // first of these 32 output columns
+                    __nv_bfloat16* dst;
+                    if (!kProject) {
+                        dst = a.c_out + (size_t)(live ? row : 0) * a.n_cols + col;
+                    } else if (col < Dq + Dk) {
+                        // a 32-column chunk lies inside one d_h-vector (d_h is a multiple of 64)
+                        const bool is_q = col < Dq;
+                        const int cc = is_q ? col : col - Dq;
+                        const int g = cc / a.d.d_h, e0 = cc - g * a.d.d_h;
+                        const double pos = (double)(a.pos0 + t);
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) {
+                            double ang = pos * a.theta[(e0 >> 1) + j];
+                            ang -= 6.283185307179586476925287 * rint(ang * 0.159154943091895335768884);
+                            float sn, cs;
+                            sincosf((float)ang, &sn, &cs);
+                            const float x0 = __uint_as_float(v[2 * j]), x1 = __uint_as_float(v[2 * j + 1]);
+                            v[2 * j] = __float_as_uint(x0 * cs - x1 * sn);
+                            v[2 * j + 1] = __float_as_uint(x0 * sn + x1 * cs);
+                        }
+                        dst = is_q ? a.q_out + (((size_t)b * a.d.n_q + g) * a.d.N + t) * a.d.d_h + e0
+                                   : a.k_cache + (((size_t)b * a.d.n_k + g) * a.S_cap + a.pos0 + t) * a.d.d_h + e0;
+                    } else {
+                        const int cc = col - Dq - Dk;
+                        const int g = cc / a.d.d_l, e0 = cc - g * a.d.d_l;
+                        dst = a.c_cache + (((size_t)b * a.d.n_c + g) * a.S_cap + a.pos0 + t) * a.d.d_l + e0;
+                    }
+                    if (live) {
+#pragma unroll
+                        for (int w2 = 0; w2 < 2; ++w2) {      // 2 x 32 bytes: whole sectors
+                            uint32_t ww[8];
+#pragma unroll
+                            for (int e = 0; e < 8; ++e)
+                                ww[e] = pack_bf16x2(__uint_as_float(v[16 * w2 + 2 * e]), __uint_as_float(v[16 * w2 + 2 * e + 1]));
+                            ptx::st_global_256(dst + w2 * 16, ww);
+                        }
+                    }
+                }
+            }
+            ptx::tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive_cluster(acc_free_leader[n & 1]);
+        }
+    }
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    ptx::cluster_arrive();     // neither CTA leaves (or frees TMEM) while the other may still signal it
+    ptx::cluster_wait();
+    if (warp == 1) ptx::tmem_dealloc_pair(tmem_base, 512);
+    if (threadIdx.x == 0 && *abort_flag) raise_status(status_word, GTA_ERR_TIMEOUT);
+}
+
+int lin_sm_count() {
+    static int n = [] {
+        int dev = 0, v = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v <= 0)
+            v = 148;
+        return v;
+    }();
+    return n;
+}
+
+template <bool kProject>
+gta_status_t launch_linear(const LinArgs& a, const void* a_ptr, const void* w_ptr, int32_t* status_word,
+                           cudaStream_t stream) {
+    CUtensorMap tm_a, tm_w;
+    {
+        const uint64_t dims[2] = {(uint64_t)a.K, (uint64_t)a.M};
+        const uint32_t box[2] = {kBlockK, kTileM};
+        if (!make_bf16_map(&tm_a, a_ptr, 2, dims, box)) return GTA_ERR_CUDA;
+    }
+    {
+        const uint64_t dims[2] = {(uint64_t)a.n_cols, (uint64_t)a.K};
+        const uint32_t box[2] = {64, kBlockK};
+        if (!make_bf16_map(&tm_w, w_ptr, 2, dims, box)) return GTA_ERR_CUDA;
+    }
+    auto kern = sm100_linear_kernel<kProject>;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kLinSmemTotal) != cudaSuccess)
+        return GTA_ERR_CUDA;
+    cudaLaunchConfig_t cfg = {};
+    cfg.blockDim = dim3(kLinThreads);
+    cfg.dynamicSmemBytes = kLinSmemTotal;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    // a persistent grid must be resident at once: as many pairs as the device can hold, asked once per device
+    static thread_local int cached_dev = -1, cached_pairs = 0;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return GTA_ERR_CUDA;
+    if (dev != cached_dev) {
+        cfg.gridDim = dim3(2 * (lin_sm_count() / 2));
+        int n = 0;
+        if (cudaOccupancyMaxActiveClusters(&n, kern, &cfg) != cudaSuccess || n < 1) return GTA_ERR_CUDA;
+        cached_dev = dev;
+        cached_pairs = n;
+    }
+    const int G = a.n_units < cached_pairs ? a.n_units : cached_pairs;
+    cfg.gridDim = dim3(2 * G);
+    if (cudaLaunchKernelEx(&cfg, kern, tm_a, tm_w, a, status_word) != cudaSuccess) return GTA_ERR_CUDA;
+    return cudaGetLastError() == cudaSuccess ? GTA_OK : GTA_ERR_CUDA;
+}
+
+bool fill_common(LinArgs& a, long long M, int K, int n_cols) {
+    if (M <= 0 || M > 0x3fffffffLL || K < kBlockK || K % kBlockK != 0 || n_cols < 128 || n_cols % 128 != 0) return false;
+    a.M = (int)M;
+    a.K = K;
+    a.n_cols = n_cols;
+    a.n_cb = (n_cols + 255) / 256;
+    const long long units = ((M + 2 * kTileM - 1) / (2 * kTileM)) * a.n_cb;
+    if (units > 0x3fffffffLL) return false;
+    a.n_units = (int)units;
+    return true;
+}
+
+}  // namespace
+
+bool sm100_linear_supported(const Dims& d, int dtype) {
+    if (dtype != GTA_BF16 || d.H % kBlockK != 0 || d.d_h % 64 != 0 || d.d_h > 2 * kMaxRopePairs || d.d_l % 64 != 0)
+        return false;
+    const int qkc = (d.n_q + d.n_k) * d.d_h + d.n_c * d.d_l;
+    return qkc % 128 == 0 && d.H % 128 == 0 && (d.n_h * d.d_h) % kBlockK == 0;
+}
+
+gta_status_t launch_sm100_project(const Dims& d, int pos0, int S_cap, double rope_base, const void* x,
+                                  const void* w_qkc, void* q_out, void* k_cache, void* c_cache,
+                                  int32_t* status_word, cudaStream_t stream) {
+    LinArgs a = {};
+    if (!fill_common(a, (long long)d.B * d.N, d.H, (d.n_q + d.n_k) * d.d_h + d.n_c * d.d_l)) return GTA_ERR_UNSUPPORTED;
+    a.d = d;
+    a.pos0 = pos0;
+    a.S_cap = S_cap;
+    a.q_out = static_cast<__nv_bfloat16*>(q_out);
+    a.k_cache = static_cast<__nv_bfloat16*>(k_cache);
+    a.c_cache = static_cast<__nv_bfloat16*>(c_cache);
+    for (int i = 0; i < d.d_h / 2; ++i) a.theta[i] = pow(rope_base, -2.0 * i / d.d_h);
+    return launch_linear<true>(a, x, w_qkc, status_word, stream);
+}
+
+gta_status_t launch_sm100_matmul(long long M, int K, int n_cols, const void* a_ptr, const void* w_ptr, void* c_out,
+                                 int32_t* status_word, cudaStream_t stream) {
+    LinArgs a = {};
+    if (!fill_common(a, M, K, n_cols)) return GTA_ERR_UNSUPPORTED;
+    a.c_out = static_cast<__nv_bfloat16*>(c_out);
+    return launch_linear<false>(a, a_ptr, w_ptr, status_word, stream);
+}
+
+}  // namespace gta

@@ -164,3 +164,24 @@ def paginate(t: dict, page_size: int, seed: int = 0, spare_pages: int = 3) -> di
     out.update(k_pool=k_pool, c_pool=c_pool, block_table=table.to(dev).contiguous(), page_size=page_size,
                max_pages=max_pages, n_pages=n_pages)
     return out
+
+
+def layer_inputs(w: Workload, device="cpu"):
+    """Dict of x, w_qkc, w_p, w_g, w_o for the whole attention layer, in the workload dtype on `device`.
+
+    x ~ N(0,1); w_qkc [H, (n_q + n_k) d_h + n_c d_l] ~ N(0, 1/H) (the query, key and latent projections side
+    by side); w_p, w_g as in prefill_inputs; w_o [n_h d_h, H] ~ N(0, 1/(n_h d_h)).
+    """
+    assert w.kind == "prefill"
+    gen = torch.Generator("cpu").manual_seed(w.seed + 17)
+    dt = w.torch_dtype()
+    H, D = w.d_model, w.n_heads * w.d_h
+    out = dict(
+        x=_randn(gen, (w.batch, w.seq, H)),
+        w_qkc=_randn(gen, (H, (w.n_q + w.n_k) * w.d_h + w.n_c * w.d_l), H ** -0.5),
+        w_p=_randn(gen, (w.n_heads, w.d_l, w.d_h), w.d_l ** -0.5),
+        w_g=_randn(gen, (H, D), H ** -0.5),
+        w_o=_randn(gen, (D, H), D ** -0.5),
+    )
+    dev = torch.device(device)
+    return {name: t.to(dev).to(dt).contiguous() for name, t in out.items()}

@@ -1,0 +1,104 @@
+"""GPU parity of the whole attention layer (projections + RoPE + cache write, operator, output projection)
+against the fp64 oracle of App. B.1.1, element by element on identical seeded inputs."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2506_17286_b200 import inputs as I
+from tests.parity_utils import assert_close, oracle_shape
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def B():
+    if not torch.cuda.is_available():
+        pytest.skip("needs a CUDA device")
+    from paper_2506_17286_b200 import build, binding
+    build.build()
+    binding.lib()
+    return binding
+
+
+def _run_layer(B, w, t, chunks, s_cap, rope_base):
+    """The layer chunk by chunk over caches that start out as N(0,1) garbage; returns u, k_cache, c_cache."""
+    g = torch.Generator("cuda").manual_seed(5)
+    k_cache = torch.randn((w.batch, w.n_k, s_cap, w.d_h), generator=g, device="cuda").to(torch.bfloat16)
+    c_cache = torch.randn((w.batch, w.n_c, s_cap, w.d_l), generator=g, device="cuda").to(torch.bfloat16)
+    k0, c0 = k_cache.clone(), c_cache.clone()
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    us, pos0 = [], 0
+    for n in chunks:
+        x = t["x"][:, pos0:pos0 + n].contiguous()
+        shape = B.make_shape(batch=w.batch, seq=n, d_model=w.d_model, n_heads=w.n_heads, n_q=w.n_q, n_k=w.n_k,
+                             n_c=w.n_c, d_h=w.d_h, d_l=w.d_l, dtype=torch.bfloat16)
+        ws = torch.full((B.layer_prefill_workspace_bytes(shape),), 0xFF, dtype=torch.uint8, device="cuda")
+        us.append(B.gta_layer_prefill(x, t["w_qkc"], t["w_p"], t["w_g"], t["w_o"], k_cache, c_cache, pos0=pos0,
+                                      rope_base=rope_base, n_q=w.n_q, workspace=ws, status_word=status))
+        pos0 += n
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    # rows behind the last written position are untouched
+    assert torch.equal(k_cache[:, :, pos0:], k0[:, :, pos0:]) and torch.equal(c_cache[:, :, pos0:], c0[:, :, pos0:])
+    return torch.cat(us, dim=1), k_cache[:, :, :pos0], c_cache[:, :, :pos0]
+
+
+def _layer_case(B, oracle, w, chunks=None, rope_base=10000.0, rows=None):
+    chunks = chunks or [w.seq]
+    assert sum(chunks) == w.seq
+    t = I.layer_inputs(w, device="cuda")
+    u, k, c = _run_layer(B, w, t, chunks, w.seq + 40, rope_base)
+    tc = {n: v.cpu() for n, v in t.items()}
+    want = oracle.layer_prefill(oracle_shape(w), tc["x"], tc["w_qkc"], tc["w_p"], tc["w_g"], tc["w_o"],
+                                rope_base=rope_base)
+    # the caches hold the rounded RoPE'd projections: a value may land on the neighbouring bf16 number where fp32
+    # and fp64 accumulation straddle a rounding boundary, nothing more
+    for name, got, ref in (("k", k, want["k"]), ("c", c, want["c"])):
+        g64 = got.double().cpu().numpy()
+        # one bf16 step of the value, plus the fp32 accumulation error itself where the value is tiny
+        # (a rotation can cancel: x0 cos - x1 sin near zero)
+        step = np.abs(ref) * 2.0 ** -7 + 3e-5
+        assert np.all(np.abs(g64 - ref) <= step), f"{name} cache differs by more than one bf16 step"
+        assert np.mean(g64 != ref) < 2e-2, f"{name} cache: too many rounding flips"
+    sel = slice(None) if rows is None else rows
+    return assert_close(u[:, sel], want["u"][:, sel], torch.bfloat16, w.name)
+
+
+LAYERS = [
+    # name, B, N, H, n_h, n_q, n_k, n_c, d_h, d_l, chunks
+    ("paper_1b_shape_small", 2, 300, 1280, 20, 5, 1, 1, 64, 128, None),
+    ("c2_shape_small", 1, 384, 512, 8, 4, 4, 1, 128, 512, None),
+    ("two_chunks", 2, 320, 256, 8, 4, 2, 2, 64, 128, [192, 128]),
+    ("ragged_chunks_one_token_last", 1, 262, 256, 4, 2, 2, 1, 128, 256, [5, 256, 1]),
+    ("odd_block_tail", 3, 130, 384, 6, 3, 3, 1, 64, 256, None),
+]
+
+
+@pytest.mark.parametrize("case", LAYERS, ids=[c[0] for c in LAYERS])
+def test_layer_prefill_small_shapes(B, oracle, case):
+    name, nb, N, H, n_h, n_q, n_k, n_c, d_h, d_l, chunks = case
+    w = I.Workload(name, "prefill", "bf16", nb, N, H, n_h, n_q, n_k, n_c, d_h, d_l, seed=71)
+    _layer_case(B, oracle, w, chunks=chunks)
+
+
+def test_layer_prefill_other_rope_base_and_late_positions(B, oracle):
+    """A chunk far into the context (positions 3000 ..): the phase of the fast pairs must survive."""
+    w = I.Workload("late", "prefill", "bf16", 1, 3200, 256, 4, 2, 2, 1, 64, 128, seed=72)
+    _layer_case(B, oracle, w, chunks=[3072, 128], rope_base=500000.0, rows=slice(3000, 3200))
+
+
+def test_layer_rejects_what_it_does_not_cover(B):
+    w = I.Workload("bad", "prefill", "bf16", 1, 64, 256, 4, 2, 2, 1, 64, 128, seed=1)
+    t = I.layer_inputs(w, device="cuda")
+    k = torch.zeros((1, 2, 64, 64), dtype=torch.bfloat16, device="cuda")
+    c = torch.zeros((1, 1, 64, 128), dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(B.GtaError) as e:     # chunk does not fit behind pos0
+        B.gta_layer_prefill(t["x"], t["w_qkc"], t["w_p"], t["w_g"], t["w_o"], k, c, pos0=1, n_q=2)
+    assert e.value.status == B.GTA_ERR_INVALID_ARG
+    with pytest.raises(B.GtaError) as e:
+        B.gta_layer_prefill(t["x"], t["w_qkc"], t["w_p"], t["w_g"], t["w_o"], k, c, rope_base=1.0, n_q=2)
+    assert e.value.status == B.GTA_ERR_INVALID_ARG
+    f = {n: v.float() for n, v in t.items()}
+    with pytest.raises(B.GtaError) as e:     # fp32: not on the tensor-core kernels
+        B.gta_layer_prefill(f["x"], f["w_qkc"], f["w_p"], f["w_g"], f["w_o"], k.float(), c.float(), n_q=2)
+    assert e.value.status == B.GTA_ERR_UNSUPPORTED

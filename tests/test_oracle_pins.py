@@ -353,3 +353,92 @@ def test_paged_append_equals_contiguous_append_seen_through_the_block_table(orac
     # pages outside the block table are untouched
     unused = sorted(set(range(kp.shape[0])) - set(table.ravel().tolist()))
     assert np.array_equal(gk[unused], kp[unused]) and np.array_equal(gc[unused], cp[unused])
+
+
+# --------------------------------------------------------------------------- whole layer (App. B.1.1)
+def test_rope_is_a_rotation_that_depends_on_relative_position_only(oracle):
+    d, n = 8, 6
+    q = _rand(n, d); k = _rand(n, d)
+    pos = np.arange(n)
+    rq, rk = oracle.rope(q, pos), oracle.rope(k, pos)
+    assert np.allclose(np.linalg.norm(rq, axis=-1), np.linalg.norm(q, axis=-1), rtol=1e-13)
+    assert np.array_equal(rq[0], q[0])                                   # position 0: the identity
+    # <RoPE(a, m), RoPE(b, n)> is a function of m - n: shift every position by 11
+    rq2, rk2 = oracle.rope(q, pos + 11), oracle.rope(k, pos + 11)
+    assert np.allclose(rq @ rk.T, rq2 @ rk2.T, rtol=0, atol=1e-12)
+    # the complex form of the same definition: (x_{2i} + j x_{2i+1}) e^{j m theta_i}, theta_i = base^(-2i/d)
+    z = (q[:, 0::2] + 1j * q[:, 1::2]) * np.exp(1j * pos[:, None] * 10000.0 ** (-np.arange(0, d, 2) / d)[None, :])
+    assert np.allclose(rq[:, 0::2], z.real, atol=1e-13) and np.allclose(rq[:, 1::2], z.imag, atol=1e-13)
+    # first pair turns by one radian per position; base changes every pair but the first
+    e0 = np.zeros((n, d)); e0[:, 0] = 1.0
+    r = oracle.rope(e0, pos, base=500.0)
+    assert np.allclose(r[:, 0], np.cos(pos)) and np.allclose(r[:, 1], np.sin(pos)) and np.all(r[:, 2:] == 0)
+    e2 = np.zeros((n, d)); e2[:, 2] = 1.0
+    assert np.allclose(oracle.rope(e2, pos, base=500.0)[:, 3], np.sin(pos * 500.0 ** (-2 / d)))
+
+
+def test_round_to_storage_is_round_to_nearest_even_bf16(oracle):
+    F32, BF16 = 0, 1
+    v = np.array([1.0, 1.0 + 2.0 ** -8, 1.0 + 2.0 ** -7, 1.0 + 3 * 2.0 ** -8, -3.0 - 2.0 ** -7, 1e-3, 0.0])
+    got = oracle.round_to_storage(v, BF16)
+    # bf16 keeps 8 significant bits: ties go to the even neighbour
+    want = np.array([1.0, 1.0, 1.0 + 2.0 ** -7, 1.0 + 2.0 ** -6, -3.0, got[5], 0.0])
+    assert np.array_equal(got, want) and abs(got[5] - 1e-3) <= 1e-3 * 2.0 ** -9
+    assert np.array_equal(oracle.round_to_storage(v, F32), v.astype(np.float32).astype(np.float64))
+
+
+def test_layer_reduces_to_rotary_multi_head_attention_times_w_o(oracle):
+    """n_q = n_k = n_c = n_h, W_P = identity (d_l = d_h), W_G = 0: u = 0.5 * MHA(RoPE(xW_Q), RoPE(xW_K), xW_C) W_O,
+    checked against a textbook attention written here (no storage rounding: storage = float64)."""
+    F64 = 2
+    B, N, H, nh, dh = 2, 9, 12, 3, 4
+    s = Shape(B, N, H, nh, nh, nh, nh, dh, dh, 1)
+    x = _rand(B, N, H)
+    w_qkc = _rand(H, 3 * nh * dh, scale=H ** -0.5)
+    w_o = _rand(nh * dh, H, scale=0.3)
+    w_p = np.broadcast_to(np.eye(dh), (nh, dh, dh)).copy()
+    w_g = np.zeros((H, nh * dh))
+    got = oracle.layer_prefill(s, x, w_qkc, w_p, w_g, w_o, rope_base=100.0, storage=F64)
+    pos = np.arange(N)
+    theta = 100.0 ** (-np.arange(0, dh, 2) / dh)
+
+    def rot(v):   # [N, dh], written with the 2x2 rotation matrices
+        out = np.zeros_like(v)
+        for t in range(N):
+            for i in range(dh // 2):
+                c_, s_ = np.cos(pos[t] * theta[i]), np.sin(pos[t] * theta[i])
+                out[t, 2 * i:2 * i + 2] = np.array([[c_, -s_], [s_, c_]]) @ v[t, 2 * i:2 * i + 2]
+        return out
+
+    want = np.zeros((B, N, H))
+    for b in range(B):
+        heads = []
+        for h in range(nh):
+            q = rot(x[b] @ w_qkc[:, h * dh:(h + 1) * dh])
+            k = rot(x[b] @ w_qkc[:, (nh + h) * dh:(nh + h + 1) * dh])
+            v = x[b] @ w_qkc[:, (2 * nh + h) * dh:(2 * nh + h + 1) * dh]
+            sc = q @ k.T / np.sqrt(dh)
+            sc[np.triu_indices(N, 1)] = -np.inf
+            heads.append(0.5 * _softmax_np(sc) @ v)
+        want[b] = np.concatenate(heads, axis=-1) @ w_o
+    assert np.allclose(got["u"], want, rtol=1e-10, atol=1e-12)
+
+
+def test_layer_is_the_operator_between_its_projections(oracle):
+    """General grouping: the layer's u equals W_O applied to the operator oracle run on the layer's own q, k, c
+    (which are the rounded RoPE'd projections), and the stored tensors are representable in bf16."""
+    BF16 = 1
+    s = Shape(2, 7, 16, 4, 2, 1, 1, 4, 8, 1)
+    x = oracle.round_to_storage(_rand(s.batch, s.seq, s.d_model), BF16)
+    w_qkc = oracle.round_to_storage(_rand(s.d_model, 2 * 4 + 4 + 8, scale=0.25), BF16)
+    w_p = _rand(s.n_heads, s.d_l, s.d_h, scale=0.3); w_g = _rand(s.d_model, s.n_heads * s.d_h, scale=0.25)
+    w_o = _rand(s.n_heads * s.d_h, s.d_model, scale=0.25)
+    r = oracle.layer_prefill(s, x, w_qkc, w_p, w_g, w_o)
+    for name in ("q", "k", "c", "o"):
+        assert np.array_equal(oracle.round_to_storage(r[name], BF16), r[name])
+    o = oracle.prefill(s, r["q"], r["k"], r["c"], x, w_p, w_g)
+    assert np.allclose(r["u"], oracle.round_to_storage(o, BF16).reshape(2, 7, -1) @ w_o, rtol=1e-12, atol=1e-14)
+    # c carries no position: token t's latent is x_t W_C whatever t is
+    assert np.array_equal(r["c"][:, 0], oracle.round_to_storage(x @ w_qkc[:, 12:], BF16))
+    # position 0 is not rotated
+    assert np.array_equal(r["k"][:, 0, 0], oracle.round_to_storage(x[:, 0] @ w_qkc[:, 8:12], BF16))
