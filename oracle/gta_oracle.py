@@ -282,14 +282,15 @@ def rope(v, positions, base: float = 10000.0):
 
 
 def layer_prefill(shape: Shape, x, w_qkc, w_p, w_g, w_o, rope_base: float = 10000.0, storage: int = BF16,
-                  n_threads: int = 0):
+                  n_threads: int = 0, rows=None):
     """The attention layer of App. B.1.1 over a prompt (positions 0 .. N-1):
         q_t, k_t = RoPE(x_t W_Q), RoPE(x_t W_K);  c_t = x_t W_C        (W_qkc = [W_Q | W_K | W_C], groups
                                                                          side by side, d_h / d_h / d_l wide)
         o_t = the operator (prefill) on q, k, c, gated by x_t;          u_t = [o_t,1; ...; o_t,n_h] W_O
     Tensors that the layer stores between its steps (q, the K and C caches, the gated heads) are rounded
     to `storage` there; everything else is float64.  Returns dict(u, q, k, c, o) as float64 arrays:
-    u [B, N, H], q [B, n_q, N, d_h], k [B, n_k, N, d_h], c [B, n_c, N, d_l], o [B, N, n_h, d_h]."""
+    u [B, N, H], q [B, n_q, N, d_h], k [B, n_k, N, d_h], c [B, n_c, N, d_l], o [B, N, n_h, d_h].
+    rows = a list of token positions: o and u are computed for those positions only ([B, R, ...])."""
     s = shape
     x64, w_qkc, w_o = _to_f64(x), _to_f64(w_qkc), _to_f64(w_o)
     B, N = s.batch, s.seq
@@ -306,9 +307,9 @@ def layer_prefill(shape: Shape, x, w_qkc, w_p, w_g, w_o, rope_base: float = 1000
     k = round_to_storage(rope(grouped(y[..., Dq:Dq + Dk], s.n_k, s.d_h), pos, rope_base), storage)
     c = round_to_storage(grouped(y[..., Dq + Dk:], s.n_c, s.d_l), storage)
     o = prefill(s, np.ascontiguousarray(q), np.ascontiguousarray(k), np.ascontiguousarray(c), x64,
-                _to_f64(w_p), _to_f64(w_g), n_threads=n_threads)
+                _to_f64(w_p), _to_f64(w_g), rows=rows, n_threads=n_threads)
     o = round_to_storage(o, storage)
-    u = o.reshape(B, N, s.n_heads * s.d_h) @ w_o
+    u = o.reshape(B, o.shape[1], s.n_heads * s.d_h) @ w_o
     return dict(u=u, q=q, k=k, c=c, o=o)
 
 

@@ -60,6 +60,48 @@ def run_prefill_chunk(w, iters, warmup, kv_len):
     return {"whole_call": _median(times), "kv_len": kv_len}
 
 
+def run_layer(w, iters, warmup):
+    """The whole attention layer on the workload's shape (gta_layer_prefill, a prompt: pos0 = 0)."""
+    dev = torch.device("cuda")
+    t = I.layer_inputs(w, device=dev)
+    shape = G.make_shape(batch=w.batch, seq=w.seq, d_model=w.d_model, n_heads=w.n_heads, n_q=w.n_q, n_k=w.n_k,
+                         n_c=w.n_c, d_h=w.d_h, d_l=w.d_l, dtype=w.torch_dtype())
+    ws = torch.zeros(G.layer_prefill_workspace_bytes(shape), dtype=torch.uint8, device=dev)
+    k_cache = torch.zeros((w.batch, w.n_k, w.seq, w.d_h), dtype=w.torch_dtype(), device=dev)
+    c_cache = torch.zeros((w.batch, w.n_c, w.seq, w.d_l), dtype=w.torch_dtype(), device=dev)
+    u = torch.empty((w.batch, w.seq, w.d_model), dtype=w.torch_dtype(), device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    stream = torch.cuda.current_stream()
+
+    def step():
+        G.gta_layer_prefill(t["x"], t["w_qkc"], t["w_p"], t["w_g"], t["w_o"], k_cache, c_cache, n_q=w.n_q, out=u,
+                            workspace=ws, status_word=status)
+
+    for _ in range(warmup):
+        step()
+    torch.cuda.synchronize()
+    times = []
+    for rep in range(3):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(iters):
+            step()
+        e1.record(stream)
+        torch.cuda.synchronize()
+        times.append(e0.elapsed_time(e1) / iters)
+    assert int(status.item()) == 0, "device status word raised"
+    M = w.batch * w.seq
+    qkc = (w.n_q + w.n_k) * w.d_h + w.n_c * w.d_l
+    D = w.n_heads * w.d_h
+    # linear maps in full, attention over the causal half (as the operator's figures count it)
+    flops = dict(project=2.0 * M * w.d_model * qkc, w_o=2.0 * M * D * w.d_model,
+                 attention=w.batch * w.n_q * (w.d_h + w.d_l) * float(w.seq) * (w.seq + 1),
+                 decoder=2.0 * M * w.n_heads * w.d_l * w.d_h, gate=2.0 * M * w.d_model * D)
+    ms = _median(times)
+    return {"whole_call": ms, "launches": G.last_launch_count(), "gflop": {k: v / 1e9 for k, v in flops.items()},
+            "tflops": sum(flops.values()) / (ms * 1e-3) / 1e12}
+
+
 def run_prefill(w, iters, warmup, stages):
     dev = torch.device("cuda")
     t = I.prefill_inputs(w, device=dev)
@@ -208,6 +250,8 @@ def main():
     ap.add_argument("--append", action="store_true", help="decode: run gta_cache_append before every step")
     ap.add_argument("--kv-len", type=int, default=0,
                     help="prefill: treat the workload's tokens as the last chunk of a context of this length")
+    ap.add_argument("--layer", action="store_true",
+                    help="prefill: the whole attention layer (projections + RoPE + cache write, operator, W_O)")
     ap.add_argument("--page-size", type=int, default=0,
                     help="decode: keep the caches in a paged pool with pages of this many tokens")
     args = ap.parse_args()
@@ -218,7 +262,9 @@ def main():
         w = I.scaled(w, seq=args.seq) if w.kind == "prefill" or w.seq > 0 else I.scaled(w, ctx_max=args.seq)
     G.lib()
     torch.cuda.set_device(0)
-    if w.kind == "prefill" and args.kv_len > w.seq:
+    if w.kind == "prefill" and args.layer:
+        res = run_layer(w, args.iters, args.warmup)
+    elif w.kind == "prefill" and args.kv_len > w.seq:
         res = run_prefill_chunk(w, args.iters, args.warmup, args.kv_len)
     elif w.kind == "prefill":
         res = run_prefill(w, args.iters, args.warmup, args.stages & 3)

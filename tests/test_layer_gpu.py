@@ -43,14 +43,14 @@ def _run_layer(B, w, t, chunks, s_cap, rope_base):
     return torch.cat(us, dim=1), k_cache[:, :, :pos0], c_cache[:, :, :pos0]
 
 
-def _layer_case(B, oracle, w, chunks=None, rope_base=10000.0, rows=None):
+def _layer_case(B, oracle, w, chunks=None, rope_base=10000.0, rows=None, sample=None):
     chunks = chunks or [w.seq]
     assert sum(chunks) == w.seq
     t = I.layer_inputs(w, device="cuda")
     u, k, c = _run_layer(B, w, t, chunks, w.seq + 40, rope_base)
     tc = {n: v.cpu() for n, v in t.items()}
     want = oracle.layer_prefill(oracle_shape(w), tc["x"], tc["w_qkc"], tc["w_p"], tc["w_g"], tc["w_o"],
-                                rope_base=rope_base)
+                                rope_base=rope_base, rows=sample)
     # the caches hold the rounded RoPE'd projections: a value may land on the neighbouring bf16 number where fp32
     # and fp64 accumulation straddle a rounding boundary, nothing more
     for name, got, ref in (("k", k, want["k"]), ("c", c, want["c"])):
@@ -60,6 +60,8 @@ def _layer_case(B, oracle, w, chunks=None, rope_base=10000.0, rows=None):
         step = np.abs(ref) * 2.0 ** -7 + 3e-5
         assert np.all(np.abs(g64 - ref) <= step), f"{name} cache differs by more than one bf16 step"
         assert np.mean(g64 != ref) < 2e-2, f"{name} cache: too many rounding flips"
+    if sample is not None:      # the oracle computed these positions only
+        return assert_close(u[:, torch.as_tensor(sample, device="cuda")], want["u"], torch.bfloat16, w.name)
     sel = slice(None) if rows is None else rows
     return assert_close(u[:, sel], want["u"][:, sel], torch.bfloat16, w.name)
 
@@ -85,6 +87,18 @@ def test_layer_prefill_other_rope_base_and_late_positions(B, oracle):
     """A chunk far into the context (positions 3000 ..): the phase of the fast pairs must survive."""
     w = I.Workload("late", "prefill", "bf16", 1, 3200, 256, 4, 2, 2, 1, 64, 128, seed=72)
     _layer_case(B, oracle, w, chunks=[3072, 128], rope_base=500000.0, rows=slice(3000, 3200))
+
+
+def _sample_positions(N, n=24, seed=0):
+    rng = np.random.default_rng(seed)
+    fixed = [0, 1, 127, 128, 255, 256, N // 2, N - 2, N - 1]
+    return sorted(set(fixed) | set(int(v) for v in rng.integers(0, N, n)))
+
+
+@pytest.mark.parametrize("name", ["c2_prefill_bf16", "x1_gta1b_prefill_bf16"])
+def test_layer_prefill_full_size_sampled_positions(B, oracle, name):
+    w = I.CONFIGS[name]
+    _layer_case(B, oracle, w, sample=_sample_positions(w.seq))
 
 
 def test_layer_rejects_what_it_does_not_cover(B):
