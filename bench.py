@@ -395,6 +395,31 @@ def run_ours(args):
     t_decode_paged = d4.elapsed_time(d5) / K_d
     assert int(status.item()) == 0, "device status word raised during the benchmark"
     del psets, ws_pg
+    # ---- the whole attention layer on the prefill workload's shape (projections + RoPE + cache write, the
+    #      operator, the output projection), back to back: context for the operator's figure, not part of `value`
+    tl = I.layer_inputs(wp, device=dev)
+    ws_l = torch.zeros(G.layer_prefill_workspace_bytes(shape_p), dtype=torch.uint8, device=dev)
+    kc_l = torch.zeros((wp.batch, wp.n_k, wp.seq, wp.d_h), dtype=torch.bfloat16, device=dev)
+    cc_l = torch.zeros((wp.batch, wp.n_c, wp.seq, wp.d_l), dtype=torch.bfloat16, device=dev)
+    u_l = torch.empty((wp.batch, wp.seq, wp.d_model), dtype=torch.bfloat16, device=dev)
+
+    def layer_call():
+        G.gta_layer_prefill(tl["x"], tl["w_qkc"], tl["w_p"], tl["w_g"], tl["w_o"], kc_l, cc_l, n_q=wp.n_q, out=u_l,
+                            workspace=ws_l, status_word=status)
+
+    K_l = max(min(K, 200), 20)
+    for i in range(3):
+        layer_call()
+    barrier()
+    l0, l1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    l0.record(stream)
+    for i in range(K_l):
+        layer_call()
+    l1.record(stream)
+    barrier()
+    t_layer = l0.elapsed_time(l1) / K_l
+    assert int(status.item()) == 0, "device status word raised during the benchmark"
+    del tl, ws_l, kc_l, cc_l, u_l
 
     total_ms = e_start.elapsed_time(e_end)
     t_attn = sum(e[0].elapsed_time(e[1]) for e in evk) / K_k
@@ -412,6 +437,7 @@ def run_ours(args):
     t_decode_b2b = max_over_ranks_(t_decode_b2b)
     t_decode_call = max_over_ranks_(t_decode_call)
     t_decode_paged = max_over_ranks_(t_decode_paged)
+    t_layer = max_over_ranks_(t_layer)
 
     fl = prefill_flops(wp)
     by = decode_bytes(wd, [wd.seq] * wd.batch)
@@ -452,6 +478,13 @@ def run_ours(args):
                                              "length vector, prepared before the loop)"}},
     }
     decode["roofline"]["frac"] = decode["roofline"]["achieved"] / decode["roofline"]["peak"]
+    M_l = wp.batch * wp.seq
+    fl_layer = fl["total"] + 2.0 * M_l * wp.d_model * ((wp.n_q + wp.n_k) * wp.d_h + wp.n_c * wp.d_l) \
+        + 2.0 * M_l * wp.n_heads * wp.d_h * wp.d_model
+    layer = {"call": "gta_layer_prefill (X [W_Q|W_K|W_C] + RoPE + cache write, the operator, W_O), back to back",
+             "ms": t_layer, "flops": fl_layer, "tflops": fl_layer / (t_layer * 1e-3) / 1e12,
+             "frac_of_sustained_peak": fl_layer / (t_layer * 1e-3) / 1e12 / peaks["bf16_tflops_sustained"],
+             "frac_of_burst_peak": fl_layer / (t_layer * 1e-3) / 1e12 / peaks["bf16_tflops"]}
     decode["paged"] = {"page_size": page_size, "ms_decode_call": t_decode_paged,
                        "achieved": by["total"] / (t_decode_paged * 1e-3) / 1e9,
                        "frac": by["total"] / (t_decode_paged * 1e-3) / 1e9 / peaks["hbm_gbs"],
@@ -550,7 +583,7 @@ def run_ours(args):
             },
             "prefill": {"ms": t_prefill, "tokens_per_s": world * wp.batch * wp.seq / (t_prefill * 1e-3),
                         "flops": fl},
-            "decode": decode, "roofline": roofline, "e2e": e2e, "cpu_baseline": cpu_baseline,
+            "layer": layer, "decode": decode, "roofline": roofline, "e2e": e2e, "cpu_baseline": cpu_baseline,
             "gpu_launches": n_launches, "clocks": clocks,
         }
         print(json.dumps(line))
