@@ -250,7 +250,7 @@ extern "C" size_t gta_layer_prefill_workspace_bytes(const gta_shape_t* shape) {
     const size_t es = elem_size(shape->dtype);
     const size_t q_bytes = align256((size_t)d.B * d.n_q * d.N * d.d_h * es);
     const size_t o_bytes = align256((size_t)d.B * d.N * d.n_h * d.d_h * es);
-    return q_bytes + o_bytes + gta_prefill_workspace_bytes(shape);
+    return q_bytes + o_bytes + align256(gta::sm100_rope_table_bytes(d)) + gta_prefill_workspace_bytes(shape);
 }
 
 extern "C" gta_status_t gta_layer_prefill(const gta_shape_t* shape, int32_t pos0, int32_t S_cap, float rope_base,
@@ -277,10 +277,11 @@ extern "C" gta_status_t gta_layer_prefill(const gta_shape_t* shape, int32_t pos0
     char* ws = static_cast<char*>(workspace);
     void* q_ws = ws;
     void* o_ws = ws + align256((size_t)d.B * d.n_q * d.N * d.d_h * es);
-    char* op_ws = static_cast<char*>(o_ws) + align256((size_t)d.B * d.N * d.n_h * d.d_h * es);
+    char* rope_ws = static_cast<char*>(o_ws) + align256((size_t)d.B * d.N * d.n_h * d.d_h * es);
+    char* op_ws = rope_ws + align256(gta::sm100_rope_table_bytes(d));
     const size_t op_ws_bytes = workspace_bytes - (size_t)(op_ws - ws);
-    st = gta::launch_sm100_project(d, pos0, S_cap, (double)rope_base, x, w_qkc, q_ws, k_cache, c_cache, status_word,
-                                   stream);
+    st = gta::launch_sm100_project(d, pos0, S_cap, (double)rope_base, x, w_qkc, q_ws, k_cache, c_cache, rope_ws,
+                                   status_word, stream);
     if (st != GTA_OK) return st;
     // the chunk's queries against everything the caches now hold for these sequences
     st = prefill_impl(shape, pos0 + d.N, S_cap, q_ws, k_cache, c_cache, x, w_p, w_g, o_ws, op_ws, op_ws_bytes,
@@ -289,7 +290,7 @@ extern "C" gta_status_t gta_layer_prefill(const gta_shape_t* shape, int32_t pos0
     const int op_launches = g_last_launches;
     st = gta::launch_sm100_matmul((long long)d.B * d.N, d.n_h * d.d_h, d.H, o_ws, w_o, u, status_word, stream);
     if (st != GTA_OK) return st;
-    g_last_launches = op_launches + 2;
+    g_last_launches = op_launches + 3;
     return GTA_OK;
 }
 

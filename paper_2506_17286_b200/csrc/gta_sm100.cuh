@@ -23,8 +23,10 @@ bool sm100_linear_supported(const Dims& d, int dtype);
 
 // [Q | K | C] = X W_qkc for the B x N tokens of a chunk that starts at position pos0: RoPE on q and k,
 // q to q_out [B, n_q, N, d_h], k and c to rows pos0 + t of the caches [B, groups, S_cap, width].
+// rope_table: sm100_rope_table_bytes(d) bytes of scratch (cos / sin of the chunk's positions).
+size_t sm100_rope_table_bytes(const Dims& d);
 gta_status_t launch_sm100_project(const Dims& d, int pos0, int S_cap, double rope_base, const void* x,
-                                  const void* w_qkc, void* q_out, void* k_cache, void* c_cache,
+                                  const void* w_qkc, void* q_out, void* k_cache, void* c_cache, void* rope_table,
                                   int32_t* status_word, cudaStream_t stream);
 
 // C[M, n_cols] = A[M, K] W[K, n_cols], row-major.
