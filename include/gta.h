@@ -233,6 +233,28 @@ GTA_API gta_status_t gta_layer_prefill(const gta_shape_t *shape, int32_t pos0, i
                                        void *cuda_stream);
 
 /*
+ * gta_layer_decode — one decode step of the whole attention layer (App. B.1.1 for the newest token;
+ * cache handling as in App. B.1.3).  For every sequence b, with p = seq_lens[b] the new token's position:
+ *
+ *   [q | k | c] = x_t[b] W_qkc;  q, k <- RoPE(., position p)        (layouts and RoPE as in gta_layer_prefill)
+ *   k_cache[b, :, p, :] = k,  c_cache[b, :, p, :] = c,  seq_lens[b] = p + 1
+ *   o = gta_decode over the p + 1 cached tokens, gated by x_t[b];    u[b] = [o_1; ...; o_{n_h}] W_o
+ *
+ *   x_t [B, H]   u [B, H]   seq_lens device int32 [B] in/out   caches as in gta_decode
+ *   workspace: gta_layer_decode_workspace_bytes(shape, S_cap), 256-byte aligned.
+ * A sequence with seq_lens[b] outside [0, S_cap) is left as it is (no row written, length unchanged),
+ * *status_word is raised to GTA_ERR_CACHE_FULL and its row of u is unspecified.
+ * Shapes as gta_layer_prefill (bf16, tensor-core kernels); the decode itself runs on whichever kernel family
+ * gta_decode picks for the shape.
+ */
+GTA_API size_t gta_layer_decode_workspace_bytes(const gta_shape_t *shape, int32_t S_cap);
+GTA_API gta_status_t gta_layer_decode(const gta_shape_t *shape, int32_t S_cap, float rope_base,
+                                      const void *x_t, const void *w_qkc, const void *w_p,
+                                      const void *w_g, const void *w_o, void *k_cache, void *c_cache,
+                                      int32_t *seq_lens, void *u, void *workspace,
+                                      size_t workspace_bytes, int32_t *status_word, void *cuda_stream);
+
+/*
  * gta_decode_static — gta_decode without a workspace argument (the paper has no counterpart: this
  * is a packaging variant of the same decode step, with the same arguments, results and errors).
  *

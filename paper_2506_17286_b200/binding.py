@@ -25,7 +25,7 @@ EXPORTS = (
     "gta_cache_append", "gta_status_string", "gta_version", "gta_prefill_path", "gta_last_launch_count",
     "gta_prefill_stages", "gta_decode_stages", "gta_decode_static", "gta_prefill_chunk",
     "gta_decode_paged_workspace_bytes", "gta_decode_paged", "gta_cache_append_paged",
-    "gta_layer_prefill_workspace_bytes", "gta_layer_prefill",
+    "gta_layer_prefill_workspace_bytes", "gta_layer_prefill", "gta_layer_decode_workspace_bytes", "gta_layer_decode",
 )
 
 
@@ -87,6 +87,10 @@ def lib():
         L.gta_layer_prefill_workspace_bytes.restype = sz
         L.gta_layer_prefill.argtypes = [sp, i32, i32, ctypes.c_float, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp, vp]
         L.gta_layer_prefill.restype = i32
+        L.gta_layer_decode_workspace_bytes.argtypes = [sp, i32]
+        L.gta_layer_decode_workspace_bytes.restype = sz
+        L.gta_layer_decode.argtypes = [sp, i32, ctypes.c_float, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp, vp]
+        L.gta_layer_decode.restype = i32
         L.gta_status_string.argtypes = [i32]
         L.gta_status_string.restype = ctypes.c_char_p
         L.gta_version.restype = i32
@@ -241,6 +245,39 @@ def gta_layer_prefill(x, w_qkc, w_p, w_g, w_o, k_cache, c_cache, *, pos0=0, rope
                                  _stream(stream))
     if st != GTA_OK:
         raise GtaError(st, "gta_layer_prefill")
+    return out
+
+
+def layer_decode_workspace_bytes(shape: GtaShape, s_cap: int) -> int:
+    return int(lib().gta_layer_decode_workspace_bytes(ctypes.byref(shape), int(s_cap)))
+
+
+def gta_layer_decode(x_t, w_qkc, w_p, w_g, w_o, k_cache, c_cache, seq_lens, *, rope_base=10000.0, n_q,
+                     softmax_scale=0.0, out=None, workspace=None, status_word=None, stream=None):
+    """u[B, H] = one decode step of the whole attention layer: the new token of every sequence is projected,
+    rotated at position seq_lens[b], written to the caches (seq_lens advances), attended and projected by w_o."""
+    _check_tensors(x_t, w_qkc, w_p, w_g, w_o, k_cache, c_cache)
+    if seq_lens.dtype != torch.int32 or seq_lens.device != x_t.device or not seq_lens.is_contiguous():
+        raise ValueError("seq_lens must be a contiguous int32 tensor on the operator's device")
+    B, H = x_t.shape
+    n_h, d_l, d_h = w_p.shape
+    n_k, s_cap, n_c = k_cache.shape[1], k_cache.shape[2], c_cache.shape[1]
+    if k_cache.shape != (B, n_k, s_cap, d_h) or c_cache.shape != (B, n_c, s_cap, d_l) \
+            or w_qkc.shape != (H, (n_q + n_k) * d_h + n_c * d_l) or w_g.shape != (H, n_h * d_h) \
+            or w_o.shape != (n_h * d_h, H) or seq_lens.shape != (B,):
+        raise ValueError("inconsistent layer tensor shapes")
+    shape = make_shape(batch=B, seq=0, d_model=H, n_heads=n_h, n_q=n_q, n_k=n_k, n_c=n_c, d_h=d_h, d_l=d_l,
+                       dtype=_dtype_code(x_t), causal=True, softmax_scale=softmax_scale)
+    if out is None:
+        out = torch.empty((B, H), dtype=x_t.dtype, device=x_t.device)
+    if workspace is None:
+        workspace = _workspace(layer_decode_workspace_bytes(shape, s_cap), x_t.device)
+    st = lib().gta_layer_decode(ctypes.byref(shape), int(s_cap), float(rope_base), _ptr(x_t), _ptr(w_qkc), _ptr(w_p),
+                                _ptr(w_g), _ptr(w_o), _ptr(k_cache), _ptr(c_cache), _ptr(seq_lens), _ptr(out),
+                                _ptr(workspace), workspace.numel() * workspace.element_size(), _ptr(status_word),
+                                _stream(stream))
+    if st != GTA_OK:
+        raise GtaError(st, "gta_layer_decode")
     return out
 
 

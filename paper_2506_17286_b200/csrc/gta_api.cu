@@ -294,6 +294,55 @@ extern "C" gta_status_t gta_layer_prefill(const gta_shape_t* shape, int32_t pos0
     return GTA_OK;
 }
 
+extern "C" size_t gta_layer_decode_workspace_bytes(const gta_shape_t* shape, int32_t S_cap) {
+    gta::Dims d;
+    if (check_shape(shape, false, &d) != GTA_OK || S_cap < 0) return 0;
+    const size_t es = elem_size(shape->dtype);
+    return align256((size_t)d.B * d.n_q * d.d_h * es) + align256((size_t)d.B * d.n_h * d.d_h * es) +
+           align256(gta::sm100_decode_prep_bytes(d)) + gta::decode_workspace_bytes(d, shape->dtype, S_cap);
+}
+
+extern "C" gta_status_t gta_layer_decode(const gta_shape_t* shape, int32_t S_cap, float rope_base, const void* x_t,
+                                         const void* w_qkc, const void* w_p, const void* w_g, const void* w_o,
+                                         void* k_cache, void* c_cache, int32_t* seq_lens, void* u, void* workspace,
+                                         size_t workspace_bytes, int32_t* status_word, void* cuda_stream) {
+    g_last_launches = 0;
+    gta::Dims d;
+    gta_status_t st = check_shape(shape, false, &d);
+    if (st != GTA_OK) return st;
+    if (S_cap <= 0 || !(rope_base > 1.0f)) return GTA_ERR_INVALID_ARG;
+    if (!x_t || !w_qkc || !w_p || !w_g || !w_o || !k_cache || !c_cache || !seq_lens || !u) return GTA_ERR_INVALID_ARG;
+    if (!aligned(x_t, 16) || !aligned(w_qkc, 16) || !aligned(w_p, 16) || !aligned(w_g, 16) || !aligned(w_o, 16) ||
+        !aligned(k_cache, 16) || !aligned(c_cache, 16) || !aligned(u, 16) || !aligned(seq_lens, 4) ||
+        !aligned(status_word, 4))
+        return GTA_ERR_INVALID_ARG;
+    if (!gta::sm100_linear_supported(d, shape->dtype) || (size_t)d.d_l * elem_size(shape->dtype) > 4096)
+        return GTA_ERR_UNSUPPORTED;
+    if (d.B == 0) return GTA_OK;
+    if (!workspace || !aligned(workspace, 256) || workspace_bytes < gta_layer_decode_workspace_bytes(shape, S_cap))
+        return GTA_ERR_WORKSPACE;
+    if ((st = check_device()) != GTA_OK) return st;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const size_t es = elem_size(shape->dtype);
+    char* ws = static_cast<char*>(workspace);
+    char* q_ws = ws;
+    char* o_ws = q_ws + align256((size_t)d.B * d.n_q * d.d_h * es);
+    char* prep_ws = o_ws + align256((size_t)d.B * d.n_h * d.d_h * es);
+    char* op_ws = prep_ws + align256(gta::sm100_decode_prep_bytes(d));
+    const size_t op_ws_bytes = workspace_bytes - (size_t)(op_ws - ws);
+    st = gta::launch_sm100_project_step(d, S_cap, (double)rope_base, x_t, w_qkc, q_ws, k_cache, c_cache, seq_lens,
+                                        prep_ws, status_word, stream);
+    if (st != GTA_OK) return st;
+    st = decode_impl(shape, q_ws, k_cache, c_cache, seq_lens, S_cap, x_t, w_p, w_g, o_ws, op_ws, op_ws_bytes,
+                     status_word, cuda_stream, 7, gta::PageMap());
+    if (st != GTA_OK) return st;
+    const int op_launches = g_last_launches;
+    st = gta::launch_sm100_matmul(d.B, d.n_h * d.d_h, d.H, o_ws, w_o, u, status_word, stream);
+    if (st != GTA_OK) return st;
+    g_last_launches = op_launches + 3;
+    return GTA_OK;
+}
+
 static gta_status_t decode_impl(const gta_shape_t* shape, const void* q, const void* k_cache, const void* c_cache,
                                 const int32_t* seq_lens, int32_t S_cap, const void* x_t, const void* w_p,
                                 const void* w_g, void* out, void* workspace, size_t workspace_bytes,

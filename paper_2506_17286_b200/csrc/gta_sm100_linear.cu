@@ -46,7 +46,8 @@ constexpr int kMaxRopePairs = 64;  // d_h <= 128
 
 struct LinArgs {
     int M, K, n_cols;        // C[M, n_cols] = A[M, K] W[K, n_cols]
-    int n_cb;                // column blocks (256 wide, the last one possibly 128)
+    int block;               // columns per block: 256, or 128 when there is a single row tile
+    int n_cb;                // column blocks (the last one possibly 128 wide)
     int n_units;             // row tiles (256 rows) x column blocks
     // plain epilogue
     __nv_bfloat16* c_out;    // [M, n_cols]
@@ -57,6 +58,9 @@ struct LinArgs {
     __nv_bfloat16* k_cache;  // [B, n_k, S_cap, d_h]
     __nv_bfloat16* c_cache;  // [B, n_c, S_cap, d_l]
     const float2* rope;      // [N, d_h / 2] (cos, sin) of position pos0 + t, pair i
+    // one new token per sequence (N = 1): its position, or -1 for a sequence whose cache is full (nothing is
+    // written for it); the table then has one row per sequence
+    const int32_t* pos_seq;
 };
 
 struct RopeArgs {
@@ -80,6 +84,30 @@ rope_table_kernel(const __grid_constant__ RopeArgs r, float2* __restrict__ table
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<uint32_t*>(&v);
+}
+
+// One decode step's bookkeeping, one CTA per sequence: the new token's position is the current length; the
+// (cos, sin) row of that position; then the length advances.  A full cache leaves the length alone,
+// raises the status word and marks the sequence with position -1.
+__global__ void __launch_bounds__(kMaxRopePairs)
+rope_decode_prep_kernel(const __grid_constant__ RopeArgs r, int S_cap, int32_t* __restrict__ seq_lens,
+                        int32_t* __restrict__ pos_out, float2* __restrict__ table, int32_t* status_word) {
+    const int b = blockIdx.x, i = threadIdx.x;
+    const int len = seq_lens[b];
+    __syncthreads();   // every thread has read the old length before thread 0 rewrites it
+    const bool ok = len >= 0 && len < S_cap;
+    if (i < r.n_pairs) {
+        double ang = (double)(ok ? len : 0) * r.theta[i];
+        ang -= 6.283185307179586476925287 * rint(ang * 0.159154943091895335768884);
+        float sn, cs;
+        sincosf((float)ang, &sn, &cs);
+        table[(size_t)b * r.n_pairs + i] = make_float2(cs, sn);
+    }
+    if (i == 0) {
+        pos_out[b] = ok ? len : -1;
+        if (ok) seq_lens[b] = len + 1;
+        else raise_status(status_word, GTA_ERR_CACHE_FULL);
+    }
 }
 
 // kProject: the epilogue of the input projections (RoPE + scatter); otherwise a plain row-major store
@@ -123,8 +151,8 @@ sm100_linear_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
         const int u = pr + n * G;
         const int cb = u % a.n_cb;
         row0 = (u / a.n_cb) * 2 * kTileM;
-        f0 = cb * 256;
-        nt = a.n_cols - f0 < 256 ? a.n_cols - f0 : 256;
+        f0 = cb * a.block;
+        nt = a.n_cols - f0 < a.block ? a.n_cols - f0 : a.block;
     };
 
     if (warp == 0) {
@@ -209,9 +237,16 @@ sm100_linear_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
             const int cols = nt / 2;                 // this warp's columns: 128 or 64
             const int c0 = half * cols;
             const int row = row0 + (int)rank * kTileM + row_in_tile;
-            const bool live = row < a.M;
+            bool live = row < a.M;
             const int b = kProject ? (live ? row / a.d.N : 0) : 0;
             const int t = kProject ? (live ? row - b * a.d.N : 0) : 0;
+            int pos = a.pos0 + t, rope_row = t;
+            if (kProject && a.pos_seq != nullptr) {
+                pos = a.pos_seq[b];
+                rope_row = b;
+                live = live && pos >= 0;
+                if (pos < 0) pos = 0;
+            }
             const uint32_t acc = tmem_base + (uint32_t)(n & 1) * 256 + lane_base + c0;
             ok = __all_sync(0xffffffffu, ptx::mbar_wait(&acc_full[n & 1], (n >> 1) & 1, abort_flag));
             if (!ok) break;
@@ -231,7 +266,7 @@ sm100_linear_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
                         const bool is_q = col < Dq;
                         const int cc = is_q ? col : col - Dq;
                         const int g = cc / a.d.d_h, e0 = cc - g * a.d.d_h;
-                        const float4* rt = reinterpret_cast<const float4*>(a.rope + ((size_t)t * (a.d.d_h >> 1) + (e0 >> 1)));
+                        const float4* rt = reinterpret_cast<const float4*>(a.rope + ((size_t)rope_row * (a.d.d_h >> 1) + (e0 >> 1)));
 #pragma unroll
                         for (int j2 = 0; j2 < 8; ++j2) {      // two pairs per 16-byte load
                             const float4 r4 = __ldg(rt + j2);
@@ -243,11 +278,11 @@ sm100_linear_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
                             v[4 * j2 + 3] = __float_as_uint(x2 * r4.w + x3 * r4.z);
                         }
                         dst = is_q ? a.q_out + (((size_t)b * a.d.n_q + g) * a.d.N + t) * a.d.d_h + e0
-                                   : a.k_cache + (((size_t)b * a.d.n_k + g) * a.S_cap + a.pos0 + t) * a.d.d_h + e0;
+                                   : a.k_cache + (((size_t)b * a.d.n_k + g) * a.S_cap + pos) * a.d.d_h + e0;
                     } else {
                         const int cc = col - Dq - Dk;
                         const int g = cc / a.d.d_l, e0 = cc - g * a.d.d_l;
-                        dst = a.c_cache + (((size_t)b * a.d.n_c + g) * a.S_cap + a.pos0 + t) * a.d.d_l + e0;
+                        dst = a.c_cache + (((size_t)b * a.d.n_c + g) * a.S_cap + pos) * a.d.d_l + e0;
                     }
                     if (live) {
 #pragma unroll
@@ -335,7 +370,8 @@ bool fill_common(LinArgs& a, long long M, int K, int n_cols) {
     a.M = (int)M;
     a.K = K;
     a.n_cols = n_cols;
-    a.n_cb = (n_cols + 255) / 256;
+    a.block = M <= 2 * kTileM ? 128 : 256;      // a single row tile: narrower blocks keep twice as many SMs busy
+    a.n_cb = (n_cols + a.block - 1) / a.block;
     const long long units = ((M + 2 * kTileM - 1) / (2 * kTileM)) * a.n_cb;
     if (units > 0x3fffffffLL) return false;
     a.n_units = (int)units;
@@ -373,6 +409,35 @@ gta_status_t launch_sm100_project(const Dims& d, int pos0, int S_cap, double rop
     rope_table_kernel<<<(d.N * r.n_pairs + 255) / 256, 256, 0, stream>>>(r, static_cast<float2*>(rope_table));
     if (cudaGetLastError() != cudaSuccess) return GTA_ERR_CUDA;
     return launch_linear<true>(a, x, w_qkc, status_word, stream);
+}
+
+size_t sm100_decode_prep_bytes(const Dims& d) {
+    return (((size_t)d.B * (d.d_h / 2) * sizeof(float2) + 255) & ~(size_t)255) + (size_t)d.B * sizeof(int32_t);
+}
+
+gta_status_t launch_sm100_project_step(const Dims& d, int S_cap, double rope_base, const void* x_t, const void* w_qkc,
+                                       void* q_out, void* k_cache, void* c_cache, int32_t* seq_lens, void* prep,
+                                       int32_t* status_word, cudaStream_t stream) {
+    LinArgs a = {};
+    Dims d1 = d;
+    d1.N = 1;
+    if (!fill_common(a, d.B, d.H, (d.n_q + d.n_k) * d.d_h + d.n_c * d.d_l)) return GTA_ERR_UNSUPPORTED;
+    a.d = d1;
+    a.S_cap = S_cap;
+    a.q_out = static_cast<__nv_bfloat16*>(q_out);
+    a.k_cache = static_cast<__nv_bfloat16*>(k_cache);
+    a.c_cache = static_cast<__nv_bfloat16*>(c_cache);
+    float2* table = static_cast<float2*>(prep);
+    int32_t* pos = reinterpret_cast<int32_t*>(static_cast<char*>(prep) +
+                                              (((size_t)d.B * (d.d_h / 2) * sizeof(float2) + 255) & ~(size_t)255));
+    a.rope = table;
+    a.pos_seq = pos;
+    RopeArgs r = {};
+    r.n_pairs = d.d_h / 2;
+    for (int i = 0; i < r.n_pairs; ++i) r.theta[i] = pow(rope_base, -2.0 * i / d.d_h);
+    rope_decode_prep_kernel<<<d.B, kMaxRopePairs, 0, stream>>>(r, S_cap, seq_lens, pos, table, status_word);
+    if (cudaGetLastError() != cudaSuccess) return GTA_ERR_CUDA;
+    return launch_linear<true>(a, x_t, w_qkc, status_word, stream);
 }
 
 gta_status_t launch_sm100_matmul(long long M, int K, int n_cols, const void* a_ptr, const void* w_ptr, void* c_out,

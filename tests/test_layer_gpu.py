@@ -101,6 +101,73 @@ def test_layer_prefill_full_size_sampled_positions(B, oracle, name):
     _layer_case(B, oracle, w, sample=_sample_positions(w.seq))
 
 
+LAYER_STEPS = [
+    # name, H, n_h, n_q, n_k, n_c, d_h, d_l, lens (tokens already cached per sequence)
+    ("c3_shape_small", 512, 8, 4, 4, 1, 128, 512, [1, 63, 64, 200, 0]),
+    ("paper_1b_shape", 1280, 20, 5, 1, 1, 64, 128, [130, 7]),
+    ("two_latents_batch_20", 256, 8, 4, 2, 2, 64, 128, [(37 * i) % 150 for i in range(20)]),
+]
+
+
+@pytest.mark.parametrize("case", LAYER_STEPS, ids=[c[0] for c in LAYER_STEPS])
+def test_layer_decode_step_equals_the_next_row_of_the_layer(B, oracle, case):
+    """Caches filled by gta_layer_prefill (one call per sequence, ragged lengths), then one gta_layer_decode step:
+    its output is row len_b of the layer oracle over len_b + 1 tokens, its cache rows the oracle's k / c there."""
+    name, H, n_h, n_q, n_k, n_c, d_h, d_l, lens = case
+    nb, cap = len(lens), max(lens) + 9
+    w = I.Workload(name, "prefill", "bf16", nb, max(lens) + 1, H, n_h, n_q, n_k, n_c, d_h, d_l, seed=73)
+    t = I.layer_inputs(w, device="cuda")          # x: the history of every sequence, the new token at row len_b
+    g = torch.Generator("cuda").manual_seed(6)
+    k_cache = torch.randn((nb, n_k, cap, d_h), generator=g, device="cuda").to(torch.bfloat16)
+    c_cache = torch.randn((nb, n_c, cap, d_l), generator=g, device="cuda").to(torch.bfloat16)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    for b, n in enumerate(lens):
+        if n > 0:
+            B.gta_layer_prefill(t["x"][b:b + 1, :n].contiguous(), t["w_qkc"], t["w_p"], t["w_g"], t["w_o"],
+                                k_cache[b:b + 1], c_cache[b:b + 1], n_q=n_q, status_word=status)
+    k0, c0 = k_cache.clone(), c_cache.clone()
+    seq_lens = torch.tensor(lens, dtype=torch.int32, device="cuda")
+    idx = torch.arange(nb, device="cuda")
+    x_t = t["x"][idx, seq_lens.long()].contiguous()
+    shape = B.make_shape(batch=nb, seq=0, d_model=H, n_heads=n_h, n_q=n_q, n_k=n_k, n_c=n_c, d_h=d_h, d_l=d_l,
+                         dtype=torch.bfloat16)
+    ws = torch.full((B.layer_decode_workspace_bytes(shape, cap),), 0xFF, dtype=torch.uint8, device="cuda")
+    u = B.gta_layer_decode(x_t, t["w_qkc"], t["w_p"], t["w_g"], t["w_o"], k_cache, c_cache, seq_lens, n_q=n_q,
+                           workspace=ws, status_word=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    assert seq_lens.tolist() == [n + 1 for n in lens]
+    tc = {n: v.cpu() for n, v in t.items()}
+    want_u = np.zeros((nb, H))
+    for b, n in enumerate(lens):
+        ws_b = I.scaled(w, batch=1, seq=n + 1)
+        r = oracle.layer_prefill(oracle_shape(ws_b), tc["x"][b:b + 1, :n + 1], tc["w_qkc"], tc["w_p"], tc["w_g"],
+                                 tc["w_o"], rows=[n])
+        want_u[b] = r["u"][0, 0]
+        for got, ref in ((k_cache[b, :, n], r["k"][0, :, n]), (c_cache[b, :, n], r["c"][0, :, n])):
+            assert np.all(np.abs(got.double().cpu().numpy() - ref) <= np.abs(ref) * 2.0 ** -7 + 3e-5)
+        # nothing but row n of this sequence's caches changed
+        keep = torch.ones(cap, dtype=torch.bool, device="cuda")
+        keep[n] = False
+        assert torch.equal(k_cache[b][:, keep], k0[b][:, keep]) and torch.equal(c_cache[b][:, keep], c0[b][:, keep])
+    assert_close(u, want_u, torch.bfloat16, name)
+
+
+def test_layer_decode_full_cache_is_skipped_and_reported(B):
+    w = I.Workload("full", "prefill", "bf16", 2, 8, 256, 4, 2, 2, 1, 64, 128, seed=2)
+    t = I.layer_inputs(w, device="cuda")
+    k = torch.zeros((2, 2, 8, 64), dtype=torch.bfloat16, device="cuda")
+    c = torch.zeros((2, 1, 8, 128), dtype=torch.bfloat16, device="cuda")
+    lens = torch.tensor([8, 3], dtype=torch.int32, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    B.gta_layer_decode(t["x"][:, 0].contiguous(), t["w_qkc"], t["w_p"], t["w_g"], t["w_o"], k, c, lens, n_q=2,
+                       status_word=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == B.GTA_ERR_CACHE_FULL
+    assert lens.tolist() == [8, 4]
+    assert not k[0].any() and not c[0].any() and k[1, :, 3].any() and not k[1, :, 4:].any()
+
+
 def test_layer_rejects_what_it_does_not_cover(B):
     w = I.Workload("bad", "prefill", "bf16", 1, 64, 256, 4, 2, 2, 1, 64, 128, seed=1)
     t = I.layer_inputs(w, device="cuda")
