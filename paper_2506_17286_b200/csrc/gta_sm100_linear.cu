@@ -43,10 +43,18 @@ constexpr uint32_t kStageBytes = kATileBytes + 2 * kBGroupBytes;   // 32 KB per 
 constexpr uint32_t kBarOffset = kLinStages * kStageBytes;
 constexpr uint32_t kLinSmemTotal = kBarOffset + 512 + 1024;        // barriers + alignment slack
 constexpr int kMaxRopePairs = 64;  // d_h <= 128
+// Without CTA pairs (at most 128 rows in all: a decode step): the A tile holds only the rows that exist,
+// rounded up to the 8-row swizzle atom, which leaves room for a much deeper ring -- with one unit per CTA
+// and few CTAs the bytes in flight per SM pace the kernel.  The MMA still reads 128 rows: the rows past the
+// tile are whatever follows in shared memory, and only feed accumulator rows that are never stored.
+constexpr int kMaxStages = 16;
+constexpr uint32_t kSoloRingBytes = 200 * 1024;
 
 struct LinArgs {
     int M, K, n_cols;        // C[M, n_cols] = A[M, K] W[K, n_cols]
-    int block;               // columns per block: 256, or 128 when there is a single row tile
+    int block;               // columns per block: 256, 128 when there is a single 256-row tile, 64 without CTA pairs
+    int n_stages;            // ring depth
+    uint32_t a_bytes;        // bytes of an A tile in the ring
     int n_cb;                // column blocks (the last one possibly 128 wide)
     int n_units;             // row tiles (256 rows) x column blocks
     // plain epilogue
@@ -111,46 +119,66 @@ rope_decode_prep_kernel(const __grid_constant__ RopeArgs r, int S_cap, int32_t* 
 }
 
 // kProject: the epilogue of the input projections (RoPE + scatter); otherwise a plain row-major store
-template <bool kProject>
+// kPair: CTA pairs (cta_group::2, M = 256); otherwise single CTAs (cta_group::1, M = 128) on 64-column units
+template <bool kProject, bool kPair>
 __global__ void __launch_bounds__(kLinThreads, 1)
 sm100_linear_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_w,
                     const __grid_constant__ LinArgs a, int32_t* status_word) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-    uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + kBarOffset);    // used in the leader CTA
-    uint64_t* empty_bar = full_bar + kLinStages;                             // both CTAs
-    uint64_t* acc_full = empty_bar + kLinStages;                             // [2] both CTAs
+    // ring: pairs keep {A, W} of a stage side by side; without pairs all A tiles come first, then all W tiles
+    const int n_stages = kPair ? kLinStages : a.n_stages;
+    const uint32_t a_stride = kPair ? kStageBytes : a.a_bytes;
+    const uint32_t b_base = kPair ? kATileBytes : (uint32_t)n_stages * a.a_bytes;
+    const uint32_t b_stride = kPair ? kStageBytes : kBGroupBytes;
+    const uint32_t a_tile_bytes = kPair ? kATileBytes : a.a_bytes;
+    const uint32_t bar_off = kPair ? kBarOffset : (uint32_t)n_stages * (a.a_bytes + kBGroupBytes);
+    uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + bar_off);       // used in the leader CTA
+    uint64_t* empty_bar = full_bar + kMaxStages;                             // both CTAs
+    uint64_t* acc_full = empty_bar + kMaxStages;                             // [2] both CTAs
     uint64_t* acc_free = acc_full + 2;                                       // [2] leader CTA: 16 warps arrive
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_free + 2);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
     volatile int* drain_flag = abort_flag + 1;   // never raised: lets the drain wait run to its limit
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const uint32_t rank = ptx::cluster_ctarank();                       // 0 = leader
-    const int G = gridDim.x >> 1, pr = blockIdx.x >> 1;
+    const uint32_t rank = kPair ? ptx::cluster_ctarank() : 0u;          // 0 = leader
+    const int G = kPair ? gridDim.x >> 1 : gridDim.x;                   // CTA pairs (or CTAs)
+    const int pr = kPair ? blockIdx.x >> 1 : blockIdx.x;
+    constexpr int kUnitRows = kPair ? 2 * kTileM : kTileM;
     const int n_items = pr < a.n_units ? (a.n_units - pr + G - 1) / G : 0;
     const int ks_total = a.K / kBlockK;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < kLinStages; ++s) { ptx::mbar_init(&full_bar[s], 2); ptx::mbar_init(&empty_bar[s], 1); }
-        for (int j = 0; j < 2; ++j) { ptx::mbar_init(&acc_full[j], 1); ptx::mbar_init(&acc_free[j], 16); }
+        for (int s = 0; s < n_stages; ++s) { ptx::mbar_init(&full_bar[s], kPair ? 2 : 1); ptx::mbar_init(&empty_bar[s], 1); }
+        for (int j = 0; j < 2; ++j) { ptx::mbar_init(&acc_full[j], 1); ptx::mbar_init(&acc_free[j], kPair ? 16 : 8); }
         *abort_flag = 0;
         *drain_flag = 0;
         ptx::fence_mbar_init();
     }
-    if (warp == 1) ptx::tmem_alloc_pair(tmem_slot, 512);
+    if (warp == 1) {
+        if (kPair) ptx::tmem_alloc_pair(tmem_slot, 512);
+        else ptx::tmem_alloc(tmem_slot, 512);
+    }
     ptx::tc_fence_before_sync();
     __syncthreads();
-    ptx::cluster_arrive();     // the peer's barriers exist before anything is signalled to them
-    ptx::cluster_wait();
+    if (kPair) {
+        ptx::cluster_arrive();     // the peer's barriers exist before anything is signalled to them
+        ptx::cluster_wait();
+    }
     ptx::tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
+    // Launched with programmatic stream serialisation: the set-up above may have run while the kernel ahead
+    // in the stream was draining.  Nothing of global memory is touched before that kernel is complete, and
+    // only then may the kernel behind this one be scheduled.
+    ptx::grid_dependency_wait();
+    ptx::grid_launch_dependents();
 
     // unit n of this pair: column block cb (consecutive pairs share a row tile), first row, first column, width
     auto unit = [&](int n, int& row0, int& f0, int& nt) {
         const int u = pr + n * G;
         const int cb = u % a.n_cb;
-        row0 = (u / a.n_cb) * 2 * kTileM;
+        row0 = (u / a.n_cb) * kUnitRows;
         f0 = cb * a.block;
         nt = a.n_cols - f0 < a.block ? a.n_cols - f0 : a.block;
     };
@@ -159,8 +187,6 @@ sm100_linear_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
         if (ptx::elect_one()) {
             ptx::prefetch_tensormap(&tm_a);
             ptx::prefetch_tensormap(&tm_w);
-            // A may be the result of the kernel before this one in the stream
-            ptx::grid_dependency_wait();
             int it = 0, s = 0;
             uint32_t ph = 0;
             bool ok = true;
@@ -168,15 +194,21 @@ sm100_linear_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
                 int row0, f0, nt;
                 unit(n, row0, f0, nt);
                 const int r0 = row0 + (int)rank * kTileM;          // this CTA's rows
-                const int n_grp = nt / 128;                         // 64-column groups this CTA stages
-                const int fc = f0 + (int)rank * (nt / 2);           // this CTA's first weight column
-                const uint32_t tx = kATileBytes + (uint32_t)n_grp * kBGroupBytes;
-                const uint32_t bar_base = ptx::map_to_cta(ptx::smem_addr(&full_bar[0]), 0);   // the leader's
-                for (int ks = 0; ks < ks_total; ++ks, ++it, s = (s + 1 == kLinStages) ? 0 : s + 1, ph ^= (s == 0)) {
+                const int n_grp = kPair ? nt / 128 : 1;             // 64-column groups this CTA stages
+                const int fc = kPair ? f0 + (int)rank * (nt / 2) : f0;   // this CTA's first weight column
+                const uint32_t tx = a_tile_bytes + (uint32_t)n_grp * kBGroupBytes;
+                const uint32_t bar_base = kPair ? ptx::map_to_cta(ptx::smem_addr(&full_bar[0]), 0) : 0u;   // the leader's
+                for (int ks = 0; ks < ks_total; ++ks, ++it, s = (s + 1 == n_stages) ? 0 : s + 1, ph ^= (s == 0)) {
                     ok = ptx::mbar_wait(&empty_bar[s], ph ^ 1, abort_flag);
                     if (!ok) break;
-                    uint8_t* a_s = smem + s * kStageBytes;
-                    uint8_t* b_s = a_s + kATileBytes;
+                    uint8_t* a_s = smem + s * a_stride;
+                    uint8_t* b_s = smem + b_base + s * b_stride;
+                    if (!kPair) {
+                        ptx::mbar_arrive_expect_tx(&full_bar[s], tx);
+                        ptx::tma_load_2d(a_s, &tm_a, &full_bar[s], ks * kBlockK, r0);
+                        ptx::tma_load_2d(b_s, &tm_w, &full_bar[s], fc, ks * kBlockK);
+                        continue;
+                    }
                     const uint32_t bar = bar_base + (uint32_t)s * 8;
                     ptx::mbar_arrive_expect_tx_cluster(bar, tx);
                     ptx::tma_load_2d_pair(a_s, &tm_a, bar, ks * kBlockK, r0);
@@ -185,9 +217,9 @@ sm100_linear_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
                 }
             }
             if (*abort_flag && rank == 0) {   // drain: every armed stage either lands or the wait gives up
-                for (int back = 1; back <= kLinStages && it - back >= 0; ++back) {
+                for (int back = 1; back <= n_stages && it - back >= 0; ++back) {
                     const int kq = it - back;
-                    ptx::mbar_wait(&full_bar[kq % kLinStages], (kq / kLinStages) & 1, drain_flag);
+                    ptx::mbar_wait(&full_bar[kq % n_stages], (kq / n_stages) & 1, drain_flag);
                 }
             }
         }
@@ -199,24 +231,30 @@ sm100_linear_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
             for (int n = 0; n < n_items && ok; ++n) {
                 int row0, f0, nt;
                 unit(n, row0, f0, nt);
-                const uint32_t idesc = ptx::make_idesc_bf16(2 * kTileM, nt, 0, 1);   // A K-major, W MN-major
+                const uint32_t idesc = ptx::make_idesc_bf16(kUnitRows, nt, 0, 1);   // A K-major, W MN-major
                 const uint32_t d_tmem = tmem_base + (uint32_t)(n & 1) * 256;
                 // the accumulator about to be overwritten (unit n - 2) must have been read by both epilogues
                 ok = ptx::mbar_wait(&acc_free[n & 1], ((n >> 1) & 1) ^ 1, abort_flag);
-                for (int ks = 0; ks < ks_total && ok; ++ks, ++it, s = (s + 1 == kLinStages) ? 0 : s + 1, ph ^= (s == 0)) {
+                for (int ks = 0; ks < ks_total && ok; ++ks, ++it, s = (s + 1 == n_stages) ? 0 : s + 1, ph ^= (s == 0)) {
                     ok = ptx::mbar_wait(&full_bar[s], ph, abort_flag);
                     if (!ok) break;
                     ptx::tc_fence_after_sync();
-                    const uint32_t a_addr = ptx::smem_addr(smem + s * kStageBytes);
-                    const uint32_t b_addr = a_addr + kATileBytes;
+                    const uint32_t a_addr = ptx::smem_addr(smem + s * a_stride);
+                    const uint32_t b_addr = ptx::smem_addr(smem + b_base + s * b_stride);
 #pragma unroll
                     for (int k4 = 0; k4 < kBlockK / 16; ++k4) {
                         const uint64_t a_desc = ptx::make_smem_desc(a_addr + k4 * 32, 16, 1024);
                         const uint64_t b_desc = ptx::make_smem_desc(b_addr + k4 * 16 * 128, 64 * 128, 1024);
-                        ptx::mma_ss_pair(d_tmem, a_desc, b_desc, idesc, (ks == 0 && k4 == 0) ? 0u : 1u);
+                        if (kPair) ptx::mma_ss_pair(d_tmem, a_desc, b_desc, idesc, (ks == 0 && k4 == 0) ? 0u : 1u);
+                        else ptx::mma_ss(d_tmem, a_desc, b_desc, idesc, (ks == 0 && k4 == 0) ? 0u : 1u);
                     }
-                    ptx::tc_commit_pair(&empty_bar[s], 3);
-                    if (ks == ks_total - 1) ptx::tc_commit_pair(&acc_full[n & 1], 3);
+                    if (kPair) {
+                        ptx::tc_commit_pair(&empty_bar[s], 3);
+                        if (ks == ks_total - 1) ptx::tc_commit_pair(&acc_full[n & 1], 3);
+                    } else {
+                        ptx::tc_commit(&empty_bar[s]);
+                        if (ks == ks_total - 1) ptx::tc_commit(&acc_full[n & 1]);
+                    }
                 }
             }
         }
@@ -227,14 +265,14 @@ sm100_linear_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
         const int half = (warp - 2) >> 2;
         const int row_in_tile = quarter * 32 + lane;
         const uint32_t lane_base = ((uint32_t)(quarter * 32) << 16);
-        const uint32_t acc_free_leader[2] = {ptx::map_to_cta(ptx::smem_addr(&acc_free[0]), 0),
-                                             ptx::map_to_cta(ptx::smem_addr(&acc_free[1]), 0)};
+        const uint32_t acc_free_leader[2] = {kPair ? ptx::map_to_cta(ptx::smem_addr(&acc_free[0]), 0) : 0u,
+                                             kPair ? ptx::map_to_cta(ptx::smem_addr(&acc_free[1]), 0) : 0u};
         const int Dq = a.d.n_q * a.d.d_h, Dk = a.d.n_k * a.d.d_h;
         bool ok = true;
         for (int n = 0; n < n_items && ok; ++n) {
             int row0, f0, nt;
             unit(n, row0, f0, nt);
-            const int cols = nt / 2;                 // this warp's columns: 128 or 64
+            const int cols = nt / 2;                 // this warp's columns: 128, 64 or 32
             const int c0 = half * cols;
             const int row = row0 + (int)rank * kTileM + row_in_tile;
             bool live = row < a.M;
@@ -298,14 +336,22 @@ sm100_linear_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
             }
             ptx::tc_fence_before_sync();
             __syncwarp();
-            if (lane == 0) ptx::mbar_arrive_cluster(acc_free_leader[n & 1]);
+            if (lane == 0) {
+                if (kPair) ptx::mbar_arrive_cluster(acc_free_leader[n & 1]);
+                else ptx::mbar_arrive(&acc_free[n & 1]);
+            }
         }
     }
     ptx::tc_fence_before_sync();
     __syncthreads();
-    ptx::cluster_arrive();     // neither CTA leaves (or frees TMEM) while the other may still signal it
-    ptx::cluster_wait();
-    if (warp == 1) ptx::tmem_dealloc_pair(tmem_base, 512);
+    if (kPair) {
+        ptx::cluster_arrive();     // neither CTA leaves (or frees TMEM) while the other may still signal it
+        ptx::cluster_wait();
+    }
+    if (warp == 1) {
+        if (kPair) ptx::tmem_dealloc_pair(tmem_base, 512);
+        else ptx::tmem_dealloc(tmem_base, 512);
+    }
     if (threadIdx.x == 0 && *abort_flag) raise_status(status_word, GTA_ERR_TIMEOUT);
 }
 
@@ -324,9 +370,10 @@ template <bool kProject>
 gta_status_t launch_linear(const LinArgs& a, const void* a_ptr, const void* w_ptr, int32_t* status_word,
                            cudaStream_t stream) {
     CUtensorMap tm_a, tm_w;
+    const bool solo = a.M <= kTileM;
     {
         const uint64_t dims[2] = {(uint64_t)a.K, (uint64_t)a.M};
-        const uint32_t box[2] = {kBlockK, kTileM};
+        const uint32_t box[2] = {kBlockK, solo ? a.a_bytes / (kBlockK * 2) : (uint32_t)kTileM};
         if (!make_bf16_map(&tm_a, a_ptr, 2, dims, box)) return GTA_ERR_CUDA;
     }
     {
@@ -334,20 +381,37 @@ gta_status_t launch_linear(const LinArgs& a, const void* a_ptr, const void* w_pt
         const uint32_t box[2] = {64, kBlockK};
         if (!make_bf16_map(&tm_w, w_ptr, 2, dims, box)) return GTA_ERR_CUDA;
     }
-    auto kern = sm100_linear_kernel<kProject>;
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kLinSmemTotal) != cudaSuccess)
-        return GTA_ERR_CUDA;
     cudaLaunchConfig_t cfg = {};
     cfg.blockDim = dim3(kLinThreads);
-    cfg.dynamicSmemBytes = kLinSmemTotal;
     cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
+    if (solo) {   // 64-column units over as many SMs as there are units
+        auto kern1 = sm100_linear_kernel<kProject, false>;
+        const uint32_t smem_bytes = (uint32_t)a.n_stages * (a.a_bytes + kBGroupBytes) + 512 + 1024;
+        if (cudaFuncSetAttribute(kern1, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes) != cudaSuccess)
+            return GTA_ERR_CUDA;
+        cfg.dynamicSmemBytes = smem_bytes;
+        cfg.gridDim = dim3(a.n_units < lin_sm_count() ? a.n_units : lin_sm_count());
+        cudaLaunchAttribute attr1[1];
+        attr1[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr1[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr1;
+        cfg.numAttrs = 1;
+        if (cudaLaunchKernelEx(&cfg, kern1, tm_a, tm_w, a, status_word) != cudaSuccess) return GTA_ERR_CUDA;
+        return cudaGetLastError() == cudaSuccess ? GTA_OK : GTA_ERR_CUDA;
+    }
+    auto kern = sm100_linear_kernel<kProject, true>;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kLinSmemTotal) != cudaSuccess)
+        return GTA_ERR_CUDA;
+    cfg.dynamicSmemBytes = kLinSmemTotal;
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = 2;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = 1;   // the occupancy query below takes the cluster attribute only
     // a persistent grid must be resident at once: as many pairs as the device can hold, asked once per device
     static thread_local int cached_dev = -1, cached_pairs = 0;
     int dev = 0;
@@ -361,6 +425,7 @@ gta_status_t launch_linear(const LinArgs& a, const void* a_ptr, const void* w_pt
     }
     const int G = a.n_units < cached_pairs ? a.n_units : cached_pairs;
     cfg.gridDim = dim3(2 * G);
+    cfg.numAttrs = 2;
     if (cudaLaunchKernelEx(&cfg, kern, tm_a, tm_w, a, status_word) != cudaSuccess) return GTA_ERR_CUDA;
     return cudaGetLastError() == cudaSuccess ? GTA_OK : GTA_ERR_CUDA;
 }
@@ -370,9 +435,21 @@ bool fill_common(LinArgs& a, long long M, int K, int n_cols) {
     a.M = (int)M;
     a.K = K;
     a.n_cols = n_cols;
-    a.block = M <= 2 * kTileM ? 128 : 256;      // a single row tile: narrower blocks keep twice as many SMs busy
+    const bool solo = M <= kTileM;
+    // a single row tile: narrower blocks keep more SMs busy
+    a.block = solo ? 64 : (M <= 2 * kTileM ? 128 : 256);
     a.n_cb = (n_cols + a.block - 1) / a.block;
-    const long long units = ((M + 2 * kTileM - 1) / (2 * kTileM)) * a.n_cb;
+    a.n_stages = kLinStages;
+    a.a_bytes = kATileBytes;
+    if (solo) {
+        a.a_bytes = (uint32_t)((M + 7) & ~7LL) * kBlockK * 2;
+        a.n_stages = (int)(kSoloRingBytes / (a.a_bytes + kBGroupBytes));
+        if (a.n_stages > kMaxStages) a.n_stages = kMaxStages;
+        // the MMA reads 16 KB from every A tile: the W tiles behind the last one must cover that
+        if ((uint32_t)a.n_stages * kBGroupBytes < kATileBytes) return false;
+    }
+    const long long unit_rows = solo ? kTileM : 2 * kTileM;
+    const long long units = ((M + unit_rows - 1) / unit_rows) * a.n_cb;
     if (units > 0x3fffffffLL) return false;
     a.n_units = (int)units;
     return true;

@@ -182,6 +182,54 @@ def run_decode_paged(w, iters, warmup, append, page_size):
             "cache_bytes": float(sum(lens)) * (w.n_k * w.d_h + w.n_c * w.d_l) * 2}
 
 
+def run_layer_decode(w, iters, warmup):
+    """One decode step of the whole attention layer per iteration (gta_layer_decode), two cache sets alternating;
+    the lengths are put back before every step (a 4-byte-per-sequence copy inside the timed loop)."""
+    dev = torch.device("cuda")
+    wl = I.scaled(w, kind="prefill", seq=1)
+    sets = []
+    for s in range(2):
+        td = I.decode_inputs(I.scaled(w, seed=w.seed + s), device=dev)
+        td["lens0"] = td["seq_lens"].clone() - 1          # the step appends the new token itself
+        td.update(I.layer_inputs(I.scaled(wl, seed=w.seed + s), device=dev))
+        td["x_t"] = td["x"][:, 0].contiguous()
+        sets.append(td)
+    td = sets[0]
+    shape = G.decode_shape(td["q"], td["k_cache"], td["c_cache"], td["x_t"], td["w_p"])
+    ws = torch.zeros(G.layer_decode_workspace_bytes(shape, td["s_cap"]), dtype=torch.uint8, device=dev)
+    u = torch.empty((w.batch, w.d_model), dtype=w.torch_dtype(), device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    stream = torch.cuda.current_stream()
+
+    def step(it):
+        td = sets[it % 2]
+        td["seq_lens"].copy_(td["lens0"])
+        G.gta_layer_decode(td["x_t"], td["w_qkc"], td["w_p"], td["w_g"], td["w_o"], td["k_cache"], td["c_cache"],
+                           td["seq_lens"], n_q=w.n_q, out=u, workspace=ws, status_word=status)
+
+    for it in range(warmup):
+        step(it)
+    torch.cuda.synchronize()
+    times = []
+    for rep in range(3):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for it in range(iters):
+            step(it)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        times.append(e0.elapsed_time(e1) / iters)
+    assert int(status.item()) == 0, "device status word raised"
+    lens = [n + 1 for n in sets[0]["lens0"].cpu().tolist()]
+    qkc = (w.n_q + w.n_k) * w.d_h + w.n_c * w.d_l
+    D = w.n_heads * w.d_h
+    cache_bytes = float(sum(lens)) * (w.n_k * w.d_h + w.n_c * w.d_l) * 2
+    weight_bytes = 2.0 * (w.d_model * qkc + w.n_heads * w.d_l * w.d_h + w.d_model * D + D * w.d_model)
+    ms = _median(times)
+    return {"whole_call": ms, "launches": G.last_launch_count(), "cache_bytes": cache_bytes,
+            "weight_bytes": weight_bytes, "gbs": (cache_bytes + weight_bytes) / (ms * 1e-3) / 1e9}
+
+
 def run_decode(w, iters, warmup, stages, append):
     dev = torch.device("cuda")
     sets = []
@@ -251,7 +299,8 @@ def main():
     ap.add_argument("--kv-len", type=int, default=0,
                     help="prefill: treat the workload's tokens as the last chunk of a context of this length")
     ap.add_argument("--layer", action="store_true",
-                    help="prefill: the whole attention layer (projections + RoPE + cache write, operator, W_O)")
+                    help="the whole attention layer (projections + RoPE + cache write, operator, W_O): "
+                         "gta_layer_prefill on a prefill workload, gta_layer_decode on a decode workload")
     ap.add_argument("--page-size", type=int, default=0,
                     help="decode: keep the caches in a paged pool with pages of this many tokens")
     args = ap.parse_args()
@@ -268,6 +317,8 @@ def main():
         res = run_prefill_chunk(w, args.iters, args.warmup, args.kv_len)
     elif w.kind == "prefill":
         res = run_prefill(w, args.iters, args.warmup, args.stages & 3)
+    elif args.layer:
+        res = run_layer_decode(w, args.iters, args.warmup)
     elif args.page_size > 0:
         res = run_decode_paged(w, args.iters, args.warmup, args.append, args.page_size)
     else:
