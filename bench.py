@@ -420,6 +420,34 @@ def run_ours(args):
     t_layer = l0.elapsed_time(l1) / K_l
     assert int(status.item()) == 0, "device status word raised during the benchmark"
     del tl, ws_l, kc_l, cc_l, u_l
+    # ---- one decode step of the whole layer on the decode workload's shape (projection of the new token + RoPE +
+    #      cache row write + length update, gta_decode, W_O), two cache sets alternating; the lengths are put back
+    #      before every step (a copy of 4 bytes per sequence inside the timed loop)
+    wl_d = I.scaled(wd, kind="prefill", seq=1)
+    tld = [I.layer_inputs(I.scaled(wl_d, seed=wd.seed + i), device=dev) for i in range(2)]
+    for t_ in tld:
+        t_["x_t"] = t_["x"][:, 0].contiguous()
+    ws_ld = torch.zeros(G.layer_decode_workspace_bytes(shape_d, wd.seq + 64), dtype=torch.uint8, device=dev)
+    u_ld = torch.empty((wd.batch, wd.d_model), dtype=torch.bfloat16, device=dev)
+
+    def layer_decode_call(i):
+        td, tl_ = sets[i % 2], tld[i % 2]
+        td["seq_lens"].copy_(td["lens0"])
+        G.gta_layer_decode(tl_["x_t"], tl_["w_qkc"], tl_["w_p"], tl_["w_g"], tl_["w_o"], td["k_cache"], td["c_cache"],
+                           td["seq_lens"], n_q=wd.n_q, out=u_ld, workspace=ws_ld, status_word=status)
+
+    for i in range(3):
+        layer_decode_call(i)
+    barrier()
+    l2, l3 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    l2.record(stream)
+    for i in range(K_d):
+        layer_decode_call(i)
+    l3.record(stream)
+    barrier()
+    t_layer_decode = l2.elapsed_time(l3) / K_d
+    assert int(status.item()) == 0, "device status word raised during the benchmark"
+    del tld, ws_ld, u_ld
 
     total_ms = e_start.elapsed_time(e_end)
     t_attn = sum(e[0].elapsed_time(e[1]) for e in evk) / K_k
@@ -438,6 +466,7 @@ def run_ours(args):
     t_decode_call = max_over_ranks_(t_decode_call)
     t_decode_paged = max_over_ranks_(t_decode_paged)
     t_layer = max_over_ranks_(t_layer)
+    t_layer_decode = max_over_ranks_(t_layer_decode)
 
     fl = prefill_flops(wp)
     by = decode_bytes(wd, [wd.seq] * wd.batch)
@@ -485,6 +514,13 @@ def run_ours(args):
              "ms": t_layer, "flops": fl_layer, "tflops": fl_layer / (t_layer * 1e-3) / 1e12,
              "frac_of_sustained_peak": fl_layer / (t_layer * 1e-3) / 1e12 / peaks["bf16_tflops_sustained"],
              "frac_of_burst_peak": fl_layer / (t_layer * 1e-3) / 1e12 / peaks["bf16_tflops"]}
+    lw_bytes = 2.0 * (wd.d_model * ((wd.n_q + wd.n_k) * wd.d_h + wd.n_c * wd.d_l) + wd.n_heads * wd.d_h * wd.d_model)
+    layer["decode_step"] = {
+        "call": "gta_layer_decode on the decode workload's shape, back to back", "ms": t_layer_decode,
+        "tokens_per_s": world * wd.batch / (t_layer_decode * 1e-3),
+        "algorithmic_bytes": by["total"] + lw_bytes,
+        "achieved": (by["total"] + lw_bytes) / (t_layer_decode * 1e-3) / 1e9,
+        "frac": (by["total"] + lw_bytes) / (t_layer_decode * 1e-3) / 1e9 / peaks["hbm_gbs"], "unit": "GB/s"}
     decode["paged"] = {"page_size": page_size, "ms_decode_call": t_decode_paged,
                        "achieved": by["total"] / (t_decode_paged * 1e-3) / 1e9,
                        "frac": by["total"] / (t_decode_paged * 1e-3) / 1e9 / peaks["hbm_gbs"],
