@@ -106,7 +106,8 @@ GTA_API gta_status_t gta_prefill(const gta_shape_t *shape, const void *q, const 
  * equals row kv_len - N + t of gta_prefill over all kv_len tokens.
  *
  *   q   [B, n_q, N, d_h]          x   [B, N, H]        out [B, N, n_h, d_h]
- *   k   [B, n_k, kv_cap, d_h]     c   [B, n_c, kv_cap, d_l]    rows 0 .. kv_len-1 are read
+ *   k   [B, n_k, kv_cap, d_h]     c   [B, n_c, kv_cap, d_l]    rows 0 .. kv_len-1 are read; the rows
+ *   behind them may hold anything (uninitialised memory, NaN bit patterns): nothing of them reaches out
  *   N <= kv_len <= kv_cap (else GTA_ERR_INVALID_ARG); kv_len = kv_cap = N is gta_prefill.
  * Workspace, weights, arithmetic, paths and errors as for gta_prefill.
  */
@@ -124,7 +125,8 @@ GTA_API gta_status_t gta_prefill_chunk(const gta_shape_t *shape, int32_t kv_len,
  *   q        [B, n_q, d_h]                 x_t [B, H]
  *   k_cache  [B, n_k, S_cap, d_h]          c_cache [B, n_c, S_cap, d_l]
  *   seq_lens device int32 [B], 0 <= seq_lens[b] <= S_cap (values above S_cap are clamped);
- *            a sequence with length 0 gets an all-zero output row
+ *            a sequence with length 0 gets an all-zero output row; cache rows at and behind
+ *            seq_lens[b] may hold anything (uninitialised memory, NaN bit patterns)
  *   w_p, w_g as in gta_prefill;  out [B, n_h, d_h]
  *   workspace: at least gta_decode_workspace_bytes(shape, S_cap) bytes, 256-byte aligned
  *     (split-KV partial results and gate partial sums).

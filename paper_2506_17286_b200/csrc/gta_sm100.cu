@@ -547,10 +547,14 @@ gta_status_t launch_sm100_prefill(const Dims& d, const void* q, const void* k, c
         CUtensorMap tm_q, tm_k, tm_c, tm_o;
         const uint32_t box[3] = {64, 128, 1}, box_k[3] = {64, 64, 1};
         const uint64_t dq[3] = {(uint64_t)d.d_h, (uint64_t)d.N, (uint64_t)d.B * d.n_q};
-        const uint64_t dk[3] = {(uint64_t)d.d_h, (uint64_t)d.S, (uint64_t)d.B * d.n_k};
-        const uint64_t dc[3] = {(uint64_t)d.d_l, (uint64_t)d.S, (uint64_t)d.B * d.n_c};
-        if (!make_bf16_map(&tm_q, q, 3, dq, box) || !make_bf16_map(&tm_k, k, 3, dk, box_k) ||
-            !make_bf16_map(&tm_c, c, 3, dc, box))
+        // K / C: Nk of the S rows of a plane take part; the rest (the unused tail of a cache, which may hold
+        // anything, NaN bit patterns included) lies outside the maps and reads as zeros
+        const uint64_t dk[3] = {(uint64_t)d.d_h, (uint64_t)d.Nk, (uint64_t)d.B * d.n_k};
+        const uint64_t dc[3] = {(uint64_t)d.d_l, (uint64_t)d.Nk, (uint64_t)d.B * d.n_c};
+        const uint64_t ak[3] = {(uint64_t)d.d_h, (uint64_t)d.S, (uint64_t)d.B * d.n_k};
+        const uint64_t ac[3] = {(uint64_t)d.d_l, (uint64_t)d.S, (uint64_t)d.B * d.n_c};
+        if (!make_bf16_map(&tm_q, q, 3, dq, box) || !make_bf16_map(&tm_k, k, 3, dk, box_k, ak) ||
+            !make_bf16_map(&tm_c, c, 3, dc, box, ac))
             return GTA_ERR_CUDA;
         {   // L [B n_q][N][d_l], stored in boxes of 128 rows x 64 columns
             const uint64_t dl[3] = {(uint64_t)d.d_l, (uint64_t)d.N, (uint64_t)d.B * d.n_q};

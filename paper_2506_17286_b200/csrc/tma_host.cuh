@@ -26,7 +26,11 @@ inline EncodeTiledFn tensor_map_encoder() {
 
 // Dense bf16 tensor of `rank` dimensions (innermost first), box `box`, 128-byte swizzle, zero
 // fill outside the tensor.  The innermost box extent must be 64 elements (one swizzle row).
-inline bool make_bf16_map(CUtensorMap* m, const void* base, int rank, const uint64_t* dims, const uint32_t* box) {
+// `alloc`, when given, holds the allocated extent of every dimension (>= dims): the strides follow the
+// allocation while only `dims` is addressable, so that rows that exist in memory but are not part of the
+// problem (the unused tail of a cache) read as zeros like everything else outside the tensor.
+inline bool make_bf16_map(CUtensorMap* m, const void* base, int rank, const uint64_t* dims, const uint32_t* box,
+                          const uint64_t* alloc = nullptr) {
     EncodeTiledFn fn = tensor_map_encoder();
     if (!fn) return false;
     cuuint64_t gdim[5], gstride[5];
@@ -36,7 +40,7 @@ inline bool make_bf16_map(CUtensorMap* m, const void* base, int rank, const uint
         gdim[i] = dims[i];
         bx[i] = box[i];
         estr[i] = 1;
-        stride *= dims[i];
+        stride *= alloc ? alloc[i] : dims[i];
         if (i < rank - 1) gstride[i] = stride;   // byte stride of dimension i+1
     }
     return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void*>(base), gdim, gstride, bx, estr,

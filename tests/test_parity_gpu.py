@@ -158,14 +158,14 @@ CHUNKS = [
 @pytest.mark.parametrize("case", CHUNKS, ids=[c[0] for c in CHUNKS])
 def test_prefill_chunk_against_a_longer_cache(B, oracle, case):
     """The chunk's rows must equal the same rows of a prefill over all kv_len tokens (oracle); the
-    cache rows past kv_len hold finite garbage that must not be read into the result."""
+    cache rows past kv_len hold NaN (what uninitialised memory may hold) and must not reach the result."""
     name, dt, nb, kv_len, N, kv_cap, H, n_h, n_q, n_k, n_c, d_h, d_l, causal = case
     w = I.Workload(name, "prefill", dt, nb, kv_len, H, n_h, n_q, n_k, n_c, d_h, d_l, seed=321)
     t = I.prefill_inputs(w, device="cuda")
     first = kv_len - N
     gen = torch.Generator(device="cuda").manual_seed(5)
-    k = torch.randn((nb, n_k, kv_cap, d_h), generator=gen, device="cuda").to(w.torch_dtype())
-    c = torch.randn((nb, n_c, kv_cap, d_l), generator=gen, device="cuda").to(w.torch_dtype())
+    k = torch.full((nb, n_k, kv_cap, d_h), float("nan"), device="cuda", dtype=w.torch_dtype())
+    c = torch.full((nb, n_c, kv_cap, d_l), float("nan"), device="cuda", dtype=w.torch_dtype())
     k[:, :, :kv_len] = t["k"]
     c[:, :, :kv_len] = t["c"]
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
@@ -181,8 +181,17 @@ def test_prefill_chunk_against_a_longer_cache(B, oracle, case):
 
 
 # --------------------------------------------------------------------------- decode
+def _nan_behind_the_live_rows(t):
+    """Cache rows at and past seq_lens[b] become NaN: what uninitialised memory may hold, and nothing of it may
+    reach the result (a masked probability times NaN would)."""
+    for b, n in enumerate(t["seq_lens"].cpu().tolist()):
+        t["k_cache"][b, :, n:] = float("nan")
+        t["c_cache"][b, :, n:] = float("nan")
+    return t
+
+
 def _decode_case(B, oracle, w, seq_lens=None, s_cap=None, sample=None):
-    t = I.decode_inputs(w, device="cuda", s_cap=s_cap, seq_lens=seq_lens)
+    t = _nan_behind_the_live_rows(I.decode_inputs(w, device="cuda", s_cap=s_cap, seq_lens=seq_lens))
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
     shape = B.decode_shape(t["q"], t["k_cache"], t["c_cache"], t["x_t"], t["w_p"])
     ws = torch.full((B.decode_workspace_bytes(shape, t["s_cap"]),), 0xFF, dtype=torch.uint8, device="cuda")
@@ -326,7 +335,8 @@ def test_append_then_decode_sequence_of_steps(B, oracle):
 # --------------------------------------------------------------------------- paged cache
 def _paged_decode_case(B, oracle, w, page_size, seq_lens=None, s_cap=None, sample=None, holes=True):
     """gta_decode_paged against the oracle reading the same pools through the same block table."""
-    t = I.paginate(I.decode_inputs(w, device="cuda", s_cap=s_cap, seq_lens=seq_lens), page_size, seed=w.seed)
+    t = I.paginate(_nan_behind_the_live_rows(I.decode_inputs(w, device="cuda", s_cap=s_cap, seq_lens=seq_lens)),
+                   page_size, seed=w.seed)
     table = t["block_table"].clone()
     if holes:   # entries no live token maps to are never read: poison them
         lens_h = t["seq_lens"].cpu().tolist()
