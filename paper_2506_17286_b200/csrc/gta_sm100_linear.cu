@@ -79,6 +79,9 @@ struct RopeArgs {
 // one thread per (token of the chunk, pair)
 __global__ void __launch_bounds__(256)
 rope_table_kernel(const __grid_constant__ RopeArgs r, float2* __restrict__ table) {
+    // launched with programmatic stream serialisation: the table may still be read by the kernel ahead
+    ptx::grid_dependency_wait();
+    ptx::grid_launch_dependents();
     const int idx = blockIdx.x * 256 + threadIdx.x;
     const int t = idx / r.n_pairs, i = idx - t * r.n_pairs;
     if (t >= r.n_tokens) return;
@@ -100,6 +103,10 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
 __global__ void __launch_bounds__(kMaxRopePairs)
 rope_decode_prep_kernel(const __grid_constant__ RopeArgs r, int S_cap, int32_t* __restrict__ seq_lens,
                         int32_t* __restrict__ pos_out, float2* __restrict__ table, int32_t* status_word) {
+    // launched with programmatic stream serialisation: lengths, positions and table belong to the kernels ahead
+    // in the stream until they are complete
+    ptx::grid_dependency_wait();
+    ptx::grid_launch_dependents();
     const int b = blockIdx.x, i = threadIdx.x;
     const int len = seq_lens[b];
     __syncthreads();   // every thread has read the old length before thread 0 rewrites it
@@ -483,8 +490,20 @@ gta_status_t launch_sm100_project(const Dims& d, int pos0, int S_cap, double rop
     r.n_pairs = d.d_h / 2;
     for (int i = 0; i < r.n_pairs; ++i) r.theta[i] = pow(rope_base, -2.0 * i / d.d_h);
     r.n_tokens = d.N;
-    rope_table_kernel<<<(d.N * r.n_pairs + 255) / 256, 256, 0, stream>>>(r, static_cast<float2*>(rope_table));
-    if (cudaGetLastError() != cudaSuccess) return GTA_ERR_CUDA;
+    {
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((d.N * r.n_pairs + 255) / 256);
+        cfg.blockDim = dim3(256);
+        cfg.stream = stream;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        if (cudaLaunchKernelEx(&cfg, rope_table_kernel, r, static_cast<float2*>(rope_table)) != cudaSuccess ||
+            cudaGetLastError() != cudaSuccess)
+            return GTA_ERR_CUDA;
+    }
     return launch_linear<true>(a, x, w_qkc, status_word, stream);
 }
 
@@ -512,8 +531,21 @@ gta_status_t launch_sm100_project_step(const Dims& d, int S_cap, double rope_bas
     RopeArgs r = {};
     r.n_pairs = d.d_h / 2;
     for (int i = 0; i < r.n_pairs; ++i) r.theta[i] = pow(rope_base, -2.0 * i / d.d_h);
-    rope_decode_prep_kernel<<<d.B, kMaxRopePairs, 0, stream>>>(r, S_cap, seq_lens, pos, table, status_word);
-    if (cudaGetLastError() != cudaSuccess) return GTA_ERR_CUDA;
+    {
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(d.B);
+        cfg.blockDim = dim3(kMaxRopePairs);
+        cfg.stream = stream;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        if (cudaLaunchKernelEx(&cfg, rope_decode_prep_kernel, r, S_cap, seq_lens, pos, table, status_word) !=
+                cudaSuccess ||
+            cudaGetLastError() != cudaSuccess)
+            return GTA_ERR_CUDA;
+    }
     return launch_linear<true>(a, x_t, w_qkc, status_word, stream);
 }
 
