@@ -257,6 +257,22 @@ GTA_API gta_status_t gta_layer_decode(const gta_shape_t *shape, int32_t S_cap, f
                                       size_t workspace_bytes, int32_t *status_word, void *cuda_stream);
 
 /*
+ * gta_layer_decode_paged — gta_layer_decode over a paged cache (pools, block table and their rules as
+ * in gta_decode_paged; the capacity of a sequence is page_size * max_pages).  The new token's key and
+ * latent rows go to row p % page_size of page block_table[b, p / page_size], p = seq_lens[b]; an entry
+ * outside [0, n_pages) raises GTA_ERR_BAD_PAGE and the row is not written.
+ */
+GTA_API size_t gta_layer_decode_paged_workspace_bytes(const gta_shape_t *shape, int32_t page_size,
+                                                      int32_t max_pages);
+GTA_API gta_status_t gta_layer_decode_paged(const gta_shape_t *shape, const int32_t *block_table,
+                                            int32_t page_size, int32_t n_pages, int32_t max_pages,
+                                            float rope_base, const void *x_t, const void *w_qkc,
+                                            const void *w_p, const void *w_g, const void *w_o,
+                                            void *k_pool, void *c_pool, int32_t *seq_lens, void *u,
+                                            void *workspace, size_t workspace_bytes,
+                                            int32_t *status_word, void *cuda_stream);
+
+/*
  * gta_decode_static — gta_decode without a workspace argument (the paper has no counterpart: this
  * is a packaging variant of the same decode step, with the same arguments, results and errors).
  *

@@ -26,6 +26,7 @@ EXPORTS = (
     "gta_prefill_stages", "gta_decode_stages", "gta_decode_static", "gta_prefill_chunk",
     "gta_decode_paged_workspace_bytes", "gta_decode_paged", "gta_cache_append_paged",
     "gta_layer_prefill_workspace_bytes", "gta_layer_prefill", "gta_layer_decode_workspace_bytes", "gta_layer_decode",
+    "gta_layer_decode_paged_workspace_bytes", "gta_layer_decode_paged",
 )
 
 
@@ -91,6 +92,11 @@ def lib():
         L.gta_layer_decode_workspace_bytes.restype = sz
         L.gta_layer_decode.argtypes = [sp, i32, ctypes.c_float, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp, vp]
         L.gta_layer_decode.restype = i32
+        L.gta_layer_decode_paged_workspace_bytes.argtypes = [sp, i32, i32]
+        L.gta_layer_decode_paged_workspace_bytes.restype = sz
+        L.gta_layer_decode_paged.argtypes = [sp, vp, i32, i32, i32, ctypes.c_float, vp, vp, vp, vp, vp, vp, vp, vp, vp,
+                                             vp, sz, vp, vp]
+        L.gta_layer_decode_paged.restype = i32
         L.gta_status_string.argtypes = [i32]
         L.gta_status_string.restype = ctypes.c_char_p
         L.gta_version.restype = i32
@@ -278,6 +284,37 @@ def gta_layer_decode(x_t, w_qkc, w_p, w_g, w_o, k_cache, c_cache, seq_lens, *, r
                                 _stream(stream))
     if st != GTA_OK:
         raise GtaError(st, "gta_layer_decode")
+    return out
+
+
+def layer_decode_paged_workspace_bytes(shape: GtaShape, page_size: int, max_pages: int) -> int:
+    return int(lib().gta_layer_decode_paged_workspace_bytes(ctypes.byref(shape), int(page_size), int(max_pages)))
+
+
+def gta_layer_decode_paged(x_t, w_qkc, w_p, w_g, w_o, k_pool, c_pool, block_table, seq_lens, *, rope_base=10000.0,
+                           n_q, softmax_scale=0.0, out=None, workspace=None, status_word=None, stream=None):
+    """gta_layer_decode over a paged cache (pools and block table as in gta_decode_paged)."""
+    _check_tensors(x_t, w_qkc, w_p, w_g, w_o, k_pool, c_pool)
+    n_pages, page_size, max_pages = _check_paged(k_pool, c_pool, block_table, seq_lens)
+    B, H = x_t.shape
+    n_h, d_l, d_h = w_p.shape
+    n_k, n_c = k_pool.shape[1], c_pool.shape[1]
+    if k_pool.shape[3] != d_h or c_pool.shape[3] != d_l or block_table.shape[0] != B \
+            or w_qkc.shape != (H, (n_q + n_k) * d_h + n_c * d_l) or w_g.shape != (H, n_h * d_h) \
+            or w_o.shape != (n_h * d_h, H):
+        raise ValueError("inconsistent layer tensor shapes")
+    shape = make_shape(batch=B, seq=0, d_model=H, n_heads=n_h, n_q=n_q, n_k=n_k, n_c=n_c, d_h=d_h, d_l=d_l,
+                       dtype=_dtype_code(x_t), causal=True, softmax_scale=softmax_scale)
+    if out is None:
+        out = torch.empty((B, H), dtype=x_t.dtype, device=x_t.device)
+    if workspace is None:
+        workspace = _workspace(layer_decode_paged_workspace_bytes(shape, page_size, max_pages), x_t.device)
+    st = lib().gta_layer_decode_paged(ctypes.byref(shape), _ptr(block_table), page_size, n_pages, max_pages,
+                                      float(rope_base), _ptr(x_t), _ptr(w_qkc), _ptr(w_p), _ptr(w_g), _ptr(w_o),
+                                      _ptr(k_pool), _ptr(c_pool), _ptr(seq_lens), _ptr(out), _ptr(workspace),
+                                      workspace.numel() * workspace.element_size(), _ptr(status_word), _stream(stream))
+    if st != GTA_OK:
+        raise GtaError(st, "gta_layer_decode_paged")
     return out
 
 

@@ -302,10 +302,56 @@ extern "C" size_t gta_layer_decode_workspace_bytes(const gta_shape_t* shape, int
            align256(gta::sm100_decode_prep_bytes(d)) + gta::decode_workspace_bytes(d, shape->dtype, S_cap);
 }
 
+static gta_status_t layer_decode_impl(const gta_shape_t* shape, int32_t S_cap, float rope_base, const void* x_t,
+                                      const void* w_qkc, const void* w_p, const void* w_g, const void* w_o,
+                                      void* k_cache, void* c_cache, int32_t* seq_lens, void* u, void* workspace,
+                                      size_t workspace_bytes, int32_t* status_word, void* cuda_stream,
+                                      const gta::PageMap& pm);
+
 extern "C" gta_status_t gta_layer_decode(const gta_shape_t* shape, int32_t S_cap, float rope_base, const void* x_t,
                                          const void* w_qkc, const void* w_p, const void* w_g, const void* w_o,
                                          void* k_cache, void* c_cache, int32_t* seq_lens, void* u, void* workspace,
                                          size_t workspace_bytes, int32_t* status_word, void* cuda_stream) {
+    return layer_decode_impl(shape, S_cap, rope_base, x_t, w_qkc, w_p, w_g, w_o, k_cache, c_cache, seq_lens, u,
+                             workspace, workspace_bytes, status_word, cuda_stream, gta::PageMap());
+}
+
+extern "C" size_t gta_layer_decode_paged_workspace_bytes(const gta_shape_t* shape, int32_t page_size,
+                                                         int32_t max_pages) {
+    gta::Dims d;
+    if (check_shape(shape, false, &d) != GTA_OK || page_size <= 0 || max_pages <= 0 ||
+        (long long)page_size * max_pages > INT32_MAX)
+        return 0;
+    const size_t es = elem_size(shape->dtype);
+    return align256((size_t)d.B * d.n_q * d.d_h * es) + align256((size_t)d.B * d.n_h * d.d_h * es) +
+           align256(gta::sm100_decode_prep_bytes(d)) +
+           gta::decode_workspace_bytes(d, shape->dtype, page_size * max_pages, page_size);
+}
+
+extern "C" gta_status_t gta_layer_decode_paged(const gta_shape_t* shape, const int32_t* block_table,
+                                               int32_t page_size, int32_t n_pages, int32_t max_pages,
+                                               float rope_base, const void* x_t, const void* w_qkc, const void* w_p,
+                                               const void* w_g, const void* w_o, void* k_pool, void* c_pool,
+                                               int32_t* seq_lens, void* u, void* workspace, size_t workspace_bytes,
+                                               int32_t* status_word, void* cuda_stream) {
+    g_last_launches = 0;
+    if (!block_table || !aligned(block_table, 4) || page_size <= 0 || n_pages <= 0 || max_pages <= 0 ||
+        (long long)page_size * max_pages > INT32_MAX)
+        return GTA_ERR_INVALID_ARG;
+    gta::PageMap pm;
+    pm.table = block_table;
+    pm.page_size = page_size;
+    pm.max_pages = max_pages;
+    pm.n_pages = n_pages;
+    return layer_decode_impl(shape, page_size * max_pages, rope_base, x_t, w_qkc, w_p, w_g, w_o, k_pool, c_pool,
+                             seq_lens, u, workspace, workspace_bytes, status_word, cuda_stream, pm);
+}
+
+static gta_status_t layer_decode_impl(const gta_shape_t* shape, int32_t S_cap, float rope_base, const void* x_t,
+                                      const void* w_qkc, const void* w_p, const void* w_g, const void* w_o,
+                                      void* k_cache, void* c_cache, int32_t* seq_lens, void* u, void* workspace,
+                                      size_t workspace_bytes, int32_t* status_word, void* cuda_stream,
+                                      const gta::PageMap& pm) {
     g_last_launches = 0;
     gta::Dims d;
     gta_status_t st = check_shape(shape, false, &d);
@@ -319,8 +365,9 @@ extern "C" gta_status_t gta_layer_decode(const gta_shape_t* shape, int32_t S_cap
     if (!gta::sm100_linear_supported(d, shape->dtype) || (size_t)d.d_l * elem_size(shape->dtype) > 4096)
         return GTA_ERR_UNSUPPORTED;
     if (d.B == 0) return GTA_OK;
-    if (!workspace || !aligned(workspace, 256) || workspace_bytes < gta_layer_decode_workspace_bytes(shape, S_cap))
-        return GTA_ERR_WORKSPACE;
+    const size_t ws_need = pm.table ? gta_layer_decode_paged_workspace_bytes(shape, pm.page_size, pm.max_pages)
+                                    : gta_layer_decode_workspace_bytes(shape, S_cap);
+    if (!workspace || !aligned(workspace, 256) || workspace_bytes < ws_need) return GTA_ERR_WORKSPACE;
     if ((st = check_device()) != GTA_OK) return st;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     const size_t es = elem_size(shape->dtype);
@@ -331,10 +378,10 @@ extern "C" gta_status_t gta_layer_decode(const gta_shape_t* shape, int32_t S_cap
     char* op_ws = prep_ws + align256(gta::sm100_decode_prep_bytes(d));
     const size_t op_ws_bytes = workspace_bytes - (size_t)(op_ws - ws);
     st = gta::launch_sm100_project_step(d, S_cap, (double)rope_base, x_t, w_qkc, q_ws, k_cache, c_cache, seq_lens,
-                                        prep_ws, status_word, stream);
+                                        prep_ws, status_word, stream, pm);
     if (st != GTA_OK) return st;
     st = decode_impl(shape, q_ws, k_cache, c_cache, seq_lens, S_cap, x_t, w_p, w_g, o_ws, op_ws, op_ws_bytes,
-                     status_word, cuda_stream, 7, gta::PageMap());
+                     status_word, cuda_stream, 7, pm);
     if (st != GTA_OK) return st;
     const int op_launches = g_last_launches;
     st = gta::launch_sm100_matmul(d.B, d.n_h * d.d_h, d.H, o_ws, w_o, u, status_word, stream);

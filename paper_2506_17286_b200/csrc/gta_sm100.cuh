@@ -31,11 +31,11 @@ gta_status_t launch_sm100_project(const Dims& d, int pos0, int S_cap, double rop
 
 // One decode step of the same projection: one new token per sequence at position seq_lens[b] (RoPE there,
 // k and c to that cache row, q to q_out [B, n_q, d_h]), then seq_lens[b] += 1; a sequence whose cache is full
-// is skipped and raises GTA_ERR_CACHE_FULL.  prep: sm100_decode_prep_bytes(d) bytes of scratch.
+// is skipped and raises GTA_ERR_CACHE_FULL.  With a page map, k_cache / c_cache are the paged pools.  prep: sm100_decode_prep_bytes(d) bytes of scratch.
 size_t sm100_decode_prep_bytes(const Dims& d);
 gta_status_t launch_sm100_project_step(const Dims& d, int S_cap, double rope_base, const void* x_t, const void* w_qkc,
                                        void* q_out, void* k_cache, void* c_cache, int32_t* seq_lens, void* prep,
-                                       int32_t* status_word, cudaStream_t stream);
+                                       int32_t* status_word, cudaStream_t stream, const PageMap& pm = PageMap());
 
 // C[M, n_cols] = A[M, K] W[K, n_cols], row-major.
 gta_status_t launch_sm100_matmul(long long M, int K, int n_cols, const void* a, const void* w, void* c_out,

@@ -69,6 +69,7 @@ struct LinArgs {
     // one new token per sequence (N = 1): its position, or -1 for a sequence whose cache is full (nothing is
     // written for it); the table then has one row per sequence
     const int32_t* pos_seq;
+    PageMap pm;              // table != nullptr: the caches are paged pools (decode step only)
 };
 
 struct RopeArgs {
@@ -322,12 +323,19 @@ sm100_linear_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
                             v[4 * j2 + 2] = __float_as_uint(x2 * r4.z - x3 * r4.w);
                             v[4 * j2 + 3] = __float_as_uint(x2 * r4.w + x3 * r4.z);
                         }
-                        dst = is_q ? a.q_out + (((size_t)b * a.d.n_q + g) * a.d.N + t) * a.d.d_h + e0
-                                   : a.k_cache + (((size_t)b * a.d.n_k + g) * a.S_cap + pos) * a.d.d_h + e0;
+                        if (is_q) {
+                            dst = a.q_out + (((size_t)b * a.d.n_q + g) * a.d.N + t) * a.d.d_h + e0;
+                        } else {
+                            const long long kr = cache_row(a.pm, b, a.d.n_k, g, a.S_cap, pos, status_word);
+                            live = live && kr >= 0;          // a block-table entry outside the pool: nothing is written
+                            dst = a.k_cache + (size_t)(kr < 0 ? 0 : kr) * a.d.d_h + e0;
+                        }
                     } else {
                         const int cc = col - Dq - Dk;
                         const int g = cc / a.d.d_l, e0 = cc - g * a.d.d_l;
-                        dst = a.c_cache + (((size_t)b * a.d.n_c + g) * a.S_cap + pos) * a.d.d_l + e0;
+                        const long long cr = cache_row(a.pm, b, a.d.n_c, g, a.S_cap, pos, status_word);
+                        live = live && cr >= 0;
+                        dst = a.c_cache + (size_t)(cr < 0 ? 0 : cr) * a.d.d_l + e0;
                     }
                     if (live) {
 #pragma unroll
@@ -513,8 +521,9 @@ size_t sm100_decode_prep_bytes(const Dims& d) {
 
 gta_status_t launch_sm100_project_step(const Dims& d, int S_cap, double rope_base, const void* x_t, const void* w_qkc,
                                        void* q_out, void* k_cache, void* c_cache, int32_t* seq_lens, void* prep,
-                                       int32_t* status_word, cudaStream_t stream) {
+                                       int32_t* status_word, cudaStream_t stream, const PageMap& pm) {
     LinArgs a = {};
+    a.pm = pm;
     Dims d1 = d;
     d1.N = 1;
     if (!fill_common(a, d.B, d.H, (d.n_q + d.n_k) * d.d_h + d.n_c * d.d_l)) return GTA_ERR_UNSUPPORTED;

@@ -122,6 +122,39 @@ def test_bad_arguments_are_rejected_on_the_host(B):
     assert B.decode_paged_workspace_bytes(good, 64, 4) == B.decode_workspace_bytes(good, 256)
     assert B.decode_paged_workspace_bytes(good, 0, 4) == 0
 
+    def layer_prefill(shape, pos0=0, s_cap=128, base=10000.0, ws_bytes=1 << 40):
+        return L.gta_layer_prefill(ctypes.byref(shape), pos0, s_cap, ctypes.c_float(base), p, p, p, p, p, p, p, p, p,
+                                   ws_bytes, None, None)
+
+    lay = _shape(B, d_model=128, n_heads=4, n_q=2, n_k=2, n_c=1, d_h=64, d_l=128)     # (2 + 2) 64 + 128 = 384 columns
+    assert layer_prefill(lay, pos0=-1) == B.GTA_ERR_INVALID_ARG
+    assert layer_prefill(lay, pos0=65) == B.GTA_ERR_INVALID_ARG           # 65 + 64 tokens do not fit 128 rows
+    assert layer_prefill(lay, base=1.0) == B.GTA_ERR_INVALID_ARG
+    assert layer_prefill(_shape(B, d_model=128, n_heads=4, n_q=2, n_k=2, n_c=1, d_h=64, d_l=128, causal=0)) \
+        == B.GTA_ERR_INVALID_ARG
+    assert layer_prefill(_shape(B, d_model=128, n_heads=4, n_q=2, n_k=1, n_c=1, d_h=64, d_l=128)) \
+        == B.GTA_ERR_UNSUPPORTED                                          # 320 projection columns: no multiple of 128
+    assert layer_prefill(_shape(B, d_model=128, n_heads=4, n_q=2, n_k=2, n_c=1, d_h=64, d_l=128, dtype=B.GTA_F32)) \
+        == B.GTA_ERR_UNSUPPORTED
+    assert layer_prefill(lay, ws_bytes=8) == B.GTA_ERR_WORKSPACE
+    assert layer_prefill(_shape(B, d_model=128, n_heads=4, n_q=2, n_k=2, n_c=1, d_h=64, d_l=128, seq=0)) == B.GTA_OK
+    assert B.layer_prefill_workspace_bytes(lay) > B.prefill_workspace_bytes(lay)
+
+    def layer_decode(shape, s_cap=128, base=10000.0, lens=p, ws_bytes=1 << 40):
+        return L.gta_layer_decode(ctypes.byref(shape), s_cap, ctypes.c_float(base), p, p, p, p, p, p, p, lens, p, p,
+                                  ws_bytes, None, None)
+
+    assert layer_decode(lay, s_cap=0) == B.GTA_ERR_INVALID_ARG
+    assert layer_decode(lay, base=0.5) == B.GTA_ERR_INVALID_ARG
+    assert layer_decode(lay, lens=None) == B.GTA_ERR_INVALID_ARG
+    assert layer_decode(lay, ws_bytes=8) == B.GTA_ERR_WORKSPACE
+    assert layer_decode(_shape(B, d_model=128, n_heads=4, n_q=2, n_k=2, n_c=1, d_h=64, d_l=128, batch=0)) == B.GTA_OK
+    assert L.gta_layer_decode_paged(ctypes.byref(lay), None, 64, 10, 4, ctypes.c_float(1e4), p, p, p, p, p, p, p, p, p,
+                                    p, 1 << 40, None, None) == B.GTA_ERR_INVALID_ARG
+    assert L.gta_layer_decode_paged(ctypes.byref(lay), p, 0, 10, 4, ctypes.c_float(1e4), p, p, p, p, p, p, p, p, p,
+                                    p, 1 << 40, None, None) == B.GTA_ERR_INVALID_ARG
+    assert B.layer_decode_paged_workspace_bytes(lay, 64, 2) == B.layer_decode_workspace_bytes(lay, 128)
+
     def append_paged(shape, table=p, page_size=64, n_new=1):
         return L.gta_cache_append_paged(ctypes.byref(shape), p, p, table, page_size, 10, 4, p, p, n_new, p, None, None)
 

@@ -131,11 +131,21 @@ def test_layer_decode_step_equals_the_next_row_of_the_layer(B, oracle, case):
     shape = B.make_shape(batch=nb, seq=0, d_model=H, n_heads=n_h, n_q=n_q, n_k=n_k, n_c=n_c, d_h=d_h, d_l=d_l,
                          dtype=torch.bfloat16)
     ws = torch.full((B.layer_decode_workspace_bytes(shape, cap),), 0xFF, dtype=torch.uint8, device="cuda")
+    # the same step over the same caches scattered into 64-token pages: bit-identical output and rows
+    pg = I.paginate(dict(k_cache=k_cache, c_cache=c_cache), 64, seed=9)
+    lens_p = seq_lens.clone()
+    u_p = B.gta_layer_decode_paged(x_t, t["w_qkc"], t["w_p"], t["w_g"], t["w_o"], pg["k_pool"], pg["c_pool"],
+                                   pg["block_table"], lens_p, n_q=n_q, status_word=status)
     u = B.gta_layer_decode(x_t, t["w_qkc"], t["w_p"], t["w_g"], t["w_o"], k_cache, c_cache, seq_lens, n_q=n_q,
                            workspace=ws, status_word=status)
     torch.cuda.synchronize()
     assert int(status.item()) == 0
-    assert seq_lens.tolist() == [n + 1 for n in lens]
+    assert seq_lens.tolist() == [n + 1 for n in lens] and lens_p.tolist() == seq_lens.tolist()
+    assert torch.equal(u_p.view(torch.int16), u.view(torch.int16))
+    for b, n in enumerate(lens):
+        page = int(pg["block_table"][b, n // 64])
+        assert torch.equal(pg["k_pool"][page, :, n % 64].view(torch.int16), k_cache[b, :, n].view(torch.int16))
+        assert torch.equal(pg["c_pool"][page, :, n % 64].view(torch.int16), c_cache[b, :, n].view(torch.int16))
     tc = {n: v.cpu() for n, v in t.items()}
     want_u = np.zeros((nb, H))
     for b, n in enumerate(lens):
