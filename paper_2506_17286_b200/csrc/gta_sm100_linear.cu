@@ -294,6 +294,19 @@ sm100_linear_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
                 if (pos < 0) pos = 0;
             }
             const uint32_t acc = tmem_base + (uint32_t)(n & 1) * 256 + lane_base + c0;
+            // (cos, sin) of the 16 pairs of piece ch, fetched one piece ahead of its use -- the first one before
+            // the accumulator is even complete: they depend on the row and the columns only
+            float4 rope_next[8];
+            auto fetch_rope = [&](int ch) {
+                const int col = f0 + c0 + ch * 32;
+                if (!kProject || ch * 32 >= cols || col >= Dq + Dk) return;
+                const int cc = col < Dq ? col : col - Dq;
+                const int e0 = cc % a.d.d_h;
+                const float4* rt = reinterpret_cast<const float4*>(a.rope + ((size_t)rope_row * (a.d.d_h >> 1) + (e0 >> 1)));
+#pragma unroll
+                for (int j2 = 0; j2 < 8; ++j2) rope_next[j2] = __ldg(rt + j2);
+            };
+            fetch_rope(0);
             ok = __all_sync(0xffffffffu, ptx::mbar_wait(&acc_full[n & 1], (n >> 1) & 1, abort_flag));
             if (!ok) break;
             ptx::tc_fence_after_sync();
@@ -302,6 +315,10 @@ sm100_linear_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
                 if (ch * 32 < cols) {
                     uint32_t v[32];
                     ptx::tmem_ld32(acc + ch * 32, v);
+                    float4 rope_cur[8];
+#pragma unroll
+                    for (int j2 = 0; j2 < 8; ++j2) rope_cur[j2] = rope_next[j2];
+                    if (ch + 1 < 4) fetch_rope(ch + 1);
                     ptx::tmem_wait_ld();
                     const int col = f0 + c0 + ch * 32;     // first of these 32 output columns
                     __nv_bfloat16* dst;
@@ -312,10 +329,9 @@ sm100_linear_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
                         const bool is_q = col < Dq;
                         const int cc = is_q ? col : col - Dq;
                         const int g = cc / a.d.d_h, e0 = cc - g * a.d.d_h;
-                        const float4* rt = reinterpret_cast<const float4*>(a.rope + ((size_t)rope_row * (a.d.d_h >> 1) + (e0 >> 1)));
 #pragma unroll
-                        for (int j2 = 0; j2 < 8; ++j2) {      // two pairs per 16-byte load
-                            const float4 r4 = __ldg(rt + j2);
+                        for (int j2 = 0; j2 < 8; ++j2) {      // two pairs per 16-byte table entry
+                            const float4 r4 = rope_cur[j2];
                             const float x0 = __uint_as_float(v[4 * j2]), x1 = __uint_as_float(v[4 * j2 + 1]);
                             const float x2 = __uint_as_float(v[4 * j2 + 2]), x3 = __uint_as_float(v[4 * j2 + 3]);
                             v[4 * j2] = __float_as_uint(x0 * r4.x - x1 * r4.y);
