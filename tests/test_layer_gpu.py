@@ -95,7 +95,7 @@ def _sample_positions(N, n=24, seed=0):
     return sorted(set(fixed) | set(int(v) for v in rng.integers(0, N, n)))
 
 
-@pytest.mark.parametrize("name", ["c2_prefill_bf16", "x1_gta1b_prefill_bf16"])
+@pytest.mark.parametrize("name", ["c2_prefill_bf16", "x1_gta1b_prefill_bf16", "c4_long_prefill_bf16"])
 def test_layer_prefill_full_size_sampled_positions(B, oracle, name):
     w = I.CONFIGS[name]
     _layer_case(B, oracle, w, sample=_sample_positions(w.seq))
