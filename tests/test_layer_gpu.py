@@ -106,6 +106,8 @@ LAYER_STEPS = [
     ("c3_shape_small", 512, 8, 4, 4, 1, 128, 512, [1, 63, 64, 200, 0]),
     ("paper_1b_shape", 1280, 20, 5, 1, 1, 64, 128, [130, 7]),
     ("two_latents_batch_20", 256, 8, 4, 2, 2, 64, 128, [(37 * i) % 150 for i in range(20)]),
+    # more than 128 sequences: the one-token projections run on CTA pairs again (two row tiles)
+    ("batch_150", 256, 8, 4, 2, 2, 64, 128, [(13 * i) % 90 for i in range(150)]),
 ]
 
 
