@@ -57,6 +57,11 @@ struct LinArgs {
     uint32_t a_bytes;        // bytes of an A tile in the ring
     int n_cb;                // column blocks (the last one possibly 128 wide)
     int n_units;             // row tiles (256 rows) x column blocks
+    // Static schedule over G CTA pairs (or CTAs): every pair takes q = n_units / G whole units (unit pr + n G,
+    // so that neighbouring pairs share a row tile); the r = n_units mod G left over are cut into two halves of
+    // 128 columns when that makes the last round shorter (2 r <= G and every block is 256 wide), else handed
+    // out whole.
+    int q, r, split_tail;
     // plain epilogue
     __nv_bfloat16* c_out;    // [M, n_cols]
     // projection epilogue: row = b N + t
@@ -154,7 +159,7 @@ sm100_linear_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
     const int G = kPair ? gridDim.x >> 1 : gridDim.x;                   // CTA pairs (or CTAs)
     const int pr = kPair ? blockIdx.x >> 1 : blockIdx.x;
     constexpr int kUnitRows = kPair ? 2 * kTileM : kTileM;
-    const int n_items = pr < a.n_units ? (a.n_units - pr + G - 1) / G : 0;
+    const int n_items = a.q + ((a.split_tail ? pr < 2 * a.r : pr < a.r) ? 1 : 0);
     const int ks_total = a.K / kBlockK;
 
     if (threadIdx.x == 0) {
@@ -184,11 +189,15 @@ sm100_linear_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
 
     // unit n of this pair: column block cb (consecutive pairs share a row tile), first row, first column, width
     auto unit = [&](int n, int& row0, int& f0, int& nt) {
-        const int u = pr + n * G;
+        int u, half = -1;
+        if (n < a.q) u = pr + n * G;
+        else if (a.split_tail) { u = G * a.q + (pr >> 1); half = pr & 1; }
+        else u = G * a.q + pr;
         const int cb = u % a.n_cb;
         row0 = (u / a.n_cb) * kUnitRows;
         f0 = cb * a.block;
         nt = a.n_cols - f0 < a.block ? a.n_cols - f0 : a.block;
+        if (half >= 0) { f0 += 128 * half; nt = 128; }
     };
 
     if (warp == 0) {
@@ -421,13 +430,18 @@ gta_status_t launch_linear(const LinArgs& a, const void* a_ptr, const void* w_pt
         if (cudaFuncSetAttribute(kern1, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes) != cudaSuccess)
             return GTA_ERR_CUDA;
         cfg.dynamicSmemBytes = smem_bytes;
-        cfg.gridDim = dim3(a.n_units < lin_sm_count() ? a.n_units : lin_sm_count());
+        const int G1 = a.n_units < lin_sm_count() ? a.n_units : lin_sm_count();
+        LinArgs a1 = a;
+        a1.q = a.n_units / G1;
+        a1.r = a.n_units % G1;
+        a1.split_tail = 0;
+        cfg.gridDim = dim3(G1);
         cudaLaunchAttribute attr1[1];
         attr1[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
         attr1[0].val.programmaticStreamSerializationAllowed = 1;
         cfg.attrs = attr1;
         cfg.numAttrs = 1;
-        if (cudaLaunchKernelEx(&cfg, kern1, tm_a, tm_w, a, status_word) != cudaSuccess) return GTA_ERR_CUDA;
+        if (cudaLaunchKernelEx(&cfg, kern1, tm_a, tm_w, a1, status_word) != cudaSuccess) return GTA_ERR_CUDA;
         return cudaGetLastError() == cudaSuccess ? GTA_OK : GTA_ERR_CUDA;
     }
     auto kern = sm100_linear_kernel<kProject, true>;
@@ -455,9 +469,13 @@ gta_status_t launch_linear(const LinArgs& a, const void* a_ptr, const void* w_pt
         cached_pairs = n;
     }
     const int G = a.n_units < cached_pairs ? a.n_units : cached_pairs;
+    LinArgs a2 = a;
+    a2.q = a.n_units / G;
+    a2.r = a.n_units % G;
+    a2.split_tail = (a.block == 256 && a.n_cols % 256 == 0 && 2 * a2.r <= G) ? 1 : 0;
     cfg.gridDim = dim3(2 * G);
     cfg.numAttrs = 2;
-    if (cudaLaunchKernelEx(&cfg, kern, tm_a, tm_w, a, status_word) != cudaSuccess) return GTA_ERR_CUDA;
+    if (cudaLaunchKernelEx(&cfg, kern, tm_a, tm_w, a2, status_word) != cudaSuccess) return GTA_ERR_CUDA;
     return cudaGetLastError() == cudaSuccess ? GTA_OK : GTA_ERR_CUDA;
 }
 
