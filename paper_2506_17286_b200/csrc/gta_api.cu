@@ -66,6 +66,21 @@ static gta_status_t append_impl(const gta_shape_t* shape, void* k_cache, void* c
                                 const void* k_new, const void* c_new, int32_t n_new, int32_t* seq_lens,
                                 int32_t* status_word, void* cuda_stream, const gta::PageMap& pm);
 
+// A block table is usable when it is there, 4-byte aligned, and the pool geometry is positive.
+static bool page_args_ok(const int32_t* block_table, int32_t page_size, int32_t n_pages, int32_t max_pages) {
+    return block_table && aligned(block_table, 4) && page_size > 0 && n_pages > 0 && max_pages > 0 &&
+           (long long)page_size * max_pages <= INT32_MAX;
+}
+
+static gta::PageMap page_map(const int32_t* block_table, int32_t page_size, int32_t n_pages, int32_t max_pages) {
+    gta::PageMap pm;
+    pm.table = block_table;
+    pm.page_size = page_size;
+    pm.max_pages = max_pages;
+    pm.n_pages = n_pages;
+    return pm;
+}
+
 extern "C" {
 
 const char* gta_status_string(gta_status_t status) {
@@ -194,12 +209,6 @@ gta_status_t gta_decode_stages(const gta_shape_t* shape, const void* q, const vo
                        status_word, cuda_stream, stages, gta::PageMap());
 }
 
-// A block table is usable when it is there, 4-byte aligned, and the pool geometry is positive.
-static bool page_args_ok(const int32_t* block_table, int32_t page_size, int32_t n_pages, int32_t max_pages) {
-    return block_table && aligned(block_table, 4) && page_size > 0 && n_pages > 0 && max_pages > 0 &&
-           (long long)page_size * max_pages <= INT32_MAX;
-}
-
 size_t gta_decode_paged_workspace_bytes(const gta_shape_t* shape, int32_t page_size, int32_t max_pages) {
     gta::Dims d;
     if (check_shape(shape, false, &d) != GTA_OK || page_size <= 0 || max_pages <= 0 ||
@@ -215,13 +224,9 @@ gta_status_t gta_decode_paged(const gta_shape_t* shape, const void* q, const voi
                               void* cuda_stream) {
     g_last_launches = 0;
     if (!page_args_ok(block_table, page_size, n_pages, max_pages)) return GTA_ERR_INVALID_ARG;
-    gta::PageMap pm;
-    pm.table = block_table;
-    pm.page_size = page_size;
-    pm.max_pages = max_pages;
-    pm.n_pages = n_pages;
     return decode_impl(shape, q, k_pool, c_pool, seq_lens, page_size * max_pages, x_t, w_p, w_g, out, workspace,
-                       workspace_bytes, status_word, cuda_stream, 7, pm);
+                       workspace_bytes, status_word, cuda_stream, 7,
+                       page_map(block_table, page_size, n_pages, max_pages));
 }
 
 gta_status_t gta_cache_append_paged(const gta_shape_t* shape, void* k_pool, void* c_pool,
@@ -230,13 +235,8 @@ gta_status_t gta_cache_append_paged(const gta_shape_t* shape, void* k_pool, void
                                     int32_t* seq_lens, int32_t* status_word, void* cuda_stream) {
     g_last_launches = 0;
     if (!page_args_ok(block_table, page_size, n_pages, max_pages)) return GTA_ERR_INVALID_ARG;
-    gta::PageMap pm;
-    pm.table = block_table;
-    pm.page_size = page_size;
-    pm.max_pages = max_pages;
-    pm.n_pages = n_pages;
     return append_impl(shape, k_pool, c_pool, page_size * max_pages, k_new, c_new, n_new, seq_lens, status_word,
-                       cuda_stream, pm);
+                       cuda_stream, page_map(block_table, page_size, n_pages, max_pages));
 }
 
 }  // extern "C"
@@ -335,16 +335,10 @@ extern "C" gta_status_t gta_layer_decode_paged(const gta_shape_t* shape, const i
                                                int32_t* seq_lens, void* u, void* workspace, size_t workspace_bytes,
                                                int32_t* status_word, void* cuda_stream) {
     g_last_launches = 0;
-    if (!block_table || !aligned(block_table, 4) || page_size <= 0 || n_pages <= 0 || max_pages <= 0 ||
-        (long long)page_size * max_pages > INT32_MAX)
-        return GTA_ERR_INVALID_ARG;
-    gta::PageMap pm;
-    pm.table = block_table;
-    pm.page_size = page_size;
-    pm.max_pages = max_pages;
-    pm.n_pages = n_pages;
+    if (!page_args_ok(block_table, page_size, n_pages, max_pages)) return GTA_ERR_INVALID_ARG;
     return layer_decode_impl(shape, page_size * max_pages, rope_base, x_t, w_qkc, w_p, w_g, w_o, k_pool, c_pool,
-                             seq_lens, u, workspace, workspace_bytes, status_word, cuda_stream, pm);
+                             seq_lens, u, workspace, workspace_bytes, status_word, cuda_stream,
+                             page_map(block_table, page_size, n_pages, max_pages));
 }
 
 static gta_status_t layer_decode_impl(const gta_shape_t* shape, int32_t S_cap, float rope_base, const void* x_t,
