@@ -129,7 +129,9 @@ GTA_API gta_status_t gta_prefill_chunk(const gta_shape_t *shape, int32_t kv_len,
  *            seq_lens[b] may hold anything (uninitialised memory, NaN bit patterns)
  *   w_p, w_g as in gta_prefill;  out [B, n_h, d_h]
  *   workspace: at least gta_decode_workspace_bytes(shape, S_cap) bytes, 256-byte aligned
- *     (split-KV partial results and gate partial sums).
+ *     (split-KV partial results and gate partial sums).  The size follows the SM count of the
+ *     device that is current when the function is asked, so ask with the device the call
+ *     will run on (this holds for every *_workspace_bytes function of the decode family).
  * Needs d_h and d_l multiples of 8 (bf16) / 4 (fp32) so that rows are 16-byte vectors,
  * d_h <= 256, d_l <= 2048.  bf16 fast path (TMA-streamed caches, tensor-core decoder) when
  * d_h = 64 or 128, d_l = 128, 256, 512 or 1024, n_q <= 8, n_k = 1, 2, 4 or 8, H a
@@ -287,8 +289,11 @@ GTA_API gta_status_t gta_layer_decode_paged(const gta_shape_t *shape, const int3
  *   - A problem whose gta_decode_workspace_bytes() exceeds GTA_STATIC_SCRATCH_BYTES is refused
  *     with GTA_ERR_STATIC_SCRATCH before anything is launched (for the bf16 kernels the need
  *     grows with batch * n_q * d_l, not with the context length).
- *   - The first call on each device looks up the array's device address (once, with that
- *     device current); make that first call outside any stream capture.
+ *   - Arguments are checked exactly as gta_decode checks them (same order, same codes; an
+ *     empty batch returns GTA_OK after those checks), then the size, then the device.
+ *   - The first call on each device that gets past those checks looks up the array's device
+ *     address (once, with that device current); make that first call outside any stream
+ *     capture.
  *   - All calls on a device share the one array and find in it whatever the previous call left;
  *     the kernels write every word before they read it, so nothing needs clearing.  Two calls
  *     that may run on the GPU at the same time (different streams, no ordering) race on it:

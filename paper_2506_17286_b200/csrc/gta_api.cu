@@ -384,14 +384,14 @@ static gta_status_t layer_decode_impl(const gta_shape_t* shape, int32_t S_cap, f
     return GTA_OK;
 }
 
-static gta_status_t decode_impl(const gta_shape_t* shape, const void* q, const void* k_cache, const void* c_cache,
-                                const int32_t* seq_lens, int32_t S_cap, const void* x_t, const void* w_p,
-                                const void* w_g, void* out, void* workspace, size_t workspace_bytes,
-                                int32_t* status_word, void* cuda_stream, int32_t stages, const gta::PageMap& pm) {
-    g_last_launches = 0;
-    if (stages < 1 || stages > 7) return GTA_ERR_INVALID_ARG;
-    gta::Dims d;
-    gta_status_t st = check_shape(shape, false, &d);
+// Host-side checks of a decode call that need no workspace and no device: the shape, the pointers
+// and their alignment, the limits of the kernels.  *empty is set when the batch is empty (nothing to do).
+gta_status_t gta::decode_check_args(const gta_shape_t* shape, const void* q, const void* k_cache, const void* c_cache,
+                                    const int32_t* seq_lens, int32_t S_cap, const void* x_t, const void* w_p,
+                                    const void* w_g, const void* out, const int32_t* status_word, gta::Dims* d,
+                                    bool* empty) {
+    *empty = false;
+    gta_status_t st = check_shape(shape, false, d);
     if (st != GTA_OK) return st;
     if (S_cap < 0) return GTA_ERR_INVALID_ARG;
     if (!q || !seq_lens || !x_t || !w_p || !w_g || !out) return GTA_ERR_INVALID_ARG;
@@ -401,8 +401,25 @@ static gta_status_t decode_impl(const gta_shape_t* shape, const void* q, const v
         !aligned(status_word, 4))
         return GTA_ERR_INVALID_ARG;
     // one latent row is spread over at most 256 threads, 16 bytes each
-    if ((size_t)d.d_l * elem_size(shape->dtype) > 4096) return GTA_ERR_UNSUPPORTED;
-    if (d.B == 0) return GTA_OK;
+    if ((size_t)d->d_l * elem_size(shape->dtype) > 4096) return GTA_ERR_UNSUPPORTED;
+    *empty = d->B == 0;
+    return GTA_OK;
+}
+
+gta_status_t gta::check_current_device() { return check_device(); }
+
+static gta_status_t decode_impl(const gta_shape_t* shape, const void* q, const void* k_cache, const void* c_cache,
+                                const int32_t* seq_lens, int32_t S_cap, const void* x_t, const void* w_p,
+                                const void* w_g, void* out, void* workspace, size_t workspace_bytes,
+                                int32_t* status_word, void* cuda_stream, int32_t stages, const gta::PageMap& pm) {
+    g_last_launches = 0;
+    if (stages < 1 || stages > 7) return GTA_ERR_INVALID_ARG;
+    gta::Dims d;
+    bool empty = false;
+    gta_status_t st = gta::decode_check_args(shape, q, k_cache, c_cache, seq_lens, S_cap, x_t, w_p, w_g, out,
+                                             status_word, &d, &empty);
+    if (st != GTA_OK) return st;
+    if (empty) return GTA_OK;
     if (!workspace || !aligned(workspace, 256) ||
         workspace_bytes < gta::decode_workspace_bytes(d, shape->dtype, S_cap, pm.table ? pm.page_size : 0))
         return GTA_ERR_WORKSPACE;

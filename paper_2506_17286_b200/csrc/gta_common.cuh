@@ -98,6 +98,14 @@ cudaError_t launch_decode_fast(const Dims& d, const void* q, const void* k_cache
                                const void* w_g, void* out, void* workspace, int32_t* status_word,
                                cudaStream_t stream, int stages, int* launches, const PageMap& pm = PageMap());
 
+// Host-side argument checks of a decode call (everything but the workspace and the device), shared by
+// gta_decode and gta_decode_static so that both report the same errors; *empty: the batch is empty.
+gta_status_t decode_check_args(const gta_shape_t* shape, const void* q, const void* k_cache, const void* c_cache,
+                               const int32_t* seq_lens, int32_t S_cap, const void* x_t, const void* w_p,
+                               const void* w_g, const void* out, const int32_t* status_word, Dims* d, bool* empty);
+// GTA_OK when the current device is one the kernels are built for, GTA_ERR_UNSUPPORTED otherwise.
+gta_status_t check_current_device();
+
 cudaError_t launch_cache_append(const Dims& d, int elem_size, void* k_cache, void* c_cache, int S_cap,
                                 const void* k_new, const void* c_new, int n_new, int32_t* seq_lens,
                                 int32_t* status_word, cudaStream_t stream, int* launches,

@@ -54,15 +54,25 @@ bool decode_fast_supported(const Dims& d, int dtype, int page_size) {
     return tok_bytes * 16 <= kStreamStageBytes;
 }
 
+// SM count of the CURRENT device (the grid, the slot count and hence the workspace size follow it),
+// looked up once per device ordinal and thread; 148 when there is no device to ask (a host without GPUs).
 static int sm_count() {
-    static int n = [] {
-        int dev = 0, v = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess ||
-            cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v <= 0)
+    static thread_local int cached_dev = -1, cached_n = 148;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) {
+        cudaGetLastError();
+        return 148;
+    }
+    if (dev != cached_dev) {
+        int v = 0;
+        if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v <= 0) {
+            cudaGetLastError();
             v = 148;
-        return v;
-    }();
-    return n;
+        }
+        cached_dev = dev;
+        cached_n = v;
+    }
+    return cached_n;
 }
 
 static FastPlan make_fast_plan(const Dims& d) {

@@ -45,16 +45,21 @@ extern "C" gta_status_t gta_decode_static(const gta_shape_t* shape, const void* 
                                           const void* c_cache, const int32_t* seq_lens, int32_t S_cap,
                                           const void* x_t, const void* w_p, const void* w_g, void* out,
                                           int32_t* status_word, void* cuda_stream) {
-    if (!shape) return GTA_ERR_INVALID_ARG;
-    if (shape->batch == 0) return GTA_OK;
-    // Size check first, on the host, before any CUDA call: a problem that does not fit the
-    // built-in array is refused, never truncated.
-    const size_t need = gta_decode_workspace_bytes(shape, S_cap);
-    if (need == 0) return GTA_ERR_INVALID_ARG;   // the shape itself is invalid
-    if (need > (size_t)GTA_STATIC_SCRATCH_BYTES) return GTA_ERR_STATIC_SCRATCH;
-    void* scratch = nullptr;
-    gta_status_t st = scratch_address(&scratch);
+    // The same host-side checks as gta_decode, in the same order, so that both calls answer a bad
+    // argument alike; nothing of CUDA has been touched yet.
+    gta::Dims d;
+    bool empty = false;
+    gta_status_t st = gta::decode_check_args(shape, q, k_cache, c_cache, seq_lens, S_cap, x_t, w_p, w_g, out,
+                                             status_word, &d, &empty);
     if (st != GTA_OK) return st;
+    if (empty) return GTA_OK;
+    // Size check, still on the host: a problem that does not fit the built-in array is refused,
+    // never truncated.
+    if (gta_decode_workspace_bytes(shape, S_cap) > (size_t)GTA_STATIC_SCRATCH_BYTES) return GTA_ERR_STATIC_SCRATCH;
+    if ((st = gta::check_current_device()) != GTA_OK) return st;
+    // Only a call that will launch looks the array up (the first one on a device loads it).
+    void* scratch = nullptr;
+    if ((st = scratch_address(&scratch)) != GTA_OK) return st;
     // Same kernels as gta_decode; they write every scratch word before reading it, so nothing in
     // the array has to be cleared between calls.
     return gta_decode(shape, q, k_cache, c_cache, seq_lens, S_cap, x_t, w_p, w_g, out, scratch,

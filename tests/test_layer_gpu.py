@@ -101,6 +101,30 @@ def test_layer_prefill_full_size_sampled_positions(B, oracle, name):
     _layer_case(B, oracle, w, sample=_sample_positions(w.seq))
 
 
+def _unrounded_case(B, oracle, w, sample=None):
+    """u of gta_layer_prefill against the layer oracle with NO rounding anywhere (storage = float64): the
+    definition of App. B.1.1 itself, whatever the kernels keep between their steps."""
+    t = I.layer_inputs(w, device="cuda")
+    u, _, _ = _run_layer(B, w, t, [w.seq], w.seq + 8, 10000.0)
+    tc = {n: v.cpu() for n, v in t.items()}
+    want = oracle.layer_prefill(oracle_shape(w), tc["x"], tc["w_qkc"], tc["w_p"], tc["w_g"], tc["w_o"], rows=sample,
+                                storage=oracle.F64)
+    got = u if sample is None else u[:, torch.as_tensor(sample, device="cuda")]
+    rel, mx = assert_close(got, want["u"], torch.bfloat16, w.name + " (unrounded oracle)")
+    print(f"\n{w.name}: u vs unrounded fp64 layer: rel-L2 {rel:.3e} max-abs {mx:.3e}")
+
+
+@pytest.mark.parametrize("case", LAYERS, ids=[c[0] for c in LAYERS])
+def test_layer_prefill_against_the_unrounded_definition_small(B, oracle, case):
+    name, nb, N, H, n_h, n_q, n_k, n_c, d_h, d_l, _ = case
+    _unrounded_case(B, oracle, I.Workload(name, "prefill", "bf16", nb, N, H, n_h, n_q, n_k, n_c, d_h, d_l, seed=74))
+
+
+def test_layer_prefill_against_the_unrounded_definition_c2_sampled(B, oracle):
+    w = I.CONFIGS["c2_prefill_bf16"]
+    _unrounded_case(B, oracle, w, sample=_sample_positions(w.seq))
+
+
 LAYER_STEPS = [
     # name, H, n_h, n_q, n_k, n_c, d_h, d_l, lens (tokens already cached per sequence)
     ("c3_shape_small", 512, 8, 4, 4, 1, 128, 512, [1, 63, 64, 200, 0]),

@@ -442,3 +442,26 @@ def test_layer_is_the_operator_between_its_projections(oracle):
     assert np.array_equal(r["c"][:, 0], oracle.round_to_storage(x @ w_qkc[:, 12:], BF16))
     # position 0 is not rotated
     assert np.array_equal(r["k"][:, 0, 0], oracle.round_to_storage(x[:, 0] @ w_qkc[:, 8:12], BF16))
+
+
+def test_layer_widens_bf16_tensors_exactly(oracle):
+    """The layer oracle fed bf16 torch tensors (what the GPU tests hand it) gives bit for bit what it gives
+    for the same values as float64 arrays and as fp32 tensors; the widening is also checked against values
+    written out by hand (2^-7 steps around 1, a subnormal-range number, negative zero)."""
+    import torch
+    s = Shape(2, 6, 16, 4, 2, 1, 1, 4, 8, 1)
+    t = dict(x=_rand(s.batch, s.seq, s.d_model), w_qkc=_rand(s.d_model, 2 * 4 + 4 + 8, scale=0.25),
+             w_p=_rand(s.n_heads, s.d_l, s.d_h, scale=0.3), w_g=_rand(s.d_model, s.n_heads * s.d_h, scale=0.25),
+             w_o=_rand(s.n_heads * s.d_h, s.d_model, scale=0.25))
+    tb = {k: torch.from_numpy(v).to(torch.bfloat16) for k, v in t.items()}
+    for storage in (1, 2):      # rounded at the stored tensors, and not rounded at all
+        r_bf = oracle.layer_prefill(s, **tb, storage=storage)
+        r_f32 = oracle.layer_prefill(s, **{k: v.float() for k, v in tb.items()}, storage=storage)
+        r_f64 = oracle.layer_prefill(s, **{k: v.double().numpy() for k, v in tb.items()}, storage=storage)
+        for name in ("u", "q", "k", "c", "o"):
+            assert np.array_equal(r_bf[name], r_f64[name]) and np.array_equal(r_f32[name], r_f64[name]), name
+    bits = torch.from_numpy(np.array([0x3F80, 0x3F81, 0xBF81, 0x0001, 0x8000, 0x4049], dtype=np.uint16)
+                            .view(np.int16)).view(torch.bfloat16)
+    want = np.array([1.0, 1.0 + 2.0 ** -7, -(1.0 + 2.0 ** -7), 2.0 ** -133, -0.0, 3.140625])
+    got = oracle._to_f64(bits)
+    assert np.array_equal(got, want) and np.signbit(got[4])
