@@ -323,3 +323,68 @@ def cache_elems(shape: Shape) -> float:
     """(n_k d_h + n_c d_l) N — Table 3, GTA row, 'KV Cache per Layer' column."""
     cs = shape.c()
     return float(lib().gta_oracle_cache_elems(ctypes.byref(cs)))
+
+
+# ----------------------------------------------------------------------------------------------
+# Comparison operators of the paper: grouped-query attention (App. B.3 "GQA", definition) and, as its
+# special case with one key / value head per query head, multi-head attention (Sec. 3.1).  Plain numpy in
+# float64, one head and one batch entry at a time, straight from the definition.
+def _kv_head(i: int, n_heads: int, n_kv: int, head_map: str) -> int:
+    """Key / value head of query head i.  "mod": i mod n_kv, the map App. B.3 prints; "blocks": contiguous
+    blocks of n_heads / n_kv query heads per key / value head (the same reading as for the maps of GTA).
+    The two differ by a renumbering of the query heads only."""
+    assert n_heads % n_kv == 0 and head_map in ("mod", "blocks")
+    return i % n_kv if head_map == "mod" else i // (n_heads // n_kv)
+
+
+def gqa_prefill(q, k, v, causal: bool = True, scale: float = 0.0, head_map: str = "blocks", rows=None):
+    """o[b, i, t] = sum_{j <= t} Softmax_j(q[b, i, t] . k[b, kv(i), j] * scale) v[b, kv(i), j]   (App. B.3, GQA,
+    attention equation; scale 0 means 1 / sqrt(d_h)).  q [B, n_h, N, d_h]; k, v [B, n_kv, N, d_h];
+    returns float64 [B, n_h, N or len(rows), d_h] (head-major)."""
+    q, k, v = _to_f64(q), _to_f64(k), _to_f64(v)
+    B, n_h, N, d_h = q.shape
+    n_kv = k.shape[1]
+    assert k.shape == (B, n_kv, N, d_h) and v.shape == (B, n_kv, N, d_h)
+    sc = scale if scale > 0 else 1.0 / np.sqrt(d_h)
+    ts = list(range(N)) if rows is None else list(rows)
+    out = np.zeros((B, n_h, len(ts), d_h))
+    for b in range(B):
+        for i in range(n_h):
+            j = _kv_head(i, n_h, n_kv, head_map)
+            for r, t in enumerate(ts):
+                last = t if causal else N - 1
+                s = (k[b, j, :last + 1] @ q[b, i, t]) * sc
+                p = np.exp(s - s.max())
+                out[b, i, r] = (p / p.sum()) @ v[b, j, :last + 1]
+    return out
+
+
+def gqa_decode(q, k_cache, v_cache, seq_lens, scale: float = 0.0, head_map: str = "blocks"):
+    """One decode step of GQA (App. B.3, decode): the new token's query heads q [B, n_h, d_h] attend the
+    seq_lens[b] cached keys / values (the new token's own included); an empty sequence gives zeros.
+    k_cache, v_cache [B, n_kv, S_cap, d_h]; returns float64 [B, n_h, d_h]."""
+    q, k_cache, v_cache = _to_f64(q), _to_f64(k_cache), _to_f64(v_cache)
+    B, n_h, d_h = q.shape
+    n_kv = k_cache.shape[1]
+    sc = scale if scale > 0 else 1.0 / np.sqrt(d_h)
+    out = np.zeros((B, n_h, d_h))
+    for b in range(B):
+        n = int(seq_lens[b])
+        if n <= 0:
+            continue
+        for i in range(n_h):
+            j = _kv_head(i, n_h, n_kv, head_map)
+            s = (k_cache[b, j, :n] @ q[b, i]) * sc
+            p = np.exp(s - s.max())
+            out[b, i] = (p / p.sum()) @ v_cache[b, j, :n]
+    return out
+
+
+def gqa_attention_cost(n_heads: int, d_h: int, n: int) -> float:
+    """2 n_h d_h N^2 — Table 3, GQA row, 'Attention' column (App. B.3 prefill)."""
+    return 2.0 * n_heads * d_h * float(n) * float(n)
+
+
+def gqa_cache_elems(n_kv: int, d_h: int, n: int) -> float:
+    """2 n_k d_h N — Table 3, GQA row, 'KV Cache per Layer' column (App. B.3 decode)."""
+    return 2.0 * n_kv * d_h * float(n)

@@ -1,4 +1,4 @@
-// tcgen05 / TMA (sm_100a) prefill path for bf16, d_h = 128.
+// tcgen05 / TMA (sm_100a) prefill path for bf16, d_h = 64 or 128.
 //
 //   sm100_attention_kernel : shared attention map per query group, online softmax, latent P C
 //       (Sec. 3.3, reformulated equation; causal sum of App. B.1.1) -> normalised L (bf16).
@@ -25,19 +25,31 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
 // per 256 query rows and the ring is three key tiles deep.  (The 128 x d_l fp32 output does not fit
 // the 512 TMEM columns next to the score tiles, so d_l is cut in slices of 256 and each slice item
 // recomputes the scores.)  Persistent: a pair walks a static list of items, heaviest (latest)
-// query tiles first, dealt to the pairs in snake order.  Per 128-key tile j:
-//   S_j = Q K_j^T            tcgen05.mma M = 256, smem x smem -> TMEM (two S buffers, ping-pong)
-//   P_j = exp2(S_j c - m)    512 softmax threads per CTA, four per row (32 keys each, row maximum
-//                            exchanged through shared memory); P_j (bf16) overwrites S_j in TMEM
-//   O  += P_j C_j            tcgen05.mma M = 256, TMEM x smem (C is the MN-major B operand) -> TMEM
-// The running maximum is only raised when it grows by more than 2^8 (the accumulators stay in
-// range and O needs rescaling on few tiles).  At the end of an item the softmax threads only hand
-// their row sums over: four epilogue warps (one per TMEM lane quarter) divide O by the row sum,
-// stage it in shared memory as bf16 and write it to L[B, n_q, N, d_l] with TMA tensor stores
-// (whole 128-byte lines, clipped at the sequence end), while the softmax threads are already on
-// the first score tile of the next item.  The ring and the score pipeline run on across items.  The lower
-// query tile of a pair sees one fully masked key tile per item (its probabilities are zero).
-constexpr int kAttnThreads = 64 + 512 + 128;   // TMA warp, MMA warp, 16 softmax warps, 4 epilogue warps
+// query tiles first, dealt to the pairs in snake order.
+//
+// The scores are produced and consumed in SUB-TILES of 64 keys (32 of each CTA's 64 keys of a ring
+// tile), four of which are in flight, each in its own 64-column TMEM buffer with its own group of
+// 128 softmax threads (a query row per thread).  Per sub-tile u (buffer and group u mod 4):
+//   S_u = Q K_u^T            tcgen05.mma M = 256, N = 64, smem x smem -> TMEM
+//   P_u = exp2(S_u c - m)    the group's threads; P_u (bf16) overwrites S_u in TMEM
+//   O  += P_u C_u            tcgen05.mma M = 256, K = 64, TMEM x smem (C is the MN-major B operand)
+// With four sub-tiles in flight the tensor pipe's own chain for a buffer (sum of sub-tile u, scores of
+// sub-tile u + 4 into the buffer it frees, two barrier hand-offs) and the softmax of a sub-tile both
+// hide behind the work on the other three; the four softmax warps of an SM sub-partition sit at
+// different points of their sub-tiles, which keeps its issue slots and its exponential unit busy.
+// The running maximum of a row is a chain over the sub-tiles: the thread of sub-tile u publishes it
+// in shared memory as soon as it has the maximum of its own sub-tile (before its exponentials) and
+// the thread of sub-tile u + 1 (the next group) picks it up there.  It is only raised when it grows
+// by more than 2^8 (the accumulators stay in range and O needs rescaling on few sub-tiles).  At the
+// end of an item the softmax threads only hand their (maximum, row sum) pairs over: four epilogue
+// warps (one per TMEM lane quarter) combine the groups' sums, divide O by the row sum, stage it in
+// shared memory as bf16 and write it to L[B, n_q, N, d_l] with TMA tensor stores (whole 128-byte
+// lines, clipped at the sequence end), while the softmax threads are already on the next item.  The
+// ring and the score pipeline run on across items.  The lower query tile of a pair sees one fully
+// masked key tile per item (its probabilities are zero).
+constexpr int kAttnGroups = 4;                     // softmax groups = score buffers = sub-tiles in flight
+constexpr int kSubKeys = 64;                       // keys per sub-tile (32 from each CTA of the pair)
+constexpr int kAttnThreads = 128 * kAttnGroups + 128 + 96;   // warps 0-15 softmax, 16-19 epilogue, 20 TMA, 21 / 22 MMA issue (sums / scores)
 constexpr int kAttnStages = 3;
 constexpr int kKeyTile = 128;
 constexpr int kSlice = 256;      // widest latent slice of an item (template parameter SLICE: 256 or 128)
@@ -51,11 +63,11 @@ constexpr uint32_t kAttnRingOff = kQBytes;
 // tile of item n + 2.  So the next item's Q is loaded long before the current item ends.
 constexpr uint32_t kAttnOutOff = kAttnRingOff + kAttnStages * kAttnStageBytes;   // the second buffer (the first is at 0)
 constexpr uint32_t kAttnOutBoxBytes = 128 * 64 * 2;
-constexpr uint32_t kAttnXchgOff = kAttnOutOff + 2 * kAttnOutBoxBytes;   // 2 KB, per lane quarter: bf16 [2][4][32] or float [4][32]
-constexpr uint32_t kAttnSumOff = kAttnXchgOff + 2 * 4 * 2 * 32 * 4;      // 4 KB: float [2 items][4 quarters][4 parts][32] row sums
-constexpr uint32_t kAttnBarOff = kAttnSumOff + 2 * 4 * 4 * 32 * 4;
+constexpr uint32_t kAttnXchgOff = kAttnOutOff + 2 * kAttnOutBoxBytes;   // 2 KB: float [4 groups][128 rows] running maxima
+constexpr uint32_t kAttnSumOff = kAttnXchgOff + kAttnGroups * 128 * 4;  // 8 KB: float2 [2 items][4 groups][128] (max, sum)
+constexpr uint32_t kAttnBarOff = kAttnSumOff + 2 * kAttnGroups * 128 * 8;
 constexpr uint32_t kAttnAlignSlack = 1024;  // checked in the kernel
-constexpr uint32_t kAttnSmemTotal = kAttnBarOff + 256 + kAttnAlignSlack;
+constexpr uint32_t kAttnSmemTotal = kAttnBarOff + 512 + kAttnAlignSlack;
 static_assert(kAttnSmemTotal <= 232448, "attention kernel shared memory exceeds the per-CTA limit");
 
 __device__ __forceinline__ float fast_exp2(float x) {
@@ -63,33 +75,45 @@ __device__ __forceinline__ float fast_exp2(float x) {
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
-// 2^x for a pair of values on the FMA pipe (x <= ~8; anything below -126 gives ~1e-38): round to the
-// nearest integer with the 1.5 * 2^23 trick, cubic for the fraction in [-1/2, 1/2] (relative error
-// < 8e-5, well inside the bf16 rounding of P), exponent patched in with integer arithmetic.  Used for
-// some of the pairs so that the MUFU unit, which paces the exponential phase, carries fewer of them.
-__device__ __forceinline__ void poly_exp2_pair(uint64_t x2, float& p0, float& p1) {
-    float x0, x1;
-    ptx::f32x2_split(x2, x0, x1);
-    x2 = ptx::f32x2(fmaxf(x0, -126.f), fmaxf(x1, -126.f));
-    const uint64_t t2 = ptx::add2(x2, ptx::f32x2(12582912.f, 12582912.f));
-    const uint64_t u2 = ptx::add2(t2, ptx::f32x2(-12582912.f, -12582912.f));
-    const uint64_t f2 = ptx::fma2(u2, ptx::f32x2(-1.f, -1.f), x2);
-    uint64_t q2 = ptx::fma2(f2, ptx::f32x2(0.05517165f, 0.05517165f), ptx::f32x2(0.24261113f, 0.24261113f));
-    q2 = ptx::fma2(f2, q2, ptx::f32x2(0.69326097f, 0.69326097f));
-    q2 = ptx::fma2(f2, q2, ptx::f32x2(0.99992806f, 0.99992806f));
-    float q0, q1, t0, t1;
-    ptx::f32x2_split(q2, q0, q1);
-    ptx::f32x2_split(t2, t0, t1);
-    p0 = __int_as_float(__float_as_int(q0) + (__float_as_int(t0) << 23));
-    p1 = __int_as_float(__float_as_int(q1) + (__float_as_int(t1) << 23));
-}
-// which of every eight pairs of exponentials run on the FMA pipe instead of the MUFU unit
-__device__ constexpr bool kPolyPair[8] = {false, false, true, false, false, true, false, true};
 __device__ __forceinline__ void epilogue_sync() {   // the four epilogue warps
     asm volatile("bar.sync 5, 128;" ::: "memory");
 }
-__device__ __forceinline__ void quarter_sync(int quarter) {   // the four softmax warps of a TMEM lane quarter
-    asm volatile("bar.sync %0, 128;" ::"r"(quarter + 1) : "memory");
+// The four warps of a softmax group (ids 1 .. 4) or the epilogue warps (id 6): one of them polls a
+// barrier of the tensor pipe, the others sleep here at no cost in issue slots until it has seen it.
+__device__ __forceinline__ void wait_group_sync(int id) {
+    asm volatile("bar.sync %0, 128;" ::"r"(id) : "memory");
+}
+// Scores of keys past `last_key` (past the sequence end, or -- causal -- after the query) become -inf.
+// Only called on boundary tiles (a warp-level branch around it costs the other tiles nothing).
+__device__ __forceinline__ void mask_chunk(uint32_t (&r)[32], int key0, int last_key) {
+#pragma unroll
+    for (int e = 0; e < 32; ++e)
+        if (key0 + e > last_key) r[e] = 0xff800000u;     // -inf
+}
+// exp2(s c - m) of 32 scores of one row (raw TMEM words), packed to bf16 pairs; their sum is added to sum2
+__device__ __forceinline__ void softmax_chunk(const uint32_t (&r)[32], uint64_t cs2, uint64_t nm2, uint64_t (&sum2)[2],
+                                              uint32_t (&packed)[16]) {
+#pragma unroll
+    for (int e = 0; e < 16; ++e) {
+        const uint64_t x2 = ptx::fma2(ptx::f32x2(__uint_as_float(r[2 * e]), __uint_as_float(r[2 * e + 1])), cs2, nm2);
+        // (a polynomial on the FMA pipe for part of the pairs, to spare the exponential unit, was measured
+        // slower here: the unit is under half busy, the issue slots are what is short)
+        float x0, x1;
+        ptx::f32x2_split(x2, x0, x1);
+        const float p0 = fast_exp2(x0), p1 = fast_exp2(x1);
+        sum2[e & 1] = ptx::add2(sum2[e & 1], ptx::f32x2(p0, p1));
+        packed[e] = pack_bf16x2(p0, p1);
+    }
+}
+// maximum of 32 scores of one row (raw TMEM words) and mx
+__device__ __forceinline__ float max_chunk(const uint32_t (&r)[32], float mx) {
+    float a = mx, b = -INFINITY;
+#pragma unroll
+    for (int e = 0; e < 32; e += 4) {
+        a = ptx::max3(a, __uint_as_float(r[e]), __uint_as_float(r[e + 1]));
+        b = ptx::max3(b, __uint_as_float(r[e + 2]), __uint_as_float(r[e + 3]));
+    }
+    return fmaxf(a, b);
 }
 struct AttnItem {
     int b, g, slice, qp, n_tiles;   // qp: pair of query tiles (2 qp, 2 qp + 1)
@@ -128,13 +152,14 @@ sm100_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     uint64_t* stage_free = bars + 1;    // this CTA; its epilogue's stores have read the buffer (one thread arrives)
     uint64_t* full = bars + 2;          // [4] leader CTA; both producers arrive
     uint64_t* empty = bars + 6;         // [4] both CTAs (multicast commit)
-    uint64_t* s_full = bars + 10;       // [2] both CTAs (multicast commit)
-    uint64_t* p_full = bars + 12;       // [2] leader CTA; 32 softmax warps arrive
-    uint64_t* o_done = bars + 14;       // both CTAs (multicast commit)
-    uint64_t* o_free = bars + 15;       // leader CTA; 8 epilogue warps arrive
-    uint64_t* epi_ready = bars + 16;    // this CTA; its 16 softmax warps arrive (row sums of an item are in place)
-    uint64_t* o_item = bars + 17;       // both CTAs (multicast commit): the last sum of an item is complete
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 18);
+    uint64_t* s_full = bars + 10;       // [4] both CTAs (multicast commit): scores of a sub-tile are in its buffer
+    uint64_t* p_full = bars + 14;       // [4] leader CTA; the 4 warps of a softmax group of both CTAs arrive
+    uint64_t* o_done = bars + 18;       // [4] both CTAs (multicast commit): the sum of a sub-tile is complete
+    uint64_t* o_free = bars + 22;       // leader CTA; 8 epilogue warps arrive
+    uint64_t* epi_ready = bars + 23;    // this CTA; its 16 softmax warps arrive (maxima and row sums of an item are in place)
+    uint64_t* o_item = bars + 24;       // both CTAs (multicast commit): the last sum of an item is complete
+    uint64_t* chain = bars + 25;        // [4 groups][4 quarters] this CTA; one warp arrives: its rows' running maxima are published
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 41);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
     volatile int* drain_flag = abort_flag + 1;
 
@@ -145,7 +170,10 @@ sm100_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     constexpr uint32_t kQLoadBytes = 128 * DH * 2;                 // this CTA's query tile
     constexpr uint32_t kKLoadBytes = (kKeyTile / 2) * DH * 2;      // this CTA's 64 keys
     constexpr uint32_t kCLoadBytes = kKeyTile * (SLICE / 2) * 2;   // this CTA's SLICE / 2 latent columns
-    const int n_slices = d.d_l / SLICE;
+    // A latent of only SLICE / 2 columns (the comparison operators with d_h = 64 values): both CTAs of the
+    // pair stage the same columns, so the second half of O repeats the first and is not stored.
+    const bool narrow = d.d_l * 2 == SLICE;
+    const int n_slices = narrow ? 1 : d.d_l / SLICE;
     const int n_qt = (d.N + 127) / 128, n_qp = (n_qt + 1) / 2;
     const int n_kt = (d.Nk + 127) / 128;          // key tiles
     const long long total = bad_align ? 0 : (long long)n_qp * n_slices * d.n_q * d.B;
@@ -154,16 +182,18 @@ sm100_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         ptx::mbar_init(q_full, 2);
         ptx::mbar_init(stage_free, 1);
         for (int s = 0; s < kAttnStages; ++s) { ptx::mbar_init(&full[s], 2); ptx::mbar_init(&empty[s], 1); }
-        for (int s = 0; s < 2; ++s) { ptx::mbar_init(&s_full[s], 1); ptx::mbar_init(&p_full[s], 32); }
-        ptx::mbar_init(o_done, 1);
+        for (int s = 0; s < kAttnGroups; ++s) {
+            ptx::mbar_init(&s_full[s], 1); ptx::mbar_init(&p_full[s], 8); ptx::mbar_init(&o_done[s], 1);
+        }
         ptx::mbar_init(o_free, 8);
-        ptx::mbar_init(epi_ready, 16);
+        ptx::mbar_init(epi_ready, 4 * kAttnGroups);
         ptx::mbar_init(o_item, 1);
+        for (int s = 0; s < 4 * kAttnGroups; ++s) ptx::mbar_init(&chain[s], 1);
         *abort_flag = 0;
         *drain_flag = 0;
         ptx::fence_mbar_init();
     }
-    if (warp == 1) ptx::tmem_alloc_pair(tmem_slot, 512);
+    if (warp == 21) ptx::tmem_alloc_pair(tmem_slot, 512);
     ptx::tc_fence_before_sync();
     __syncthreads();
     ptx::cluster_arrive();     // the peer's barriers exist before anything is signalled to them
@@ -179,7 +209,7 @@ sm100_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     const uint32_t tmem_base = *tmem_slot;
     const uint32_t tmem_o = tmem_base + 256;
 
-    if (warp == 0) {
+    if (warp == 20) {
         if (ptx::elect_one()) {
             ptx::prefetch_tensormap(&tm_q); ptx::prefetch_tensormap(&tm_k); ptx::prefetch_tensormap(&tm_c);
             const uint32_t q_full_leader = ptx::map_to_cta(ptx::smem_addr(q_full), 0);
@@ -200,7 +230,7 @@ sm100_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                 for (int j = 0; j < w.n_tiles; ++j, ++tj) {
                     const int s = tj % kAttnStages;
                     const uint32_t ph = (tj / kAttnStages) & 1;
-                    ok = ptx::mbar_wait(&empty[s], ph ^ 1, abort_flag);
+                    ok = ptx::mbar_wait_backoff(&empty[s], ph ^ 1, abort_flag, 64);   // the ring is three tiles ahead
                     if (!ok) break;
                     uint8_t* k_s = smem + kAttnRingOff + s * kAttnStageBytes;
                     uint8_t* c_s = k_s + kKHalfBytes;
@@ -209,7 +239,7 @@ sm100_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                     const int key0 = j * kKeyTile + (int)rank * 64;         // this CTA's 64 keys of the tile
                     ptx::tma_load_3d_pair(k_s, &tm_k, bar, 0, key0, w.b * d.n_k + kg);
                     if (DH == 128) ptx::tma_load_3d_pair(k_s + 8192, &tm_k, bar, 64, key0, w.b * d.n_k + kg);
-                    const int col0 = w.slice * SLICE + (int)rank * (SLICE / 2);     // this CTA's latent columns
+                    const int col0 = narrow ? 0 : w.slice * SLICE + (int)rank * (SLICE / 2);     // this CTA's latent columns
                     ptx::tma_load_3d_pair(c_s, &tm_c, bar, col0, j * kKeyTile, w.b * d.n_c + cg);
                     if (SLICE == 256)
                         ptx::tma_load_3d_pair(c_s + 16384, &tm_c, bar, col0 + 64, j * kKeyTile, w.b * d.n_c + cg);
@@ -224,189 +254,202 @@ sm100_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                 }
             }
         }
-    } else if (warp == 1) {
+    } else if (warp == 21 || warp == 22) {
+        // Two threads of the leader CTA feed the tensor pipe: one issues the score MMAs (S_u = Q K_u^T), the
+        // other the sums (O += P_u C_u).  A single thread's instruction stream -- waits, descriptors, MMAs,
+        // commits, one instruction every few cycles -- is what paced the pipe when one thread did both.
+        // The two are ordered through barriers only: the scores of sub-tile u + 4 go into the buffer of
+        // sub-tile u once its sum is COMPLETE (o_done), the sum of sub-tile u follows its probabilities
+        // (p_full), which follow its scores (s_full).
         if (rank == 0 && ptx::elect_one()) {
-            constexpr uint32_t idesc_qk = ptx::make_idesc_bf16(256, kKeyTile, 0, 0);   // both K-major
+            constexpr uint32_t idesc_qk = ptx::make_idesc_bf16(256, kSubKeys, 0, 0);   // both K-major
             constexpr uint32_t idesc_pv = ptx::make_idesc_bf16(256, SLICE, 0, 1);      // B = C, MN-major
+            const uint32_t smem_base = ptx::smem_addr(smem);
+            // descriptors differ in the start address only: base + (address >> 4)
+            const uint64_t desc_kmajor = ptx::make_smem_desc(0, 16, 1024);
+            const uint64_t desc_latent = ptx::make_smem_desc(0, 16384, 1024);
             bool ok = true;
-            // S = Q K^T of ring tile tj; `first`: first key tile of its item n
-            auto issue_qk = [&](int tj, int n, bool first) {
-                if (first) ok = ptx::mbar_wait(q_full, n & 1, abort_flag);
-                if (ok) ok = ptx::mbar_wait(&full[tj % kAttnStages], (tj / kAttnStages) & 1, abort_flag);
-                if (!ok) return;
-                ptx::tc_fence_after_sync();
-                const uint32_t q_addr = ptx::smem_addr(smem + ((n & 1) ? kAttnOutOff : 0u));
-                const uint32_t k_addr = ptx::smem_addr(smem + kAttnRingOff + (tj % kAttnStages) * kAttnStageBytes);
-                const uint32_t s_tmem = tmem_base + (tj & 1) * 128;
+            int u = 0;                  // sub-tiles so far over all items: buffer and group u & 3, ring tile u >> 1
+            AttnItem w;
+            for (int n = 0; ok && attn_item(d, n_kt, n_qp, n_slices, total, G, pr, n, &w); ++n) {
+                const int n_sub = 2 * w.n_tiles;
+                if (warp == 22) {
+                    // ---- scores
+                    const uint32_t q_lo = (smem_base + ((n & 1) ? kAttnOutOff : 0u)) >> 4;
+                    for (int j = 0; j < n_sub && ok; ++j, ++u) {
+                        const int tile = u >> 1, stage = tile % kAttnStages;
+                        if (u >= kAttnGroups) ok = ptx::mbar_wait(&o_done[u & 3], ((u - kAttnGroups) >> 2) & 1, abort_flag);
+                        if (ok && j == 0) ok = ptx::mbar_wait(q_full, n & 1, abort_flag);
+                        if (ok && (j & 1) == 0) ok = ptx::mbar_wait(&full[stage], (tile / kAttnStages) & 1, abort_flag);
+                        if (!ok) break;
+                        ptx::tc_fence_after_sync();
+                        // this CTA's keys 32 (j & 1) .. of its 64 keys of the ring tile: 32 rows of 128 bytes further
+                        // on; 32 bytes per k-step inside a 64-column half, the next half 16 KB (Q) / 8 KB (K) on
+                        uint64_t dq = desc_kmajor + q_lo;
+                        uint64_t dk = desc_kmajor + ((smem_base + kAttnRingOff + stage * kAttnStageBytes + (j & 1) * 4096) >> 4);
+                        const uint32_t s_tmem = tmem_base + (u & 3) * kSubKeys;
 #pragma unroll
-                for (int k8 = 0; k8 < DH / 16; ++k8)
-                    ptx::mma_ss_pair(s_tmem, ptx::make_smem_desc(q_addr + (k8 >> 2) * 16384 + (k8 & 3) * 32, 16, 1024),
-                                     ptx::make_smem_desc(k_addr + (k8 >> 2) * 8192 + (k8 & 3) * 32, 16, 1024), idesc_qk,
-                                     k8 ? 1u : 0u);
-                ptx::tc_commit_pair(&s_full[tj & 1], 3);
-            };
-            int tj = 0;
-            AttnItem w, nxt;
-            bool have = attn_item(d, n_kt, n_qp, n_slices, total, G, pr, 0, &w);
-            if (have) issue_qk(0, 0, true);
-            for (int n = 0; have && ok; ++n) {
-                const bool have_next = attn_item(d, n_kt, n_qp, n_slices, total, G, pr, n + 1, &nxt);
-                for (int j = 0; j < w.n_tiles && ok; ++j, ++tj) {
-                    // look ahead: the next score tile goes to the tensor pipe before this tile's P C, so
-                    // the softmax warps never wait for scores.  Across items too, when the next
-                    // item's Q has landed (it normally has: it is loaded into the other buffer well
-                    // before this item ends); otherwise after this item's last P C, below.
-                    bool next_item_early = false;
-                    if (j + 1 < w.n_tiles) {
-                        issue_qk(tj + 1, n, false);
-                    } else if (have_next && ptx::mbar_test_wait(q_full, (n + 1) & 1)) {
-                        issue_qk(tj + 1, n + 1, true);
-                        next_item_early = true;
+                        for (int k8 = 0; k8 < DH / 16; ++k8) {
+                            ptx::mma_ss_pair(s_tmem, dq, dk, idesc_qk, (uint32_t)k8);
+                            const bool wrap = (k8 & 3) == 3;
+                            dq += wrap ? (16384 - 96) >> 4 : 2;
+                            dk += wrap ? (8192 - 96) >> 4 : 2;
+                        }
+                        ptx::tc_commit_pair(&s_full[u & 3], 3);
                     }
-                    if (!ok) break;
-                    ok = ptx::mbar_wait(&p_full[tj & 1], (tj >> 1) & 1, abort_flag);
-                    if (ok && j == 0 && n > 0) ok = ptx::mbar_wait(o_free, (n - 1) & 1, abort_flag);
-                    if (!ok) break;
-                    ptx::tc_fence_after_sync();
-                    const uint32_t c_addr =
-                        ptx::smem_addr(smem + kAttnRingOff + (tj % kAttnStages) * kAttnStageBytes + kKHalfBytes);
-                    const uint32_t p_tmem = tmem_base + (tj & 1) * 128;
+                } else {
+                    // ---- sums
+                    for (int j = 0; j < n_sub && ok; ++j, ++u) {
+                        const int tile = u >> 1, stage = tile % kAttnStages, sub = j & 1;
+                        ok = ptx::mbar_wait(&p_full[u & 3], (u >> 2) & 1, abort_flag);
+                        if (ok && j == 0 && n > 0) ok = ptx::mbar_wait(o_free, (n - 1) & 1, abort_flag);
+                        if (!ok) break;
+                        ptx::tc_fence_after_sync();
+                        // P columns 16 kk .. are the keys 32 sub + 16 (kk & 1) .. of CTA kk >> 1, i.e. rows
+                        // 64 (kk >> 1) + 32 sub + 16 (kk & 1) .. of the 128-key latent tile (2 KB per 16 rows)
+                        uint64_t dc = desc_latent + ((smem_base + kAttnRingOff + stage * kAttnStageBytes + kKHalfBytes + sub * 4096) >> 4);
+                        uint32_t p_tmem = tmem_base + (u & 3) * kSubKeys;
 #pragma unroll
-                    for (int k8 = 0; k8 < 8; ++k8)
-                        ptx::mma_ts_pair(tmem_o, p_tmem + k8 * 8, ptx::make_smem_desc(c_addr + k8 * 2048, 16384, 1024),
-                                         idesc_pv, (j > 0 || k8 > 0) ? 1u : 0u);
-                    ptx::tc_commit_pair(o_done, 3);
-                    if (j + 1 == w.n_tiles) ptx::tc_commit_pair(o_item, 3);   // for the epilogue warps
-                    ptx::tc_commit_pair(&empty[tj % kAttnStages], 3);
-                    if (j + 1 == w.n_tiles && have_next && !next_item_early)
-                        issue_qk(tj + 1, n + 1, true);
+                        for (int kk = 0; kk < 4; ++kk) {
+                            ptx::mma_ts_pair(tmem_o, p_tmem, dc, idesc_pv, (j > 0 || kk > 0) ? 1u : 0u);
+                            p_tmem += 8;
+                            dc += (kk == 1) ? (3 * 2048) >> 4 : 2048 >> 4;
+                        }
+                        ptx::tc_commit_pair(&o_done[u & 3], 3);
+                        if (j + 1 == n_sub) ptx::tc_commit_pair(o_item, 3);   // for the epilogue warps
+                        // both halves of the ring tile are used up (its scores were complete before these sums began)
+                        if (sub == 1) ptx::tc_commit_pair(&empty[stage], 3);
+                    }
                 }
-                w = nxt;
-                have = have_next;
             }
         }
-    } else if (warp < 18) {
-        // 16 softmax warps: four per TMEM lane quarter (warp % 4), each thread 32 of the 128 keys of its
-        // row and 64 of the 256 output columns.  Four warps per scheduler hide the latencies of the
-        // TMEM loads, the exchange and the exponentials behind one another.
+    } else if (warp < 4 * kAttnGroups) {
+        // Four softmax groups of four warps (one per TMEM lane quarter), a query row per thread.  Group g
+        // takes the sub-tiles u with u mod 4 = g (score buffer g).  Per sub-tile: (1) the row maximum of the
+        // 64 scores; (2) the chain: take the running maximum that the previous group's thread of this row
+        // published for the sub-tile before, raise it if this sub-tile exceeds it by more than 2^8, publish
+        // it; (3) the exponentials, 32 keys at a time, P written over S; (4) rarely, O rescaled.  Step (2)
+        // is all that orders the groups.
+        const int wg = warp >> 2;
         const int quarter = warp & 3;
-        const int part = (warp - 2) >> 2;            // which 32 keys of a tile / which 64 output columns
         const int row = quarter * 32 + lane;
         const uint32_t lane_base = ((uint32_t)(quarter * 32) << 16);
         const float c_scale = d.scale * 1.4426950408889634f;
-        const uint32_t p_full_leader[2] = {ptx::map_to_cta(ptx::smem_addr(&p_full[0]), 0),
-                                           ptx::map_to_cta(ptx::smem_addr(&p_full[1]), 0)};
-        __nv_bfloat16* xm = reinterpret_cast<__nv_bfloat16*>(xchg);   // [4 quarters][2][4][32] partial row maxima
-        float* xsum = reinterpret_cast<float*>(smem + kAttnSumOff);
+        const uint32_t p_full_leader = ptx::map_to_cta(ptx::smem_addr(&p_full[wg]), 0);
+        const uint32_t s_tmem = tmem_base + lane_base + wg * kSubKeys;
+        const int wg_prev = (wg + kAttnGroups - 1) & (kAttnGroups - 1);
+        float* m_pub = xchg + wg * 128 + row;                 // written by this thread, read by the next group's
+        const volatile float* m_in = xchg + wg_prev * 128 + row;
+        uint64_t* chain_out = &chain[wg * 4 + quarter];
+        uint64_t* chain_in = &chain[wg_prev * 4 + quarter];
+        float2* xsum = reinterpret_cast<float2*>(smem + kAttnSumOff);
+        const uint64_t cs2 = ptx::f32x2(c_scale, c_scale);
         // A wait that gives up raises the CTA's abort flag, after which every wait returns at once:
-        // these warps then run their loops to the end all the same (on meaningless data), so that
-        // the named barriers below are always reached by all of their threads.
+        // these warps then run their loops to the end all the same (on meaningless data).
         bool ok = true;
-        int tj = 0;
-        AttnItem w;
-        for (int n = 0; attn_item(d, n_kt, n_qp, n_slices, total, G, pr, n, &w); ++n) {
+        int u = 0;                                  // sub-tiles so far, over all items
+        AttnItem w, nxt;
+        bool have = attn_item(d, n_kt, n_qp, n_slices, total, G, pr, 0, &w);
+        for (int n = 0; have; ++n) {
+            const bool have_next = attn_item(d, n_kt, n_qp, n_slices, total, G, pr, n + 1, &nxt);
             const int t = (2 * w.qp + (int)rank) * 128 + row;
-            float m = -INFINITY, l = 0.f;            // m in scaled (log2) units; l = this thread's share of the row sum
-            for (int j = 0; j < w.n_tiles; ++j, ++tj) {
-                ok = __all_sync(0xffffffffu, ptx::mbar_wait(&s_full[tj & 1], (tj >> 1) & 1, abort_flag));
+            const int last_key = d.causal ? min(t + d.Nk - d.N, d.Nk - 1) : d.Nk - 1;
+            const int n_sub = 2 * w.n_tiles;
+            float m_own = -INFINITY, l = 0.f;       // m in scaled (log2) units; l: this group's share of the row sum, relative to m_own
+            for (int j = 0; j < n_sub; ++j, ++u) {
+                if ((u & (kAttnGroups - 1)) != wg) continue;
+                // one warp of the group polls for the scores (on a scheduler of its own: group g's poller is its
+                // warp of lane quarter g), the other three are woken through a named barrier
+                if (quarter == wg) ok = __all_sync(0xffffffffu, ptx::mbar_wait(&s_full[wg], (u >> 2) & 1, abort_flag));
+                wait_group_sync(1 + wg);
                 ptx::tc_fence_after_sync();
-                const uint32_t s_tmem = tmem_base + lane_base + (tj & 1) * 128;
-                float sv[32];
-                {
-                    uint32_t r0[32];
-                    ptx::tmem_ld32(s_tmem + part * 32, r0);
+                // columns 0 .. 31 of the buffer: keys key_a .. of the ring tile's first half (the leader CTA's),
+                // columns 32 .. 63: keys key_b .. of its second half
+                const int key_a = (j >> 1) * kKeyTile + (j & 1) * 32, key_b = key_a + 64;
+                const bool boundary = key_b + 31 > last_key;
+                uint32_t ra[32];
+                // ---- (1) row maximum (the two 32-key halves in a rolled loop, like the exponentials below: the
+                //      warps of a scheduler share a small instruction cache with the thread that issues the MMAs)
+                float mx = -INFINITY;
+#pragma unroll
+                for (int c = 0; c < 2; ++c) {
+                    ptx::tmem_ld32(s_tmem + c * 32, ra);
                     ptx::tmem_wait_ld();
-#pragma unroll
-                    for (int e = 0; e < 32; ++e) sv[e] = __uint_as_float(r0[e]);
+                    if (boundary) mask_chunk(ra, c ? key_b : key_a, last_key);
+                    mx = max_chunk(ra, mx);
                 }
-                // mask: keys past the sequence end, and (causal) keys after the query, on boundary tiles
-                const int key0 = j * kKeyTile + part * 32;
-                const int last_key = d.causal ? min(t + d.Nk - d.N, d.Nk - 1) : d.Nk - 1;
-                if (key0 + 31 > last_key) {
-#pragma unroll
-                    for (int e = 0; e < 32; ++e)
-                        if (key0 + e > last_key) sv[e] = -INFINITY;
+                ptx::tmem_ld32(s_tmem, ra);            // the first 32 scores again for step (3), under the chain
+                const float m_tile = mx * c_scale;     // c_scale > 0
+                // ---- (2) the chain of running maxima (every sub-tile but the very first waits for the one
+                //      before it, every sub-tile but the very last signals the one after it: strict rotation)
+                if (u > 0) ok = __all_sync(0xffffffffu, ptx::mbar_wait(chain_in, ((u - 1) >> 2) & 1, abort_flag));
+                const float m_prev = (j == 0) ? -INFINITY : *m_in;
+                const bool raise = m_tile > m_prev + 8.f;     // also true on the first live sub-tile (m_prev = -inf)
+                const float m = raise ? m_tile : m_prev;
+                *m_pub = m;
+                __syncwarp();
+                if (lane == 0 && (have_next || j + 1 < n_sub)) ptx::mbar_arrive(chain_out);
+                if (m != m_own) {                     // this group's sum follows the maximum (other groups may have raised it)
+                    l *= fast_exp2(m_own - m);        // m_own = -inf: l is 0 and stays 0
+                    m_own = m;
                 }
-                float mx[2] = {ptx::max3(sv[0], sv[1], sv[2]), ptx::max3(sv[3], sv[4], sv[5])};
-#pragma unroll
-                for (int e = 6; e < 30; e += 4) {
-                    mx[0] = ptx::max3(mx[0], sv[e], sv[e + 1]);
-                    mx[1] = ptx::max3(mx[1], sv[e + 2], sv[e + 3]);
-                }
-                const float m_part = ptx::max3(mx[0], mx[1], fmaxf(sv[30], sv[31])) * c_scale;   // c_scale > 0
-                __nv_bfloat16* xs = xm + (quarter * 2 + (tj & 1)) * 128;   // 512 bytes per quarter, shared with xl
-                xs[part * 32 + lane] = __float2bfloat16_ru(m_part);
-                quarter_sync(quarter);
-                const float m_tile = fmaxf(fmaxf(__bfloat162float(xs[lane]), __bfloat162float(xs[32 + lane])),
-                                           fmaxf(__bfloat162float(xs[64 + lane]), __bfloat162float(xs[96 + lane])));
-                float alpha = 1.f;
-                const bool raise = m_tile > m + 8.f;     // also true on the first live tile (m = -inf); same in all four threads
-                if (raise) {
-                    alpha = fast_exp2(m - m_tile);
-                    m = m_tile;
-                }
+                // ---- (3) exponentials, 32 keys at a time (the scores are read from TMEM a second time: keeping
+                //      all 64 in registers across the chain costs more in spills than the second load)
                 const float neg_m = (m == -INFINITY) ? 0.f : -m;   // a fully masked row keeps p = 0
-                const uint64_t cs2 = ptx::f32x2(c_scale, c_scale), nm2 = ptx::f32x2(neg_m, neg_m);
+                const uint64_t nm2 = ptx::f32x2(neg_m, neg_m);
                 uint64_t sum2[2] = {0ull, 0ull};         // two-wide fp32 arithmetic: half the issue slots
                 uint32_t packed[16];
 #pragma unroll
-                for (int e = 0; e < 16; ++e) {
-                    const uint64_t x2 = ptx::fma2(ptx::f32x2(sv[2 * e], sv[2 * e + 1]), cs2, nm2);
-                    float p0, p1;
-                    if (kPolyPair[e & 7]) {
-                        poly_exp2_pair(x2, p0, p1);
-                    } else {
-                        float x0, x1;
-                        ptx::f32x2_split(x2, x0, x1);
-                        p0 = fast_exp2(x0);
-                        p1 = fast_exp2(x1);
-                    }
-                    sum2[e & 1] = ptx::add2(sum2[e & 1], ptx::f32x2(p0, p1));
-                    packed[e] = pack_bf16x2(p0, p1);
+                for (int c = 0; c < 2; ++c) {
+                    ptx::tmem_wait_ld();
+                    if (boundary) mask_chunk(ra, c ? key_b : key_a, last_key);
+                    softmax_chunk(ra, cs2, nm2, sum2, packed);
+                    if (c == 0) ptx::tmem_ld32(s_tmem + 32, ra);
+                    // P_u (bf16 pairs): 32 keys = 16 packed columns of the buffer, columns whose scores this thread
+                    // has already loaded
+                    ptx::tmem_st16(s_tmem + c * 16, packed);
                 }
                 float s0, s1;
                 ptx::f32x2_split(ptx::add2(sum2[0], sum2[1]), s0, s1);
-                l = l * alpha + (s0 + s1);
-                // P_j (bf16 pairs): this thread's 32 keys = packed columns [16 part, 16 part + 16) of S_j
-                // (columns that other threads of the row read as scores: they did so before the exchange)
-                ptx::tmem_st16(s_tmem + part * 16, packed);
-                if (tj > 0) {
-                    // Every completion of o_done is waited for, in order, whether or not O has to be
-                    // rescaled (on the first tile of an item it never is): a parity wait is only
-                    // meaningful one phase at a time.
-                    ok = __all_sync(0xffffffffu, ptx::mbar_wait(o_done, (tj - 1) & 1, abort_flag));
-                    if (j > 0 && __any_sync(0xffffffffu, raise)) {
-                        ptx::tc_fence_after_sync();
+                l += s0 + s1;
+                // ---- (4) O holds the sums of the sub-tiles before this one relative to m_prev: rescale it when
+                //      the maximum was raised.  The sum of sub-tile u - 1 must be complete first; its barrier
+                //      (one per buffer) completes once per four sub-tiles, and when the scores of sub-tile u exist
+                //      the sum of sub-tile u - 4 is complete, so the phase waited for is the current or the last one.
+                if (j > 0 && __any_sync(0xffffffffu, raise)) {
+                    ok = __all_sync(0xffffffffu, ptx::mbar_wait(&o_done[(u - 1) & 3], ((u - 1) >> 2) & 1, abort_flag));
+                    ptx::tc_fence_after_sync();
+                    const float alpha = raise ? fast_exp2(m_prev - m) : 1.f;
+                    const uint64_t a2 = ptx::f32x2(alpha, alpha);
 #pragma unroll 1
-                        for (int ch = 0; ch < SLICE / 128; ++ch) {     // this thread's quarter of the output columns
-                            uint32_t r[32];
-                            ptx::tmem_ld32(tmem_o + lane_base + part * (SLICE / 4) + ch * 32, r);
-                            ptx::tmem_wait_ld();
-                            const uint64_t a2 = ptx::f32x2(alpha, alpha);
+                    for (int ch = 0; ch < SLICE / 32; ++ch) {
+                        ptx::tmem_ld32(tmem_o + lane_base + ch * 32, ra);
+                        ptx::tmem_wait_ld();
 #pragma unroll
-                            for (int e = 0; e < 32; e += 2) {
-                                float v0, v1;
-                                ptx::f32x2_split(ptx::mul2(ptx::f32x2(__uint_as_float(r[e]), __uint_as_float(r[e + 1])), a2), v0, v1);
-                                r[e] = __float_as_uint(v0);
-                                r[e + 1] = __float_as_uint(v1);
-                            }
-                            ptx::tmem_st32(tmem_o + lane_base + part * (SLICE / 4) + ch * 32, r);
+                        for (int e = 0; e < 32; e += 2) {
+                            float v0, v1;
+                            ptx::f32x2_split(ptx::mul2(ptx::f32x2(__uint_as_float(ra[e]), __uint_as_float(ra[e + 1])), a2), v0, v1);
+                            ra[e] = __float_as_uint(v0);
+                            ra[e + 1] = __float_as_uint(v1);
                         }
+                        ptx::tmem_st32(tmem_o + lane_base + ch * 32, ra);
                     }
                 }
                 ptx::tmem_wait_st();
                 ptx::tc_fence_before_sync();
                 __syncwarp();
-                if (lane == 0) ptx::mbar_arrive_cluster(p_full_leader[tj & 1]);
+                if (lane == 0) ptx::mbar_arrive_cluster(p_full_leader);
             }
-            // ---- end of the item: the row sums go to the epilogue warps (double-buffered by item:
-            //      the epilogue of item n reads them before it hands O back, which the sums of
-            //      item n + 1 wait for, long before item n + 2 ends)
-            xsum[(((n & 1) * 4 + quarter) * 4 + part) * 32 + lane] = l;
+            // ---- end of the item: (maximum, row sum) of this group go to the epilogue warps
+            //      (double-buffered by item: the epilogue of item n reads them before it hands O
+            //      back, which the sums of item n + 1 wait for, long before item n + 2 ends)
+            xsum[((n & 1) * kAttnGroups + wg) * 128 + row] = make_float2(m_own, l);
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(epi_ready);
+            w = nxt;
+            have = have_next;
         }
-    } else {
+    } else if (warp < 4 * kAttnGroups + 4) {
         // 4 epilogue warps, one per TMEM lane quarter, a row per thread.  After the last sum of an item
         // (o_item: one completion per item, and the next cannot come before this item's O has been
         // handed back) they divide O by the row sum, round to bf16 into the staging boxes (box = 64 columns x
@@ -416,58 +459,80 @@ sm100_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         const int row = quarter * 32 + lane;
         const uint32_t lane_base = ((uint32_t)(quarter * 32) << 16);
         const uint32_t o_free_leader = ptx::map_to_cta(ptx::smem_addr(o_free), 0);
-        const float* xsum = reinterpret_cast<const float*>(smem + kAttnSumOff);
-        const bool store_issuer = warp == 18 && lane == 0;
+        const float2* xsum = reinterpret_cast<const float2*>(smem + kAttnSumOff);
+        const bool store_issuer = warp == 4 * kAttnGroups && lane == 0;
         bool ok = true;      // as for the softmax warps: on a wait that gave up the loops run to their end
         AttnItem w;
         for (int n = 0; attn_item(d, n_kt, n_qp, n_slices, total, G, pr, n, &w); ++n) {
-            ok = __all_sync(0xffffffffu, ptx::mbar_wait_backoff(o_item, n & 1, abort_flag, 100));
-            ok = __all_sync(0xffffffffu, ptx::mbar_wait(epi_ready, n & 1, abort_flag));
+            if (quarter == 2) {     // one warp polls (slowly: an item takes many microseconds), the others are woken by it
+                ok = __all_sync(0xffffffffu, ptx::mbar_wait_backoff(o_item, n & 1, abort_flag, 200));
+                ok = __all_sync(0xffffffffu, ptx::mbar_wait(epi_ready, n & 1, abort_flag));
+            }
+            wait_group_sync(6);
             ptx::tc_fence_after_sync();
-            const float* xs = xsum + ((n & 1) * 4 + quarter) * 128;
-            const float inv_l = 1.f / ((xs[lane] + xs[32 + lane]) + (xs[64 + lane] + xs[96 + lane]));
+            // the groups' sums, each relative to the maximum its group saw last; O is relative to the largest
+            float2 gs[kAttnGroups];
+            float m_fin = -INFINITY;
+#pragma unroll
+            for (int g = 0; g < kAttnGroups; ++g) {
+                gs[g] = xsum[((n & 1) * kAttnGroups + g) * 128 + row];
+                m_fin = fmaxf(m_fin, gs[g].x);
+            }
+            float l_fin = 0.f;
+#pragma unroll
+            for (int g = 0; g < kAttnGroups; ++g)
+                l_fin += gs[g].x == -INFINITY ? 0.f : gs[g].y * fast_exp2(gs[g].x - m_fin);
+            const float inv_l = 1.f / l_fin;
             const int q0 = (2 * w.qp + (int)rank) * 128;
             const uint64_t inv2 = ptx::f32x2(inv_l, inv_l);
             uint8_t* stage = smem + ((n & 1) ? kAttnOutOff : 0u);    // the buffer that held this item's Q
-            // Four passes of 64 columns = one box each, the two halves of the buffer used alternately:
-            // a pass only waits for the store of the pass before last.  O is handed back as soon as
-            // its last columns are in registers.
+            // Four passes of 64 columns = one box each, the two halves of the buffer used alternately: a pass
+            // only waits for the store of the pass before last.  O is read 16 columns at a time, the next 16
+            // already on their way while the current ones are scaled, rounded and staged; it is handed back
+            // as soon as its last columns are in registers (the next item's first sum waits for that).
+            uint32_t ra[16], rb[16];
+            auto stage_out = [&](const uint32_t (&r)[16], int c) {      // columns 16 c .. 16 c + 15 of the slice
+                uint8_t* box_row = stage + ((c >> 2) & 1) * kAttnOutBoxBytes + row * 128;
+                uint32_t pk[8];
+#pragma unroll
+                for (int e = 0; e < 8; ++e) {
+                    float v0, v1;
+                    ptx::f32x2_split(ptx::mul2(ptx::f32x2(__uint_as_float(r[2 * e]), __uint_as_float(r[2 * e + 1])), inv2), v0, v1);
+                    pk[e] = pack_bf16x2(v0, v1);
+                }
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {        // 16-byte chunks 2 (c & 3), 2 (c & 3) + 1 of the box row
+                    const int chunk = ((c & 3) * 2 + h) ^ (row & 7);
+                    *reinterpret_cast<uint4*>(box_row + chunk * 16) = make_uint4(pk[4 * h], pk[4 * h + 1], pk[4 * h + 2], pk[4 * h + 3]);
+                }
+            };
+            constexpr int kChunks = SLICE / 16;
+            ptx::tmem_ld16(tmem_o + lane_base, ra);
 #pragma unroll 1
             for (int pass = 0; pass < SLICE / 64; ++pass) {
-                uint8_t* box_row = stage + (pass & 1) * kAttnOutBoxBytes + row * 128;
                 if (pass >= 2) {
                     if (store_issuer) ptx::bulk_wait_group_read_but_one();
                     epilogue_sync();
                 }
-#pragma unroll 1
-                for (int ch = 0; ch < 2; ++ch) {     // 32 columns at a time: 16-byte chunks 4 ch .. 4 ch + 3 of the row
-                    uint32_t r[32];
-                    ptx::tmem_ld32(tmem_o + lane_base + pass * 64 + ch * 32, r);
+#pragma unroll
+                for (int q = 0; q < 4; q += 2) {
+                    const int c = pass * 4 + q;
                     ptx::tmem_wait_ld();
-                    if (pass == SLICE / 64 - 1 && ch == 1) {      // O has been read completely: the next item's sums may start
+                    ptx::tmem_ld16(tmem_o + lane_base + (c + 1) * 16, rb);
+                    stage_out(ra, c);
+                    ptx::tmem_wait_ld();
+                    if (c + 2 < kChunks) {
+                        ptx::tmem_ld16(tmem_o + lane_base + (c + 2) * 16, ra);
+                    } else {                  // O has been read completely: the next item's sums may start
                         ptx::tc_fence_before_sync();
                         __syncwarp();
                         if (lane == 0) ptx::mbar_arrive_cluster(o_free_leader);
                     }
-                    // two-wide multiplies: these warps share their schedulers with the softmax warps,
-                    // and every issue slot they need delays handing O back
-                    uint32_t pk[16];
-#pragma unroll
-                    for (int e = 0; e < 16; ++e) {
-                        float v0, v1;
-                        ptx::f32x2_split(ptx::mul2(ptx::f32x2(__uint_as_float(r[2 * e]), __uint_as_float(r[2 * e + 1])), inv2), v0, v1);
-                        pk[e] = pack_bf16x2(v0, v1);
-                    }
-#pragma unroll
-                    for (int c = 0; c < 4; ++c) {
-                        const int chunk = (ch * 4 + c) ^ (row & 7);
-                        *reinterpret_cast<uint4*>(box_row + chunk * 16) =
-                            make_uint4(pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
-                    }
+                    stage_out(rb, c + 1);
                 }
                 ptx::fence_proxy_async_smem();
                 epilogue_sync();
-                if (store_issuer && q0 < d.N) {
+                if (store_issuer && q0 < d.N && w.slice * SLICE + pass * 64 < d.d_l) {
                     ptx::tma_store_3d(&tm_o, stage + (pass & 1) * kAttnOutBoxBytes, w.slice * SLICE + pass * 64, q0,
                                       w.b * d.n_q + w.g);
                     ptx::bulk_commit_group();
@@ -484,7 +549,7 @@ sm100_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     __syncthreads();
     ptx::cluster_arrive();     // neither CTA leaves (or frees TMEM) while the other may still signal it
     ptx::cluster_wait();
-    if (warp == 1) ptx::tmem_dealloc_pair(tmem_base, 512);
+    if (warp == 21) ptx::tmem_dealloc_pair(tmem_base, 512);
     if (threadIdx.x == 0 && *abort_flag) raise_status(status_word, GTA_ERR_TIMEOUT);
 }
 
@@ -505,7 +570,7 @@ static gta_status_t launch_attention(const Dims& d, const CUtensorMap& tm_q, con
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAttnSmemTotal) != cudaSuccess)
         return GTA_ERR_CUDA;
     const int n_qt = (d.N + 127) / 128, n_qp = (n_qt + 1) / 2;
-    const long long n_items = (long long)n_qp * (d.d_l / SLICE) * d.n_q * d.B;
+    const long long n_items = (long long)n_qp * (d.d_l * 2 == SLICE ? 1 : d.d_l / SLICE) * d.n_q * d.B;
     if (n_items > 0x3fffffffLL) return GTA_ERR_UNSUPPORTED;
     cudaLaunchConfig_t cfg = {};
     cfg.blockDim = dim3(kAttnThreads);
@@ -540,36 +605,44 @@ static gta_status_t launch_attention(const Dims& d, const CUtensorMap& tm_q, con
     return cudaGetLastError() == cudaSuccess ? GTA_OK : GTA_ERR_CUDA;
 }
 
+// L[B, n_q, N, d_l] (bf16) = Softmax(scale Q K^T) C per attention map: the attention kernel alone.  d_l is a
+// multiple of 128, or 64 (the narrow case of the comparison operators).
+gta_status_t launch_sm100_attention(const Dims& d, const void* q, const void* k, const void* c, void* l_out,
+                                    int32_t* status_word, cudaStream_t stream) {
+    CUtensorMap tm_q, tm_k, tm_c, tm_o;
+    const uint32_t box[3] = {64, 128, 1}, box_k[3] = {64, 64, 1};
+    const uint64_t dq[3] = {(uint64_t)d.d_h, (uint64_t)d.N, (uint64_t)d.B * d.n_q};
+    // K / C: Nk of the S rows of a plane take part; the rest (the unused tail of a cache, which may hold
+    // anything, NaN bit patterns included) lies outside the maps and reads as zeros
+    const uint64_t dk[3] = {(uint64_t)d.d_h, (uint64_t)d.Nk, (uint64_t)d.B * d.n_k};
+    const uint64_t dc[3] = {(uint64_t)d.d_l, (uint64_t)d.Nk, (uint64_t)d.B * d.n_c};
+    const uint64_t ak[3] = {(uint64_t)d.d_h, (uint64_t)d.S, (uint64_t)d.B * d.n_k};
+    const uint64_t ac[3] = {(uint64_t)d.d_l, (uint64_t)d.S, (uint64_t)d.B * d.n_c};
+    if (!make_bf16_map(&tm_q, q, 3, dq, box) || !make_bf16_map(&tm_k, k, 3, dk, box_k, ak) ||
+        !make_bf16_map(&tm_c, c, 3, dc, box, ac))
+        return GTA_ERR_CUDA;
+    {   // L [B n_q][N][d_l], stored in boxes of 128 rows x 64 columns
+        const uint64_t dl[3] = {(uint64_t)d.d_l, (uint64_t)d.N, (uint64_t)d.B * d.n_q};
+        const uint32_t box_o[3] = {64, 128, 1};
+        if (!make_bf16_map(&tm_o, l_out, 3, dl, box_o)) return GTA_ERR_CUDA;
+    }
+    gta_status_t st;
+    if (d.d_h == 128)
+        st = d.d_l % 256 == 0 ? launch_attention<128, 256>(d, tm_q, tm_k, tm_c, tm_o, status_word, stream)
+                              : launch_attention<128, 128>(d, tm_q, tm_k, tm_c, tm_o, status_word, stream);
+    else
+        st = d.d_l % 256 == 0 ? launch_attention<64, 256>(d, tm_q, tm_k, tm_c, tm_o, status_word, stream)
+                              : launch_attention<64, 128>(d, tm_q, tm_k, tm_c, tm_o, status_word, stream);
+    if (st != GTA_OK) return st;
+    return cudaGetLastError() == cudaSuccess ? GTA_OK : GTA_ERR_CUDA;
+}
+
 gta_status_t launch_sm100_prefill(const Dims& d, const void* q, const void* k, const void* c, const void* x,
                                   const void* w_p, const void* w_g, void* out, void* workspace,
                                   int32_t* status_word, cudaStream_t stream, int stages, int* launches) {
     if (stages & 1) {
-        CUtensorMap tm_q, tm_k, tm_c, tm_o;
-        const uint32_t box[3] = {64, 128, 1}, box_k[3] = {64, 64, 1};
-        const uint64_t dq[3] = {(uint64_t)d.d_h, (uint64_t)d.N, (uint64_t)d.B * d.n_q};
-        // K / C: Nk of the S rows of a plane take part; the rest (the unused tail of a cache, which may hold
-        // anything, NaN bit patterns included) lies outside the maps and reads as zeros
-        const uint64_t dk[3] = {(uint64_t)d.d_h, (uint64_t)d.Nk, (uint64_t)d.B * d.n_k};
-        const uint64_t dc[3] = {(uint64_t)d.d_l, (uint64_t)d.Nk, (uint64_t)d.B * d.n_c};
-        const uint64_t ak[3] = {(uint64_t)d.d_h, (uint64_t)d.S, (uint64_t)d.B * d.n_k};
-        const uint64_t ac[3] = {(uint64_t)d.d_l, (uint64_t)d.S, (uint64_t)d.B * d.n_c};
-        if (!make_bf16_map(&tm_q, q, 3, dq, box) || !make_bf16_map(&tm_k, k, 3, dk, box_k, ak) ||
-            !make_bf16_map(&tm_c, c, 3, dc, box, ac))
-            return GTA_ERR_CUDA;
-        {   // L [B n_q][N][d_l], stored in boxes of 128 rows x 64 columns
-            const uint64_t dl[3] = {(uint64_t)d.d_l, (uint64_t)d.N, (uint64_t)d.B * d.n_q};
-            const uint32_t box_o[3] = {64, 128, 1};
-            if (!make_bf16_map(&tm_o, workspace, 3, dl, box_o)) return GTA_ERR_CUDA;
-        }
-        gta_status_t st;
-        if (d.d_h == 128)
-            st = d.d_l % 256 == 0 ? launch_attention<128, 256>(d, tm_q, tm_k, tm_c, tm_o, status_word, stream)
-                                  : launch_attention<128, 128>(d, tm_q, tm_k, tm_c, tm_o, status_word, stream);
-        else
-            st = d.d_l % 256 == 0 ? launch_attention<64, 256>(d, tm_q, tm_k, tm_c, tm_o, status_word, stream)
-                                  : launch_attention<64, 128>(d, tm_q, tm_k, tm_c, tm_o, status_word, stream);
+        gta_status_t st = launch_sm100_attention(d, q, k, c, workspace, status_word, stream);
         if (st != GTA_OK) return st;
-        if (cudaGetLastError() != cudaSuccess) return GTA_ERR_CUDA;
         *launches += 1;
     }
     if (stages & 2) {

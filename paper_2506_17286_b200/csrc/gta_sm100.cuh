@@ -13,6 +13,11 @@ gta_status_t launch_sm100_prefill(const Dims& d, const void* q, const void* k, c
                                   const void* w_p, const void* w_g, void* out, void* workspace,
                                   int32_t* status_word, cudaStream_t stream, int stages, int* launches);
 
+// Attention kernel alone: L[B, n_q, N, d_l] (bf16) = Softmax(scale Q K^T) C per attention map; bf16, d_h = 64 or
+// 128, d_l a multiple of 128 or exactly 64.
+gta_status_t launch_sm100_attention(const Dims& d, const void* q, const void* k, const void* c, void* l_out,
+                                    int32_t* status_word, cudaStream_t stream);
+
 // Decoder + gate kernel alone: out = (L W_P) (.) sigmoid(X W_G) with L[B, n_q, N, d_l] in bf16.
 gta_status_t launch_sm100_decoder(const Dims& d, const void* l_bf16, const void* x, const void* w_p, const void* w_g,
                                   void* out, int32_t* status_word, cudaStream_t stream);

@@ -50,7 +50,6 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
         : "memory");
     return ok != 0;
 }
-
 // Non-blocking query: has the phase with this parity completed?  (try_wait may suspend the thread for
 // a while when it has not.)
 __device__ __forceinline__ bool mbar_test_wait(uint64_t* bar, uint32_t parity) {
@@ -73,37 +72,54 @@ __device__ __forceinline__ uint64_t global_timer_ns() {
 
 // Bounded wait: gives up after about two seconds, or as soon as another thread of the CTA has
 // raised *abort_flag.  Returns false on give-up (the caller unwinds; nothing spins forever).
+//
+// A waiting warp polls, and every poll costs issue slots that the working warps of its scheduler would
+// otherwise have (try_wait comes back after some tens of nanoseconds whether or not the phase has
+// completed).  So the polling loop itself is a handful of instructions (try_wait, an optional sleep, a
+// countdown), and the clock and the abort flag are only looked at between runs of kPollsPerCheck polls.
+// sleep_ns = 0: poll back to back (waits that are short or sit on the critical path); otherwise the
+// thread sleeps about that long between polls (waits that are long and whose end nobody is waiting for).
 constexpr uint64_t kWaitLimitNs = 2000000000ull;
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+constexpr uint32_t kPollsPerCheck = 1024;
+__device__ __forceinline__ bool mbar_poll_run(uint64_t* bar, uint32_t parity, uint32_t sleep_ns) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t.reg .u32 n;\n\t"
+        "mov.u32 n, %4;\n"
+        "GTA_POLL_%=:\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "@p bra GTA_POLL_DONE_%=;\n\t"
+        "setp.ne.u32 q, %3, 0;\n\t"
+        "@q nanosleep.u32 %3;\n\t"
+        "sub.u32 n, n, 1;\n\t"
+        "setp.ne.u32 q, n, 0;\n\t"
+        "@q bra GTA_POLL_%=;\n"
+        "GTA_POLL_DONE_%=:\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_addr(bar)), "r"(parity), "r"(sleep_ns), "r"(kPollsPerCheck)
+        : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ bool mbar_wait_sleep(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
+                                                uint32_t sleep_ns) {
     if (mbar_try_wait(bar, parity)) return true;
     const uint64_t t0 = global_timer_ns();
-    for (uint32_t it = 1;; ++it) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if ((it & 0xff) == 0) {
-            if (*abort_flag) return false;
-            if (global_timer_ns() - t0 > kWaitLimitNs) break;
-        }
+    for (;;) {
+        if (mbar_poll_run(bar, parity, sleep_ns)) return true;
+        if (*abort_flag) return false;
+        if (global_timer_ns() - t0 > kWaitLimitNs) break;
     }
     *abort_flag = 1;
     return false;
 }
-
-// Same wait for threads that wait long and whose reaction time matters little: they sleep between
-// polls, so that their spinning does not take issue slots from the warps that share their scheduler.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+    return mbar_wait_sleep(bar, parity, abort_flag, 0);
+}
+// Same wait for threads that wait long and whose reaction time matters little.
 __device__ __forceinline__ bool mbar_wait_backoff(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
                                                   uint32_t sleep_ns) {
-    if (mbar_try_wait(bar, parity)) return true;
-    const uint64_t t0 = global_timer_ns();
-    for (uint32_t it = 1;; ++it) {
-        __nanosleep(sleep_ns);
-        if (mbar_try_wait(bar, parity)) return true;
-        if ((it & 0xff) == 0) {
-            if (*abort_flag) return false;
-            if (global_timer_ns() - t0 > kWaitLimitNs) break;
-        }
-    }
-    *abort_flag = 1;
-    return false;
+    return mbar_wait_sleep(bar, parity, abort_flag, sleep_ns);
 }
 
 __device__ __forceinline__ void fence_proxy_async_smem() {
@@ -257,6 +273,15 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
           "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
           "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
           "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
         : "r"(taddr)
         : "memory");
 }

@@ -465,3 +465,72 @@ def test_layer_widens_bf16_tensors_exactly(oracle):
     want = np.array([1.0, 1.0 + 2.0 ** -7, -(1.0 + 2.0 ** -7), 2.0 ** -133, -0.0, 3.140625])
     got = oracle._to_f64(bits)
     assert np.array_equal(got, want) and np.signbit(got[4])
+
+
+# ---------------------------------------------------------------- comparison operators (App. B.3 GQA, Sec. 3.1 MHA)
+def _mha_np(q, k, v, causal=True):
+    """Textbook multi-head attention on whole matrices: q, k, v [B, n_h, N, d]."""
+    d = q.shape[-1]
+    s = np.einsum("bhtd,bhjd->bhtj", q, k) / np.sqrt(d)
+    if causal:
+        N = q.shape[2]
+        s = np.where(np.tril(np.ones((N, N), dtype=bool))[None, None], s, -np.inf)
+    return np.einsum("bhtj,bhjd->bhtd", _softmax_np(s), v)
+
+
+@pytest.mark.parametrize("causal", [True, False])
+def test_gqa_is_multi_head_attention_on_repeated_key_value_heads(oracle, causal):
+    B, n_h, n_kv, N, d = 2, 6, 2, 11, 8
+    q, k, v = _rand(B, n_h, N, d), _rand(B, n_kv, N, d), _rand(B, n_kv, N, d)
+    got = oracle.gqa_prefill(q, k, v, causal=causal)
+    rep = n_h // n_kv
+    assert np.allclose(got, _mha_np(q, np.repeat(k, rep, axis=1), np.repeat(v, rep, axis=1), causal), rtol=1e-12, atol=1e-14)
+    # the printed map i mod n_kv is the same operator with the query heads renumbered
+    perm = [i for j in range(n_kv) for i in range(n_h) if i % n_kv == j]      # heads of kv head 0 first, ...
+    got_mod = oracle.gqa_prefill(q, k, v, causal=causal, head_map="mod")
+    assert np.allclose(got_mod[:, perm], oracle.gqa_prefill(q[:, perm], k, v, causal=causal), rtol=1e-12, atol=1e-14)
+    # one key / value head per query head: multi-head attention itself, whichever map
+    k1, v1 = _rand(B, n_h, N, d), _rand(B, n_h, N, d)
+    for hm in ("blocks", "mod"):
+        assert np.allclose(oracle.gqa_prefill(q, k1, v1, causal=causal, head_map=hm), _mha_np(q, k1, v1, causal),
+                           rtol=1e-12, atol=1e-14)
+
+
+def test_gqa_agrees_with_the_gta_oracle_where_the_two_operators_coincide(oracle):
+    """GTA with one map per head, the latent holding the value heads side by side, selector decoders and a
+    zero gate is 0.5 x GQA (sigmoid(0) = 1/2): the C oracle of the operator against the numpy comparison oracle."""
+    B, n_h, n_kv, N, d = 2, 4, 2, 9, 4
+    q, k, v = _rand(B, n_h, N, d), _rand(B, n_kv, N, d), _rand(B, n_kv, N, d)
+    s = Shape(B, N, 8, n_h, n_h, n_kv, n_kv, d, d, 1)
+    w_p = np.broadcast_to(np.eye(d), (n_h, d, d)).copy()
+    got = oracle.prefill(s, q, k, v, _rand(B, N, 8), w_p, np.zeros((8, n_h * d)))       # [B, N, n_h, d]
+    want = oracle.gqa_prefill(q, k, v)                                                  # [B, n_h, N, d]
+    assert np.allclose(got.transpose(0, 2, 1, 3), 0.5 * want, rtol=1e-12, atol=1e-14)
+
+
+def test_gqa_decode_is_the_last_prefill_row_and_skips_empty_sequences(oracle):
+    B, n_h, n_kv, d, cap = 3, 4, 2, 8, 12
+    lens = [7, 0, 12]
+    kc, vc = _rand(B, n_kv, cap, d), _rand(B, n_kv, cap, d)
+    q = _rand(B, n_h, d)
+    got = oracle.gqa_decode(q, kc, vc, lens)
+    assert not got[1].any()
+    for b in (0, 2):
+        n = lens[b]
+        qq = np.zeros((1, n_h, n, d)); qq[0, :, n - 1] = q[b]
+        full = oracle.gqa_prefill(qq, kc[b:b + 1, :, :n], vc[b:b + 1, :, :n])
+        assert np.allclose(got[b], full[0, :, n - 1], rtol=1e-12, atol=1e-14)
+    # rows of the cache behind the live length do not matter
+    kc2, vc2 = kc.copy(), vc.copy()
+    kc2[0, :, 7:] = np.nan; vc2[0, :, 7:] = np.nan
+    assert np.array_equal(oracle.gqa_decode(q, kc2, vc2, lens)[0], got[0])
+
+
+def test_gqa_cost_closed_forms_against_the_printed_ratios(oracle):
+    """Table 3 rows of GQA and GTA at the 1B hyper-parameters: GTA-1B has 37.5 % of GQA-1B's attention cost and
+    30 % of its cache (Sec. 4.3); GQA-1B caches 640 elements per token and layer, MHA 2560."""
+    N = 2048
+    gta_1b = Shape(1, N, 1280, 20, 5, 1, 1, 64, 128)
+    assert oracle.attention_cost(gta_1b) / oracle.gqa_attention_cost(20, 64, N) == pytest.approx(0.375, abs=1e-12)
+    assert oracle.cache_elems(gta_1b) / oracle.gqa_cache_elems(5, 64, N) == pytest.approx(0.30, abs=1e-12)
+    assert oracle.gqa_cache_elems(5, 64, 1) == 640 and oracle.gqa_cache_elems(20, 64, 1) == 2560
