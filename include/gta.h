@@ -339,6 +339,20 @@ GTA_API int gta_prefill_path(const gta_shape_t *shape);
  */
 GTA_API int gta_last_launch_count(void);
 
+/*
+ * Test hook (no counterpart in the paper).  Every wait inside the kernels is bounded: a thread
+ * that waits longer than a time limit gives up, tells the other threads of its CTA and of its
+ * cluster, the kernel unwinds (outstanding copies and MMAs are waited for, tensor memory is
+ * freed), raises GTA_ERR_TIMEOUT in the status word and returns; the context stays usable.
+ * This call lets a test exercise that path of the tensor-core attention kernel on a healthy
+ * GPU: limit_ns replaces the limit of its waits (0 = the built-in two seconds), and with
+ * withhold_first_arrive != 0 one softmax warp of every CTA pair keeps its first arrival to
+ * itself, so that the first sum of every pair is never released and the limit runs out.
+ * The settings live in device memory of the current device and hold for later launches on it
+ * until they are changed back; the call synchronises the device.  Not for production use.
+ */
+GTA_API gta_status_t gta_debug_attention_wait(uint64_t limit_ns, int32_t withhold_first_arrive);
+
 #ifdef __cplusplus
 }
 #endif

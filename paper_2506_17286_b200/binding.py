@@ -26,7 +26,7 @@ EXPORTS = (
     "gta_prefill_stages", "gta_decode_stages", "gta_decode_static", "gta_prefill_chunk",
     "gta_decode_paged_workspace_bytes", "gta_decode_paged", "gta_cache_append_paged",
     "gta_layer_prefill_workspace_bytes", "gta_layer_prefill", "gta_layer_decode_workspace_bytes", "gta_layer_decode",
-    "gta_layer_decode_paged_workspace_bytes", "gta_layer_decode_paged",
+    "gta_layer_decode_paged_workspace_bytes", "gta_layer_decode_paged", "gta_debug_attention_wait",
 )
 
 
@@ -103,6 +103,8 @@ def lib():
         L.gta_prefill_path.argtypes = [sp]
         L.gta_prefill_path.restype = i32
         L.gta_last_launch_count.restype = i32
+        L.gta_debug_attention_wait.argtypes = [ctypes.c_uint64, i32]
+        L.gta_debug_attention_wait.restype = i32
         _lib = L
     return _lib
 
@@ -113,6 +115,14 @@ def status_string(status: int) -> str:
 
 def version() -> int:
     return int(lib().gta_version())
+
+
+def debug_attention_wait(limit_ns: int = 0, withhold_first_arrive: bool = False) -> None:
+    """Test hook: time limit of the attention kernel's bounded waits (0 = built-in) and the switch that
+    makes the first sum of every CTA pair wait in vain (see gta_debug_attention_wait in include/gta.h)."""
+    st = lib().gta_debug_attention_wait(int(limit_ns), int(bool(withhold_first_arrive)))
+    if st != GTA_OK:
+        raise GtaError(st, "gta_debug_attention_wait")
 
 
 def last_launch_count() -> int:

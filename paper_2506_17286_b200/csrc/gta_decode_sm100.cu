@@ -245,7 +245,7 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
             if (lane == 0 && *abort_flag) {
                 for (int back = 1; back <= kStreamStages && it - back >= 0; ++back) {
                     const int iq = it - back;
-                    ptx::mbar_wait(&full_bar[iq % kStreamStages], (iq / kStreamStages) & 1, drain_flag);
+                    ptx::mbar_wait_drain(&full_bar[iq % kStreamStages], (iq / kStreamStages) & 1, drain_flag);
                 }
             }
         }

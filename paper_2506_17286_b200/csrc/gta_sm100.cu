@@ -115,6 +115,13 @@ __device__ __forceinline__ float max_chunk(const uint32_t (&r)[32], float mx) {
     }
     return fmaxf(a, b);
 }
+// Test hooks of the bounded waits (gta_debug_attention_wait): the time limit of every wait of the attention
+// kernel, and a switch that makes one softmax warp keep its very first arrival to itself, so that the
+// thread that issues the sums runs into that limit and the whole unwinding path can be exercised on a
+// healthy GPU.  Both live in device memory of the library and are read once per thread at kernel start.
+static __device__ unsigned long long g_attn_wait_limit_ns = ptx::kWaitLimitNs;
+static __device__ int g_attn_withhold_first_arrive = 0;
+
 struct AttnItem {
     int b, g, slice, qp, n_tiles;   // qp: pair of query tiles (2 qp, 2 qp + 1)
 };
@@ -148,7 +155,7 @@ sm100_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     float* xchg = reinterpret_cast<float*>(smem + kAttnXchgOff);
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kAttnBarOff);
-    uint64_t* q_full = bars;            // leader CTA; both producers arrive
+    uint64_t* q_full = bars;            // [2] (slots 0 and 41) leader CTA; both producers arrive; item n uses barrier n & 1
     uint64_t* stage_free = bars + 1;    // this CTA; its epilogue's stores have read the buffer (one thread arrives)
     uint64_t* full = bars + 2;          // [4] leader CTA; both producers arrive
     uint64_t* empty = bars + 6;         // [4] both CTAs (multicast commit)
@@ -159,12 +166,19 @@ sm100_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     uint64_t* epi_ready = bars + 23;    // this CTA; its 16 softmax warps arrive (maxima and row sums of an item are in place)
     uint64_t* o_item = bars + 24;       // both CTAs (multicast commit): the last sum of an item is complete
     uint64_t* chain = bars + 25;        // [4 groups][4 quarters] this CTA; one warp arrives: its rows' running maxima are published
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 41);
+    uint64_t* mma_drain = bars + 42;    // [2] leader CTA: used once by an MMA-issuing thread that unwinds (all its MMAs are done)
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 44);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
     volatile int* drain_flag = abort_flag + 1;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = ptx::cluster_ctarank();          // 0 = leader
+    const uint64_t wait_limit = g_attn_wait_limit_ns;
+    const bool withhold_first_arrive = g_attn_withhold_first_arrive != 0;
+    // every wait of this kernel: bounded by wait_limit, ended early by the CTA's abort flag
+    auto wait = [&](uint64_t* bar, uint32_t parity, uint32_t sleep_ns = 0) {
+        return ptx::mbar_wait_sleep(bar, parity, abort_flag, sleep_ns, wait_limit);
+    };
     const int G = gridDim.x >> 1, pr = blockIdx.x >> 1;    // CTA pairs, this pair
     const bool bad_align = (uint32_t)(smem - smem_raw) > kAttnAlignSlack;   // cannot happen with a 256-byte aligned window
     constexpr uint32_t kQLoadBytes = 128 * DH * 2;                 // this CTA's query tile
@@ -179,7 +193,10 @@ sm100_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     const long long total = bad_align ? 0 : (long long)n_qp * n_slices * d.n_q * d.B;
 
     if (threadIdx.x == 0) {
-        ptx::mbar_init(q_full, 2);
+        ptx::mbar_init(&q_full[0], 2);
+        ptx::mbar_init(&q_full[41], 2);
+        ptx::mbar_init(&mma_drain[0], 1);
+        ptx::mbar_init(&mma_drain[1], 1);
         ptx::mbar_init(stage_free, 1);
         for (int s = 0; s < kAttnStages; ++s) { ptx::mbar_init(&full[s], 2); ptx::mbar_init(&empty[s], 1); }
         for (int s = 0; s < kAttnGroups; ++s) {
@@ -212,25 +229,27 @@ sm100_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     if (warp == 20) {
         if (ptx::elect_one()) {
             ptx::prefetch_tensormap(&tm_q); ptx::prefetch_tensormap(&tm_k); ptx::prefetch_tensormap(&tm_c);
-            const uint32_t q_full_leader = ptx::map_to_cta(ptx::smem_addr(q_full), 0);
             int tj = 0;                 // key tiles issued so far (ring position), across items
+            int n_armed = 0;            // query tiles whose load has been issued
             bool ok = true;
             AttnItem w;
             for (int n = 0; ok && attn_item(d, n_kt, n_qp, n_slices, total, G, pr, n, &w); ++n) {
+                const uint32_t q_full_leader = ptx::map_to_cta(ptx::smem_addr(&q_full[(n & 1) * 41]), 0);
                 const int kg = d.q_to_k(w.g), cg = d.q_to_c(w.g);
                 const int q0 = (2 * w.qp + (int)rank) * 128;       // this CTA's query rows
                 // buffer n & 1 is free once the epilogue of item n - 2 has stored out of it (which
                 // also means every Q K^T of that item is done); every completion is waited for, in order
-                if (n >= 2) ok = ptx::mbar_wait(stage_free, n & 1, abort_flag);
+                if (n >= 2) ok = wait(stage_free, n & 1);
                 if (!ok) break;
                 uint8_t* q_s = smem + ((n & 1) ? kAttnOutOff : 0u);
                 ptx::mbar_arrive_expect_tx_cluster(q_full_leader, kQLoadBytes);
+                ++n_armed;
                 ptx::tma_load_3d_pair(q_s, &tm_q, q_full_leader, 0, q0, w.b * d.n_q + w.g);
                 if (DH == 128) ptx::tma_load_3d_pair(q_s + 16384, &tm_q, q_full_leader, 64, q0, w.b * d.n_q + w.g);
                 for (int j = 0; j < w.n_tiles; ++j, ++tj) {
                     const int s = tj % kAttnStages;
                     const uint32_t ph = (tj / kAttnStages) & 1;
-                    ok = ptx::mbar_wait_backoff(&empty[s], ph ^ 1, abort_flag, 64);   // the ring is three tiles ahead
+                    ok = wait(&empty[s], ph ^ 1, 64);   // the ring is three tiles ahead
                     if (!ok) break;
                     uint8_t* k_s = smem + kAttnRingOff + s * kAttnStageBytes;
                     uint8_t* c_s = k_s + kKHalfBytes;
@@ -245,12 +264,18 @@ sm100_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                         ptx::tma_load_3d_pair(c_s + 16384, &tm_c, bar, col0 + 64, j * kKeyTile, w.b * d.n_c + cg);
                 }
             }
-            if (*abort_flag && rank == 0) {   // drain what was armed (bounded), so no copy lands after exit
-                ptx::mbar_wait(q_full, 0, drain_flag);
-                ptx::mbar_wait(q_full, 1, drain_flag);
+            if (*abort_flag && rank == 0) {
+                // Unwinding: wait (bounded) for the copies that were armed, so that none lands after the CTA has
+                // left.  At most the last two query tiles and the last three ring tiles can be outstanding (the
+                // loads before them were consumed before their buffers were armed again), each on a barrier whose
+                // earlier phases are complete, so a parity wait for its latest phase is unambiguous.
+                for (int back = 1; back <= 2 && n_armed - back >= 0; ++back) {
+                    const int m = n_armed - back;
+                    ptx::mbar_wait_drain(&q_full[(m & 1) * 41], (m >> 1) & 1, drain_flag);
+                }
                 for (int back = 1; back <= kAttnStages && tj - back >= 0; ++back) {
                     const int jq = tj - back;
-                    ptx::mbar_wait(&full[jq % kAttnStages], (jq / kAttnStages) & 1, drain_flag);
+                    ptx::mbar_wait_drain(&full[jq % kAttnStages], (jq / kAttnStages) & 1, drain_flag);
                 }
             }
         }
@@ -278,9 +303,9 @@ sm100_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                     const uint32_t q_lo = (smem_base + ((n & 1) ? kAttnOutOff : 0u)) >> 4;
                     for (int j = 0; j < n_sub && ok; ++j, ++u) {
                         const int tile = u >> 1, stage = tile % kAttnStages;
-                        if (u >= kAttnGroups) ok = ptx::mbar_wait(&o_done[u & 3], ((u - kAttnGroups) >> 2) & 1, abort_flag);
-                        if (ok && j == 0) ok = ptx::mbar_wait(q_full, n & 1, abort_flag);
-                        if (ok && (j & 1) == 0) ok = ptx::mbar_wait(&full[stage], (tile / kAttnStages) & 1, abort_flag);
+                        if (u >= kAttnGroups) ok = wait(&o_done[u & 3], ((u - kAttnGroups) >> 2) & 1);
+                        if (ok && j == 0) ok = wait(&q_full[(n & 1) * 41], (n >> 1) & 1);
+                        if (ok && (j & 1) == 0) ok = wait(&full[stage], (tile / kAttnStages) & 1);
                         if (!ok) break;
                         ptx::tc_fence_after_sync();
                         // this CTA's keys 32 (j & 1) .. of its 64 keys of the ring tile: 32 rows of 128 bytes further
@@ -301,8 +326,8 @@ sm100_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                     // ---- sums
                     for (int j = 0; j < n_sub && ok; ++j, ++u) {
                         const int tile = u >> 1, stage = tile % kAttnStages, sub = j & 1;
-                        ok = ptx::mbar_wait(&p_full[u & 3], (u >> 2) & 1, abort_flag);
-                        if (ok && j == 0 && n > 0) ok = ptx::mbar_wait(o_free, (n - 1) & 1, abort_flag);
+                        ok = wait(&p_full[u & 3], (u >> 2) & 1);
+                        if (ok && j == 0 && n > 0) ok = wait(o_free, (n - 1) & 1);
                         if (!ok) break;
                         ptx::tc_fence_after_sync();
                         // P columns 16 kk .. are the keys 32 sub + 16 (kk & 1) .. of CTA kk >> 1, i.e. rows
@@ -321,6 +346,13 @@ sm100_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                         if (sub == 1) ptx::tc_commit_pair(&empty[stage], 3);
                     }
                 }
+            }
+            if (*abort_flag) {
+                // Unwinding: the MMAs this thread has issued must be complete before tensor memory is freed.
+                // A commit on a barrier that is used for nothing else completes when they all are.
+                uint64_t* bar = &mma_drain[warp - 21];
+                ptx::tc_commit_pair(bar, 1);
+                ptx::mbar_wait_drain(bar, 0, drain_flag);
             }
         }
     } else if (warp < 4 * kAttnGroups) {
@@ -360,7 +392,7 @@ sm100_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                 if ((u & (kAttnGroups - 1)) != wg) continue;
                 // one warp of the group polls for the scores (on a scheduler of its own: group g's poller is its
                 // warp of lane quarter g), the other three are woken through a named barrier
-                if (quarter == wg) ok = __all_sync(0xffffffffu, ptx::mbar_wait(&s_full[wg], (u >> 2) & 1, abort_flag));
+                if (quarter == wg) ok = __all_sync(0xffffffffu, wait(&s_full[wg], (u >> 2) & 1));
                 wait_group_sync(1 + wg);
                 ptx::tc_fence_after_sync();
                 // columns 0 .. 31 of the buffer: keys key_a .. of the ring tile's first half (the leader CTA's),
@@ -382,7 +414,7 @@ sm100_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                 const float m_tile = mx * c_scale;     // c_scale > 0
                 // ---- (2) the chain of running maxima (every sub-tile but the very first waits for the one
                 //      before it, every sub-tile but the very last signals the one after it: strict rotation)
-                if (u > 0) ok = __all_sync(0xffffffffu, ptx::mbar_wait(chain_in, ((u - 1) >> 2) & 1, abort_flag));
+                if (u > 0) ok = __all_sync(0xffffffffu, wait(chain_in, ((u - 1) >> 2) & 1));
                 const float m_prev = (j == 0) ? -INFINITY : *m_in;
                 const bool raise = m_tile > m_prev + 8.f;     // also true on the first live sub-tile (m_prev = -inf)
                 const float m = raise ? m_tile : m_prev;
@@ -417,7 +449,7 @@ sm100_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                 //      (one per buffer) completes once per four sub-tiles, and when the scores of sub-tile u exist
                 //      the sum of sub-tile u - 4 is complete, so the phase waited for is the current or the last one.
                 if (j > 0 && __any_sync(0xffffffffu, raise)) {
-                    ok = __all_sync(0xffffffffu, ptx::mbar_wait(&o_done[(u - 1) & 3], ((u - 1) >> 2) & 1, abort_flag));
+                    ok = __all_sync(0xffffffffu, wait(&o_done[(u - 1) & 3], ((u - 1) >> 2) & 1));
                     ptx::tc_fence_after_sync();
                     const float alpha = raise ? fast_exp2(m_prev - m) : 1.f;
                     const uint64_t a2 = ptx::f32x2(alpha, alpha);
@@ -438,7 +470,8 @@ sm100_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                 ptx::tmem_wait_st();
                 ptx::tc_fence_before_sync();
                 __syncwarp();
-                if (lane == 0) ptx::mbar_arrive_cluster(p_full_leader);
+                if (lane == 0 && !(withhold_first_arrive && u == 0 && quarter == 0 && rank == 0))
+                    ptx::mbar_arrive_cluster(p_full_leader);
             }
             // ---- end of the item: (maximum, row sum) of this group go to the epilogue warps
             //      (double-buffered by item: the epilogue of item n reads them before it hands O
@@ -465,8 +498,8 @@ sm100_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         AttnItem w;
         for (int n = 0; attn_item(d, n_kt, n_qp, n_slices, total, G, pr, n, &w); ++n) {
             if (quarter == 2) {     // one warp polls (slowly: an item takes many microseconds), the others are woken by it
-                ok = __all_sync(0xffffffffu, ptx::mbar_wait_backoff(o_item, n & 1, abort_flag, 200));
-                ok = __all_sync(0xffffffffu, ptx::mbar_wait(epi_ready, n & 1, abort_flag));
+                ok = __all_sync(0xffffffffu, wait(o_item, n & 1, 200));
+                ok = __all_sync(0xffffffffu, wait(epi_ready, n & 1));
             }
             wait_group_sync(6);
             ptx::tc_fence_after_sync();
@@ -554,6 +587,17 @@ sm100_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
 }
 
 // --------------------------------------------------------------------------- host side
+gta_status_t sm100_attention_debug_wait(unsigned long long limit_ns, int withhold_first_arrive) {
+    const unsigned long long lim = limit_ns ? limit_ns : ptx::kWaitLimitNs;
+    const int sw = withhold_first_arrive ? 1 : 0;
+    if (cudaMemcpyToSymbol(g_attn_wait_limit_ns, &lim, sizeof(lim)) != cudaSuccess ||
+        cudaMemcpyToSymbol(g_attn_withhold_first_arrive, &sw, sizeof(sw)) != cudaSuccess) {
+        cudaGetLastError();
+        return GTA_ERR_CUDA;
+    }
+    return GTA_OK;
+}
+
 bool sm100_prefill_supported(const Dims& d, int dtype) {
     // the decoder + gate kernel cuts the output columns in blocks of at least 128 inside one attention map
     const bool blocks_ok = d.n_q > 0 && ((d.n_h / d.n_q) * d.d_h) % 128 == 0;

@@ -18,6 +18,9 @@ gta_status_t launch_sm100_prefill(const Dims& d, const void* q, const void* k, c
 gta_status_t launch_sm100_attention(const Dims& d, const void* q, const void* k, const void* c, void* l_out,
                                     int32_t* status_word, cudaStream_t stream);
 
+// Test hooks of the attention kernel's bounded waits (see gta_debug_attention_wait in gta.h).
+gta_status_t sm100_attention_debug_wait(unsigned long long limit_ns, int withhold_first_arrive);
+
 // Decoder + gate kernel alone: out = (L W_P) (.) sigmoid(X W_G) with L[B, n_q, N, d_l] in bf16.
 gta_status_t launch_sm100_decoder(const Dims& d, const void* l_bf16, const void* x, const void* w_p, const void* w_g,
                                   void* out, int32_t* status_word, cudaStream_t stream);

@@ -231,7 +231,7 @@ sm100_decoder_kernel(const __grid_constant__ CUtensorMap tm_l, const __grid_cons
             if (*abort_flag && rank == 0) {   // drain: every armed stage either lands or the wait gives up
                 for (int back = 1; back <= n_stages && it - back >= 0; ++back) {
                     const int kq = it - back;
-                    ptx::mbar_wait(&full_bar[kq % n_stages], (kq / n_stages) & 1, drain_flag);
+                    ptx::mbar_wait_drain(&full_bar[kq % n_stages], (kq / n_stages) & 1, drain_flag);
                 }
             }
         }

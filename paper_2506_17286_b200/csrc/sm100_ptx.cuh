@@ -101,20 +101,48 @@ __device__ __forceinline__ bool mbar_poll_run(uint64_t* bar, uint32_t parity, ui
         : "memory");
     return ok != 0;
 }
+// Raises the abort flag of this CTA and of every other CTA of its cluster (the flag sits at the same
+// shared-memory offset in all of them), so that a peer that waits for this CTA learns of the give-up
+// within one run of polls instead of running into its own time limit.
+__device__ __forceinline__ void raise_abort_cluster(volatile int* abort_flag) {
+    *abort_flag = 1;
+    uint32_t n_ranks, my_rank;
+    asm volatile("mov.u32 %0, %%cluster_nctarank;" : "=r"(n_ranks));
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(my_rank));
+    const uint32_t local = smem_addr(const_cast<int*>(abort_flag));
+    for (uint32_t r = 0; r < n_ranks; ++r) {
+        if (r == my_rank) continue;
+        uint32_t remote;
+        asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local), "r"(r));
+        asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(remote), "r"(1u) : "memory");
+    }
+}
 __device__ __forceinline__ bool mbar_wait_sleep(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
-                                                uint32_t sleep_ns) {
+                                                uint32_t sleep_ns, uint64_t limit_ns = kWaitLimitNs) {
     if (mbar_try_wait(bar, parity)) return true;
     const uint64_t t0 = global_timer_ns();
     for (;;) {
-        if (mbar_poll_run(bar, parity, sleep_ns)) return true;
         if (*abort_flag) return false;
-        if (global_timer_ns() - t0 > kWaitLimitNs) break;
+        if (mbar_poll_run(bar, parity, sleep_ns)) return true;
+        if (global_timer_ns() - t0 > limit_ns) break;
     }
-    *abort_flag = 1;
+    raise_abort_cluster(abort_flag);
     return false;
 }
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
     return mbar_wait_sleep(bar, parity, abort_flag, 0);
+}
+// The wait of an unwinding producer for the copies it has armed (so that none lands after the CTA has
+// left): bounded like the others, with a flag of its own that nobody raises, and no word to the peers.
+__device__ __forceinline__ bool mbar_wait_drain(uint64_t* bar, uint32_t parity, volatile int* drain_flag) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const uint64_t t0 = global_timer_ns();
+    for (;;) {
+        if (mbar_poll_run(bar, parity, 0)) return true;
+        if (global_timer_ns() - t0 > kWaitLimitNs) break;
+    }
+    *drain_flag = 1;
+    return false;
 }
 // Same wait for threads that wait long and whose reaction time matters little.
 __device__ __forceinline__ bool mbar_wait_backoff(uint64_t* bar, uint32_t parity, volatile int* abort_flag,

@@ -35,3 +35,22 @@ def assert_close(got, want, dtype, what=""):
         assert rel_l2 <= BF16_REL_L2, f"{what}: rel-L2 {rel_l2:.3e} > {BF16_REL_L2}"
         assert max_abs <= BF16_MAX_ABS, f"{what}: max-abs {max_abs:.3e} > {BF16_MAX_ABS}"
     return rel_l2, max_abs
+
+
+class Guarded:
+    """A device buffer between two guard bands (a page of 0xA5 bytes before and after it): a store that
+    strays past either end of an output or a workspace shows up in check()."""
+    GUARD = 4096
+
+    def __init__(self, shape, dtype, device="cuda", fill_byte=0xFF):
+        n = int(np.prod(shape)) * torch.empty((), dtype=dtype).element_size()
+        self.nbytes = n
+        self.raw = torch.full((2 * self.GUARD + ((n + 255) & ~255),), 0xA5, dtype=torch.uint8, device=device)
+        body = self.raw[self.GUARD:self.GUARD + n]
+        body.fill_(fill_byte)                    # NaN bit patterns for the floating-point types
+        self.t = body.view(dtype).view(shape)
+
+    def check(self, what=""):
+        g = self.GUARD
+        assert bool((self.raw[:g] == 0xA5).all()), f"{what}: bytes before the buffer were overwritten"
+        assert bool((self.raw[g + self.nbytes:] == 0xA5).all()), f"{what}: bytes behind the buffer were overwritten"

@@ -5,7 +5,7 @@ import pytest
 import torch
 
 from paper_2506_17286_b200 import inputs as I
-from tests.parity_utils import assert_close, oracle_shape
+from tests.parity_utils import Guarded, assert_close, oracle_shape
 
 pytestmark = pytest.mark.gpu
 
@@ -26,17 +26,21 @@ def _run_layer(B, w, t, chunks, s_cap, rope_base):
     k_cache = torch.full((w.batch, w.n_k, s_cap, w.d_h), float("nan"), device="cuda", dtype=torch.bfloat16)
     c_cache = torch.full((w.batch, w.n_c, s_cap, w.d_l), float("nan"), device="cuda", dtype=torch.bfloat16)
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
-    us, pos0 = [], 0
+    us, pos0, guards = [], 0, []
     for n in chunks:
         x = t["x"][:, pos0:pos0 + n].contiguous()
         shape = B.make_shape(batch=w.batch, seq=n, d_model=w.d_model, n_heads=w.n_heads, n_q=w.n_q, n_k=w.n_k,
                              n_c=w.n_c, d_h=w.d_h, d_l=w.d_l, dtype=torch.bfloat16)
-        ws = torch.full((B.layer_prefill_workspace_bytes(shape),), 0xFF, dtype=torch.uint8, device="cuda")
+        ws = Guarded((B.layer_prefill_workspace_bytes(shape),), torch.uint8)
+        ug = Guarded((w.batch, n, w.d_model), torch.bfloat16)
         us.append(B.gta_layer_prefill(x, t["w_qkc"], t["w_p"], t["w_g"], t["w_o"], k_cache, c_cache, pos0=pos0,
-                                      rope_base=rope_base, n_q=w.n_q, workspace=ws, status_word=status))
+                                      rope_base=rope_base, n_q=w.n_q, workspace=ws.t, out=ug.t, status_word=status))
+        guards += [ws, ug]
         pos0 += n
     torch.cuda.synchronize()
     assert int(status.item()) == 0
+    for g in guards:
+        g.check(w.name)
     # rows behind the last written position are untouched, everything before is written
     assert torch.isnan(k_cache[:, :, pos0:]).all() and torch.isnan(c_cache[:, :, pos0:]).all()
     assert not torch.isnan(k_cache[:, :, :pos0]).any() and not torch.isnan(c_cache[:, :, :pos0]).any()

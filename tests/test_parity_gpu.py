@@ -6,7 +6,7 @@ import pytest
 import torch
 
 from paper_2506_17286_b200 import inputs as I
-from tests.parity_utils import assert_close, cpu, oracle_shape
+from tests.parity_utils import Guarded, assert_close, cpu, oracle_shape
 
 pytestmark = pytest.mark.gpu
 
@@ -26,12 +26,15 @@ def _prefill_case(B, oracle, w, causal=True, rows=None, scale=0.0, project=True)
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
     shape = B.make_shape(batch=w.batch, seq=w.seq, d_model=w.d_model, n_heads=w.n_heads, n_q=w.n_q, n_k=w.n_k,
                          n_c=w.n_c, d_h=w.d_h, d_l=w.d_l, dtype=w.torch_dtype())
-    # a workspace full of NaN bit patterns: nothing may be read before the library wrote it
-    ws = torch.full((B.prefill_workspace_bytes(shape),), 0xFF, dtype=torch.uint8, device="cuda")
+    # a workspace full of NaN bit patterns: nothing may be read before the library wrote it; guard bands
+    # around the workspace and the output: nothing may be written outside them
+    ws = Guarded((B.prefill_workspace_bytes(shape),), torch.uint8)
+    og = Guarded((w.batch, w.seq, w.n_heads, w.d_h), w.torch_dtype())
     out = B.gta_prefill(t["q"], t["k"], t["c"], t["x"], t["w_p"], t["w_g"], causal=causal,
-                        softmax_scale=scale, status_word=status, workspace=ws)
+                        softmax_scale=scale, status_word=status, workspace=ws.t, out=og.t)
     torch.cuda.synchronize()
     assert int(status.item()) == 0
+    ws.check(w.name + " workspace"); og.check(w.name + " out")
     tc = cpu(t)
     want = oracle.prefill(oracle_shape(w, causal=int(causal), scale=scale), tc["q"], tc["k"], tc["c"], tc["x"],
                           tc["w_p"], tc["w_g"], rows=rows)
@@ -194,11 +197,13 @@ def _decode_case(B, oracle, w, seq_lens=None, s_cap=None, sample=None):
     t = _nan_behind_the_live_rows(I.decode_inputs(w, device="cuda", s_cap=s_cap, seq_lens=seq_lens))
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
     shape = B.decode_shape(t["q"], t["k_cache"], t["c_cache"], t["x_t"], t["w_p"])
-    ws = torch.full((B.decode_workspace_bytes(shape, t["s_cap"]),), 0xFF, dtype=torch.uint8, device="cuda")
+    ws = Guarded((B.decode_workspace_bytes(shape, t["s_cap"]),), torch.uint8)
+    og = Guarded((w.batch, w.n_heads, w.d_h), w.torch_dtype())
     out = B.gta_decode(t["q"], t["k_cache"], t["c_cache"], t["seq_lens"], t["x_t"], t["w_p"], t["w_g"],
-                       status_word=status, workspace=ws)
+                       status_word=status, workspace=ws.t, out=og.t)
     torch.cuda.synchronize()
     assert int(status.item()) == 0
+    ws.check(w.name + " workspace"); og.check(w.name + " out")
     idx = list(range(w.batch)) if sample is None else sample
     sel = torch.as_tensor(idx, device="cuda", dtype=torch.long)
     lens = t["seq_lens"][sel].cpu().numpy()
@@ -485,3 +490,33 @@ def test_block_table_entry_outside_the_pool_raises_the_status_word(B, page_size)
     assert int(status.item()) == B.GTA_ERR_BAD_PAGE
     changed = (t["k_pool"] != before_k).flatten(1).any(1).sum().item()
     assert changed == 2   # the two good sequences wrote one row each, each in a page of its own
+
+
+# --------------------------------------------------------------------------- bounded waits
+def test_a_wait_that_runs_out_unwinds_the_attention_kernel(B, oracle):
+    """With the test hook one softmax warp of every CTA pair keeps its first arrival to itself and the waits
+    give up after 2 ms: the call must come back (no hang), report GTA_ERR_TIMEOUT in the status word, leave the
+    context usable, and the next ordinary call must give bit for bit what the call before gave."""
+    w = I.Workload("timeout", "prefill", "bf16", 1, 200, 128, 4, 1, 1, 1, 128, 256, seed=99)   # one item, two key tiles
+    t = I.prefill_inputs(w, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    args = (t["q"], t["k"], t["c"], t["x"], t["w_p"], t["w_g"])
+    before = B.gta_prefill(*args, status_word=status).clone()
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    B.debug_attention_wait(limit_ns=2_000_000, withhold_first_arrive=True)
+    try:
+        junk = B.gta_prefill(*args, status_word=status)
+        torch.cuda.synchronize()                      # returns: every wait is bounded
+        assert int(status.item()) == B.GTA_ERR_TIMEOUT
+        del junk
+    finally:
+        B.debug_attention_wait(limit_ns=0, withhold_first_arrive=False)
+    status.zero_()
+    after = B.gta_prefill(*args, status_word=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    assert torch.equal(after.view(torch.int16), before.view(torch.int16))
+    tc = cpu(t)
+    want = oracle.prefill(oracle_shape(w), tc["q"], tc["k"], tc["c"], tc["x"], tc["w_p"], tc["w_g"])
+    assert_close(after, want, torch.bfloat16, "after a timed-out call")
