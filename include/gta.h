@@ -306,6 +306,32 @@ GTA_API gta_status_t gta_decode_static(const gta_shape_t *shape, const void *q, 
                                        int32_t *status_word, void *cuda_stream);
 
 /*
+ * Comparison operators of the paper, in the same harness: grouped-query attention (App. B.3, "GQA",
+ * definition; with n_k_groups = n_heads it is the multi-head attention of Sec. 3.1), so that the
+ * ratios the paper states analytically (Table 3; Sec. 4.3: 37.5 % of the attention cost, 30 % of
+ * the cache at the 1B hyper-parameters) can be measured on the same kernels:
+ *     o[b, i, t] = sum_{j <= t} Softmax_j(q[b, i, t] . k[b, kv(i), j] * scale) v[b, kv(i), j]
+ * with kv(i) = floor(i * n_kv / n_h): contiguous blocks of query heads per key / value head, the
+ * same reading as for the maps of GTA (App. B.3 prints i mod n_kv, which is this operator with
+ * the query heads renumbered).  Of the shape only batch, seq (prefill), n_heads, n_k_groups (the
+ * number of key / value heads), head_dim, causal, dtype and softmax_scale are read.
+ *   gta_ref_gqa_prefill:  q [B, n_h, N, d_h]; k, v [B, n_kv, N, d_h]; out [B, n_h, N, d_h] (head-major).
+ *   gta_ref_gqa_decode:   q [B, n_h, d_h]; k_cache, v_cache [B, n_kv, S_cap, d_h]; seq_lens device
+ *     int32 [B] counting the new token (already in the caches); out [B, n_h, d_h]; a sequence of
+ *     length 0 gives zeros.  workspace: gta_ref_gqa_decode_workspace_bytes(shape), 256-byte aligned.
+ * bf16 with d_h = 64 or 128 only (decode also: at most 8 query heads per key / value head,
+ * B * n_kv <= 512); anything else returns GTA_ERR_UNSUPPORTED.  Status word, stream and error
+ * behaviour as for gta_prefill / gta_decode.
+ */
+GTA_API gta_status_t gta_ref_gqa_prefill(const gta_shape_t *shape, const void *q, const void *k, const void *v,
+                                         void *out, int32_t *status_word, void *cuda_stream);
+GTA_API size_t gta_ref_gqa_decode_workspace_bytes(const gta_shape_t *shape);
+GTA_API gta_status_t gta_ref_gqa_decode(const gta_shape_t *shape, const void *q, const void *k_cache,
+                                        const void *v_cache, const int32_t *seq_lens, int32_t S_cap,
+                                        void *out, void *workspace, size_t workspace_bytes,
+                                        int32_t *status_word, void *cuda_stream);
+
+/*
  * Profiling aids (no counterpart in the paper): the same calls restricted to a subset of their
  * kernels, so that each kernel can be timed or captured alone.  `stages` is a bit mask;
  * gta_prefill_stages: 1 = attention kernel (writes L to the workspace), 2 = decoder + gate

@@ -27,6 +27,7 @@ EXPORTS = (
     "gta_decode_paged_workspace_bytes", "gta_decode_paged", "gta_cache_append_paged",
     "gta_layer_prefill_workspace_bytes", "gta_layer_prefill", "gta_layer_decode_workspace_bytes", "gta_layer_decode",
     "gta_layer_decode_paged_workspace_bytes", "gta_layer_decode_paged", "gta_debug_attention_wait",
+    "gta_ref_gqa_prefill", "gta_ref_gqa_decode_workspace_bytes", "gta_ref_gqa_decode",
 )
 
 
@@ -103,6 +104,12 @@ def lib():
         L.gta_prefill_path.argtypes = [sp]
         L.gta_prefill_path.restype = i32
         L.gta_last_launch_count.restype = i32
+        L.gta_ref_gqa_prefill.argtypes = [sp, vp, vp, vp, vp, vp, vp]
+        L.gta_ref_gqa_prefill.restype = i32
+        L.gta_ref_gqa_decode_workspace_bytes.argtypes = [sp]
+        L.gta_ref_gqa_decode_workspace_bytes.restype = sz
+        L.gta_ref_gqa_decode.argtypes = [sp, vp, vp, vp, vp, i32, vp, vp, sz, vp, vp]
+        L.gta_ref_gqa_decode.restype = i32
         L.gta_debug_attention_wait.argtypes = [ctypes.c_uint64, i32]
         L.gta_debug_attention_wait.restype = i32
         _lib = L
@@ -474,6 +481,58 @@ def gta_cache_append_paged(k_pool, c_pool, block_table, k_new, c_new, seq_lens, 
     if st != GTA_OK:
         raise GtaError(st, "gta_cache_append_paged")
     return seq_lens
+
+
+def gqa_shape(*, batch, seq, n_heads, n_kv, d_h, dtype, causal=True, softmax_scale=0.0) -> GtaShape:
+    """Shape of the comparison operators: only batch, seq, n_heads, n_k (key / value heads), d_h are read."""
+    return make_shape(batch=batch, seq=seq, d_model=8, n_heads=n_heads, n_q=n_heads, n_k=n_kv, n_c=n_kv, d_h=d_h,
+                      d_l=d_h, dtype=dtype, causal=causal, softmax_scale=softmax_scale)
+
+
+def gta_ref_gqa_prefill(q, k, v, *, causal=True, softmax_scale=0.0, out=None, status_word=None, stream=None):
+    """Grouped-query attention (App. B.3 of the paper), the comparison operator: q [B, n_h, N, d_h],
+    k, v [B, n_kv, N, d_h] -> out [B, n_h, N, d_h]."""
+    _check_tensors(q, k, v)
+    B, n_h, N, d_h = q.shape
+    n_kv = k.shape[1]
+    if k.shape != (B, n_kv, N, d_h) or v.shape != k.shape:
+        raise ValueError("inconsistent tensor shapes")
+    shape = gqa_shape(batch=B, seq=N, n_heads=n_h, n_kv=n_kv, d_h=d_h, dtype=_dtype_code(q), causal=causal,
+                      softmax_scale=softmax_scale)
+    if out is None:
+        out = torch.empty((B, n_h, N, d_h), dtype=q.dtype, device=q.device)
+    st = lib().gta_ref_gqa_prefill(ctypes.byref(shape), _ptr(q), _ptr(k), _ptr(v), _ptr(out), _ptr(status_word),
+                                   _stream(stream))
+    if st != GTA_OK:
+        raise GtaError(st, "gta_ref_gqa_prefill")
+    return out
+
+
+def gqa_decode_workspace_bytes(shape: GtaShape) -> int:
+    return int(lib().gta_ref_gqa_decode_workspace_bytes(ctypes.byref(shape)))
+
+
+def gta_ref_gqa_decode(q, k_cache, v_cache, seq_lens, *, softmax_scale=0.0, out=None, workspace=None, status_word=None,
+                       stream=None):
+    """One decode step of grouped-query attention: q [B, n_h, d_h], caches [B, n_kv, S_cap, d_h], seq_lens int32 [B]
+    (counting the new token) -> out [B, n_h, d_h]."""
+    _check_tensors(q, k_cache, v_cache)
+    B, n_h, d_h = q.shape
+    n_kv, s_cap = k_cache.shape[1], k_cache.shape[2]
+    if k_cache.shape != (B, n_kv, s_cap, d_h) or v_cache.shape != k_cache.shape or seq_lens.shape != (B,) \
+            or seq_lens.dtype != torch.int32:
+        raise ValueError("inconsistent tensor shapes")
+    shape = gqa_shape(batch=B, seq=0, n_heads=n_h, n_kv=n_kv, d_h=d_h, dtype=_dtype_code(q), softmax_scale=softmax_scale)
+    if out is None:
+        out = torch.empty((B, n_h, d_h), dtype=q.dtype, device=q.device)
+    if workspace is None:
+        workspace = _workspace(gqa_decode_workspace_bytes(shape), q.device)
+    st = lib().gta_ref_gqa_decode(ctypes.byref(shape), _ptr(q), _ptr(k_cache), _ptr(v_cache), _ptr(seq_lens), int(s_cap),
+                                  _ptr(out), _ptr(workspace), workspace.numel() * workspace.element_size(),
+                                  _ptr(status_word), _stream(stream))
+    if st != GTA_OK:
+        raise GtaError(st, "gta_ref_gqa_decode")
+    return out
 
 
 def _gcd(a, b):

@@ -468,3 +468,77 @@ static gta_status_t append_impl(const gta_shape_t* shape, void* k_cache, void* c
     g_last_launches = launches;
     return GTA_OK;
 }
+
+// ---- comparison operators of the paper (App. B.3, GQA; with one key / value head per query head, the MHA of
+//      Sec. 3.1) on the same tensor-core attention kernel and the same stream / merge kernels
+static gta_status_t gqa_check(const gta_shape_t* s, bool need_seq, float* scale) {
+    if (!s) return GTA_ERR_INVALID_ARG;
+    if (s->batch < 0 || (need_seq && s->seq < 0) || s->n_heads < 1 || s->n_k_groups < 1 || s->head_dim < 1)
+        return GTA_ERR_INVALID_ARG;
+    if (s->n_heads % s->n_k_groups) return GTA_ERR_INVALID_ARG;
+    if (s->dtype != GTA_F32 && s->dtype != GTA_BF16) return GTA_ERR_INVALID_ARG;
+    if (s->causal != 0 && s->causal != 1) return GTA_ERR_INVALID_ARG;
+    if (!(s->softmax_scale >= 0.f) || isinf(s->softmax_scale)) return GTA_ERR_INVALID_ARG;
+    if (s->dtype != GTA_BF16 || (s->head_dim != 64 && s->head_dim != 128) || s->batch > 65535 || s->n_heads > 65535)
+        return GTA_ERR_UNSUPPORTED;
+    *scale = s->softmax_scale > 0.f ? s->softmax_scale : 1.0f / sqrtf((float)s->head_dim);
+    return GTA_OK;
+}
+
+extern "C" gta_status_t gta_ref_gqa_prefill(const gta_shape_t* shape, const void* q, const void* k, const void* v,
+                                            void* out, int32_t* status_word, void* cuda_stream) {
+    g_last_launches = 0;
+    float scale = 0.f;
+    gta_status_t st = gqa_check(shape, true, &scale);
+    if (st != GTA_OK) return st;
+    if (!q || !k || !v || !out) return GTA_ERR_INVALID_ARG;
+    if (!aligned(q, 16) || !aligned(k, 16) || !aligned(v, 16) || !aligned(out, 16) || !aligned(status_word, 4))
+        return GTA_ERR_INVALID_ARG;
+    if (shape->batch == 0 || shape->seq == 0) return GTA_OK;
+    if ((st = check_device()) != GTA_OK) return st;
+    // one attention map per query head; the value heads take the place of the latent (d_h wide, one "latent
+    // group" per key / value head); the attention kernel's normalised output is the operator's output
+    gta::Dims d = {};
+    d.B = shape->batch; d.N = shape->seq; d.H = 64; d.n_h = shape->n_heads; d.n_q = shape->n_heads;
+    d.n_k = shape->n_k_groups; d.n_c = shape->n_k_groups; d.d_h = shape->head_dim; d.d_l = shape->head_dim;
+    d.causal = shape->causal; d.scale = scale; d.Nk = d.N; d.S = d.N;
+    st = gta::launch_sm100_attention(d, q, k, v, out, status_word, static_cast<cudaStream_t>(cuda_stream));
+    if (st != GTA_OK) return st;
+    g_last_launches = 1;
+    return GTA_OK;
+}
+
+extern "C" size_t gta_ref_gqa_decode_workspace_bytes(const gta_shape_t* shape) {
+    float scale = 0.f;
+    if (gqa_check(shape, false, &scale) != GTA_OK) return 0;
+    if (!gta::gqa_decode_supported(shape->batch, shape->n_heads, shape->n_k_groups, shape->head_dim, shape->dtype)) return 0;
+    return gta::gqa_decode_workspace_bytes(shape->batch, shape->n_heads, shape->n_k_groups, shape->head_dim);
+}
+
+extern "C" gta_status_t gta_ref_gqa_decode(const gta_shape_t* shape, const void* q, const void* k_cache,
+                                           const void* v_cache, const int32_t* seq_lens, int32_t S_cap, void* out,
+                                           void* workspace, size_t workspace_bytes, int32_t* status_word,
+                                           void* cuda_stream) {
+    g_last_launches = 0;
+    float scale = 0.f;
+    gta_status_t st = gqa_check(shape, false, &scale);
+    if (st != GTA_OK) return st;
+    if (S_cap <= 0) return GTA_ERR_INVALID_ARG;
+    if (!q || !k_cache || !v_cache || !seq_lens || !out) return GTA_ERR_INVALID_ARG;
+    if (!aligned(q, 16) || !aligned(k_cache, 16) || !aligned(v_cache, 16) || !aligned(out, 16) ||
+        !aligned(seq_lens, 4) || !aligned(status_word, 4))
+        return GTA_ERR_INVALID_ARG;
+    if (!gta::gqa_decode_supported(shape->batch, shape->n_heads, shape->n_k_groups, shape->head_dim, shape->dtype))
+        return GTA_ERR_UNSUPPORTED;
+    if (shape->batch == 0) return GTA_OK;
+    if (!workspace || !aligned(workspace, 256) || workspace_bytes < gta_ref_gqa_decode_workspace_bytes(shape))
+        return GTA_ERR_WORKSPACE;
+    if ((st = check_device()) != GTA_OK) return st;
+    int launches = 0;
+    cudaError_t err = gta::launch_gqa_decode(shape->batch, shape->n_heads, shape->n_k_groups, shape->head_dim, scale, q,
+                                             k_cache, v_cache, seq_lens, S_cap, out, workspace, status_word,
+                                             static_cast<cudaStream_t>(cuda_stream), &launches);
+    if (err != cudaSuccess) return GTA_ERR_CUDA;
+    g_last_launches = launches;
+    return GTA_OK;
+}

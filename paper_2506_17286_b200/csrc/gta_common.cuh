@@ -106,6 +106,13 @@ gta_status_t decode_check_args(const gta_shape_t* shape, const void* q, const vo
 // GTA_OK when the current device is one the kernels are built for, GTA_ERR_UNSUPPORTED otherwise.
 gta_status_t check_current_device();
 
+// Comparison operator (App. B.3, GQA / Sec. 3.1, MHA): one decode step on the stream and merge kernels.
+bool gqa_decode_supported(int B, int n_h, int n_kv, int d_h, int dtype);
+size_t gqa_decode_workspace_bytes(int B, int n_h, int n_kv, int d_h);
+cudaError_t launch_gqa_decode(int B, int n_h, int n_kv, int d_h, float scale, const void* q, const void* k_cache,
+                              const void* v_cache, const int32_t* seq_lens, int S_cap, void* out, void* workspace,
+                              int32_t* status_word, cudaStream_t stream, int* launches);
+
 cudaError_t launch_cache_append(const Dims& d, int elem_size, void* k_cache, void* c_cache, int S_cap,
                                 const void* k_new, const void* c_new, int n_new, int32_t* seq_lens,
                                 int32_t* status_word, cudaStream_t stream, int* launches,

@@ -44,7 +44,7 @@ static size_t align256f(size_t v) { return (v + 255) & ~(size_t)255; }
 bool decode_fast_supported(const Dims& d, int dtype, int page_size) {
     if (dtype != GTA_BF16 || (d.d_h != 128 && d.d_h != 64)) return false;
     if (page_size % kStreamMaxT != 0) return false;              // a sub-tile never straddles two pages
-    if (d.d_l != 128 && d.d_l != 256 && d.d_l != 512 && d.d_l != 1024) return false;
+    if (d.d_l != 64 && d.d_l != 128 && d.d_l != 256 && d.d_l != 512 && d.d_l != 1024) return false;
     if (d.n_q < 1 || d.n_q > 8) return false;                    // the maps are the rows of the warp-level MMAs
     if (d.n_k != 1 && d.n_k != 2 && d.n_k != 4 && d.n_k != 8) return false;   // key groups are dealt to the 8 warps
     if (d.H % 64 != 0 || d.B > kStreamMaxBatch) return false;
@@ -82,7 +82,7 @@ static FastPlan make_fast_plan(const Dims& d) {
     // Narrow caches (a 64-token sub-tile within 32 KB): two CTAs per SM with half-size ring stages.  The
     // work per byte is the same, but a sub-tile is small against its fixed latency chain (barrier,
     // score -> softmax -> latent sum), which two independent CTAs on an SM hide behind one another.
-    p.occ = (d.d_l == 128 && kStreamMaxT * tok_bytes <= kStreamStageBytes / 2) ? 2 : 1;
+    p.occ = (d.d_l <= 128 && kStreamMaxT * tok_bytes <= kStreamStageBytes / 2) ? 2 : 1;
     while (t * 2 * tok_bytes <= kStreamStageBytes / p.occ && t * 2 <= kStreamMaxT) t *= 2;
     p.T = t;
     const int ctas = p.occ * sm_count();
@@ -402,14 +402,21 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
                         const uint32_t a0 = mine ? pa[kt][0] : 0u, a2 = mine ? pa[kt][1] : 0u;
                         const int token = 16 * kt + (mat & 1) * 8 + mrow;
                         const uint32_t crow = cbase + token * 128;
+                        if constexpr (NT == 1) {     // 64 latent columns: one 8-column n-tile per warp
+                            const int chunk = warp;   // 16-byte chunk of the latent row
+                            uint32_t c0, c1;
+                            ptx::ldsm_x2_trans(crow + (((chunk & 7) ^ (token & 7)) << 4), c0, c1);
+                            ptx::mma_bf16_16816(acc[0], a0, 0u, a2, 0u, c0, c1);
+                        } else {
 #pragma unroll
-                        for (int np = 0; np < NT / 2; ++np) {
-                            const int chunk = warp * NT + 2 * np + (mat >> 1);   // 16-byte chunk of the latent row
-                            uint32_t c0, c1, c2, c3;
-                            ptx::ldsm_x4_trans(crow + (chunk >> 3) * tile_bytes + (((chunk & 7) ^ (token & 7)) << 4),
-                                               c0, c1, c2, c3);
-                            ptx::mma_bf16_16816(acc[2 * np], a0, 0u, a2, 0u, c0, c1);
-                            ptx::mma_bf16_16816(acc[2 * np + 1], a0, 0u, a2, 0u, c2, c3);
+                            for (int np = 0; np < NT / 2; ++np) {
+                                const int chunk = warp * NT + 2 * np + (mat >> 1);   // 16-byte chunk of the latent row
+                                uint32_t c0, c1, c2, c3;
+                                ptx::ldsm_x4_trans(crow + (chunk >> 3) * tile_bytes + (((chunk & 7) ^ (token & 7)) << 4),
+                                                   c0, c1, c2, c3);
+                                ptx::mma_bf16_16816(acc[2 * np], a0, 0u, a2, 0u, c0, c1);
+                                ptx::mma_bf16_16816(acc[2 * np + 1], a0, 0u, a2, 0u, c2, c3);
+                            }
                         }
                     }
                 }
@@ -425,8 +432,9 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
 
 // ---------------------------------------------------------------------------------------------
 // Log-sum-exp merge of the split-KV slots of one (attention map, sequence) pair per
-// CTA into the normalised latent L[n_q][B][d_l] (bf16), which the tcgen05 decoder + gate kernel of
-// the prefill path then consumes with the batch in the role of the token axis.
+// CTA into the normalised latent (bf16), row (g, b) at l_out + g stride_g + b stride_b: L[n_q][B][d_l] for the
+// tcgen05 decoder + gate kernel of the prefill path, which then consumes it with the batch in the role of the
+// token axis (the comparison operators take it head by head as their output).
 // Launched with programmatic stream serialisation: while the stream kernel still runs, the CTA
 // works out from the sequence lengths (inputs, not results of that kernel) which stream CTAs own
 // sub-tiles of its sequence -- the same arithmetic as in the stream kernel: prefix sums of
@@ -435,7 +443,7 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
 __global__ void __launch_bounds__(256)
 decode_merge_kernel(Dims d, int G, int T, int S_cap, const int32_t* __restrict__ seq_lens,
                     const float* __restrict__ part_o, const float* __restrict__ part_ml,
-                    __nv_bfloat16* __restrict__ l_out) {
+                    __nv_bfloat16* __restrict__ l_out, long long stride_g, long long stride_b) {
     __shared__ long long red_s[2][8];
     __shared__ int live_s[kFinMaxSlots];        // slot j of the range holds something
     ptx::grid_launch_dependents();
@@ -508,18 +516,17 @@ decode_merge_kernel(Dims d, int G, int T, int S_cap, const int32_t* __restrict__
     uint2 packed;
     packed.x = pack_bf16(acc.x * inv_l, acc.y * inv_l);
     packed.y = pack_bf16(acc.z * inv_l, acc.w * inv_l);
-    *reinterpret_cast<uint2*>(l_out + ((size_t)g * d.B + b) * d.d_l + col) = packed;
+    *reinterpret_cast<uint2*>(l_out + g * stride_g + b * stride_b + col) = packed;
 }
 
 // ---------------------------------------------------------------------------------------------
-cudaError_t launch_decode_fast(const Dims& d, const void* q, const void* k_cache, const void* c_cache,
-                               const int32_t* seq_lens, int S_cap, const void* x_t, const void* w_p,
-                               const void* w_g, void* out, void* workspace, int32_t* status_word,
-                               cudaStream_t stream, int stages, int* launches, const PageMap& pm) {
-    const FastPlan p = make_fast_plan(d);
-    float* part_o = reinterpret_cast<float*>(workspace);
-    float* part_ml = reinterpret_cast<float*>(static_cast<char*>(workspace) + p.off_ml);
-    __nv_bfloat16* l_g = reinterpret_cast<__nv_bfloat16*>(static_cast<char*>(workspace) + p.off_l);
+// Stream kernel (stages & 2) and merge kernel (stages & 4) of one decode step: the normalised latent rows go to
+// l_out (row (g, b) at g stride_g + b stride_b elements).
+static cudaError_t launch_stream_and_merge(const Dims& d, const FastPlan& p, const void* q, const void* k_cache,
+                                           const void* c_cache, const int32_t* seq_lens, int S_cap, float* part_o,
+                                           float* part_ml, __nv_bfloat16* l_out, long long stride_g,
+                                           long long stride_b, int32_t* status_word, cudaStream_t stream, int stages,
+                                           int* launches, const PageMap& pm) {
     cudaError_t err;
     if (stages & 2) {
         CUtensorMap tm_k, tm_c;
@@ -560,16 +567,20 @@ cudaError_t launch_decode_fast(const Dims& d, const void* q, const void* k_cache
             else if (d.n_c == 1) GTA_LAUNCH_STREAM_(NT, 1, true, 1);                                       \
             else GTA_LAUNCH_STREAM_(NT, 1, false, 1);                                                      \
         } while (0)
-#define GTA_LAUNCH_STREAM_NARROW()   /* d_l = 128, two CTAs per SM */                                      \
+#define GTA_LAUNCH_STREAM_NARROW(NT)   /* d_l <= 128, two CTAs per SM */                                   \
         do {                                                                                               \
-            if (d.d_h == 128 && d.n_c == 1) GTA_LAUNCH_STREAM_(2, 2, true, 2);                             \
-            else if (d.d_h == 128) GTA_LAUNCH_STREAM_(2, 2, false, 2);                                     \
-            else if (d.n_c == 1) GTA_LAUNCH_STREAM_(2, 1, true, 2);                                        \
-            else GTA_LAUNCH_STREAM_(2, 1, false, 2);                                                       \
+            if (d.d_h == 128 && d.n_c == 1) GTA_LAUNCH_STREAM_(NT, 2, true, 2);                            \
+            else if (d.d_h == 128) GTA_LAUNCH_STREAM_(NT, 2, false, 2);                                    \
+            else if (d.n_c == 1) GTA_LAUNCH_STREAM_(NT, 1, true, 2);                                       \
+            else GTA_LAUNCH_STREAM_(NT, 1, false, 2);                                                      \
         } while (0)
         switch (d.d_l) {
+            case 64:
+                if (p.occ == 2) GTA_LAUNCH_STREAM_NARROW(1);
+                else GTA_LAUNCH_STREAM(1);
+                break;
             case 128:
-                if (p.occ == 2) GTA_LAUNCH_STREAM_NARROW();
+                if (p.occ == 2) GTA_LAUNCH_STREAM_NARROW(2);
                 else GTA_LAUNCH_STREAM(2);
                 break;
             case 256: GTA_LAUNCH_STREAM(4); break;
@@ -593,16 +604,91 @@ cudaError_t launch_decode_fast(const Dims& d, const void* q, const void* k_cache
         cfg.attrs = attr;
         cfg.numAttrs = 1;
         err = cudaLaunchKernelEx(&cfg, decode_merge_kernel, d, p.G, p.T, S_cap, seq_lens, (const float*)part_o,
-                                 (const float*)part_ml, l_g);
+                                 (const float*)part_ml, l_out, stride_g, stride_b);
         if (err != cudaSuccess) return err;
+        *launches += 1;
+    }
+    return cudaSuccess;
+}
+
+cudaError_t launch_decode_fast(const Dims& d, const void* q, const void* k_cache, const void* c_cache,
+                               const int32_t* seq_lens, int S_cap, const void* x_t, const void* w_p,
+                               const void* w_g, void* out, void* workspace, int32_t* status_word,
+                               cudaStream_t stream, int stages, int* launches, const PageMap& pm) {
+    const FastPlan p = make_fast_plan(d);
+    float* part_o = reinterpret_cast<float*>(workspace);
+    float* part_ml = reinterpret_cast<float*>(static_cast<char*>(workspace) + p.off_ml);
+    __nv_bfloat16* l_g = reinterpret_cast<__nv_bfloat16*>(static_cast<char*>(workspace) + p.off_l);
+    cudaError_t err = launch_stream_and_merge(d, p, q, k_cache, c_cache, seq_lens, S_cap, part_o, part_ml, l_g,
+                                              (long long)d.B * d.d_l, d.d_l, status_word, stream, stages, launches, pm);
+    if (err != cudaSuccess) return err;
+    if (stages & 4) {
         // the batch takes the role of the token axis: L [n_q][B][d_l], x_t [B][H], out [B][n_h][d_h]
         Dims dd = d;
         dd.B = 1;
         dd.N = d.B;
         if (launch_sm100_decoder(dd, l_g, x_t, w_p, w_g, out, status_word, stream) != GTA_OK) return cudaErrorUnknown;
-        *launches += 2;
+        *launches += 1;
     }
     return cudaSuccess;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Comparison operator (App. B.3, GQA; one key / value head per query head gives the multi-head attention of
+// Sec. 3.1): one decode step on the same stream and merge kernels.  Every (sequence, key / value head) pair
+// is streamed as a sequence of its own whose maps are the n_h / n_kv query heads that share the head, whose
+// key group is the head's K rows and whose "latent" is the head's V rows (d_h wide); no decoder, no gate:
+// the merged, normalised rows ARE the output [B, n_h, d_h].
+__global__ void gqa_expand_lens_kernel(const int32_t* __restrict__ seq_lens, int32_t* __restrict__ out, int B, int n_kv) {
+    ptx::grid_dependency_wait();          // the lengths may come from the kernel before (an append)
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < B * n_kv) out[i] = seq_lens[i / n_kv];
+}
+
+static Dims gqa_stream_dims(int B, int n_h, int n_kv, int d_h, float scale) {
+    Dims d = {};
+    d.B = B * n_kv; d.N = 0; d.H = 64; d.n_h = n_h / n_kv; d.n_q = n_h / n_kv; d.n_k = 1; d.n_c = 1;
+    d.d_h = d_h; d.d_l = d_h; d.causal = 1; d.scale = scale; d.Nk = 0; d.S = 0;
+    return d;
+}
+
+bool gqa_decode_supported(int B, int n_h, int n_kv, int d_h, int dtype) {
+    if (dtype != GTA_BF16 || n_kv < 1 || n_h % n_kv != 0 || (d_h != 64 && d_h != 128)) return false;
+    const int r = n_h / n_kv;
+    return r >= 1 && r <= 8 && (long long)B * n_kv <= kStreamMaxBatch;
+}
+
+size_t gqa_decode_workspace_bytes(int B, int n_h, int n_kv, int d_h) {
+    const Dims d = gqa_stream_dims(B, n_h, n_kv, d_h, 1.f);
+    return make_fast_plan(d).off_l + align256f((size_t)d.B * sizeof(int32_t));
+}
+
+cudaError_t launch_gqa_decode(int B, int n_h, int n_kv, int d_h, float scale, const void* q, const void* k_cache,
+                              const void* v_cache, const int32_t* seq_lens, int S_cap, void* out, void* workspace,
+                              int32_t* status_word, cudaStream_t stream, int* launches) {
+    const Dims d = gqa_stream_dims(B, n_h, n_kv, d_h, scale);
+    const FastPlan p = make_fast_plan(d);
+    float* part_o = reinterpret_cast<float*>(workspace);
+    float* part_ml = reinterpret_cast<float*>(static_cast<char*>(workspace) + p.off_ml);
+    int32_t* lens = reinterpret_cast<int32_t*>(static_cast<char*>(workspace) + p.off_l);
+    {
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((d.B + 255) / 256);
+        cfg.blockDim = dim3(256);
+        cfg.stream = stream;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        cudaError_t err = cudaLaunchKernelEx(&cfg, gqa_expand_lens_kernel, seq_lens, lens, B, n_kv);
+        if (err != cudaSuccess) return err;
+        *launches += 1;
+    }
+    // row (g, b') of the merge = query head j r + g of sequence b, b' = b n_kv + j: out + (b' r + g) d_h
+    return launch_stream_and_merge(d, p, q, k_cache, v_cache, lens, S_cap, part_o, part_ml,
+                                   static_cast<__nv_bfloat16*>(out), d.d_l, (long long)d.n_q * d.d_l, status_word, stream,
+                                   6, launches, PageMap());
 }
 
 }  // namespace gta

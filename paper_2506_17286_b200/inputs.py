@@ -185,3 +185,31 @@ def layer_inputs(w: Workload, device="cpu"):
     )
     dev = torch.device(device)
     return {name: t.to(dev).to(dt).contiguous() for name, t in out.items()}
+
+
+def gqa_prefill_inputs(batch, n_heads, n_kv, seq, d_h, seed=0, device="cpu"):
+    """q [B, n_h, N, d_h], k, v [B, n_kv, N, d_h] ~ N(0,1) in bf16 for the comparison operators (drawn on
+    `device` from a generator seeded there: the full-size workloads are too large to draw on the host)."""
+    dev = torch.device(device)
+    gen = torch.Generator(dev).manual_seed(seed)
+
+    def draw(*shape):
+        return torch.randn(shape, generator=gen, dtype=torch.float32, device=dev).to(torch.bfloat16)
+
+    return dict(q=draw(batch, n_heads, seq, d_h), k=draw(batch, n_kv, seq, d_h), v=draw(batch, n_kv, seq, d_h))
+
+
+def gqa_decode_inputs(batch, n_heads, n_kv, d_h, seq_lens, s_cap=None, seed=0, device="cpu"):
+    """q [B, n_h, d_h], k_cache, v_cache [B, n_kv, S_cap, d_h] ~ N(0,1) in bf16 (everywhere, also behind the
+    live lengths), seq_lens int32 [B]."""
+    dev = torch.device(device)
+    gen = torch.Generator(dev).manual_seed(seed)
+    lens = torch.as_tensor(seq_lens, dtype=torch.int32)
+    if s_cap is None:
+        s_cap = int(lens.max().item()) + 64
+
+    def draw(*shape):
+        return torch.randn(shape, generator=gen, dtype=torch.float32, device=dev).to(torch.bfloat16)
+
+    return dict(q=draw(batch, n_heads, d_h), k_cache=draw(batch, n_kv, s_cap, d_h), v_cache=draw(batch, n_kv, s_cap, d_h),
+                seq_lens=lens.to(dev), s_cap=s_cap)
