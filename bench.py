@@ -329,6 +329,8 @@ def run_ours(args):
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=dev)
     G.lib()
+    global MIN_TIMED_MS
+    MIN_TIMED_MS = float(args.min_timed_ms)
     peaks = load_peaks()
     traffic = load_traffic()
     stream = torch.cuda.current_stream()
@@ -350,10 +352,11 @@ def run_ours(args):
         pass
     sampler = ClockSampler(gpu_id)
 
-    def timed_loop(step, n_iter, before_rep=None, min_ms=MIN_TIMED_MS, max_reps=400):
+    def timed_loop(step, n_iter, before_rep=None, min_ms=None, max_reps=400):
         """`n_iter` calls of step(i) between two CUDA events, repeated until `min_ms` of device time
         have been measured (at least 3 repetitions); `before_rep` runs untimed before each repetition.
         Returns (median ms per call over the repetitions, max over ranks; record of the loop)."""
+        min_ms = MIN_TIMED_MS if min_ms is None else min(min_ms, MIN_TIMED_MS)
         if before_rep:
             before_rep()
         for i in range(3):
@@ -503,6 +506,20 @@ def run_ours(args):
     clk_k = sampler.window(t0k, time.time())
     t_attn, t_dec_k = mx(statistics.median(acc["attn"])), mx(statistics.median(acc["dec"]))
     assert int(status.item()) == 0, "device status word raised during the benchmark"
+
+    if args.step_only:
+        # the timed region alone (for a profiler's launch list of exactly the kernels of a step): a short line
+        if rank == 0:
+            fl_ = prefill_flops(wp)
+            print(json.dumps({"metric": METRIC, "value": whole_job_rate(fl_["total"], world, t_prefill) / 1e12,
+                              "unit": UNIT, "n_gpus": world, "steps": K, "warmup": args.warmup,
+                              "ms_per_step": total_ms / K, "step_only": True,
+                              "kernels_ms": {"prefill_attention": t_attn, "prefill_decoder_gate": t_dec_k,
+                                             "decode_leg": t_decode_leg}, "gpu_launches": n_launches}))
+        sampler.stop()
+        if dist is not None:
+            dist.destroy_process_group()
+        return 0
 
     # ---- decode leg alone, back to back (append + decode, alternating cache sets): the figure the
     #      decode roofline is quoted on; launch gaps between calls are inside the timed region
@@ -898,6 +915,10 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--step-only", action="store_true",
+                    help="run the timed region and the per-kernel loop only and print a short line (for a launch list)")
+    ap.add_argument("--min-timed-ms", type=float, default=MIN_TIMED_MS,
+                    help="device time every timed loop is repeated up to (lower it for a profiler's launch list)")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
