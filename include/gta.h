@@ -306,6 +306,35 @@ GTA_API gta_status_t gta_decode_static(const gta_shape_t *shape, const void *q, 
                                        int32_t *status_word, void *cuda_stream);
 
 /*
+ * 8-bit caches (the paper has no such format; Sec. 5.3 and App. C.2 only observe that the decode
+ * step is bound by the bytes of the cache, the larger the context and the slower the memory the
+ * more).  Reading taken here: K and C rows are kept as e4m3 codes (8-bit floats: 1 sign, 4
+ * exponent, 3 mantissa bits, bias 7, no infinities, largest value 448) with ONE fp32 scale per
+ * cached row (token and group):
+ *     scale = max|row| / 448 (1 for an all-zero row),  code = round-to-nearest-even(x / scale),
+ * both divisions in fp32, magnitudes saturating at 448; the operator runs on code * scale.
+ *   k_codes uint8 [B, n_k, S_cap, d_h]   k_scales float [B, n_k, S_cap]
+ *   c_codes uint8 [B, n_c, S_cap, d_l]   c_scales float [B, n_c, S_cap]
+ * gta_cache_append_fp8 quantises k_new [B, n_k, n_new, d_h] / c_new [B, n_c, n_new, d_l] (in the
+ * shape's dtype) into rows [len, len + n_new) and advances seq_lens, with the overflow rule of
+ * gta_cache_append; codes and scales are bit-exact functions of the new rows.  gta_decode_fp8 is
+ * gta_decode over such caches (q, x_t, w_p, w_g, out in the shape's dtype; rows at and behind
+ * seq_lens[b] may hold anything).  Needs d_h and d_l multiples of 16, d_l <= 2048; contiguous
+ * caches only.  These calls run on the plain-ALU kernels: they halve the cache but are not at the
+ * HBM roofline (the measured figures are in the benchmark's output).
+ */
+GTA_API size_t gta_decode_fp8_workspace_bytes(const gta_shape_t *shape, int32_t S_cap);
+GTA_API gta_status_t gta_cache_append_fp8(const gta_shape_t *shape, void *k_codes, void *c_codes,
+                                          float *k_scales, float *c_scales, int32_t S_cap,
+                                          const void *k_new, const void *c_new, int32_t n_new,
+                                          int32_t *seq_lens, int32_t *status_word, void *cuda_stream);
+GTA_API gta_status_t gta_decode_fp8(const gta_shape_t *shape, const void *q, const void *k_codes,
+                                    const void *c_codes, const float *k_scales, const float *c_scales,
+                                    const int32_t *seq_lens, int32_t S_cap, const void *x_t,
+                                    const void *w_p, const void *w_g, void *out, void *workspace,
+                                    size_t workspace_bytes, int32_t *status_word, void *cuda_stream);
+
+/*
  * Comparison operators of the paper, in the same harness: grouped-query attention (App. B.3, "GQA",
  * definition; with n_k_groups = n_heads it is the multi-head attention of Sec. 3.1), so that the
  * ratios the paper states analytically (Table 3; Sec. 4.3: 37.5 % of the attention cost, 30 % of

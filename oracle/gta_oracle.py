@@ -388,3 +388,86 @@ def gqa_attention_cost(n_heads: int, d_h: int, n: int) -> float:
 def gqa_cache_elems(n_kv: int, d_h: int, n: int) -> float:
     """2 n_k d_h N — Table 3, GQA row, 'KV Cache per Layer' column (App. B.3 decode)."""
     return 2.0 * n_kv * d_h * float(n)
+
+
+# ----------------------------------------------------------------------------------------------
+# Lower-precision caches (the direction of Sec. 5.3 / App. C.2: decode is bound by the bytes of the cache).
+# Reading taken here, the paper fixing none: K and C rows are stored as 8-bit floats of the e4m3 format (1 sign,
+# 4 exponent, 3 mantissa bits, bias 7, no infinities, largest finite value 448; the "fn" variant of the OCP 8-bit
+# floating point specification) with ONE fp32 scale per cached row (token and group):
+#     scale = max|row| / 448   (1 for an all-zero row),   code = round-to-nearest-even_e4m3(x / scale),
+# both divisions in fp32, and the operator then runs unchanged on the dequantised values code * scale.
+def e4m3_table():
+    """Value of each of the 256 e4m3 codes, from the format's definition (codes 0x7f / 0xff are NaN)."""
+    vals = np.zeros(256, dtype=np.float64)
+    for code in range(256):
+        sign = -1.0 if code & 0x80 else 1.0
+        e, m = (code >> 3) & 0xF, code & 0x7
+        if e == 0xF and m == 0x7:
+            vals[code] = np.nan
+        elif e == 0:
+            vals[code] = sign * (m / 8.0) * 2.0 ** -6          # subnormal
+        else:
+            vals[code] = sign * (1.0 + m / 8.0) * 2.0 ** (e - 7)
+    return vals
+
+
+def round_to_e4m3(y):
+    """fp32 values -> e4m3 codes (uint8): nearest representable value, ties to the even code, magnitudes above 448
+    saturate to 448 (no infinities in this format)."""
+    y = np.asarray(y, dtype=np.float32)
+    mags = e4m3_table()[:0x7F]                        # the 127 finite non-negative values, ascending with the code
+    a = np.minimum(np.abs(y).astype(np.float64), 448.0)
+    hi = np.clip(np.searchsorted(mags, a, side="left"), 0, 0x7E)
+    lo = np.maximum(hi - 1, 0)
+    d_hi, d_lo = mags[hi] - a, a - mags[lo]
+    pick_lo = (d_lo < d_hi) | ((d_lo == d_hi) & (lo % 2 == 0))
+    code = np.where(pick_lo, lo, hi).astype(np.uint8)
+    return code | np.where(np.signbit(y), 0x80, 0).astype(np.uint8)
+
+
+def quantize_rows_e4m3(x):
+    """Rows (last axis) of x -> (codes uint8 like x, scales float32 without the last axis)."""
+    xf = _to_f64(x).astype(np.float32)                 # the stored values are exact in fp32 (bf16 / fp32 storage)
+    amax = np.abs(xf).max(axis=-1)
+    scale = np.where(amax > 0, amax / np.float32(448.0), np.float32(1.0)).astype(np.float32)
+    return round_to_e4m3(xf / scale[..., None]), scale
+
+
+def dequantize_e4m3(codes, scales):
+    """float64 values code * scale."""
+    return e4m3_table()[np.asarray(codes, dtype=np.uint8)] * np.asarray(scales, dtype=np.float64)[..., None]
+
+
+def cache_append_fp8(k_codes, k_scales, c_codes, c_scales, k_new, c_new, seq_lens):
+    """Quantising append: rows [len, len + n_new) of every group of sequence b take the codes and scales of
+    k_new [B, n_k, n_new, d_h] / c_new [B, n_c, n_new, d_l]; a sequence whose rows do not fit is skipped (length
+    unchanged).  Returns new arrays (k_codes, k_scales, c_codes, c_scales, seq_lens, overflowed)."""
+    kc, ks, cc, cs = (np.array(a, copy=True) for a in (k_codes, k_scales, c_codes, c_scales))
+    lens = np.array(seq_lens, dtype=np.int32, copy=True)
+    kq, kqs = quantize_rows_e4m3(k_new)
+    cq, cqs = quantize_rows_e4m3(c_new)
+    n_new, cap, overflowed = kq.shape[2], kc.shape[2], 0
+    for b in range(kc.shape[0]):
+        if lens[b] < 0 or lens[b] + n_new > cap:
+            overflowed = 1
+            continue
+        kc[b, :, lens[b]:lens[b] + n_new] = kq[b]; ks[b, :, lens[b]:lens[b] + n_new] = kqs[b]
+        cc[b, :, lens[b]:lens[b] + n_new] = cq[b]; cs[b, :, lens[b]:lens[b] + n_new] = cqs[b]
+        lens[b] += n_new
+    return kc, ks, cc, cs, lens, overflowed
+
+
+def decode_fp8(shape: Shape, q, k_codes, k_scales, c_codes, c_scales, seq_lens, x_t, w_p, w_g, n_threads: int = 0):
+    """The decode step (App. B.1.3) over caches held as e4m3 codes + per-row scales: dequantise in float64, then
+    the unchanged operator oracle.  Rows at and behind seq_lens[b] are never read (they are zeroed here first, so
+    that NaN codes or scales there cannot leak through a 0 * NaN)."""
+    s_cap = k_codes.shape[2]
+    k = dequantize_e4m3(k_codes, k_scales)
+    c = dequantize_e4m3(c_codes, c_scales)
+    for b in range(shape.batch):
+        n = max(0, min(int(seq_lens[b]), s_cap))
+        k[b, :, n:] = 0.0
+        c[b, :, n:] = 0.0
+    return decode(shape, _to_f64(q), np.ascontiguousarray(k), np.ascontiguousarray(c), seq_lens, s_cap, _to_f64(x_t),
+                  _to_f64(w_p), _to_f64(w_g), n_threads=n_threads)

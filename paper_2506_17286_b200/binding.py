@@ -28,6 +28,7 @@ EXPORTS = (
     "gta_layer_prefill_workspace_bytes", "gta_layer_prefill", "gta_layer_decode_workspace_bytes", "gta_layer_decode",
     "gta_layer_decode_paged_workspace_bytes", "gta_layer_decode_paged", "gta_debug_attention_wait",
     "gta_ref_gqa_prefill", "gta_ref_gqa_decode_workspace_bytes", "gta_ref_gqa_decode",
+    "gta_decode_fp8_workspace_bytes", "gta_cache_append_fp8", "gta_decode_fp8",
 )
 
 
@@ -110,6 +111,12 @@ def lib():
         L.gta_ref_gqa_decode_workspace_bytes.restype = sz
         L.gta_ref_gqa_decode.argtypes = [sp, vp, vp, vp, vp, i32, vp, vp, sz, vp, vp]
         L.gta_ref_gqa_decode.restype = i32
+        L.gta_decode_fp8_workspace_bytes.argtypes = [sp, i32]
+        L.gta_decode_fp8_workspace_bytes.restype = sz
+        L.gta_cache_append_fp8.argtypes = [sp, vp, vp, vp, vp, i32, vp, vp, i32, vp, vp, vp]
+        L.gta_cache_append_fp8.restype = i32
+        L.gta_decode_fp8.argtypes = [sp, vp, vp, vp, vp, vp, vp, i32, vp, vp, vp, vp, vp, sz, vp, vp]
+        L.gta_decode_fp8.restype = i32
         L.gta_debug_attention_wait.argtypes = [ctypes.c_uint64, i32]
         L.gta_debug_attention_wait.restype = i32
         _lib = L
@@ -481,6 +488,64 @@ def gta_cache_append_paged(k_pool, c_pool, block_table, k_new, c_new, seq_lens, 
     if st != GTA_OK:
         raise GtaError(st, "gta_cache_append_paged")
     return seq_lens
+
+
+def _check_fp8_caches(k_codes, c_codes, k_scales, c_scales):
+    B, n_k, s_cap, d_h = k_codes.shape
+    n_c, d_l = c_codes.shape[1], c_codes.shape[3]
+    if k_codes.dtype != torch.uint8 or c_codes.dtype != torch.uint8 or k_scales.dtype != torch.float32 \
+            or c_scales.dtype != torch.float32 or c_codes.shape != (B, n_c, s_cap, d_l) \
+            or k_scales.shape != (B, n_k, s_cap) or c_scales.shape != (B, n_c, s_cap):
+        raise ValueError("8-bit caches: codes uint8 [B, groups, S_cap, width], scales float32 [B, groups, S_cap]")
+    for t in (k_codes, c_codes, k_scales, c_scales):
+        if not t.is_contiguous() or t.device.type != "cuda":
+            raise ValueError("cache tensors must be contiguous CUDA tensors")
+    return B, n_k, n_c, s_cap, d_h, d_l
+
+
+def gta_cache_append_fp8(k_codes, c_codes, k_scales, c_scales, k_new, c_new, seq_lens, *, status_word=None, stream=None):
+    """Quantises k_new [B, n_k, n_new, d_h] / c_new [B, n_c, n_new, d_l] to e4m3 codes + per-row scales behind the
+    live rows of the 8-bit caches and advances seq_lens."""
+    B, n_k, n_c, s_cap, d_h, d_l = _check_fp8_caches(k_codes, c_codes, k_scales, c_scales)
+    _check_tensors(k_new, c_new)
+    n_new = k_new.shape[2]
+    if k_new.shape != (B, n_k, n_new, d_h) or c_new.shape != (B, n_c, n_new, d_l):
+        raise ValueError("inconsistent new-row shapes")
+    n_q = n_k * n_c          # any map count that both group counts divide: the append does not look at it
+    shape = make_shape(batch=B, seq=0, d_model=8, n_heads=n_q, n_q=n_q, n_k=n_k, n_c=n_c, d_h=d_h, d_l=d_l,
+                       dtype=_dtype_code(k_new))
+    st = lib().gta_cache_append_fp8(ctypes.byref(shape), _ptr(k_codes), _ptr(c_codes), _ptr(k_scales), _ptr(c_scales),
+                                    int(s_cap), _ptr(k_new), _ptr(c_new), int(n_new), _ptr(seq_lens), _ptr(status_word),
+                                    _stream(stream))
+    if st != GTA_OK:
+        raise GtaError(st, "gta_cache_append_fp8")
+    return seq_lens
+
+
+def decode_fp8_workspace_bytes(shape: GtaShape, s_cap: int) -> int:
+    return int(lib().gta_decode_fp8_workspace_bytes(ctypes.byref(shape), int(s_cap)))
+
+
+def gta_decode_fp8(q, k_codes, c_codes, k_scales, c_scales, seq_lens, x_t, w_p, w_g, *, softmax_scale=0.0, out=None,
+                   workspace=None, status_word=None, stream=None):
+    """gta_decode over 8-bit caches (e4m3 codes + one fp32 scale per cached row)."""
+    B, n_k, n_c, s_cap, d_h, d_l = _check_fp8_caches(k_codes, c_codes, k_scales, c_scales)
+    _check_tensors(q, x_t, w_p, w_g)
+    n_q, n_h, H = q.shape[1], w_p.shape[0], x_t.shape[1]
+    if q.shape != (B, n_q, d_h) or w_p.shape != (n_h, d_l, d_h) or w_g.shape != (H, n_h * d_h) or x_t.shape != (B, H):
+        raise ValueError("inconsistent operator tensor shapes")
+    shape = make_shape(batch=B, seq=0, d_model=H, n_heads=n_h, n_q=n_q, n_k=n_k, n_c=n_c, d_h=d_h, d_l=d_l,
+                       dtype=_dtype_code(q), softmax_scale=softmax_scale)
+    if out is None:
+        out = torch.empty((B, n_h, d_h), dtype=q.dtype, device=q.device)
+    if workspace is None:
+        workspace = _workspace(decode_fp8_workspace_bytes(shape, s_cap), q.device)
+    st = lib().gta_decode_fp8(ctypes.byref(shape), _ptr(q), _ptr(k_codes), _ptr(c_codes), _ptr(k_scales), _ptr(c_scales),
+                              _ptr(seq_lens), int(s_cap), _ptr(x_t), _ptr(w_p), _ptr(w_g), _ptr(out), _ptr(workspace),
+                              workspace.numel() * workspace.element_size(), _ptr(status_word), _stream(stream))
+    if st != GTA_OK:
+        raise GtaError(st, "gta_decode_fp8")
+    return out
 
 
 def gqa_shape(*, batch, seq, n_heads, n_kv, d_h, dtype, causal=True, softmax_scale=0.0) -> GtaShape:

@@ -542,3 +542,69 @@ extern "C" gta_status_t gta_ref_gqa_decode(const gta_shape_t* shape, const void*
     g_last_launches = launches;
     return GTA_OK;
 }
+
+// ---- 8-bit caches (e4m3 codes + one fp32 scale per cached row)
+static gta_status_t fp8_check(const gta_shape_t* shape, gta::Dims* d) {
+    gta_status_t st = check_shape(shape, false, d);
+    if (st != GTA_OK) return st;
+    if (d->d_h % 16 || d->d_l % 16 || d->d_l > 2048) return GTA_ERR_UNSUPPORTED;   // rows are read as 16-byte vectors of codes
+    return GTA_OK;
+}
+
+extern "C" size_t gta_decode_fp8_workspace_bytes(const gta_shape_t* shape, int32_t S_cap) {
+    gta::Dims d;
+    if (fp8_check(shape, &d) != GTA_OK || S_cap < 0) return 0;
+    return gta::decode_fp8_workspace_bytes(d, S_cap);
+}
+
+extern "C" gta_status_t gta_cache_append_fp8(const gta_shape_t* shape, void* k_codes, void* c_codes, float* k_scales,
+                                             float* c_scales, int32_t S_cap, const void* k_new, const void* c_new,
+                                             int32_t n_new, int32_t* seq_lens, int32_t* status_word, void* cuda_stream) {
+    g_last_launches = 0;
+    gta::Dims d;
+    gta_status_t st = fp8_check(shape, &d);
+    if (st != GTA_OK) return st;
+    if (S_cap < 0 || n_new < 0) return GTA_ERR_INVALID_ARG;
+    if (!k_codes || !c_codes || !k_scales || !c_scales || !k_new || !c_new || !seq_lens) return GTA_ERR_INVALID_ARG;
+    if (!aligned(k_codes, 16) || !aligned(c_codes, 16) || !aligned(k_scales, 4) || !aligned(c_scales, 4) ||
+        !aligned(k_new, 16) || !aligned(c_new, 16) || !aligned(seq_lens, 4) || !aligned(status_word, 4))
+        return GTA_ERR_INVALID_ARG;
+    if (d.B == 0 || n_new == 0) return GTA_OK;
+    if ((st = check_device()) != GTA_OK) return st;
+    int launches = 0;
+    cudaError_t err = gta::launch_cache_append_fp8(d, shape->dtype, k_codes, c_codes, k_scales, c_scales, S_cap, k_new,
+                                                   c_new, n_new, seq_lens, status_word,
+                                                   static_cast<cudaStream_t>(cuda_stream), &launches);
+    if (err != cudaSuccess) return GTA_ERR_CUDA;
+    g_last_launches = launches;
+    return GTA_OK;
+}
+
+extern "C" gta_status_t gta_decode_fp8(const gta_shape_t* shape, const void* q, const void* k_codes, const void* c_codes,
+                                       const float* k_scales, const float* c_scales, const int32_t* seq_lens,
+                                       int32_t S_cap, const void* x_t, const void* w_p, const void* w_g, void* out,
+                                       void* workspace, size_t workspace_bytes, int32_t* status_word,
+                                       void* cuda_stream) {
+    g_last_launches = 0;
+    gta::Dims d;
+    gta_status_t st = fp8_check(shape, &d);
+    if (st != GTA_OK) return st;
+    if (S_cap <= 0) return GTA_ERR_INVALID_ARG;
+    if (!q || !k_codes || !c_codes || !k_scales || !c_scales || !seq_lens || !x_t || !w_p || !w_g || !out)
+        return GTA_ERR_INVALID_ARG;
+    if (!aligned(q, 16) || !aligned(k_codes, 16) || !aligned(c_codes, 16) || !aligned(k_scales, 4) ||
+        !aligned(c_scales, 4) || !aligned(x_t, 16) || !aligned(w_p, 16) || !aligned(w_g, 16) || !aligned(out, 16) ||
+        !aligned(seq_lens, 4) || !aligned(status_word, 4))
+        return GTA_ERR_INVALID_ARG;
+    if (d.B == 0) return GTA_OK;
+    if (!workspace || !aligned(workspace, 256) || workspace_bytes < gta::decode_fp8_workspace_bytes(d, S_cap))
+        return GTA_ERR_WORKSPACE;
+    if ((st = check_device()) != GTA_OK) return st;
+    int launches = 0;
+    cudaError_t err = gta::launch_decode_fp8(d, shape->dtype, q, k_codes, c_codes, k_scales, c_scales, seq_lens, S_cap,
+                                             x_t, w_p, w_g, out, workspace, status_word,
+                                             static_cast<cudaStream_t>(cuda_stream), &launches);
+    if (err != cudaSuccess) return GTA_ERR_CUDA;
+    g_last_launches = launches;
+    return GTA_OK;
+}

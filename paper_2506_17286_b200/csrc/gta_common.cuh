@@ -106,6 +106,17 @@ gta_status_t decode_check_args(const gta_shape_t* shape, const void* q, const vo
 // GTA_OK when the current device is one the kernels are built for, GTA_ERR_UNSUPPORTED otherwise.
 gta_status_t check_current_device();
 
+// Decode and append over 8-bit caches (e4m3 codes [B, groups, S_cap, width] + one fp32 scale per row
+// [B, groups, S_cap]); plain-ALU kernels.
+size_t decode_fp8_workspace_bytes(const Dims& d, int S_cap);
+cudaError_t launch_decode_fp8(const Dims& d, int dtype, const void* q, const void* k_codes, const void* c_codes,
+                              const float* k_scale, const float* c_scale, const int32_t* seq_lens, int S_cap,
+                              const void* x_t, const void* w_p, const void* w_g, void* out, void* workspace,
+                              int32_t* status_word, cudaStream_t stream, int* launches);
+cudaError_t launch_cache_append_fp8(const Dims& d, int dtype, void* k_codes, void* c_codes, float* k_scale,
+                                    float* c_scale, int S_cap, const void* k_new, const void* c_new, int n_new,
+                                    int32_t* seq_lens, int32_t* status_word, cudaStream_t stream, int* launches);
+
 // Comparison operator (App. B.3, GQA / Sec. 3.1, MHA): one decode step on the stream and merge kernels.
 bool gqa_decode_supported(int B, int n_h, int n_kv, int d_h, int dtype);
 size_t gqa_decode_workspace_bytes(int B, int n_h, int n_kv, int d_h);

@@ -9,6 +9,8 @@
 //       split over H; partial sums to workspace.
 //   decode_finish_kernel  : log-sum-exp merge of the chunk partials, decoder GEMV with
 //       W_P,i for 8 sequences per CTA (weights reused), gate sigmoid, store.
+#include <type_traits>
+
 #include "gta_common.cuh"
 
 namespace gta {
@@ -76,19 +78,41 @@ template <> struct Vec16<__nv_bfloat16> {
     }
 };
 
+// e4m3 codes (1 sign, 4 exponent, 3 mantissa bits, bias 7): the seven low bits, put where fp32 keeps the low four
+// exponent bits and the top three mantissa bits, are the value times 2^-120 -- for the subnormal codes too --,
+// so one exact multiplication by 2^120 finishes the conversion.
+struct Fp8 { uint8_t bits; };
+__device__ __forceinline__ float e4m3_to_f32(uint32_t b) {
+    return __uint_as_float(((b & 0x80u) << 24) | ((b & 0x7fu) << 20)) * 1.329227995784916e36f;   // 2^120
+}
+template <> struct Vec16<Fp8> {
+    static constexpr int N = 16;
+    static __device__ __forceinline__ void load(const Fp8* p, float (&v)[16]) {
+        const uint4 r = __ldg(reinterpret_cast<const uint4*>(p));
+        const uint32_t w[4] = {r.x, r.y, r.z, r.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+#pragma unroll
+            for (int j = 0; j < 4; ++j) v[4 * i + j] = e4m3_to_f32(w[i] >> (8 * j));
+    }
+};
+
 template <typename T> __device__ __forceinline__ float exp_fn(float x);
 template <> __device__ __forceinline__ float exp_fn<float>(float x) { return expf(x); }
 template <> __device__ __forceinline__ float exp_fn<__nv_bfloat16>(float x) { return __expf(x); }
 
 // Dynamic shared memory of decode_partial_kernel (floats):
 //   q_s [n_q][d_h] | p_s [chunk][n_q] | ml_s [n_q][2] | red [R][d_l]
-template <typename T, int NGB>
+// CT: storage type of the caches (T, or Fp8 with one fp32 scale per cached row in k_scale / c_scale).
+template <typename T, int NGB, typename CT = T>
 __global__ void __launch_bounds__(kDecodeThreads)
 decode_partial_kernel(Dims d, int chunk, int n_chunks, int S_cap, const T* __restrict__ q,
-                      const T* __restrict__ k_cache, const T* __restrict__ c_cache,
+                      const CT* __restrict__ k_cache, const CT* __restrict__ c_cache,
                       const int32_t* __restrict__ seq_lens, float* __restrict__ part_o,
-                      float* __restrict__ part_ml, PageMap pm, int32_t* status_word) {
-    constexpr int VEC = Vec16<T>::N;
+                      float* __restrict__ part_ml, PageMap pm, int32_t* status_word,
+                      const float* __restrict__ k_scale, const float* __restrict__ c_scale) {
+    constexpr int VEC = Vec16<CT>::N;
+    constexpr bool kScaled = !std::is_same<CT, T>::value;
     const int b = blockIdx.y, ck = blockIdx.x;
     int len = seq_lens[b];
     len = len < 0 ? 0 : (len > S_cap ? S_cap : len);
@@ -122,19 +146,20 @@ decode_partial_kernel(Dims d, int chunk, int n_chunks, int S_cap, const T* __res
             const bool live = j < n_tok;
             // (a block-table entry outside the pool raises the status word; row 0 of the pool stands in)
             const long long k_idx = cache_row(pm, b, d.n_k, kg, S_cap, j_begin + (live ? j : 0), status_word);
-            const T* k_row = k_cache + (size_t)(k_idx < 0 ? 0 : k_idx) * d.d_h;
+            const CT* k_row = k_cache + (size_t)(k_idx < 0 ? 0 : k_idx) * d.d_h;
+            const float row_scale = kScaled ? d.scale * k_scale[k_idx < 0 ? 0 : k_idx] : d.scale;
             for (int gi = 0; gi < q_per_k; ++gi) {
                 const int g = kg * q_per_k + gi;
                 float dot = 0.f;
                 for (int v = sl; v < vecs_per_row; v += lpr) {
                     float kv[VEC];
-                    Vec16<T>::load(k_row + v * VEC, kv);
+                    Vec16<CT>::load(k_row + v * VEC, kv);
                     const float* qv = q_s + g * d.d_h + v * VEC;
 #pragma unroll
                     for (int e = 0; e < VEC; ++e) dot = fmaf(qv[e], kv[e], dot);
                 }
                 for (int o = lpr >> 1; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
-                if (live && sl == 0) p_s[j * d.n_q + g] = dot * d.scale;
+                if (live && sl == 0) p_s[j * d.n_q + g] = dot * row_scale;
             }
         }
     }
@@ -169,9 +194,9 @@ decode_partial_kernel(Dims d, int chunk, int n_chunks, int S_cap, const T* __res
     const int r = tid / tpr, v = tid % tpr;
     const int maps_per_c = d.n_q / d.n_c;
     for (int cg = 0; cg < d.n_c; ++cg) {
-        auto c_row = [&](int j) -> const T* {   // latent row of token j_begin + j, this thread's vector
+        auto c_idx = [&](int j) -> size_t {   // row of token j_begin + j in the latent cache
             const long long idx = cache_row(pm, b, d.n_c, cg, S_cap, j_begin + j, status_word);
-            return c_cache + (size_t)(idx < 0 ? 0 : idx) * d.d_l + v * VEC;
+            return (size_t)(idx < 0 ? 0 : idx);
         };
         for (int g0 = cg * maps_per_c; g0 < (cg + 1) * maps_per_c; g0 += NGB) {
             float acc[NGB][VEC];
@@ -180,17 +205,23 @@ decode_partial_kernel(Dims d, int chunk, int n_chunks, int S_cap, const T* __res
 #pragma unroll
                 for (int e = 0; e < VEC; ++e) acc[gi][e] = 0.f;
             if (active) {
+                constexpr int U = kScaled ? 2 : 4;         // independent 16-byte loads in flight
                 int j = r;
-                for (; j + 3 * R < n_tok; j += 4 * R) {   // four independent 16-byte loads in flight
-                    float cv[4][VEC];
+                for (; j + (U - 1) * R < n_tok; j += U * R) {
+                    float cv[U][VEC];
+                    float cs[U];
 #pragma unroll
-                    for (int u = 0; u < 4; ++u) Vec16<T>::load(c_row(j + u * R), cv[u]);
+                    for (int u = 0; u < U; ++u) {
+                        const size_t idx = c_idx(j + u * R);
+                        Vec16<CT>::load(c_cache + idx * d.d_l + v * VEC, cv[u]);
+                        cs[u] = kScaled ? c_scale[idx] : 1.f;
+                    }
 #pragma unroll
-                    for (int u = 0; u < 4; ++u) {
+                    for (int u = 0; u < U; ++u) {
                         const float* pj = p_s + (j + u * R) * d.n_q + g0;
 #pragma unroll
                         for (int gi = 0; gi < NGB; ++gi) {
-                            const float p = pj[gi];
+                            const float p = pj[gi] * cs[u];      // the row's scale folded into its probability
 #pragma unroll
                             for (int e = 0; e < VEC; ++e) acc[gi][e] = fmaf(p, cv[u][e], acc[gi][e]);
                         }
@@ -198,11 +229,13 @@ decode_partial_kernel(Dims d, int chunk, int n_chunks, int S_cap, const T* __res
                 }
                 for (; j < n_tok; j += R) {
                     float cv[VEC];
-                    Vec16<T>::load(c_row(j), cv);
+                    const size_t idx = c_idx(j);
+                    Vec16<CT>::load(c_cache + idx * d.d_l + v * VEC, cv);
+                    const float cs = kScaled ? c_scale[idx] : 1.f;
                     const float* pj = p_s + j * d.n_q + g0;
 #pragma unroll
                     for (int gi = 0; gi < NGB; ++gi) {
-                        const float p = pj[gi];
+                        const float p = pj[gi] * cs;
 #pragma unroll
                         for (int e = 0; e < VEC; ++e) acc[gi][e] = fmaf(p, cv[e], acc[gi][e]);
                     }
@@ -370,7 +403,7 @@ static cudaError_t launch_decode_typed(const Dims& d, const void* q, const void*
             }                                                                                          \
             kern<<<grid, kDecodeThreads, smem, stream>>>(d, p.chunk, p.n_chunks, S_cap, (const T*)q,   \
                                                          (const T*)k_cache, (const T*)c_cache, seq_lens, \
-                                                         part_o, part_ml, pm, status_word);            \
+                                                         part_o, part_ml, pm, status_word, nullptr, nullptr); \
         } while (0)
         if (maps_per_c % 8 == 0) GTA_LAUNCH_PARTIAL(8);
         else if (maps_per_c % 4 == 0) GTA_LAUNCH_PARTIAL(4);
@@ -395,6 +428,144 @@ static cudaError_t launch_decode_typed(const Dims& d, const void* q, const void*
         *launches += 1;
     }
     return cudaSuccess;
+}
+
+// ---- 8-bit caches: e4m3 codes with one fp32 scale per cached row (token and group).  Reading (the paper
+//      fixes none; its Sec. 5.3 / App. C.2 only observe that decode is bound by the bytes of the cache):
+//      scale = max|row| / 448 (1 for an all-zero row), code = round-to-nearest-even(x / scale), both
+//      divisions in fp32; the operator runs on code * scale.
+size_t decode_fp8_workspace_bytes(const Dims& d, int S_cap) { return make_plan(d, S_cap).total; }
+
+template <typename T>
+static cudaError_t launch_decode_fp8_typed(const Dims& d, const void* q, const void* k_codes, const void* c_codes,
+                                           const float* k_scale, const float* c_scale, const int32_t* seq_lens,
+                                           int S_cap, const void* x_t, const void* w_p, const void* w_g, void* out,
+                                           void* workspace, int32_t* status_word, cudaStream_t stream, int* launches) {
+    const DecodePlan p = make_plan(d, S_cap);
+    float* part_o = reinterpret_cast<float*>(workspace);
+    float* part_ml = reinterpret_cast<float*>(static_cast<char*>(workspace) + p.off_ml);
+    float* z_part = reinterpret_cast<float*>(static_cast<char*>(workspace) + p.off_z);
+    cudaError_t err;
+    dim3 ggrid((d.n_h * d.d_h + 127) / 128, p.gate_splits);
+    decode_gate_kernel<T><<<ggrid, 128, 0, stream>>>(d, p.gate_slice, (const T*)x_t, (const T*)w_g, z_part);
+    if ((err = cudaGetLastError()) != cudaSuccess) return err;
+    {
+        constexpr int VEC = 16;
+        const int tpr = d.d_l / VEC;
+        const int R = kDecodeThreads / tpr;
+        const size_t smem = ((size_t)d.n_q * d.d_h + (size_t)p.chunk * d.n_q + 2 * d.n_q + (size_t)R * d.d_l) * sizeof(float);
+        const int maps_per_c = d.n_q / d.n_c;
+        dim3 grid(p.n_chunks, d.B);
+#define GTA_LAUNCH_PARTIAL8(NGB)                                                                       \
+        do {                                                                                           \
+            auto kern = decode_partial_kernel<T, NGB, Fp8>;                                            \
+            if (smem > 48 * 1024) {                                                                    \
+                err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem); \
+                if (err != cudaSuccess) return err;                                                    \
+            }                                                                                          \
+            kern<<<grid, kDecodeThreads, smem, stream>>>(d, p.chunk, p.n_chunks, S_cap, (const T*)q,   \
+                                                         (const Fp8*)k_codes, (const Fp8*)c_codes, seq_lens, \
+                                                         part_o, part_ml, PageMap(), status_word, k_scale, c_scale); \
+        } while (0)
+        if (maps_per_c % 4 == 0) GTA_LAUNCH_PARTIAL8(4);
+        else if (maps_per_c % 2 == 0) GTA_LAUNCH_PARTIAL8(2);
+        else GTA_LAUNCH_PARTIAL8(1);
+#undef GTA_LAUNCH_PARTIAL8
+        if ((err = cudaGetLastError()) != cudaSuccess) return err;
+    }
+    {
+        const int KH = kDecodeThreads / d.d_h > 0 ? kDecodeThreads / d.d_h : 1;
+        const size_t smem = ((size_t)kFinishSeqs * d.d_l + (size_t)KH * kFinishSeqs * d.d_h + p.n_chunks) * sizeof(float);
+        auto kern = decode_finish_kernel<T>;
+        if (smem > 48 * 1024) {
+            err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+            if (err != cudaSuccess) return err;
+        }
+        dim3 grid(d.n_h, (d.B + kFinishSeqs - 1) / kFinishSeqs);
+        kern<<<grid, kDecodeThreads, smem, stream>>>(d, p.chunk, p.n_chunks, S_cap, p.gate_splits, seq_lens, part_o,
+                                                    part_ml, z_part, (const T*)w_p, (T*)out);
+        if ((err = cudaGetLastError()) != cudaSuccess) return err;
+    }
+    *launches += 3;
+    return cudaSuccess;
+}
+
+cudaError_t launch_decode_fp8(const Dims& d, int dtype, const void* q, const void* k_codes, const void* c_codes,
+                              const float* k_scale, const float* c_scale, const int32_t* seq_lens, int S_cap,
+                              const void* x_t, const void* w_p, const void* w_g, void* out, void* workspace,
+                              int32_t* status_word, cudaStream_t stream, int* launches) {
+    if (dtype == GTA_F32)
+        return launch_decode_fp8_typed<float>(d, q, k_codes, c_codes, k_scale, c_scale, seq_lens, S_cap, x_t, w_p, w_g,
+                                              out, workspace, status_word, stream, launches);
+    return launch_decode_fp8_typed<__nv_bfloat16>(d, q, k_codes, c_codes, k_scale, c_scale, seq_lens, S_cap, x_t, w_p,
+                                                  w_g, out, workspace, status_word, stream, launches);
+}
+
+// Quantising append: one warp per new row (token and group): the row's largest magnitude, its scale, its codes.
+// One CTA per sequence; the length advances when all its rows are written.  src rows [B][groups][n_new][width].
+__device__ __forceinline__ uint32_t f32_to_e4m3(float y) {
+    uint16_t r;   // the low byte of the pair is the second source operand
+    asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(r) : "f"(0.f), "f"(y));
+    return r & 0xffu;
+}
+template <typename T>
+__device__ __forceinline__ void quantise_row(const T* __restrict__ src, uint8_t* __restrict__ dst,
+                                             float* __restrict__ scale_out, int width, int lane) {
+    float amax = 0.f;
+    for (int e = lane; e < width; e += 32) amax = fmaxf(amax, fabsf(to_f32(src[e])));
+    amax = warp_max(amax);
+    const float scale = amax > 0.f ? __fdiv_rn(amax, 448.f) : 1.f;
+    for (int e = lane * 4; e < width; e += 128) {        // widths are multiples of 8: four codes per store
+        uint32_t w = 0;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) w |= f32_to_e4m3(__fdiv_rn(to_f32(src[e + i]), scale)) << (8 * i);
+        *reinterpret_cast<uint32_t*>(dst + e) = w;
+    }
+    if (lane == 0) *scale_out = scale;
+}
+template <typename T>
+__global__ void __launch_bounds__(256)
+append_fp8_kernel(Dims d, int S_cap, int n_new, uint8_t* __restrict__ k_codes, uint8_t* __restrict__ c_codes,
+                  float* __restrict__ k_scale, float* __restrict__ c_scale, const T* __restrict__ k_new,
+                  const T* __restrict__ c_new, int32_t* __restrict__ seq_lens, int32_t* status_word) {
+    const int b = blockIdx.x, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int len = seq_lens[b];
+    __syncthreads();   // every thread has read the old length before thread 0 rewrites it
+    if (len < 0 || (long long)len + n_new > S_cap) {
+        if (threadIdx.x == 0) raise_status(status_word, GTA_ERR_CACHE_FULL);
+        return;
+    }
+    const int k_rows = d.n_k * n_new, rows = k_rows + d.n_c * n_new;
+    for (int r = warp; r < rows; r += 8) {
+        if (r < k_rows) {
+            const int g = r / n_new, n = r % n_new;
+            const size_t row = ((size_t)b * d.n_k + g) * S_cap + len + n;
+            quantise_row(k_new + (((size_t)b * d.n_k + g) * n_new + n) * d.d_h, k_codes + row * d.d_h, k_scale + row,
+                         d.d_h, lane);
+        } else {
+            const int g = (r - k_rows) / n_new, n = (r - k_rows) % n_new;
+            const size_t row = ((size_t)b * d.n_c + g) * S_cap + len + n;
+            quantise_row(c_new + (((size_t)b * d.n_c + g) * n_new + n) * d.d_l, c_codes + row * d.d_l, c_scale + row,
+                         d.d_l, lane);
+        }
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) seq_lens[b] = len + n_new;
+}
+
+cudaError_t launch_cache_append_fp8(const Dims& d, int dtype, void* k_codes, void* c_codes, float* k_scale,
+                                    float* c_scale, int S_cap, const void* k_new, const void* c_new, int n_new,
+                                    int32_t* seq_lens, int32_t* status_word, cudaStream_t stream, int* launches) {
+    if (dtype == GTA_F32)
+        append_fp8_kernel<float><<<d.B, 256, 0, stream>>>(d, S_cap, n_new, (uint8_t*)k_codes, (uint8_t*)c_codes, k_scale,
+                                                           c_scale, (const float*)k_new, (const float*)c_new, seq_lens,
+                                                           status_word);
+    else
+        append_fp8_kernel<__nv_bfloat16><<<d.B, 256, 0, stream>>>(d, S_cap, n_new, (uint8_t*)k_codes, (uint8_t*)c_codes,
+                                                                   k_scale, c_scale, (const __nv_bfloat16*)k_new,
+                                                                   (const __nv_bfloat16*)c_new, seq_lens, status_word);
+    *launches += 1;
+    return cudaGetLastError();
 }
 
 cudaError_t launch_decode(const Dims& d, int dtype, const void* q, const void* k_cache, const void* c_cache,

@@ -1,0 +1,140 @@
+"""GPU parity of the 8-bit caches (e4m3 codes + one fp32 scale per cached row): the quantising append is a
+bit-exact function of the new rows, the decode step over such caches matches the fp64 oracle on the dequantised
+values within the bf16 bounds."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2506_17286_b200 import inputs as I
+from tests.parity_utils import Guarded, assert_close, oracle_shape
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def B():
+    if not torch.cuda.is_available():
+        pytest.skip("needs a CUDA device")
+    from paper_2506_17286_b200 import build, binding
+    build.build()
+    binding.lib()
+    return binding
+
+
+@pytest.mark.parametrize("dt", ["bf16", "f32"])
+@pytest.mark.parametrize("n_new", [1, 3, 300])
+def test_quantising_append_is_bit_exact(B, oracle, dt, n_new):
+    tdt = torch.bfloat16 if dt == "bf16" else torch.float32
+    nb, n_k, n_c, d_h, d_l, cap = 6, 4, 2, 64, 128, 512
+    g = torch.Generator("cpu").manual_seed(31 + n_new)
+    k_new = (torch.randn(nb, n_k, n_new, d_h, generator=g) * 3).to(tdt)
+    c_new = torch.randn(nb, n_c, n_new, d_l, generator=g).to(tdt)
+    k_new[0, 0, 0] = 0                                   # an all-zero row keeps scale 1
+    c_new[1, 1, n_new - 1, 5] = 1000.0                   # one dominant element
+    k_codes = torch.randint(0, 255, (nb, n_k, cap, d_h), generator=g, dtype=torch.uint8)
+    c_codes = torch.randint(0, 255, (nb, n_c, cap, d_l), generator=g, dtype=torch.uint8)
+    k_scales = torch.rand(nb, n_k, cap, generator=g)
+    c_scales = torch.rand(nb, n_c, cap, generator=g)
+    lens = torch.tensor([0, 1, cap - n_new, cap - n_new + 1, cap, 17], dtype=torch.int32)   # two do not fit
+    want = oracle.cache_append_fp8(k_codes.numpy(), k_scales.numpy(), c_codes.numpy(), c_scales.numpy(), k_new, c_new,
+                                   lens.numpy())
+    dev = [t.cuda() for t in (k_codes, c_codes, k_scales, c_scales)]
+    lens_d = lens.cuda()
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    B.gta_cache_append_fp8(*dev, k_new.cuda(), c_new.cuda(), lens_d, status_word=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == B.GTA_ERR_CACHE_FULL
+    assert lens_d.cpu().numpy().tolist() == want[4].tolist()
+    for got, ref, what in zip(dev, (want[0], want[2], want[1], want[3]), ("k codes", "c codes", "k scales", "c scales")):
+        g_ = got.cpu().numpy()
+        if g_.dtype == np.float32:                       # compared as bit patterns
+            assert np.array_equal(g_.view(np.uint32), np.asarray(ref, dtype=np.float32).view(np.uint32)), what
+        else:
+            # -0 and +0 are the same stored value as far as the operator goes, the codes 0x00 / 0x80 are not:
+            # the cast keeps the sign of a value that rounds to zero, and so does the oracle
+            assert np.array_equal(g_, ref), what
+
+
+def _decode_case(B, oracle, w, lens, sample=None):
+    nb = w.batch
+    cap = max(lens) + 7
+    t = I.decode_inputs(w, device="cuda", s_cap=cap, seq_lens=lens)
+    kq, ks = oracle.quantize_rows_e4m3(t["k_cache"].cpu())
+    cq, cs = oracle.quantize_rows_e4m3(t["c_cache"].cpu())
+    for b, n in enumerate(lens):                          # what uninitialised memory may hold behind the live rows
+        kq[b, :, n:] = 0x7F; cq[b, :, n:] = 0xFF; ks[b, :, n:] = np.nan; cs[b, :, n:] = np.inf
+    dev = [torch.from_numpy(a).cuda() for a in (kq, cq, ks, cs)]
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    shape = B.decode_shape(t["q"], t["k_cache"], t["c_cache"], t["x_t"], t["w_p"])
+    ws = Guarded((B.decode_fp8_workspace_bytes(shape, cap),), torch.uint8)
+    og = Guarded((nb, w.n_heads, w.d_h), w.torch_dtype())
+    out = B.gta_decode_fp8(t["q"], *dev, t["seq_lens"], t["x_t"], t["w_p"], t["w_g"], out=og.t, workspace=ws.t,
+                           status_word=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    ws.check("fp8 decode workspace"); og.check("fp8 decode out")
+    idx = list(range(nb)) if sample is None else sample
+    ws_ = I.scaled(w, batch=len(idx))
+    want = oracle.decode_fp8(oracle_shape(ws_, seq=0), t["q"][idx].cpu(), kq[idx], ks[idx], cq[idx], cs[idx],
+                             [lens[i] for i in idx], t["x_t"][idx].cpu(), t["w_p"].cpu(), t["w_g"].cpu())
+    return assert_close(out[idx], want, w.torch_dtype(), w.name)
+
+
+FP8_DECODE = [
+    # name, dtype, B, H, n_h, n_q, n_k, n_c, d_h, d_l, lens
+    ("bf16_ragged", "bf16", 5, 256, 8, 4, 4, 1, 128, 512, [1, 63, 64, 65, 700]),
+    ("bf16_empty_and_shared_keys", "bf16", 4, 128, 8, 4, 2, 2, 64, 128, [0, 512, 1, 300]),
+    ("bf16_paper_1b_shape", "bf16", 2, 1280, 20, 5, 1, 1, 64, 128, [333, 1000]),
+    ("f32_general", "f32", 3, 96, 6, 6, 3, 1, 32, 64, [100, 7, 260]),
+    ("bf16_dl1024_eight_maps", "bf16", 3, 512, 16, 8, 8, 1, 128, 1024, [257, 1, 1000]),
+]
+
+
+@pytest.mark.parametrize("case", FP8_DECODE, ids=[c[0] for c in FP8_DECODE])
+def test_fp8_decode_small_shapes(B, oracle, case):
+    name, dt, nb, H, n_h, n_q, n_k, n_c, d_h, d_l, lens = case
+    w = I.Workload(name, "decode", dt, nb, 0, H, n_h, n_q, n_k, n_c, d_h, d_l, seed=61)
+    _decode_case(B, oracle, w, lens)
+
+
+def test_fp8_decode_config3_shape_sampled_sequences(B, oracle):
+    w = I.CONFIGS["c3_decode_bf16"]
+    _decode_case(B, oracle, w, [w.seq] * w.batch, sample=[0, 9, 31])
+
+
+def test_append_then_decode_over_fp8_caches(B, oracle):
+    """The GPU's own quantising append feeds the GPU decode: the result is the oracle's on the oracle's append."""
+    w = I.Workload("steps", "decode", "bf16", 3, 0, 128, 8, 4, 2, 1, 64, 256, seed=62)
+    lens, cap = [5, 0, 130], 140
+    t = I.decode_inputs(w, device="cuda", s_cap=cap, seq_lens=lens)
+    kq = np.zeros((3, 2, cap, 64), np.uint8); ks = np.ones((3, 2, cap), np.float32)
+    cq = np.zeros((3, 1, cap, 256), np.uint8); cs = np.ones((3, 1, cap), np.float32)
+    dev = [torch.from_numpy(a).cuda() for a in (kq, cq, ks, cs)]
+    lens_d = torch.zeros(3, dtype=torch.int32, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    # prefill-style bulk append of each sequence's history, one call per sequence (ragged lengths)
+    for b, n in enumerate(lens):
+        if n == 0:
+            continue
+        sub = [d_[b:b + 1] for d_ in dev]
+        B.gta_cache_append_fp8(*sub, t["k_cache"][b:b + 1, :, :n].contiguous(), t["c_cache"][b:b + 1, :, :n].contiguous(),
+                               lens_d[b:b + 1], status_word=status)
+    # then one new token for all of them
+    B.gta_cache_append_fp8(*dev, t["k_new"], t["c_new"], lens_d, status_word=status)
+    out = B.gta_decode_fp8(t["q"], *dev, lens_d, t["x_t"], t["w_p"], t["w_g"], status_word=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0 and lens_d.tolist() == [n + 1 for n in lens]
+    k_hist, c_hist = t["k_cache"].cpu(), t["c_cache"].cpu()
+    kq_r, ks_r, cq_r, cs_r = kq.copy(), ks.copy(), cq.copy(), cs.copy()
+    for b, n in enumerate(lens):
+        if n:
+            a, s_ = oracle.quantize_rows_e4m3(k_hist[b, :, :n]); kq_r[b, :, :n] = a; ks_r[b, :, :n] = s_
+            a, s_ = oracle.quantize_rows_e4m3(c_hist[b, :, :n]); cq_r[b, :, :n] = a; cs_r[b, :, :n] = s_
+    kq_r, ks_r, cq_r, cs_r, lens_r, ov = oracle.cache_append_fp8(kq_r, ks_r, cq_r, cs_r, t["k_new"].cpu(), t["c_new"].cpu(),
+                                                                  np.array(lens, np.int32))
+    assert ov == 0
+    assert np.array_equal(dev[0].cpu().numpy(), kq_r) and np.array_equal(dev[1].cpu().numpy(), cq_r)
+    assert np.array_equal(dev[2].cpu().numpy().view(np.uint32), ks_r.view(np.uint32))
+    want = oracle.decode_fp8(oracle_shape(w, seq=0), t["q"].cpu(), kq_r, ks_r, cq_r, cs_r, lens_r, t["x_t"].cpu(),
+                             t["w_p"].cpu(), t["w_g"].cpu())
+    assert_close(out, want, torch.bfloat16, "append then decode (fp8 caches)")

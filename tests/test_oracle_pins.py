@@ -534,3 +534,61 @@ def test_gqa_cost_closed_forms_against_the_printed_ratios(oracle):
     assert oracle.attention_cost(gta_1b) / oracle.gqa_attention_cost(20, 64, N) == pytest.approx(0.375, abs=1e-12)
     assert oracle.cache_elems(gta_1b) / oracle.gqa_cache_elems(5, 64, N) == pytest.approx(0.30, abs=1e-12)
     assert oracle.gqa_cache_elems(5, 64, 1) == 640 and oracle.gqa_cache_elems(20, 64, 1) == 2560
+
+
+# ---------------------------------------------------------------- 8-bit caches (e4m3 codes + one scale per row)
+def test_e4m3_rounding_against_the_format_and_a_library_cast(oracle):
+    """Values written out from the format's definition, ties to even, saturation at 448, and every fp32 value of a
+    dense sweep against torch's own float8_e4m3fn cast (an independent implementation of the same format)."""
+    import torch
+    tab = oracle.e4m3_table()
+    assert tab[0x7E] == 448.0 and tab[0x38] == 1.0 and tab[0x01] == 2.0 ** -9 and tab[0x08] == 2.0 ** -6
+    assert tab[0xB8] == -1.0 and np.isnan(tab[0x7F]) and tab[0x3C] == 1.5
+    r = oracle.round_to_e4m3
+    assert r(np.float32(1.0)) == 0x38 and r(np.float32(-448.0)) == 0xFE and r(np.float32(1e9)) == 0x7E
+    assert r(np.float32(1.0625)) == 0x38 and r(np.float32(1.1875)) == 0x3A      # ties: 1.0625 -> 1.0, 1.1875 -> 1.25
+    assert r(np.float32(2.0 ** -10)) == 0x00 and r(np.float32(3 * 2.0 ** -10)) == 0x02   # ties among the subnormals
+    y = np.concatenate([np.linspace(-460, 460, 200001), np.linspace(-0.05, 0.05, 50001), _rand(100000) * 30]).astype(np.float32)
+    want = torch.from_numpy(np.clip(y, -448, 448)).to(torch.float8_e4m3fn).view(torch.uint8).numpy()
+    got = r(y)
+    same = (got == want) | ((tab[got] == 0) & (tab[want] == 0))          # +0 / -0 of tiny negatives may differ in sign
+    assert same.all()
+
+
+def test_quantised_rows_are_within_half_a_step_and_all_zero_rows_keep_scale_one(oracle):
+    x = _rand(3, 2, 5, 64)
+    x[1, 0, 2] = 0.0
+    codes, scales = oracle.quantize_rows_e4m3(x.astype(np.float32))
+    assert codes.dtype == np.uint8 and scales.shape == (3, 2, 5) and scales[1, 0, 2] == 1.0
+    back = oracle.dequantize_e4m3(codes, scales)
+    amax = np.abs(x).max(axis=-1, keepdims=True)
+    assert np.all(np.abs(back - x) <= np.maximum(np.abs(x) * 2.0 ** -4, amax / 448 * 2.0 ** -10) * 1.0001 + 1e-12)
+    big = np.argmax(np.abs(x), axis=-1)                                  # the largest element of a row maps to +-448 exactly
+    top = np.take_along_axis(oracle.e4m3_table()[codes], big[..., None], axis=-1)[..., 0]
+    nz = amax[..., 0] > 0
+    assert np.all(np.abs(top[nz]) == 448.0)
+
+
+def test_fp8_decode_is_the_operator_on_the_dequantised_caches_and_append_skips_full_sequences(oracle):
+    s = Shape(3, 0, 16, 4, 2, 2, 1, 8, 16, 1)
+    cap = 9
+    k, c = _rand(3, 2, cap, 8), _rand(3, 1, cap, 16)
+    kq, ks = oracle.quantize_rows_e4m3(k.astype(np.float32))
+    cq, cs = oracle.quantize_rows_e4m3(c.astype(np.float32))
+    lens = np.array([4, 9, 0], dtype=np.int32)
+    k_new, c_new = _rand(3, 2, 1, 8).astype(np.float32), _rand(3, 1, 1, 16).astype(np.float32)
+    kq2, ks2, cq2, cs2, lens2, ov = oracle.cache_append_fp8(kq, ks, cq, cs, k_new, c_new, lens)
+    assert ov == 1 and lens2.tolist() == [5, 9, 1]
+    assert np.array_equal(kq2[1], kq[1]) and np.array_equal(cs2[1], cs[1])          # the full sequence is untouched
+    nk, nks = oracle.quantize_rows_e4m3(k_new)
+    assert np.array_equal(kq2[0, :, 4], nk[0, :, 0]) and np.array_equal(ks2[2, :, 0], nks[2, :, 0])
+    assert np.array_equal(kq2[0, :, :4], kq[0, :, :4]) and np.array_equal(kq2[0, :, 5:], kq[0, :, 5:])
+    t = dict(q=_rand(3, 2, 8), x_t=_rand(3, 16), w_p=_rand(4, 16, 8, scale=0.25), w_g=_rand(16, 32, scale=0.25))
+    got = oracle.decode_fp8(s, t["q"], kq2, ks2, cq2, cs2, lens2, t["x_t"], t["w_p"], t["w_g"])
+    want = oracle.decode(s, t["q"], oracle.dequantize_e4m3(kq2, ks2), oracle.dequantize_e4m3(cq2, cs2), lens2, cap,
+                         t["x_t"], t["w_p"], t["w_g"])
+    assert np.array_equal(got, want)
+    # garbage (NaN codes and scales) behind the live rows does not matter
+    kq3, ks3 = kq2.copy(), ks2.copy()
+    kq3[0, :, 5:] = 0x7F; ks3[0, :, 5:] = np.nan
+    assert np.array_equal(oracle.decode_fp8(s, t["q"], kq3, ks3, cq2, cs2, lens2, t["x_t"], t["w_p"], t["w_g"])[0], got[0])
