@@ -763,6 +763,39 @@ def run_ours(args):
     comparisons["paper"] = {"attention_cost_ratio_1b": 0.375, "cache_ratio_1b": 0.30,
                             "source": "Sec. 4.3 / Table 3 of the paper (analytic, GTA-1B against GQA-1B)"}
 
+    # ---- 8-bit caches on the c3 shape: e4m3 codes + one fp32 scale per cached row (quantised on the device by the
+    #      library's own append, outside the timed loop); the decode step runs on the plain-ALU kernels
+    def fp8_leg():
+        ctx, nb = wd.seq, wd.batch
+        caches = []
+        for i in range(2):
+            td = I.decode_inputs(I.scaled(wd, seed=wd.seed + 10 + i), device=dev, s_cap=ctx + 64)
+            kq = torch.zeros((nb, wd.n_k, ctx + 64, wd.d_h), dtype=torch.uint8, device=dev)
+            cq = torch.zeros((nb, wd.n_c, ctx + 64, wd.d_l), dtype=torch.uint8, device=dev)
+            ks = torch.ones((nb, wd.n_k, ctx + 64), dtype=torch.float32, device=dev)
+            cs = torch.ones((nb, wd.n_c, ctx + 64), dtype=torch.float32, device=dev)
+            lens = torch.zeros(nb, dtype=torch.int32, device=dev)
+            G.gta_cache_append_fp8(kq, cq, ks, cs, td["k_cache"][:, :, :ctx].contiguous(),
+                                   td["c_cache"][:, :, :ctx].contiguous(), lens, status_word=status)
+            caches.append(dict(kq=kq, cq=cq, ks=ks, cs=cs, lens=lens, q=td["q"], x_t=td["x_t"], w_p=td["w_p"], w_g=td["w_g"]))
+        ws8 = torch.empty(G.decode_fp8_workspace_bytes(shape_d, ctx + 64), dtype=torch.uint8, device=dev)
+
+        def call(i):
+            c = caches[i % 2]
+            G.gta_decode_fp8(c["q"], c["kq"], c["cq"], c["ks"], c["cs"], c["lens"], c["x_t"], c["w_p"], c["w_g"], out=out_d,
+                             workspace=ws8, status_word=status)
+        t8, rec8 = timed_loop(call, 20, min_ms=150.0)
+        cache_bytes = float(nb) * ctx * ((wd.n_k * wd.d_h + wd.n_c * wd.d_l) + 4 * (wd.n_k + wd.n_c))
+        nbytes = cache_bytes + by["weights"] + by["vectors"]
+        r = hbm_roofline(nbytes, t8, peaks, rec8["clocks"],
+                         note="gta_decode_fp8 back to back, two cache sets alternating; bytes = codes + scales of the live "
+                              "rows + weights + vectors; plain-ALU kernels (correct, not at the roofline)")
+        r["cache_bytes_vs_bf16"] = cache_bytes / by["cache"]
+        r["ms_vs_bf16_decode_call"] = t8 / t_decode_call
+        return r
+
+    fp8_cache = fp8_leg()
+
     # ---- c5: 128 ragged sequences (1024 .. 32768 cached tokens, 8.9 GB live), gta_cache_append + gta_decode per step
     w5 = I.CONFIGS["c5_ragged_decode_bf16"]
     t5 = I.decode_inputs(w5, device=dev)
@@ -898,7 +931,8 @@ def run_ours(args):
             },
             "prefill": {"ms": t_prefill, "tokens_per_s": world * wp.batch * wp.seq / (t_prefill * 1e-3),
                         "flops": fl},
-            "layer": layer, "decode": decode, "legs": legs, "comparison_with_gqa": comparisons, "roofline": roofline,
+            "layer": layer, "decode": decode, "legs": legs, "comparison_with_gqa": comparisons, "fp8_cache_decode": fp8_cache,
+            "roofline": roofline,
             "e2e": e2e,
             "cpu_baseline": cpu_baseline, "gpu_launches": n_launches, "clocks": clocks,
         }
