@@ -306,6 +306,28 @@ GTA_API gta_status_t gta_decode_static(const gta_shape_t *shape, const void *q, 
                                        int32_t *status_word, void *cuda_stream);
 
 /*
+ * gta_decode_append — one decode step including the append of its token (App. B.1.3: the new
+ * token's keys and latents join the caches, then its queries attend over all of them):
+ * the same result, cache contents, lengths and status as
+ *     gta_cache_append(shape, k_cache, c_cache, S_cap, k_new, c_new, 1, seq_lens, ...);
+ *     gta_decode(shape, q, k_cache, c_cache, seq_lens, S_cap, x_t, w_p, w_g, out, ...);
+ * bit for bit, in one call.  seq_lens (device int32 [B], in / out) does NOT count the new token
+ * on entry and does on return; k_new [B, n_k, d_h], c_new [B, n_c, d_l]; a sequence whose cache
+ * is full (or whose length is negative) keeps its cache and length, is attended over as it is,
+ * and raises GTA_ERR_CACHE_FULL in the status word.  On the bf16 fast path of gta_decode the
+ * append costs no kernel of its own: the CTA that streams the end of a sequence puts the new
+ * rows over the corresponding rows of its shared-memory tile and writes them to the caches, and
+ * the lengths advance in the last kernel of the step, after every reader of them is done.
+ * Everywhere else the call runs the two calls above one after the other.  Workspace as for
+ * gta_decode.
+ */
+GTA_API gta_status_t gta_decode_append(const gta_shape_t *shape, const void *q, void *k_cache, void *c_cache,
+                                       const void *k_new, const void *c_new, int32_t *seq_lens, int32_t S_cap,
+                                       const void *x_t, const void *w_p, const void *w_g, void *out,
+                                       void *workspace, size_t workspace_bytes, int32_t *status_word,
+                                       void *cuda_stream);
+
+/*
  * 8-bit caches (the paper has no such format; Sec. 5.3 and App. C.2 only observe that the decode
  * step is bound by the bytes of the cache, the larger the context and the slower the memory the
  * more).  Reading taken here: K and C rows are kept as e4m3 codes (8-bit floats: 1 sign, 4

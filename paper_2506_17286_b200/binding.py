@@ -28,7 +28,7 @@ EXPORTS = (
     "gta_layer_prefill_workspace_bytes", "gta_layer_prefill", "gta_layer_decode_workspace_bytes", "gta_layer_decode",
     "gta_layer_decode_paged_workspace_bytes", "gta_layer_decode_paged", "gta_debug_attention_wait",
     "gta_ref_gqa_prefill", "gta_ref_gqa_decode_workspace_bytes", "gta_ref_gqa_decode",
-    "gta_decode_fp8_workspace_bytes", "gta_cache_append_fp8", "gta_decode_fp8",
+    "gta_decode_fp8_workspace_bytes", "gta_cache_append_fp8", "gta_decode_fp8", "gta_decode_append",
 )
 
 
@@ -117,6 +117,8 @@ def lib():
         L.gta_cache_append_fp8.restype = i32
         L.gta_decode_fp8.argtypes = [sp, vp, vp, vp, vp, vp, vp, i32, vp, vp, vp, vp, vp, sz, vp, vp]
         L.gta_decode_fp8.restype = i32
+        L.gta_decode_append.argtypes = [sp, vp, vp, vp, vp, vp, vp, i32, vp, vp, vp, vp, vp, sz, vp, vp]
+        L.gta_decode_append.restype = i32
         L.gta_debug_attention_wait.argtypes = [ctypes.c_uint64, i32]
         L.gta_debug_attention_wait.restype = i32
         _lib = L
@@ -374,6 +376,27 @@ def gta_decode(q, k_cache, c_cache, seq_lens, x_t, w_p, w_g, *, softmax_scale=0.
     st = lib().gta_decode(*args) if stages == 7 else lib().gta_decode_stages(*args, stages)
     if st != GTA_OK:
         raise GtaError(st, "gta_decode")
+    return out
+
+
+def gta_decode_append(q, k_cache, c_cache, k_new, c_new, seq_lens, x_t, w_p, w_g, *, softmax_scale=0.0, out=None,
+                      workspace=None, status_word=None, stream=None):
+    """One decode step including the append of its token: k_new [B, n_k, 1, d_h] / c_new [B, n_c, 1, d_l] join the
+    caches at row seq_lens[b], seq_lens advances, the new token's queries attend over everything."""
+    _check_tensors(q, k_cache, c_cache, k_new, c_new, x_t, w_p, w_g)
+    shape = decode_shape(q, k_cache, c_cache, x_t, w_p, softmax_scale=softmax_scale)
+    B, n_k, s_cap, d_h = k_cache.shape
+    if k_new.numel() != B * n_k * d_h or c_new.numel() != B * c_cache.shape[1] * c_cache.shape[3]:
+        raise ValueError("k_new / c_new hold one row per sequence and group")
+    if out is None:
+        out = torch.empty((B, w_p.shape[0], d_h), dtype=q.dtype, device=q.device)
+    if workspace is None:
+        workspace = _workspace(decode_workspace_bytes(shape, s_cap), q.device)
+    st = lib().gta_decode_append(ctypes.byref(shape), _ptr(q), _ptr(k_cache), _ptr(c_cache), _ptr(k_new), _ptr(c_new),
+                                 _ptr(seq_lens), int(s_cap), _ptr(x_t), _ptr(w_p), _ptr(w_g), _ptr(out), _ptr(workspace),
+                                 workspace.numel() * workspace.element_size(), _ptr(status_word), _stream(stream))
+    if st != GTA_OK:
+        raise GtaError(st, "gta_decode_append")
     return out
 
 

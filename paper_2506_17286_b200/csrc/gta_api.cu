@@ -608,3 +608,39 @@ extern "C" gta_status_t gta_decode_fp8(const gta_shape_t* shape, const void* q, 
     g_last_launches = launches;
     return GTA_OK;
 }
+
+// ---- append + decode in one call
+extern "C" gta_status_t gta_decode_append(const gta_shape_t* shape, const void* q, void* k_cache, void* c_cache,
+                                          const void* k_new, const void* c_new, int32_t* seq_lens, int32_t S_cap,
+                                          const void* x_t, const void* w_p, const void* w_g, void* out, void* workspace,
+                                          size_t workspace_bytes, int32_t* status_word, void* cuda_stream) {
+    g_last_launches = 0;
+    gta::Dims d;
+    bool empty = false;
+    gta_status_t st = gta::decode_check_args(shape, q, k_cache, c_cache, seq_lens, S_cap, x_t, w_p, w_g, out, status_word,
+                                             &d, &empty);
+    if (st != GTA_OK) return st;
+    if (S_cap <= 0 || !k_new || !c_new || !aligned(k_new, 16) || !aligned(c_new, 16)) return GTA_ERR_INVALID_ARG;
+    if (empty) return GTA_OK;
+    if (!workspace || !aligned(workspace, 256) || workspace_bytes < gta::decode_workspace_bytes(d, shape->dtype, S_cap))
+        return GTA_ERR_WORKSPACE;
+    if ((st = check_device()) != GTA_OK) return st;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    int launches = 0;
+    cudaError_t err;
+    if (gta::decode_fast_supported(d, shape->dtype, 0)) {
+        // one pass: the stream kernel puts the new rows into the caches and attends over them, the lengths advance
+        // in the last kernel of the step
+        err = gta::launch_decode_fast(d, q, k_cache, c_cache, seq_lens, S_cap, x_t, w_p, w_g, out, workspace, status_word,
+                                      stream, 7, &launches, gta::PageMap(), k_new, c_new);
+    } else {
+        err = gta::launch_cache_append(d, (int)elem_size(shape->dtype), k_cache, c_cache, S_cap, k_new, c_new, 1, seq_lens,
+                                       status_word, stream, &launches);
+        if (err == cudaSuccess)
+            err = gta::launch_decode(d, shape->dtype, q, k_cache, c_cache, seq_lens, S_cap, x_t, w_p, w_g, out, workspace,
+                                     status_word, stream, 7, &launches);
+    }
+    if (err != cudaSuccess) return GTA_ERR_CUDA;
+    g_last_launches = launches;
+    return GTA_OK;
+}

@@ -96,7 +96,8 @@ size_t decode_fast_workspace_bytes(const Dims& d);
 cudaError_t launch_decode_fast(const Dims& d, const void* q, const void* k_cache, const void* c_cache,
                                const int32_t* seq_lens, int S_cap, const void* x_t, const void* w_p,
                                const void* w_g, void* out, void* workspace, int32_t* status_word,
-                               cudaStream_t stream, int stages, int* launches, const PageMap& pm = PageMap());
+                               cudaStream_t stream, int stages, int* launches, const PageMap& pm = PageMap(),
+                               const void* k_new = nullptr, const void* c_new = nullptr);
 
 // Host-side argument checks of a decode call (everything but the workspace and the device), shared by
 // gta_decode and gta_decode_static so that both report the same errors; *empty: the batch is empty.

@@ -111,6 +111,18 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     return *reinterpret_cast<uint32_t*>(&v);
 }
 __device__ __forceinline__ int clamp_len(int len, int S_cap) { return len < 0 ? 0 : (len > S_cap ? S_cap : len); }
+// Length a decode step attends over.  With `append` (the fused append + decode step) the stored length does not
+// count the new token yet: a sequence with room for it (0 <= len < S_cap) attends over len + 1 tokens, the last
+// of which comes from the new rows; a full or invalid one is left as it is (and reported by the kernel).
+struct StepLens {
+    const int32_t* seq_lens;
+    int S_cap, append;
+    __device__ __forceinline__ bool appends(int b) const {
+        const int len = seq_lens[b];
+        return append && len >= 0 && len < S_cap;
+    }
+    __device__ __forceinline__ int len(int b) const { return clamp_len(seq_lens[b], S_cap) + (appends(b) ? 1 : 0); }
+};
 
 // Shared-memory layout of one ring stage (all tiles are [T rows][64 bf16] = T x 128 bytes with
 // the 128-byte TMA swizzle: the 16-byte chunk c of row r sits at chunk c ^ (r & 7)):
@@ -123,7 +135,12 @@ template <int NT, int KH, bool ONE_C, int OCC>
 __global__ void __launch_bounds__(kStreamThreads, OCC)
 decode_stream_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_c, Dims d,
                      int T, int S_cap, const __nv_bfloat16* __restrict__ q, const int32_t* __restrict__ seq_lens,
-                     float* __restrict__ part_o, float* __restrict__ part_ml, int32_t* status_word, PageMap pm) {
+                     float* __restrict__ part_o, float* __restrict__ part_ml, int32_t* status_word, PageMap pm,
+                     const uint4* __restrict__ k_new, const uint4* __restrict__ c_new, uint4* __restrict__ k_rows,
+                     uint4* __restrict__ c_rows) {
+    // k_new != nullptr: the fused append + decode step (contiguous caches).  k_new [B][n_k][d_h] / c_new
+    // [B][n_c][d_l] are the new token's rows, k_rows / c_rows the caches as writable 16-byte vectors.
+    const StepLens L{seq_lens, S_cap, k_new != nullptr};
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     uint8_t* ring = smem;                                                              // 3 x 64 KB
@@ -160,7 +177,7 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
         const int per = (d.B + kStreamThreads - 1) / kStreamThreads;
         const int lo = min(tid * per, d.B), hi = min(lo + per, d.B);
         int sum = 0;
-        for (int b = lo; b < hi; ++b) sum += (clamp_len(seq_lens[b], S_cap) + T - 1) / T;
+        for (int b = lo; b < hi; ++b) sum += (L.len(b) + T - 1) / T;
         int incl = sum;
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
@@ -179,10 +196,14 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
         for (int w = 0; w < warp; ++w) base += scan_tmp[w];
         for (int b = lo; b < hi; ++b) {
             prefix[b] = base;
-            base += (clamp_len(seq_lens[b], S_cap) + T - 1) / T;
+            base += (L.len(b) + T - 1) / T;
         }
         if (tid == kStreamThreads - 1) prefix[d.B] = base;
         __syncthreads();
+    }
+    if (L.append && cta == 0) {      // a sequence without room for the new token is left as it is and reported
+        for (int b = tid; b < d.B; b += kStreamThreads)
+            if (!L.appends(b)) raise_status(status_word, GTA_ERR_CACHE_FULL);
     }
     const long long n_st = prefix[d.B];
     const long long st_begin = ((long long)cta * n_st) / G, st_end = ((long long)(cta + 1) * n_st) / G;
@@ -292,9 +313,24 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
             l_run = 0.f;
         };
 
+        // Fused append: the new token's rows of the current sequence, two 16-byte vectors per thread at most
+        // (vector v < k_vecs belongs to K, the others to C), fetched when the sequence is taken up so that the
+        // latency has passed when its last sub-tile -- the one that holds the new token -- comes round.
+        const int k_vecs = d.n_k * KH * 8, new_vecs = k_vecs + n_c_tiles * 8;      // 8 vectors per 64-column tile row
+        uint4 nv[2];
+        auto load_new = [&](int b) {
+            if (!L.appends(b)) return;
+#pragma unroll
+            for (int i = 0; i < 2; ++i) {
+                const int v = tid + i * kStreamConsumers;
+                if (v < k_vecs) nv[i] = __ldg(k_new + (size_t)b * k_vecs + v);
+                else if (v < new_vecs) nv[i] = __ldg(c_new + (size_t)b * (new_vecs - k_vecs) + (v - k_vecs));
+            }
+        };
         int b = b0;
         long long k = st_begin - prefix[b0];
         load_q(b);
+        load_new(b);
         int it = 0;
         bool ok = true;
         for (long long st = st_begin; st < st_end; ++st, ++it, ++k) {
@@ -303,13 +339,38 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
                 do { ++b; } while (prefix[b + 1] == prefix[b]);
                 k = 0;
                 load_q(b);
+                load_new(b);
             }
             const int s = it % kStreamStages;
             const uint32_t ph = (it / kStreamStages) & 1;
             ok = __all_sync(0xffffffffu, ptx::mbar_wait(&full_bar[s], ph, abort_flag));
             if (!ok) break;
-            const int len = clamp_len(seq_lens[b], S_cap);
+            const int len = L.len(b);
             const int n_valid = min(T, len - (int)k * T);
+            // the sub-tile that ends the sequence holds the new token (row n_valid - 1): what TMA brought for that
+            // row is whatever the cache held; the new rows are put over it here, and written to the caches
+            const bool patch = L.appends(b) && ((int)k + 1) * T >= len;
+            if (patch) {
+                const int row = n_valid - 1;
+#pragma unroll
+                for (int i = 0; i < 2; ++i) {
+                    const int v = tid + i * kStreamConsumers;
+                    if (v < new_vecs) {
+                        // vector v: tile v >> 3 of the stage (K tiles first, then the C tiles), 16-byte chunk v & 7
+                        uint8_t* p = ring + s * kStageBytes + (v >> 3) * tile_bytes + row * 128 + (((v & 7) ^ (row & 7)) << 4);
+                        *reinterpret_cast<uint4*>(p) = nv[i];
+                        if (v < k_vecs) {       // K row of group v / (8 KH): vector v % (8 KH) of its d_h columns
+                            const int g = v / (8 * KH);
+                            k_rows[(((size_t)b * d.n_k + g) * S_cap + (len - 1)) * (8 * KH) + v % (8 * KH)] = nv[i];
+                        } else {
+                            const int cv = v - k_vecs, g = cv / (8 * NT);
+                            c_rows[(((size_t)b * d.n_c + g) * S_cap + (len - 1)) * (8 * NT) + cv % (8 * NT)] = nv[i];
+                        }
+                    }
+                }
+                ptx::fence_proxy_async_smem();   // the next TMA write of this stage follows generic writes
+                consumer_sync();                 // the scores below read the row
+            }
             const uint32_t stage = ring_addr + s * kStageBytes;
             float* sb = s_buf + (it & 1) * (NQ * T);
 
@@ -443,14 +504,15 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
 __global__ void __launch_bounds__(256)
 decode_merge_kernel(Dims d, int G, int T, int S_cap, const int32_t* __restrict__ seq_lens,
                     const float* __restrict__ part_o, const float* __restrict__ part_ml,
-                    __nv_bfloat16* __restrict__ l_out, long long stride_g, long long stride_b) {
+                    __nv_bfloat16* __restrict__ l_out, long long stride_g, long long stride_b, int append) {
+    const StepLens L{seq_lens, S_cap, append};
     __shared__ long long red_s[2][8];
     __shared__ int live_s[kFinMaxSlots];        // slot j of the range holds something
     ptx::grid_launch_dependents();
     const int g = blockIdx.x, b = blockIdx.y, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     long long before = 0, total = 0;            // sub-tiles of the sequences before b, of all sequences
     for (int i = tid; i < d.B; i += 256) {
-        const int n = (clamp_len(seq_lens[i], S_cap) + T - 1) / T;
+        const int n = (L.len(i) + T - 1) / T;
         total += n;
         if (i < b) before += n;
     }
@@ -464,7 +526,7 @@ decode_merge_kernel(Dims d, int G, int T, int S_cap, const int32_t* __restrict__
     long long s_lo = 0, n_st = 0;
 #pragma unroll
     for (int w = 0; w < 8; ++w) { s_lo += red_s[0][w]; n_st += red_s[1][w]; }
-    const long long s_hi = s_lo + (clamp_len(seq_lens[b], S_cap) + T - 1) / T;
+    const long long s_hi = s_lo + (L.len(b) + T - 1) / T;
     // the owner of sub-tile st is the largest c with floor(c n / G) <= st = floor(((st + 1) G - 1) / n)
     int c_lo = 0, c_hi = -1;
     if (s_hi > s_lo) {
@@ -526,7 +588,8 @@ static cudaError_t launch_stream_and_merge(const Dims& d, const FastPlan& p, con
                                            const void* c_cache, const int32_t* seq_lens, int S_cap, float* part_o,
                                            float* part_ml, __nv_bfloat16* l_out, long long stride_g,
                                            long long stride_b, int32_t* status_word, cudaStream_t stream, int stages,
-                                           int* launches, const PageMap& pm) {
+                                           int* launches, const PageMap& pm, const void* k_new = nullptr,
+                                           const void* c_new = nullptr) {
     cudaError_t err;
     if (stages & 2) {
         CUtensorMap tm_k, tm_c;
@@ -557,7 +620,9 @@ static cudaError_t launch_stream_and_merge(const Dims& d, const FastPlan& p, con
             cfg.attrs = attr;                                                                              \
             cfg.numAttrs = 1;                                                                              \
             err = cudaLaunchKernelEx(&cfg, kern, tm_k, tm_c, d, p.T, S_cap, (const __nv_bfloat16*)q,       \
-                                     seq_lens, part_o, part_ml, status_word, pm);                          \
+                                     seq_lens, part_o, part_ml, status_word, pm, (const uint4*)k_new,      \
+                                     (const uint4*)c_new, (uint4*)const_cast<void*>(k_cache),              \
+                                     (uint4*)const_cast<void*>(c_cache));                                  \
             if (err != cudaSuccess) return err;                                                            \
         } while (0)
 #define GTA_LAUNCH_STREAM(NT)                                                                              \
@@ -604,30 +669,36 @@ static cudaError_t launch_stream_and_merge(const Dims& d, const FastPlan& p, con
         cfg.attrs = attr;
         cfg.numAttrs = 1;
         err = cudaLaunchKernelEx(&cfg, decode_merge_kernel, d, p.G, p.T, S_cap, seq_lens, (const float*)part_o,
-                                 (const float*)part_ml, l_out, stride_g, stride_b);
+                                 (const float*)part_ml, l_out, stride_g, stride_b, k_new != nullptr ? 1 : 0);
         if (err != cudaSuccess) return err;
         *launches += 1;
     }
     return cudaSuccess;
 }
 
+// k_new / c_new != nullptr: the fused append + decode step -- seq_lens does not count the new token yet, the stream
+// kernel puts its rows into the caches and attends over them, the decoder kernel advances the lengths at the end.
 cudaError_t launch_decode_fast(const Dims& d, const void* q, const void* k_cache, const void* c_cache,
                                const int32_t* seq_lens, int S_cap, const void* x_t, const void* w_p,
                                const void* w_g, void* out, void* workspace, int32_t* status_word,
-                               cudaStream_t stream, int stages, int* launches, const PageMap& pm) {
+                               cudaStream_t stream, int stages, int* launches, const PageMap& pm, const void* k_new,
+                               const void* c_new) {
     const FastPlan p = make_fast_plan(d);
     float* part_o = reinterpret_cast<float*>(workspace);
     float* part_ml = reinterpret_cast<float*>(static_cast<char*>(workspace) + p.off_ml);
     __nv_bfloat16* l_g = reinterpret_cast<__nv_bfloat16*>(static_cast<char*>(workspace) + p.off_l);
     cudaError_t err = launch_stream_and_merge(d, p, q, k_cache, c_cache, seq_lens, S_cap, part_o, part_ml, l_g,
-                                              (long long)d.B * d.d_l, d.d_l, status_word, stream, stages, launches, pm);
+                                              (long long)d.B * d.d_l, d.d_l, status_word, stream, stages, launches, pm,
+                                              k_new, c_new);
     if (err != cudaSuccess) return err;
     if (stages & 4) {
         // the batch takes the role of the token axis: L [n_q][B][d_l], x_t [B][H], out [B][n_h][d_h]
         Dims dd = d;
         dd.B = 1;
         dd.N = d.B;
-        if (launch_sm100_decoder(dd, l_g, x_t, w_p, w_g, out, status_word, stream) != GTA_OK) return cudaErrorUnknown;
+        if (launch_sm100_decoder(dd, l_g, x_t, w_p, w_g, out, status_word, stream,
+                                 k_new ? const_cast<int32_t*>(seq_lens) : nullptr, d.B, S_cap) != GTA_OK)
+            return cudaErrorUnknown;
         *launches += 1;
     }
     return cudaSuccess;

@@ -22,8 +22,11 @@ gta_status_t launch_sm100_attention(const Dims& d, const void* q, const void* k,
 gta_status_t sm100_attention_debug_wait(unsigned long long limit_ns, int withhold_first_arrive);
 
 // Decoder + gate kernel alone: out = (L W_P) (.) sigmoid(X W_G) with L[B, n_q, N, d_l] in bf16.
+// step_lens (optional; the fused append + decode step): lengths that the kernel advances by one, where there is room
+// below step_cap, once the kernel before it in the stream is complete.
 gta_status_t launch_sm100_decoder(const Dims& d, const void* l_bf16, const void* x, const void* w_p, const void* w_g,
-                                  void* out, int32_t* status_word, cudaStream_t stream);
+                                  void* out, int32_t* status_word, cudaStream_t stream, int32_t* step_lens = nullptr,
+                                  int step_batch = 0, int step_cap = 0);
 
 // Linear maps of the attention layer around the operator (App. B.1.1), bf16 with fp32 accumulation.
 // True when the tcgen05 kernel covers the layer's projections for this shape.

@@ -116,7 +116,11 @@ template <bool kPair>
 __global__ void __launch_bounds__(kDecThreads, 1)
 sm100_decoder_kernel(const __grid_constant__ CUtensorMap tm_l, const __grid_constant__ CUtensorMap tm_x,
                      const __grid_constant__ CUtensorMap tm_wp, const __grid_constant__ CUtensorMap tm_wg,
-                     Dims d, Schedule sch, __nv_bfloat16* __restrict__ out, int32_t* status_word) {
+                     Dims d, Schedule sch, __nv_bfloat16* __restrict__ out, int32_t* status_word,
+                     int32_t* step_lens, int step_batch, int step_cap) {
+    // step_lens != nullptr (the fused append + decode step): once the kernel before this one is complete --
+    // and with it every reader of the sequence lengths --, the producer thread of CTA 0 advances the length
+    // of every sequence that had room for its new token.
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     // ring: pairs keep {A, B} of a stage side by side; without pairs all A tiles come first, then all B tiles
@@ -201,7 +205,15 @@ sm100_decoder_kernel(const __grid_constant__ CUtensorMap tm_l, const __grid_cons
                                 ptx::tma_load_2d(b_s + grp * kBGroupBytes, &tm_wg, bar, fc + grp * 64, ks * kBlockK);
                         } else {
                             const int kk = ks - ks_g;
-                            if (!l_ready) { ptx::grid_dependency_wait(); l_ready = true; }
+                            if (!l_ready) {
+                                ptx::grid_dependency_wait();
+                                l_ready = true;
+                                if (step_lens != nullptr && blockIdx.x == 0)
+                                    for (int sb = 0; sb < step_batch; ++sb) {
+                                        const int len = step_lens[sb];
+                                        if (len >= 0 && len < step_cap) step_lens[sb] = len + 1;
+                                    }
+                            }
                             ptx::tma_load_3d(a_s, &tm_l, bar, kk * kBlockK, t0, w.b * d.n_q + g);
                             for (int grp = 0; grp < n_grp; ++grp)
                                 ptx::tma_load_3d(b_s + grp * kBGroupBytes, &tm_wp, bar, wp_col[grp], kk * kBlockK,
@@ -220,7 +232,15 @@ sm100_decoder_kernel(const __grid_constant__ CUtensorMap tm_l, const __grid_cons
                         // L comes from the kernel before this one in the stream; this kernel is
                         // launched with programmatic serialisation, so the gate phase above (X, W_G
                         // only) may already have run while that kernel was draining
-                        if (!l_ready) { ptx::grid_dependency_wait(); l_ready = true; }
+                        if (!l_ready) {
+                                ptx::grid_dependency_wait();
+                                l_ready = true;
+                                if (step_lens != nullptr && blockIdx.x == 0)
+                                    for (int sb = 0; sb < step_batch; ++sb) {
+                                        const int len = step_lens[sb];
+                                        if (len >= 0 && len < step_cap) step_lens[sb] = len + 1;
+                                    }
+                            }
                         ptx::tma_load_3d_pair(a_s, &tm_l, bar, kk * kBlockK, t0, w.b * d.n_q + g);
                         for (int grp = 0; grp < n_grp; ++grp)
                             ptx::tma_load_3d_pair(b_s + grp * kBGroupBytes, &tm_wp, bar, wp_col[grp], kk * kBlockK,
@@ -375,7 +395,8 @@ int sm_count() {
 }  // namespace
 
 gta_status_t launch_sm100_decoder(const Dims& d, const void* l_bf16, const void* x, const void* w_p, const void* w_g,
-                                  void* out, int32_t* status_word, cudaStream_t stream) {
+                                  void* out, int32_t* status_word, cudaStream_t stream, int32_t* step_lens,
+                                  int step_batch, int step_cap) {
     CUtensorMap tm_l, tm_x, tm_wp, tm_wg;
     const bool solo = d.N <= kTileM;                                    // one row tile: no CTA pairs
     const uint32_t a_rows = solo ? (uint32_t)((d.N + 7) & ~7) : kTileM; // rows of an A tile
@@ -432,7 +453,7 @@ gta_status_t launch_sm100_decoder(const Dims& d, const void* l_bf16, const void*
         cfg.attrs = attr;
         cfg.numAttrs = 1;
         if (cudaLaunchKernelEx(&cfg, sm100_decoder_kernel<false>, tm_l, tm_x, tm_wp, tm_wg, d, s, (__nv_bfloat16*)out,
-                               status_word) != cudaSuccess)
+                               status_word, step_lens, step_batch, step_cap) != cudaSuccess)
             return GTA_ERR_CUDA;
         return cudaGetLastError() == cudaSuccess ? GTA_OK : GTA_ERR_CUDA;
     }
@@ -482,7 +503,7 @@ gta_status_t launch_sm100_decoder(const Dims& d, const void* l_bf16, const void*
     cfg.gridDim = dim3(2 * G);
     cfg.numAttrs = 2;
     if (cudaLaunchKernelEx(&cfg, sm100_decoder_kernel<true>, tm_l, tm_x, tm_wp, tm_wg, d, s, (__nv_bfloat16*)out,
-                           status_word) != cudaSuccess)
+                           status_word, step_lens, step_batch, step_cap) != cudaSuccess)
         return GTA_ERR_CUDA;
     return cudaGetLastError() == cudaSuccess ? GTA_OK : GTA_ERR_CUDA;
 }

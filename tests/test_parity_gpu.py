@@ -520,3 +520,50 @@ def test_a_wait_that_runs_out_unwinds_the_attention_kernel(B, oracle):
     tc = cpu(t)
     want = oracle.prefill(oracle_shape(w), tc["q"], tc["k"], tc["c"], tc["x"], tc["w_p"], tc["w_g"])
     assert_close(after, want, torch.bfloat16, "after a timed-out call")
+
+
+# --------------------------------------------------------------------------- append + decode in one call
+STEP_CASES = [
+    # name, dtype, H, n_h, n_q, n_k, n_c, d_h, d_l, lens BEFORE the step, S_cap
+    ("bf16_around_the_sub_tiles", "bf16", 256, 8, 4, 4, 1, 128, 512, [0, 1, 30, 31, 32, 33, 63, 64, 65, 700], 720),
+    ("bf16_full_and_nearly_full", "bf16", 128, 4, 2, 2, 1, 128, 256, [128, 127, 5, 126], 128),
+    ("bf16_two_latents_dh64", "bf16", 128, 8, 4, 2, 2, 64, 128, [200, 0, 129, 63, 64], 256),
+    ("bf16_paper_1b_shape", "bf16", 1280, 20, 5, 1, 1, 64, 128, [333, 127, 128], 400),
+    ("bf16_batch_40", "bf16", 256, 8, 4, 4, 1, 128, 512, [(37 * i) % 300 for i in range(40)], 320),
+    ("f32_plain_alu_kernels", "f32", 96, 6, 6, 3, 1, 32, 64, [100, 7, 0, 260], 261),
+]
+
+
+@pytest.mark.parametrize("case", STEP_CASES, ids=[c[0] for c in STEP_CASES])
+def test_decode_append_equals_append_then_decode(B, oracle, case):
+    name, dt, H, n_h, n_q, n_k, n_c, d_h, d_l, lens, cap = case
+    w = I.Workload(name, "decode", dt, len(lens), 0, H, n_h, n_q, n_k, n_c, d_h, d_l, seed=83)
+    t = I.decode_inputs(w, device="cuda", s_cap=cap, seq_lens=lens)
+    status_a = torch.zeros(1, dtype=torch.int32, device="cuda")
+    status_b = torch.zeros(1, dtype=torch.int32, device="cuda")
+    # the two calls
+    k_a, c_a, lens_a = t["k_cache"].clone(), t["c_cache"].clone(), t["seq_lens"].clone()
+    B.gta_cache_append(k_a, c_a, t["k_new"], t["c_new"], lens_a, status_word=status_a)
+    want = B.gta_decode(t["q"], k_a, c_a, lens_a, t["x_t"], t["w_p"], t["w_g"], status_word=status_a)
+    # the one call, twice in a row on fresh copies (leftovers in the workspace must not matter)
+    shape = B.decode_shape(t["q"], t["k_cache"], t["c_cache"], t["x_t"], t["w_p"])
+    ws = Guarded((B.decode_workspace_bytes(shape, cap),), torch.uint8)
+    for rep in range(2):
+        k_b, c_b, lens_b = t["k_cache"].clone(), t["c_cache"].clone(), t["seq_lens"].clone()
+        status_b.zero_()
+        og = Guarded(tuple(want.shape), want.dtype)
+        got = B.gta_decode_append(t["q"], k_b, c_b, t["k_new"], t["c_new"], lens_b, t["x_t"], t["w_p"], t["w_g"],
+                                  out=og.t, workspace=ws.t, status_word=status_b)
+        torch.cuda.synchronize()
+        ws.check(name + " workspace"); og.check(name + " out")
+        assert int(status_b.item()) == int(status_a.item())
+        assert int(status_b.item()) == (B.GTA_ERR_CACHE_FULL if any(n >= cap for n in lens) else 0)
+        assert lens_b.tolist() == lens_a.tolist() == [n + 1 if n < cap else n for n in lens]
+        bits = torch.int16 if dt == "bf16" else torch.int32
+        assert torch.equal(k_b.view(bits), k_a.view(bits)) and torch.equal(c_b.view(bits), c_a.view(bits))
+        assert torch.equal(got.view(bits), want.view(bits))
+    live = max(lens_a.tolist())
+    ref = oracle.decode(oracle_shape(w, seq=0), t["q"].cpu(), k_a[:, :, :live].contiguous().cpu(),
+                        c_a[:, :, :live].contiguous().cpu(), lens_a.cpu().numpy(), live, t["x_t"].cpu(), t["w_p"].cpu(),
+                        t["w_g"].cpu())
+    assert_close(got, ref, w.torch_dtype(), name)
