@@ -5,13 +5,13 @@
 
 One *step* is one pass of the whole hot path over one synthetic batch:
   prefill leg : gta_prefill on workload c2 (B=4, N=2048, H=2048, 16 heads / 4 maps, d_h=128, d_l=512, bf16)
-  decode leg  : gta_cache_append (one token per sequence) + gta_decode on workload c3
-                (B=32, context 4096, same layer shape, bf16), rotating between two cache sets.
+  decode leg  : gta_decode_append (the append of one token per sequence and the decode step in one call) on
+                workload c3 (B=32, context 4096, same layer shape, bf16), rotating between two cache sets.
 The headline `value` is prefill TFLOP/s (causal-useful flops / device time of the prefill legs);
 the decode leg is reported under "decode" (tokens/s, HBM GB/s).  The two largest workloads are
 timed in loops of their own and reported under "legs": c4 (one 16384-token prompt, d_l = 1024:
-gta_prefill) and c5 (128 ragged sequences of 1024..32768 cached tokens: gta_cache_append +
-gta_decode per step), each with its own roofline.  Inputs are resident in HBM for `value`; "e2e"
+gta_prefill) and c5 (128 ragged sequences of 1024..32768 cached tokens: gta_decode_append
+per step), each with its own roofline.  Inputs are resident in HBM for `value`; "e2e"
 repeats the prefill through the public call with pinned HOST buffers, host->device and
 device->host copies inside the timed region.  Prints ONE JSON line on rank 0.
 
@@ -425,15 +425,21 @@ def run_ours(args):
             td["pool"].copy_(td["lens0"].unsqueeze(0).expand(LENS_POOL, -1))
 
     def decode_leg(i, ev=None):
+        # one decode step including the append of its token (gta_decode_append: one call, no append kernel)
         td = sets[i % 2]
         lens = td["pool"][(i // 2) % LENS_POOL]            # this step's own length vector (wd.seq - 1)
-        G.gta_cache_append(td["k_cache"], td["c_cache"], td["k_new"], td["c_new"], lens, status_word=status)
-        launches["n"] += G.last_launch_count()
         if ev is not None:
             ev.record(stream)
+        G.gta_decode_append(td["q"], td["k_cache"], td["c_cache"], td["k_new"], td["c_new"], lens, td["x_t"], td["w_p"],
+                            td["w_g"], out=out_d, workspace=ws_d, status_word=status)
+        launches["n"] += G.last_launch_count()
+
+    def decode_leg_two_calls(i):
+        td = sets[i % 2]
+        lens = td["pool"][(i // 2) % LENS_POOL]
+        G.gta_cache_append(td["k_cache"], td["c_cache"], td["k_new"], td["c_new"], lens, status_word=status)
         G.gta_decode(td["q"], td["k_cache"], td["c_cache"], lens, td["x_t"], td["w_p"], td["w_g"],
                      out=out_d, workspace=ws_d, status_word=status)
-        launches["n"] += G.last_launch_count()
 
     for i in range(max(args.warmup, 3)):
         prefill_leg(); decode_leg(i)
@@ -525,6 +531,7 @@ def run_ours(args):
     #      decode roofline is quoted on; launch gaps between calls are inside the timed region
     K_d = max(K, 40)
     t_decode_b2b, rec_decode_b2b = timed_loop(lambda i: decode_leg(i), K_d, before_rep=reset_lens)
+    t_decode_two, rec_decode_two = timed_loop(decode_leg_two_calls, K_d, before_rep=reset_lens, min_ms=250.0)
     # ---- the gta_decode call alone, back to back (no append; same alternation)
     for td in sets:
         td["seq_lens"].copy_(td["lens0"] + 1)
@@ -811,9 +818,8 @@ def run_ours(args):
 
     def c5_step(i):
         lens = pool5[i % N5]
-        G.gta_cache_append(t5["k_cache"], t5["c_cache"], t5["k_new"], t5["c_new"], lens, status_word=status)
-        G.gta_decode(t5["q"], t5["k_cache"], t5["c_cache"], lens, t5["x_t"], t5["w_p"], t5["w_g"], out=out_5,
-                     workspace=ws_5, status_word=status)
+        G.gta_decode_append(t5["q"], t5["k_cache"], t5["c_cache"], t5["k_new"], t5["c_new"], lens, t5["x_t"], t5["w_p"],
+                            t5["w_g"], out=out_5, workspace=ws_5, status_word=status)
 
     def c5_call(i):
         G.gta_decode(t5["q"], t5["k_cache"], t5["c_cache"], lens5, t5["x_t"], t5["w_p"], t5["w_g"], out=out_5,
@@ -865,10 +871,13 @@ def run_ours(args):
                                                  "included); bytes = live cache + weights + vectors"),
                                "decode_stream", "c3")
     decode_roof["with_append"] = hbm_roofline(by["total"], t_decode_b2b, peaks, rec_decode_b2b["clocks"],
-                                              note="loop of gta_cache_append + gta_decode (each step on its own "
-                                                   "length vector, prepared before the loop)")
+                                              note="loop of gta_decode_append, the step with the append of its token "
+                                                   "in one call (each step on its own length vector, prepared "
+                                                   "before the loop)")
+    decode_roof["with_append_two_calls"] = hbm_roofline(by["total"], t_decode_two, peaks, rec_decode_two["clocks"],
+                                                        note="the same step as gta_cache_append + gta_decode")
     decode = {
-        "workload": wd.name, "step": "gta_cache_append + gta_decode, back to back, two cache sets alternating",
+        "workload": wd.name, "step": "gta_decode_append (append + decode in one call), back to back, two cache sets alternating",
         "ms": t_decode_b2b, "tokens_per_s": world * wd.batch / (t_decode_b2b * 1e-3),
         "ms_decode_call": t_decode_call, "ms_in_step": t_decode_leg, "ms_in_step_decode_call_only": t_decode,
         "roofline": decode_roof, "cpu_baseline": cpu_c3,
@@ -892,7 +901,7 @@ def run_ours(args):
         "c2_prefill_bf16": {"call": "gta_prefill inside the timed step", "ms": t_prefill,
                             "tokens_per_s": world * wp.batch * wp.seq / (t_prefill * 1e-3),
                             "roofline": roofline["whole_prefill"], "cpu_baseline": cpu_baseline},
-        "c3_decode_bf16": {"call": "gta_cache_append + gta_decode, back to back", "ms": t_decode_b2b,
+        "c3_decode_bf16": {"call": "gta_decode_append (append + decode in one call), back to back", "ms": t_decode_b2b,
                            "tokens_per_s": world * wd.batch / (t_decode_b2b * 1e-3),
                            "roofline": decode_roof["with_append"], "roofline_decode_call_only": decode_roof,
                            "cpu_baseline": cpu_c3},
@@ -906,7 +915,7 @@ def run_ours(args):
                                         kernel="prefill_decoder_gate", timing="looped alone")],
             "cpu_baseline": cpu_c4},
         "c5_ragged_decode_bf16": {
-            "call": "gta_cache_append + gta_decode per step, back to back (each step on its own length vector)",
+            "call": "gta_decode_append per step (append + decode in one call), back to back (each step on its own length vector)",
             "ms": t_c5, "tokens_per_s": world * w5.batch / (t_c5 * 1e-3), "loop": rec_c5,
             "live_cache_bytes": by5["cache"], "mean_context": sum(lens5_host) / len(lens5_host),
             "roofline": hbm_roofline(by5["total"] + append_bytes5, t_c5, peaks, rec_c5["clocks"]),
@@ -922,7 +931,7 @@ def run_ours(args):
             "config": {
                 "workload": wp.name, "decode_workload": wd.name, "also": [wd.name, w4.name, w5.name],
                 "prefill_path": {1: "plain-ALU", 2: "tcgen05"}.get(path),
-                "step": "gta_prefill(c2) then gta_cache_append + gta_decode(c3)",
+                "step": "gta_prefill(c2) then gta_decode_append(c3): the decode step with the append of its token",
                 "l2": "working set per step ~415 MB > 126 MB L2: the prefill leg touches 136 MB, the decode leg "
                       "streams 279 MB and alternates between two cache sets",
                 "timed_region": f"exactly {K} steps, repeated {n_reps} times ({device_total:.0f} ms of device time); "
