@@ -205,6 +205,29 @@ GTA_API gta_status_t gta_cache_append_paged(const gta_shape_t *shape, void *k_po
                                             int32_t *status_word, void *cuda_stream);
 
 /*
+ * gta_prefill_chunk_paged — gta_prefill_chunk with the attended keys and latents in a paged cache (pools,
+ * block table and their rules as in gta_decode_paged): attended position j of sequence b, 0 <= j < kv_len, is
+ * row j % page_size of page block_table[b, j / page_size].  Every sequence has the same kv_len, with
+ * N <= kv_len <= page_size * max_pages (else GTA_ERR_INVALID_ARG).  Only the block-table entries of
+ * positions below kv_len are read; the rows of a sequence's last page behind kv_len, and every page no
+ * such entry names, may hold anything (uninitialised memory, NaN bit patterns): nothing of them reaches
+ * out.  An entry in use outside [0, n_pages) raises *status_word to GTA_ERR_BAD_PAGE; no memory outside
+ * the pools is touched, and the keys of such a page take no part in the affected sequence's result
+ * (they are left out of the softmax on the plain-ALU kernels and read as zero rows on the tensor-core
+ * kernels, so that result is unspecified).
+ * q, x, weights, out, workspace (gta_prefill_workspace_bytes), arithmetic and errors as for
+ * gta_prefill_chunk; the tensor-core path applies when, in addition to gta_prefill's rules, page_size is
+ * a multiple of 64, other page sizes run on the plain-ALU kernels.
+ */
+GTA_API gta_status_t gta_prefill_chunk_paged(const gta_shape_t *shape, int32_t kv_len, const void *q,
+                                             const void *k_pool, const void *c_pool,
+                                             const int32_t *block_table, int32_t page_size, int32_t n_pages,
+                                             int32_t max_pages, const void *x, const void *w_p,
+                                             const void *w_g, void *out, void *workspace,
+                                             size_t workspace_bytes, int32_t *status_word,
+                                             void *cuda_stream);
+
+/*
  * gta_layer_prefill — the whole attention layer of App. B.1.1 for a chunk of N tokens per sequence
  * that starts at position pos0 (pos0 = 0: a prompt):
  *
@@ -235,6 +258,25 @@ GTA_API gta_status_t gta_layer_prefill(const gta_shape_t *shape, int32_t pos0, i
                                        void *k_cache, void *c_cache, void *u, void *workspace,
                                        size_t workspace_bytes, int32_t *status_word,
                                        void *cuda_stream);
+
+/*
+ * gta_layer_prefill_paged — gta_layer_prefill over a paged cache (pools, block table and their rules as in
+ * gta_decode_paged; the capacity of a sequence, page_size * max_pages, takes the place of S_cap): the
+ * chunk's keys and latents are written to the rows the block table assigns to positions
+ * pos0 .. pos0 + N - 1, and the chunk attends positions 0 .. pos0 + N - 1 as gta_prefill_chunk_paged
+ * does.  The block-table entries of positions below pos0 + N are read; a row whose entry lies outside
+ * [0, n_pages) is not written and raises *status_word to GTA_ERR_BAD_PAGE.  The caller owns the
+ * assignment of pages; two sequences must not be given the same page for the chunk's positions.
+ * workspace: gta_layer_prefill_workspace_bytes(shape).  Shapes and errors as gta_layer_prefill, plus
+ * GTA_ERR_INVALID_ARG for a bad block table or pool geometry.
+ */
+GTA_API gta_status_t gta_layer_prefill_paged(const gta_shape_t *shape, int32_t pos0, float rope_base,
+                                             const void *x, const void *w_qkc, const void *w_p,
+                                             const void *w_g, const void *w_o, void *k_pool,
+                                             void *c_pool, const int32_t *block_table,
+                                             int32_t page_size, int32_t n_pages, int32_t max_pages,
+                                             void *u, void *workspace, size_t workspace_bytes,
+                                             int32_t *status_word, void *cuda_stream);
 
 /*
  * gta_layer_decode — one decode step of the whole attention layer (App. B.1.1 for the newest token;

@@ -29,6 +29,7 @@ EXPORTS = (
     "gta_layer_decode_paged_workspace_bytes", "gta_layer_decode_paged", "gta_debug_attention_wait",
     "gta_ref_gqa_prefill", "gta_ref_gqa_decode_workspace_bytes", "gta_ref_gqa_decode",
     "gta_decode_fp8_workspace_bytes", "gta_cache_append_fp8", "gta_decode_fp8", "gta_decode_append",
+    "gta_prefill_chunk_paged", "gta_layer_prefill_paged",
 )
 
 
@@ -70,6 +71,11 @@ def lib():
         L.gta_prefill_stages.restype = i32
         L.gta_prefill_chunk.argtypes = [sp, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp, vp]
         L.gta_prefill_chunk.restype = i32
+        L.gta_prefill_chunk_paged.argtypes = [sp, i32, vp, vp, vp, vp, i32, i32, i32, vp, vp, vp, vp, vp, sz, vp, vp]
+        L.gta_prefill_chunk_paged.restype = i32
+        L.gta_layer_prefill_paged.argtypes = [sp, i32, ctypes.c_float, vp, vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, vp,
+                                              vp, sz, vp, vp]
+        L.gta_layer_prefill_paged.restype = i32
         L.gta_decode_stages.argtypes = [sp, vp, vp, vp, vp, i32, vp, vp, vp, vp, vp, sz, vp, vp, i32]
         L.gta_decode_stages.restype = i32
         L.gta_decode_workspace_bytes.argtypes = [sp, i32]
@@ -245,6 +251,75 @@ def gta_prefill_chunk(q, k, c, x, w_p, w_g, kv_len, *, causal=True, softmax_scal
                                  workspace.numel() * workspace.element_size(), _ptr(status_word), _stream(stream))
     if st != GTA_OK:
         raise GtaError(st, "gta_prefill_chunk")
+    return out
+
+
+def _check_pools(k_pool, c_pool, block_table):
+    if block_table.dtype != torch.int32 or block_table.device != k_pool.device or not block_table.is_contiguous() \
+            or block_table.dim() != 2:
+        raise ValueError("block_table must be a contiguous int32 [B, max_pages] tensor on the pools' device")
+    n_pages, n_k, page_size, d_h = k_pool.shape
+    n_c, d_l = c_pool.shape[1], c_pool.shape[3]
+    if c_pool.shape != (n_pages, n_c, page_size, d_l):
+        raise ValueError("inconsistent pool tensor shapes")
+    return n_pages, page_size, block_table.shape[1]
+
+
+def gta_prefill_chunk_paged(q, k_pool, c_pool, block_table, x, w_p, w_g, kv_len, *, causal=True, softmax_scale=0.0,
+                            out=None, workspace=None, status_word=None, stream=None):
+    """gta_prefill_chunk over a paged cache: the N queries are the last N of kv_len positions, whose keys and
+    latents are read from k_pool [n_pages,n_k,page_size,d_h], c_pool [n_pages,n_c,page_size,d_l] through
+    block_table int32 [B,max_pages]."""
+    _check_tensors(q, k_pool, c_pool, x, w_p, w_g)
+    n_pages, page_size, max_pages = _check_pools(k_pool, c_pool, block_table)
+    B, n_q, N, d_h = q.shape
+    n_k, n_c, d_l = k_pool.shape[1], c_pool.shape[1], c_pool.shape[3]
+    n_h, H = w_p.shape[0], x.shape[2]
+    if k_pool.shape[3] != d_h or block_table.shape[0] != B or x.shape != (B, N, H) \
+            or w_p.shape != (n_h, d_l, d_h) or w_g.shape != (H, n_h * d_h):
+        raise ValueError("inconsistent operator tensor shapes")
+    shape = make_shape(batch=B, seq=N, d_model=H, n_heads=n_h, n_q=n_q, n_k=n_k, n_c=n_c, d_h=d_h, d_l=d_l,
+                       dtype=_dtype_code(q), causal=causal, softmax_scale=softmax_scale)
+    if out is None:
+        out = torch.empty((B, N, n_h, d_h), dtype=q.dtype, device=q.device)
+    if workspace is None:
+        workspace = _workspace(prefill_workspace_bytes(shape), q.device)
+    st = lib().gta_prefill_chunk_paged(ctypes.byref(shape), int(kv_len), _ptr(q), _ptr(k_pool), _ptr(c_pool),
+                                       _ptr(block_table), page_size, n_pages, max_pages, _ptr(x), _ptr(w_p),
+                                       _ptr(w_g), _ptr(out), _ptr(workspace),
+                                       workspace.numel() * workspace.element_size(), _ptr(status_word),
+                                       _stream(stream))
+    if st != GTA_OK:
+        raise GtaError(st, "gta_prefill_chunk_paged")
+    return out
+
+
+def gta_layer_prefill_paged(x, w_qkc, w_p, w_g, w_o, k_pool, c_pool, block_table, *, pos0=0, rope_base=10000.0, n_q,
+                            softmax_scale=0.0, out=None, workspace=None, status_word=None, stream=None):
+    """gta_layer_prefill over a paged cache: the chunk's keys and latents are written to the pages that
+    block_table assigns to positions pos0 .. pos0+N-1, and the chunk attends everything up to there."""
+    _check_tensors(x, w_qkc, w_p, w_g, w_o, k_pool, c_pool)
+    n_pages, page_size, max_pages = _check_pools(k_pool, c_pool, block_table)
+    B, N, H = x.shape
+    n_h, d_l, d_h = w_p.shape
+    n_k, n_c = k_pool.shape[1], c_pool.shape[1]
+    if k_pool.shape[3] != d_h or c_pool.shape[3] != d_l or block_table.shape[0] != B \
+            or w_qkc.shape != (H, (n_q + n_k) * d_h + n_c * d_l) or w_g.shape != (H, n_h * d_h) \
+            or w_o.shape != (n_h * d_h, H):
+        raise ValueError("inconsistent layer tensor shapes")
+    shape = make_shape(batch=B, seq=N, d_model=H, n_heads=n_h, n_q=n_q, n_k=n_k, n_c=n_c, d_h=d_h, d_l=d_l,
+                       dtype=_dtype_code(x), causal=True, softmax_scale=softmax_scale)
+    if out is None:
+        out = torch.empty((B, N, H), dtype=x.dtype, device=x.device)
+    if workspace is None:
+        workspace = _workspace(layer_prefill_workspace_bytes(shape), x.device)
+    st = lib().gta_layer_prefill_paged(ctypes.byref(shape), int(pos0), float(rope_base), _ptr(x), _ptr(w_qkc),
+                                       _ptr(w_p), _ptr(w_g), _ptr(w_o), _ptr(k_pool), _ptr(c_pool),
+                                       _ptr(block_table), page_size, n_pages, max_pages, _ptr(out), _ptr(workspace),
+                                       workspace.numel() * workspace.element_size(), _ptr(status_word),
+                                       _stream(stream))
+    if st != GTA_OK:
+        raise GtaError(st, "gta_layer_prefill_paged")
     return out
 
 

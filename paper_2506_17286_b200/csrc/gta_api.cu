@@ -57,7 +57,7 @@ size_t elem_size(int dtype) { return dtype == GTA_F32 ? 4 : 2; }
 static gta_status_t prefill_impl(const gta_shape_t* shape, int32_t kv_len, int32_t kv_cap, const void* q,
                                  const void* k, const void* c, const void* x, const void* w_p, const void* w_g,
                                  void* out, void* workspace, size_t workspace_bytes, int32_t* status_word,
-                                 void* cuda_stream, int32_t stages);
+                                 void* cuda_stream, int32_t stages, const gta::PageMap& pm);
 static gta_status_t decode_impl(const gta_shape_t* shape, const void* q, const void* k_cache, const void* c_cache,
                                 const int32_t* seq_lens, int32_t S_cap, const void* x_t, const void* w_p,
                                 const void* w_g, void* out, void* workspace, size_t workspace_bytes,
@@ -138,7 +138,7 @@ gta_status_t gta_prefill_stages(const gta_shape_t* shape, const void* q, const v
                                 int32_t stages) {
     if (!shape) return GTA_ERR_INVALID_ARG;
     return prefill_impl(shape, shape->seq, shape->seq, q, k, c, x, w_p, w_g, out, workspace, workspace_bytes,
-                        status_word, cuda_stream, stages);
+                        status_word, cuda_stream, stages, gta::PageMap());
 }
 
 gta_status_t gta_prefill_chunk(const gta_shape_t* shape, int32_t kv_len, int32_t kv_cap, const void* q,
@@ -148,7 +148,21 @@ gta_status_t gta_prefill_chunk(const gta_shape_t* shape, int32_t kv_len, int32_t
     if (!shape) return GTA_ERR_INVALID_ARG;
     if (kv_len < shape->seq || kv_cap < kv_len) return GTA_ERR_INVALID_ARG;
     return prefill_impl(shape, kv_len, kv_cap, q, k, c, x, w_p, w_g, out, workspace, workspace_bytes, status_word,
-                        cuda_stream, 3);
+                        cuda_stream, 3, gta::PageMap());
+}
+
+gta_status_t gta_prefill_chunk_paged(const gta_shape_t* shape, int32_t kv_len, const void* q, const void* k_pool,
+                                     const void* c_pool, const int32_t* block_table, int32_t page_size,
+                                     int32_t n_pages, int32_t max_pages, const void* x, const void* w_p,
+                                     const void* w_g, void* out, void* workspace, size_t workspace_bytes,
+                                     int32_t* status_word, void* cuda_stream) {
+    g_last_launches = 0;
+    if (!shape) return GTA_ERR_INVALID_ARG;
+    if (!page_args_ok(block_table, page_size, n_pages, max_pages)) return GTA_ERR_INVALID_ARG;
+    if (kv_len < shape->seq || (long long)kv_len > (long long)page_size * max_pages) return GTA_ERR_INVALID_ARG;
+    return prefill_impl(shape, kv_len, page_size * max_pages, q, k_pool, c_pool, x, w_p, w_g, out, workspace,
+                        workspace_bytes, status_word, cuda_stream, 3,
+                        page_map(block_table, page_size, n_pages, max_pages));
 }
 
 }  // extern "C"
@@ -156,7 +170,7 @@ gta_status_t gta_prefill_chunk(const gta_shape_t* shape, int32_t kv_len, int32_t
 static gta_status_t prefill_impl(const gta_shape_t* shape, int32_t kv_len, int32_t kv_cap, const void* q,
                                  const void* k, const void* c, const void* x, const void* w_p, const void* w_g,
                                  void* out, void* workspace, size_t workspace_bytes, int32_t* status_word,
-                                 void* cuda_stream, int32_t stages) {
+                                 void* cuda_stream, int32_t stages, const gta::PageMap& pm) {
     g_last_launches = 0;
     if (stages < 1 || stages > 3) return GTA_ERR_INVALID_ARG;
     gta::Dims d;
@@ -177,13 +191,15 @@ static gta_status_t prefill_impl(const gta_shape_t* shape, int32_t kv_len, int32
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     int launches = 0;
     cudaError_t err;
-    if (path == 2) {
-        st = gta::launch_sm100_prefill(d, q, k, c, x, w_p, w_g, out, workspace, status_word, stream, stages, &launches);
+    // paged pools: the tensor-core attention kernel loads blocks of 64 tokens, each inside one page
+    if (path == 2 && (pm.table == nullptr || pm.page_size % 64 == 0)) {
+        st = gta::launch_sm100_prefill(d, q, k, c, x, w_p, w_g, out, workspace, status_word, stream, stages, &launches,
+                                       pm);
         if (st != GTA_OK) return st;
         err = cudaSuccess;
     } else {
         err = gta::launch_generic_prefill(d, shape->dtype, q, k, c, x, w_p, w_g, out,
-                                          static_cast<float*>(workspace), stream, stages, &launches);
+                                          static_cast<float*>(workspace), stream, stages, &launches, pm, status_word);
     }
     if (err != cudaSuccess) return GTA_ERR_CUDA;
     g_last_launches = launches;
@@ -259,10 +275,38 @@ extern "C" size_t gta_layer_prefill_workspace_bytes(const gta_shape_t* shape) {
     return q_bytes + o_bytes + align256(gta::sm100_rope_table_bytes(d)) + gta_prefill_workspace_bytes(shape);
 }
 
+static gta_status_t layer_prefill_impl(const gta_shape_t* shape, int32_t pos0, int32_t S_cap, float rope_base,
+                                       const void* x, const void* w_qkc, const void* w_p, const void* w_g,
+                                       const void* w_o, void* k_cache, void* c_cache, void* u, void* workspace,
+                                       size_t workspace_bytes, int32_t* status_word, void* cuda_stream,
+                                       const gta::PageMap& pm);
+
 extern "C" gta_status_t gta_layer_prefill(const gta_shape_t* shape, int32_t pos0, int32_t S_cap, float rope_base,
                                           const void* x, const void* w_qkc, const void* w_p, const void* w_g,
                                           const void* w_o, void* k_cache, void* c_cache, void* u, void* workspace,
                                           size_t workspace_bytes, int32_t* status_word, void* cuda_stream) {
+    return layer_prefill_impl(shape, pos0, S_cap, rope_base, x, w_qkc, w_p, w_g, w_o, k_cache, c_cache, u, workspace,
+                              workspace_bytes, status_word, cuda_stream, gta::PageMap());
+}
+
+extern "C" gta_status_t gta_layer_prefill_paged(const gta_shape_t* shape, int32_t pos0, float rope_base,
+                                                const void* x, const void* w_qkc, const void* w_p, const void* w_g,
+                                                const void* w_o, void* k_pool, void* c_pool,
+                                                const int32_t* block_table, int32_t page_size, int32_t n_pages,
+                                                int32_t max_pages, void* u, void* workspace, size_t workspace_bytes,
+                                                int32_t* status_word, void* cuda_stream) {
+    g_last_launches = 0;
+    if (!page_args_ok(block_table, page_size, n_pages, max_pages)) return GTA_ERR_INVALID_ARG;
+    return layer_prefill_impl(shape, pos0, page_size * max_pages, rope_base, x, w_qkc, w_p, w_g, w_o, k_pool, c_pool, u,
+                              workspace, workspace_bytes, status_word, cuda_stream,
+                              page_map(block_table, page_size, n_pages, max_pages));
+}
+
+static gta_status_t layer_prefill_impl(const gta_shape_t* shape, int32_t pos0, int32_t S_cap, float rope_base,
+                                       const void* x, const void* w_qkc, const void* w_p, const void* w_g,
+                                       const void* w_o, void* k_cache, void* c_cache, void* u, void* workspace,
+                                       size_t workspace_bytes, int32_t* status_word, void* cuda_stream,
+                                       const gta::PageMap& pm) {
     g_last_launches = 0;
     gta::Dims d;
     gta_status_t st = check_shape(shape, true, &d);
@@ -287,11 +331,11 @@ extern "C" gta_status_t gta_layer_prefill(const gta_shape_t* shape, int32_t pos0
     char* op_ws = rope_ws + align256(gta::sm100_rope_table_bytes(d));
     const size_t op_ws_bytes = workspace_bytes - (size_t)(op_ws - ws);
     st = gta::launch_sm100_project(d, pos0, S_cap, (double)rope_base, x, w_qkc, q_ws, k_cache, c_cache, rope_ws,
-                                   status_word, stream);
+                                   status_word, stream, pm);
     if (st != GTA_OK) return st;
     // the chunk's queries against everything the caches now hold for these sequences
     st = prefill_impl(shape, pos0 + d.N, S_cap, q_ws, k_cache, c_cache, x, w_p, w_g, o_ws, op_ws, op_ws_bytes,
-                      status_word, cuda_stream, 3);
+                      status_word, cuda_stream, 3, pm);
     if (st != GTA_OK) return st;
     const int op_launches = g_last_launches;
     st = gta::launch_sm100_matmul((long long)d.B * d.N, d.n_h * d.d_h, d.H, o_ws, w_o, u, status_word, stream);

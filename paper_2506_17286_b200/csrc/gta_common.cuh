@@ -79,7 +79,8 @@ __device__ __forceinline__ long long cache_row(const PageMap& pm, int b, int gro
 // adds the number of launches it made to *launches.
 cudaError_t launch_generic_prefill(const Dims& d, int dtype, const void* q, const void* k, const void* c,
                                    const void* x, const void* w_p, const void* w_g, void* out,
-                                   float* o_lat_ws, cudaStream_t stream, int stages, int* launches);
+                                   float* o_lat_ws, cudaStream_t stream, int stages, int* launches,
+                                   const PageMap& pm = PageMap(), int32_t* status_word = nullptr);
 
 cudaError_t launch_generic_attention_bf16(const Dims& d, const void* q, const void* k, const void* c,
                                           void* o_lat_bf16, cudaStream_t stream, int* launches);

@@ -15,7 +15,7 @@ constexpr int kMaxAccPerLane = 32;  // d_l <= 32 * 32
 template <typename T, typename TO>
 __global__ void __launch_bounds__(kAttnWarps * 32)
 generic_attention_kernel(Dims d, const T* __restrict__ q, const T* __restrict__ k,
-                         const T* __restrict__ c, TO* __restrict__ o_lat) {
+                         const T* __restrict__ c, TO* __restrict__ o_lat, const PageMap pm, int32_t* status_word) {
     extern __shared__ float q_smem[];  // [kAttnWarps][d_h]
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int t = blockIdx.x * kAttnWarps + warp;
@@ -23,8 +23,8 @@ generic_attention_kernel(Dims d, const T* __restrict__ q, const T* __restrict__ 
     if (t >= d.N) return;  // no block-wide barrier below
     const int kg = d.q_to_k(g), cg = d.q_to_c(g);
     const T* q_row = q + (((size_t)b * d.n_q + g) * d.N + t) * d.d_h;
-    const T* k_base = k + ((size_t)b * d.n_k + kg) * (size_t)d.S * d.d_h;
-    const T* c_base = c + ((size_t)b * d.n_c + cg) * (size_t)d.S * d.d_l;
+    // rows of the attended keys and latents: planes of S rows, or (with a page map) pages of a pool; a key whose
+    // block-table entry lies outside the pool takes no part (its score stays -inf)
     float* qs = q_smem + warp * d.d_h;
     for (int e = lane; e < d.d_h; e += 32) qs[e] = to_f32(q_row[e]);
     __syncwarp();
@@ -39,14 +39,22 @@ generic_attention_kernel(Dims d, const T* __restrict__ q, const T* __restrict__ 
     for (int j0 = 0; j0 < n_keys; j0 += 32) {
         const int j = j0 + lane;
         float s = -INFINITY;
+        long long c_idx = -1;
         if (j < n_keys) {
-            const T* k_row = k_base + (size_t)j * d.d_h;
-            float dot = 0.f;
-            for (int e = 0; e < d.d_h; ++e) dot = fmaf(qs[e], to_f32(k_row[e]), dot);
-            s = dot * d.scale;
+            const long long k_idx = cache_row(pm, b, d.n_k, kg, d.S, j, status_word);
+            c_idx = cache_row(pm, b, d.n_c, cg, d.S, j, status_word);
+            if (k_idx >= 0 && c_idx >= 0) {
+                const T* k_row = k + (size_t)k_idx * d.d_h;
+                float dot = 0.f;
+                for (int e = 0; e < d.d_h; ++e) dot = fmaf(qs[e], to_f32(k_row[e]), dot);
+                s = dot * d.scale;
+            } else {
+                c_idx = -1;
+            }
         }
-        const float m_new = fmaxf(m, warp_max(s));  // finite: lane 0 always holds a live key
-        const float p = (j < n_keys) ? expf(s - m_new) : 0.f;
+        const float m_new = fmaxf(m, warp_max(s));
+        if (m_new == -INFINITY) continue;            // only keys on bad pages so far
+        const float p = (c_idx >= 0) ? expf(s - m_new) : 0.f;
         const float corr = expf(m - m_new);          // exp(-inf) = 0 on the first tile
         l = l * corr + warp_sum(p);
         m = m_new;
@@ -55,7 +63,9 @@ generic_attention_kernel(Dims d, const T* __restrict__ q, const T* __restrict__ 
         const int live = min(32, n_keys - j0);
         for (int jj = 0; jj < live; ++jj) {
             const float pj = __shfl_sync(0xffffffffu, p, jj);
-            const T* c_row = c_base + (size_t)(j0 + jj) * d.d_l;
+            const long long cj = __shfl_sync(0xffffffffu, c_idx, jj);
+            if (cj < 0) continue;
+            const T* c_row = c + (size_t)cj * d.d_l;
 #pragma unroll
             for (int a = 0; a < kMaxAccPerLane; ++a) {
                 const int col = lane + 32 * a;
@@ -63,7 +73,7 @@ generic_attention_kernel(Dims d, const T* __restrict__ q, const T* __restrict__ 
             }
         }
     }
-    const float inv_l = 1.f / l;
+    const float inv_l = l > 0.f ? 1.f / l : 0.f;
     TO* o_row = o_lat + (((size_t)b * d.n_q + g) * d.N + t) * d.d_l;
 #pragma unroll
     for (int a = 0; a < kMaxAccPerLane; ++a) {
@@ -157,12 +167,13 @@ generic_decoder_kernel(Dims d, const float* __restrict__ o_lat, const T* __restr
 template <typename T>
 static cudaError_t launch_typed(const Dims& d, const void* q, const void* k, const void* c, const void* x,
                                 const void* w_p, const void* w_g, void* out, float* o_lat_ws,
-                                cudaStream_t stream, int stages, int* launches) {
+                                cudaStream_t stream, int stages, int* launches, const PageMap& pm,
+                                int32_t* status_word) {
     if (stages & 1) {
         dim3 grid_a((d.N + kAttnWarps - 1) / kAttnWarps, d.n_q, d.B);
         const size_t smem = (size_t)kAttnWarps * d.d_h * sizeof(float);
         generic_attention_kernel<T, float><<<grid_a, kAttnWarps * 32, smem, stream>>>(
-            d, (const T*)q, (const T*)k, (const T*)c, o_lat_ws);
+            d, (const T*)q, (const T*)k, (const T*)c, o_lat_ws, pm, status_word);
         cudaError_t err = cudaGetLastError();
         if (err != cudaSuccess) return err;
         *launches += 1;
@@ -179,10 +190,12 @@ static cudaError_t launch_typed(const Dims& d, const void* q, const void* k, con
 
 cudaError_t launch_generic_prefill(const Dims& d, int dtype, const void* q, const void* k, const void* c,
                                    const void* x, const void* w_p, const void* w_g, void* out,
-                                   float* o_lat_ws, cudaStream_t stream, int stages, int* launches) {
+                                   float* o_lat_ws, cudaStream_t stream, int stages, int* launches,
+                                   const PageMap& pm, int32_t* status_word) {
     if (dtype == GTA_F32)
-        return launch_typed<float>(d, q, k, c, x, w_p, w_g, out, o_lat_ws, stream, stages, launches);
-    return launch_typed<__nv_bfloat16>(d, q, k, c, x, w_p, w_g, out, o_lat_ws, stream, stages, launches);
+        return launch_typed<float>(d, q, k, c, x, w_p, w_g, out, o_lat_ws, stream, stages, launches, pm, status_word);
+    return launch_typed<__nv_bfloat16>(d, q, k, c, x, w_p, w_g, out, o_lat_ws, stream, stages, launches, pm,
+                                       status_word);
 }
 
 // Attention stage only, bf16 storage in and out (L written as bf16): feeds the tensor-core
@@ -192,7 +205,8 @@ cudaError_t launch_generic_attention_bf16(const Dims& d, const void* q, const vo
     dim3 grid_a((d.N + kAttnWarps - 1) / kAttnWarps, d.n_q, d.B);
     const size_t smem = (size_t)kAttnWarps * d.d_h * sizeof(float);
     generic_attention_kernel<__nv_bfloat16, __nv_bfloat16><<<grid_a, kAttnWarps * 32, smem, stream>>>(
-        d, (const __nv_bfloat16*)q, (const __nv_bfloat16*)k, (const __nv_bfloat16*)c, (__nv_bfloat16*)o_lat_bf16);
+        d, (const __nv_bfloat16*)q, (const __nv_bfloat16*)k, (const __nv_bfloat16*)c, (__nv_bfloat16*)o_lat_bf16,
+        PageMap(), nullptr);
     *launches += 1;
     return cudaGetLastError();
 }

@@ -150,7 +150,7 @@ template <int DH, int SLICE>
 __global__ void __launch_bounds__(kAttnThreads, 1)
 sm100_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                        const __grid_constant__ CUtensorMap tm_c, const __grid_constant__ CUtensorMap tm_o, Dims d,
-                       int32_t* status_word) {
+                       const PageMap pm, int32_t* status_word) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     float* xchg = reinterpret_cast<float*>(smem + kAttnXchgOff);
@@ -167,6 +167,7 @@ sm100_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     uint64_t* o_item = bars + 24;       // both CTAs (multicast commit): the last sum of an item is complete
     uint64_t* chain = bars + 25;        // [4 groups][4 quarters] this CTA; one warp arrives: its rows' running maxima are published
     uint64_t* mma_drain = bars + 42;    // [2] leader CTA: used once by an MMA-issuing thread that unwinds (all its MMAs are done)
+    uint64_t* tail_bar = bars + 46;     // this CTA, paged pools only: the latent block whose last rows the producer clears
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 44);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
     volatile int* drain_flag = abort_flag + 1;
@@ -187,6 +188,7 @@ sm100_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     // A latent of only SLICE / 2 columns (the comparison operators with d_h = 64 values): both CTAs of the
     // pair stage the same columns, so the second half of O repeats the first and is not stored.
     const bool narrow = d.d_l * 2 == SLICE;
+    const bool paged = pm.table != nullptr;
     const int n_slices = narrow ? 1 : d.d_l / SLICE;
     const int n_qt = (d.N + 127) / 128, n_qp = (n_qt + 1) / 2;
     const int n_kt = (d.Nk + 127) / 128;          // key tiles
@@ -198,6 +200,7 @@ sm100_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         ptx::mbar_init(&mma_drain[0], 1);
         ptx::mbar_init(&mma_drain[1], 1);
         ptx::mbar_init(stage_free, 1);
+        ptx::mbar_init(tail_bar, 1);
         for (int s = 0; s < kAttnStages; ++s) { ptx::mbar_init(&full[s], 2); ptx::mbar_init(&empty[s], 1); }
         for (int s = 0; s < kAttnGroups; ++s) {
             ptx::mbar_init(&s_full[s], 1); ptx::mbar_init(&p_full[s], 8); ptx::mbar_init(&o_done[s], 1);
@@ -231,6 +234,18 @@ sm100_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
             ptx::prefetch_tensormap(&tm_q); ptx::prefetch_tensormap(&tm_k); ptx::prefetch_tensormap(&tm_c);
             int tj = 0;                 // key tiles issued so far (ring position), across items
             int n_armed = 0;            // query tiles whose load has been issued
+            int tail_armed = 0;         // loads through tail_bar
+            const uint32_t tail_bar_addr = ptx::map_to_cta(ptx::smem_addr(tail_bar), rank);
+            // (row, plane) coordinates of the 64 cached tokens from `token` on of sequence b in a pool of `groups`
+            auto page_block = [&](int b, int token, int groups, int grp, int& row, int& plane) {
+                row = pm.page_size;     // past the page: the box reads as zeros
+                plane = 0;
+                if (token >= d.Nk) return;
+                const int page = pm.table[(size_t)b * pm.max_pages + token / pm.page_size];
+                if (page < 0 || page >= pm.n_pages) { raise_status(status_word, GTA_ERR_BAD_PAGE); return; }
+                row = token % pm.page_size;
+                plane = page * groups + grp;
+            };
             bool ok = true;
             AttnItem w;
             for (int n = 0; ok && attn_item(d, n_kt, n_qp, n_slices, total, G, pr, n, &w); ++n) {
@@ -254,16 +269,62 @@ sm100_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                     uint8_t* k_s = smem + kAttnRingOff + s * kAttnStageBytes;
                     uint8_t* c_s = k_s + kKHalfBytes;
                     const uint32_t bar = ptx::map_to_cta(ptx::smem_addr(&full[s]), 0);
-                    ptx::mbar_arrive_expect_tx_cluster(bar, kKLoadBytes + kCLoadBytes);
                     const int key0 = j * kKeyTile + (int)rank * 64;         // this CTA's 64 keys of the tile
-                    ptx::tma_load_3d_pair(k_s, &tm_k, bar, 0, key0, w.b * d.n_k + kg);
-                    if (DH == 128) ptx::tma_load_3d_pair(k_s + 8192, &tm_k, bar, 64, key0, w.b * d.n_k + kg);
                     const int col0 = narrow ? 0 : w.slice * SLICE + (int)rank * (SLICE / 2);     // this CTA's latent columns
-                    ptx::tma_load_3d_pair(c_s, &tm_c, bar, col0, j * kKeyTile, w.b * d.n_c + cg);
-                    if (SLICE == 256)
-                        ptx::tma_load_3d_pair(c_s + 16384, &tm_c, bar, col0 + 64, j * kKeyTile, w.b * d.n_c + cg);
+                    if (!paged) {
+                        ptx::mbar_arrive_expect_tx_cluster(bar, kKLoadBytes + kCLoadBytes);
+                        ptx::tma_load_3d_pair(k_s, &tm_k, bar, 0, key0, w.b * d.n_k + kg);
+                        if (DH == 128) ptx::tma_load_3d_pair(k_s + 8192, &tm_k, bar, 64, key0, w.b * d.n_k + kg);
+                        ptx::tma_load_3d_pair(c_s, &tm_c, bar, col0, j * kKeyTile, w.b * d.n_c + cg);
+                        if (SLICE == 256)
+                            ptx::tma_load_3d_pair(c_s + 16384, &tm_c, bar, col0 + 64, j * kKeyTile, w.b * d.n_c + cg);
+                        continue;
+                    }
+                    // Paged pools: the maps are [pages x groups][page_size][width] and every load is a block of 64
+                    // tokens, which lies inside one page (page_size is a multiple of 64).  A block past the attended
+                    // keys, or one whose page number is outside the pool, is loaded from a row coordinate past the
+                    // page, i.e. as zeros.
+                    int k_row, k_plane, c_row[2], c_plane[2];
+                    page_block(w.b, key0, d.n_k, kg, k_row, k_plane);
+                    page_block(w.b, j * kKeyTile, d.n_c, cg, c_row[0], c_plane[0]);
+                    page_block(w.b, j * kKeyTile + 64, d.n_c, cg, c_row[1], c_plane[1]);
+                    // The block that holds position Nk: its rows from Nk on exist in the page and may hold anything.
+                    // As keys they are masked, but as latent rows they would meet their zero probabilities in the
+                    // sum (0 x NaN), so this block goes through a barrier of this CTA, the thread clears those rows
+                    // in shared memory, and only then arrives at the tile's barrier.
+                    const int tail_h = (d.Nk & 63) ? (d.Nk - j * kKeyTile) >> 6 : -1;     // 0 or 1: the tile's half with that block
+                    const bool tail = (tail_h == 0 || tail_h == 1) && c_row[tail_h & 1] < pm.page_size;
+                    if (tail) {
+                        ptx::mbar_expect_tx_cluster(bar, kKLoadBytes + kCLoadBytes / 2);
+                        ptx::mbar_arrive_expect_tx(tail_bar, kCLoadBytes / 2);
+                        ++tail_armed;
+                    } else {
+                        ptx::mbar_arrive_expect_tx_cluster(bar, kKLoadBytes + kCLoadBytes);
+                    }
+                    ptx::tma_load_3d_pair(k_s, &tm_k, bar, 0, k_row, k_plane);
+                    if (DH == 128) ptx::tma_load_3d_pair(k_s + 8192, &tm_k, bar, 64, k_row, k_plane);
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+                        const uint32_t hb = (tail && h == tail_h) ? tail_bar_addr : bar;
+                        ptx::tma_load_3d_pair(c_s + h * 8192, &tm_c, hb, col0, c_row[h], c_plane[h]);
+                        if (SLICE == 256)
+                            ptx::tma_load_3d_pair(c_s + 16384 + h * 8192, &tm_c, hb, col0 + 64, c_row[h], c_plane[h]);
+                    }
+                    if (tail) {
+                        ok = wait(tail_bar, (tail_armed - 1) & 1);
+                        if (!ok) break;
+                        const int live = d.Nk & 63;                       // rows of the block that are keys
+                        const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
+                        for (int grp = 0; grp < SLICE / 128; ++grp) {     // 64-column groups of this CTA: 128 bytes a row
+                            uint4* z = reinterpret_cast<uint4*>(c_s + grp * 16384 + tail_h * 8192 + live * 128);
+                            for (int i = 0; i < (64 - live) * 8; ++i) z[i] = zero;
+                        }
+                        ptx::fence_proxy_async_smem();                    // the MMAs read these rows through the async proxy
+                        ptx::mbar_arrive_release_cluster(bar);
+                    }
                 }
             }
+            if (*abort_flag && tail_armed > 0) ptx::mbar_wait_drain(tail_bar, (tail_armed - 1) & 1, drain_flag);
             if (*abort_flag && rank == 0) {
                 // Unwinding: wait (bounded) for the copies that were armed, so that none lands after the CTA has
                 // left.  At most the last two query tiles and the last three ring tiles can be outstanding (the
@@ -307,6 +368,7 @@ sm100_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                         if (ok && j == 0) ok = wait(&q_full[(n & 1) * 41], (n >> 1) & 1);
                         if (ok && (j & 1) == 0) ok = wait(&full[stage], (tile / kAttnStages) & 1);
                         if (!ok) break;
+                        if (paged) ptx::fence_acq_rel_cluster();   // rows of the tile that the peer's producer cleared
                         ptx::tc_fence_after_sync();
                         // this CTA's keys 32 (j & 1) .. of its 64 keys of the ring tile: 32 rows of 128 bytes further
                         // on; 32 bytes per k-step inside a 64-column half, the next half 16 KB (Q) / 8 KB (K) on
@@ -607,7 +669,7 @@ bool sm100_prefill_supported(const Dims& d, int dtype) {
 
 // One instantiation of the attention kernel: its occupancy (asked once per device) and its launch.
 template <int DH, int SLICE>
-static gta_status_t launch_attention(const Dims& d, const CUtensorMap& tm_q, const CUtensorMap& tm_k,
+static gta_status_t launch_attention(const Dims& d, const PageMap& pm, const CUtensorMap& tm_q, const CUtensorMap& tm_k,
                                      const CUtensorMap& tm_c, const CUtensorMap& tm_o, int32_t* status_word,
                                      cudaStream_t stream) {
     auto kern = sm100_attention_kernel<DH, SLICE>;
@@ -645,26 +707,36 @@ static gta_status_t launch_attention(const Dims& d, const CUtensorMap& tm_q, con
     const int pairs = (int)(n_items < cached_pairs ? n_items : cached_pairs);
     cfg.gridDim = dim3(2 * pairs);
     cfg.numAttrs = 2;
-    if (cudaLaunchKernelEx(&cfg, kern, tm_q, tm_k, tm_c, tm_o, d, status_word) != cudaSuccess) return GTA_ERR_CUDA;
+    if (cudaLaunchKernelEx(&cfg, kern, tm_q, tm_k, tm_c, tm_o, d, pm, status_word) != cudaSuccess) return GTA_ERR_CUDA;
     return cudaGetLastError() == cudaSuccess ? GTA_OK : GTA_ERR_CUDA;
 }
 
 // L[B, n_q, N, d_l] (bf16) = Softmax(scale Q K^T) C per attention map: the attention kernel alone.  d_l is a
 // multiple of 128, or 64 (the narrow case of the comparison operators).
 gta_status_t launch_sm100_attention(const Dims& d, const void* q, const void* k, const void* c, void* l_out,
-                                    int32_t* status_word, cudaStream_t stream) {
+                                    int32_t* status_word, cudaStream_t stream, const PageMap& pm) {
     CUtensorMap tm_q, tm_k, tm_c, tm_o;
     const uint32_t box[3] = {64, 128, 1}, box_k[3] = {64, 64, 1};
     const uint64_t dq[3] = {(uint64_t)d.d_h, (uint64_t)d.N, (uint64_t)d.B * d.n_q};
-    // K / C: Nk of the S rows of a plane take part; the rest (the unused tail of a cache, which may hold
-    // anything, NaN bit patterns included) lies outside the maps and reads as zeros
-    const uint64_t dk[3] = {(uint64_t)d.d_h, (uint64_t)d.Nk, (uint64_t)d.B * d.n_k};
-    const uint64_t dc[3] = {(uint64_t)d.d_l, (uint64_t)d.Nk, (uint64_t)d.B * d.n_c};
-    const uint64_t ak[3] = {(uint64_t)d.d_h, (uint64_t)d.S, (uint64_t)d.B * d.n_k};
-    const uint64_t ac[3] = {(uint64_t)d.d_l, (uint64_t)d.S, (uint64_t)d.B * d.n_c};
-    if (!make_bf16_map(&tm_q, q, 3, dq, box) || !make_bf16_map(&tm_k, k, 3, dk, box_k, ak) ||
-        !make_bf16_map(&tm_c, c, 3, dc, box, ac))
-        return GTA_ERR_CUDA;
+    if (pm.table != nullptr) {
+        // paged pools [n_pages, groups, page_size, width]: one plane per (page, group), blocks of 64 tokens
+        if (pm.page_size % 64 != 0) return GTA_ERR_UNSUPPORTED;
+        const uint64_t pk[3] = {(uint64_t)d.d_h, (uint64_t)pm.page_size, (uint64_t)pm.n_pages * d.n_k};
+        const uint64_t pc[3] = {(uint64_t)d.d_l, (uint64_t)pm.page_size, (uint64_t)pm.n_pages * d.n_c};
+        if (!make_bf16_map(&tm_q, q, 3, dq, box) || !make_bf16_map(&tm_k, k, 3, pk, box_k) ||
+            !make_bf16_map(&tm_c, c, 3, pc, box_k))
+            return GTA_ERR_CUDA;
+    } else {
+        // K / C: Nk of the S rows of a plane take part; the rest (the unused tail of a cache, which may hold
+        // anything, NaN bit patterns included) lies outside the maps and reads as zeros
+        const uint64_t dk[3] = {(uint64_t)d.d_h, (uint64_t)d.Nk, (uint64_t)d.B * d.n_k};
+        const uint64_t dc[3] = {(uint64_t)d.d_l, (uint64_t)d.Nk, (uint64_t)d.B * d.n_c};
+        const uint64_t ak[3] = {(uint64_t)d.d_h, (uint64_t)d.S, (uint64_t)d.B * d.n_k};
+        const uint64_t ac[3] = {(uint64_t)d.d_l, (uint64_t)d.S, (uint64_t)d.B * d.n_c};
+        if (!make_bf16_map(&tm_q, q, 3, dq, box) || !make_bf16_map(&tm_k, k, 3, dk, box_k, ak) ||
+            !make_bf16_map(&tm_c, c, 3, dc, box, ac))
+            return GTA_ERR_CUDA;
+    }
     {   // L [B n_q][N][d_l], stored in boxes of 128 rows x 64 columns
         const uint64_t dl[3] = {(uint64_t)d.d_l, (uint64_t)d.N, (uint64_t)d.B * d.n_q};
         const uint32_t box_o[3] = {64, 128, 1};
@@ -672,20 +744,21 @@ gta_status_t launch_sm100_attention(const Dims& d, const void* q, const void* k,
     }
     gta_status_t st;
     if (d.d_h == 128)
-        st = d.d_l % 256 == 0 ? launch_attention<128, 256>(d, tm_q, tm_k, tm_c, tm_o, status_word, stream)
-                              : launch_attention<128, 128>(d, tm_q, tm_k, tm_c, tm_o, status_word, stream);
+        st = d.d_l % 256 == 0 ? launch_attention<128, 256>(d, pm, tm_q, tm_k, tm_c, tm_o, status_word, stream)
+                              : launch_attention<128, 128>(d, pm, tm_q, tm_k, tm_c, tm_o, status_word, stream);
     else
-        st = d.d_l % 256 == 0 ? launch_attention<64, 256>(d, tm_q, tm_k, tm_c, tm_o, status_word, stream)
-                              : launch_attention<64, 128>(d, tm_q, tm_k, tm_c, tm_o, status_word, stream);
+        st = d.d_l % 256 == 0 ? launch_attention<64, 256>(d, pm, tm_q, tm_k, tm_c, tm_o, status_word, stream)
+                              : launch_attention<64, 128>(d, pm, tm_q, tm_k, tm_c, tm_o, status_word, stream);
     if (st != GTA_OK) return st;
     return cudaGetLastError() == cudaSuccess ? GTA_OK : GTA_ERR_CUDA;
 }
 
 gta_status_t launch_sm100_prefill(const Dims& d, const void* q, const void* k, const void* c, const void* x,
                                   const void* w_p, const void* w_g, void* out, void* workspace,
-                                  int32_t* status_word, cudaStream_t stream, int stages, int* launches) {
+                                  int32_t* status_word, cudaStream_t stream, int stages, int* launches,
+                                  const PageMap& pm) {
     if (stages & 1) {
-        gta_status_t st = launch_sm100_attention(d, q, k, c, workspace, status_word, stream);
+        gta_status_t st = launch_sm100_attention(d, q, k, c, workspace, status_word, stream, pm);
         if (st != GTA_OK) return st;
         *launches += 1;
     }

@@ -11,12 +11,14 @@ bool sm100_prefill_supported(const Dims& d, int dtype);
 // Enqueues the tensor-core prefill (attention kernel + decoder kernel) on `stream`.
 gta_status_t launch_sm100_prefill(const Dims& d, const void* q, const void* k, const void* c, const void* x,
                                   const void* w_p, const void* w_g, void* out, void* workspace,
-                                  int32_t* status_word, cudaStream_t stream, int stages, int* launches);
+                                  int32_t* status_word, cudaStream_t stream, int stages, int* launches,
+                                  const PageMap& pm = PageMap());
 
 // Attention kernel alone: L[B, n_q, N, d_l] (bf16) = Softmax(scale Q K^T) C per attention map; bf16, d_h = 64 or
-// 128, d_l a multiple of 128 or exactly 64.
+// 128, d_l a multiple of 128 or exactly 64.  With a page map, k and c are paged pools (page_size a multiple of 64)
+// and token t of sequence b is looked up through the block table.
 gta_status_t launch_sm100_attention(const Dims& d, const void* q, const void* k, const void* c, void* l_out,
-                                    int32_t* status_word, cudaStream_t stream);
+                                    int32_t* status_word, cudaStream_t stream, const PageMap& pm = PageMap());
 
 // Test hooks of the attention kernel's bounded waits (see gta_debug_attention_wait in gta.h).
 gta_status_t sm100_attention_debug_wait(unsigned long long limit_ns, int withhold_first_arrive);
@@ -33,12 +35,13 @@ gta_status_t launch_sm100_decoder(const Dims& d, const void* l_bf16, const void*
 bool sm100_linear_supported(const Dims& d, int dtype);
 
 // [Q | K | C] = X W_qkc for the B x N tokens of a chunk that starts at position pos0: RoPE on q and k,
-// q to q_out [B, n_q, N, d_h], k and c to rows pos0 + t of the caches [B, groups, S_cap, width].
+// q to q_out [B, n_q, N, d_h], k and c to rows pos0 + t of the caches [B, groups, S_cap, width] (with a page map:
+// of the paged pools, S_cap then being page_size * max_pages).
 // rope_table: sm100_rope_table_bytes(d) bytes of scratch (cos / sin of the chunk's positions).
 size_t sm100_rope_table_bytes(const Dims& d);
 gta_status_t launch_sm100_project(const Dims& d, int pos0, int S_cap, double rope_base, const void* x,
                                   const void* w_qkc, void* q_out, void* k_cache, void* c_cache, void* rope_table,
-                                  int32_t* status_word, cudaStream_t stream);
+                                  int32_t* status_word, cudaStream_t stream, const PageMap& pm = PageMap());
 
 // One decode step of the same projection: one new token per sequence at position seq_lens[b] (RoPE there,
 // k and c to that cache row, q to q_out [B, n_q, d_h]), then seq_lens[b] += 1; a sequence whose cache is full

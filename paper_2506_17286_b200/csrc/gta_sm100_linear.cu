@@ -517,7 +517,7 @@ size_t sm100_rope_table_bytes(const Dims& d) { return (size_t)d.N * (d.d_h / 2) 
 
 gta_status_t launch_sm100_project(const Dims& d, int pos0, int S_cap, double rope_base, const void* x,
                                   const void* w_qkc, void* q_out, void* k_cache, void* c_cache, void* rope_table,
-                                  int32_t* status_word, cudaStream_t stream) {
+                                  int32_t* status_word, cudaStream_t stream, const PageMap& pm) {
     LinArgs a = {};
     if (!fill_common(a, (long long)d.B * d.N, d.H, (d.n_q + d.n_k) * d.d_h + d.n_c * d.d_l)) return GTA_ERR_UNSUPPORTED;
     a.d = d;
@@ -527,6 +527,7 @@ gta_status_t launch_sm100_project(const Dims& d, int pos0, int S_cap, double rop
     a.k_cache = static_cast<__nv_bfloat16*>(k_cache);
     a.c_cache = static_cast<__nv_bfloat16*>(c_cache);
     a.rope = static_cast<const float2*>(rope_table);
+    a.pm = pm;
     RopeArgs r = {};
     r.pos0 = pos0;
     r.n_pairs = d.d_h / 2;

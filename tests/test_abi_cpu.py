@@ -163,6 +163,30 @@ def test_bad_arguments_are_rejected_on_the_host(B):
     assert append_paged(good, n_new=-1) == B.GTA_ERR_INVALID_ARG
     assert append_paged(good, n_new=0) == B.GTA_OK
 
+    def chunk_paged(shape, kv_len, table=p, page_size=64, n_pages=10, max_pages=4, ws_bytes=1 << 40):
+        return L.gta_prefill_chunk_paged(ctypes.byref(shape), kv_len, p, p, p, table, page_size, n_pages, max_pages,
+                                         p, p, p, p, p, ws_bytes, None, None)
+
+    assert chunk_paged(good, n, table=None) == B.GTA_ERR_INVALID_ARG
+    assert chunk_paged(good, n, table=odd) == B.GTA_ERR_INVALID_ARG
+    assert chunk_paged(good, n, page_size=0) == B.GTA_ERR_INVALID_ARG
+    assert chunk_paged(good, n - 1) == B.GTA_ERR_INVALID_ARG             # fewer keys than queries
+    assert chunk_paged(good, 64 * 4 + 1) == B.GTA_ERR_INVALID_ARG        # more keys than the block table covers
+    assert chunk_paged(good, n, ws_bytes=8) == B.GTA_ERR_WORKSPACE
+    assert chunk_paged(_shape(B, seq=0), 16) == B.GTA_OK                 # no queries: no-op
+    assert L.gta_prefill_chunk_paged(None, 8, p, p, p, p, 64, 10, 4, p, p, p, p, p, 1 << 40, None,
+                                     None) == B.GTA_ERR_INVALID_ARG
+
+    def layer_prefill_paged(shape, pos0=0, table=p, page_size=64, max_pages=2, base=10000.0, ws_bytes=1 << 40):
+        return L.gta_layer_prefill_paged(ctypes.byref(shape), pos0, ctypes.c_float(base), p, p, p, p, p, p, p, table,
+                                         page_size, 10, max_pages, p, p, ws_bytes, None, None)
+
+    assert layer_prefill_paged(lay, table=None) == B.GTA_ERR_INVALID_ARG
+    assert layer_prefill_paged(lay, page_size=-4) == B.GTA_ERR_INVALID_ARG
+    assert layer_prefill_paged(lay, pos0=65) == B.GTA_ERR_INVALID_ARG     # 65 + 64 tokens do not fit two pages
+    assert layer_prefill_paged(lay, base=1.0) == B.GTA_ERR_INVALID_ARG
+    assert layer_prefill_paged(lay, ws_bytes=8) == B.GTA_ERR_WORKSPACE
+
 
 def test_binding_rejects_cpu_tensors_and_missing_library(B, monkeypatch):
     import torch
