@@ -384,10 +384,15 @@ GTA_API gta_status_t gta_decode_append(const gta_shape_t *shape, const void *q, 
  * gta_cache_append; codes and scales are bit-exact functions of the new rows.  gta_decode_fp8 is
  * gta_decode over such caches (q, x_t, w_p, w_g, out in the shape's dtype; rows at and behind
  * seq_lens[b] may hold anything).  Needs d_h and d_l multiples of 16, d_l <= 2048; contiguous
- * caches only.  These calls run on the plain-ALU kernels: they halve the cache but are not at the
- * HBM roofline (the measured figures are in the benchmark's output).
+ * caches only.  gta_decode_fp8 has a streaming path (TMA ring, warp-level MMAs on the e4m3 codes
+ * themselves, query rows and probabilities carried as sums of two e4m3 numbers, merge and tensor-core
+ * decoder kernels of gta_decode) for bf16 operator tensors with d_h = 128, one latent group,
+ * d_l in {128, 256, 512, 1024}, at most 8 maps over 1, 2, 4 or 8 key groups, S_cap a multiple of 4
+ * and 16-byte aligned scale arrays; everything else, and the append, runs on the plain-ALU kernels.
+ * gta_decode_fp8_path says which (0 unsupported, 1 plain-ALU, 2 streaming, alignment aside).
  */
 GTA_API size_t gta_decode_fp8_workspace_bytes(const gta_shape_t *shape, int32_t S_cap);
+GTA_API int gta_decode_fp8_path(const gta_shape_t *shape, int32_t S_cap);
 GTA_API gta_status_t gta_cache_append_fp8(const gta_shape_t *shape, void *k_codes, void *c_codes,
                                           float *k_scales, float *c_scales, int32_t S_cap,
                                           const void *k_new, const void *c_new, int32_t n_new,

@@ -29,7 +29,7 @@ EXPORTS = (
     "gta_layer_decode_paged_workspace_bytes", "gta_layer_decode_paged", "gta_debug_attention_wait",
     "gta_ref_gqa_prefill", "gta_ref_gqa_decode_workspace_bytes", "gta_ref_gqa_decode",
     "gta_decode_fp8_workspace_bytes", "gta_cache_append_fp8", "gta_decode_fp8", "gta_decode_append",
-    "gta_prefill_chunk_paged", "gta_layer_prefill_paged",
+    "gta_prefill_chunk_paged", "gta_layer_prefill_paged", "gta_decode_fp8_path",
 )
 
 
@@ -119,6 +119,8 @@ def lib():
         L.gta_ref_gqa_decode.restype = i32
         L.gta_decode_fp8_workspace_bytes.argtypes = [sp, i32]
         L.gta_decode_fp8_workspace_bytes.restype = sz
+        L.gta_decode_fp8_path.argtypes = [sp, i32]
+        L.gta_decode_fp8_path.restype = i32
         L.gta_cache_append_fp8.argtypes = [sp, vp, vp, vp, vp, i32, vp, vp, i32, vp, vp, vp]
         L.gta_cache_append_fp8.restype = i32
         L.gta_decode_fp8.argtypes = [sp, vp, vp, vp, vp, vp, vp, i32, vp, vp, vp, vp, vp, sz, vp, vp]
@@ -618,6 +620,11 @@ def gta_cache_append_fp8(k_codes, c_codes, k_scales, c_scales, k_new, c_new, seq
     if st != GTA_OK:
         raise GtaError(st, "gta_cache_append_fp8")
     return seq_lens
+
+
+def decode_fp8_path(shape: GtaShape, s_cap: int) -> int:
+    """0 unsupported, 1 plain-ALU kernels, 2 streaming kernels."""
+    return int(lib().gta_decode_fp8_path(ctypes.byref(shape), int(s_cap)))
 
 
 def decode_fp8_workspace_bytes(shape: GtaShape, s_cap: int) -> int:

@@ -595,10 +595,26 @@ static gta_status_t fp8_check(const gta_shape_t* shape, gta::Dims* d) {
     return GTA_OK;
 }
 
+// enough for either kernel family (which one runs also depends on the alignment of the scale arrays)
+static size_t fp8_workspace(const gta::Dims& d, int dtype, int S_cap) {
+    size_t need = gta::decode_fp8_workspace_bytes(d, S_cap);
+    if (gta::decode_fp8_fast_supported(d, dtype, S_cap)) {
+        const size_t fast = gta::decode_fp8_fast_workspace_bytes(d);
+        need = fast > need ? fast : need;
+    }
+    return need;
+}
+
 extern "C" size_t gta_decode_fp8_workspace_bytes(const gta_shape_t* shape, int32_t S_cap) {
     gta::Dims d;
     if (fp8_check(shape, &d) != GTA_OK || S_cap < 0) return 0;
-    return gta::decode_fp8_workspace_bytes(d, S_cap);
+    return fp8_workspace(d, shape->dtype, S_cap);
+}
+
+extern "C" int gta_decode_fp8_path(const gta_shape_t* shape, int32_t S_cap) {
+    gta::Dims d;
+    if (fp8_check(shape, &d) != GTA_OK || S_cap <= 0) return 0;
+    return gta::decode_fp8_fast_supported(d, shape->dtype, S_cap) ? 2 : 1;
 }
 
 extern "C" gta_status_t gta_cache_append_fp8(const gta_shape_t* shape, void* k_codes, void* c_codes, float* k_scales,
@@ -641,13 +657,19 @@ extern "C" gta_status_t gta_decode_fp8(const gta_shape_t* shape, const void* q, 
         !aligned(seq_lens, 4) || !aligned(status_word, 4))
         return GTA_ERR_INVALID_ARG;
     if (d.B == 0) return GTA_OK;
-    if (!workspace || !aligned(workspace, 256) || workspace_bytes < gta::decode_fp8_workspace_bytes(d, S_cap))
+    if (!workspace || !aligned(workspace, 256) || workspace_bytes < fp8_workspace(d, shape->dtype, S_cap))
         return GTA_ERR_WORKSPACE;
     if ((st = check_device()) != GTA_OK) return st;
     int launches = 0;
-    cudaError_t err = gta::launch_decode_fp8(d, shape->dtype, q, k_codes, c_codes, k_scales, c_scales, seq_lens, S_cap,
-                                             x_t, w_p, w_g, out, workspace, status_word,
-                                             static_cast<cudaStream_t>(cuda_stream), &launches);
+    cudaError_t err;
+    // the streaming kernel copies the scale rows in 16-byte pieces
+    if (gta::decode_fp8_fast_supported(d, shape->dtype, S_cap) && aligned(k_scales, 16) && aligned(c_scales, 16))
+        err = gta::launch_decode_fp8_fast(d, q, k_codes, c_codes, k_scales, c_scales, seq_lens, S_cap, x_t, w_p, w_g, out,
+                                          workspace, status_word, static_cast<cudaStream_t>(cuda_stream), &launches);
+    else
+        err = gta::launch_decode_fp8(d, shape->dtype, q, k_codes, c_codes, k_scales, c_scales, seq_lens, S_cap,
+                                     x_t, w_p, w_g, out, workspace, status_word,
+                                     static_cast<cudaStream_t>(cuda_stream), &launches);
     if (err != cudaSuccess) return GTA_ERR_CUDA;
     g_last_launches = launches;
     return GTA_OK;

@@ -111,6 +111,13 @@ gta_status_t check_current_device();
 // Decode and append over 8-bit caches (e4m3 codes [B, groups, S_cap, width] + one fp32 scale per row
 // [B, groups, S_cap]); plain-ALU kernels.
 size_t decode_fp8_workspace_bytes(const Dims& d, int S_cap);
+// 8-bit caches on the bandwidth-oriented kernels (bf16 operator tensors, d_h = 128, one latent group, ...)
+bool decode_fp8_fast_supported(const Dims& d, int dtype, int S_cap);
+size_t decode_fp8_fast_workspace_bytes(const Dims& d);
+cudaError_t launch_decode_fp8_fast(const Dims& d, const void* q, const void* k_codes, const void* c_codes,
+                                   const float* k_scale, const float* c_scale, const int32_t* seq_lens, int S_cap,
+                                   const void* x_t, const void* w_p, const void* w_g, void* out, void* workspace,
+                                   int32_t* status_word, cudaStream_t stream, int* launches);
 cudaError_t launch_decode_fp8(const Dims& d, int dtype, const void* q, const void* k_codes, const void* c_codes,
                               const float* k_scale, const float* c_scale, const int32_t* seq_lens, int S_cap,
                               const void* x_t, const void* w_p, const void* w_g, void* out, void* workspace,

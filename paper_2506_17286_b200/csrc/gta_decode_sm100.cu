@@ -676,6 +676,359 @@ static cudaError_t launch_stream_and_merge(const Dims& d, const FastPlan& p, con
     return cudaSuccess;
 }
 
+// ---------------------------------------------------------------------------------------------
+// The stream kernel for 8-bit caches: K and C rows as e4m3 codes with one fp32 scale per cached row.
+// Same schedule, ring, barriers and partial results as decode_stream_kernel; what differs is the arithmetic:
+//   * the warp-level MMAs are m16n8k32 on e4m3 operands, so the codes go from shared memory into the tensor
+//     pipe as they are.  The other operand has to be e4m3 too, and one e4m3 number (4 significant bits) cannot
+//     hold a bf16 query element or a probability (8 significant bits): each is written as the SUM OF TWO e4m3
+//     numbers -- x scaled by a power of two, p1 = x rounded to e4m3, p2 = x - p1 (exact: what is left has at
+//     most 4 significant bits) -- and the two pieces take rows g and g + 8 of the 16-row operand, so one MMA
+//     multiplies both; the two halves of the accumulator are added afterwards.  The sum is exact for every
+//     element above 2^-10 of its row's largest; below that the error is 2^-18 of the largest.
+//   * a key row's scale multiplies its score after the MMA.  A latent row's scale s_j would have to multiply
+//     its probability before the MMA; instead log2(s_j) is added to the score that the WEIGHTS are taken from,
+//     w_j = 2^(score_j + log2 s_j - m), with m the running maximum of those shifted scores, so that the
+//     weights again fill [0, 1] and sum_j w_j code_j = sum_j 2^(score_j - m) c_j; the row sum l is taken from
+//     the unshifted scores against the same m.  (m, l, sums) is a valid partial for the merge kernel: any
+//     reference m works as long as nothing overflows, and 2^(score - m) <= 1 / min s_j.
+//   * the latent operand B[token][column] is read with transposing 16-bit ldmatrix loads, which deliver two
+//     tokens x two columns per register; a byte permute of two such registers gives four tokens of one
+//     column.  Which tokens share a register is a permutation of the 32 tokens of a k-step that the weight
+//     fragments follow, and the even / odd column split is undone when the sums are written.
+// d_h = 128 (a key row is one 128-byte swizzle row), one latent group, d_l = 128 CH; T = 32 or 64 tokens.
+template <int CH>
+__global__ void __launch_bounds__(kStreamThreads, 1)
+decode_stream_fp8_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_c, Dims d,
+                         int T, int S_cap, const __nv_bfloat16* __restrict__ q, const float* __restrict__ k_scale,
+                         const float* __restrict__ c_scale, const int32_t* __restrict__ seq_lens,
+                         float* __restrict__ part_o, float* __restrict__ part_ml, int32_t* status_word) {
+    const StepLens L{seq_lens, S_cap, 0};
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    constexpr int KTM = kStreamMaxT / 32;                      // most 32-token MMA k-steps per sub-tile
+    const uint32_t tile_bytes = (uint32_t)T * 128;
+    const uint32_t c_off = (uint32_t)d.n_k * tile_bytes;       // the CH latent tiles follow the n_k key tiles
+    const uint32_t scale_off = c_off + CH * tile_bytes;        // then [n_k][T] key scales and [T] latent scales
+    const uint32_t stage_stride = scale_off + (((uint32_t)(d.n_k + 1) * T * 4 + 1023) & ~1023u);
+    uint8_t* ring = smem;
+    float* s_buf = reinterpret_cast<float*>(smem + kStreamStages * stage_stride);        // [2][n_q][T]
+    int32_t* prefix = reinterpret_cast<int32_t*>(s_buf + 2 * 8 * kStreamMaxT);           // [B + 1]
+    int32_t* scan_tmp = prefix + kStreamMaxBatch + 2;                                    // [kStreamThreads]
+    uint64_t* full_bar = reinterpret_cast<uint64_t*>(scan_tmp + kStreamThreads);
+    uint64_t* empty_bar = full_bar + kStreamStages;
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(empty_bar + kStreamStages);
+    volatile int* drain_flag = abort_flag + 1;
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int G = gridDim.x, cta = blockIdx.x;
+    const int NQ = d.n_q;
+    if (tid == kStreamConsumers) {
+        ptx::prefetch_tensormap(&tm_k);
+        ptx::prefetch_tensormap(&tm_c);
+    }
+    // launched with programmatic stream serialisation: nothing of global memory is read before the kernel ahead
+    // (a quantising append) is complete, and only then may the kernels behind this one be scheduled
+    ptx::grid_dependency_wait();
+    ptx::grid_launch_dependents();
+
+    {   // exclusive prefix sum of the sub-tile counts (as in decode_stream_kernel)
+        const int per = (d.B + kStreamThreads - 1) / kStreamThreads;
+        const int lo = min(tid * per, d.B), hi = min(lo + per, d.B);
+        int sum = 0;
+        for (int b = lo; b < hi; ++b) sum += (L.len(b) + T - 1) / T;
+        int incl = sum;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int v = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += v;
+        }
+        if (lane == 31) scan_tmp[warp] = incl;
+        if (tid == 0) {
+            for (int s = 0; s < kStreamStages; ++s) { ptx::mbar_init(&full_bar[s], 1); ptx::mbar_init(&empty_bar[s], 8); }
+            *abort_flag = 0;
+            *drain_flag = 0;
+            ptx::fence_mbar_init();
+        }
+        __syncthreads();
+        int base = incl - sum;
+        for (int w = 0; w < warp; ++w) base += scan_tmp[w];
+        for (int b = lo; b < hi; ++b) {
+            prefix[b] = base;
+            base += (L.len(b) + T - 1) / T;
+        }
+        if (tid == kStreamThreads - 1) prefix[d.B] = base;
+        __syncthreads();
+    }
+    const long long n_st = prefix[d.B];
+    const long long st_begin = ((long long)cta * n_st) / G, st_end = ((long long)(cta + 1) * n_st) / G;
+    if (st_begin >= st_end) return;      // uniform: nothing armed
+    int b0;
+    {
+        int lo = 0, hi = d.B - 1;
+        while (lo < hi) {
+            const int mid = (lo + hi + 1) >> 1;
+            if (prefix[mid] <= st_begin) lo = mid; else hi = mid - 1;
+        }
+        b0 = lo;
+    }
+
+    if (warp == kStreamConsumers / 32) {
+        // ------------------------------------------------------------------ producer: one load per lane
+        const uint64_t policy = ptx::l2_evict_first_policy();
+        const int n_tiles = d.n_k + CH, n_ops = n_tiles + d.n_k + 1;      // tensor tiles, then the scale rows
+        int b = b0;
+        long long k = st_begin - prefix[b0];
+        int it = 0;
+        bool ok = true;
+        for (long long st = st_begin; st < st_end; ++st, ++it, ++k) {
+            while (k >= prefix[b + 1] - prefix[b]) { ++b; k = 0; }
+            const int s = it % kStreamStages;
+            const uint32_t ph = (it / kStreamStages) & 1;
+            const int tok0 = (int)k * T;
+            const uint32_t n_sc = (uint32_t)min(T, S_cap - tok0) * 4;     // bytes of a scale row (S_cap is a multiple of 4)
+            if (lane == 0) {
+                ok = ptx::mbar_wait(&empty_bar[s], ph ^ 1, abort_flag);
+                if (ok) ptx::mbar_arrive_expect_tx(&full_bar[s], scale_off + (uint32_t)(d.n_k + 1) * n_sc);
+            }
+            ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
+            if (!ok) break;
+            uint8_t* stage = ring + s * stage_stride;
+            for (int op = lane; op < n_ops; op += 32) {
+                if (op < d.n_k)
+                    ptx::tma_load_3d_hint(stage + op * tile_bytes, &tm_k, &full_bar[s], 0, tok0, b * d.n_k + op, policy);
+                else if (op < n_tiles)
+                    ptx::tma_load_3d_hint(stage + op * tile_bytes, &tm_c, &full_bar[s], (op - d.n_k) * 128, tok0, b, policy);
+                else if (op < n_tiles + d.n_k)
+                    ptx::bulk_load_1d(stage + scale_off + (op - n_tiles) * T * 4,
+                                      k_scale + ((size_t)b * d.n_k + (op - n_tiles)) * S_cap + tok0, n_sc, &full_bar[s]);
+                else
+                    ptx::bulk_load_1d(stage + scale_off + d.n_k * T * 4, c_scale + (size_t)b * S_cap + tok0, n_sc,
+                                      &full_bar[s]);
+            }
+        }
+        if (lane == 0 && *abort_flag) {
+            for (int back = 1; back <= kStreamStages && it - back >= 0; ++back) {
+                const int iq = it - back;
+                ptx::mbar_wait_drain(&full_bar[iq % kStreamStages], (iq / kStreamStages) & 1, drain_flag);
+            }
+        }
+    } else {
+        // ------------------------------------------------------------------ consumers
+        const int quad = lane >> 2, sub = lane & 3;       // MMA fragment coordinates
+        const int mat = lane >> 3, mrow = lane & 7;       // ldmatrix: which 8x8 matrix, which row of it
+        const int qpk = NQ / d.n_k;                       // maps per key group
+        const int kg_w = warp % d.n_k;                    // this warp scores key group kg_w
+        const int KT = T >> 5;                            // 32-token MMA k-steps per sub-tile
+        const int n_units = (T >> 3) * d.n_k;             // (8-token n-tile, key group) scoring units
+        const uint32_t ring_addr = ptx::smem_addr(ring);
+        const bool map_lane = quad < NQ;
+        float m_run = -INFINITY, l_run = 0.f;
+        float acc[2 * CH][4];
+#pragma unroll
+        for (int n = 0; n < 2 * CH; ++n) acc[n][0] = acc[n][1] = acc[n][2] = acc[n][3] = 0.f;
+        uint32_t qa[4][4];                                // A fragments of the query pieces, d_h = 4 k-steps of 32
+        float q_mul = 0.f;                                // power-of-two scale of the query row x softmax scale x log2(e)
+
+        // x0 .. x3 -> the four codes of each piece, packed lowest element first
+        auto split4 = [](float x0, float x1, float x2, float x3, uint32_t& hi, uint32_t& lo) {
+            const uint32_t h01 = ptx::cvt_e4m3x2(x0, x1), h23 = ptx::cvt_e4m3x2(x2, x3);
+            const float2 b01 = ptx::e4m3x2_to_f32(h01), b23 = ptx::e4m3x2_to_f32(h23);
+            hi = h01 | (h23 << 16);
+            lo = ptx::cvt_e4m3x2(x0 - b01.x, x1 - b01.y) | (ptx::cvt_e4m3x2(x2 - b23.x, x3 - b23.y) << 16);
+        };
+        auto load_q = [&](int b) {
+            const bool live = quad < qpk;
+            const __nv_bfloat16* qrow = q + ((size_t)b * NQ + kg_w * qpk + (live ? quad : 0)) * 128;
+            float v[4][8];
+            float amax = 0.f;
+#pragma unroll
+            for (int ks = 0; ks < 4; ++ks) {
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {             // elements 32 ks + 16 h + 4 sub .. + 3
+                    const uint2 raw = __ldg(reinterpret_cast<const uint2*>(qrow + 32 * ks + 16 * h + 4 * sub));
+                    const float2 lo = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&raw.x));
+                    const float2 hi = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&raw.y));
+                    v[ks][4 * h] = live ? lo.x : 0.f; v[ks][4 * h + 1] = live ? lo.y : 0.f;
+                    v[ks][4 * h + 2] = live ? hi.x : 0.f; v[ks][4 * h + 3] = live ? hi.y : 0.f;
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) amax = fmaxf(amax, fabsf(v[ks][4 * h + e]));
+                }
+            }
+            amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 1));
+            amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, 2));
+            // power of two that brings the row's largest element into [128, 256) (e4m3 reaches 448)
+            uint32_t e = (__float_as_uint(amax) >> 23) & 0xffu;
+            e = e < 8u ? 8u : e;
+            const float scale = __uint_as_float((e - 7u) << 23), inv = __uint_as_float((261u - e) << 23);
+            q_mul = scale * d.scale * 1.4426950408889634f;
+#pragma unroll
+            for (int ks = 0; ks < 4; ++ks) {
+                split4(v[ks][0] * inv, v[ks][1] * inv, v[ks][2] * inv, v[ks][3] * inv, qa[ks][0], qa[ks][1]);
+                split4(v[ks][4] * inv, v[ks][5] * inv, v[ks][6] * inv, v[ks][7] * inv, qa[ks][2], qa[ks][3]);
+            }
+        };
+        auto flush = [&](int b) {
+            const int slot = cta + b;
+            if (map_lane) {
+                float* o = part_o + ((size_t)slot * NQ + quad) * d.d_l + warp * (CH * 16) + 4 * sub;
+#pragma unroll
+                for (int c = 0; c < CH; ++c) {
+                    // even / odd columns of the chunk, pieces added, the weights' factor 2^8 taken out
+                    const float4 v = make_float4((acc[2 * c][0] + acc[2 * c][2]) * 0.00390625f,
+                                                 (acc[2 * c + 1][0] + acc[2 * c + 1][2]) * 0.00390625f,
+                                                 (acc[2 * c][1] + acc[2 * c][3]) * 0.00390625f,
+                                                 (acc[2 * c + 1][1] + acc[2 * c + 1][3]) * 0.00390625f);
+                    *reinterpret_cast<float4*>(o + 16 * c) = v;
+                }
+                if (warp == 0 && sub == 0) {
+                    part_ml[((size_t)slot * NQ + quad) * 2] = m_run;
+                    part_ml[((size_t)slot * NQ + quad) * 2 + 1] = l_run;
+                }
+            }
+#pragma unroll
+            for (int n = 0; n < 2 * CH; ++n) acc[n][0] = acc[n][1] = acc[n][2] = acc[n][3] = 0.f;
+            m_run = -INFINITY;
+            l_run = 0.f;
+        };
+
+        int b = b0;
+        long long k = st_begin - prefix[b0];
+        load_q(b);
+        int it = 0;
+        bool ok = true;
+        for (long long st = st_begin; st < st_end; ++st, ++it, ++k) {
+            if (k >= prefix[b + 1] - prefix[b]) {
+                flush(b);
+                do { ++b; } while (prefix[b + 1] == prefix[b]);
+                k = 0;
+                load_q(b);
+            }
+            const int s = it % kStreamStages;
+            const uint32_t ph = (it / kStreamStages) & 1;
+            ok = __all_sync(0xffffffffu, ptx::mbar_wait(&full_bar[s], ph, abort_flag));
+            if (!ok) break;
+            const int n_valid = min(T, L.len(b) - (int)k * T);
+            const uint32_t stage = ring_addr + s * stage_stride;
+            const float* ksc = reinterpret_cast<const float*>(ring + s * stage_stride + scale_off);
+            const float* csc = ksc + d.n_k * T;
+            float* sb = s_buf + (it & 1) * (NQ * T);
+
+            // ---- scores of the maps of key group kg_w, 8 tokens per unit
+            for (int u = warp; u < n_units; u += 8) {
+                const int nt = u / d.n_k;
+                const int token = nt * 8 + mrow;
+                const uint32_t krow = stage + (uint32_t)kg_w * tile_bytes + token * 128;
+                float sc[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+                for (int kp = 0; kp < 2; ++kp) {
+                    const int chunk = 4 * kp + mat;     // 16-byte chunk (16 codes) of the key row
+                    uint32_t k0, k1, k2, k3;
+                    ptx::ldsm_x4(krow + (((chunk & 7) ^ (token & 7)) << 4), k0, k1, k2, k3);
+                    ptx::mma_e4m3_16832(sc, qa[2 * kp][0], qa[2 * kp][1], qa[2 * kp][2], qa[2 * kp][3], k0, k1);
+                    ptx::mma_e4m3_16832(sc, qa[2 * kp + 1][0], qa[2 * kp + 1][1], qa[2 * kp + 1][2], qa[2 * kp + 1][3], k2, k3);
+                }
+                if (quad < qpk) {
+                    const int t0 = nt * 8 + 2 * sub;
+                    const float2 ks2 = *reinterpret_cast<const float2*>(ksc + kg_w * T + t0);
+                    float2 v;
+                    v.x = t0 < n_valid ? (sc[0] + sc[2]) * q_mul * ks2.x : -INFINITY;
+                    v.y = t0 + 1 < n_valid ? (sc[1] + sc[3]) * q_mul * ks2.y : -INFINITY;
+                    *reinterpret_cast<float2*>(sb + (kg_w * qpk + quad) * T + t0) = v;
+                }
+            }
+            // ---- rows past the live length hold whatever the cache holds there (NaN codes included): their
+            //      weights are zero, so the latent rows are cleared
+            if (n_valid < T) {
+                const int vec_per_row = CH * 8;
+                const int n_vec = (T - n_valid) * vec_per_row;
+                for (int idx = tid; idx < n_vec; idx += kStreamConsumers) {
+                    const int row = n_valid + idx / vec_per_row, v = idx % vec_per_row;
+                    uint8_t* p = ring + s * stage_stride + c_off + (v >> 3) * tile_bytes + row * 128 + (v & 7) * 16;
+                    *reinterpret_cast<uint4*>(p) = make_uint4(0u, 0u, 0u, 0u);
+                }
+                ptx::fence_proxy_async_smem();   // the next TMA write of this stage follows generic writes
+            }
+            consumer_sync();
+
+            // ---- softmax state of map `quad` and the weight fragments: lane (quad, sub) holds, of every 32-token
+            //      k-step, tokens 8 j + 2 sub + {0, 1} for j = 0 .. 3 (j = 0, 1 in the first register, 2, 3 in the second)
+            uint32_t pa[KTM][4];
+            float alpha = 1.f;
+            {
+                float sv[KTM][8], sw[KTM][8];
+                float m_t = -INFINITY;
+#pragma unroll
+                for (int kt = 0; kt < KTM; ++kt) {
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        float2 x = make_float2(-INFINITY, -INFINITY), y = x;
+                        if (kt < KT && map_lane) {
+                            const int t0 = 32 * kt + 8 * j + 2 * sub;
+                            x = *reinterpret_cast<const float2*>(sb + quad * T + t0);
+                            const float2 cs = *reinterpret_cast<const float2*>(csc + t0);
+                            y.x = x.x == -INFINITY ? -INFINITY : x.x + __log2f(cs.x);
+                            y.y = x.y == -INFINITY ? -INFINITY : x.y + __log2f(cs.y);
+                        }
+                        sv[kt][2 * j] = x.x; sv[kt][2 * j + 1] = x.y;
+                        sw[kt][2 * j] = y.x; sw[kt][2 * j + 1] = y.y;
+                        m_t = fmaxf(m_t, fmaxf(y.x, y.y));
+                    }
+                }
+                m_t = fmaxf(m_t, __shfl_xor_sync(0xffffffffu, m_t, 1));
+                m_t = fmaxf(m_t, __shfl_xor_sync(0xffffffffu, m_t, 2));
+                const float m_new = fmaxf(m_run, m_t);
+                const bool any = map_lane && m_new > -INFINITY;     // false: only rows with a zero scale so far
+                const float m_sub = any ? m_new : 0.f;
+                alpha = any ? ex2f(m_run - m_new) : 1.f;
+                float sum = 0.f;
+#pragma unroll
+                for (int kt = 0; kt < KTM; ++kt) {
+                    float w[8];
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) {
+                        w[e] = ex2f(sw[kt][e] - m_sub) * 256.f;
+                        sum += any ? ex2f(sv[kt][e] - m_sub) : 0.f;
+                    }
+                    split4(w[0], w[1], w[2], w[3], pa[kt][0], pa[kt][1]);
+                    split4(w[4], w[5], w[6], w[7], pa[kt][2], pa[kt][3]);
+                }
+                sum += __shfl_xor_sync(0xffffffffu, sum, 1);
+                sum += __shfl_xor_sync(0xffffffffu, sum, 2);
+                l_run = l_run * alpha + sum;
+                m_run = any ? m_new : m_run;
+            }
+#pragma unroll
+            for (int n = 0; n < 2 * CH; ++n) { acc[n][0] *= alpha; acc[n][1] *= alpha; acc[n][2] *= alpha; acc[n][3] *= alpha; }
+
+            // ---- latent sums of this warp's 16 CH columns, all maps and both pieces at once
+#pragma unroll
+            for (int kt = 0; kt < KTM; ++kt) {
+                if (kt < KT) {
+                    const int token = 32 * kt + 8 * mat + mrow;
+#pragma unroll
+                    for (int c = 0; c < CH; ++c) {
+                        const int chunk = warp * CH + c;      // 16-byte chunk (16 columns) of the latent row
+                        uint32_t r0, r1, r2, r3;
+                        ptx::ldsm_x4_trans(stage + c_off + (chunk >> 3) * tile_bytes + token * 128 +
+                                               (((chunk & 7) ^ (token & 7)) << 4), r0, r1, r2, r3);
+                        // r_i: tokens 8 i + 2 sub + {0, 1} x columns 2 quad + {0, 1}
+                        const uint32_t be0 = ptx::byte_perm(r0, r1, 0x6420u), be1 = ptx::byte_perm(r2, r3, 0x6420u);
+                        const uint32_t bo0 = ptx::byte_perm(r0, r1, 0x7531u), bo1 = ptx::byte_perm(r2, r3, 0x7531u);
+                        ptx::mma_e4m3_16832(acc[2 * c], pa[kt][0], pa[kt][1], pa[kt][2], pa[kt][3], be0, be1);
+                        ptx::mma_e4m3_16832(acc[2 * c + 1], pa[kt][0], pa[kt][1], pa[kt][2], pa[kt][3], bo0, bo1);
+                    }
+                }
+            }
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(&empty_bar[s]);
+        }
+        if (ok) flush(b);
+    }
+    __syncthreads();
+    if (tid == 0 && *abort_flag) raise_status(status_word, GTA_ERR_TIMEOUT);
+}
+
 // k_new / c_new != nullptr: the fused append + decode step -- seq_lens does not count the new token yet, the stream
 // kernel puts its rows into the caches and attends over them, the decoder kernel advances the lengths at the end.
 cudaError_t launch_decode_fast(const Dims& d, const void* q, const void* k_cache, const void* c_cache,
@@ -701,6 +1054,108 @@ cudaError_t launch_decode_fast(const Dims& d, const void* q, const void* k_cache
             return cudaErrorUnknown;
         *launches += 1;
     }
+    return cudaSuccess;
+}
+
+// ---------------------------------------------------------------------------------------------
+// One decode step over 8-bit caches on the stream kernel above, the merge kernel and the tcgen05 decoder kernel.
+bool decode_fp8_fast_supported(const Dims& d, int dtype, int S_cap) {
+    if (dtype != GTA_BF16 || d.d_h != 128 || d.n_c != 1) return false;
+    if (d.d_l != 128 && d.d_l != 256 && d.d_l != 512 && d.d_l != 1024) return false;
+    if (d.n_q < 1 || d.n_q > 8) return false;
+    if (d.n_k != 1 && d.n_k != 2 && d.n_k != 4 && d.n_k != 8) return false;
+    if (d.H % 64 != 0 || d.B > kStreamMaxBatch) return false;
+    if (S_cap % 4 != 0) return false;                           // scale rows are copied in 16-byte pieces
+    if (((d.n_h / d.n_q) * d.d_h) % (d.B > 128 ? 128 : 64) != 0) return false;
+    return (d.n_k * 128 + d.d_l) * 32 <= kStreamStageBytes;     // a 32-token sub-tile fits a ring stage
+}
+
+static FastPlan make_fp8_plan(const Dims& d) {
+    FastPlan p;
+    const int tok_bytes = d.n_k * 128 + d.d_l;
+    p.occ = 1;
+    p.T = tok_bytes * 64 <= kStreamStageBytes ? 64 : 32;
+    const int ctas = sm_count();
+    p.G = ctas < kFinMaxSlots - kStreamMaxBatch ? ctas : kFinMaxSlots - kStreamMaxBatch;
+    p.slots = p.G + d.B;
+    p.off_ml = align256f((size_t)p.slots * d.n_q * d.d_l * sizeof(float));
+    p.off_l = p.off_ml + align256f((size_t)p.slots * d.n_q * 2 * sizeof(float));
+    p.total = p.off_l + align256f((size_t)d.n_q * d.B * d.d_l * sizeof(__nv_bfloat16));
+    return p;
+}
+
+size_t decode_fp8_fast_workspace_bytes(const Dims& d) { return make_fp8_plan(d).total; }
+
+cudaError_t launch_decode_fp8_fast(const Dims& d, const void* q, const void* k_codes, const void* c_codes,
+                                   const float* k_scale, const float* c_scale, const int32_t* seq_lens, int S_cap,
+                                   const void* x_t, const void* w_p, const void* w_g, void* out, void* workspace,
+                                   int32_t* status_word, cudaStream_t stream, int* launches) {
+    const FastPlan p = make_fp8_plan(d);
+    float* part_o = reinterpret_cast<float*>(workspace);
+    float* part_ml = reinterpret_cast<float*>(static_cast<char*>(workspace) + p.off_ml);
+    __nv_bfloat16* l_g = reinterpret_cast<__nv_bfloat16*>(static_cast<char*>(workspace) + p.off_l);
+    cudaError_t err;
+    {
+        CUtensorMap tm_k, tm_c;
+        const uint32_t box[3] = {128, (uint32_t)p.T, 1};
+        const uint64_t dk[3] = {128, (uint64_t)S_cap, (uint64_t)d.B * d.n_k};
+        const uint64_t dc[3] = {(uint64_t)d.d_l, (uint64_t)S_cap, (uint64_t)d.B};
+        if (!make_u8_map(&tm_k, k_codes, 3, dk, box) || !make_u8_map(&tm_c, c_codes, 3, dc, box))
+            return cudaErrorInvalidValue;
+        const int CH = d.d_l / 128;
+        const size_t stage = (size_t)(d.n_k + CH) * p.T * 128 + ((((size_t)d.n_k + 1) * p.T * 4 + 1023) & ~(size_t)1023);
+        const size_t smem = kStreamStages * stage + 2 * 8 * kStreamMaxT * sizeof(float) +
+                            (size_t)(kStreamMaxBatch + 2 + kStreamThreads) * sizeof(int32_t) +
+                            2 * kStreamStages * sizeof(uint64_t) + 16 + 1024;
+#define GTA_LAUNCH_FP8(CHV)                                                                                \
+        do {                                                                                               \
+            auto kern = decode_stream_fp8_kernel<CHV>;                                                     \
+            err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);      \
+            if (err != cudaSuccess) return err;                                                            \
+            cudaLaunchConfig_t cfg = {};                                                                   \
+            cfg.gridDim = dim3(p.G);                                                                       \
+            cfg.blockDim = dim3(kStreamThreads);                                                           \
+            cfg.dynamicSmemBytes = smem;                                                                   \
+            cfg.stream = stream;                                                                           \
+            cudaLaunchAttribute attr[1];                                                                   \
+            attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;                               \
+            attr[0].val.programmaticStreamSerializationAllowed = 1;                                        \
+            cfg.attrs = attr;                                                                              \
+            cfg.numAttrs = 1;                                                                              \
+            err = cudaLaunchKernelEx(&cfg, kern, tm_k, tm_c, d, p.T, S_cap, (const __nv_bfloat16*)q, k_scale, \
+                                     c_scale, seq_lens, part_o, part_ml, status_word);                     \
+            if (err != cudaSuccess) return err;                                                            \
+        } while (0)
+        switch (CH) {
+            case 1: GTA_LAUNCH_FP8(1); break;
+            case 2: GTA_LAUNCH_FP8(2); break;
+            case 4: GTA_LAUNCH_FP8(4); break;
+            default: GTA_LAUNCH_FP8(8); break;
+        }
+#undef GTA_LAUNCH_FP8
+        if ((err = cudaGetLastError()) != cudaSuccess) return err;
+        *launches += 1;
+    }
+    {
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(d.n_q, d.B);
+        cfg.blockDim = dim3(256);
+        cfg.stream = stream;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        err = cudaLaunchKernelEx(&cfg, decode_merge_kernel, d, p.G, p.T, S_cap, seq_lens, (const float*)part_o,
+                                 (const float*)part_ml, l_g, (long long)d.B * d.d_l, (long long)d.d_l, 0);
+        if (err != cudaSuccess) return err;
+        *launches += 1;
+    }
+    Dims dd = d;      // the batch takes the role of the token axis
+    dd.B = 1;
+    dd.N = d.B;
+    if (launch_sm100_decoder(dd, l_g, x_t, w_p, w_g, out, status_word, stream) != GTA_OK) return cudaErrorUnknown;
+    *launches += 1;
     return cudaSuccess;
 }
 

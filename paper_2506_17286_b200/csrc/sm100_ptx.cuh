@@ -4,6 +4,8 @@
 // signals the barriers of both CTAs of a pair).
 #pragma once
 
+#include <cuda_fp16.h>
+
 #include <cuda.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -242,6 +244,41 @@ __device__ __forceinline__ void mma_bf16_16816(float (&d)[4], uint32_t a0, uint3
         "{%0, %1, %2, %3};"
         : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
         : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+// D (16 x 8, fp32) += A (16 x 32, row) B (32 x 8, col) on 8-bit floats of the e4m3 format.  Lane (g = lane / 4,
+// s = lane % 4): a0 = A[g][4 s .. 4 s + 3], a1 = A[g + 8][same], a2 / a3 = the same rows, columns + 16 (lowest byte =
+// lowest column); b0 = B[4 s .. 4 s + 3][g], b1 = rows + 16; d0, d1 = D[g][2 s, 2 s + 1], d2, d3 = D[g + 8][same].
+__device__ __forceinline__ void mma_e4m3_16832(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                               uint32_t b0, uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k32.row.col.f32.e4m3.e4m3.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
+        "{%0, %1, %2, %3};"
+        : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+// Two fp32 values -> two e4m3 codes (round to nearest even, saturating at 448): lo in bits 0-7, hi in bits 8-15.
+__device__ __forceinline__ uint32_t cvt_e4m3x2(float lo, float hi) {
+    uint16_t r;
+    asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+// Two e4m3 codes (bits 0-7, 8-15) -> their exact values (every e4m3 value is an f16 value).
+__device__ __forceinline__ float2 e4m3x2_to_f32(uint32_t pair) {
+    uint32_t h2;
+    asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(h2) : "h"((uint16_t)pair));
+    return __half22float2(*reinterpret_cast<__half2*>(&h2));
+}
+__device__ __forceinline__ uint32_t byte_perm(uint32_t a, uint32_t b, uint32_t sel) {
+    uint32_t d;
+    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(sel));
+    return d;
+}
+// Untiled bulk copy global -> shared of `bytes` (a multiple of 16; both addresses 16-byte aligned), counted on `bar`.
+__device__ __forceinline__ void bulk_load_1d(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(smem_addr(dst)), "l"(reinterpret_cast<uint64_t>(src)), "r"(bytes), "r"(smem_addr(bar))
+                 : "memory");
 }
 
 // ------------------------------------------------------------------ tensor memory

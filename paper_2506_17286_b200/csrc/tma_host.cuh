@@ -48,4 +48,23 @@ inline bool make_bf16_map(CUtensorMap* m, const void* base, int rank, const uint
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Dense tensor of bytes (8-bit codes), same conventions: the innermost box extent is 128 bytes (one swizzle row).
+inline bool make_u8_map(CUtensorMap* m, const void* base, int rank, const uint64_t* dims, const uint32_t* box) {
+    EncodeTiledFn fn = tensor_map_encoder();
+    if (!fn) return false;
+    cuuint64_t gdim[5], gstride[5];
+    cuuint32_t bx[5], estr[5];
+    uint64_t stride = 1;
+    for (int i = 0; i < rank; ++i) {
+        gdim[i] = dims[i];
+        bx[i] = box[i];
+        estr[i] = 1;
+        stride *= dims[i];
+        if (i < rank - 1) gstride[i] = stride;
+    }
+    return fn(m, CU_TENSOR_MAP_DATA_TYPE_UINT8, (cuuint32_t)rank, const_cast<void*>(base), gdim, gstride, bx, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 }  // namespace gta

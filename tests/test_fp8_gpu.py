@@ -55,9 +55,9 @@ def test_quantising_append_is_bit_exact(B, oracle, dt, n_new):
             assert np.array_equal(g_, ref), what
 
 
-def _decode_case(B, oracle, w, lens, sample=None):
+def _decode_case(B, oracle, w, lens, sample=None, cap=None, path=None):
     nb = w.batch
-    cap = max(lens) + 7
+    cap = cap or max(lens) + 7
     t = I.decode_inputs(w, device="cuda", s_cap=cap, seq_lens=lens)
     kq, ks = oracle.quantize_rows_e4m3(t["k_cache"].cpu())
     cq, cs = oracle.quantize_rows_e4m3(t["c_cache"].cpu())
@@ -66,6 +66,8 @@ def _decode_case(B, oracle, w, lens, sample=None):
     dev = [torch.from_numpy(a).cuda() for a in (kq, cq, ks, cs)]
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
     shape = B.decode_shape(t["q"], t["k_cache"], t["c_cache"], t["x_t"], t["w_p"])
+    if path is not None:
+        assert B.decode_fp8_path(shape, cap) == path
     ws = Guarded((B.decode_fp8_workspace_bytes(shape, cap),), torch.uint8)
     og = Guarded((nb, w.n_heads, w.d_h), w.torch_dtype())
     out = B.gta_decode_fp8(t["q"], *dev, t["seq_lens"], t["x_t"], t["w_p"], t["w_g"], out=og.t, workspace=ws.t,
@@ -97,9 +99,37 @@ def test_fp8_decode_small_shapes(B, oracle, case):
     _decode_case(B, oracle, w, lens)
 
 
+FP8_STREAM = [
+    # name, B, H, n_h, n_q, n_k, d_l, lens, cap  (bf16, d_h = 128, one latent group: the streaming kernels)
+    ("ragged_64_token_subtiles", 5, 256, 8, 4, 4, 512, [1, 63, 64, 65, 700], 708),
+    ("dl1024_eight_maps_32_token_subtiles", 3, 512, 16, 8, 8, 1024, [257, 1, 1000], 1004),
+    ("dl128_five_maps_one_key_group", 2, 1280, 10, 5, 1, 128, [333, 1000], 1024),
+    ("dl256_empty_sequences_shared_keys", 6, 256, 8, 4, 2, 256, [0, 512, 1, 0, 300, 33], 512),
+    ("one_map_full_cache", 2, 128, 2, 1, 1, 256, [256, 255], 256),
+    ("many_sequences", 150, 256, 8, 4, 4, 512, [((7 * i) % 130) for i in range(150)], 132),
+]
+
+
+@pytest.mark.parametrize("case", FP8_STREAM, ids=[c[0] for c in FP8_STREAM])
+def test_fp8_decode_streaming_kernels(B, oracle, case):
+    name, nb, H, n_h, n_q, n_k, d_l, lens, cap = case
+    w = I.Workload(name, "decode", "bf16", nb, 0, H, n_h, n_q, n_k, 1, 128, d_l, seed=63)
+    rel, mx = _decode_case(B, oracle, w, lens, cap=cap, path=2)
+    print(f"\n{name}: rel-L2 {rel:.3e} max-abs {mx:.3e}")
+
+
 def test_fp8_decode_config3_shape_sampled_sequences(B, oracle):
     w = I.CONFIGS["c3_decode_bf16"]
-    _decode_case(B, oracle, w, [w.seq] * w.batch, sample=[0, 9, 31])
+    rel, mx = _decode_case(B, oracle, w, [w.seq] * w.batch, sample=[0, 9, 31], cap=w.seq + 64, path=2)
+    print(f"\nc3 shape over 8-bit caches: rel-L2 {rel:.3e} max-abs {mx:.3e}")
+
+
+def test_fp8_decode_config5_shape_ragged_sampled_sequences(B, oracle):
+    """The ragged workload's shape (8 maps over 8 key groups, d_l = 1024) at a tenth of its lengths."""
+    w = I.scaled(I.CONFIGS["c5_ragged_decode_bf16"], batch=24)
+    g = torch.Generator("cpu").manual_seed(5)
+    lens = torch.randint(100, 3300, (24,), generator=g).tolist()
+    _decode_case(B, oracle, w, lens, sample=[0, 11, 23], cap=3304, path=2)
 
 
 def test_append_then_decode_over_fp8_caches(B, oracle):
