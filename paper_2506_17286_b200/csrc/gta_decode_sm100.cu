@@ -696,6 +696,12 @@ static cudaError_t launch_stream_and_merge(const Dims& d, const FastPlan& p, con
 //     tokens x two columns per register; a byte permute of two such registers gives four tokens of one
 //     column.  Which tokens share a register is a permutation of the 32 tokens of a k-step that the weight
 //     fragments follow, and the even / odd column split is undone when the sums are written.
+//   * the exponentials and the e4m3 conversions of the weights are done once per CTA (each warp takes T / 8
+//     tokens) and handed to the other warps through shared memory in fragment order, not once per warp.
+// What bounds it: on this architecture the warp-level e4m3 MMA is carried out as f16 MMAs behind conversions of its
+// operands on the conversion unit (16 lanes per clock and SM: measured 3.4 conversion instructions per MMA, that
+// unit 58 % busy), so the kernel runs at about the token rate of the bf16 kernel -- half its byte rate.  Converting
+// the codes to f16 here and issuing f16 MMAs (for the scores only, or for both contractions) was measured slower.
 // d_h = 128 (a key row is one 128-byte swizzle row), one latent group, d_l = 128 CH; T = 32 or 64 tokens.
 template <int CH>
 __global__ void __launch_bounds__(kStreamThreads, 1)
@@ -712,8 +718,10 @@ decode_stream_fp8_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_
     const uint32_t scale_off = c_off + CH * tile_bytes;        // then [n_k][T] key scales and [T] latent scales
     const uint32_t stage_stride = scale_off + (((uint32_t)(d.n_k + 1) * T * 4 + 1023) & ~1023u);
     uint8_t* ring = smem;
-    float* s_buf = reinterpret_cast<float*>(smem + kStreamStages * stage_stride);        // [2][n_q][T]
-    int32_t* prefix = reinterpret_cast<int32_t*>(s_buf + 2 * 8 * kStreamMaxT);           // [B + 1]
+    float* s_buf = reinterpret_cast<float*>(smem + kStreamStages * stage_stride);        // [2][2][n_q][T]: scores, shifted scores
+    uint4* w_buf = reinterpret_cast<uint4*>(s_buf + 4 * 8 * kStreamMaxT);                // [KTM][8 maps][4]: weight fragments
+    float* den_buf = reinterpret_cast<float*>(w_buf + KTM * 32);                         // [8 warps][32 lanes]: row-sum shares
+    int32_t* prefix = reinterpret_cast<int32_t*>(den_buf + 256);                         // [B + 1]
     int32_t* scan_tmp = prefix + kStreamMaxBatch + 2;                                    // [kStreamThreads]
     uint64_t* full_bar = reinterpret_cast<uint64_t*>(scan_tmp + kStreamThreads);
     uint64_t* empty_bar = full_bar + kStreamStages;
@@ -912,7 +920,8 @@ decode_stream_fp8_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_
             const uint32_t stage = ring_addr + s * stage_stride;
             const float* ksc = reinterpret_cast<const float*>(ring + s * stage_stride + scale_off);
             const float* csc = ksc + d.n_k * T;
-            float* sb = s_buf + (it & 1) * (NQ * T);
+            float* sb = s_buf + (it & 1) * (2 * NQ * T);      // scores [n_q][T]
+            float* sbw = sb + NQ * T;                          // scores shifted by log2 of the latent row's scale
 
             // ---- scores of the maps of key group kg_w, 8 tokens per unit
             for (int u = warp; u < n_units; u += 8) {
@@ -931,10 +940,14 @@ decode_stream_fp8_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_
                 if (quad < qpk) {
                     const int t0 = nt * 8 + 2 * sub;
                     const float2 ks2 = *reinterpret_cast<const float2*>(ksc + kg_w * T + t0);
-                    float2 v;
+                    const float2 cs2 = *reinterpret_cast<const float2*>(csc + t0);
+                    float2 v, y;
                     v.x = t0 < n_valid ? (sc[0] + sc[2]) * q_mul * ks2.x : -INFINITY;
                     v.y = t0 + 1 < n_valid ? (sc[1] + sc[3]) * q_mul * ks2.y : -INFINITY;
+                    y.x = t0 < n_valid ? v.x + __log2f(cs2.x) : -INFINITY;
+                    y.y = t0 + 1 < n_valid ? v.y + __log2f(cs2.y) : -INFINITY;
                     *reinterpret_cast<float2*>(sb + (kg_w * qpk + quad) * T + t0) = v;
+                    *reinterpret_cast<float2*>(sbw + (kg_w * qpk + quad) * T + t0) = y;
                 }
             }
             // ---- rows past the live length hold whatever the cache holds there (NaN codes included): their
@@ -951,52 +964,70 @@ decode_stream_fp8_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_
             }
             consumer_sync();
 
-            // ---- softmax state of map `quad` and the weight fragments: lane (quad, sub) holds, of every 32-token
-            //      k-step, tokens 8 j + 2 sub + {0, 1} for j = 0 .. 3 (j = 0, 1 in the first register, 2, 3 in the second)
-            uint32_t pa[KTM][4];
-            float alpha = 1.f;
+            // ---- (A) every warp: the running maximum of map `quad` over the shifted scores of all T tokens
+            float alpha = 1.f, m_sub = 0.f;
+            bool any = false;
             {
-                float sv[KTM][8], sw[KTM][8];
                 float m_t = -INFINITY;
 #pragma unroll
                 for (int kt = 0; kt < KTM; ++kt) {
+                    if (kt < KT && map_lane) {
 #pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        float2 x = make_float2(-INFINITY, -INFINITY), y = x;
-                        if (kt < KT && map_lane) {
-                            const int t0 = 32 * kt + 8 * j + 2 * sub;
-                            x = *reinterpret_cast<const float2*>(sb + quad * T + t0);
-                            const float2 cs = *reinterpret_cast<const float2*>(csc + t0);
-                            y.x = x.x == -INFINITY ? -INFINITY : x.x + __log2f(cs.x);
-                            y.y = x.y == -INFINITY ? -INFINITY : x.y + __log2f(cs.y);
+                        for (int j = 0; j < 4; ++j) {
+                            const float2 y = *reinterpret_cast<const float2*>(sbw + quad * T + 32 * kt + 8 * j + 2 * sub);
+                            m_t = fmaxf(m_t, fmaxf(y.x, y.y));
                         }
-                        sv[kt][2 * j] = x.x; sv[kt][2 * j + 1] = x.y;
-                        sw[kt][2 * j] = y.x; sw[kt][2 * j + 1] = y.y;
-                        m_t = fmaxf(m_t, fmaxf(y.x, y.y));
                     }
                 }
                 m_t = fmaxf(m_t, __shfl_xor_sync(0xffffffffu, m_t, 1));
                 m_t = fmaxf(m_t, __shfl_xor_sync(0xffffffffu, m_t, 2));
                 const float m_new = fmaxf(m_run, m_t);
-                const bool any = map_lane && m_new > -INFINITY;     // false: only rows with a zero scale so far
-                const float m_sub = any ? m_new : 0.f;
+                any = map_lane && m_new > -INFINITY;       // false: nothing but rows with a zero scale so far
+                m_sub = any ? m_new : 0.f;
                 alpha = any ? ex2f(m_run - m_new) : 1.f;
+                m_run = any ? m_new : m_run;
+            }
+            // ---- (B) the weights of T / 8 tokens per warp (the exponentials and the conversions are the costly part
+            //      of a sub-tile: each is done once per CTA, not once per warp) go to shared memory as the 16-bit halves
+            //      of the fragment registers of the lanes that need them: lane (quad, s') holds, of k-step kt, the token
+            //      pairs 32 kt + 8 j + 2 s' + {0, 1}, j = 0 .. 3, in {a0, a1, a2, a3} = {piece 1 of j = 0 | 1, piece 2 of
+            //      j = 0 | 1, piece 1 of j = 2 | 3, piece 2 of j = 2 | 3}
+            {
+                const int ppw = T >> 4;                    // token pairs per warp
+                float den = 0.f;
+                if (sub < ppw) {
+                    const int gp = warp * ppw + sub;       // token pair 2 gp, 2 gp + 1 of the sub-tile
+                    float2 x = make_float2(-INFINITY, -INFINITY), y = x;
+                    if (map_lane) {
+                        x = *reinterpret_cast<const float2*>(sb + quad * T + 2 * gp);
+                        y = *reinterpret_cast<const float2*>(sbw + quad * T + 2 * gp);
+                    }
+                    const float w0 = ex2f(y.x - m_sub) * 256.f, w1 = ex2f(y.y - m_sub) * 256.f;
+                    den = any ? ex2f(x.x - m_sub) + ex2f(x.y - m_sub) : 0.f;
+                    const uint32_t hi = ptx::cvt_e4m3x2(w0, w1);
+                    const float2 back = ptx::e4m3x2_to_f32(hi);
+                    const uint32_t lo = ptx::cvt_e4m3x2(w0 - back.x, w1 - back.y);
+                    const int r = gp & 15, j = r >> 2;
+                    uint16_t* wp = reinterpret_cast<uint16_t*>(w_buf + ((gp >> 4) * 8 + quad) * 4 + (r & 3));
+                    wp[(j >> 1) * 4 + (j & 1)] = (uint16_t)hi;
+                    wp[(j >> 1) * 4 + 2 + (j & 1)] = (uint16_t)lo;
+                }
+                den_buf[warp * 32 + lane] = den;
+            }
+            consumer_sync();
+            uint32_t pa[KTM][4];
+#pragma unroll
+            for (int kt = 0; kt < KTM; ++kt) {
+                const uint4 f = kt < KT ? w_buf[(kt * 8 + quad) * 4 + sub] : make_uint4(0u, 0u, 0u, 0u);
+                pa[kt][0] = f.x; pa[kt][1] = f.y; pa[kt][2] = f.z; pa[kt][3] = f.w;
+            }
+            if (warp == 0) {                               // the row sum is kept (and written out) by warp 0 alone
                 float sum = 0.f;
 #pragma unroll
-                for (int kt = 0; kt < KTM; ++kt) {
-                    float w[8];
-#pragma unroll
-                    for (int e = 0; e < 8; ++e) {
-                        w[e] = ex2f(sw[kt][e] - m_sub) * 256.f;
-                        sum += any ? ex2f(sv[kt][e] - m_sub) : 0.f;
-                    }
-                    split4(w[0], w[1], w[2], w[3], pa[kt][0], pa[kt][1]);
-                    split4(w[4], w[5], w[6], w[7], pa[kt][2], pa[kt][3]);
-                }
+                for (int w8 = 0; w8 < 8; ++w8) sum += den_buf[w8 * 32 + lane];
                 sum += __shfl_xor_sync(0xffffffffu, sum, 1);
                 sum += __shfl_xor_sync(0xffffffffu, sum, 2);
                 l_run = l_run * alpha + sum;
-                m_run = any ? m_new : m_run;
             }
 #pragma unroll
             for (int n = 0; n < 2 * CH; ++n) { acc[n][0] *= alpha; acc[n][1] *= alpha; acc[n][2] *= alpha; acc[n][3] *= alpha; }
@@ -1104,7 +1135,8 @@ cudaError_t launch_decode_fp8_fast(const Dims& d, const void* q, const void* k_c
             return cudaErrorInvalidValue;
         const int CH = d.d_l / 128;
         const size_t stage = (size_t)(d.n_k + CH) * p.T * 128 + ((((size_t)d.n_k + 1) * p.T * 4 + 1023) & ~(size_t)1023);
-        const size_t smem = kStreamStages * stage + 2 * 8 * kStreamMaxT * sizeof(float) +
+        const size_t smem = kStreamStages * stage + 4 * 8 * kStreamMaxT * sizeof(float) +      // scores, shifted scores
+                            (kStreamMaxT / 32) * 32 * 16 + 256 * sizeof(float) +               // weight fragments, row-sum shares
                             (size_t)(kStreamMaxBatch + 2 + kStreamThreads) * sizeof(int32_t) +
                             2 * kStreamStages * sizeof(uint64_t) + 16 + 1024;
 #define GTA_LAUNCH_FP8(CHV)                                                                                \
