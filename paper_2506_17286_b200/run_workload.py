@@ -1,7 +1,7 @@
 """Run one named synthetic workload through the C-ABI library and print per-kernel device times.
 
     python -m paper_2506_17286_b200.run_workload c3_decode_bf16 [--iters 20] [--warmup 3]
-           [--batch B] [--seq N] [--stages MASK] [--append] [--page-size P] [--kv-len L]
+           [--batch B] [--seq N] [--stages MASK] [--append] [--fp8] [--page-size P] [--kv-len L]
 
 A small, self-contained driver for timing or profiling one call at a time (the benchmark
 times the whole step).  Times are CUDA-event times on the launching stream; between
@@ -287,6 +287,60 @@ def run_decode(w, iters, warmup, stages, append):
     return res
 
 
+def run_decode_fp8(w, iters, warmup):
+    """gta_decode_fp8 over caches quantised (outside the timed loop) by the library's own gta_cache_append_fp8."""
+    dev = torch.device("cuda")
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    sets = []
+    for s in range(2):
+        td = I.decode_inputs(I.scaled(w, seed=w.seed + s), device=dev, s_cap=(w.seq or w.ctx_max) + 64)
+        cap, nb = td["s_cap"], w.batch
+        kq = torch.zeros((nb, w.n_k, cap, w.d_h), dtype=torch.uint8, device=dev)
+        cq = torch.zeros((nb, w.n_c, cap, w.d_l), dtype=torch.uint8, device=dev)
+        ks = torch.ones((nb, w.n_k, cap), dtype=torch.float32, device=dev)
+        cs = torch.ones((nb, w.n_c, cap), dtype=torch.float32, device=dev)
+        for b in range(nb):                      # sequence by sequence: the lengths may be ragged
+            n = int(td["seq_lens"][b])
+            if n == 0:
+                continue
+            zero = torch.zeros(1, dtype=torch.int32, device=dev)
+            G.gta_cache_append_fp8(kq[b:b + 1], cq[b:b + 1], ks[b:b + 1], cs[b:b + 1],
+                                   td["k_cache"][b:b + 1, :, :n].contiguous(), td["c_cache"][b:b + 1, :, :n].contiguous(),
+                                   zero, status_word=status)
+        sets.append(dict(kq=kq, cq=cq, ks=ks, cs=cs, lens=td["seq_lens"], q=td["q"], x_t=td["x_t"], w_p=td["w_p"],
+                         w_g=td["w_g"], cap=cap))
+        del td
+    shape = G.make_shape(batch=w.batch, seq=0, d_model=w.d_model, n_heads=w.n_heads, n_q=w.n_q, n_k=w.n_k, n_c=w.n_c,
+                         d_h=w.d_h, d_l=w.d_l, dtype=w.torch_dtype())
+    cap = sets[0]["cap"]
+    ws = torch.zeros(G.decode_fp8_workspace_bytes(shape, cap), dtype=torch.uint8, device=dev)
+    out = torch.empty((w.batch, w.n_heads, w.d_h), dtype=w.torch_dtype(), device=dev)
+    stream = torch.cuda.current_stream()
+
+    def step(it):
+        c = sets[it % 2]
+        G.gta_decode_fp8(c["q"], c["kq"], c["cq"], c["ks"], c["cs"], c["lens"], c["x_t"], c["w_p"], c["w_g"], out=out,
+                         workspace=ws, status_word=status)
+    for it in range(warmup):
+        step(it)
+    torch.cuda.synchronize()
+    times = []
+    for rep in range(3):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for it in range(iters):
+            step(it)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        times.append(e0.elapsed_time(e1) / iters)
+    assert int(status.item()) == 0, "device status word raised"
+    live = float(sets[0]["lens"].sum())
+    cache_bytes = live * ((w.n_k * w.d_h + w.n_c * w.d_l) + 4 * (w.n_k + w.n_c))
+    ms = _median(times)
+    return {"whole_call": ms, "path": G.decode_fp8_path(shape, cap), "launches": G.last_launch_count(),
+            "cache_bytes": cache_bytes, "cache_gbs": cache_bytes / (ms * 1e-3) / 1e9}
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("workload", choices=sorted(I.CONFIGS))
@@ -301,6 +355,8 @@ def main():
     ap.add_argument("--layer", action="store_true",
                     help="the whole attention layer (projections + RoPE + cache write, operator, W_O): "
                          "gta_layer_prefill on a prefill workload, gta_layer_decode on a decode workload")
+    ap.add_argument("--fp8", action="store_true",
+                    help="decode: caches as e4m3 codes with one scale per cached row (gta_decode_fp8)")
     ap.add_argument("--page-size", type=int, default=0,
                     help="decode: keep the caches in a paged pool with pages of this many tokens")
     args = ap.parse_args()
@@ -319,6 +375,8 @@ def main():
         res = run_prefill(w, args.iters, args.warmup, args.stages & 3)
     elif args.layer:
         res = run_layer_decode(w, args.iters, args.warmup)
+    elif args.fp8:
+        res = run_decode_fp8(w, args.iters, args.warmup)
     elif args.page_size > 0:
         res = run_decode_paged(w, args.iters, args.warmup, args.append, args.page_size)
     else:
