@@ -51,6 +51,7 @@ KERNEL_SOURCES = {
     "prefill_attention": "paper_2506_17286_b200/csrc/gta_sm100.cu",
     "prefill_decoder_gate": "paper_2506_17286_b200/csrc/gta_sm100_decoder.cu",
     "decode_stream": "paper_2506_17286_b200/csrc/gta_decode_sm100.cu",
+    "decode_stream_fp8": "paper_2506_17286_b200/csrc/gta_decode_sm100.cu",
 }
 
 
@@ -799,6 +800,9 @@ def run_ours(args):
                               "rows + weights + vectors; streaming kernel with warp-level e4m3 MMAs, paced by its consumer "
                               "warps (those MMAs are carried out as f16 MMAs behind operand conversions on this architecture)")
         r["path"] = G.decode_fp8_path(shape_d, ctx + 64)
+        tr = traffic.get(("decode_stream_fp8", "c3"))
+        r["traffic"] = tr["bytes"] if tr else None
+        r["traffic_source"] = tr["source"] if tr else None
         r["cache_bytes_vs_bf16"] = cache_bytes / by["cache"]
         r["ms_vs_bf16_decode_call"] = t8 / t_decode_call
         return r
