@@ -236,15 +236,24 @@ sm100_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
             int n_armed = 0;            // query tiles whose load has been issued
             int tail_armed = 0;         // loads through tail_bar
             const uint32_t tail_bar_addr = ptx::map_to_cta(ptx::smem_addr(tail_bar), rank);
-            // (row, plane) coordinates of the 64 cached tokens from `token` on of sequence b in a pool of `groups`
-            auto page_block = [&](int b, int token, int groups, int grp, int& row, int& plane) {
+            // Block-table entries of the two 64-token halves of key tile j of sequence b (kPastKeys for a half past the
+            // attended keys, whose entry may not exist).  They are fetched one tile ahead, before the wait for the ring
+            // stage: a table look-up behind that wait would add its latency to every tile.
+            constexpr int kPastKeys = -0x40000000;
+            auto page_entries = [&](int b, int j, int& e0, int& e1) {
+                const int t0 = j * kKeyTile;
+                const int32_t* row = pm.table + (size_t)b * pm.max_pages;
+                e0 = t0 < d.Nk ? row[t0 / pm.page_size] : kPastKeys;
+                e1 = t0 + 64 < d.Nk ? row[(t0 + 64) / pm.page_size] : kPastKeys;
+            };
+            // (row, plane) coordinates of the 64 cached tokens from `token` on, given their block-table entry
+            auto page_block = [&](int entry, int token, int groups, int grp, int& row, int& plane) {
                 row = pm.page_size;     // past the page: the box reads as zeros
                 plane = 0;
-                if (token >= d.Nk) return;
-                const int page = pm.table[(size_t)b * pm.max_pages + token / pm.page_size];
-                if (page < 0 || page >= pm.n_pages) { raise_status(status_word, GTA_ERR_BAD_PAGE); return; }
+                if (entry == kPastKeys) return;
+                if (entry < 0 || entry >= pm.n_pages) { raise_status(status_word, GTA_ERR_BAD_PAGE); return; }
                 row = token % pm.page_size;
-                plane = page * groups + grp;
+                plane = entry * groups + grp;
             };
             bool ok = true;
             AttnItem w;
@@ -261,9 +270,13 @@ sm100_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                 ++n_armed;
                 ptx::tma_load_3d_pair(q_s, &tm_q, q_full_leader, 0, q0, w.b * d.n_q + w.g);
                 if (DH == 128) ptx::tma_load_3d_pair(q_s + 16384, &tm_q, q_full_leader, 64, q0, w.b * d.n_q + w.g);
+                int e_cur[2] = {kPastKeys, kPastKeys}, e_next[2] = {kPastKeys, kPastKeys};
+                if (paged) page_entries(w.b, 0, e_next[0], e_next[1]);
                 for (int j = 0; j < w.n_tiles; ++j, ++tj) {
                     const int s = tj % kAttnStages;
                     const uint32_t ph = (tj / kAttnStages) & 1;
+                    e_cur[0] = e_next[0]; e_cur[1] = e_next[1];
+                    if (paged && j + 1 < w.n_tiles) page_entries(w.b, j + 1, e_next[0], e_next[1]);
                     ok = wait(&empty[s], ph ^ 1, 64);   // the ring is three tiles ahead
                     if (!ok) break;
                     uint8_t* k_s = smem + kAttnRingOff + s * kAttnStageBytes;
@@ -285,9 +298,9 @@ sm100_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                     // keys, or one whose page number is outside the pool, is loaded from a row coordinate past the
                     // page, i.e. as zeros.
                     int k_row, k_plane, c_row[2], c_plane[2];
-                    page_block(w.b, key0, d.n_k, kg, k_row, k_plane);
-                    page_block(w.b, j * kKeyTile, d.n_c, cg, c_row[0], c_plane[0]);
-                    page_block(w.b, j * kKeyTile + 64, d.n_c, cg, c_row[1], c_plane[1]);
+                    page_block(rank ? e_cur[1] : e_cur[0], key0, d.n_k, kg, k_row, k_plane);
+                    page_block(e_cur[0], j * kKeyTile, d.n_c, cg, c_row[0], c_plane[0]);
+                    page_block(e_cur[1], j * kKeyTile + 64, d.n_c, cg, c_row[1], c_plane[1]);
                     // The block that holds position Nk: its rows from Nk on exist in the page and may hold anything.
                     // As keys they are masked, but as latent rows they would meet their zero probabilities in the
                     // sum (0 x NaN), so this block goes through a barrier of this CTA, the thread clears those rows
@@ -368,7 +381,9 @@ sm100_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                         if (ok && j == 0) ok = wait(&q_full[(n & 1) * 41], (n >> 1) & 1);
                         if (ok && (j & 1) == 0) ok = wait(&full[stage], (tile / kAttnStages) & 1);
                         if (!ok) break;
-                        if (paged) ptx::fence_acq_rel_cluster();   // rows of the tile that the peer's producer cleared
+                        // the one tile of which the producers cleared rows (the block that holds position Nk): the
+                        // peer's stores are ordered before its arrival by a release, taken here by an acquire fence
+                        if (paged && (d.Nk & 63) != 0 && (j >> 1) == (d.Nk >> 7)) ptx::fence_acq_rel_cluster();
                         ptx::tc_fence_after_sync();
                         // this CTA's keys 32 (j & 1) .. of its 64 keys of the ring tile: 32 rows of 128 bytes further
                         // on; 32 bytes per k-step inside a 64-column half, the next half 16 KB (Q) / 8 KB (K) on

@@ -26,8 +26,9 @@ def _median(xs):
     return statistics.median(xs) if xs else 0.0
 
 
-def run_prefill_chunk(w, iters, warmup, kv_len):
-    """The last w.seq positions of a kv_len-token context as one chunk (gta_prefill_chunk)."""
+def run_prefill_chunk(w, iters, warmup, kv_len, page_size=0):
+    """The last w.seq positions of a kv_len-token context as one chunk (gta_prefill_chunk; with a page size the
+    keys and latents sit in a pool of pages dealt out in random order: gta_prefill_chunk_paged)."""
     dev = torch.device("cuda")
     t = I.prefill_inputs(w, device=dev)
     gen = torch.Generator(device=dev).manual_seed(w.seed)
@@ -40,9 +41,17 @@ def run_prefill_chunk(w, iters, warmup, kv_len):
     status = torch.zeros(1, dtype=torch.int32, device=dev)
     stream = torch.cuda.current_stream()
 
+    if page_size > 0:
+        pg = I.paginate(dict(k_cache=k, c_cache=c), page_size, seed=w.seed)
+        k_pool, c_pool, table = pg["k_pool"], pg["c_pool"], pg["block_table"]
+
     def step():
-        G.gta_prefill_chunk(t["q"], k, c, t["x"], t["w_p"], t["w_g"], kv_len, out=out, workspace=ws,
-                            status_word=status)
+        if page_size > 0:
+            G.gta_prefill_chunk_paged(t["q"], k_pool, c_pool, table, t["x"], t["w_p"], t["w_g"], kv_len, out=out,
+                                      workspace=ws, status_word=status)
+        else:
+            G.gta_prefill_chunk(t["q"], k, c, t["x"], t["w_p"], t["w_g"], kv_len, out=out, workspace=ws,
+                                status_word=status)
 
     for _ in range(warmup):
         step()
@@ -57,7 +66,7 @@ def run_prefill_chunk(w, iters, warmup, kv_len):
         torch.cuda.synchronize()
         times.append(e0.elapsed_time(e1) / iters)
     assert int(status.item()) == 0, "device status word raised"
-    return {"whole_call": _median(times), "kv_len": kv_len}
+    return {"whole_call": _median(times), "kv_len": kv_len, "page_size": page_size}
 
 
 def run_layer(w, iters, warmup):
@@ -358,7 +367,7 @@ def main():
     ap.add_argument("--fp8", action="store_true",
                     help="decode: caches as e4m3 codes with one scale per cached row (gta_decode_fp8)")
     ap.add_argument("--page-size", type=int, default=0,
-                    help="decode: keep the caches in a paged pool with pages of this many tokens")
+                    help="keep the caches in a paged pool with pages of this many tokens (decode, or a prefill chunk)")
     args = ap.parse_args()
     w = I.CONFIGS[args.workload]
     if args.batch:
@@ -369,8 +378,8 @@ def main():
     torch.cuda.set_device(0)
     if w.kind == "prefill" and args.layer:
         res = run_layer(w, args.iters, args.warmup)
-    elif w.kind == "prefill" and args.kv_len > w.seq:
-        res = run_prefill_chunk(w, args.iters, args.warmup, args.kv_len)
+    elif w.kind == "prefill" and (args.kv_len > w.seq or args.page_size > 0):
+        res = run_prefill_chunk(w, args.iters, args.warmup, max(args.kv_len, w.seq), args.page_size)
     elif w.kind == "prefill":
         res = run_prefill(w, args.iters, args.warmup, args.stages & 3)
     elif args.layer:
