@@ -809,6 +809,34 @@ def run_ours(args):
 
     fp8_cache = fp8_leg()
 
+    # ---- the c3 shape with its caches left in page-locked host memory and read in place at every step (the setting
+    #      of the paper's offload experiments): bound by the host link, not by HBM
+    def offload_leg():
+        ctx, nb = wd.seq, wd.batch
+        sets = []
+        for i in range(2):
+            td = I.decode_inputs(I.scaled(wd, seed=wd.seed + 20 + i), device=dev, s_cap=ctx + 64)
+            for name in ("k_cache", "c_cache"):
+                h = torch.empty(td[name].shape, dtype=td[name].dtype, pin_memory=True)
+                h.copy_(td[name])
+                td[name] = h
+            sets.append(td)
+        torch.cuda.synchronize()
+        wsh = torch.empty(G.decode_hostcache_workspace_bytes(shape_d, ctx + 64), dtype=torch.uint8, device=dev)
+
+        def call(i):
+            c = sets[i % 2]
+            G.gta_decode_hostcache(c["q"], c["k_cache"], c["c_cache"], c["seq_lens"], c["x_t"], c["w_p"], c["w_g"],
+                                   out=out_d, workspace=wsh, status_word=status)
+        th, rech = timed_loop(call, 4, min_ms=100.0)
+        return {"call": "gta_decode_hostcache back to back, two cache sets alternating", "ms": th,
+                "cache_bytes_over_host_link": by["cache"], "host_link_gbs": by["cache"] / (th * 1e-3) / 1e9,
+                "tokens_per_s": nb / (th * 1e-3), "ms_vs_device_resident_step": th / t_decode_call,
+                "note": "bound by the host link (PCIe), so the step time follows the bytes of the cache per token: "
+                        "(n_k d_h + n_c d_l) elements, Table 3 of the paper", "loop": rech}
+
+    offloaded = offload_leg()
+
     # ---- c5: 128 ragged sequences (1024 .. 32768 cached tokens, 8.9 GB live), gta_cache_append + gta_decode per step
     w5 = I.CONFIGS["c5_ragged_decode_bf16"]
     t5 = I.decode_inputs(w5, device=dev)
@@ -947,6 +975,7 @@ def run_ours(args):
             "prefill": {"ms": t_prefill, "tokens_per_s": world * wp.batch * wp.seq / (t_prefill * 1e-3),
                         "flops": fl},
             "layer": layer, "decode": decode, "legs": legs, "comparison_with_gqa": comparisons, "fp8_cache_decode": fp8_cache,
+            "host_cache_decode": offloaded,
             "roofline": roofline,
             "e2e": e2e,
             "cpu_baseline": cpu_baseline, "gpu_launches": n_launches, "clocks": clocks,

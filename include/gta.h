@@ -370,6 +370,26 @@ GTA_API gta_status_t gta_decode_append(const gta_shape_t *shape, const void *q, 
                                        void *cuda_stream);
 
 /*
+ * gta_decode_hostcache — gta_decode with the K and C caches left in HOST memory (the setting of the paper's
+ * offload experiments, Sec. 5.3 and App. C.2: the cache stays in host memory and crosses the host link
+ * at every step, so the step is bound by the bytes of the cache all the more).  k_cache and c_cache are
+ * addresses of page-locked host memory that the device can read directly (cudaHostAlloc / cudaMallocHost,
+ * or cudaHostRegister'ed memory with its device pointer; on a system with unified addressing the host
+ * pointer itself); layouts, lengths, all other arguments (device memory as before), result and errors
+ * are those of gta_decode.  The cache is read in place with ordinary 16-byte loads by the plain-ALU
+ * kernels, every live row exactly once per step: no staging copy and no device memory for the cache.
+ * Pageable host memory is not accepted by the hardware: passing it is an error the library cannot
+ * detect (the kernel faults).  The call also works on device-resident caches (it is then simply the
+ * plain-ALU decode path).  workspace: gta_decode_hostcache_workspace_bytes(shape, S_cap).
+ */
+GTA_API size_t gta_decode_hostcache_workspace_bytes(const gta_shape_t *shape, int32_t S_cap);
+GTA_API gta_status_t gta_decode_hostcache(const gta_shape_t *shape, const void *q, const void *k_cache,
+                                          const void *c_cache, const int32_t *seq_lens, int32_t S_cap,
+                                          const void *x_t, const void *w_p, const void *w_g, void *out,
+                                          void *workspace, size_t workspace_bytes,
+                                          int32_t *status_word, void *cuda_stream);
+
+/*
  * 8-bit caches (the paper has no such format; Sec. 5.3 and App. C.2 only observe that the decode
  * step is bound by the bytes of the cache, the larger the context and the slower the memory the
  * more).  Reading taken here: K and C rows are kept as e4m3 codes (8-bit floats: 1 sign, 4

@@ -30,6 +30,7 @@ EXPORTS = (
     "gta_ref_gqa_prefill", "gta_ref_gqa_decode_workspace_bytes", "gta_ref_gqa_decode",
     "gta_decode_fp8_workspace_bytes", "gta_cache_append_fp8", "gta_decode_fp8", "gta_decode_append",
     "gta_prefill_chunk_paged", "gta_layer_prefill_paged", "gta_decode_fp8_path",
+    "gta_decode_hostcache_workspace_bytes", "gta_decode_hostcache",
 )
 
 
@@ -82,6 +83,10 @@ def lib():
         L.gta_decode_workspace_bytes.restype = sz
         L.gta_decode.argtypes = [sp, vp, vp, vp, vp, i32, vp, vp, vp, vp, vp, sz, vp, vp]
         L.gta_decode.restype = i32
+        L.gta_decode_hostcache_workspace_bytes.argtypes = [sp, i32]
+        L.gta_decode_hostcache_workspace_bytes.restype = sz
+        L.gta_decode_hostcache.argtypes = [sp, vp, vp, vp, vp, i32, vp, vp, vp, vp, vp, sz, vp, vp]
+        L.gta_decode_hostcache.restype = i32
         L.gta_decode_static.argtypes = [sp, vp, vp, vp, vp, i32, vp, vp, vp, vp, vp, vp]
         L.gta_decode_static.restype = i32
         L.gta_cache_append.argtypes = [sp, vp, vp, i32, vp, vp, i32, vp, vp, vp]
@@ -453,6 +458,44 @@ def gta_decode(q, k_cache, c_cache, seq_lens, x_t, w_p, w_g, *, softmax_scale=0.
     st = lib().gta_decode(*args) if stages == 7 else lib().gta_decode_stages(*args, stages)
     if st != GTA_OK:
         raise GtaError(st, "gta_decode")
+    return out
+
+
+def decode_hostcache_workspace_bytes(shape: GtaShape, s_cap: int) -> int:
+    return int(lib().gta_decode_hostcache_workspace_bytes(ctypes.byref(shape), int(s_cap)))
+
+
+def gta_decode_hostcache(q, k_cache, c_cache, seq_lens, x_t, w_p, w_g, *, softmax_scale=0.0, out=None, workspace=None,
+                         status_word=None, stream=None):
+    """gta_decode with k_cache / c_cache in page-locked HOST memory (pinned CPU tensors, read in place over the
+    host link; CUDA tensors are accepted too); everything else lives on the device."""
+    _check_tensors(q, x_t, w_p, w_g)
+    for t in (k_cache, c_cache):
+        if t.dtype != q.dtype or not t.is_contiguous():
+            raise ValueError("the caches must be contiguous and of the operator's dtype")
+        if t.device.type == "cpu" and not t.is_pinned():
+            raise ValueError("a cache in host memory must be page-locked (tensor.pin_memory())")
+        if t.device.type == "cuda" and t.device != q.device:
+            raise ValueError("a cache in device memory must live on the operator's device")
+    if seq_lens.dtype != torch.int32 or seq_lens.device != q.device or not seq_lens.is_contiguous():
+        raise ValueError("seq_lens must be a contiguous int32 tensor on the operator's device")
+    B, n_q, d_h = q.shape
+    s_cap = k_cache.shape[2]
+    shape = decode_shape(q, k_cache, c_cache, x_t, w_p, softmax_scale=softmax_scale)
+    n_h, d_l, H = shape.n_heads, shape.latent_dim, shape.d_model
+    if k_cache.shape != (B, shape.n_k_groups, s_cap, d_h) or c_cache.shape != (B, shape.n_c_groups, s_cap, d_l) \
+            or x_t.shape != (B, H) or w_p.shape != (n_h, d_l, d_h) or w_g.shape != (H, n_h * d_h) \
+            or seq_lens.shape != (B,):
+        raise ValueError("inconsistent operator tensor shapes")
+    if out is None:
+        out = torch.empty((B, n_h, d_h), dtype=q.dtype, device=q.device)
+    if workspace is None:
+        workspace = _workspace(decode_hostcache_workspace_bytes(shape, s_cap), q.device)
+    st = lib().gta_decode_hostcache(ctypes.byref(shape), _ptr(q), _ptr(k_cache), _ptr(c_cache), _ptr(seq_lens), s_cap,
+                                    _ptr(x_t), _ptr(w_p), _ptr(w_g), _ptr(out), _ptr(workspace),
+                                    workspace.numel() * workspace.element_size(), _ptr(status_word), _stream(stream))
+    if st != GTA_OK:
+        raise GtaError(st, "gta_decode_hostcache")
     return out
 
 

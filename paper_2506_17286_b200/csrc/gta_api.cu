@@ -675,6 +675,36 @@ extern "C" gta_status_t gta_decode_fp8(const gta_shape_t* shape, const void* q, 
     return GTA_OK;
 }
 
+// ---- caches in page-locked host memory
+extern "C" size_t gta_decode_hostcache_workspace_bytes(const gta_shape_t* shape, int32_t S_cap) {
+    gta::Dims d;
+    if (check_shape(shape, false, &d) != GTA_OK || S_cap < 0) return 0;
+    return gta::decode_plain_workspace_bytes(d, S_cap);
+}
+
+extern "C" gta_status_t gta_decode_hostcache(const gta_shape_t* shape, const void* q, const void* k_cache,
+                                             const void* c_cache, const int32_t* seq_lens, int32_t S_cap,
+                                             const void* x_t, const void* w_p, const void* w_g, void* out,
+                                             void* workspace, size_t workspace_bytes, int32_t* status_word,
+                                             void* cuda_stream) {
+    g_last_launches = 0;
+    gta::Dims d;
+    bool empty = false;
+    gta_status_t st = gta::decode_check_args(shape, q, k_cache, c_cache, seq_lens, S_cap, x_t, w_p, w_g, out, status_word,
+                                             &d, &empty);
+    if (st != GTA_OK) return st;
+    if (empty) return GTA_OK;
+    if (!workspace || !aligned(workspace, 256) || workspace_bytes < gta::decode_plain_workspace_bytes(d, S_cap))
+        return GTA_ERR_WORKSPACE;
+    if ((st = check_device()) != GTA_OK) return st;
+    int launches = 0;
+    cudaError_t err = gta::launch_decode_plain(d, shape->dtype, q, k_cache, c_cache, seq_lens, S_cap, x_t, w_p, w_g, out,
+                                               workspace, status_word, static_cast<cudaStream_t>(cuda_stream), &launches);
+    if (err != cudaSuccess) return GTA_ERR_CUDA;
+    g_last_launches = launches;
+    return GTA_OK;
+}
+
 // ---- append + decode in one call
 extern "C" gta_status_t gta_decode_append(const gta_shape_t* shape, const void* q, void* k_cache, void* c_cache,
                                           const void* k_new, const void* c_new, int32_t* seq_lens, int32_t S_cap,

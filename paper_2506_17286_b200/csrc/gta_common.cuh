@@ -90,6 +90,13 @@ cudaError_t launch_decode(const Dims& d, int dtype, const void* q, const void* k
                           const void* w_g, void* out, void* workspace, int32_t* status_word,
                           cudaStream_t stream, int stages, int* launches, const PageMap& pm = PageMap());
 size_t decode_workspace_bytes(const Dims& d, int dtype, int S_cap, int page_size = 0);
+// The plain-ALU decode kernels regardless of shape (caches reachable by ordinary loads: device memory or mapped,
+// page-locked host memory).
+size_t decode_plain_workspace_bytes(const Dims& d, int S_cap);
+cudaError_t launch_decode_plain(const Dims& d, int dtype, const void* q, const void* k_cache, const void* c_cache,
+                                const int32_t* seq_lens, int S_cap, const void* x_t, const void* w_p,
+                                const void* w_g, void* out, void* workspace, int32_t* status_word,
+                                cudaStream_t stream, int* launches);
 
 // bf16 bandwidth-oriented decode (persistent streaming kernel + cluster finish kernel).
 bool decode_fast_supported(const Dims& d, int dtype, int page_size = 0);

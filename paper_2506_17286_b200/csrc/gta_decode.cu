@@ -568,6 +568,21 @@ cudaError_t launch_cache_append_fp8(const Dims& d, int dtype, void* k_codes, voi
     return cudaGetLastError();
 }
 
+size_t decode_plain_workspace_bytes(const Dims& d, int S_cap) { return make_plan(d, S_cap).total; }
+
+// The plain-ALU kernels whatever the shape: they read the caches with ordinary 16-byte loads, which is what a cache
+// in page-locked host memory (reached over the host link) needs; the TMA path is kept to device memory.
+cudaError_t launch_decode_plain(const Dims& d, int dtype, const void* q, const void* k_cache, const void* c_cache,
+                                const int32_t* seq_lens, int S_cap, const void* x_t, const void* w_p,
+                                const void* w_g, void* out, void* workspace, int32_t* status_word,
+                                cudaStream_t stream, int* launches) {
+    if (dtype == GTA_F32)
+        return launch_decode_typed<float>(d, q, k_cache, c_cache, seq_lens, S_cap, x_t, w_p, w_g, out,
+                                          workspace, status_word, stream, 7, launches, PageMap());
+    return launch_decode_typed<__nv_bfloat16>(d, q, k_cache, c_cache, seq_lens, S_cap, x_t, w_p, w_g, out,
+                                              workspace, status_word, stream, 7, launches, PageMap());
+}
+
 cudaError_t launch_decode(const Dims& d, int dtype, const void* q, const void* k_cache, const void* c_cache,
                           const int32_t* seq_lens, int S_cap, const void* x_t, const void* w_p,
                           const void* w_g, void* out, void* workspace, int32_t* status_word,

@@ -1,7 +1,7 @@
 """Run one named synthetic workload through the C-ABI library and print per-kernel device times.
 
     python -m paper_2506_17286_b200.run_workload c3_decode_bf16 [--iters 20] [--warmup 3]
-           [--batch B] [--seq N] [--stages MASK] [--append] [--fp8] [--page-size P] [--kv-len L]
+           [--batch B] [--seq N] [--stages MASK] [--append] [--fp8] [--host-cache] [--page-size P] [--kv-len L]
 
 A small, self-contained driver for timing or profiling one call at a time (the benchmark
 times the whole step).  Times are CUDA-event times on the launching stream; between
@@ -296,6 +296,48 @@ def run_decode(w, iters, warmup, stages, append):
     return res
 
 
+def run_decode_hostcache(w, iters, warmup):
+    """gta_decode_hostcache: the caches stay in page-locked host memory and are read in place at every step."""
+    dev = torch.device("cuda")
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    sets = []
+    for s in range(2):
+        td = I.decode_inputs(I.scaled(w, seed=w.seed + s), device=dev)
+        for name in ("k_cache", "c_cache"):
+            h = torch.empty(td[name].shape, dtype=td[name].dtype, pin_memory=True)
+            h.copy_(td[name])
+            td[name] = h
+        sets.append(td)
+    torch.cuda.synchronize()
+    td = sets[0]
+    shape = G.decode_shape(td["q"], td["k_cache"], td["c_cache"], td["x_t"], td["w_p"])
+    ws = torch.zeros(G.decode_hostcache_workspace_bytes(shape, td["s_cap"]), dtype=torch.uint8, device=dev)
+    out = torch.empty((w.batch, w.n_heads, w.d_h), dtype=w.torch_dtype(), device=dev)
+    stream = torch.cuda.current_stream()
+
+    def step(it):
+        c = sets[it % 2]
+        G.gta_decode_hostcache(c["q"], c["k_cache"], c["c_cache"], c["seq_lens"], c["x_t"], c["w_p"], c["w_g"], out=out,
+                               workspace=ws, status_word=status)
+    for it in range(warmup):
+        step(it)
+    torch.cuda.synchronize()
+    times = []
+    for rep in range(3):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for it in range(iters):
+            step(it)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        times.append(e0.elapsed_time(e1) / iters)
+    assert int(status.item()) == 0, "device status word raised"
+    cache_bytes = float(td["seq_lens"].sum()) * (w.n_k * w.d_h + w.n_c * w.d_l) * td["k_cache"].element_size()
+    ms = _median(times)
+    return {"whole_call": ms, "launches": G.last_launch_count(), "cache_bytes": cache_bytes,
+            "host_link_gbs": cache_bytes / (ms * 1e-3) / 1e9}
+
+
 def run_decode_fp8(w, iters, warmup):
     """gta_decode_fp8 over caches quantised (outside the timed loop) by the library's own gta_cache_append_fp8."""
     dev = torch.device("cuda")
@@ -364,6 +406,8 @@ def main():
     ap.add_argument("--layer", action="store_true",
                     help="the whole attention layer (projections + RoPE + cache write, operator, W_O): "
                          "gta_layer_prefill on a prefill workload, gta_layer_decode on a decode workload")
+    ap.add_argument("--host-cache", action="store_true",
+                    help="decode: caches in page-locked host memory, read in place (gta_decode_hostcache)")
     ap.add_argument("--fp8", action="store_true",
                     help="decode: caches as e4m3 codes with one scale per cached row (gta_decode_fp8)")
     ap.add_argument("--page-size", type=int, default=0,
@@ -386,6 +430,8 @@ def main():
         res = run_layer_decode(w, args.iters, args.warmup)
     elif args.fp8:
         res = run_decode_fp8(w, args.iters, args.warmup)
+    elif args.host_cache:
+        res = run_decode_hostcache(w, args.iters, args.warmup)
     elif args.page_size > 0:
         res = run_decode_paged(w, args.iters, args.warmup, args.append, args.page_size)
     else:

@@ -100,6 +100,15 @@ def test_bad_arguments_are_rejected_on_the_host(B):
     assert decode(_shape(B, d_l=4096)) == B.GTA_ERR_UNSUPPORTED
     assert decode(_shape(B, batch=0)) == B.GTA_OK
 
+    def decode_host(shape, s_cap=128, ws=p, ws_bytes=1 << 40, lens=p):
+        return L.gta_decode_hostcache(ctypes.byref(shape), p, p, p, lens, s_cap, p, p, p, p, ws, ws_bytes, None, None)
+
+    assert decode_host(good, s_cap=-1) == B.GTA_ERR_INVALID_ARG
+    assert decode_host(good, lens=None) == B.GTA_ERR_INVALID_ARG
+    assert decode_host(good, ws_bytes=8) == B.GTA_ERR_WORKSPACE
+    assert decode_host(_shape(B, batch=0)) == B.GTA_OK
+    assert B.decode_hostcache_workspace_bytes(good, 1000) > 0
+
     def append(shape, n_new=1, lens=p):
         return L.gta_cache_append(ctypes.byref(shape), p, p, 128, p, p, n_new, lens, None, None)
 
