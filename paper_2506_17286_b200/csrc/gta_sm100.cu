@@ -42,9 +42,9 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
 // the thread of sub-tile u + 1 (the next group) picks it up there.  It is only raised when it grows
 // by more than 2^8 (the accumulators stay in range and O needs rescaling on few sub-tiles).  At the
 // end of an item the softmax threads only hand their (maximum, row sum) pairs over: four epilogue
-// warps (one per TMEM lane quarter) combine the groups' sums, divide O by the row sum, stage it in
-// shared memory as bf16 and write it to L[B, n_q, N, d_l] with TMA tensor stores (whole 128-byte
-// lines, clipped at the sequence end), while the softmax threads are already on the next item.  The
+// warps (one per TMEM lane quarter) combine the groups' sums, divide O by the row sum, round it to
+// bf16 and write it to L[B, n_q, N, d_l] with 32-byte stores (a full sector of the thread's own row,
+// nothing past the sequence end), while the softmax threads are already on the next item.  The
 // ring and the score pipeline run on across items.  The lower query tile of a pair sees one fully
 // masked key tile per item (its probabilities are zero).
 constexpr int kAttnGroups = 4;                     // softmax groups = score buffers = sub-tiles in flight
@@ -74,9 +74,6 @@ __device__ __forceinline__ float fast_exp2(float x) {
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
-}
-__device__ __forceinline__ void epilogue_sync() {   // the four epilogue warps
-    asm volatile("bar.sync 5, 128;" ::: "memory");
 }
 // The four warps of a softmax group (ids 1 .. 4) or the epilogue warps (id 6): one of them polls a
 // barrier of the tensor pipe, the others sleep here at no cost in issue slots until it has seen it.
@@ -149,7 +146,7 @@ __device__ __forceinline__ bool attn_item(const Dims& d, int n_kt, int n_qp, int
 template <int DH, int SLICE>
 __global__ void __launch_bounds__(kAttnThreads, 1)
 sm100_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
-                       const __grid_constant__ CUtensorMap tm_c, const __grid_constant__ CUtensorMap tm_o, Dims d,
+                       const __grid_constant__ CUtensorMap tm_c, __nv_bfloat16* __restrict__ l_out, Dims d,
                        const PageMap pm, int32_t* status_word) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -560,26 +557,26 @@ sm100_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
             have = have_next;
         }
     } else if (warp < 4 * kAttnGroups + 4) {
-        // 4 epilogue warps, one per TMEM lane quarter, a row per thread.  After the last sum of an item
-        // (o_item: one completion per item, and the next cannot come before this item's O has been
-        // handed back) they divide O by the row sum, round to bf16 into the staging boxes (box = 64 columns x
-        // 128 rows, 128-byte swizzle: 16-byte chunk c of row r sits at chunk c ^ (r & 7)) and store
-        // them with TMA: two passes of 128 columns.  O is handed back as soon as it has been read.
+        // 4 epilogue warps, one per TMEM lane quarter, a row per thread.  When the softmax groups have left their
+        // (maximum, row sum) pairs (epi_ready) the row's normaliser is worked out; after the last sum of the item
+        // (o_item: one completion per item, and the next cannot come before this item's O has been handed back) O is
+        // read 16 columns at a time, the next 16 already on their way while the current ones are scaled, rounded to
+        // bf16 and written straight to L with one 32-byte store per thread (a full sector of the thread's own row):
+        // nothing between the read and the hand-back waits for a staging buffer or a store, so O is back with the
+        // MMA threads after one pass over its columns.  (An earlier form staged 64-column boxes in shared memory
+        // for TMA stores and held O for 2.7 us per item; handing it back sooner did not change the kernel's time,
+        // which is set by the steady rate of the score-buffer loop, but this form needs no staging buffer.)
         const int quarter = warp & 3;
         const int row = quarter * 32 + lane;
         const uint32_t lane_base = ((uint32_t)(quarter * 32) << 16);
         const uint32_t o_free_leader = ptx::map_to_cta(ptx::smem_addr(o_free), 0);
         const float2* xsum = reinterpret_cast<const float2*>(smem + kAttnSumOff);
-        const bool store_issuer = warp == 4 * kAttnGroups && lane == 0;
+        const bool poller = quarter == 2;    // one warp polls, the others are woken by it through a named barrier
         bool ok = true;      // as for the softmax warps: on a wait that gave up the loops run to their end
         AttnItem w;
         for (int n = 0; attn_item(d, n_kt, n_qp, n_slices, total, G, pr, n, &w); ++n) {
-            if (quarter == 2) {     // one warp polls (slowly: an item takes many microseconds), the others are woken by it
-                ok = __all_sync(0xffffffffu, wait(o_item, n & 1, 200));
-                ok = __all_sync(0xffffffffu, wait(epi_ready, n & 1));
-            }
+            if (poller) ok = __all_sync(0xffffffffu, wait(epi_ready, n & 1, 200));
             wait_group_sync(6);
-            ptx::tc_fence_after_sync();
             // the groups' sums, each relative to the maximum its group saw last; O is relative to the largest
             float2 gs[kAttnGroups];
             float m_fin = -INFINITY;
@@ -593,16 +590,20 @@ sm100_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
             for (int g = 0; g < kAttnGroups; ++g)
                 l_fin += gs[g].x == -INFINITY ? 0.f : gs[g].y * fast_exp2(gs[g].x - m_fin);
             const float inv_l = 1.f / l_fin;
-            const int q0 = (2 * w.qp + (int)rank) * 128;
             const uint64_t inv2 = ptx::f32x2(inv_l, inv_l);
-            uint8_t* stage = smem + ((n & 1) ? kAttnOutOff : 0u);    // the buffer that held this item's Q
-            // Four passes of 64 columns = one box each, the two halves of the buffer used alternately: a pass
-            // only waits for the store of the pass before last.  O is read 16 columns at a time, the next 16
-            // already on their way while the current ones are scaled, rounded and staged; it is handed back
-            // as soon as its last columns are in registers (the next item's first sum waits for that).
+            const int t = (2 * w.qp + (int)rank) * 128 + row;             // this thread's query row
+            const int col0 = w.slice * SLICE;
+            // narrow latent: the second half of the slice repeats the first and is not stored
+            const int n_cols = narrow ? SLICE / 2 : SLICE;
+            __nv_bfloat16* dst = l_out + ((size_t)(w.b * d.n_q + w.g) * d.N + (t < d.N ? t : 0)) * d.d_l + col0;
+            const bool live = t < d.N;
+            if (poller) ok = __all_sync(0xffffffffu, wait(o_item, n & 1, 64));
+            wait_group_sync(6);
+            ptx::tc_fence_after_sync();
+            // every score MMA of the item is complete too: its query tile's buffer may take the tile of item n + 2
+            if (warp == 4 * kAttnGroups && lane == 0) ptx::mbar_arrive(stage_free);
             uint32_t ra[16], rb[16];
-            auto stage_out = [&](const uint32_t (&r)[16], int c) {      // columns 16 c .. 16 c + 15 of the slice
-                uint8_t* box_row = stage + ((c >> 2) & 1) * kAttnOutBoxBytes + row * 128;
+            auto write_out = [&](const uint32_t (&r)[16], int c) {      // columns 16 c .. 16 c + 15 of the slice
                 uint32_t pk[8];
 #pragma unroll
                 for (int e = 0; e < 8; ++e) {
@@ -610,48 +611,24 @@ sm100_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
                     ptx::f32x2_split(ptx::mul2(ptx::f32x2(__uint_as_float(r[2 * e]), __uint_as_float(r[2 * e + 1])), inv2), v0, v1);
                     pk[e] = pack_bf16x2(v0, v1);
                 }
-#pragma unroll
-                for (int h = 0; h < 2; ++h) {        // 16-byte chunks 2 (c & 3), 2 (c & 3) + 1 of the box row
-                    const int chunk = ((c & 3) * 2 + h) ^ (row & 7);
-                    *reinterpret_cast<uint4*>(box_row + chunk * 16) = make_uint4(pk[4 * h], pk[4 * h + 1], pk[4 * h + 2], pk[4 * h + 3]);
-                }
+                if (live && c * 16 < n_cols) ptx::st_global_256(dst + c * 16, pk);
             };
             constexpr int kChunks = SLICE / 16;
             ptx::tmem_ld16(tmem_o + lane_base, ra);
 #pragma unroll 1
-            for (int pass = 0; pass < SLICE / 64; ++pass) {
-                if (pass >= 2) {
-                    if (store_issuer) ptx::bulk_wait_group_read_but_one();
-                    epilogue_sync();
+            for (int c = 0; c < kChunks; c += 2) {
+                ptx::tmem_wait_ld();
+                ptx::tmem_ld16(tmem_o + lane_base + (c + 1) * 16, rb);
+                write_out(ra, c);
+                ptx::tmem_wait_ld();
+                if (c + 2 < kChunks) {
+                    ptx::tmem_ld16(tmem_o + lane_base + (c + 2) * 16, ra);
+                } else {                  // O has been read completely: the next item's sums may start
+                    ptx::tc_fence_before_sync();
+                    __syncwarp();
+                    if (lane == 0) ptx::mbar_arrive_cluster(o_free_leader);
                 }
-#pragma unroll
-                for (int q = 0; q < 4; q += 2) {
-                    const int c = pass * 4 + q;
-                    ptx::tmem_wait_ld();
-                    ptx::tmem_ld16(tmem_o + lane_base + (c + 1) * 16, rb);
-                    stage_out(ra, c);
-                    ptx::tmem_wait_ld();
-                    if (c + 2 < kChunks) {
-                        ptx::tmem_ld16(tmem_o + lane_base + (c + 2) * 16, ra);
-                    } else {                  // O has been read completely: the next item's sums may start
-                        ptx::tc_fence_before_sync();
-                        __syncwarp();
-                        if (lane == 0) ptx::mbar_arrive_cluster(o_free_leader);
-                    }
-                    stage_out(rb, c + 1);
-                }
-                ptx::fence_proxy_async_smem();
-                epilogue_sync();
-                if (store_issuer && q0 < d.N && w.slice * SLICE + pass * 64 < d.d_l) {
-                    ptx::tma_store_3d(&tm_o, stage + (pass & 1) * kAttnOutBoxBytes, w.slice * SLICE + pass * 64, q0,
-                                      w.b * d.n_q + w.g);
-                    ptx::bulk_commit_group();
-                }
-            }
-            // the buffer may take the query tile of item n + 2 once the stores have read it
-            if (store_issuer) {
-                ptx::bulk_wait_group_read_all();
-                ptx::mbar_arrive(stage_free);
+                write_out(rb, c + 1);
             }
         }
     }
@@ -685,7 +662,7 @@ bool sm100_prefill_supported(const Dims& d, int dtype) {
 // One instantiation of the attention kernel: its occupancy (asked once per device) and its launch.
 template <int DH, int SLICE>
 static gta_status_t launch_attention(const Dims& d, const PageMap& pm, const CUtensorMap& tm_q, const CUtensorMap& tm_k,
-                                     const CUtensorMap& tm_c, const CUtensorMap& tm_o, int32_t* status_word,
+                                     const CUtensorMap& tm_c, __nv_bfloat16* l_out, int32_t* status_word,
                                      cudaStream_t stream) {
     auto kern = sm100_attention_kernel<DH, SLICE>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kAttnSmemTotal) != cudaSuccess)
@@ -722,7 +699,7 @@ static gta_status_t launch_attention(const Dims& d, const PageMap& pm, const CUt
     const int pairs = (int)(n_items < cached_pairs ? n_items : cached_pairs);
     cfg.gridDim = dim3(2 * pairs);
     cfg.numAttrs = 2;
-    if (cudaLaunchKernelEx(&cfg, kern, tm_q, tm_k, tm_c, tm_o, d, pm, status_word) != cudaSuccess) return GTA_ERR_CUDA;
+    if (cudaLaunchKernelEx(&cfg, kern, tm_q, tm_k, tm_c, l_out, d, pm, status_word) != cudaSuccess) return GTA_ERR_CUDA;
     return cudaGetLastError() == cudaSuccess ? GTA_OK : GTA_ERR_CUDA;
 }
 
@@ -730,7 +707,8 @@ static gta_status_t launch_attention(const Dims& d, const PageMap& pm, const CUt
 // multiple of 128, or 64 (the narrow case of the comparison operators).
 gta_status_t launch_sm100_attention(const Dims& d, const void* q, const void* k, const void* c, void* l_out,
                                     int32_t* status_word, cudaStream_t stream, const PageMap& pm) {
-    CUtensorMap tm_q, tm_k, tm_c, tm_o;
+    CUtensorMap tm_q, tm_k, tm_c;
+    __nv_bfloat16* l_bf16 = static_cast<__nv_bfloat16*>(l_out);
     const uint32_t box[3] = {64, 128, 1}, box_k[3] = {64, 64, 1};
     const uint64_t dq[3] = {(uint64_t)d.d_h, (uint64_t)d.N, (uint64_t)d.B * d.n_q};
     if (pm.table != nullptr) {
@@ -752,18 +730,13 @@ gta_status_t launch_sm100_attention(const Dims& d, const void* q, const void* k,
             !make_bf16_map(&tm_c, c, 3, dc, box, ac))
             return GTA_ERR_CUDA;
     }
-    {   // L [B n_q][N][d_l], stored in boxes of 128 rows x 64 columns
-        const uint64_t dl[3] = {(uint64_t)d.d_l, (uint64_t)d.N, (uint64_t)d.B * d.n_q};
-        const uint32_t box_o[3] = {64, 128, 1};
-        if (!make_bf16_map(&tm_o, l_out, 3, dl, box_o)) return GTA_ERR_CUDA;
-    }
     gta_status_t st;
     if (d.d_h == 128)
-        st = d.d_l % 256 == 0 ? launch_attention<128, 256>(d, pm, tm_q, tm_k, tm_c, tm_o, status_word, stream)
-                              : launch_attention<128, 128>(d, pm, tm_q, tm_k, tm_c, tm_o, status_word, stream);
+        st = d.d_l % 256 == 0 ? launch_attention<128, 256>(d, pm, tm_q, tm_k, tm_c, l_bf16, status_word, stream)
+                              : launch_attention<128, 128>(d, pm, tm_q, tm_k, tm_c, l_bf16, status_word, stream);
     else
-        st = d.d_l % 256 == 0 ? launch_attention<64, 256>(d, pm, tm_q, tm_k, tm_c, tm_o, status_word, stream)
-                              : launch_attention<64, 128>(d, pm, tm_q, tm_k, tm_c, tm_o, status_word, stream);
+        st = d.d_l % 256 == 0 ? launch_attention<64, 256>(d, pm, tm_q, tm_k, tm_c, l_bf16, status_word, stream)
+                              : launch_attention<64, 128>(d, pm, tm_q, tm_k, tm_c, l_bf16, status_word, stream);
     if (st != GTA_OK) return st;
     return cudaGetLastError() == cudaSuccess ? GTA_OK : GTA_ERR_CUDA;
 }
