@@ -395,15 +395,24 @@ sm100_linear_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
     if (threadIdx.x == 0 && *abort_flag) raise_status(status_word, GTA_ERR_TIMEOUT);
 }
 
+// SM count of the CURRENT device, looked up once per device ordinal and thread
 int lin_sm_count() {
-    static int n = [] {
-        int dev = 0, v = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess ||
-            cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v <= 0)
+    static thread_local int cached_dev = -1, cached_n = 148;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) {
+        cudaGetLastError();
+        return 148;
+    }
+    if (dev != cached_dev) {
+        int v = 0;
+        if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v <= 0) {
+            cudaGetLastError();
             v = 148;
-        return v;
-    }();
-    return n;
+        }
+        cached_dev = dev;
+        cached_n = v;
+    }
+    return cached_n;
 }
 
 template <bool kProject>
