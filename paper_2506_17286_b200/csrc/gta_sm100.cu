@@ -160,7 +160,11 @@ sm100_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
     uint64_t* p_full = bars + 14;       // [4] leader CTA; the 4 warps of a softmax group of both CTAs arrive
     uint64_t* o_done = bars + 18;       // [4] both CTAs (multicast commit): the sum of a sub-tile is complete
     uint64_t* o_free = bars + 22;       // leader CTA; 8 epilogue warps arrive
-    uint64_t* epi_ready = bars + 23;    // this CTA; its 16 softmax warps arrive (maxima and row sums of an item are in place)
+    // this CTA; its 16 softmax warps arrive (maxima and row sums of an item are in place).  One barrier for the even
+    // items (slot 23) and one for the odd ones (slot 47): a group that is done with item n early goes on to a short
+    // item n + 1 and may arrive for it before the last group has arrived for item n; on a single barrier that arrival
+    // would complete item n's phase with that group's pair still missing.
+    uint64_t* epi_ready = bars + 23;
     uint64_t* o_item = bars + 24;       // both CTAs (multicast commit): the last sum of an item is complete
     uint64_t* chain = bars + 25;        // [4 groups][4 quarters] this CTA; one warp arrives: its rows' running maxima are published
     uint64_t* mma_drain = bars + 42;    // [2] leader CTA: used once by an MMA-issuing thread that unwinds (all its MMAs are done)
@@ -203,7 +207,8 @@ sm100_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
             ptx::mbar_init(&s_full[s], 1); ptx::mbar_init(&p_full[s], 8); ptx::mbar_init(&o_done[s], 1);
         }
         ptx::mbar_init(o_free, 8);
-        ptx::mbar_init(epi_ready, 4 * kAttnGroups);
+        ptx::mbar_init(&epi_ready[0], 4 * kAttnGroups);
+        ptx::mbar_init(&epi_ready[24], 4 * kAttnGroups);
         ptx::mbar_init(o_item, 1);
         for (int s = 0; s < 4 * kAttnGroups; ++s) ptx::mbar_init(&chain[s], 1);
         *abort_flag = 0;
@@ -552,7 +557,7 @@ sm100_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
             //      back, which the sums of item n + 1 wait for, long before item n + 2 ends)
             xsum[((n & 1) * kAttnGroups + wg) * 128 + row] = make_float2(m_own, l);
             __syncwarp();
-            if (lane == 0) ptx::mbar_arrive(epi_ready);
+            if (lane == 0) ptx::mbar_arrive(&epi_ready[(n & 1) * 24]);
             w = nxt;
             have = have_next;
         }
@@ -575,7 +580,7 @@ sm100_attention_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_co
         bool ok = true;      // as for the softmax warps: on a wait that gave up the loops run to their end
         AttnItem w;
         for (int n = 0; attn_item(d, n_kt, n_qp, n_slices, total, G, pr, n, &w); ++n) {
-            if (poller) ok = __all_sync(0xffffffffu, wait(epi_ready, n & 1, 200));
+            if (poller) ok = __all_sync(0xffffffffu, wait(&epi_ready[(n & 1) * 24], (n >> 1) & 1, 200));
             wait_group_sync(6);
             // the groups' sums, each relative to the maximum its group saw last; O is relative to the largest
             float2 gs[kAttnGroups];

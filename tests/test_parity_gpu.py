@@ -110,7 +110,7 @@ def test_prefill_repeated_runs_with_several_items_per_cta(B, oracle):
     want = oracle.prefill(oracle_shape(w), tc["q"], tc["k"], tc["c"], tc["x"], tc["w_p"], tc["w_g"], rows=rows)
     sel = torch.as_tensor(rows, device="cuda", dtype=torch.long)
     first = None
-    for rep in range(12):
+    for rep in range(60):
         out = B.gta_prefill(t["q"], t["k"], t["c"], t["x"], t["w_p"], t["w_g"])
         torch.cuda.synchronize()
         assert_close(out[:, sel], want, torch.bfloat16, f"repeat {rep}")
