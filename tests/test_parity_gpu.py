@@ -567,3 +567,42 @@ def test_decode_append_equals_append_then_decode(B, oracle, case):
                         c_a[:, :, :live].contiguous().cpu(), lens_a.cpu().numpy(), live, t["x_t"].cpu(), t["w_p"].cpu(),
                         t["w_g"].cpu())
     assert_close(got, ref, w.torch_dtype(), name)
+
+
+def _step_full_size(B, oracle, w, sample):
+    """The fused step as the benchmark times it (full size, lengths that do not count the new token yet): result on
+    sampled sequences against the oracle over the caches WITH the new rows, the new rows bit for bit in every
+    sequence's cache, the rows around them untouched, the lengths advanced."""
+    t = I.decode_inputs(w, device="cuda")
+    lens_after = t["seq_lens"].clone()
+    lens = lens_after - 1                                   # the caches hold all tokens but the one being decoded
+    pos = lens.long()
+    ar = torch.arange(w.batch, device="cuda")
+    k_before = t["k_cache"][ar, :, pos + 1].clone()         # the row behind the new one must stay as it is
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    out = B.gta_decode_append(t["q"], t["k_cache"], t["c_cache"], t["k_new"], t["c_new"], lens, t["x_t"], t["w_p"],
+                              t["w_g"], status_word=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0 and torch.equal(lens, lens_after)
+    assert torch.equal(t["k_cache"][ar, :, pos].view(torch.int16), t["k_new"][:, :, 0].view(torch.int16))
+    assert torch.equal(t["c_cache"][ar, :, pos].view(torch.int16), t["c_new"][:, :, 0].view(torch.int16))
+    assert torch.equal(t["k_cache"][ar, :, pos + 1].view(torch.int16), k_before.view(torch.int16))
+    sel = torch.as_tensor(sample, device="cuda", dtype=torch.long)
+    sub = lens_after[sel].cpu().numpy()
+    cap = int(sub.max())
+    want = oracle.decode(oracle_shape(I.scaled(w, batch=len(sample)), seq=0), t["q"][sel].cpu(),
+                         t["k_cache"][sel][:, :, :cap].contiguous().cpu(), t["c_cache"][sel][:, :, :cap].contiguous().cpu(),
+                         sub, cap, t["x_t"][sel].cpu(), t["w_p"].cpu(), t["w_g"].cpu())
+    assert_close(out[sel], want, torch.bfloat16, w.name + " fused step")
+
+
+def test_decode_append_config3_full_size_sampled_sequences(B, oracle):
+    w = I.CONFIGS["c3_decode_bf16"]
+    _step_full_size(B, oracle, w, [0, 7, 16, 31])
+
+
+def test_decode_append_config5_full_size_sampled_sequences(B, oracle):
+    w = I.CONFIGS["c5_ragged_decode_bf16"]
+    lens = I.decode_seq_lens(w).numpy()
+    order = np.argsort(lens)
+    _step_full_size(B, oracle, w, sorted({int(order[0]), int(order[-1]), int(order[len(order) // 2]), 0, 127}))
