@@ -343,8 +343,16 @@ decode_stream_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_cons
             }
             const int s = it % kStreamStages;
             const uint32_t ph = (it / kStreamStages) & 1;
-            ok = __all_sync(0xffffffffu, ptx::mbar_wait(&full_bar[s], ph, abort_flag));
-            if (!ok) break;
+            // A wait that gives up raises the CTA's abort flag, after which every wait returns at once.  The warp does
+            // NOT leave the loop then: other consumer warps may already stand at a CTA barrier of this or a later
+            // sub-tile, which needs all eight.  It skips the work and keeps the appointments (as many barriers as the
+            // sub-tile has) to the end of its range; nothing is flushed.
+            ok = __all_sync(0xffffffffu, ptx::mbar_wait(&full_bar[s], ph, abort_flag));   // (once false, false for good: the flag)
+            if (!ok) {
+                if (L.appends(b) && ((int)k + 1) * T >= L.len(b)) consumer_sync();
+                consumer_sync();
+                continue;
+            }
             const int len = L.len(b);
             const int n_valid = min(T, len - (int)k * T);
             // the sub-tile that ends the sequence holds the new token (row n_valid - 1): what TMA brought for that
@@ -905,7 +913,8 @@ decode_stream_fp8_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_
         load_q(b);
         int it = 0;
         bool ok = true;
-        for (long long st = st_begin; st < st_end; ++st, ++it, ++k) {
+        long long st = st_begin;
+        for (; st < st_end; ++st, ++it, ++k) {
             if (k >= prefix[b + 1] - prefix[b]) {
                 flush(b);
                 do { ++b; } while (prefix[b + 1] == prefix[b]);
@@ -915,7 +924,7 @@ decode_stream_fp8_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_
             const int s = it % kStreamStages;
             const uint32_t ph = (it / kStreamStages) & 1;
             ok = __all_sync(0xffffffffu, ptx::mbar_wait(&full_bar[s], ph, abort_flag));
-            if (!ok) break;
+            if (!ok) break;      // (the appointments of the remaining sub-tiles are kept below)
             const int n_valid = min(T, L.len(b) - (int)k * T);
             const uint32_t stage = ring_addr + s * stage_stride;
             const float* ksc = reinterpret_cast<const float*>(ring + s * stage_stride + scale_off);
@@ -1055,6 +1064,13 @@ decode_stream_fp8_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_
             if (lane == 0) ptx::mbar_arrive(&empty_bar[s]);
         }
         if (ok) flush(b);
+        // A wait that gave up (it raises the CTA's abort flag, after which every wait returns at once): other consumer
+        // warps may already stand at a CTA barrier of this or a later sub-tile, which needs all eight, so the warp
+        // keeps its appointments -- two barriers per sub-tile -- to the end of the range before it leaves.
+        for (; st < st_end; ++st) {
+            consumer_sync();
+            consumer_sync();
+        }
     }
     __syncthreads();
     if (tid == 0 && *abort_flag) raise_status(status_word, GTA_ERR_TIMEOUT);
