@@ -60,21 +60,25 @@ size_t decode_workspace_bytes(const Dims& d, int dtype, int S_cap, int page_size
 template <typename T> struct Vec16;
 template <> struct Vec16<float> {
     static constexpr int N = 4;
+    static __device__ __forceinline__ void widen(const uint4& r, float (&v)[4]) {
+        v[0] = __uint_as_float(r.x); v[1] = __uint_as_float(r.y); v[2] = __uint_as_float(r.z); v[3] = __uint_as_float(r.w);
+    }
     static __device__ __forceinline__ void load(const float* p, float (&v)[4]) {
-        const float4 r = __ldg(reinterpret_cast<const float4*>(p));
-        v[0] = r.x; v[1] = r.y; v[2] = r.z; v[3] = r.w;
+        widen(__ldg(reinterpret_cast<const uint4*>(p)), v);
     }
 };
 template <> struct Vec16<__nv_bfloat16> {
     static constexpr int N = 8;
-    static __device__ __forceinline__ void load(const __nv_bfloat16* p, float (&v)[8]) {
-        const uint4 r = __ldg(reinterpret_cast<const uint4*>(p));
+    static __device__ __forceinline__ void widen(const uint4& r, float (&v)[8]) {
         const uint32_t w[4] = {r.x, r.y, r.z, r.w};
 #pragma unroll
         for (int i = 0; i < 4; ++i) {  // bf16 is the upper half of an fp32
             v[2 * i] = __uint_as_float(w[i] << 16);
             v[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
         }
+    }
+    static __device__ __forceinline__ void load(const __nv_bfloat16* p, float (&v)[8]) {
+        widen(__ldg(reinterpret_cast<const uint4*>(p)), v);
     }
 };
 
@@ -87,13 +91,15 @@ __device__ __forceinline__ float e4m3_to_f32(uint32_t b) {
 }
 template <> struct Vec16<Fp8> {
     static constexpr int N = 16;
-    static __device__ __forceinline__ void load(const Fp8* p, float (&v)[16]) {
-        const uint4 r = __ldg(reinterpret_cast<const uint4*>(p));
+    static __device__ __forceinline__ void widen(const uint4& r, float (&v)[16]) {
         const uint32_t w[4] = {r.x, r.y, r.z, r.w};
 #pragma unroll
         for (int i = 0; i < 4; ++i)
 #pragma unroll
             for (int j = 0; j < 4; ++j) v[4 * i + j] = e4m3_to_f32(w[i] >> (8 * j));
+    }
+    static __device__ __forceinline__ void load(const Fp8* p, float (&v)[16]) {
+        widen(__ldg(reinterpret_cast<const uint4*>(p)), v);
     }
 };
 
@@ -104,7 +110,11 @@ template <> __device__ __forceinline__ float exp_fn<__nv_bfloat16>(float x) { re
 // Dynamic shared memory of decode_partial_kernel (floats):
 //   q_s [n_q][d_h] | p_s [chunk][n_q] | ml_s [n_q][2] | red [R][d_l]
 // CT: storage type of the caches (T, or Fp8 with one fp32 scale per cached row in k_scale / c_scale).
-template <typename T, int NGB, typename CT = T>
+// kReadOnce: every cached row is loaded exactly once, for caches that sit behind the host link, where a row
+// that is loaded again crosses the link again: a key row's vector is kept in registers for all the maps of its
+// key group, and the maps of a latent group need not be a multiple of NGB (the last accumulators of the last
+// pass idle).  On device memory the repeated loads hit L1 / L2 and the leaner loops are faster.
+template <typename T, int NGB, typename CT = T, bool kReadOnce = false>
 __global__ void __launch_bounds__(kDecodeThreads)
 decode_partial_kernel(Dims d, int chunk, int n_chunks, int S_cap, const T* __restrict__ q,
                       const CT* __restrict__ k_cache, const CT* __restrict__ c_cache,
@@ -132,7 +142,76 @@ decode_partial_kernel(Dims d, int chunk, int n_chunks, int S_cap, const T* __res
     __syncthreads();
 
     // ---- scores: LPR lanes share one K row, one 16-byte vector per lane and step ----
-    {
+    if constexpr (kReadOnce) {
+        constexpr int kScoreRows = 4;                       // rows per lane group whose loads are issued together
+        constexpr int kMapsAtOnce = 8;                      // maps of a key group per pass over a row's registers
+        constexpr int kSlots = (256 / VEC + 31) / 32;       // vectors per lane and row (d_h <= 256): 2 for fp32, else 1
+        const int vecs_per_row = d.d_h / VEC;
+        int lpr = 1;
+        while (lpr < vecs_per_row && lpr < 32) lpr <<= 1;
+        const int rows_per_warp = 32 / lpr;
+        const int sub = lane / lpr, sl = lane % lpr;
+        const int q_per_k = d.n_q / d.n_k;
+        const int n_row_iters = (n_tok + rows_per_warp - 1) / rows_per_warp;
+        const int total_iters = d.n_k * n_row_iters;
+        constexpr int kWarps = kDecodeThreads / 32;
+        for (int it0 = warp; it0 < total_iters; it0 += kWarps * kScoreRows) {
+            uint4 raw[kScoreRows][kSlots];
+            float row_scale[kScoreRows];
+#pragma unroll
+            for (int u = 0; u < kScoreRows; ++u) {
+                const int it = it0 + u * kWarps;
+                const bool in = it < total_iters;
+                const int kg = in ? it / n_row_iters : 0;
+                const int j = in ? (it % n_row_iters) * rows_per_warp + sub : 0;
+                const long long k_idx = cache_row(pm, b, d.n_k, kg, S_cap, j_begin + (j < n_tok ? j : 0), status_word);
+                const CT* k_row = k_cache + (size_t)(k_idx < 0 ? 0 : k_idx) * d.d_h;
+                row_scale[u] = kScaled ? d.scale * k_scale[k_idx < 0 ? 0 : k_idx] : d.scale;
+#pragma unroll
+                for (int s = 0; s < kSlots; ++s) {
+                    raw[u][s] = make_uint4(0u, 0u, 0u, 0u);
+                    if (in && j < n_tok && sl + s * lpr < vecs_per_row)
+                        raw[u][s] = __ldg(reinterpret_cast<const uint4*>(k_row + (sl + s * lpr) * VEC));
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < kScoreRows; ++u) {
+                const int it = it0 + u * kWarps;
+                if (it >= total_iters) break;       // uniform over the warp
+                const int kg = it / n_row_iters;
+                const int j = (it % n_row_iters) * rows_per_warp + sub;
+                float kv[kSlots][VEC];
+#pragma unroll
+                for (int s = 0; s < kSlots; ++s) Vec16<CT>::widen(raw[u][s], kv[s]);
+                for (int g0 = 0; g0 < q_per_k; g0 += kMapsAtOnce) {
+                    float dot[kMapsAtOnce];
+#pragma unroll
+                    for (int gi = 0; gi < kMapsAtOnce; ++gi) {
+                        dot[gi] = 0.f;
+                        if (g0 + gi < q_per_k) {
+                            const float* qv = q_s + (kg * q_per_k + g0 + gi) * d.d_h + sl * VEC;
+#pragma unroll
+                            for (int s = 0; s < kSlots; ++s) {
+                                if (sl + s * lpr < vecs_per_row) {
+#pragma unroll
+                                    for (int e = 0; e < VEC; ++e) dot[gi] = fmaf(qv[s * lpr * VEC + e], kv[s][e], dot[gi]);
+                                }
+                            }
+                        }
+                    }
+                    for (int o = lpr >> 1; o > 0; o >>= 1) {
+#pragma unroll
+                        for (int gi = 0; gi < kMapsAtOnce; ++gi) dot[gi] += __shfl_xor_sync(0xffffffffu, dot[gi], o);
+                    }
+                    if (j < n_tok && sl == 0) {
+#pragma unroll
+                        for (int gi = 0; gi < kMapsAtOnce; ++gi)
+                            if (g0 + gi < q_per_k) p_s[j * d.n_q + kg * q_per_k + g0 + gi] = dot[gi] * row_scale[u];
+                    }
+                }
+            }
+        }
+    } else {
         const int vecs_per_row = d.d_h / VEC;
         int lpr = 1;
         while (lpr < vecs_per_row && lpr < 32) lpr <<= 1;
@@ -198,7 +277,8 @@ decode_partial_kernel(Dims d, int chunk, int n_chunks, int S_cap, const T* __res
             const long long idx = cache_row(pm, b, d.n_c, cg, S_cap, j_begin + j, status_word);
             return (size_t)(idx < 0 ? 0 : idx);
         };
-        for (int g0 = cg * maps_per_c; g0 < (cg + 1) * maps_per_c; g0 += NGB) {
+        const int g_end = (cg + 1) * maps_per_c;
+        for (int g0 = cg * maps_per_c; g0 < g_end; g0 += NGB) {
             float acc[NGB][VEC];
 #pragma unroll
             for (int gi = 0; gi < NGB; ++gi)
@@ -221,6 +301,7 @@ decode_partial_kernel(Dims d, int chunk, int n_chunks, int S_cap, const T* __res
                         const float* pj = p_s + (j + u * R) * d.n_q + g0;
 #pragma unroll
                         for (int gi = 0; gi < NGB; ++gi) {
+                            if (kReadOnce && g0 + gi >= g_end) break;
                             const float p = pj[gi] * cs[u];      // the row's scale folded into its probability
 #pragma unroll
                             for (int e = 0; e < VEC; ++e) acc[gi][e] = fmaf(p, cv[u][e], acc[gi][e]);
@@ -235,6 +316,7 @@ decode_partial_kernel(Dims d, int chunk, int n_chunks, int S_cap, const T* __res
                     const float* pj = p_s + j * d.n_q + g0;
 #pragma unroll
                     for (int gi = 0; gi < NGB; ++gi) {
+                        if (kReadOnce && g0 + gi >= g_end) break;
                         const float p = pj[gi] * cs;
 #pragma unroll
                         for (int e = 0; e < VEC; ++e) acc[gi][e] = fmaf(p, cv[e], acc[gi][e]);
@@ -244,6 +326,7 @@ decode_partial_kernel(Dims d, int chunk, int n_chunks, int S_cap, const T* __res
             // reduce the R row slots through shared memory, one map at a time
 #pragma unroll
             for (int gi = 0; gi < NGB; ++gi) {
+                if (kReadOnce && g0 + gi >= g_end) break;      // uniform over the CTA
                 __syncthreads();
                 if (active) {
 #pragma unroll
@@ -370,7 +453,8 @@ decode_finish_kernel(Dims d, int chunk, int n_chunks, int S_cap, int gate_splits
     }
 }
 
-template <typename T>
+// kReadOnce: the caches are read over the host link (see decode_partial_kernel)
+template <typename T, bool kReadOnce = false>
 static cudaError_t launch_decode_typed(const Dims& d, const void* q, const void* k_cache, const void* c_cache,
                                        const int32_t* seq_lens, int S_cap, const void* x_t, const void* w_p,
                                        const void* w_g, void* out, void* workspace, int32_t* status_word,
@@ -396,7 +480,7 @@ static cudaError_t launch_decode_typed(const Dims& d, const void* q, const void*
         dim3 grid(p.n_chunks, d.B);
 #define GTA_LAUNCH_PARTIAL(NGB)                                                                        \
         do {                                                                                           \
-            auto kern = decode_partial_kernel<T, NGB>;                                                 \
+            auto kern = decode_partial_kernel<T, NGB, T, kReadOnce>;                                   \
             if (smem > 48 * 1024) {                                                                    \
                 err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem); \
                 if (err != cudaSuccess) return err;                                                    \
@@ -405,7 +489,12 @@ static cudaError_t launch_decode_typed(const Dims& d, const void* q, const void*
                                                          (const T*)k_cache, (const T*)c_cache, seq_lens, \
                                                          part_o, part_ml, pm, status_word, nullptr, nullptr); \
         } while (0)
-        if (maps_per_c % 8 == 0) GTA_LAUNCH_PARTIAL(8);
+        if (kReadOnce) {    // as few passes over the latent rows as the accumulators allow
+            if (maps_per_c >= 5) GTA_LAUNCH_PARTIAL(8);
+            else if (maps_per_c >= 3) GTA_LAUNCH_PARTIAL(4);
+            else if (maps_per_c == 2) GTA_LAUNCH_PARTIAL(2);
+            else GTA_LAUNCH_PARTIAL(1);
+        } else if (maps_per_c % 8 == 0) GTA_LAUNCH_PARTIAL(8);
         else if (maps_per_c % 4 == 0) GTA_LAUNCH_PARTIAL(4);
         else if (maps_per_c % 2 == 0) GTA_LAUNCH_PARTIAL(2);
         else GTA_LAUNCH_PARTIAL(1);
@@ -577,10 +666,10 @@ cudaError_t launch_decode_plain(const Dims& d, int dtype, const void* q, const v
                                 const void* w_g, void* out, void* workspace, int32_t* status_word,
                                 cudaStream_t stream, int* launches) {
     if (dtype == GTA_F32)
-        return launch_decode_typed<float>(d, q, k_cache, c_cache, seq_lens, S_cap, x_t, w_p, w_g, out,
-                                          workspace, status_word, stream, 7, launches, PageMap());
-    return launch_decode_typed<__nv_bfloat16>(d, q, k_cache, c_cache, seq_lens, S_cap, x_t, w_p, w_g, out,
-                                              workspace, status_word, stream, 7, launches, PageMap());
+        return launch_decode_typed<float, true>(d, q, k_cache, c_cache, seq_lens, S_cap, x_t, w_p, w_g, out,
+                                                workspace, status_word, stream, 7, launches, PageMap());
+    return launch_decode_typed<__nv_bfloat16, true>(d, q, k_cache, c_cache, seq_lens, S_cap, x_t, w_p, w_g, out,
+                                                    workspace, status_word, stream, 7, launches, PageMap());
 }
 
 cudaError_t launch_decode(const Dims& d, int dtype, const void* q, const void* k_cache, const void* c_cache,

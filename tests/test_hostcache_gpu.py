@@ -66,6 +66,10 @@ HOST_CASES = [
     ("bf16_empty_and_shared_keys", "bf16", 4, 128, 8, 4, 2, 2, 64, 128, [0, 512, 1, 300]),
     ("bf16_paper_1b_grouping", "bf16", 2, 1280, 20, 5, 1, 1, 64, 128, [333, 1000]),
     ("f32_general", "f32", 3, 96, 6, 6, 3, 1, 32, 64, [100, 7, 260]),
+    # more maps on one key / latent group than one pass of the kernel holds (8): two passes, the second ragged
+    ("bf16_twelve_maps_one_group", "bf16", 2, 128, 12, 12, 1, 1, 64, 128, [130, 77]),
+    # three maps per latent group (a ragged pass of four) and key rows of two 16-byte vectors per lane
+    ("f32_wide_heads_three_maps_per_latent", "f32", 2, 64, 6, 6, 2, 2, 256, 256, [50, 129]),
 ]
 
 
