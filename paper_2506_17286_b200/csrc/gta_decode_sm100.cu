@@ -1142,7 +1142,12 @@ cudaError_t launch_decode_fp8_fast(const Dims& d, const void* q, const void* k_c
     float* part_ml = reinterpret_cast<float*>(static_cast<char*>(workspace) + p.off_ml);
     __nv_bfloat16* l_g = reinterpret_cast<__nv_bfloat16*>(static_cast<char*>(workspace) + p.off_l);
     cudaError_t err;
-    {
+    if (decode_fp8_tc_supported(d, p.T)) {     // the tokens as the rows of tcgen05 MMAs
+        err = launch_decode_fp8_tc_stream(d, p.G, S_cap, q, k_codes, c_codes, k_scale, c_scale, seq_lens, part_o, part_ml,
+                                          status_word, stream);
+        if (err != cudaSuccess) return err;
+        *launches += 1;
+    } else {
         CUtensorMap tm_k, tm_c;
         const uint32_t box[3] = {128, (uint32_t)p.T, 1};
         const uint64_t dk[3] = {128, (uint64_t)S_cap, (uint64_t)d.B * d.n_k};
