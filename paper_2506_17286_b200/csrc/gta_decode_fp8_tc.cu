@@ -23,7 +23,12 @@
 //
 // Schedule, ring, scale rows, partial results (slot c + b: running maximum, row sum, unnormalised latent sums) are
 // those of the other stream kernels, so decode_merge_kernel and the decoder kernel follow unchanged.
-// Warps 0-3: token / column threads (TMEM lane quarters), warp 4: TMA producer, warp 5: MMA issue.
+// Warps 0-3 (group A, one per TMEM lane quarter): read a sub-tile's scores, keep the running maxima, leave the
+// exponents of the weights and of the row-sum terms in shared memory.  Warps 4-7 (group B, again one per lane
+// quarter): exponentials, the weights' pieces into the B operand, rescaling of the sums when a maximum has grown,
+// the partial result at the end of a sequence.  A works on sub-tile i + 1 while B works on sub-tile i: a single
+// warp per scheduler runs at the latency of its dependent instructions, not at its issue rate, so the chain of a
+// sub-tile is cut in two.  Warp 8: TMA producer.  Warp 9: MMA issue.
 #include "gta_common.cuh"
 #include "gta_sm100.cuh"
 #include "sm100_ptx.cuh"
@@ -34,10 +39,11 @@ namespace {
 
 constexpr int kTcT = 64;                        // tokens per sub-tile
 constexpr int kTcStages = 3;
-constexpr int kTcThreads = 192;
+constexpr int kTcThreads = 320;
 constexpr int kTcMaxBatch = 512;
 constexpr uint32_t kTcTile = kTcT * 128;        // bytes of a [64 tokens][128 codes] tile
 constexpr uint32_t kTcOperand = 16 * 128;       // bytes of a [16 rows][128 codes] B operand (Q pieces, weights' pieces)
+constexpr uint32_t kTcExpBytes = 2 * 2 * 8 * kTcT * 4;   // exponents handed from group A to group B
 constexpr uint32_t kTcTmemCols = 256;           // 2 x 64 score columns, 64 sum columns
 constexpr float kTcWeightScale = 64.f;          // the weights are scaled into e4m3's range ...
 constexpr float kTcLag = 2.f;                   // ... with room for a running maximum that lags by 2^2
@@ -67,12 +73,16 @@ __host__ __device__ inline TcSmem tc_smem_layout(int n_k, int ch) {
     s.q_off = kTcStages * s.stage_stride;            // [2 sequence parities][16][128]
     s.p_off = s.q_off + 2 * kTcOperand;              // [2 sub-tile parities][16][128]
     s.misc_off = s.p_off + 2 * kTcOperand;
-    // prefix [B + 2] | scan [kTcThreads] | mx [2][4][8] | l_red [4][8] | qmul [2][8] | 16 barriers | 4 words
-    s.total = s.misc_off + (kTcMaxBatch + 2 + kTcThreads) * 4 + (64 + 32 + 16) * 4 + 16 * 8 + 16 + 1024;
+    // exponents [2][2][8][64] | prefix [B + 2] | scan [kTcThreads] | mx [2][4][8] | l_red [4][8] | qmul [2][8] |
+    // hdr [2][8 alpha, 8 maxima, grow, pad 7] | 24 barriers | 4 words
+    s.total = s.misc_off + kTcExpBytes + (kTcMaxBatch + 2 + kTcThreads) * 4 + (64 + 32 + 16 + 48) * 4 + 24 * 8 + 16 + 1024;
     return s;
 }
 
-template <int CH>
+// CH: 128-column blocks of the latent; NK: key groups; QPK: maps per key group (compile-time, so that the per-map
+// loops of the token threads unroll into straight code: those threads run one warp per scheduler, at the latency of
+// every instruction they issue).
+template <int CH, int NK, int QPK>
 __global__ void __launch_bounds__(kTcThreads, 1)
 decode_stream_fp8_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_c, Dims d,
                             int S_cap, const __nv_bfloat16* __restrict__ q, const float* __restrict__ k_scale,
@@ -80,47 +90,53 @@ decode_stream_fp8_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __gr
                             float* __restrict__ part_o, float* __restrict__ part_ml, int32_t* status_word) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-    const TcSmem lay = tc_smem_layout(d.n_k, CH);
+    const TcSmem lay = tc_smem_layout(NK, CH);
     uint8_t* ring = smem;
     uint8_t* q_buf = smem + lay.q_off;
     uint8_t* p_buf = smem + lay.p_off;
-    int32_t* prefix = reinterpret_cast<int32_t*>(smem + lay.misc_off);       // [B + 1]
+    float* e_buf = reinterpret_cast<float*>(smem + lay.misc_off);             // [2 parities][weights, row sums][8 maps][64 tokens]
+    int32_t* prefix = reinterpret_cast<int32_t*>(smem + lay.misc_off + kTcExpBytes);   // [B + 1]
     int32_t* scan_tmp = prefix + kTcMaxBatch + 2;                             // [kTcThreads]
     float* mx_buf = reinterpret_cast<float*>(scan_tmp + kTcThreads);          // [2 parities][4 warps][8 maps]
     float* l_red = mx_buf + 64;                                               // [4 warps][8 maps]
     float* qmul = l_red + 32;                                                 // [2 parities][8 maps]
-    uint64_t* full_bar = reinterpret_cast<uint64_t*>(qmul + 16);              // [3] TMA bytes of a stage have landed
+    float* hdr = qmul + 16;                                                   // [2 parities][8 alpha | 8 maxima | grow | -]
+    uint64_t* full_bar = reinterpret_cast<uint64_t*>(hdr + 48);               // [3] TMA bytes of a stage have landed
     uint64_t* empty_bar = full_bar + kTcStages;                               // [3] the sums of its sub-tile are complete
     uint64_t* s_ready = empty_bar + kTcStages;                                // [2] scores of sub-tile i are in buffer i & 1
-    uint64_t* p_ready = s_ready + 2;                                          // [2] 4 warps: weights written, scores read, O rescaled
+    uint64_t* p_ready = s_ready + 2;                                          // [2] 4 warps of B: weights written, O rescaled
     uint64_t* pv_done = p_ready + 2;                                          // [2] the sums of sub-tile i are complete
     uint64_t* q_ready = pv_done + 2;                                          // [2] 4 warps: query pieces of sequence n in buffer n & 1
-    uint64_t* drain_bar = q_ready + 2;
+    uint64_t* s_free = q_ready + 2;                                           // [2] 4 warps of A: the scores have been read
+    uint64_t* xy_ready = s_free + 2;                                          // [2] 4 warps of A: exponents and header of sub-tile i
+    uint64_t* xy_free = xy_ready + 2;                                         // [2] 4 warps of B: ... have been read
+    uint64_t* drain_bar = xy_free + 2;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(drain_bar + 1);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
     volatile int* drain_flag = abort_flag + 1;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int G = gridDim.x, cta = blockIdx.x;
-    const int NQ = d.n_q;
-    const int qpk = NQ / d.n_k;                       // maps per key group
+    constexpr int NQ = NK * QPK;
+    constexpr int qpk = QPK;
 
     if (tid == 0) {
         for (int s = 0; s < kTcStages; ++s) { ptx::mbar_init(&full_bar[s], 1); ptx::mbar_init(&empty_bar[s], 1); }
         for (int s = 0; s < 2; ++s) {
             ptx::mbar_init(&s_ready[s], 1); ptx::mbar_init(&p_ready[s], 4);
             ptx::mbar_init(&pv_done[s], 1); ptx::mbar_init(&q_ready[s], 4);
+            ptx::mbar_init(&s_free[s], 4); ptx::mbar_init(&xy_ready[s], 4); ptx::mbar_init(&xy_free[s], 4);
         }
         ptx::mbar_init(drain_bar, 1);
         *abort_flag = 0;
         *drain_flag = 0;
         ptx::fence_mbar_init();
     }
-    if (warp == 4 && lane == 0) {
+    if (warp == 8 && lane == 0) {
         ptx::prefetch_tensormap(&tm_k);
         ptx::prefetch_tensormap(&tm_c);
     }
-    if (warp == 5) ptx::tmem_alloc(tmem_slot, kTcTmemCols);
+    if (warp == 9) ptx::tmem_alloc(tmem_slot, kTcTmemCols);
     // rows of the B operands that belong to no map stay zero for the whole kernel
     for (uint32_t i = tid; i < 4 * kTcOperand / 16; i += kTcThreads)
         reinterpret_cast<uint4*>(q_buf)[i] = make_uint4(0u, 0u, 0u, 0u);
@@ -171,10 +187,10 @@ decode_stream_fp8_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __gr
     const int k0 = n_sub > 0 ? (int)(st_begin - prefix[b0]) : 0;     // first sub-tile of sequence b0 in this range
     const uint32_t ring_addr = ptx::smem_addr(ring);
 
-    if (n_sub > 0 && warp == 4) {
+    if (n_sub > 0 && warp == 8) {
         // ------------------------------------------------------------------ producer: one load per lane
         const uint64_t policy = ptx::l2_evict_first_policy();
-        const int n_tiles = d.n_k + CH, n_ops = n_tiles + d.n_k + 1;      // tensor tiles, then the scale rows
+        const int n_tiles = NK + CH, n_ops = n_tiles + NK + 1;      // tensor tiles, then the scale rows
         int b = b0, k = k0, it = 0;
         bool ok = true;
         for (; it < n_sub; ++it, ++k) {
@@ -185,21 +201,21 @@ decode_stream_fp8_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __gr
             const uint32_t n_sc = (uint32_t)min(kTcT, S_cap - tok0) * 4;   // bytes of a scale row (S_cap is a multiple of 4)
             if (lane == 0) {
                 ok = ptx::mbar_wait(&empty_bar[s], ph ^ 1, abort_flag);
-                if (ok) ptx::mbar_arrive_expect_tx(&full_bar[s], lay.scale_off + (uint32_t)(d.n_k + 1) * n_sc);
+                if (ok) ptx::mbar_arrive_expect_tx(&full_bar[s], lay.scale_off + (uint32_t)(NK + 1) * n_sc);
             }
             ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
             if (!ok) break;
             uint8_t* stage = ring + s * lay.stage_stride;
             for (int op = lane; op < n_ops; op += 32) {
-                if (op < d.n_k)
-                    ptx::tma_load_3d_hint(stage + op * kTcTile, &tm_k, &full_bar[s], 0, tok0, b * d.n_k + op, policy);
+                if (op < NK)
+                    ptx::tma_load_3d_hint(stage + op * kTcTile, &tm_k, &full_bar[s], 0, tok0, b * NK + op, policy);
                 else if (op < n_tiles)
-                    ptx::tma_load_3d_hint(stage + op * kTcTile, &tm_c, &full_bar[s], (op - d.n_k) * 128, tok0, b, policy);
-                else if (op < n_tiles + d.n_k)
+                    ptx::tma_load_3d_hint(stage + op * kTcTile, &tm_c, &full_bar[s], (op - NK) * 128, tok0, b, policy);
+                else if (op < n_tiles + NK)
                     ptx::bulk_load_1d(stage + lay.scale_off + (op - n_tiles) * kTcT * 4,
-                                      k_scale + ((size_t)b * d.n_k + (op - n_tiles)) * S_cap + tok0, n_sc, &full_bar[s]);
+                                      k_scale + ((size_t)b * NK + (op - n_tiles)) * S_cap + tok0, n_sc, &full_bar[s]);
                 else
-                    ptx::bulk_load_1d(stage + lay.scale_off + d.n_k * kTcT * 4, c_scale + (size_t)b * S_cap + tok0, n_sc,
+                    ptx::bulk_load_1d(stage + lay.scale_off + NK * kTcT * 4, c_scale + (size_t)b * S_cap + tok0, n_sc,
                                       &full_bar[s]);
             }
         }
@@ -209,7 +225,7 @@ decode_stream_fp8_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __gr
                 ptx::mbar_wait_drain(&full_bar[iq % kTcStages], (iq / kTcStages) & 1, drain_flag);
             }
         }
-    } else if (n_sub > 0 && warp == 5) {
+    } else if (n_sub > 0 && warp == 9) {
         // ------------------------------------------------------------------ MMA issue (one thread)
         if (ptx::elect_one()) {
             constexpr uint32_t idesc_s = ptx::make_idesc_e4m3(128, 16, 0, 0);    // key tile and query pieces, both K-major
@@ -229,13 +245,15 @@ decode_stream_fp8_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __gr
                 const int s = j % kTcStages;
                 if (first && !ptx::mbar_wait(&q_ready[sn & 1], (sn >> 1) & 1, abort_flag)) return false;
                 if (!ptx::mbar_wait(&full_bar[s], (j / kTcStages) & 1, abort_flag)) return false;
+                // the buffer held the scores of sub-tile j - 2
+                if (j >= 2 && !ptx::mbar_wait(&s_free[j & 1], ((j >> 1) - 1) & 1, abort_flag)) return false;
                 ptx::tc_fence_after_sync();
                 const uint32_t stage = ring_addr + s * lay.stage_stride;
                 const uint64_t dq = desc_kmajor + ((q_addr + (sn & 1) * kTcOperand) >> 4);
                 // The 128 rows of A are the 64 tokens of key group 2 kp and, 8 KB further on, the same 64 tokens of key
                 // group 2 kp + 1 (the tiles of a stage lie back to back; behind the last key tile come latent rows,
                 // whose "scores" nobody reads): lanes 0-63 and 64-127 of the accumulator.
-                for (int kp = 0; 2 * kp < d.n_k; ++kp) {
+                for (int kp = 0; 2 * kp < NK; ++kp) {
                     const uint64_t dk = desc_kmajor + ((stage + 2 * kp * kTcTile) >> 4);
 #pragma unroll
                     for (int ks = 0; ks < 4; ++ks)      // 32 codes = 32 bytes of the 128-byte rows per step
@@ -247,8 +265,7 @@ decode_stream_fp8_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __gr
             };
             ok = issue_scores(0);
             for (int i = 0; i < n_sub && ok; ++i) {
-                // the scores of the next sub-tile go into the other buffer, which the token threads have read
-                // (their arrival for sub-tile i - 1 was waited for below)
+                // the scores of the next sub-tile go into the other buffer, once group A has read it
                 if (i + 1 < n_sub) ok = issue_scores(i + 1);
                 if (!ok) break;
                 bool first = (i == 0);
@@ -262,7 +279,7 @@ decode_stream_fp8_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __gr
                 const uint64_t dp = desc_kmajor + ((p_addr + (i & 1) * kTcOperand) >> 4);
 #pragma unroll
                 for (int c = 0; c < CH; ++c) {
-                    const uint64_t dc = desc_latent + ((stage + (d.n_k + c) * kTcTile) >> 4);
+                    const uint64_t dc = desc_latent + ((stage + (NK + c) * kTcTile) >> 4);
 #pragma unroll
                     for (int kk = 0; kk < 2; ++kk)      // 32 tokens = 4096 bytes of the tile, 32 bytes of the weights' rows
                         ptx::mma_ss_f8(tmem_o + c * 16, dc + kk * (4096 >> 4), dp + 2 * kk, idesc_o,
@@ -276,24 +293,36 @@ decode_stream_fp8_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __gr
                 ptx::mbar_wait_drain(drain_bar, 0, drain_flag);
             }
         }
-    } else if (n_sub > 0 && warp < 4) {
-        // ------------------------------------------------------------------ token / column threads
-        const uint32_t lane_base = ((uint32_t)(warp * 32) << 16);
+    } else if (n_sub > 0 && warp < 8) {
+        // ------------------------------------------------------------------ groups A and B
+        // Scores: quarters 0 / 1 hold tokens 0-31 / 32-63 for the even key groups, quarters 2 / 3 the same tokens for
+        // the odd ones; a thread of B takes over the (token, maps) of the thread of A in the same place.  Sums: lane
+        // 32 quarter + lane is a latent column of each 128-column block.
+        const bool group_b = warp >= 4;
+        const int quarter = warp & 3;
+        const int gtid = tid & 127;                      // thread index inside the group
+        const uint32_t lane_base = ((uint32_t)(quarter * 32) << 16);
         const uint32_t tmem_o = tmem_base + 128 + lane_base;
-        // Scores: warps 0 / 1 hold tokens 0-31 / 32-63 for the even key groups, warps 2 / 3 the same tokens for the
-        // odd ones.  Sums: lane 32 warp + lane is a latent column of each 128-column block.
-        const int half = warp >> 1;
-        const int token = (warp & 1) * 32 + lane;        // of the sub-tile
+        const int half = quarter >> 1;
+        const int token = (quarter & 1) * 32 + lane;     // of the sub-tile
         const uint32_t tok_swz = (uint32_t)token >> 4, tok_low = (uint32_t)token & 15u;
-        float m_run[8], l_thr[8];
+        int kg_of[8];                       // key group of map g
+        bool mine[8];                       // this thread handles map g
 #pragma unroll
-        for (int g = 0; g < 8; ++g) { m_run[g] = -INFINITY; l_thr[g] = 0.f; }
+        for (int g = 0; g < 8; ++g) {
+            kg_of[g] = g / qpk;
+            mine[g] = g < NQ && (kg_of[g] & 1) == half;
+        }
+        int b = b0, k = k0, n = 0;          // sequence, its sub-tile, its ordinal in this range
+        int len_b = tc_len(seq_lens, b, S_cap), n_sub_b = prefix[b + 1] - prefix[b];
+        bool ok = true, first = true;
 
+        if (!group_b) {
         // the query pieces of sequence b into buffer par: warp w takes the maps 2 w and 2 w + 1, a lane four elements
         auto write_q = [&](int b, int par) {
 #pragma unroll
             for (int h = 0; h < 2; ++h) {
-                const int g = 2 * warp + h;
+                const int g = 2 * quarter + h;
                 if (g < NQ) {     // uniform over the warp
                     const uint2 raw = __ldg(reinterpret_cast<const uint2*>(q + ((size_t)b * NQ + g) * 128 + 4 * lane));
                     const float2 v01 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&raw.x));
@@ -327,55 +356,52 @@ decode_stream_fp8_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __gr
             return (nb < d.B && prefix[nb] < st_end) ? nb : -1;
         };
 
-        int b = b0, k = k0, n = 0;          // sequence, its sub-tile, its ordinal in this range
-        int len_b = tc_len(seq_lens, b, S_cap), n_sub_b = prefix[b + 1] - prefix[b];
-        int kg_of[8];                       // key group of map g
-        bool mine[8];                       // this thread scores map g
-#pragma unroll
-        for (int g = 0; g < 8; ++g) {
-            kg_of[g] = g / qpk;
-            mine[g] = g < NQ && (kg_of[g] & 1) == half;
-        }
-        write_q(b, 0);
-        tc_group_sync();                    // qmul of the first sequence is visible to all
-        bool ok = true, first = true;
-        for (int i = 0; i < n_sub; ++i, ++k) {
-            if (k >= n_sub_b) {
-                do { ++b; } while (prefix[b + 1] == prefix[b]);
-                k = 0;
-                ++n;
-                first = true;
-                len_b = tc_len(seq_lens, b, S_cap);
-                n_sub_b = prefix[b + 1] - prefix[b];
-            }
-            if (first) {    // the buffer of the sequence before this one is free: every score of it has been read
-                const int nb = next_seq(b);
-                if (nb >= 0) write_q(nb, (n + 1) & 1);
-            }
-            const int s = i % kTcStages;
-            const int n_valid = min(kTcT, len_b - k * kTcT);
-            uint8_t* stage = ring + s * lay.stage_stride;
-            const float* ksc = reinterpret_cast<const float*>(stage + lay.scale_off);
-            const float* csc = ksc + d.n_k * kTcT;
-            ok = ptx::mbar_wait(&full_bar[s], (i / kTcStages) & 1, abort_flag) && ok;
-            ok = ptx::mbar_wait(&s_ready[i & 1], (i >> 1) & 1, abort_flag) && ok;
-            ptx::tc_fence_after_sync();
 
-            // ---- this token's scores of this thread's maps, plain (x) and shifted by log2 of the latent row's scale (y)
-            float x[8], y[8];
+            float m_run[8];
 #pragma unroll
-            for (int g = 0; g < 8; ++g) x[g] = y[g] = -INFINITY;
-            {
+            for (int g = 0; g < 8; ++g) m_run[g] = -INFINITY;
+            write_q(b, 0);
+            asm volatile("bar.sync 1, 128;" ::: "memory");      // qmul of the first sequence is visible to all of A
+            for (int i = 0; i < n_sub; ++i, ++k) {
+                if (k >= n_sub_b) {
+                    do { ++b; } while (prefix[b + 1] == prefix[b]);
+                    k = 0;
+                    ++n;
+                    first = true;
+                    len_b = tc_len(seq_lens, b, S_cap);
+                    n_sub_b = prefix[b + 1] - prefix[b];
+#pragma unroll
+                    for (int g = 0; g < 8; ++g) m_run[g] = -INFINITY;
+                }
+                if (first) {    // the buffer of the sequence before this one is free: every score of it has been read
+                    const int nb = next_seq(b);
+                    if (nb >= 0) write_q(nb, (n + 1) & 1);
+                }
+                const int s = i % kTcStages;
+                const int n_valid = min(kTcT, len_b - k * kTcT);
+                const float* ksc = reinterpret_cast<const float*>(ring + s * lay.stage_stride + lay.scale_off);
+                const float* csc = ksc + NK * kTcT;
+                ok = ptx::mbar_wait(&full_bar[s], (i / kTcStages) & 1, abort_flag) && ok;
+                ok = ptx::mbar_wait(&s_ready[i & 1], (i >> 1) & 1, abort_flag) && ok;
+                ptx::tc_fence_after_sync();
+
+                // ---- this token's scores of this thread's maps, plain (x) and shifted by log2 of the latent row's scale (y)
+                float x[8], y[8];
+#pragma unroll
+                for (int g = 0; g < 8; ++g) x[g] = y[g] = -INFINITY;
                 const bool live = token < n_valid;
                 const float shift = live ? __log2f(csc[token]) : 0.f;
                 uint32_t r[2][16];
 #pragma unroll
                 for (int kp = 0; kp < 2; ++kp)
-                    if (2 * kp < d.n_k) ptx::tmem_ld16(tmem_base + lane_base + (i & 1) * 64 + kp * 16, r[kp]);
+                    if (2 * kp < NK) ptx::tmem_ld16(tmem_base + lane_base + (i & 1) * 64 + kp * 16, r[kp]);
                 ptx::tmem_wait_ld();
+                ptx::tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(&s_free[i & 1]);
 #pragma unroll
                 for (int kp = 0; kp < 2; ++kp) {
-                    if (2 * kp + half < d.n_k) {
+                    if (2 * kp + half < NK) {
                         const float ks = live ? ksc[(2 * kp + half) * kTcT + token] : 0.f;
 #pragma unroll
                         for (int g = 0; g < 8; ++g) {
@@ -390,138 +416,235 @@ decode_stream_fp8_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __gr
                 for (int g = 0; g < 8; ++g) {
                     if (mine[g]) {      // uniform over the warp
                         const float mw = ptx::warp_max_redux(y[g]);
-                        if (lane == 0) mx_buf[((i & 1) * 4 + warp) * 8 + g] = mw;
+                        if (lane == 0) mx_buf[((i & 1) * 4 + quarter) * 8 + g] = mw;
                     }
                 }
-            }
-            // ---- rows past the live length hold whatever the cache holds there (NaN codes included): their
-            //      weights are zero, so the latent rows are cleared
-            if (n_valid < kTcT) {
-                const int n_vec = (kTcT - n_valid) * CH * 8;
-                for (int idx = tid; idx < n_vec; idx += 128) {
-                    const int row = n_valid + idx / (CH * 8), v = idx % (CH * 8);
-                    *reinterpret_cast<uint4*>(stage + (d.n_k + (v >> 3)) * kTcTile + row * 128 + (v & 7) * 16) =
-                        make_uint4(0u, 0u, 0u, 0u);
-                }
-            }
-            tc_group_sync();
+                asm volatile("bar.sync 1, 128;" ::: "memory");
 
-            // ---- the running maxima; the sums so far are rescaled when one of them grows
-            float alpha[8], m_sub[8];
-            bool grow = false;
+                // ---- the running maxima: a reference is raised only when the sub-tile exceeds it by more than kTcLag
+                //      (the weights, scaled by kTcWeightScale, then stay within e4m3's range: 64 x 2^2 = 256 <= 448)
+                float alpha[8], m_sub[8];
+                bool grow = false;
 #pragma unroll
-            for (int g = 0; g < 8; ++g) {
-                alpha[g] = 1.f;
-                m_sub[g] = 0.f;
-                if (g < NQ) {
-                    // the reference is raised only when the sub-tile exceeds it by more than kTcLag (the weights,
-                    // scaled by kTcWeightScale, then stay within e4m3's range: 64 x 2^2 = 256 <= 448)
-                    const int w0 = (i & 1) * 4 + 2 * (kg_of[g] & 1);      // the two warps that score map g
-                    const float m_tile = fmaxf(mx_buf[w0 * 8 + g], mx_buf[(w0 + 1) * 8 + g]);
-                    const bool up = m_tile > m_run[g] + kTcLag;
-                    grow = grow || up;
-                    alpha[g] = up ? tc_ex2(m_run[g] - m_tile) : 1.f;
-                    m_run[g] = up ? m_tile : m_run[g];
-                    m_sub[g] = m_run[g] > -INFINITY ? m_run[g] : 0.f;
-                    l_thr[g] *= alpha[g];
+                for (int g = 0; g < 8; ++g) {
+                    alpha[g] = 1.f;
+                    m_sub[g] = 0.f;
+                    if (g < NQ) {
+                        const int w0 = (i & 1) * 4 + 2 * (kg_of[g] & 1);      // the two warps that score map g
+                        const float m_tile = fmaxf(mx_buf[w0 * 8 + g], mx_buf[(w0 + 1) * 8 + g]);
+                        const bool up = m_tile > m_run[g] + kTcLag;
+                        grow = grow || up;
+                        alpha[g] = up ? tc_ex2(m_run[g] - m_tile) : 1.f;
+                        m_run[g] = up ? m_tile : m_run[g];
+                        m_sub[g] = m_run[g] > -INFINITY ? m_run[g] : 0.f;
+                    }
                 }
-            }
-            if (grow && !first) {       // uniform over the CTA; the first sub-tile of a sequence overwrites the sums
-                ok = ptx::mbar_wait(&pv_done[(i - 1) & 1], ((i - 1) >> 1) & 1, abort_flag) && ok;
-                ptx::tc_fence_after_sync();
-#pragma unroll
-                for (int c = 0; c < CH; ++c) {
-                    uint32_t r[16];
-                    ptx::tmem_ld16(tmem_o + c * 16, r);
-                    ptx::tmem_wait_ld();
-#pragma unroll
-                    for (int e = 0; e < 16; ++e) r[e] = __float_as_uint(__uint_as_float(r[e]) * alpha[e >> 1]);
-                    ptx::tmem_st16(tmem_o + c * 16, r);
-                }
-                ptx::tmem_wait_st();
-            }
-            // ---- the weights' pieces of this token into the B operand of the sums (free once the sums of sub-tile
-            //      i - 2 are complete)
-            if (i >= 2) ok = ptx::mbar_wait(&pv_done[i & 1], ((i >> 1) - 1) & 1, abort_flag) && ok;
-            {
-                uint8_t* dst = p_buf + (i & 1) * kTcOperand + tok_low;
+                // ---- hand-over to group B (the buffers of sub-tile i - 2 have been read)
+                if (i >= 2) ok = ptx::mbar_wait(&xy_free[i & 1], ((i >> 1) - 1) & 1, abort_flag) && ok;
+                float* eb = e_buf + (i & 1) * (2 * 8 * kTcT) + token;
 #pragma unroll
                 for (int g = 0; g < 8; ++g) {
                     if (mine[g]) {
-                        const float w = tc_ex2(y[g] - m_sub[g]) * kTcWeightScale;
-                        l_thr[g] += tc_ex2(x[g] - m_sub[g]);
-                        const uint32_t hi = ptx::cvt_e4m3x2(w, 0.f);
-                        const uint32_t lo = ptx::cvt_e4m3x2(w - ptx::e4m3x2_to_f32(hi).x, 0.f);
-                        // rows 2 g and 2 g + 1 of the operand, byte `token` (128-byte swizzle)
-                        dst[(2 * g) * 128 + ((tok_swz ^ ((2 * g) & 7)) << 4)] = (uint8_t)hi;
-                        dst[(2 * g + 1) * 128 + ((tok_swz ^ ((2 * g + 1) & 7)) << 4)] = (uint8_t)lo;
+                        eb[g * kTcT] = y[g] - m_sub[g];
+                        eb[(8 + g) * kTcT] = x[g] - m_sub[g];
                     }
                 }
-            }
-            ptx::fence_proxy_async_smem();      // the weights and the cleared rows, before the tensor pipe reads them
-            ptx::tc_fence_before_sync();
-            __syncwarp();
-            if (lane == 0) ptx::mbar_arrive(&p_ready[i & 1]);
-            first = false;
-
-            // ---- the last sub-tile of the sequence in this range: its partial result goes to slot cta + b
-            const bool last = (i + 1 == n_sub) || (k + 1 >= n_sub_b);
-            if (last) {
-                ok = ptx::mbar_wait(&pv_done[i & 1], (i >> 1) & 1, abort_flag) && ok;
-                ptx::tc_fence_after_sync();
-                const size_t slot = (size_t)cta + b;
+                if (gtid < 8) {
+                    float a = 1.f, m = -INFINITY;
 #pragma unroll
-                for (int c = 0; c < CH; ++c) {
-                    uint32_t r[16];
-                    ptx::tmem_ld16(tmem_o + c * 16, r);
-                    ptx::tmem_wait_ld();
-#pragma unroll
-                    for (int g = 0; g < 8; ++g)
-                        if (g < NQ)     // both pieces, the weights' factor taken out
-                            part_o[(slot * NQ + g) * d.d_l + c * 128 + warp * 32 + lane] =
-                                (__uint_as_float(r[2 * g]) + __uint_as_float(r[2 * g + 1])) * (1.f / kTcWeightScale);
+                    for (int g = 0; g < 8; ++g) if (g == gtid) { a = alpha[g]; m = m_run[g]; }
+                    hdr[(i & 1) * 24 + gtid] = a;
+                    hdr[(i & 1) * 24 + 8 + gtid] = m;
+                    if (gtid == 0) hdr[(i & 1) * 24 + 16] = grow ? 1.f : 0.f;
                 }
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(&xy_ready[i & 1]);
+                first = false;
+            }
+        } else {
+            float l_thr[8], m_cur[8];
+#pragma unroll
+            for (int g = 0; g < 8; ++g) { l_thr[g] = 0.f; m_cur[g] = -INFINITY; }
+            for (int i = 0; i < n_sub; ++i, ++k) {
+                if (k >= n_sub_b) {
+                    do { ++b; } while (prefix[b + 1] == prefix[b]);
+                    k = 0;
+                    first = true;
+                    len_b = tc_len(seq_lens, b, S_cap);
+                    n_sub_b = prefix[b + 1] - prefix[b];
+                }
+                const int s = i % kTcStages;
+                const int n_valid = min(kTcT, len_b - k * kTcT);
+                uint8_t* stage = ring + s * lay.stage_stride;
+                ok = ptx::mbar_wait(&xy_ready[i & 1], (i >> 1) & 1, abort_flag) && ok;
+                float alpha[8];
+#pragma unroll
+                for (int g = 0; g < 8; ++g) {
+                    alpha[g] = g < NQ ? hdr[(i & 1) * 24 + g] : 1.f;
+                    m_cur[g] = g < NQ ? hdr[(i & 1) * 24 + 8 + g] : -INFINITY;
+                    l_thr[g] *= alpha[g];
+                }
+                const bool grow = hdr[(i & 1) * 24 + 16] != 0.f;
+                float ew[8], el[8];
+                const float* eb = e_buf + (i & 1) * (2 * 8 * kTcT) + token;
+#pragma unroll
+                for (int g = 0; g < 8; ++g) {
+                    ew[g] = el[g] = -INFINITY;
+                    if (mine[g]) { ew[g] = eb[g * kTcT]; el[g] = eb[(8 + g) * kTcT]; }
+                }
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(&xy_free[i & 1]);
+
+                // ---- rows past the live length hold whatever the cache holds there (NaN codes included): their
+                //      weights are zero, so the latent rows are cleared
+                if (n_valid < kTcT) {
+                    ok = ptx::mbar_wait(&full_bar[s], (i / kTcStages) & 1, abort_flag) && ok;
+                    const int n_vec = (kTcT - n_valid) * CH * 8;
+                    for (int idx = gtid; idx < n_vec; idx += 128) {
+                        const int row = n_valid + idx / (CH * 8), v = idx % (CH * 8);
+                        *reinterpret_cast<uint4*>(stage + (NK + (v >> 3)) * kTcTile + row * 128 + (v & 7) * 16) =
+                            make_uint4(0u, 0u, 0u, 0u);
+                    }
+                }
+                // ---- the sums so far are rescaled when a maximum has grown (the first sub-tile of a sequence
+                //      overwrites them)
+                if (grow && !first) {       // uniform over the group
+                    ok = ptx::mbar_wait(&pv_done[(i - 1) & 1], ((i - 1) >> 1) & 1, abort_flag) && ok;
+                    ptx::tc_fence_after_sync();
+#pragma unroll
+                    for (int c = 0; c < CH; ++c) {
+                        uint32_t r[16];
+                        ptx::tmem_ld16(tmem_o + c * 16, r);
+                        ptx::tmem_wait_ld();
+#pragma unroll
+                        for (int e = 0; e < 16; ++e) r[e] = __float_as_uint(__uint_as_float(r[e]) * alpha[e >> 1]);
+                        ptx::tmem_st16(tmem_o + c * 16, r);
+                    }
+                    ptx::tmem_wait_st();
+                }
+                // ---- the weights' pieces of this token into the B operand of the sums (free once the sums of
+                //      sub-tile i - 2 are complete)
+                if (i >= 2) ok = ptx::mbar_wait(&pv_done[i & 1], ((i >> 1) - 1) & 1, abort_flag) && ok;
                 {
+                    uint8_t* dst = p_buf + (i & 1) * kTcOperand + tok_low;
+#pragma unroll
+                    for (int g = 0; g < 8; ++g) {
+                        if (mine[g]) {
+                            const float w = tc_ex2(ew[g]) * kTcWeightScale;
+                            l_thr[g] += tc_ex2(el[g]);
+                            const uint32_t hi = ptx::cvt_e4m3x2(w, 0.f);
+                            const uint32_t lo = ptx::cvt_e4m3x2(w - ptx::e4m3x2_to_f32(hi).x, 0.f);
+                            // rows 2 g and 2 g + 1 of the operand, byte `token` (128-byte swizzle)
+                            dst[(2 * g) * 128 + ((tok_swz ^ ((2 * g) & 7)) << 4)] = (uint8_t)hi;
+                            dst[(2 * g + 1) * 128 + ((tok_swz ^ ((2 * g + 1) & 7)) << 4)] = (uint8_t)lo;
+                        }
+                    }
+                }
+                ptx::fence_proxy_async_smem();      // the weights and the cleared rows, before the tensor pipe reads them
+                ptx::tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(&p_ready[i & 1]);
+                first = false;
+
+                // ---- the last sub-tile of the sequence in this range: its partial result goes to slot cta + b
+                const bool last = (i + 1 == n_sub) || (k + 1 >= n_sub_b);
+                if (last) {
+                    ok = ptx::mbar_wait(&pv_done[i & 1], (i >> 1) & 1, abort_flag) && ok;
+                    ptx::tc_fence_after_sync();
+                    const size_t slot = (size_t)cta + b;
+#pragma unroll
+                    for (int c = 0; c < CH; ++c) {
+                        uint32_t r[16];
+                        ptx::tmem_ld16(tmem_o + c * 16, r);
+                        ptx::tmem_wait_ld();
+#pragma unroll
+                        for (int g = 0; g < 8; ++g)
+                            if (g < NQ)     // both pieces, the weights' factor taken out
+                                part_o[(slot * NQ + g) * d.d_l + c * 128 + quarter * 32 + lane] =
+                                    (__uint_as_float(r[2 * g]) + __uint_as_float(r[2 * g + 1])) * (1.f / kTcWeightScale);
+                    }
 #pragma unroll
                     for (int g = 0; g < 8; ++g) {
                         if (mine[g]) {
                             float v = l_thr[g];
 #pragma unroll
                             for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-                            if (lane == 0) l_red[warp * 8 + g] = v;
+                            if (lane == 0) l_red[quarter * 8 + g] = v;
                         }
                     }
-                }
-                tc_group_sync();
-                if (tid < NQ) {
-                    float mg = -INFINITY;
+                    asm volatile("bar.sync 2, 128;" ::: "memory");
+                    if (gtid < NQ) {
+                        float mg = -INFINITY;
 #pragma unroll
-                    for (int g = 0; g < 8; ++g) if (g == tid) mg = m_run[g];
-                    part_ml[(slot * NQ + tid) * 2] = mg;
-                    const int w0 = 2 * ((tid / qpk) & 1);      // the two warps that hold map tid's row-sum shares
-                    part_ml[(slot * NQ + tid) * 2 + 1] = l_red[w0 * 8 + tid] + l_red[(w0 + 1) * 8 + tid];
-                }
+                        for (int g = 0; g < 8; ++g) if (g == gtid) mg = m_cur[g];
+                        const int w0 = 2 * ((gtid / qpk) & 1);      // the two warps that hold map gtid's row-sum shares
+                        part_ml[(slot * NQ + gtid) * 2] = mg;
+                        part_ml[(slot * NQ + gtid) * 2 + 1] = l_red[w0 * 8 + gtid] + l_red[(w0 + 1) * 8 + gtid];
+                    }
 #pragma unroll
-                for (int g = 0; g < 8; ++g) { m_run[g] = -INFINITY; l_thr[g] = 0.f; }
-                ptx::tc_fence_before_sync();
+                    for (int g = 0; g < 8; ++g) l_thr[g] = 0.f;
+                    ptx::tc_fence_before_sync();
+                }
             }
         }
         (void)ok;
     }
     ptx::tc_fence_before_sync();
     __syncthreads();
-    if (warp == 5) ptx::tmem_dealloc(tmem_base, kTcTmemCols);
+    if (warp == 9) ptx::tmem_dealloc(tmem_base, kTcTmemCols);
     if (tid == 0 && *abort_flag) raise_status(status_word, GTA_ERR_TIMEOUT);
 }
 
 }  // namespace
 
-// d_h = 128, one latent group, d_l = 128, 256 or 512, at most four key groups, sub-tiles of 64 tokens that fit the ring
+// d_h = 128, one latent group, d_l = 128, 256 or 512, 1, 2 or 4 key groups with 1, 2, 4 or 8 maps each (at most 8
+// maps), sub-tiles of 64 tokens that fit the ring
 bool decode_fp8_tc_supported(const Dims& d, int T) {
-    if (T != kTcT || d.d_h != 128 || d.n_c != 1 || d.n_k > 4 || d.n_q > 8 || d.B > kTcMaxBatch) return false;
+    if (T != kTcT || d.d_h != 128 || d.n_c != 1 || d.n_q > 8 || d.B > kTcMaxBatch) return false;
+    if (d.n_k != 1 && d.n_k != 2 && d.n_k != 4) return false;
+    const int qpk = d.n_q / d.n_k;
+    if (qpk != 1 && qpk != 2 && qpk != 4 && qpk != 8) return false;
     if (d.d_l != 128 && d.d_l != 256 && d.d_l != 512) return false;
     return tc_smem_layout(d.n_k, d.d_l / 128).total <= 232448u;
 }
+
+namespace {
+template <int CH, int NK, int QPK>
+cudaError_t launch_tc(const CUtensorMap& tm_k, const CUtensorMap& tm_c, const Dims& d, int G, int S_cap, const void* q,
+                      const float* k_scale, const float* c_scale, const int32_t* seq_lens, float* part_o, float* part_ml,
+                      int32_t* status_word, cudaStream_t stream) {
+    auto kern = decode_stream_fp8_tc_kernel<CH, NK, QPK>;
+    const size_t smem = tc_smem_layout(NK, CH).total;
+    cudaError_t err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (err != cudaSuccess) return err;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(G);
+    cfg.blockDim = dim3(kTcThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kern, tm_k, tm_c, d, S_cap, (const __nv_bfloat16*)q, k_scale, c_scale, seq_lens, part_o,
+                              part_ml, status_word);
+}
+template <int CH>
+cudaError_t launch_tc_groups(const CUtensorMap& tm_k, const CUtensorMap& tm_c, const Dims& d, int G, int S_cap,
+                             const void* q, const float* k_scale, const float* c_scale, const int32_t* seq_lens,
+                             float* part_o, float* part_ml, int32_t* status_word, cudaStream_t stream) {
+#define GTA_TC_CASE(NKV, QPKV)                                                                                     \
+    if (d.n_k == NKV && d.n_q == NKV * QPKV)                                                                       \
+        return launch_tc<CH, NKV, QPKV>(tm_k, tm_c, d, G, S_cap, q, k_scale, c_scale, seq_lens, part_o, part_ml,   \
+                                        status_word, stream)
+    GTA_TC_CASE(1, 1); GTA_TC_CASE(1, 2); GTA_TC_CASE(1, 4); GTA_TC_CASE(1, 8);
+    GTA_TC_CASE(2, 1); GTA_TC_CASE(2, 2); GTA_TC_CASE(2, 4);
+    GTA_TC_CASE(4, 1); GTA_TC_CASE(4, 2);
+#undef GTA_TC_CASE
+    return cudaErrorInvalidValue;
+}
+}  // namespace
 
 cudaError_t launch_decode_fp8_tc_stream(const Dims& d, int G, int S_cap, const void* q, const void* k_codes,
                                         const void* c_codes, const float* k_scale, const float* c_scale,
@@ -532,34 +655,13 @@ cudaError_t launch_decode_fp8_tc_stream(const Dims& d, int G, int S_cap, const v
     const uint64_t dk[3] = {128, (uint64_t)S_cap, (uint64_t)d.B * d.n_k};
     const uint64_t dc[3] = {(uint64_t)d.d_l, (uint64_t)S_cap, (uint64_t)d.B};
     if (!make_u8_map(&tm_k, k_codes, 3, dk, box) || !make_u8_map(&tm_c, c_codes, 3, dc, box)) return cudaErrorInvalidValue;
-    const int CH = d.d_l / 128;
-    const size_t smem = tc_smem_layout(d.n_k, CH).total;
     cudaError_t err;
-#define GTA_LAUNCH_FP8_TC(CHV)                                                                             \
-    do {                                                                                                   \
-        auto kern = decode_stream_fp8_tc_kernel<CHV>;                                                      \
-        err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);          \
-        if (err != cudaSuccess) return err;                                                                \
-        cudaLaunchConfig_t cfg = {};                                                                       \
-        cfg.gridDim = dim3(G);                                                                             \
-        cfg.blockDim = dim3(kTcThreads);                                                                   \
-        cfg.dynamicSmemBytes = smem;                                                                       \
-        cfg.stream = stream;                                                                               \
-        cudaLaunchAttribute attr[1];                                                                       \
-        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;                                   \
-        attr[0].val.programmaticStreamSerializationAllowed = 1;                                            \
-        cfg.attrs = attr;                                                                                  \
-        cfg.numAttrs = 1;                                                                                  \
-        err = cudaLaunchKernelEx(&cfg, kern, tm_k, tm_c, d, S_cap, (const __nv_bfloat16*)q, k_scale, c_scale, \
-                                 seq_lens, part_o, part_ml, status_word);                                  \
-        if (err != cudaSuccess) return err;                                                                \
-    } while (0)
-    switch (CH) {
-        case 1: GTA_LAUNCH_FP8_TC(1); break;
-        case 2: GTA_LAUNCH_FP8_TC(2); break;
-        default: GTA_LAUNCH_FP8_TC(4); break;
+    switch (d.d_l / 128) {
+        case 1: err = launch_tc_groups<1>(tm_k, tm_c, d, G, S_cap, q, k_scale, c_scale, seq_lens, part_o, part_ml, status_word, stream); break;
+        case 2: err = launch_tc_groups<2>(tm_k, tm_c, d, G, S_cap, q, k_scale, c_scale, seq_lens, part_o, part_ml, status_word, stream); break;
+        default: err = launch_tc_groups<4>(tm_k, tm_c, d, G, S_cap, q, k_scale, c_scale, seq_lens, part_o, part_ml, status_word, stream); break;
     }
-#undef GTA_LAUNCH_FP8_TC
+    if (err != cudaSuccess) return err;
     return cudaGetLastError();
 }
 
