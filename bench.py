@@ -51,7 +51,7 @@ KERNEL_SOURCES = {
     "prefill_attention": "paper_2506_17286_b200/csrc/gta_sm100.cu",
     "prefill_decoder_gate": "paper_2506_17286_b200/csrc/gta_sm100_decoder.cu",
     "decode_stream": "paper_2506_17286_b200/csrc/gta_decode_sm100.cu",
-    "decode_stream_fp8": "paper_2506_17286_b200/csrc/gta_decode_sm100.cu",
+    "decode_stream_fp8": "paper_2506_17286_b200/csrc/gta_decode_fp8_tc.cu",
 }
 
 
@@ -797,8 +797,8 @@ def run_ours(args):
         nbytes = cache_bytes + by["weights"] + by["vectors"]
         r = hbm_roofline(nbytes, t8, peaks, rec8["clocks"],
                          note="gta_decode_fp8 back to back, two cache sets alternating; bytes = codes + scales of the live "
-                              "rows + weights + vectors; streaming kernel with warp-level e4m3 MMAs, paced by its consumer "
-                              "warps (those MMAs are carried out as f16 MMAs behind operand conversions on this architecture)")
+                              "rows + weights + vectors; tcgen05 streaming kernel (kind::f8f6f4, the cached tokens on the rows "
+                              "of the MMAs), then the merge and decoder kernels of the bf16 step")
         r["path"] = G.decode_fp8_path(shape_d, ctx + 64)
         tr = traffic.get(("decode_stream_fp8", "c3"))
         r["traffic"] = tr["bytes"] if tr else None

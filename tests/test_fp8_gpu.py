@@ -55,10 +55,12 @@ def test_quantising_append_is_bit_exact(B, oracle, dt, n_new):
             assert np.array_equal(g_, ref), what
 
 
-def _decode_case(B, oracle, w, lens, sample=None, cap=None, path=None):
+def _decode_case(B, oracle, w, lens, sample=None, cap=None, path=None, reshape_keys=None):
     nb = w.batch
     cap = cap or max(lens) + 7
     t = I.decode_inputs(w, device="cuda", s_cap=cap, seq_lens=lens)
+    if reshape_keys is not None:
+        reshape_keys(t)
     kq, ks = oracle.quantize_rows_e4m3(t["k_cache"].cpu())
     cq, cs = oracle.quantize_rows_e4m3(t["c_cache"].cpu())
     for b, n in enumerate(lens):                          # what uninitialised memory may hold behind the live rows
@@ -107,6 +109,14 @@ FP8_STREAM = [
     ("dl256_empty_sequences_shared_keys", 6, 256, 8, 4, 2, 256, [0, 512, 1, 0, 300, 33], 512),
     ("one_map_full_cache", 2, 128, 2, 1, 1, 256, [256, 255], 256),
     ("many_sequences", 150, 256, 8, 4, 4, 512, [((7 * i) % 130) for i in range(150)], 132),
+    # the remaining (key groups, maps per group) instantiations of the tensor-memory kernel
+    ("eight_maps_one_key_group_dl128", 4, 256, 8, 8, 1, 128, [640, 64, 129, 1], 640),
+    ("eight_maps_two_key_groups_dl256", 3, 256, 8, 8, 2, 256, [500, 0, 191], 512),
+    ("eight_maps_four_key_groups_dl512", 3, 256, 8, 8, 4, 512, [320, 65, 128], 320),
+    ("two_maps_two_key_groups_dl128", 5, 128, 4, 2, 2, 128, [1, 2, 63, 300, 64], 304),
+    ("two_maps_one_key_group_dl512", 2, 128, 4, 2, 1, 512, [200, 450], 452),
+    ("four_maps_one_key_group_dl256", 3, 128, 8, 4, 1, 256, [1000, 7, 128], 1000),
+    ("long_sequences_many_subtiles_per_cta", 2, 256, 8, 4, 4, 512, [20000, 12345], 20000),
 ]
 
 
@@ -116,6 +126,25 @@ def test_fp8_decode_streaming_kernels(B, oracle, case):
     w = I.Workload(name, "decode", "bf16", nb, 0, H, n_h, n_q, n_k, 1, 128, d_l, seed=63)
     rel, mx = _decode_case(B, oracle, w, lens, cap=cap, path=2)
     print(f"\n{name}: rel-L2 {rel:.3e} max-abs {mx:.3e}")
+
+
+@pytest.mark.parametrize("slope", [0.002, 0.02, -0.004])
+def test_fp8_decode_scores_that_keep_rising_or_falling(B, oracle, slope):
+    """Keys that point along their map's query with a length that grows (or shrinks) with the position: the reference
+    maximum of the softmax is raised at almost every sub-tile (slope 0.002: by about two binary orders per sub-tile,
+    0.02: by twenty) or set once and never again (negative slope), so the rescaling of the sums kept in tensor memory,
+    the lag of the reference and weights that underflow are all exercised."""
+    w = I.Workload("rising", "decode", "bf16", 3, 0, 256, 8, 4, 4, 1, 128, 512, seed=64)
+    lens = [1000, 700, 130]
+
+    def keys_along_queries(t):
+        q = t["q"].float()                                   # [B, n_q, d_h]; one map per key group here
+        pos = torch.arange(t["k_cache"].shape[2], device=q.device, dtype=torch.float32)
+        length = slope * pos if slope > 0 else 4.0 + slope * pos
+        noise = t["k_cache"].float() * 0.05
+        t["k_cache"].copy_((q[:, :, None, :] * length[None, None, :, None] + noise).to(t["k_cache"].dtype))
+    rel, mx = _decode_case(B, oracle, w, lens, cap=1000, path=2, reshape_keys=keys_along_queries)
+    print(f"\nslope {slope}: rel-L2 {rel:.3e} max-abs {mx:.3e}")
 
 
 def test_fp8_decode_config3_shape_sampled_sequences(B, oracle):
