@@ -222,6 +222,14 @@ SMALL_DECODE = [
     ("bf16_shared_keys_two_latents", "bf16", 3, 128, 8, 4, 2, 2, 64, 128, [200, 5, 129]),
     ("bf16_paper_1b_shape", "bf16", 2, 1280, 20, 5, 1, 1, 64, 128, [333, 1000]),
     ("bf16_eight_maps", "bf16", 9, 512, 16, 8, 8, 1, 128, 1024, [257, 256, 255, 1, 2, 1000, 64, 128, 511]),
+    # the other (sub-tile, key groups, maps per group) instantiations of the tensor-memory stream kernel
+    ("bf16_eight_maps_four_key_groups_dl512", "bf16", 4, 256, 16, 8, 4, 1, 128, 512, [700, 31, 32, 33]),
+    ("bf16_four_maps_two_key_groups_dl512", "bf16", 5, 256, 8, 4, 2, 1, 128, 512, [1, 450, 0, 96, 65]),
+    ("bf16_four_maps_one_key_group_dl512", "bf16", 3, 256, 8, 4, 1, 1, 128, 512, [500, 64, 17]),
+    ("bf16_eight_maps_four_key_groups_dl1024", "bf16", 4, 256, 16, 8, 4, 1, 128, 1024, [300, 15, 16, 17]),
+    ("bf16_eight_maps_two_key_groups_dl1024", "bf16", 3, 256, 16, 8, 2, 1, 128, 1024, [1, 129, 48]),
+    ("bf16_eight_maps_one_key_group_dl1024", "bf16", 3, 256, 8, 8, 1, 1, 128, 1024, [200, 0, 33]),
+    ("bf16_long_sequences_many_sub_tiles_per_cta", "bf16", 2, 256, 8, 4, 4, 1, 128, 512, [20000, 12345]),
     ("f32_general", "f32", 3, 96, 6, 6, 3, 1, 32, 64, [100, 7, 260]),
     # more than 16 sequences: the finish goes through the merge kernel + the tensor-core decoder kernel
     # (without CTA pairs up to 128 sequences, with them above)
@@ -530,6 +538,10 @@ STEP_CASES = [
     ("bf16_two_latents_dh64", "bf16", 128, 8, 4, 2, 2, 64, 128, [200, 0, 129, 63, 64], 256),
     ("bf16_paper_1b_shape", "bf16", 1280, 20, 5, 1, 1, 64, 128, [333, 127, 128], 400),
     ("bf16_batch_40", "bf16", 256, 8, 4, 4, 1, 128, 512, [(37 * i) % 300 for i in range(40)], 320),
+    # 16-token sub-tiles (eight key groups on the rows of one MMA), lengths around them, a full cache
+    ("bf16_eight_key_groups_dl1024", "bf16", 512, 16, 8, 8, 1, 128, 1024, [0, 1, 14, 15, 16, 17, 31, 32, 300, 304], 304),
+    ("bf16_two_maps_per_key_group_dl512", "bf16", 256, 16, 8, 4, 1, 128, 512, [95, 96, 97, 0, 640], 641),
+    ("bf16_one_key_group_dl1024", "bf16", 256, 8, 8, 1, 1, 128, 1024, [47, 48, 200], 208),
     ("f32_plain_alu_kernels", "f32", 96, 6, 6, 3, 1, 32, 64, [100, 7, 0, 260], 261),
 ]
 
