@@ -50,7 +50,7 @@ MIN_TIMED_MS = 500.0     # device time every timed loop is repeated up to, whate
 KERNEL_SOURCES = {
     "prefill_attention": "paper_2506_17286_b200/csrc/gta_sm100.cu",
     "prefill_decoder_gate": "paper_2506_17286_b200/csrc/gta_sm100_decoder.cu",
-    "decode_stream": "paper_2506_17286_b200/csrc/gta_decode_sm100.cu",
+    "decode_stream": "paper_2506_17286_b200/csrc/gta_decode_tc.cu",
     "decode_stream_fp8": "paper_2506_17286_b200/csrc/gta_decode_fp8_tc.cu",
 }
 

@@ -599,10 +599,10 @@ static cudaError_t launch_stream_and_merge(const Dims& d, const FastPlan& p, con
                                            int* launches, const PageMap& pm, const void* k_new = nullptr,
                                            const void* c_new = nullptr) {
     cudaError_t err;
-    if ((stages & 2) && decode_tc_supported(d, p.T, p.occ, pm.table != nullptr)) {
+    if ((stages & 2) && decode_tc_supported(d, p.T, p.occ, pm.table ? pm.page_size : 0)) {
         // the cached tokens as the rows of tcgen05 MMAs (gta_decode_tc.cu)
         err = launch_decode_tc_stream(d, p.G, p.T, S_cap, q, k_cache, c_cache, seq_lens, part_o, part_ml, status_word,
-                                      stream, k_new, c_new);
+                                      stream, k_new, c_new, pm);
         if (err != cudaSuccess) return err;
         *launches += 1;
     } else if (stages & 2) {

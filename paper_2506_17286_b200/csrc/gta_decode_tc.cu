@@ -88,7 +88,7 @@ decode_stream_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_c
                         int S_cap, const __nv_bfloat16* __restrict__ q, const int32_t* __restrict__ seq_lens,
                         float* __restrict__ part_o, float* __restrict__ part_ml, int32_t* status_word,
                         const uint4* __restrict__ k_new, const uint4* __restrict__ c_new, uint4* __restrict__ k_rows,
-                        uint4* __restrict__ c_rows) {
+                        uint4* __restrict__ c_rows, const PageMap pm) {
     constexpr int NQ = NK * QPK;
     constexpr int R = 128 / T;                        // key groups on the rows of one score MMA
     constexpr int SETS = (NK + R - 1) / R;
@@ -206,7 +206,16 @@ decode_stream_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_c
             while (k >= prefix[b + 1] - prefix[b]) { ++b; k = 0; }
             const int s = it % kBtStages;
             const uint32_t ph = (it / kBtStages) & 1;
-            const int tok0 = k * T;
+            // Contiguous caches: rows tok0 .. of plane b groups + g.  Paged pool: the sub-tile lies inside one page
+            // (T divides the page size), at rows tok0 % page_size .. of plane page groups + g; the block-table entry
+            // is fetched before the wait for the stage.  An entry outside the pool raises the status word, and the
+            // load (of page 0 then) still completes the stage.
+            int tok0 = k * T, plane = b;
+            if (pm.table != nullptr) {
+                const int page = page_of(pm, b, tok0, lane == 0 ? status_word : nullptr);
+                plane = page < 0 ? 0 : page;
+                tok0 %= pm.page_size;
+            }
             if (lane == 0) {
                 ok = ptx::mbar_wait(&empty_bar[s], ph ^ 1, abort_flag);
                 if (ok) ptx::mbar_arrive_expect_tx(&full_bar[s], (uint32_t)n_ops * tb);
@@ -216,9 +225,9 @@ decode_stream_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_c
             uint8_t* stage = ring + s * lay.stage_stride;
             for (int op = lane; op < n_ops; op += 32) {
                 if (op < 2 * NK)        // half op / NK of key group op % NK
-                    ptx::tma_load_3d_hint(stage + op * tb, &tm_k, &full_bar[s], (op / NK) * 64, tok0, b * NK + op % NK, policy);
+                    ptx::tma_load_3d_hint(stage + op * tb, &tm_k, &full_bar[s], (op / NK) * 64, tok0, plane * NK + op % NK, policy);
                 else
-                    ptx::tma_load_3d_hint(stage + op * tb, &tm_c, &full_bar[s], (op - 2 * NK) * 64, tok0, b, policy);
+                    ptx::tma_load_3d_hint(stage + op * tb, &tm_c, &full_bar[s], (op - 2 * NK) * 64, tok0, plane, policy);
             }
         }
         if (lane == 0 && *abort_flag) {
@@ -610,7 +619,7 @@ decode_stream_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_c
 template <int T, int NK, int QPK, int CH>
 cudaError_t launch_bt(const CUtensorMap& tm_k, const CUtensorMap& tm_c, const Dims& d, int G, int S_cap, const void* q,
                       const int32_t* seq_lens, float* part_o, float* part_ml, int32_t* status_word, cudaStream_t stream,
-                      const void* k_new, const void* c_new, void* k_cache, void* c_cache) {
+                      const void* k_new, const void* c_new, void* k_cache, void* c_cache, const PageMap& pm) {
     auto kern = decode_stream_tc_kernel<T, NK, QPK, CH>;
     const size_t smem = bt_smem_layout(T, NK, CH).total;
     cudaError_t err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
@@ -626,7 +635,7 @@ cudaError_t launch_bt(const CUtensorMap& tm_k, const CUtensorMap& tm_c, const Di
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     return cudaLaunchKernelEx(&cfg, kern, tm_k, tm_c, d, S_cap, (const __nv_bfloat16*)q, seq_lens, part_o, part_ml,
-                              status_word, (const uint4*)k_new, (const uint4*)c_new, (uint4*)k_cache, (uint4*)c_cache);
+                              status_word, (const uint4*)k_new, (const uint4*)c_new, (uint4*)k_cache, (uint4*)c_cache, pm);
 }
 
 // the instantiations: (sub-tile, key groups, maps per group, 128-column latent blocks)
@@ -636,9 +645,10 @@ cudaError_t launch_bt(const CUtensorMap& tm_k, const CUtensorMap& tm_c, const Di
 
 }  // namespace
 
-// d_h = 128, one latent group, contiguous caches, one CTA per SM, and one of the instantiated shapes
-bool decode_tc_supported(const Dims& d, int T, int occ, bool paged) {
-    if (paged || occ != 1 || d.d_h != 128 || d.n_c != 1 || d.B > kBtMaxBatch) return false;
+// d_h = 128, one latent group, one CTA per SM, one of the instantiated shapes; a paged pool's pages hold whole sub-tiles
+bool decode_tc_supported(const Dims& d, int T, int occ, int page_size) {
+    if (occ != 1 || d.d_h != 128 || d.n_c != 1 || d.B > kBtMaxBatch) return false;
+    if (page_size % T != 0) return false;
     const int ch = d.d_l / 128, qpk = d.n_k > 0 ? d.n_q / d.n_k : 0;
     if (d.d_l % 128 != 0) return false;
 #define GTA_BT_MATCH(TV, NKV, QPKV, CHV) if (T == TV && d.n_k == NKV && qpk == QPKV && ch == CHV) return true;
@@ -649,11 +659,15 @@ bool decode_tc_supported(const Dims& d, int T, int occ, bool paged) {
 
 cudaError_t launch_decode_tc_stream(const Dims& d, int G, int T, int S_cap, const void* q, const void* k_cache,
                                     const void* c_cache, const int32_t* seq_lens, float* part_o, float* part_ml,
-                                    int32_t* status_word, cudaStream_t stream, const void* k_new, const void* c_new) {
+                                    int32_t* status_word, cudaStream_t stream, const void* k_new, const void* c_new,
+                                    const PageMap& pm) {
     CUtensorMap tm_k, tm_c;
     const uint32_t box[3] = {64, (uint32_t)T, 1};
-    const uint64_t dk[3] = {(uint64_t)d.d_h, (uint64_t)S_cap, (uint64_t)d.B * d.n_k};
-    const uint64_t dc[3] = {(uint64_t)d.d_l, (uint64_t)S_cap, (uint64_t)d.B};
+    // planes of rows: one per (sequence, group), S_cap rows each -- or one per (page, group), page_size rows
+    const uint64_t rows = pm.table ? (uint64_t)pm.page_size : (uint64_t)S_cap;
+    const uint64_t outer = pm.table ? (uint64_t)pm.n_pages : (uint64_t)d.B;
+    const uint64_t dk[3] = {(uint64_t)d.d_h, rows, outer * d.n_k};
+    const uint64_t dc[3] = {(uint64_t)d.d_l, rows, outer};
     if (!make_bf16_map(&tm_k, k_cache, 3, dk, box) || !make_bf16_map(&tm_c, c_cache, 3, dc, box))
         return cudaErrorInvalidValue;
     const int ch = d.d_l / 128, qpk = d.n_q / d.n_k;
@@ -661,7 +675,7 @@ cudaError_t launch_decode_tc_stream(const Dims& d, int G, int T, int S_cap, cons
 #define GTA_BT_LAUNCH(TV, NKV, QPKV, CHV)                                                                          \
     if (T == TV && d.n_k == NKV && qpk == QPKV && ch == CHV)                                                       \
         err = launch_bt<TV, NKV, QPKV, CHV>(tm_k, tm_c, d, G, S_cap, q, seq_lens, part_o, part_ml, status_word,    \
-                                            stream, k_new, c_new, const_cast<void*>(k_cache), const_cast<void*>(c_cache));
+                                            stream, k_new, c_new, const_cast<void*>(k_cache), const_cast<void*>(c_cache), pm);
     GTA_BT_SHAPES(GTA_BT_LAUNCH)
 #undef GTA_BT_LAUNCH
     if (err != cudaSuccess) return err;

@@ -66,9 +66,10 @@ cudaError_t launch_decode_fp8_tc_stream(const Dims& d, int G, int S_cap, const v
 // The stream kernel of a decode step over bf16 caches on the tcgen05 tensor pipe (gta_decode_tc.cu): same schedule
 // (G CTAs, sub-tiles of T tokens), step lengths and partial results as decode_stream_kernel; k_new / c_new != nullptr:
 // the fused append + decode step.
-bool decode_tc_supported(const Dims& d, int T, int occ, bool paged);
+bool decode_tc_supported(const Dims& d, int T, int occ, int page_size);
 cudaError_t launch_decode_tc_stream(const Dims& d, int G, int T, int S_cap, const void* q, const void* k_cache,
                                     const void* c_cache, const int32_t* seq_lens, float* part_o, float* part_ml,
-                                    int32_t* status_word, cudaStream_t stream, const void* k_new, const void* c_new);
+                                    int32_t* status_word, cudaStream_t stream, const void* k_new, const void* c_new,
+                                    const PageMap& pm);
 
 }  // namespace gta
