@@ -117,6 +117,8 @@ FP8_STREAM = [
     ("two_maps_one_key_group_dl512", 2, 128, 4, 2, 1, 512, [200, 450], 452),
     ("four_maps_one_key_group_dl256", 3, 128, 8, 4, 1, 256, [1000, 7, 128], 1000),
     ("long_sequences_many_subtiles_per_cta", 2, 256, 8, 4, 4, 512, [20000, 12345], 20000),
+    ("batch_400_many_empty", 400, 256, 8, 4, 4, 512, [0 if i % 7 == 3 else 1 + (13 * i) % 70 for i in range(400)], 72),
+    ("all_sequences_empty", 6, 256, 8, 4, 4, 512, [0, 0, 0, 0, 0, 0], 64),
 ]
 
 

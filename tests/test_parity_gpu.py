@@ -230,6 +230,10 @@ SMALL_DECODE = [
     ("bf16_eight_maps_two_key_groups_dl1024", "bf16", 3, 256, 16, 8, 2, 1, 128, 1024, [1, 129, 48]),
     ("bf16_eight_maps_one_key_group_dl1024", "bf16", 3, 256, 8, 8, 1, 1, 128, 1024, [200, 0, 33]),
     ("bf16_long_sequences_many_sub_tiles_per_cta", "bf16", 2, 256, 8, 4, 4, 1, 128, 512, [20000, 12345]),
+    # more sequences than the stream kernel has threads (the prefix sum takes two per thread), many of them empty;
+    # and a batch with nothing cached at all (no CTA has a sub-tile)
+    ("bf16_batch_400_c3_grouping", "bf16", 400, 256, 8, 4, 4, 1, 128, 512, [0 if i % 7 == 3 else 1 + (13 * i) % 70 for i in range(400)]),
+    ("bf16_all_sequences_empty_c3_grouping", "bf16", 6, 256, 8, 4, 4, 1, 128, 512, [0, 0, 0, 0, 0, 0]),
     ("f32_general", "f32", 3, 96, 6, 6, 3, 1, 32, 64, [100, 7, 260]),
     # more than 16 sequences: the finish goes through the merge kernel + the tensor-core decoder kernel
     # (without CTA pairs up to 128 sequences, with them above)
