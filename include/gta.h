@@ -499,6 +499,16 @@ GTA_API int gta_last_launch_count(void);
  */
 GTA_API gta_status_t gta_debug_attention_wait(uint64_t limit_ns, int32_t withhold_first_arrive);
 
+/*
+ * The same test hook for the two decode stream kernels that keep their sums in tensor memory (bf16 caches and 8-bit
+ * caches; App. B.1.3 is the step they compute): limit_ns replaces the limit of their waits (0 = the built-in two
+ * seconds), and with withhold_first_arrive != 0 one warp of every CTA keeps its first "weights written" arrival to
+ * itself, so that the thread that issues the sums runs into the limit; the kernel then unwinds as described above
+ * (what it leaves in the workspace and in `out` is meaningless) and raises GTA_ERR_TIMEOUT.  Same lifetime of the
+ * settings; the call synchronises the device.  Not for production use.
+ */
+GTA_API gta_status_t gta_debug_decode_wait(uint64_t limit_ns, int32_t withhold_first_arrive);
+
 #ifdef __cplusplus
 }
 #endif

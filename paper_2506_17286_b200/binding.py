@@ -27,6 +27,7 @@ EXPORTS = (
     "gta_decode_paged_workspace_bytes", "gta_decode_paged", "gta_cache_append_paged",
     "gta_layer_prefill_workspace_bytes", "gta_layer_prefill", "gta_layer_decode_workspace_bytes", "gta_layer_decode",
     "gta_layer_decode_paged_workspace_bytes", "gta_layer_decode_paged", "gta_debug_attention_wait",
+    "gta_debug_decode_wait",
     "gta_ref_gqa_prefill", "gta_ref_gqa_decode_workspace_bytes", "gta_ref_gqa_decode",
     "gta_decode_fp8_workspace_bytes", "gta_cache_append_fp8", "gta_decode_fp8", "gta_decode_append",
     "gta_prefill_chunk_paged", "gta_layer_prefill_paged", "gta_decode_fp8_path",
@@ -134,6 +135,8 @@ def lib():
         L.gta_decode_append.restype = i32
         L.gta_debug_attention_wait.argtypes = [ctypes.c_uint64, i32]
         L.gta_debug_attention_wait.restype = i32
+        L.gta_debug_decode_wait.argtypes = [ctypes.c_uint64, i32]
+        L.gta_debug_decode_wait.restype = i32
         _lib = L
     return _lib
 
@@ -144,6 +147,13 @@ def status_string(status: int) -> str:
 
 def version() -> int:
     return int(lib().gta_version())
+
+
+def debug_decode_wait(limit_ns: int = 0, withhold_first_arrive: bool = False) -> None:
+    """Test hook of the tensor-memory decode stream kernels' bounded waits (see gta_debug_decode_wait in include/gta.h)."""
+    st = lib().gta_debug_decode_wait(int(limit_ns), int(bool(withhold_first_arrive)))
+    if st != GTA_OK:
+        raise GtaError(st, "gta_debug_decode_wait")
 
 
 def debug_attention_wait(limit_ns: int = 0, withhold_first_arrive: bool = False) -> None:

@@ -108,6 +108,14 @@ gta_status_t gta_debug_attention_wait(uint64_t limit_ns, int32_t withhold_first_
     return gta::sm100_attention_debug_wait(limit_ns, withhold_first_arrive);
 }
 
+gta_status_t gta_debug_decode_wait(uint64_t limit_ns, int32_t withhold_first_arrive) {
+    gta_status_t st = check_device();
+    if (st != GTA_OK) return st;
+    st = gta::decode_tc_debug_wait(limit_ns, withhold_first_arrive);
+    if (st != GTA_OK) return st;
+    return gta::decode_fp8_tc_debug_wait(limit_ns, withhold_first_arrive);
+}
+
 int gta_prefill_path(const gta_shape_t* shape) {
     gta::Dims d;
     if (check_shape(shape, true, &d) != GTA_OK) return 0;

@@ -37,6 +37,12 @@
 namespace gta {
 namespace {
 
+// Test hooks of the bounded waits (gta_debug_decode_wait): the time limit of every wait of this kernel, and a switch
+// that makes one warp of group B keep its very first arrival to itself, so that the MMA warp runs into that limit and
+// the whole unwinding path can be exercised on a healthy GPU.  Read once per thread at kernel start.
+__device__ unsigned long long g_tc_wait_limit_ns = ptx::kWaitLimitNs;
+__device__ int g_tc_withhold_first_arrive = 0;
+
 constexpr int kTcT = 64;                        // tokens per sub-tile
 constexpr int kTcStages = 3;
 constexpr int kTcThreads = 320;
@@ -114,6 +120,10 @@ decode_stream_fp8_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __gr
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(drain_bar + 1);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
     volatile int* drain_flag = abort_flag + 1;
+    const uint64_t wait_limit = g_tc_wait_limit_ns;
+    const bool withhold_first_arrive = g_tc_withhold_first_arrive != 0;
+    // every wait of this kernel: bounded by wait_limit, ended early by the CTA's abort flag
+    auto wait = [&](uint64_t* bar, uint32_t parity) { return ptx::mbar_wait_sleep(bar, parity, abort_flag, 0, wait_limit); };
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int G = gridDim.x, cta = blockIdx.x;
@@ -200,7 +210,7 @@ decode_stream_fp8_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __gr
             const int tok0 = k * kTcT;
             const uint32_t n_sc = (uint32_t)min(kTcT, S_cap - tok0) * 4;   // bytes of a scale row (S_cap is a multiple of 4)
             if (lane == 0) {
-                ok = ptx::mbar_wait(&empty_bar[s], ph ^ 1, abort_flag);
+                ok = wait(&empty_bar[s], ph ^ 1);
                 if (ok) ptx::mbar_arrive_expect_tx(&full_bar[s], lay.scale_off + (uint32_t)(NK + 1) * n_sc);
             }
             ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
@@ -243,10 +253,10 @@ decode_stream_fp8_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __gr
                 while (sk >= prefix[sb + 1] - prefix[sb]) { ++sb; sk = 0; first = true; }
                 if (first && j > 0) ++sn;
                 const int s = j % kTcStages;
-                if (first && !ptx::mbar_wait(&q_ready[sn & 1], (sn >> 1) & 1, abort_flag)) return false;
-                if (!ptx::mbar_wait(&full_bar[s], (j / kTcStages) & 1, abort_flag)) return false;
+                if (first && !wait(&q_ready[sn & 1], (sn >> 1) & 1)) return false;
+                if (!wait(&full_bar[s], (j / kTcStages) & 1)) return false;
                 // the buffer held the scores of sub-tile j - 2
-                if (j >= 2 && !ptx::mbar_wait(&s_free[j & 1], ((j >> 1) - 1) & 1, abort_flag)) return false;
+                if (j >= 2 && !wait(&s_free[j & 1], ((j >> 1) - 1) & 1)) return false;
                 ptx::tc_fence_after_sync();
                 const uint32_t stage = ring_addr + s * lay.stage_stride;
                 const uint64_t dq = desc_kmajor + ((q_addr + (sn & 1) * kTcOperand) >> 4);
@@ -271,7 +281,7 @@ decode_stream_fp8_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __gr
                 bool first = (i == 0);
                 while (pk >= prefix[pb + 1] - prefix[pb]) { ++pb; pk = 0; first = true; }
                 ++pk;
-                ok = ptx::mbar_wait(&p_ready[i & 1], (i >> 1) & 1, abort_flag);
+                ok = wait(&p_ready[i & 1], (i >> 1) & 1);
                 if (!ok) break;
                 ptx::tc_fence_after_sync();
                 const int s = i % kTcStages;
@@ -381,8 +391,8 @@ decode_stream_fp8_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __gr
                 const int n_valid = min(kTcT, len_b - k * kTcT);
                 const float* ksc = reinterpret_cast<const float*>(ring + s * lay.stage_stride + lay.scale_off);
                 const float* csc = ksc + NK * kTcT;
-                ok = ptx::mbar_wait(&full_bar[s], (i / kTcStages) & 1, abort_flag) && ok;
-                ok = ptx::mbar_wait(&s_ready[i & 1], (i >> 1) & 1, abort_flag) && ok;
+                ok = wait(&full_bar[s], (i / kTcStages) & 1) && ok;
+                ok = wait(&s_ready[i & 1], (i >> 1) & 1) && ok;
                 ptx::tc_fence_after_sync();
 
                 // ---- this token's scores of this thread's maps, plain (x) and shifted by log2 of the latent row's scale (y)
@@ -440,7 +450,7 @@ decode_stream_fp8_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __gr
                     }
                 }
                 // ---- hand-over to group B (the buffers of sub-tile i - 2 have been read)
-                if (i >= 2) ok = ptx::mbar_wait(&xy_free[i & 1], ((i >> 1) - 1) & 1, abort_flag) && ok;
+                if (i >= 2) ok = wait(&xy_free[i & 1], ((i >> 1) - 1) & 1) && ok;
                 float* eb = e_buf + (i & 1) * (2 * 8 * kTcT) + token;
 #pragma unroll
                 for (int g = 0; g < 8; ++g) {
@@ -476,7 +486,7 @@ decode_stream_fp8_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __gr
                 const int s = i % kTcStages;
                 const int n_valid = min(kTcT, len_b - k * kTcT);
                 uint8_t* stage = ring + s * lay.stage_stride;
-                ok = ptx::mbar_wait(&xy_ready[i & 1], (i >> 1) & 1, abort_flag) && ok;
+                ok = wait(&xy_ready[i & 1], (i >> 1) & 1) && ok;
                 float alpha[8];
 #pragma unroll
                 for (int g = 0; g < 8; ++g) {
@@ -498,7 +508,7 @@ decode_stream_fp8_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __gr
                 // ---- rows past the live length hold whatever the cache holds there (NaN codes included): their
                 //      weights are zero, so the latent rows are cleared
                 if (n_valid < kTcT) {
-                    ok = ptx::mbar_wait(&full_bar[s], (i / kTcStages) & 1, abort_flag) && ok;
+                    ok = wait(&full_bar[s], (i / kTcStages) & 1) && ok;
                     const int n_vec = (kTcT - n_valid) * CH * 8;
                     for (int idx = gtid; idx < n_vec; idx += 128) {
                         const int row = n_valid + idx / (CH * 8), v = idx % (CH * 8);
@@ -509,7 +519,7 @@ decode_stream_fp8_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __gr
                 // ---- the sums so far are rescaled when a maximum has grown (the first sub-tile of a sequence
                 //      overwrites them)
                 if (grow && !first) {       // uniform over the group
-                    ok = ptx::mbar_wait(&pv_done[(i - 1) & 1], ((i - 1) >> 1) & 1, abort_flag) && ok;
+                    ok = wait(&pv_done[(i - 1) & 1], ((i - 1) >> 1) & 1) && ok;
                     ptx::tc_fence_after_sync();
 #pragma unroll
                     for (int c = 0; c < CH; ++c) {
@@ -524,7 +534,7 @@ decode_stream_fp8_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __gr
                 }
                 // ---- the weights' pieces of this token into the B operand of the sums (free once the sums of
                 //      sub-tile i - 2 are complete)
-                if (i >= 2) ok = ptx::mbar_wait(&pv_done[i & 1], ((i >> 1) - 1) & 1, abort_flag) && ok;
+                if (i >= 2) ok = wait(&pv_done[i & 1], ((i >> 1) - 1) & 1) && ok;
                 {
                     uint8_t* dst = p_buf + (i & 1) * kTcOperand + tok_low;
 #pragma unroll
@@ -543,13 +553,13 @@ decode_stream_fp8_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __gr
                 ptx::fence_proxy_async_smem();      // the weights and the cleared rows, before the tensor pipe reads them
                 ptx::tc_fence_before_sync();
                 __syncwarp();
-                if (lane == 0) ptx::mbar_arrive(&p_ready[i & 1]);
+                if (lane == 0 && !(withhold_first_arrive && i == 0 && quarter == 0)) ptx::mbar_arrive(&p_ready[i & 1]);
                 first = false;
 
                 // ---- the last sub-tile of the sequence in this range: its partial result goes to slot cta + b
                 const bool last = (i + 1 == n_sub) || (k + 1 >= n_sub_b);
                 if (last) {
-                    ok = ptx::mbar_wait(&pv_done[i & 1], (i >> 1) & 1, abort_flag) && ok;
+                    ok = wait(&pv_done[i & 1], (i >> 1) & 1) && ok;
                     ptx::tc_fence_after_sync();
                     const size_t slot = (size_t)cta + b;
 #pragma unroll
@@ -663,6 +673,17 @@ cudaError_t launch_decode_fp8_tc_stream(const Dims& d, int G, int S_cap, const v
     }
     if (err != cudaSuccess) return err;
     return cudaGetLastError();
+}
+
+gta_status_t decode_fp8_tc_debug_wait(unsigned long long limit_ns, int withhold_first_arrive) {
+    const unsigned long long lim = limit_ns ? limit_ns : ptx::kWaitLimitNs;
+    const int sw = withhold_first_arrive ? 1 : 0;
+    if (cudaMemcpyToSymbol(g_tc_wait_limit_ns, &lim, sizeof(lim)) != cudaSuccess ||
+        cudaMemcpyToSymbol(g_tc_withhold_first_arrive, &sw, sizeof(sw)) != cudaSuccess) {
+        cudaGetLastError();
+        return GTA_ERR_CUDA;
+    }
+    return GTA_OK;
 }
 
 }  // namespace gta

@@ -34,6 +34,12 @@
 namespace gta {
 namespace {
 
+// Test hooks of the bounded waits (gta_debug_decode_wait): the time limit of every wait of this kernel, and a switch
+// that makes one warp of group B keep its very first arrival to itself, so that the MMA warp runs into that limit and
+// the whole unwinding path can be exercised on a healthy GPU.  Read once per thread at kernel start.
+__device__ unsigned long long g_bt_wait_limit_ns = ptx::kWaitLimitNs;
+__device__ int g_bt_withhold_first_arrive = 0;
+
 constexpr int kBtStages = 3;
 constexpr int kBtThreads = 320;
 constexpr int kBtMaxBatch = 512;
@@ -121,6 +127,10 @@ decode_stream_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_c
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(drain_bar + 1);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
     volatile int* drain_flag = abort_flag + 1;
+    const uint64_t wait_limit = g_bt_wait_limit_ns;
+    const bool withhold_first_arrive = g_bt_withhold_first_arrive != 0;
+    // every wait of this kernel: bounded by wait_limit, ended early by the CTA's abort flag
+    auto wait = [&](uint64_t* bar, uint32_t parity) { return ptx::mbar_wait_sleep(bar, parity, abort_flag, 0, wait_limit); };
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int G = gridDim.x, cta = blockIdx.x;
@@ -217,7 +227,7 @@ decode_stream_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_c
                 tok0 %= pm.page_size;
             }
             if (lane == 0) {
-                ok = ptx::mbar_wait(&empty_bar[s], ph ^ 1, abort_flag);
+                ok = wait(&empty_bar[s], ph ^ 1);
                 if (ok) ptx::mbar_arrive_expect_tx(&full_bar[s], (uint32_t)n_ops * tb);
             }
             ok = __shfl_sync(0xffffffffu, (int)ok, 0) != 0;
@@ -253,10 +263,10 @@ decode_stream_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_c
             if (first && j > 0) ++sn;
             const int s = j % kBtStages;
             // (every lane of the warp waits: its lanes share the append below; the outcome is made uniform)
-            bool w = !first || ptx::mbar_wait(&q_ready[sn & 1], (sn >> 1) & 1, abort_flag);
-            w = w && ptx::mbar_wait(&full_bar[s], (j / kBtStages) & 1, abort_flag);
+            bool w = !first || wait(&q_ready[sn & 1], (sn >> 1) & 1);
+            w = w && wait(&full_bar[s], (j / kBtStages) & 1);
             // the buffer held the scores of sub-tile j - 2
-            w = w && (j < 2 || ptx::mbar_wait(&s_free[j & 1], ((j >> 1) - 1) & 1, abort_flag));
+            w = w && (j < 2 || wait(&s_free[j & 1], ((j >> 1) - 1) & 1));
             if (!__all_sync(0xffffffffu, w)) return false;
             const uint32_t stage = ring_addr + s * lay.stage_stride;
             // the sub-tile that ends a sequence of the fused step holds the new token (its last live row): what TMA
@@ -313,7 +323,7 @@ decode_stream_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_c
             bool first = (i == 0);
             while (pk >= prefix[pb + 1] - prefix[pb]) { ++pb; pk = 0; first = true; }
             ++pk;
-            ok = __all_sync(0xffffffffu, ptx::mbar_wait(&p_ready[i & 1], (i >> 1) & 1, abort_flag));
+            ok = __all_sync(0xffffffffu, wait(&p_ready[i & 1], (i >> 1) & 1));
             if (!ok) break;
             ptx::tc_fence_after_sync();
             if (lane == 0) {
@@ -394,7 +404,7 @@ decode_stream_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_c
                     if (nb >= 0) write_q(nb, (n + 1) & 1);
                 }
                 const int n_valid = min(T, len_b - k * T);
-                ok = ptx::mbar_wait(&s_ready[i & 1], (i >> 1) & 1, abort_flag) && ok;
+                ok = wait(&s_ready[i & 1], (i >> 1) & 1) && ok;
                 ptx::tc_fence_after_sync();
 
                 // ---- this (key group, token)'s scores of the key group's maps, in log2 units
@@ -445,7 +455,7 @@ decode_stream_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_c
                     }
                 }
                 // ---- hand-over to group B (the buffers of sub-tile i - 2 have been read)
-                if (i >= 2) ok = ptx::mbar_wait(&xy_free[i & 1], ((i >> 1) - 1) & 1, abort_flag) && ok;
+                if (i >= 2) ok = wait(&xy_free[i & 1], ((i >> 1) - 1) & 1) && ok;
 #pragma unroll
                 for (int set = 0; set < SETS; ++set) {
                     const int kg = set * R + gsel;
@@ -490,7 +500,7 @@ decode_stream_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_c
                 const int s = i % kBtStages;
                 const int n_valid = min(T, len_b - k * T);
                 uint8_t* stage = ring + s * lay.stage_stride;
-                ok = ptx::mbar_wait(&xy_ready[i & 1], (i >> 1) & 1, abort_flag) && ok;
+                ok = wait(&xy_ready[i & 1], (i >> 1) & 1) && ok;
                 float alpha[8];
 #pragma unroll
                 for (int g = 0; g < 8; ++g) {
@@ -520,7 +530,7 @@ decode_stream_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_c
                 // ---- rows past the live length hold whatever the cache holds there (NaN patterns included): their
                 //      weights are zero, so the latent rows are cleared
                 if (n_valid < T) {
-                    ok = ptx::mbar_wait(&full_bar[s], (i / kBtStages) & 1, abort_flag) && ok;
+                    ok = wait(&full_bar[s], (i / kBtStages) & 1) && ok;
                     const int n_vec = (T - n_valid) * CH * 16;
                     for (int idx = gtid; idx < n_vec; idx += 128) {
                         const int row = n_valid + idx / (CH * 16), v = idx % (CH * 16);
@@ -531,7 +541,7 @@ decode_stream_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_c
                 // ---- the sums so far are rescaled when a maximum was raised (the first sub-tile of a sequence
                 //      overwrites them)
                 if (grow && !first) {       // uniform over the group
-                    ok = ptx::mbar_wait(&pv_done[(i - 1) & 1], ((i - 1) >> 1) & 1, abort_flag) && ok;
+                    ok = wait(&pv_done[(i - 1) & 1], ((i - 1) >> 1) & 1) && ok;
                     ptx::tc_fence_after_sync();
 #pragma unroll
                     for (int c = 0; c < CH; ++c) {
@@ -546,7 +556,7 @@ decode_stream_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_c
                 }
                 // ---- the weights of this (key group, token) into the B operand of the sums (free once the sums of
                 //      sub-tile i - 2 are complete)
-                if (i >= 2) ok = ptx::mbar_wait(&pv_done[i & 1], ((i >> 1) - 1) & 1, abort_flag) && ok;
+                if (i >= 2) ok = wait(&pv_done[i & 1], ((i >> 1) - 1) & 1) && ok;
 #pragma unroll
                 for (int set = 0; set < SETS; ++set) {
                     const int kg = set * R + gsel;
@@ -563,13 +573,13 @@ decode_stream_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_c
                 ptx::fence_proxy_async_smem();      // the weights and the cleared rows, before the tensor pipe reads them
                 ptx::tc_fence_before_sync();
                 __syncwarp();
-                if (lane == 0) ptx::mbar_arrive(&p_ready[i & 1]);
+                if (lane == 0 && !(withhold_first_arrive && i == 0 && quarter == 0)) ptx::mbar_arrive(&p_ready[i & 1]);
                 first = false;
 
                 // ---- the last sub-tile of the sequence in this range: its partial result goes to slot cta + b
                 const bool last = (i + 1 == n_sub) || (k + 1 >= n_sub_b);
                 if (last) {
-                    ok = ptx::mbar_wait(&pv_done[i & 1], (i >> 1) & 1, abort_flag) && ok;
+                    ok = wait(&pv_done[i & 1], (i >> 1) & 1) && ok;
                     ptx::tc_fence_after_sync();
                     const size_t slot = (size_t)cta + b;
 #pragma unroll
@@ -680,6 +690,17 @@ cudaError_t launch_decode_tc_stream(const Dims& d, int G, int T, int S_cap, cons
 #undef GTA_BT_LAUNCH
     if (err != cudaSuccess) return err;
     return cudaGetLastError();
+}
+
+gta_status_t decode_tc_debug_wait(unsigned long long limit_ns, int withhold_first_arrive) {
+    const unsigned long long lim = limit_ns ? limit_ns : ptx::kWaitLimitNs;
+    const int sw = withhold_first_arrive ? 1 : 0;
+    if (cudaMemcpyToSymbol(g_bt_wait_limit_ns, &lim, sizeof(lim)) != cudaSuccess ||
+        cudaMemcpyToSymbol(g_bt_withhold_first_arrive, &sw, sizeof(sw)) != cudaSuccess) {
+        cudaGetLastError();
+        return GTA_ERR_CUDA;
+    }
+    return GTA_OK;
 }
 
 }  // namespace gta

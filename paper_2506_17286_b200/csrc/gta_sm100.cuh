@@ -72,4 +72,8 @@ cudaError_t launch_decode_tc_stream(const Dims& d, int G, int T, int S_cap, cons
                                     int32_t* status_word, cudaStream_t stream, const void* k_new, const void* c_new,
                                     const PageMap& pm);
 
+// Test hooks of the bounded waits of the two tensor-memory decode stream kernels (see gta_debug_decode_wait in gta.h).
+gta_status_t decode_tc_debug_wait(unsigned long long limit_ns, int withhold_first_arrive);
+gta_status_t decode_fp8_tc_debug_wait(unsigned long long limit_ns, int withhold_first_arrive);
+
 }  // namespace gta

@@ -149,6 +149,37 @@ def test_fp8_decode_scores_that_keep_rising_or_falling(B, oracle, slope):
     print(f"\nslope {slope}: rel-L2 {rel:.3e} max-abs {mx:.3e}")
 
 
+def test_a_wait_that_runs_out_unwinds_the_fp8_stream_kernel(B, oracle):
+    """One warp of every CTA keeps its first "weights written" arrival to itself and the waits give up after 2 ms:
+    the call comes back with GTA_ERR_TIMEOUT, and the next ordinary call gives bit for bit what the call before gave."""
+    w = I.Workload("timeout8", "decode", "bf16", 3, 0, 256, 8, 4, 4, 1, 128, 512, seed=65)
+    lens, cap = [200, 64, 33], 208
+    t = I.decode_inputs(w, device="cuda", s_cap=cap, seq_lens=lens)
+    kq, ks = oracle.quantize_rows_e4m3(t["k_cache"].cpu())
+    cq, cs = oracle.quantize_rows_e4m3(t["c_cache"].cpu())
+    dev = [torch.from_numpy(a).cuda() for a in (kq, cq, ks, cs)]
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    args = (t["q"], *dev, t["seq_lens"], t["x_t"], t["w_p"], t["w_g"])
+    shape = B.decode_shape(t["q"], t["k_cache"], t["c_cache"], t["x_t"], t["w_p"])
+    assert B.decode_fp8_path(shape, cap) == 2
+    before = B.gta_decode_fp8(*args, status_word=status).clone()
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    B.debug_decode_wait(limit_ns=2_000_000, withhold_first_arrive=True)
+    try:
+        junk = B.gta_decode_fp8(*args, status_word=status)
+        torch.cuda.synchronize()                      # returns: every wait is bounded
+        assert int(status.item()) == B.GTA_ERR_TIMEOUT
+        del junk
+    finally:
+        B.debug_decode_wait(limit_ns=0, withhold_first_arrive=False)
+    status.zero_()
+    after = B.gta_decode_fp8(*args, status_word=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    assert torch.equal(after.view(torch.int16), before.view(torch.int16))
+
+
 def test_fp8_decode_config3_shape_sampled_sequences(B, oracle):
     w = I.CONFIGS["c3_decode_bf16"]
     rel, mx = _decode_case(B, oracle, w, [w.seq] * w.batch, sample=[0, 9, 31], cap=w.seq + 64, path=2)

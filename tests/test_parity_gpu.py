@@ -534,6 +534,36 @@ def test_a_wait_that_runs_out_unwinds_the_attention_kernel(B, oracle):
     assert_close(after, want, torch.bfloat16, "after a timed-out call")
 
 
+def test_a_wait_that_runs_out_unwinds_the_decode_stream_kernel(B, oracle):
+    """The same for the decode stream kernel that keeps its sums in tensor memory: one warp of every CTA keeps its
+    first "weights written" arrival to itself and the waits give up after 2 ms; the call comes back with
+    GTA_ERR_TIMEOUT, and the next ordinary call gives bit for bit what the call before gave."""
+    w = I.Workload("timeout", "decode", "bf16", 3, 0, 256, 8, 4, 4, 1, 128, 512, seed=98)
+    lens = [200, 64, 33]
+    t = I.decode_inputs(w, device="cuda", s_cap=208, seq_lens=lens)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    args = (t["q"], t["k_cache"], t["c_cache"], t["seq_lens"], t["x_t"], t["w_p"], t["w_g"])
+    before = B.gta_decode(*args, status_word=status).clone()
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    B.debug_decode_wait(limit_ns=2_000_000, withhold_first_arrive=True)
+    try:
+        junk = B.gta_decode(*args, status_word=status)
+        torch.cuda.synchronize()                      # returns: every wait is bounded
+        assert int(status.item()) == B.GTA_ERR_TIMEOUT
+        del junk
+    finally:
+        B.debug_decode_wait(limit_ns=0, withhold_first_arrive=False)
+    status.zero_()
+    after = B.gta_decode(*args, status_word=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    assert torch.equal(after.view(torch.int16), before.view(torch.int16))
+    want = oracle.decode(oracle_shape(w, seq=0), t["q"].cpu(), t["k_cache"].cpu(), t["c_cache"].cpu(), lens, 208,
+                         t["x_t"].cpu(), t["w_p"].cpu(), t["w_g"].cpu())
+    assert_close(after, want, torch.bfloat16, "after a timed-out call")
+
+
 # --------------------------------------------------------------------------- append + decode in one call
 STEP_CASES = [
     # name, dtype, H, n_h, n_q, n_k, n_c, d_h, d_l, lens BEFORE the step, S_cap
