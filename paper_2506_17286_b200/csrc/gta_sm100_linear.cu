@@ -34,7 +34,7 @@ namespace gta {
 namespace {
 
 constexpr int kLinStages = 6;
-constexpr int kLinThreads = 320;
+constexpr int kLinThreads = 352;    // warp 0 TMA, warp 1 MMA issue, warps 2-9 epilogue, warp 10 second MMA issuer (one-tile form)
 constexpr int kTileM = 128;        // rows per CTA and unit
 constexpr int kBlockK = 64;        // K elements per pipeline stage (one 128-byte swizzle row)
 constexpr uint32_t kATileBytes = kTileM * kBlockK * 2;   // 16 KB
@@ -161,10 +161,14 @@ sm100_linear_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
     constexpr int kUnitRows = kPair ? 2 * kTileM : kTileM;
     const int n_items = a.q + ((a.split_tail ? pr < 2 * a.r : pr < a.r) ? 1 : 0);
     const int ks_total = a.K / kBlockK;
+    // One-tile form: a single thread's instruction stream (wait, descriptors, four MMAs, commit per k-block) is what
+    // paces a CTA there, so two threads issue -- the even and the odd k-blocks, into accumulators of their own that the
+    // epilogue adds.
+    const bool two_issuers = !kPair && ks_total >= 2;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < n_stages; ++s) { ptx::mbar_init(&full_bar[s], kPair ? 2 : 1); ptx::mbar_init(&empty_bar[s], 1); }
-        for (int j = 0; j < 2; ++j) { ptx::mbar_init(&acc_full[j], 1); ptx::mbar_init(&acc_free[j], kPair ? 16 : 8); }
+        for (int j = 0; j < 2; ++j) { ptx::mbar_init(&acc_full[j], two_issuers ? 2 : 1); ptx::mbar_init(&acc_free[j], kPair ? 16 : 8); }
         *abort_flag = 0;
         *drain_flag = 0;
         ptx::fence_mbar_init();
@@ -240,6 +244,41 @@ sm100_linear_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
                 }
             }
         }
+    } else if (!kPair && (warp == 1 || warp == 10)) {
+        // one-tile form: issuer `me` takes the k-blocks it = me, me + 2, ... (all of them without a second issuer)
+        const int me = warp == 1 ? 0 : 1, step = two_issuers ? 2 : 1;
+        if ((me == 0 || two_issuers) && ptx::elect_one()) {
+            const uint64_t desc_a0 = ptx::make_smem_desc(0, 16, 1024);
+            const uint64_t desc_b0 = ptx::make_smem_desc(0, 64 * 128, 1024);
+            const uint32_t smem_a = ptx::smem_addr(smem), smem_b = ptx::smem_addr(smem + b_base);
+            bool ok = true;
+            int it0 = 0;                 // first k-block of the unit in the ring's count
+            for (int n = 0; n < n_items && ok; ++n, it0 += ks_total) {
+                int row0, f0, nt;
+                unit(n, row0, f0, nt);
+                const uint32_t idesc = ptx::make_idesc_bf16(kTileM, nt, 0, 1);   // A K-major, W MN-major
+                const uint32_t d_tmem = tmem_base + (uint32_t)(n & 1) * 256 + (uint32_t)me * 64;
+                ok = ptx::mbar_wait(&acc_free[n & 1], ((n >> 1) & 1) ^ 1, abort_flag);
+                bool first = true;
+                int it = it0 + ((it0 + me) & (step - 1));
+                int s = it % n_stages;                       // stage and phase kept as counters (no division per k-block)
+                uint32_t ph = (uint32_t)(it / n_stages) & 1u;
+                for (; it < it0 + ks_total && ok; it += step, s += step) {
+                    if (s >= n_stages) { s -= n_stages; ph ^= 1u; }
+                    ok = ptx::mbar_wait(&full_bar[s], ph, abort_flag);
+                    if (!ok) break;
+                    ptx::tc_fence_after_sync();
+                    const uint64_t a_desc = desc_a0 + ((smem_a + (uint32_t)s * a_stride) >> 4);
+                    const uint64_t b_desc = desc_b0 + ((smem_b + (uint32_t)s * b_stride) >> 4);
+#pragma unroll
+                    for (int k4 = 0; k4 < kBlockK / 16; ++k4)
+                        ptx::mma_ss(d_tmem, a_desc + 2 * k4, b_desc + k4 * ((16 * 128) >> 4), idesc, (first && k4 == 0) ? 0u : 1u);
+                    first = false;
+                    ptx::tc_commit(&empty_bar[s]);
+                }
+                if (ok) ptx::tc_commit(&acc_full[n & 1]);
+            }
+        }
     } else if (warp == 1) {
         if (rank == 0 && ptx::elect_one()) {
             int it = 0, s = 0;
@@ -275,7 +314,7 @@ sm100_linear_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
                 }
             }
         }
-    } else {
+    } else if (warp >= 2 && warp < 10) {
         // epilogue: warp w may touch TMEM lanes [32 (w % 4), 32 (w % 4) + 32); the two warps of a
         // quarter take one half of the unit's columns each
         const int quarter = warp & 3;
@@ -324,6 +363,13 @@ sm100_linear_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_const
                 if (ch * 32 < cols) {
                     uint32_t v[32];
                     ptx::tmem_ld32(acc + ch * 32, v);
+                    if (two_issuers) {       // the second issuer's share of the sum (64 columns further on)
+                        uint32_t v2[32];
+                        ptx::tmem_ld32(acc + 64 + ch * 32, v2);
+                        ptx::tmem_wait_ld();
+#pragma unroll
+                        for (int e = 0; e < 32; ++e) v[e] = __float_as_uint(__uint_as_float(v[e]) + __uint_as_float(v2[e]));
+                    }
                     float4 rope_cur[8];
 #pragma unroll
                     for (int j2 = 0; j2 < 8; ++j2) rope_cur[j2] = rope_next[j2];
