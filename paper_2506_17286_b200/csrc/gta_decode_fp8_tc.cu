@@ -43,13 +43,12 @@ namespace {
 __device__ unsigned long long g_tc_wait_limit_ns = ptx::kWaitLimitNs;
 __device__ int g_tc_withhold_first_arrive = 0;
 
-constexpr int kTcT = 64;                        // tokens per sub-tile
+constexpr int kTcMaxT = 64;                     // most tokens per sub-tile (64, or 32 for wide tokens)
 constexpr int kTcStages = 3;
 constexpr int kTcThreads = 320;
 constexpr int kTcMaxBatch = 512;
-constexpr uint32_t kTcTile = kTcT * 128;        // bytes of a [64 tokens][128 codes] tile
 constexpr uint32_t kTcOperand = 16 * 128;       // bytes of a [16 rows][128 codes] B operand (Q pieces, weights' pieces)
-constexpr uint32_t kTcExpBytes = 2 * 2 * 8 * kTcT * 4;   // exponents handed from group A to group B
+constexpr uint32_t kTcExpBytes = 2 * 2 * 8 * kTcMaxT * 4;   // exponents handed from group A to group B
 constexpr uint32_t kTcTmemCols = 256;           // 2 x 64 score columns, 64 sum columns
 constexpr float kTcWeightScale = 64.f;          // the weights are scaled into e4m3's range ...
 constexpr float kTcLag = 2.f;                   // ... with room for a running maximum that lags by 2^2
@@ -72,10 +71,10 @@ __device__ __forceinline__ uint32_t tc_swz(int row, int col) {
 struct TcSmem {
     uint32_t stage_stride, scale_off, q_off, p_off, misc_off, total;
 };
-__host__ __device__ inline TcSmem tc_smem_layout(int n_k, int ch) {
+__host__ __device__ inline TcSmem tc_smem_layout(int T, int n_k, int ch) {
     TcSmem s;
-    s.scale_off = (uint32_t)(n_k + ch) * kTcTile;
-    s.stage_stride = s.scale_off + (((uint32_t)(n_k + 1) * kTcT * 4 + 1023u) & ~1023u);
+    s.scale_off = (uint32_t)(n_k + ch) * (uint32_t)T * 128u;
+    s.stage_stride = s.scale_off + (((uint32_t)(n_k + 1) * T * 4 + 1023u) & ~1023u);
     s.q_off = kTcStages * s.stage_stride;            // [2 sequence parities][16][128]
     s.p_off = s.q_off + 2 * kTcOperand;              // [2 sub-tile parities][16][128]
     s.misc_off = s.p_off + 2 * kTcOperand;
@@ -88,7 +87,7 @@ __host__ __device__ inline TcSmem tc_smem_layout(int n_k, int ch) {
 // CH: 128-column blocks of the latent; NK: key groups; QPK: maps per key group (compile-time, so that the per-map
 // loops of the token threads unroll into straight code: those threads run one warp per scheduler, at the latency of
 // every instruction they issue).
-template <int CH, int NK, int QPK>
+template <int T, int CH, int NK, int QPK>
 __global__ void __launch_bounds__(kTcThreads, 1)
 decode_stream_fp8_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_c, Dims d,
                             int S_cap, const __nv_bfloat16* __restrict__ q, const float* __restrict__ k_scale,
@@ -96,7 +95,13 @@ decode_stream_fp8_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __gr
                             float* __restrict__ part_o, float* __restrict__ part_ml, int32_t* status_word) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-    const TcSmem lay = tc_smem_layout(NK, CH);
+    constexpr int kTcT = T;
+    constexpr uint32_t kTcTile = T * 128;            // bytes of a [T tokens][128 codes] tile
+    constexpr int R = 128 / T;                        // key groups on the 128 rows of a score MMA
+    constexpr int SETS = (NK + R - 1) / R;
+    constexpr int WPG = T / 32;                       // warps of a group per key group
+    static_assert(SETS <= 2 && NK * QPK <= 8 && CH <= 8, "instantiation outside the kernel's limits");
+    const TcSmem lay = tc_smem_layout(T, NK, CH);
     uint8_t* ring = smem;
     uint8_t* q_buf = smem + lay.q_off;
     uint8_t* p_buf = smem + lay.p_off;
@@ -263,8 +268,8 @@ decode_stream_fp8_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __gr
                 // The 128 rows of A are the 64 tokens of key group 2 kp and, 8 KB further on, the same 64 tokens of key
                 // group 2 kp + 1 (the tiles of a stage lie back to back; behind the last key tile come latent rows,
                 // whose "scores" nobody reads): lanes 0-63 and 64-127 of the accumulator.
-                for (int kp = 0; 2 * kp < NK; ++kp) {
-                    const uint64_t dk = desc_kmajor + ((stage + 2 * kp * kTcTile) >> 4);
+                for (int kp = 0; kp < SETS; ++kp) {
+                    const uint64_t dk = desc_kmajor + ((stage + kp * R * kTcTile) >> 4);
 #pragma unroll
                     for (int ks = 0; ks < 4; ++ks)      // 32 codes = 32 bytes of the 128-byte rows per step
                         ptx::mma_ss_f8(tmem_base + (j & 1) * 64 + kp * 16, dk + 2 * ks, dq + 2 * ks, idesc_s, ks > 0 ? 1u : 0u);
@@ -291,7 +296,7 @@ decode_stream_fp8_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __gr
                 for (int c = 0; c < CH; ++c) {
                     const uint64_t dc = desc_latent + ((stage + (NK + c) * kTcTile) >> 4);
 #pragma unroll
-                    for (int kk = 0; kk < 2; ++kk)      // 32 tokens = 4096 bytes of the tile, 32 bytes of the weights' rows
+                    for (int kk = 0; kk < T / 32; ++kk)      // 32 tokens = 4096 bytes of the tile, 32 bytes of the weights' rows
                         ptx::mma_ss_f8(tmem_o + c * 16, dc + kk * (4096 >> 4), dp + 2 * kk, idesc_o,
                                        (first && kk == 0) ? 0u : 1u);
                 }
@@ -313,15 +318,15 @@ decode_stream_fp8_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __gr
         const int gtid = tid & 127;                      // thread index inside the group
         const uint32_t lane_base = ((uint32_t)(quarter * 32) << 16);
         const uint32_t tmem_o = tmem_base + 128 + lane_base;
-        const int half = quarter >> 1;
-        const int token = (quarter & 1) * 32 + lane;     // of the sub-tile
+        const int half = gtid / T;                       // key group of this thread inside a set of R
+        const int token = gtid % T;                      // of the sub-tile
         const uint32_t tok_swz = (uint32_t)token >> 4, tok_low = (uint32_t)token & 15u;
         int kg_of[8];                       // key group of map g
         bool mine[8];                       // this thread handles map g
 #pragma unroll
         for (int g = 0; g < 8; ++g) {
             kg_of[g] = g / qpk;
-            mine[g] = g < NQ && (kg_of[g] & 1) == half;
+            mine[g] = g < NQ && (kg_of[g] % R) == half;
         }
         int b = b0, k = k0, n = 0;          // sequence, its sub-tile, its ordinal in this range
         int len_b = tc_len(seq_lens, b, S_cap), n_sub_b = prefix[b + 1] - prefix[b];
@@ -404,18 +409,18 @@ decode_stream_fp8_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __gr
                 uint32_t r[2][16];
 #pragma unroll
                 for (int kp = 0; kp < 2; ++kp)
-                    if (2 * kp < NK) ptx::tmem_ld16(tmem_base + lane_base + (i & 1) * 64 + kp * 16, r[kp]);
+                    if (kp < SETS) ptx::tmem_ld16(tmem_base + lane_base + (i & 1) * 64 + kp * 16, r[kp]);
                 ptx::tmem_wait_ld();
                 ptx::tc_fence_before_sync();
                 __syncwarp();
                 if (lane == 0) ptx::mbar_arrive(&s_free[i & 1]);
 #pragma unroll
                 for (int kp = 0; kp < 2; ++kp) {
-                    if (2 * kp + half < NK) {
-                        const float ks = live ? ksc[(2 * kp + half) * kTcT + token] : 0.f;
+                    if (kp < SETS && kp * R + half < NK) {
+                        const float ks = live ? ksc[(kp * R + half) * kTcT + token] : 0.f;
 #pragma unroll
                         for (int g = 0; g < 8; ++g) {
-                            if (mine[g] && (kg_of[g] >> 1) == kp && live) {
+                            if (mine[g] && (kg_of[g] / R) == kp && live) {
                                 x[g] = (__uint_as_float(r[kp][2 * g]) + __uint_as_float(r[kp][2 * g + 1])) * qmul[(n & 1) * 8 + g] * ks;
                                 y[g] = x[g] + shift;
                             }
@@ -440,8 +445,9 @@ decode_stream_fp8_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __gr
                     alpha[g] = 1.f;
                     m_sub[g] = 0.f;
                     if (g < NQ) {
-                        const int w0 = (i & 1) * 4 + 2 * (kg_of[g] & 1);      // the two warps that score map g
-                        const float m_tile = fmaxf(mx_buf[w0 * 8 + g], mx_buf[(w0 + 1) * 8 + g]);
+                        const int w0 = (i & 1) * 4 + WPG * (kg_of[g] % R);    // the warps that score map g
+                        float m_tile = mx_buf[w0 * 8 + g];
+                        if (WPG == 2) m_tile = fmaxf(m_tile, mx_buf[(w0 + 1) * 8 + g]);
                         const bool up = m_tile > m_run[g] + kTcLag;
                         grow = grow || up;
                         alpha[g] = up ? tc_ex2(m_run[g] - m_tile) : 1.f;
@@ -587,9 +593,9 @@ decode_stream_fp8_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __gr
                         float mg = -INFINITY;
 #pragma unroll
                         for (int g = 0; g < 8; ++g) if (g == gtid) mg = m_cur[g];
-                        const int w0 = 2 * ((gtid / qpk) & 1);      // the two warps that hold map gtid's row-sum shares
+                        const int w0 = WPG * ((gtid / qpk) % R);    // the warps that hold map gtid's row-sum shares
                         part_ml[(slot * NQ + gtid) * 2] = mg;
-                        part_ml[(slot * NQ + gtid) * 2 + 1] = l_red[w0 * 8 + gtid] + l_red[(w0 + 1) * 8 + gtid];
+                        part_ml[(slot * NQ + gtid) * 2 + 1] = l_red[w0 * 8 + gtid] + (WPG == 2 ? l_red[(w0 + 1) * 8 + gtid] : 0.f);
                     }
 #pragma unroll
                     for (int g = 0; g < 8; ++g) l_thr[g] = 0.f;
@@ -607,24 +613,35 @@ decode_stream_fp8_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __gr
 
 }  // namespace
 
-// d_h = 128, one latent group, d_l = 128, 256 or 512, 1, 2 or 4 key groups with 1, 2, 4 or 8 maps each (at most 8
-// maps), sub-tiles of 64 tokens that fit the ring
+// the instantiations: (sub-tile, 128-column latent blocks, key groups, maps per group).  64-token sub-tiles where a
+// token is at most 1 KB of codes and scales (d_l <= 512, at most four key groups), 32-token ones above that.
+#define GTA_TC_SHAPES(X)                                                                                   \
+    X(64, 1, 1, 1) X(64, 1, 1, 2) X(64, 1, 1, 4) X(64, 1, 1, 8) X(64, 1, 2, 1) X(64, 1, 2, 2) X(64, 1, 2, 4)   \
+    X(64, 1, 4, 1) X(64, 1, 4, 2)                                                                          \
+    X(64, 2, 1, 1) X(64, 2, 1, 2) X(64, 2, 1, 4) X(64, 2, 1, 8) X(64, 2, 2, 1) X(64, 2, 2, 2) X(64, 2, 2, 4)   \
+    X(64, 2, 4, 1) X(64, 2, 4, 2)                                                                          \
+    X(64, 4, 1, 1) X(64, 4, 1, 2) X(64, 4, 1, 4) X(64, 4, 1, 8) X(64, 4, 2, 1) X(64, 4, 2, 2) X(64, 4, 2, 4)   \
+    X(64, 4, 4, 1) X(64, 4, 4, 2)                                                                          \
+    X(32, 8, 8, 1) X(32, 8, 4, 2) X(32, 8, 4, 1) X(32, 8, 2, 4) X(32, 8, 1, 8) X(32, 4, 8, 1)
+
+// d_h = 128, one latent group, one of the instantiated shapes with the sub-tile size the plan has chosen
 bool decode_fp8_tc_supported(const Dims& d, int T) {
-    if (T != kTcT || d.d_h != 128 || d.n_c != 1 || d.n_q > 8 || d.B > kTcMaxBatch) return false;
-    if (d.n_k != 1 && d.n_k != 2 && d.n_k != 4) return false;
-    const int qpk = d.n_q / d.n_k;
-    if (qpk != 1 && qpk != 2 && qpk != 4 && qpk != 8) return false;
-    if (d.d_l != 128 && d.d_l != 256 && d.d_l != 512) return false;
-    return tc_smem_layout(d.n_k, d.d_l / 128).total <= 232448u;
+    if (d.d_h != 128 || d.n_c != 1 || d.n_k < 1 || d.n_q % d.n_k != 0 || d.d_l % 128 != 0 || d.B > kTcMaxBatch) return false;
+    const int ch = d.d_l / 128, qpk = d.n_q / d.n_k;
+#define GTA_TC_MATCH(TV, CHV, NKV, QPKV) \
+    if (T == TV && ch == CHV && d.n_k == NKV && qpk == QPKV) return tc_smem_layout(TV, NKV, CHV).total <= 232448u;
+    GTA_TC_SHAPES(GTA_TC_MATCH)
+#undef GTA_TC_MATCH
+    return false;
 }
 
 namespace {
-template <int CH, int NK, int QPK>
+template <int T, int CH, int NK, int QPK>
 cudaError_t launch_tc(const CUtensorMap& tm_k, const CUtensorMap& tm_c, const Dims& d, int G, int S_cap, const void* q,
                       const float* k_scale, const float* c_scale, const int32_t* seq_lens, float* part_o, float* part_ml,
                       int32_t* status_word, cudaStream_t stream) {
-    auto kern = decode_stream_fp8_tc_kernel<CH, NK, QPK>;
-    const size_t smem = tc_smem_layout(NK, CH).total;
+    auto kern = decode_stream_fp8_tc_kernel<T, CH, NK, QPK>;
+    const size_t smem = tc_smem_layout(T, NK, CH).total;
     cudaError_t err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (err != cudaSuccess) return err;
     cudaLaunchConfig_t cfg = {};
@@ -640,37 +657,25 @@ cudaError_t launch_tc(const CUtensorMap& tm_k, const CUtensorMap& tm_c, const Di
     return cudaLaunchKernelEx(&cfg, kern, tm_k, tm_c, d, S_cap, (const __nv_bfloat16*)q, k_scale, c_scale, seq_lens, part_o,
                               part_ml, status_word);
 }
-template <int CH>
-cudaError_t launch_tc_groups(const CUtensorMap& tm_k, const CUtensorMap& tm_c, const Dims& d, int G, int S_cap,
-                             const void* q, const float* k_scale, const float* c_scale, const int32_t* seq_lens,
-                             float* part_o, float* part_ml, int32_t* status_word, cudaStream_t stream) {
-#define GTA_TC_CASE(NKV, QPKV)                                                                                     \
-    if (d.n_k == NKV && d.n_q == NKV * QPKV)                                                                       \
-        return launch_tc<CH, NKV, QPKV>(tm_k, tm_c, d, G, S_cap, q, k_scale, c_scale, seq_lens, part_o, part_ml,   \
-                                        status_word, stream)
-    GTA_TC_CASE(1, 1); GTA_TC_CASE(1, 2); GTA_TC_CASE(1, 4); GTA_TC_CASE(1, 8);
-    GTA_TC_CASE(2, 1); GTA_TC_CASE(2, 2); GTA_TC_CASE(2, 4);
-    GTA_TC_CASE(4, 1); GTA_TC_CASE(4, 2);
-#undef GTA_TC_CASE
-    return cudaErrorInvalidValue;
-}
 }  // namespace
 
-cudaError_t launch_decode_fp8_tc_stream(const Dims& d, int G, int S_cap, const void* q, const void* k_codes,
+cudaError_t launch_decode_fp8_tc_stream(const Dims& d, int G, int T, int S_cap, const void* q, const void* k_codes,
                                         const void* c_codes, const float* k_scale, const float* c_scale,
                                         const int32_t* seq_lens, float* part_o, float* part_ml, int32_t* status_word,
                                         cudaStream_t stream) {
     CUtensorMap tm_k, tm_c;
-    const uint32_t box[3] = {128, (uint32_t)kTcT, 1};
+    const uint32_t box[3] = {128, (uint32_t)T, 1};
     const uint64_t dk[3] = {128, (uint64_t)S_cap, (uint64_t)d.B * d.n_k};
     const uint64_t dc[3] = {(uint64_t)d.d_l, (uint64_t)S_cap, (uint64_t)d.B};
     if (!make_u8_map(&tm_k, k_codes, 3, dk, box) || !make_u8_map(&tm_c, c_codes, 3, dc, box)) return cudaErrorInvalidValue;
-    cudaError_t err;
-    switch (d.d_l / 128) {
-        case 1: err = launch_tc_groups<1>(tm_k, tm_c, d, G, S_cap, q, k_scale, c_scale, seq_lens, part_o, part_ml, status_word, stream); break;
-        case 2: err = launch_tc_groups<2>(tm_k, tm_c, d, G, S_cap, q, k_scale, c_scale, seq_lens, part_o, part_ml, status_word, stream); break;
-        default: err = launch_tc_groups<4>(tm_k, tm_c, d, G, S_cap, q, k_scale, c_scale, seq_lens, part_o, part_ml, status_word, stream); break;
-    }
+    const int ch = d.d_l / 128, qpk = d.n_q / d.n_k;
+    cudaError_t err = cudaErrorInvalidValue;
+#define GTA_TC_LAUNCH(TV, CHV, NKV, QPKV)                                                                         \
+    if (T == TV && ch == CHV && d.n_k == NKV && qpk == QPKV)                                                      \
+        err = launch_tc<TV, CHV, NKV, QPKV>(tm_k, tm_c, d, G, S_cap, q, k_scale, c_scale, seq_lens, part_o, part_ml, \
+                                            status_word, stream);
+    GTA_TC_SHAPES(GTA_TC_LAUNCH)
+#undef GTA_TC_LAUNCH
     if (err != cudaSuccess) return err;
     return cudaGetLastError();
 }

@@ -1149,7 +1149,7 @@ cudaError_t launch_decode_fp8_fast(const Dims& d, const void* q, const void* k_c
     __nv_bfloat16* l_g = reinterpret_cast<__nv_bfloat16*>(static_cast<char*>(workspace) + p.off_l);
     cudaError_t err;
     if (decode_fp8_tc_supported(d, p.T)) {     // the tokens as the rows of tcgen05 MMAs
-        err = launch_decode_fp8_tc_stream(d, p.G, S_cap, q, k_codes, c_codes, k_scale, c_scale, seq_lens, part_o, part_ml,
+        err = launch_decode_fp8_tc_stream(d, p.G, p.T, S_cap, q, k_codes, c_codes, k_scale, c_scale, seq_lens, part_o, part_ml,
                                           status_word, stream);
         if (err != cudaSuccess) return err;
         *launches += 1;

@@ -58,7 +58,7 @@ gta_status_t launch_sm100_matmul(long long M, int K, int n_cols, const void* a, 
 // The stream kernel of a decode step over 8-bit caches on the tcgen05 tensor pipe (gta_decode_fp8_tc.cu): same
 // schedule (G CTAs, sub-tiles of T tokens) and partial results as decode_stream_fp8_kernel.
 bool decode_fp8_tc_supported(const Dims& d, int T);
-cudaError_t launch_decode_fp8_tc_stream(const Dims& d, int G, int S_cap, const void* q, const void* k_codes,
+cudaError_t launch_decode_fp8_tc_stream(const Dims& d, int G, int T, int S_cap, const void* q, const void* k_codes,
                                         const void* c_codes, const float* k_scale, const float* c_scale,
                                         const int32_t* seq_lens, float* part_o, float* part_ml, int32_t* status_word,
                                         cudaStream_t stream);

@@ -117,6 +117,12 @@ FP8_STREAM = [
     ("two_maps_one_key_group_dl512", 2, 128, 4, 2, 1, 512, [200, 450], 452),
     ("four_maps_one_key_group_dl256", 3, 128, 8, 4, 1, 256, [1000, 7, 128], 1000),
     ("long_sequences_many_subtiles_per_cta", 2, 256, 8, 4, 4, 512, [20000, 12345], 20000),
+    # 32-token sub-tiles (a token wider than 1 KB): four key groups on the rows of a score MMA, up to two such sets
+    ("dl1024_eight_maps_four_key_groups", 3, 512, 16, 8, 4, 1024, [257, 1, 1000], 1004),
+    ("dl1024_four_maps_four_key_groups", 3, 256, 8, 4, 4, 1024, [300, 31, 33], 304),
+    ("dl1024_eight_maps_two_key_groups", 2, 256, 8, 8, 2, 1024, [129, 64], 132),
+    ("dl1024_eight_maps_one_key_group", 2, 256, 8, 8, 1, 1024, [200, 95], 200),
+    ("dl512_eight_key_groups", 3, 512, 16, 8, 8, 512, [100, 0, 333], 336),
     ("batch_400_many_empty", 400, 256, 8, 4, 4, 512, [0 if i % 7 == 3 else 1 + (13 * i) % 70 for i in range(400)], 72),
     ("all_sequences_empty", 6, 256, 8, 4, 4, 512, [0, 0, 0, 0, 0, 0], 64),
 ]
