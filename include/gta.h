@@ -405,8 +405,8 @@ GTA_API gta_status_t gta_decode_hostcache(const gta_shape_t *shape, const void *
  * gta_decode over such caches (q, x_t, w_p, w_g, out in the shape's dtype; rows at and behind
  * seq_lens[b] may hold anything).  Needs d_h and d_l multiples of 16, d_l <= 2048; contiguous
  * caches only.  gta_decode_fp8 has a streaming path (TMA ring, tensor-core MMAs on the e4m3 codes
- * themselves -- tcgen05 with the cached tokens as the MMA rows for up to four key groups of 1, 2, 4 or
- * 8 maps and d_l <= 512, warp-level MMAs otherwise --, query rows and probabilities carried as sums of
+ * themselves -- tcgen05 with the cached tokens as the MMA rows where every key group has 1, 2, 4 or 8
+ * maps, warp-level MMAs otherwise --, query rows and probabilities carried as sums of
  * two e4m3 numbers, merge and tensor-core decoder kernels of gta_decode) for bf16 operator tensors with
  * d_h = 128, one latent group, d_l in {128, 256, 512, 1024}, at most 8 maps over 1, 2, 4 or 8 key groups,
  * S_cap a multiple of 4 and 16-byte aligned scale arrays; everything else, and the append, runs on the
