@@ -622,7 +622,8 @@ decode_stream_fp8_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __gr
     X(64, 2, 4, 1) X(64, 2, 4, 2)                                                                          \
     X(64, 4, 1, 1) X(64, 4, 1, 2) X(64, 4, 1, 4) X(64, 4, 1, 8) X(64, 4, 2, 1) X(64, 4, 2, 2) X(64, 4, 2, 4)   \
     X(64, 4, 4, 1) X(64, 4, 4, 2)                                                                          \
-    X(32, 8, 8, 1) X(32, 8, 4, 2) X(32, 8, 4, 1) X(32, 8, 2, 4) X(32, 8, 1, 8) X(32, 4, 8, 1)
+    X(32, 8, 1, 1) X(32, 8, 1, 2) X(32, 8, 1, 4) X(32, 8, 1, 8) X(32, 8, 2, 1) X(32, 8, 2, 2) X(32, 8, 2, 4)   \
+    X(32, 8, 4, 1) X(32, 8, 4, 2) X(32, 8, 8, 1) X(32, 4, 8, 1) X(32, 2, 8, 1) X(32, 1, 8, 1)
 
 // d_h = 128, one latent group, one of the instantiated shapes with the sub-tile size the plan has chosen
 bool decode_fp8_tc_supported(const Dims& d, int T) {

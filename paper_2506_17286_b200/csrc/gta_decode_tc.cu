@@ -648,10 +648,17 @@ cudaError_t launch_bt(const CUtensorMap& tm_k, const CUtensorMap& tm_c, const Di
                               status_word, (const uint4*)k_new, (const uint4*)c_new, (uint4*)k_cache, (uint4*)c_cache, pm);
 }
 
-// the instantiations: (sub-tile, key groups, maps per group, 128-column latent blocks)
-#define GTA_BT_SHAPES(X)                                                                       \
-    X(32, 4, 1, 4) X(32, 4, 2, 4) X(32, 2, 2, 4) X(32, 1, 4, 4)                                \
-    X(16, 8, 1, 8) X(16, 4, 2, 8) X(16, 2, 4, 8) X(16, 1, 8, 8)
+// The instantiations: (sub-tile, key groups, maps per group, 128-column latent blocks); the sub-tile is the one the
+// stream kernels' plan arrives at (the largest of 16, 32, 64 tokens whose rows fit a 64 KB ring stage).  They are the
+// groupings on which this kernel was measured faster than decode_stream_kernel (32 sequences of 4096 tokens, every
+// grouping of 1, 2, 4, 8 key groups x 1, 2, 4, 8 maps with at most 8 maps, d_l = 256, 512, 1024): those whose key
+// groups fill, or nearly fill, the 128 rows of the score MMAs, i.e. whose sub-tiles are 48 - 64 KB.  With fewer key
+// groups a sub-tile is small against the microsecond its chain through the two token-warp groups and the MMA warp
+// takes, and the warp-level kernel is 3 - 15 % faster.
+#define GTA_BT_SHAPES(X) \
+    X(64, 1, 1, 2) X(64, 1, 2, 2) X(64, 2, 1, 2) X(64, 2, 2, 2) X(64, 2, 4, 2) X(32, 4, 1, 2) X(32, 4, 2, 2) X(16, 8, 1, 2) \
+    X(32, 4, 1, 4) X(32, 4, 2, 4) X(16, 8, 1, 4) \
+    X(16, 8, 1, 8)
 
 }  // namespace
 

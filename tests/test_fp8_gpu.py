@@ -123,6 +123,12 @@ FP8_STREAM = [
     ("dl1024_eight_maps_two_key_groups", 2, 256, 8, 8, 2, 1024, [129, 64], 132),
     ("dl1024_eight_maps_one_key_group", 2, 256, 8, 8, 1, 1024, [200, 95], 200),
     ("dl512_eight_key_groups", 3, 512, 16, 8, 8, 512, [100, 0, 333], 336),
+    ("dl128_eight_key_groups", 2, 512, 8, 8, 8, 128, [70, 33], 72),
+    ("dl256_eight_key_groups", 2, 512, 8, 8, 8, 256, [31, 260], 260),
+    ("dl1024_one_map", 2, 128, 2, 1, 1, 1024, [150, 33], 152),
+    ("dl1024_four_maps_one_key_group", 2, 128, 4, 4, 1, 1024, [64, 97], 100),
+    ("dl1024_two_maps_two_key_groups", 2, 128, 4, 2, 2, 1024, [200, 32], 200),
+    ("dl1024_four_maps_two_key_groups", 2, 128, 4, 4, 2, 1024, [129, 1], 132),
     ("batch_400_many_empty", 400, 256, 8, 4, 4, 512, [0 if i % 7 == 3 else 1 + (13 * i) % 70 for i in range(400)], 72),
     ("all_sequences_empty", 6, 256, 8, 4, 4, 512, [0, 0, 0, 0, 0, 0], 64),
 ]

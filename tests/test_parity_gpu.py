@@ -230,6 +230,20 @@ SMALL_DECODE = [
     ("bf16_eight_maps_two_key_groups_dl1024", "bf16", 3, 256, 16, 8, 2, 1, 128, 1024, [1, 129, 48]),
     ("bf16_eight_maps_one_key_group_dl1024", "bf16", 3, 256, 8, 8, 1, 1, 128, 1024, [200, 0, 33]),
     ("bf16_long_sequences_many_sub_tiles_per_cta", "bf16", 2, 256, 8, 4, 4, 1, 128, 512, [20000, 12345]),
+    # 64-token sub-tiles (d_l = 256, one or two key groups: two key groups on the rows of a score MMA)
+    ("bf16_eight_maps_one_key_group_dl256", "bf16", 3, 256, 8, 8, 1, 1, 128, 256, [500, 64, 65]),
+    ("bf16_eight_maps_two_key_groups_dl256", "bf16", 4, 256, 8, 8, 2, 1, 128, 256, [63, 300, 0, 128]),
+    ("bf16_four_maps_one_key_group_dl256", "bf16", 2, 128, 4, 4, 1, 1, 128, 256, [1000, 127]),
+    ("bf16_eight_maps_four_key_groups_dl256", "bf16", 3, 256, 8, 8, 4, 1, 128, 256, [200, 31, 97]),
+    ("bf16_eight_key_groups_dl256", "bf16", 3, 512, 8, 8, 8, 1, 128, 256, [100, 15, 49]),
+    # the remaining groupings at d_l = 512 and 1024
+    ("bf16_one_map_dl512", "bf16", 2, 128, 2, 1, 1, 1, 128, 512, [300, 33]),
+    ("bf16_eight_maps_one_key_group_dl512", "bf16", 2, 256, 8, 8, 1, 1, 128, 512, [260, 95]),
+    ("bf16_eight_maps_two_key_groups_dl512", "bf16", 2, 256, 8, 8, 2, 1, 128, 512, [64, 129]),
+    ("bf16_eight_key_groups_dl512", "bf16", 3, 512, 8, 8, 8, 1, 128, 512, [100, 16, 47]),
+    ("bf16_one_map_dl1024", "bf16", 2, 128, 2, 1, 1, 1, 128, 1024, [150, 17]),
+    ("bf16_four_maps_two_key_groups_dl1024", "bf16", 2, 128, 4, 4, 2, 1, 128, 1024, [90, 33]),
+    ("bf16_four_maps_four_key_groups_dl1024", "bf16", 2, 128, 4, 4, 4, 1, 128, 1024, [48, 200]),
     # more sequences than the stream kernel has threads (the prefix sum takes two per thread), many of them empty;
     # and a batch with nothing cached at all (no CTA has a sub-tile)
     ("bf16_batch_400_c3_grouping", "bf16", 400, 256, 8, 4, 4, 1, 128, 512, [0 if i % 7 == 3 else 1 + (13 * i) % 70 for i in range(400)]),
@@ -576,6 +590,8 @@ STEP_CASES = [
     ("bf16_eight_key_groups_dl1024", "bf16", 512, 16, 8, 8, 1, 128, 1024, [0, 1, 14, 15, 16, 17, 31, 32, 300, 304], 304),
     ("bf16_two_maps_per_key_group_dl512", "bf16", 256, 16, 8, 4, 1, 128, 512, [95, 96, 97, 0, 640], 641),
     ("bf16_one_key_group_dl1024", "bf16", 256, 8, 8, 1, 1, 128, 1024, [47, 48, 200], 208),
+    ("bf16_64_token_sub_tiles_dl256", "bf16", 256, 8, 8, 2, 1, 128, 256, [63, 64, 65, 0, 127, 128, 300], 301),
+    ("bf16_eight_key_groups_dl256", "bf16", 512, 8, 8, 8, 1, 128, 256, [15, 16, 17, 100], 104),
     ("f32_plain_alu_kernels", "f32", 96, 6, 6, 3, 1, 32, 64, [100, 7, 0, 260], 261),
 ]
 
