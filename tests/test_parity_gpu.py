@@ -401,6 +401,9 @@ PAGED_DECODE = [
     ("bf16_pages_of_128_batch_40", "bf16", 40, 256, 8, 4, 4, 1, 128, 512, 128, [1 + (37 * i) % 600 for i in range(40)]),
     ("bf16_pages_of_256_paper_1b_shape", "bf16", 3, 1280, 20, 5, 1, 1, 64, 128, 256, [333, 1000, 256]),
     ("bf16_pages_of_64_two_latents", "bf16", 5, 256, 8, 4, 4, 2, 128, 256, 64, [129, 1, 64, 400, 33]),
+    # 16-token and 64-token sub-tiles of the tensor-memory stream kernel behind a block table
+    ("bf16_pages_of_64_eight_key_groups_dl1024", "bf16", 4, 512, 8, 8, 8, 1, 128, 1024, 64, [257, 15, 64, 500]),
+    ("bf16_pages_of_128_two_key_groups_dl256", "bf16", 4, 256, 8, 4, 2, 1, 128, 256, 128, [300, 0, 128, 65]),
     # page sizes the streaming kernel does not take (no multiple of 64), and fp32: the plain-ALU kernels
     ("bf16_pages_of_16", "bf16", 4, 128, 4, 2, 2, 1, 128, 256, 16, [0, 512, 1, 300]),
     ("bf16_pages_of_48", "bf16", 3, 128, 8, 4, 2, 2, 64, 128, 48, [200, 5, 129]),
